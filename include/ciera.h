@@ -1,0 +1,219 @@
+/*
+ * ciera.h -- C ABI of the B200 (sm_100a) exponent-reuse codec.
+ *
+ * The library implements the data-parallel hot path of CIERA's "Exponent Reuse based
+ * Compression" (paper Section 3.1, Algorithm 1) and the gain rule of "Benefit-driven
+ * Selective Compression" (Section 3.2):
+ *
+ *   sender    split every weight into exponent and sign-plus-mantissa, compare the exponents
+ *             with a cached copy block by block, emit (bitmap, sign-plus-mantissa of all
+ *             values, exponents of changed blocks), refresh the cache for changed blocks;
+ *   receiver  patch its exponent cache with the changed blocks, merge cache and
+ *             sign-plus-mantissa back into bit-identical weights.
+ *
+ * Conventions
+ *   - Every function returns a ciera_status (0 = CIERA_OK, negative = error).  Nothing throws,
+ *     nothing is printed, and no codec state lives in the library: caches, messages and scratch
+ *     are the caller's buffers.
+ *   - "dev" pointers are CUDA device pointers, "host" pointers are ordinary host pointers.
+ *     The library never allocates device memory: the caller owns every device buffer and
+ *     passes scratch space explicitly.  The only host allocation is the plan object.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Device work is
+ *     enqueued on it and the call returns without waiting, unless stated otherwise.
+ *   - Errors found on the device (a wait that ran out, a message whose length contradicts its
+ *     bitmap) are written to the caller's `status_dev` word: 0 = none, otherwise the first
+ *     ciera_status that was raised.  The word is only ever written on error; clear it yourself.
+ *   - A *unit* is one shard of one tensor: N consecutive values.  Units are independent; one call
+ *     processes a whole table of them ("batched launch over simulated shards").
+ *
+ * Wire format of one unit's message (b bits per value, m = b - 8 sign-plus-mantissa bits,
+ * block size B, nb = ceil(N/B) blocks; Section 3.2 for the sizes, Algorithm 1 for the order
+ * bitmap, mant, payload):
+ *
+ *   [ bitmap : ceil(nb/8) bytes, block k -> byte k>>3 bit k&7, unused high bits 0 ]
+ *   [ zero pad to a multiple of 16 ]
+ *   [ sm     : N*m/8 bytes; bf16: byte j = sign<<7 | mantissa(7);
+ *              fp32: bytes 3j..3j+2 = (sign<<23 | mantissa(23)) little-endian ]
+ *   [ zero pad to a multiple of 16 ]
+ *   [ payload: for every changed block in ascending k, its exponent bytes (B of them, fewer
+ *              for a short last block) ]
+ *
+ * No header travels: the payload length follows from the bitmap.  The paper's byte count
+ * S_{s+m} + S_bm + (changed exponent bytes) is ciera_message_bytes(); the length that has to
+ * be moved (it includes the two pads, at most 30 bytes) is what ciera_encode reports.
+ * Bytes of a slot past the reported length are unspecified.
+ */
+#ifndef CIERA_H
+#define CIERA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define CIERA_API __attribute__((visibility("default")))
+#else
+#define CIERA_API
+#endif
+
+typedef enum ciera_status {
+    CIERA_OK = 0,
+    CIERA_ERR_INVALID_ARG = -1, /* null pointer, zero block, bad enum, inconsistent sizes      */
+    CIERA_ERR_UNSUPPORTED = -2, /* block size outside the supported set                         */
+    CIERA_ERR_MISALIGNED = -3,  /* an offset or base pointer is not a multiple of 16 bytes      */
+    CIERA_ERR_CAPACITY = -4,    /* a message slot, plan image or scratch buffer is too small    */
+    CIERA_ERR_CUDA = -5,        /* a CUDA runtime call failed (see ciera_last_cuda_error)       */
+    CIERA_ERR_TIMEOUT = -6,     /* device: a bounded wait on another tile ran out               */
+    CIERA_ERR_CORRUPT = -7,     /* device: message length disagrees with its bitmap             */
+    CIERA_ERR_NOT_BOUND = -8    /* the plan has no device image yet (ciera_plan_bind)           */
+} ciera_status;
+
+typedef enum ciera_dtype {
+    CIERA_BF16 = 0, /* b = 16: 1 sign, 8 exponent, 7 mantissa bits  -> m = 8  */
+    CIERA_FP32 = 1  /* b = 32: 1 sign, 8 exponent, 23 mantissa bits -> m = 24 */
+} ciera_dtype;
+
+/* One unit = one shard of one tensor.  All offsets are in BYTES from the base pointer of the
+ * respective buffer and must be multiples of 16. */
+typedef struct ciera_unit {
+    uint64_t n_values;     /* N; may be 0, may be smaller than the block size                   */
+    uint64_t weights_off;  /* into the weights buffer (encode: input, decode: output)           */
+    uint64_t cache_off;    /* into the exponent cache (1 byte per value)                        */
+    uint64_t msg_off;      /* into the message buffer: start of this unit's slot                */
+    uint64_t msg_capacity; /* size of the slot, >= ciera_message_capacity(N, dtype, block)      */
+} ciera_unit;
+
+/* ---- sizes (host, pure functions; Section 3.2) ------------------------------------------- */
+
+/* Smallest and largest supported block size B (a power of two in this range). */
+#define CIERA_MIN_BLOCK 16u
+#define CIERA_MAX_BLOCK 4096u
+
+/* Slot size that always suffices: every block changed (payload = N exponent bytes). */
+CIERA_API size_t ciera_message_capacity(uint64_t n_values, int dtype, uint32_t block);
+/* Offset of the sign-plus-mantissa section / of the payload section inside a slot. */
+CIERA_API size_t ciera_sm_offset(uint64_t n_values, uint32_t block);
+CIERA_API size_t ciera_payload_offset(uint64_t n_values, int dtype, uint32_t block);
+/* The paper's transmitted bytes S_{s+m} + S_bm + payload_bytes (no pads). */
+CIERA_API size_t ciera_message_bytes(uint64_t n_values, int dtype, uint32_t block, uint64_t payload_bytes);
+
+/* ---- plan: the tile table of a unit table -------------------------------------------------- */
+
+/* A plan splits every unit into tiles of ciera_plan_tile_values() consecutive values (one tile
+ * is the work of one thread block) and holds the device-side table that the kernels read.  It
+ * is immutable after ciera_plan_bind and may be shared by any number of calls and streams. */
+typedef struct ciera_plan ciera_plan;
+
+/* Host only.  Validates the units (alignment, capacity, block size) and builds the table.
+ * `units_host` is copied.  Destroy with ciera_plan_destroy. */
+CIERA_API int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units, int dtype, uint32_t block,
+                      ciera_plan** plan_out);
+CIERA_API void ciera_plan_destroy(ciera_plan* plan);
+
+CIERA_API uint32_t ciera_plan_n_units(const ciera_plan* plan);
+CIERA_API uint32_t ciera_plan_n_tiles(const ciera_plan* plan);
+CIERA_API uint32_t ciera_plan_tile_values(const ciera_plan* plan);
+CIERA_API uint64_t ciera_plan_total_values(const ciera_plan* plan);
+/* Bytes of device memory the table needs (>= 16), and the host image that has to be there. */
+CIERA_API size_t ciera_plan_device_bytes(const ciera_plan* plan);
+CIERA_API const void* ciera_plan_host_image(const ciera_plan* plan);
+/* Bytes of scratch one ciera_encode call needs (tile status words for the look-back). */
+CIERA_API size_t ciera_plan_workspace_bytes(const ciera_plan* plan);
+
+/* Copies the table into caller-owned device memory `plan_dev` (>= ciera_plan_device_bytes,
+ * 16-byte aligned) on `stream`, waits for the copy, and remembers the pointer.  The memory must
+ * stay valid and unmodified for as long as the plan is used. */
+CIERA_API int ciera_plan_bind(ciera_plan* plan, void* plan_dev, size_t plan_dev_bytes, void* stream);
+
+/* ---- caches (Algorithm 1: persistent sender / receiver state) ------------------------------ */
+
+/* cache := exponents of `weights_dev`, or all zero if weights_dev == NULL.  The paper starts
+ * "after model initialization and warmup" without fixing the first cache state; initialising
+ * both sides from the same weights (as if they had been sent uncompressed), or both to zero,
+ * keeps them in agreement. */
+CIERA_API int ciera_cache_init(const ciera_plan* plan, void* cache_dev, const void* weights_dev, void* stream);
+/* cache := exponents of `weights_dev`, unconditionally (e.g. after a checkpoint restore). */
+CIERA_API int ciera_cache_update(const ciera_plan* plan, void* cache_dev, const void* weights_dev, void* stream);
+
+/* ---- sender: Algorithm 1, sender part; Section 3.1 ----------------------------------------- */
+
+/*
+ * For every unit: split, block-wise change detection against `sender_cache_dev`, write the
+ * message into the unit's slot of `messages_dev`, refresh the cache for changed blocks.
+ *   weights_dev         in   values of the plan's dtype at units[].weights_off
+ *   sender_cache_dev    i/o  1 byte per value at units[].cache_off
+ *   messages_dev        out  slots at units[].msg_off
+ *   wire_bytes_dev      out  [n_units] bytes that have to travel (payload offset + payload bytes;
+ *                            0 for an empty unit)
+ *   changed_blocks_dev  out  [n_units] number of set bitmap bits
+ *   workspace_dev       scratch of ciera_plan_workspace_bytes(), 16-byte aligned; cleared by the
+ *                            call itself; must not be shared by calls that can overlap on the GPU
+ *   status_dev          i/o  device error word (may be NULL)
+ * One kernel launch (plus one memset of the scratch) for the whole table.
+ */
+CIERA_API int ciera_encode(const ciera_plan* plan, const void* weights_dev, void* sender_cache_dev, void* messages_dev,
+                 uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* workspace_dev,
+                 int32_t* status_dev, void* stream);
+
+/* ---- transport stand-in: Send / Recv of Algorithm 1 on one GPU ----------------------------- */
+
+/* Copies, for every unit, the first wire_bytes_dev[u] bytes of its slot from `src_messages_dev`
+ * to the same slot of `dst_messages_dev` (one kernel; the lengths are read on the device).  This
+ * stands where the Allgather of the messages would be. */
+CIERA_API int ciera_transport(const ciera_plan* plan, const void* src_messages_dev, void* dst_messages_dev,
+                    const uint64_t* wire_bytes_dev, void* stream);
+
+/* ---- receiver: Algorithm 1, receiver part; Section 3.1 ------------------------------------- */
+
+/*
+ * For every unit: read the bitmap, overwrite the cached exponents of changed blocks with the
+ * payload, merge cache and sign-plus-mantissa into `weights_out_dev`.
+ *   messages_dev        in   slots at units[].msg_off
+ *   receiver_cache_dev  i/o  1 byte per value at units[].cache_off
+ *   weights_out_dev     out  reconstructed values at units[].weights_off
+ *   wire_bytes_dev      in   optional (may be NULL): lengths as reported by the sender; a unit
+ *                            whose bitmap implies a different length raises CIERA_ERR_CORRUPT in
+ *                            status_dev (its output is then unspecified)
+ */
+CIERA_API int ciera_decode(const ciera_plan* plan, const void* messages_dev, void* receiver_cache_dev,
+                 void* weights_out_dev, const uint64_t* wire_bytes_dev, int32_t* status_dev, void* stream);
+
+/* ---- selective compression: the gain rule of Section 3.2 (host only) ----------------------- */
+
+typedef struct ciera_gain_in {
+    uint64_t n_values;    /* N^i                                                               */
+    int32_t dtype;        /* ciera_dtype                                                        */
+    uint32_t block;       /* B (any positive value; only sizes are computed)                    */
+    double q;             /* block change rate q_i in [0, 1] (measured offline / by a previous encode) */
+    int32_t world_size;   /* W, used by the alpha-beta model only                               */
+    int32_t overlapped;   /* non-zero: T_hash = T_cmp = 0 on the critical path (pipelining)     */
+    double alpha;         /* Comm(S) = alpha + (W-1) * S / beta when n_points < 2               */
+    double beta;          /* bytes per second                                                   */
+    const double* table_bytes; /* optional measured Comm(): n_points ascending payload sizes... */
+    const double* table_secs;  /* ...and their latencies; linear interpolation, the first/last
+                                  segment is extended outside the table                         */
+    int32_t n_points;
+    double t_hash;        /* seconds: change detection of the shard                             */
+    double t_cmp;         /* seconds: sender-side packing                                       */
+    double t_decmp;       /* seconds: receiver-side patch + merge                               */
+} ciera_gain_in;
+
+/* g = Comm(S) - ( Comm(S_{s+m} + S_bm + q S_e) + T_hash + T_cmp + T_decmp ), and the decision
+ * "compress iff g > 0".  Either output pointer may be NULL. */
+CIERA_API int ciera_should_compress(const ciera_gain_in* in, double* gain_seconds_out, int* decision_out);
+
+/* ---- diagnostics ---------------------------------------------------------------------------- */
+
+/* cudaError_t of the last failing runtime call made by the calling thread inside this library. */
+CIERA_API int ciera_last_cuda_error(void);
+/* Number of kernels this library has launched from the calling process (for launch accounting). */
+CIERA_API uint64_t ciera_kernel_launch_count(void);
+CIERA_API const char* ciera_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CIERA_H */

@@ -1,0 +1,205 @@
+// Host side of libciera: size rules, the plan (tile table), the gain rule, diagnostics.
+#include <new>
+
+#include "ciera_internal.cuh"
+
+namespace ciera {
+
+static thread_local int g_last_cuda_error = 0;
+static std::atomic<uint64_t> g_launches{0};
+
+int record_cuda_error(cudaError_t e) {
+    g_last_cuda_error = (int)e;
+    return CIERA_ERR_CUDA;
+}
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+int check_launch() {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return record_cuda_error(e);
+    return CIERA_OK;
+}
+
+static bool valid_dtype(int dtype) { return dtype == CIERA_BF16 || dtype == CIERA_FP32; }
+static uint32_t sm_bytes_of(int dtype) { return dtype == CIERA_BF16 ? 1u : 3u; }
+static uint32_t value_bytes_of(int dtype) { return dtype == CIERA_BF16 ? 2u : 4u; }
+
+// log2 of a power of two, or -1.
+static int exact_log2(uint32_t x) {
+    if (x == 0 || (x & (x - 1))) return -1;
+    int l = 0;
+    while ((1u << l) != x) ++l;
+    return l;
+}
+
+}  // namespace ciera
+
+using namespace ciera;
+
+// ---------------------------------------------------------------------------------- sizes
+
+extern "C" size_t ciera_sm_offset(uint64_t n, uint32_t block) {
+    if (block == 0) return 0;
+    uint64_t nb = (n + block - 1) / block;
+    return (size_t)pad16((nb + 7) / 8);
+}
+
+extern "C" size_t ciera_payload_offset(uint64_t n, int dtype, uint32_t block) {
+    if (block == 0 || !valid_dtype(dtype)) return 0;
+    return ciera_sm_offset(n, block) + (size_t)pad16(n * sm_bytes_of(dtype));
+}
+
+extern "C" size_t ciera_message_capacity(uint64_t n, int dtype, uint32_t block) {
+    if (n == 0 || block == 0 || !valid_dtype(dtype)) return 0;
+    return ciera_payload_offset(n, dtype, block) + (size_t)n;
+}
+
+extern "C" size_t ciera_message_bytes(uint64_t n, int dtype, uint32_t block, uint64_t payload_bytes) {
+    if (block == 0 || !valid_dtype(dtype)) return 0;
+    uint64_t nb = (n + block - 1) / block;
+    return (size_t)(n * sm_bytes_of(dtype) + (nb + 7) / 8 + payload_bytes);
+}
+
+// ---------------------------------------------------------------------------------- plan
+
+extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units, int dtype, uint32_t block,
+                                 ciera_plan** plan_out) {
+    if (!plan_out) return CIERA_ERR_INVALID_ARG;
+    *plan_out = nullptr;
+    if ((!units_host && n_units) || !valid_dtype(dtype)) return CIERA_ERR_INVALID_ARG;
+    if (block == 0) return CIERA_ERR_INVALID_ARG;
+    int l2 = exact_log2(block);
+    if (l2 < 0 || block < CIERA_MIN_BLOCK || block > CIERA_MAX_BLOCK) return CIERA_ERR_UNSUPPORTED;
+
+    uint64_t n_tiles = 0, total = 0;
+    for (uint32_t u = 0; u < n_units; ++u) {
+        const ciera_unit& un = units_host[u];
+        if ((un.weights_off | un.cache_off | un.msg_off) & 15ull) return CIERA_ERR_MISALIGNED;
+        if (un.n_values >= (1ull << 48)) return CIERA_ERR_UNSUPPORTED;
+        if (un.msg_capacity < ciera_message_capacity(un.n_values, dtype, block)) return CIERA_ERR_CAPACITY;
+        n_tiles += (un.n_values + kTileValues - 1) / kTileValues;
+        total += un.n_values;
+    }
+    if (n_tiles >= 0x7fffffffull) return CIERA_ERR_UNSUPPORTED;  // grid.x limit
+
+    ciera_plan* p = new (std::nothrow) ciera_plan;
+    if (!p) return CIERA_ERR_INVALID_ARG;
+    p->dtype = dtype;
+    p->block = block;
+    p->log2b = (uint32_t)l2;
+    p->n_units = n_units;
+    p->total_values = total;
+    for (uint32_t u = 0; u < n_units; ++u) p->has_empty_units |= units_host[u].n_values == 0;
+    p->units.assign(units_host, units_host + n_units);
+    p->tiles.reserve((size_t)n_tiles);
+    const uint32_t vb = value_bytes_of(dtype);
+    for (uint32_t u = 0; u < n_units; ++u) {
+        const ciera_unit& un = units_host[u];
+        uint32_t nt = (uint32_t)((un.n_values + kTileValues - 1) / kTileValues);
+        uint32_t first = (uint32_t)p->tiles.size();
+        for (uint32_t j = 0; j < nt; ++j) {
+            TileDesc t;
+            t.w_off = un.weights_off + (uint64_t)j * kTileValues * vb;
+            t.c_off = un.cache_off + (uint64_t)j * kTileValues;
+            t.msg_off = un.msg_off;
+            t.n_unit = un.n_values;
+            t.unit = u;
+            t.tile_in_unit = j;
+            t.first_tile = first;
+            t.n_tiles_unit = nt;
+            p->tiles.push_back(t);
+        }
+    }
+    *plan_out = p;
+    return CIERA_OK;
+}
+
+extern "C" void ciera_plan_destroy(ciera_plan* plan) { delete plan; }
+
+extern "C" uint32_t ciera_plan_n_units(const ciera_plan* p) { return p ? p->n_units : 0; }
+extern "C" uint32_t ciera_plan_n_tiles(const ciera_plan* p) { return p ? (uint32_t)p->tiles.size() : 0; }
+extern "C" uint32_t ciera_plan_tile_values(const ciera_plan*) { return kTileValues; }
+extern "C" uint64_t ciera_plan_total_values(const ciera_plan* p) { return p ? p->total_values : 0; }
+
+extern "C" size_t ciera_plan_device_bytes(const ciera_plan* p) {
+    if (!p) return 0;
+    size_t b = p->tiles.size() * sizeof(TileDesc);
+    return b ? b : 16;
+}
+extern "C" const void* ciera_plan_host_image(const ciera_plan* p) { return p ? p->tiles.data() : nullptr; }
+
+extern "C" size_t ciera_plan_workspace_bytes(const ciera_plan* p) {
+    if (!p) return 0;
+    size_t b = p->tiles.size() * sizeof(unsigned long long);
+    return b ? b : 16;
+}
+
+extern "C" int ciera_plan_bind(ciera_plan* p, void* plan_dev, size_t plan_dev_bytes, void* stream) {
+    if (!p || !plan_dev) return CIERA_ERR_INVALID_ARG;
+    if ((uintptr_t)plan_dev & 15u) return CIERA_ERR_MISALIGNED;
+    size_t need = p->tiles.size() * sizeof(TileDesc);
+    if (plan_dev_bytes < need) return CIERA_ERR_CAPACITY;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (need) {
+        cudaError_t e = cudaMemcpyAsync(plan_dev, p->tiles.data(), need, cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) return record_cuda_error(e);
+    }
+    p->tiles_dev = (const TileDesc*)plan_dev;
+    return CIERA_OK;
+}
+
+// ---------------------------------------------------------------------------------- gain rule
+
+static double comm_seconds(const ciera_gain_in* in, double bytes) {
+    if (in->n_points < 2 || !in->table_bytes || !in->table_secs)
+        return in->alpha + (double)(in->world_size - 1) * bytes / in->beta;
+    int i = 0;
+    while (i < in->n_points - 2 && bytes > in->table_bytes[i + 1]) ++i;
+    double x0 = in->table_bytes[i], x1 = in->table_bytes[i + 1];
+    double y0 = in->table_secs[i], y1 = in->table_secs[i + 1];
+    return y0 + (bytes - x0) * (y1 - y0) / (x1 - x0);
+}
+
+extern "C" int ciera_should_compress(const ciera_gain_in* in, double* gain_seconds_out, int* decision_out) {
+    if (!in || !valid_dtype(in->dtype) || in->block == 0) return CIERA_ERR_INVALID_ARG;
+    if (!(in->q >= 0.0 && in->q <= 1.0)) return CIERA_ERR_INVALID_ARG;
+    if (in->n_points >= 2 && in->table_bytes && in->table_secs) {
+        for (int i = 0; i + 1 < in->n_points; ++i)
+            if (!(in->table_bytes[i + 1] > in->table_bytes[i])) return CIERA_ERR_INVALID_ARG;
+    } else if (!(in->beta > 0.0) || in->world_size < 1) {
+        return CIERA_ERR_INVALID_ARG;
+    }
+    const double n = (double)in->n_values;
+    const double s_full = n * value_bytes_of(in->dtype);
+    const double s_exp = n;  // 8 exponent bits per value
+    const double s_sm = s_full - s_exp;
+    const uint64_t blocks = (in->n_values + in->block - 1) / in->block;
+    const double s_bm = (double)((blocks + 7) / 8);
+    const double sent = s_sm + s_bm + in->q * s_exp;
+    const double sender = in->overlapped ? 0.0 : in->t_hash + in->t_cmp;
+    const double g = comm_seconds(in, s_full) - (comm_seconds(in, sent) + sender + in->t_decmp);
+    if (gain_seconds_out) *gain_seconds_out = g;
+    if (decision_out) *decision_out = g > 0.0 ? 1 : 0;
+    return CIERA_OK;
+}
+
+// ---------------------------------------------------------------------------------- diagnostics
+
+extern "C" int ciera_last_cuda_error(void) { return g_last_cuda_error; }
+extern "C" uint64_t ciera_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+extern "C" const char* ciera_status_string(int s) {
+    switch (s) {
+        case CIERA_OK: return "ok";
+        case CIERA_ERR_INVALID_ARG: return "invalid argument";
+        case CIERA_ERR_UNSUPPORTED: return "unsupported block size or unit size";
+        case CIERA_ERR_MISALIGNED: return "offset or pointer not 16-byte aligned";
+        case CIERA_ERR_CAPACITY: return "buffer or message slot too small";
+        case CIERA_ERR_CUDA: return "CUDA runtime error";
+        case CIERA_ERR_TIMEOUT: return "device wait ran out";
+        case CIERA_ERR_CORRUPT: return "message length contradicts its bitmap";
+        case CIERA_ERR_NOT_BOUND: return "plan not bound to device memory";
+        default: return "unknown status";
+    }
+}

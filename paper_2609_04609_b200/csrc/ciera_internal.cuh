@@ -1,0 +1,97 @@
+// Internal declarations shared by the translation units of libciera (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+#include <vector>
+
+#include "ciera.h"
+
+namespace ciera {
+
+// One tile = kTileValues consecutive values of one unit = the work of one thread block.
+// Each thread owns kVPT consecutive values ("a group"): 16 values are 16 exponent bytes, i.e.
+// one 128-bit access on each of the byte-wide streams (cache, sm, payload).
+constexpr int kThreads = 512;
+constexpr int kVPT = 16;
+constexpr int kTileValues = kThreads * kVPT;  // 8192
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxBlocksPerTile = kTileValues / CIERA_MIN_BLOCK;  // 512
+constexpr int kBitmapWords = kMaxBlocksPerTile / 32;              // 16
+
+// Device-side tile descriptor: everything a thread block needs, in one 48-byte record so that
+// a single dependent load stands between block start and the first data load.
+struct __align__(16) TileDesc {
+    uint64_t w_off;         // byte offset of the tile's first value in the weights buffer
+    uint64_t c_off;         // byte offset of the tile's first value in the cache
+    uint64_t msg_off;       // byte offset of the unit's message slot
+    uint64_t n_unit;        // N of the unit
+    uint32_t unit;          // index into the per-unit outputs
+    uint32_t tile_in_unit;  // 0 .. n_tiles_unit-1
+    uint32_t first_tile;    // table index of the unit's first tile
+    uint32_t n_tiles_unit;  // tiles of this unit
+};
+static_assert(sizeof(TileDesc) == 48, "TileDesc must stay three 16-byte words");
+
+// Tile status word used by the single-pass look-back of the encode kernel.
+//   bits 63:62  0 = empty, 1 = aggregate of this tile, 2 = inclusive prefix up to this tile
+//   bits 61:56  the tile's own bitmap bits when a tile holds fewer than 8 blocks
+//   bits 55:0   payload bytes
+constexpr unsigned long long kFlagAggregate = 1ull << 62;
+constexpr unsigned long long kFlagPrefix = 2ull << 62;
+constexpr unsigned long long kValueMask = (1ull << 56) - 1;
+constexpr int kBitsShift = 56;
+
+// Upper bound on polls of one status word before a tile gives up and raises CIERA_ERR_TIMEOUT.
+constexpr uint32_t kMaxPolls = 1u << 21;
+
+template <int DT>
+struct Traits;
+template <>
+struct Traits<CIERA_BF16> {
+    static constexpr int kValueBytes = 2;
+    static constexpr int kSmBytes = 1;
+};
+template <>
+struct Traits<CIERA_FP32> {
+    static constexpr int kValueBytes = 4;
+    static constexpr int kSmBytes = 3;
+};
+
+__host__ __device__ inline uint64_t pad16(uint64_t x) { return (x + 15ull) & ~15ull; }
+__host__ __device__ inline uint64_t num_blocks(uint64_t n, uint32_t log2b) {
+    return (n + (1ull << log2b) - 1) >> log2b;
+}
+__host__ __device__ inline uint64_t bitmap_bytes(uint64_t n, uint32_t log2b) { return (num_blocks(n, log2b) + 7) >> 3; }
+__host__ __device__ inline uint64_t sm_offset(uint64_t n, uint32_t log2b) { return pad16(bitmap_bytes(n, log2b)); }
+__host__ __device__ inline uint64_t payload_offset(uint64_t n, uint32_t sm_bytes_per_value, uint32_t log2b) {
+    return sm_offset(n, log2b) + pad16(n * sm_bytes_per_value);
+}
+
+// Bytes of a message slot that one tile moves in the transport kernel: slot capacity <= tiles * this.
+__host__ __device__ inline uint64_t transport_chunk_bytes(uint32_t sm_bytes_per_value) {
+    return (uint64_t)kTileValues * (sm_bytes_per_value + 1) + 96;
+}
+
+}  // namespace ciera
+
+// The plan object behind the opaque handle.
+struct ciera_plan {
+    int dtype = 0;
+    uint32_t block = 0;
+    uint32_t log2b = 0;
+    uint32_t n_units = 0;
+    uint64_t total_values = 0;
+    bool has_empty_units = false;
+    std::vector<ciera_unit> units;
+    std::vector<ciera::TileDesc> tiles;
+    const ciera::TileDesc* tiles_dev = nullptr;
+};
+
+namespace ciera {
+int record_cuda_error(cudaError_t e);          // stores e for ciera_last_cuda_error, returns CIERA_ERR_CUDA
+void count_launch();                           // launch accounting
+int check_launch();                            // cudaGetLastError -> status
+}  // namespace ciera

@@ -1,0 +1,112 @@
+"""Device-side state of one table of units (e.g. one MoE layer) and the per-iteration step.
+
+Plumbing only: torch allocates the buffers and provides streams / events; every data-path
+operation is a call into the C-ABI library (``ciera.encode``, ``ciera.transport``,
+``ciera.decode``).  One ``LayerCodec`` plays both roles of the paper's Algorithm 1 on a single
+GPU: the sender with its cache, and one receiver with its own cache; the device-to-device
+``transport`` stands where the Allgather of the messages would be.
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import ciera
+from .workloads import VALUE_BYTES, layout_units
+
+
+class LayerCodec:
+    def __init__(self, units: np.ndarray, dtype: str, block: int, weights_bytes: int, cache_bytes: int,
+                 msg_bytes: int, device="cuda:0", with_output: bool = True):
+        self.dtype_name = dtype
+        self.dtype = ciera.DTYPE_CODES[dtype]
+        self.block = block
+        self.device = torch.device(device)
+        self.plan = ciera.Plan(units, self.dtype, block, self.device)
+        self.units = self.plan.units
+        dev = self.device
+        u8 = dict(dtype=torch.uint8, device=dev)
+        self.weights_bytes, self.cache_bytes, self.msg_bytes = weights_bytes, cache_bytes, msg_bytes
+        self.sender_cache = torch.zeros(max(cache_bytes, 16), **u8)
+        self.receiver_cache = torch.zeros(max(cache_bytes, 16), **u8)
+        self.msg_send = torch.zeros(max(msg_bytes, 16), **u8)
+        self.msg_recv = torch.zeros(max(msg_bytes, 16), **u8)
+        self.weights_out = torch.zeros(max(weights_bytes, 16), **u8) if with_output else None
+        n = max(self.plan.n_units, 1)
+        self.wire_bytes = torch.zeros(n, dtype=torch.int64, device=dev)
+        self.changed_blocks = torch.zeros(n, dtype=torch.int32, device=dev)
+        self.workspace = self.plan.new_workspace()
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    @classmethod
+    def from_tensors(cls, tensor_numels: Sequence[int], n_shards: int, dtype: str, block: int, device="cuda:0",
+                     **kw) -> "LayerCodec":
+        code = ciera.DTYPE_CODES[dtype]
+        units, wb, cb, mb = layout_units(tensor_numels, n_shards, VALUE_BYTES[dtype],
+                                         lambda n: ciera.message_capacity(n, code, block))
+        return cls(units, dtype, block, wb, cb, mb, device, **kw)
+
+    # -- Algorithm 1 state --------------------------------------------------------------------
+    def init_caches(self, weights: Optional[torch.Tensor], stream=None) -> None:
+        """Both caches := exponents(weights) (or zero when ``weights`` is None)."""
+        ciera.cache_init(self.plan, self.sender_cache, weights, stream)
+        ciera.cache_init(self.plan, self.receiver_cache, weights, stream)
+
+    # -- the three stages -----------------------------------------------------------------------
+    def encode(self, weights: torch.Tensor, stream=None) -> None:
+        ciera.encode(self.plan, weights, self.sender_cache, self.msg_send, self.wire_bytes, self.changed_blocks,
+                     self.workspace, self.status, stream)
+
+    def transport(self, stream=None) -> None:
+        ciera.transport(self.plan, self.msg_send, self.msg_recv, self.wire_bytes, stream)
+
+    def decode(self, weights_out: Optional[torch.Tensor] = None, stream=None, check_length: bool = True) -> None:
+        out = self.weights_out if weights_out is None else weights_out
+        ciera.decode(self.plan, self.msg_recv, self.receiver_cache, out,
+                     self.wire_bytes if check_length else None, self.status, stream)
+
+    def step(self, weights: torch.Tensor, weights_out: Optional[torch.Tensor] = None, stream=None) -> None:
+        self.encode(weights, stream)
+        self.transport(stream)
+        self.decode(weights_out, stream)
+
+    def check_status(self) -> None:
+        s = int(self.status.item())
+        if s != 0:
+            raise ciera.CieraError("device status", s)
+
+    # -- accounting -------------------------------------------------------------------------------
+    def paper_bytes(self) -> int:
+        """Transmitted bytes of the last encode by the paper's count (no pads)."""
+        wire = self.wire_bytes.cpu().numpy()
+        total = 0
+        for u, w in zip(self.units, wire):
+            n = int(u["n_values"])
+            if n == 0:
+                continue
+            payload = int(w) - ciera.payload_offset(n, self.dtype, self.block)
+            total += ciera.message_bytes(n, self.dtype, self.block, payload)
+        return total
+
+    def n_blocks(self) -> int:
+        n = self.units["n_values"].astype(np.int64)
+        return int(((n + self.block - 1) // self.block).sum())
+
+
+def pipelined_step(layers: List[LayerCodec], weights: List[torch.Tensor], outs: List[Optional[torch.Tensor]],
+                   s_enc: torch.cuda.Stream, s_dec: torch.cuda.Stream, events=None) -> None:
+    """One iteration over a stack of layers on two streams: the sender-side work of layer l+1
+    (encode, then the transport of its message) runs on ``s_enc`` while the receiver-side
+    decode of layer l runs on ``s_dec`` -- the shape of the paper's computation-communication
+    pipelining, where only the decompression of layer l stays on the critical path."""
+    n = len(layers)
+    if events is None:
+        events = [torch.cuda.Event() for _ in range(n)]
+    for l in range(n):
+        layers[l].encode(weights[l], s_enc)
+        layers[l].transport(s_enc)
+        events[l].record(s_enc)
+        s_dec.wait_event(events[l])
+        layers[l].decode(outs[l], s_dec)

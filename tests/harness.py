@@ -1,0 +1,101 @@
+"""Test-side runners: the CPU oracle over a whole unit table, and comparison with the CUDA path.
+
+Lives in tests/ and is used by tests only.  The oracle runner keeps its own flat caches in the
+same layout as the device buffers so that results can be compared byte for byte."""
+import numpy as np
+import torch
+
+from oracle import ciera_oracle as ora
+
+VB = {0: 2, 1: 4}
+WDT = {0: np.uint16, 1: np.uint32}
+
+
+class OracleTable:
+    def __init__(self, units, dtype, block, cache_bytes, msg_bytes):
+        self.units, self.dtype, self.block = units, dtype, block
+        self.cache_s = np.zeros(max(cache_bytes, 16), np.uint8)
+        self.cache_r = np.zeros(max(cache_bytes, 16), np.uint8)
+        self.msg_bytes = msg_bytes
+
+    def _w(self, w_flat, u):
+        lo = int(u["weights_off"]) // VB[self.dtype]
+        return w_flat[lo : lo + int(u["n_values"])]
+
+    def init_caches(self, w_flat):
+        for u in self.units:
+            n, co = int(u["n_values"]), int(u["cache_off"])
+            c = ora.cache_init(None if w_flat is None else self._w(w_flat, u), n, self.dtype)
+            self.cache_s[co : co + n] = c
+            self.cache_r[co : co + n] = c
+
+    def step(self, w_flat):
+        """Encode + decode every unit.  Returns dict with flat message buffer (only the first
+        wire[u] bytes of each slot are meaningful), wire, changed, payload, recon."""
+        nu = len(self.units)
+        msgs = np.zeros(max(self.msg_bytes, 16), np.uint8)
+        wire = np.zeros(nu, np.uint64)
+        chg = np.zeros(nu, np.uint32)
+        pay = np.zeros(nu, np.uint64)
+        recon = np.zeros_like(w_flat)
+        for i, u in enumerate(self.units):
+            n, co, mo = int(u["n_values"]), int(u["cache_off"]), int(u["msg_off"])
+            cs = self.cache_s[co : co + n].copy()
+            m, wb, pb, cb = ora.encode(self._w(w_flat, u), cs, self.dtype, self.block)
+            self.cache_s[co : co + n] = cs
+            msgs[mo : mo + wb] = m
+            wire[i], chg[i], pay[i] = wb, cb, pb
+            cr = self.cache_r[co : co + n].copy()
+            out = ora.decode(m, cr, self.dtype, self.block)
+            self.cache_r[co : co + n] = cr
+            lo = int(u["weights_off"]) // VB[self.dtype]
+            recon[lo : lo + n] = out
+        return dict(msgs=msgs, wire=wire, chg=chg, pay=pay, recon=recon)
+
+
+def to_dev_bytes(bits: np.ndarray, device) -> torch.Tensor:
+    """Raw bytes of a host bit-pattern array, on the device (padded to >= 16 bytes)."""
+    b = np.ascontiguousarray(bits).view(np.uint8)
+    if b.size < 16:
+        b = np.concatenate([b, np.zeros(16 - b.size, np.uint8)])
+    return torch.from_numpy(b.copy()).to(device)
+
+
+def dev_to_bits(t: torch.Tensor, dtype: int, n: int) -> np.ndarray:
+    return t.cpu().numpy().view(WDT[dtype])[:n]
+
+
+def compare_step(codec, exp, w_flat, label=""):
+    """Bit-exact comparison of one finished GPU step (codec: LayerCodec) with the oracle's."""
+    units = codec.units
+    nu = len(units)
+    wire = codec.wire_bytes.cpu().numpy().astype(np.uint64)[:nu]
+    chg = codec.changed_blocks.cpu().numpy().astype(np.uint32)[:nu]
+    assert np.array_equal(wire, exp["wire"]), f"{label}: wire bytes differ"
+    assert np.array_equal(chg, exp["chg"]), f"{label}: changed-block counts differ"
+    ms = codec.msg_send.cpu().numpy()
+    mr = codec.msg_recv.cpu().numpy()
+    for i, u in enumerate(units):
+        mo, wb = int(u["msg_off"]), int(wire[i])
+        if not np.array_equal(ms[mo : mo + wb], exp["msgs"][mo : mo + wb]):
+            bad = np.nonzero(ms[mo : mo + wb] != exp["msgs"][mo : mo + wb])[0]
+            raise AssertionError(f"{label}: message of unit {i} (N={int(u['n_values'])}) differs at bytes {bad[:8]}")
+        assert np.array_equal(mr[mo : mo + wb], exp["msgs"][mo : mo + wb]), f"{label}: transported message {i}"
+    return wire, chg
+
+
+def compare_caches(codec, table, label=""):
+    cs = codec.sender_cache.cpu().numpy()
+    cr = codec.receiver_cache.cpu().numpy()
+    for i, u in enumerate(codec.units):
+        co, n = int(u["cache_off"]), int(u["n_values"])
+        assert np.array_equal(cs[co : co + n], table.cache_s[co : co + n]), f"{label}: sender cache unit {i}"
+        assert np.array_equal(cr[co : co + n], table.cache_r[co : co + n]), f"{label}: receiver cache unit {i}"
+
+
+def compare_recon(codec, exp, w_flat, dtype, label=""):
+    out = codec.weights_out.cpu().numpy().view(WDT[dtype])
+    for i, u in enumerate(codec.units):
+        lo, n = int(u["weights_off"]) // VB[dtype], int(u["n_values"])
+        assert np.array_equal(out[lo : lo + n], exp["recon"][lo : lo + n]), f"{label}: reconstruction unit {i}"
+        assert np.array_equal(out[lo : lo + n], w_flat[lo : lo + n]), f"{label}: round trip unit {i}"

