@@ -1,0 +1,574 @@
+#!/usr/bin/env python
+"""Benchmark of the exponent-reuse codec hot path on B200.
+
+One *step* = one pass of the whole path over one iterate of the synthetic weight trajectory:
+for every layer, sender-side encode, the device-to-device transport that stands where the
+Allgather would be, and receiver-side decode -- layer-pipelined on two streams.
+
+Workload at one GPU: the full OLMoE-1B-7B expert stack (16 layers x 64 experts x 3 matrices,
+bf16, 6.44 G values = 12.9 GB), 16 simulated shards per matrix, block size 512, with the
+clustered update model (a fraction f = 0.22 of 512-aligned segments receives an Adam-like
+update each iteration; the rest is bit-identical), which reproduces the block change rate the
+paper reports for OLMoE expert-FFN shards.  Two consecutive iterates are kept on the device and
+the steps alternate between them (the set of changed exponents between A and B is the same in
+both directions), so every step is a real encode against a cache left by the previous one and
+the K timed steps run back to back.
+
+Prints ONE JSON line (rank 0).  ``--impl reference`` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "encode/decode GB/s of weights"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic of one encode launch per value, from the ncu capture summarised under profiles/
+# (dram__bytes_read.sum + dram__bytes_write.sum of a smaller case, divided by its values); None
+# until a capture exists for the current kernel.
+NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE = None
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=16, help="layers of the expert stack (16 = full model)")
+    ap.add_argument("--experts", type=int, default=64)
+    ap.add_argument("--shards", type=int, default=16)
+    ap.add_argument("--block", type=int, default=512)
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
+    ap.add_argument("--update", default="clustered", choices=["clustered", "adam"])
+    ap.add_argument("--f", type=float, default=0.22, help="fraction of segments updated (clustered model)")
+    ap.add_argument("--schedule", default="pipelined", choices=["pipelined", "serial"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-regimes", action="store_true")
+    ap.add_argument("--cpu-sample-units", type=int, default=1024)
+    return ap.parse_args()
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(p))["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# --------------------------------------------------------------------------------- clocks
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs
+    (read-only queries)."""
+
+    def __init__(self, index: int, uuid: str = "", period_s: float = 0.05):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if uuid else b"")
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join()
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------------- workload
+
+
+def build_stack(args, device, seed_base):
+    """Layers of the expert stack with two consecutive iterates W_a, W_b per layer on the device."""
+    import torch
+
+    from paper_2609_04609_b200 import runtime
+    from paper_2609_04609_b200 import workloads as wl
+
+    shapes = [r * c for r, c in wl.olmoe_layer_shapes(args.experts)]
+    layers, wa, wb = [], [], []
+    for l in range(args.layers):
+        codec = runtime.LayerCodec.from_tensors(shapes, args.shards, args.dtype, args.block, device)
+        n = codec.weights_bytes // wl.VALUE_BYTES[args.dtype]
+        gen = wl.make_generator(seed_base + l, device)
+        w = wl.init_weights(n, args.dtype, gen)
+        step = (lambda x: wl.step_clustered(x, gen, f=args.f, seg=512)) if args.update == "clustered" else (
+            lambda x: wl.step_adam_like(x, gen))
+        for _ in range(4):  # iterations 1..4 of the trajectory
+            w = step(w)
+        w5 = step(w)  # iteration 5
+        layers.append(codec)
+        wa.append(w.view(torch.uint8))
+        wb.append(w5.view(torch.uint8))
+        codec.init_caches(wa[-1])
+    torch.cuda.synchronize()
+    return layers, wa, wb
+
+
+def algorithmic_bytes(n_values, q, dtype):
+    """HBM bytes per launch the method needs: (encode, transport, decode)."""
+    vb, smb = (2, 1) if dtype == "bf16" else (4, 3)
+    enc = n_values * (vb + 1 + smb + 2 * q)
+    tra = 2 * n_values * (smb + q)
+    dec = n_values * (smb + (1 - q) + q + vb + q)
+    return enc, tra, dec
+
+
+def run_step(layers, weights, s_enc, s_dec, events, schedule, timers=None):
+    """encode+transport of layer l on s_enc, decode of layer l on s_dec (same stream if serial)."""
+    import torch
+
+    for l, (codec, w) in enumerate(zip(layers, weights)):
+        if timers is not None:
+            t = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
+            t[0].record(s_enc)
+        codec.encode(w, s_enc)
+        if timers is not None:
+            t[1].record(s_enc)
+            t[2].record(s_enc)
+        codec.transport(s_enc)
+        if timers is not None:
+            t[3].record(s_enc)
+        if schedule == "pipelined":
+            events[l].record(s_enc)
+            s_dec.wait_event(events[l])
+        if timers is not None:
+            t[4].record(s_dec)
+        codec.decode(None, s_dec)
+        if timers is not None:
+            t[5].record(s_dec)
+            timers.append(t)
+
+
+def oracle_roundtrip_units(units, w_prev, w_cur, dtype_code, block, vb, threads):
+    """CPU oracle (as it stands) on a list of units: cache init from w_prev, encode + decode of
+    w_cur.  Returns seconds of wall time with ``threads`` host threads."""
+    from concurrent.futures import ThreadPoolExecutor
+
+    from oracle import ciera_oracle as ora
+
+    ora.build()
+    wdt = np.uint16 if dtype_code == 0 else np.uint32
+    prev = w_prev.view(wdt)
+    cur = w_cur.view(wdt)
+    jobs = []
+    for u in units:
+        lo, n = int(u["weights_off"]) // vb, int(u["n_values"])
+        jobs.append((prev[lo : lo + n], cur[lo : lo + n]))
+    caches = [ora.cache_init(p, p.size, dtype_code) for p, _ in jobs]
+    caches_r = [c.copy() for c in caches]
+
+    def work(i):
+        m, wb, pb, cb = ora.encode(jobs[i][1], caches[i], dtype_code, block)
+        out = ora.decode(m, caches_r[i], dtype_code, block)
+        return np.array_equal(out, jobs[i][1])
+
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        ok = list(ex.map(work, range(len(jobs))))
+    dt = time.perf_counter() - t0
+    assert all(ok), "oracle round trip failed"
+    return dt, sum(j[1].size for j in jobs)
+
+
+# --------------------------------------------------------------------------------- reference arm
+
+
+def run_reference(args):
+    """Times the CPU oracle on the host cores, on a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+
+    from paper_2609_04609_b200 import workloads as wl
+    from oracle import ciera_oracle as ora
+
+    ora.build()
+    code = 0 if args.dtype == "bf16" else 1
+    vb = wl.VALUE_BYTES[args.dtype]
+    shapes = [r * c for r, c in wl.olmoe_layer_shapes(args.experts)]
+    n_units = min(args.cpu_sample_units, len(shapes) * args.shards)
+    units, wbytes, _, _ = wl.layout_units(shapes, args.shards, vb, lambda n: ora.message_capacity(n, code, args.block))
+    units = units[:n_units]
+    n = int(units[-1]["weights_off"]) // vb + int(units[-1]["n_values"])
+    gen = wl.make_generator(1234 + 3)
+    w = wl.init_weights(n, args.dtype, gen)
+    step = (lambda x: wl.step_clustered(x, gen, f=args.f, seg=512)) if args.update == "clustered" else (
+        lambda x: wl.step_adam_like(x, gen))
+    w1 = step(w)
+    a = wl.as_bits(w).view(np.uint8)
+    b = wl.as_bits(w1).view(np.uint8)
+    threads = os.cpu_count() or 1
+    times = []
+    nvals = 0
+    for i in range(args.warmup + args.steps):
+        prev, cur = (a, b) if i % 2 == 0 else (b, a)
+        dt, nvals = oracle_roundtrip_units(units, prev, cur, code, args.block, vb, threads)
+        if i >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * float(np.mean(times))
+    gbps = nvals * vb / (ms * 1e-3) / 1e9
+    sample = f"{n_units} of {len(shapes) * args.shards * args.layers} units ({nvals} values) per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": gbps, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
+        "config": workload_config(args),
+        "cpu_baseline": {"value": gbps, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbps, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def workload_config(args):
+    full = args.layers == 16 and args.experts == 64
+    name = ("config3: full OLMoE-1B-7B expert stack" if full else "reduced OLMoE expert stack")
+    return {
+        "workload": f"{name}, {args.layers} layers x {args.experts} experts x 3 matrices (2048x1024, 2048x1024, "
+                    f"1024x2048) {args.dtype}, {args.shards} simulated shards per matrix, block {args.block}, "
+                    f"update model {args.update}" + (f" f={args.f}" if args.update == "clustered" else ""),
+        "l2": "inputs larger than L2 (no flush needed)",
+        "schedule": args.schedule,
+        "round_trip": "encode + device-to-device transport + decode",
+    }
+
+
+# --------------------------------------------------------------------------------- main arm
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2609_04609_b200 import ciera, runtime
+    from paper_2609_04609_b200 import workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the codec has no CPU path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    peak, peak_kind = measured_peak()
+    vb = wl.VALUE_BYTES[args.dtype]
+    layers, wa, wb = build_stack(args, device, seed_base=1234 + 3 + 1000 * rank)
+    n_values = sum(c.plan.total_values for c in layers)
+    weight_bytes = n_values * vb
+    s_enc, s_dec = torch.cuda.Stream(), torch.cuda.Stream()
+    if args.schedule == "serial":
+        s_dec = s_enc
+    events = [torch.cuda.Event() for _ in layers]
+
+    def weights_of(i):
+        return wb if i % 2 == 0 else wa
+
+    step_i = 0
+    for _ in range(max(args.warmup, 3)):
+        run_step(layers, weights_of(step_i), s_enc, s_dec, events, args.schedule)
+        step_i += 1
+    barrier()
+
+    # ---- timed region: exactly K steps, device-timed, launch accounting, clocks sampled
+    try:
+        uuid = "GPU-" + str(torch.cuda.get_device_properties(device).uuid)
+    except Exception:
+        uuid = ""
+    sampler = ClockSampler(local_rank, uuid)
+    timers = []
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = ciera.kernel_launch_count()
+    sampler.start()
+    barrier()
+    cur = torch.cuda.current_stream()
+    ev0.record(cur)
+    s_enc.wait_event(ev0)
+    s_dec.wait_event(ev0)
+    for _ in range(args.steps):
+        run_step(layers, weights_of(step_i), s_enc, s_dec, events, args.schedule, timers)
+        step_i += 1
+    cur.wait_stream(s_enc)
+    cur.wait_stream(s_dec)
+    ev1.record(cur)
+    barrier()
+    clocks = sampler.stop()
+    launches = ciera.kernel_launch_count() - launches0
+    ms_total = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([ms_total], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    for c in layers:
+        c.check_status()
+
+    # ---- what was moved: change rates and the paper's byte count of the last step
+    changed = sum(int(c.changed_blocks.sum().item()) for c in layers)
+    blocks = sum(c.n_blocks() for c in layers)
+    q = changed / blocks
+    paper_bytes = sum(c.paper_bytes() for c in layers)
+    enc_ms = float(np.mean([t[0].elapsed_time(t[1]) for t in timers]))
+    tra_ms = float(np.mean([t[2].elapsed_time(t[3]) for t in timers]))
+    dec_ms = float(np.mean([t[4].elapsed_time(t[5]) for t in timers]))
+    n_layer = layers[0].plan.total_values
+    a_enc, a_tra, a_dec = algorithmic_bytes(n_layer, q, args.dtype)
+    enc_gbs = a_enc / (enc_ms * 1e-3) / 1e9
+
+    # ---- correctness at full size: exact round trip everywhere, oracle on sampled units
+    last_w = weights_of(step_i - 1)
+    prev_w = weights_of(step_i)
+    verified = all(torch.equal(c.weights_out[: w.numel()], w) for c, w in zip(layers, last_w))
+    verified = verified and all(torch.equal(c.sender_cache, c.receiver_cache) for c in layers)
+    sampled = 0
+    if rank == 0:
+        from oracle import ciera_oracle as ora
+
+        ora.build()
+        code = ciera.DTYPE_CODES[args.dtype]
+        wdt = np.uint16 if code == 0 else np.uint32
+        rng = np.random.default_rng(0)
+        for l in sorted(set(rng.integers(0, len(layers), 4).tolist())):
+            c = layers[l]
+            for ui in rng.integers(0, len(c.units), 4):
+                u = c.units[ui]
+                lo, n, mo, co = int(u["weights_off"]), int(u["n_values"]), int(u["msg_off"]), int(u["cache_off"])
+                w_prev = prev_w[l][lo : lo + n * vb].cpu().numpy().view(wdt)
+                w_cur = last_w[l][lo : lo + n * vb].cpu().numpy().view(wdt)
+                cache = ora.cache_init(w_prev, n, code)
+                m, wbytes, _, cb = ora.encode(w_cur, cache, code, args.block)
+                got = c.msg_recv[mo : mo + wbytes].cpu().numpy()
+                verified = verified and int(c.wire_bytes[ui].item()) == wbytes and np.array_equal(got, m)
+                verified = verified and int(c.changed_blocks[ui].item()) == cb
+                verified = verified and np.array_equal(c.sender_cache[co : co + n].cpu().numpy(), cache)
+                sampled += 1
+
+    out = {
+        "metric": METRIC,
+        "value": world * weight_bytes / (ms_per_step * 1e-3) / 1e9,
+        "unit": "GB/s",
+        "n_gpus": world,
+        "steps": args.steps,
+        "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_per_step,
+        "higher_is_better": True,
+        "scaling": "weak",
+        "vs_baseline": None,
+        "dtype": "u32",
+        "data": "synthetic",
+        "config": workload_config(args),
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "verified_bit_exact": bool(verified),
+        "oracle_sampled_units": sampled,
+        "block_change_rate_q": q,
+        "bytes_ratio": paper_bytes / weight_bytes,
+        "encode_GBps_of_weights": n_layer * vb / (enc_ms * 1e-3) / 1e9,
+        "decode_GBps_of_weights": n_layer * vb / (dec_ms * 1e-3) / 1e9,
+        "transport_GBps": a_tra / (tra_ms * 1e-3) / 1e9,
+        "decode_hbm_GBps": a_dec / (dec_ms * 1e-3) / 1e9,
+        "kernel_ms": {"encode": enc_ms, "transport": tra_ms, "decode": dec_ms, "per": "layer launch, timed region"},
+        "roofline": {
+            "bound": "hbm", "kernel": "encode_kernel", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
+            "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBps": enc_gbs / NOMINAL_HBM_GBS,
+            "traffic": (NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE * n_layer if NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE else None),
+            "algorithmic_bytes_per_launch": a_enc,
+        },
+    }
+
+    # ---- per-kernel numbers with each kernel alone on the GPU, three change regimes (one layer)
+    if not args.no_regimes and rank == 0:
+        out["kernels_alone"] = kernels_alone(args, layers[0], wa[0], wb[0], peak)
+
+    # ---- end to end through the host-buffer entry point (weights start and end in host memory)
+    if not args.no_e2e:
+        out["e2e"] = e2e(args, layers, wa, wb, world, rank, barrier)
+
+    # ---- the oracle on this machine's host cores (rank 0, one GPU only)
+    if not args.no_cpu_baseline and rank == 0 and world == 1:
+        threads = os.cpu_count() or 1
+        units = layers[0].units[: args.cpu_sample_units]
+        hi = int(units[-1]["weights_off"]) + int(units[-1]["n_values"]) * vb
+        a = wa[0][:hi].cpu().numpy()
+        b = wb[0][:hi].cpu().numpy()
+        dt, nv = oracle_roundtrip_units(units, a, b, ciera.DTYPE_CODES[args.dtype], args.block, vb, threads)
+        out["cpu_baseline"] = {"value": nv * vb / dt / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
+                               "sample": f"{len(units)} of {sum(len(c.units) for c in layers)} units "
+                                         f"({nv} values), encode+decode round trip, {dt:.2f} s wall"}
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def kernels_alone(args, codec, w_a, w_b, peak):
+    """Each kernel timed alone (events on its stream, nothing else running) on one layer, at block
+    change rates ~0 (nothing changed), the workload's own, and 1 (every block changed)."""
+    import torch
+
+    res = {}
+    vb = 2 if args.dtype == "bf16" else 4
+    n = codec.plan.total_values
+    # lowest exponent bit flipped everywhere: every block changes
+    if vb == 2:
+        w_c = (w_a.view(torch.int16) ^ 0x0080).view(torch.uint8)
+    else:
+        w_c = (w_a.view(torch.int32) ^ 0x00800000).view(torch.uint8)
+
+    def timed(fn, reps=5):
+        ts = []
+        for _ in range(reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return float(np.median(ts))
+
+    for name, first, second in (("q0", w_a, w_a), ("workload", w_a, w_b), ("q1", w_a, w_c)):
+        enc, tra, dec = [], [], []
+        for _ in range(5):
+            codec.init_caches(first)
+            enc.append(timed(lambda: codec.encode(second), 1))
+            tra.append(timed(lambda: codec.transport(), 1))
+            dec.append(timed(lambda: codec.decode(), 1))
+        q = int(codec.changed_blocks.sum().item()) / codec.n_blocks()
+        a_enc, a_tra, a_dec = algorithmic_bytes(n, q, args.dtype)
+        e, t, d = float(np.median(enc)), float(np.median(tra)), float(np.median(dec))
+        res[name] = {
+            "q": q,
+            "encode_ms": e, "encode_hbm_GBps": a_enc / e / 1e6, "encode_frac": a_enc / e / 1e6 / peak,
+            "encode_GBps_of_weights": n * vb / e / 1e6,
+            "transport_ms": t, "transport_hbm_GBps": a_tra / t / 1e6, "transport_frac": a_tra / t / 1e6 / peak,
+            "decode_ms": d, "decode_hbm_GBps": a_dec / d / 1e6, "decode_frac": a_dec / d / 1e6 / peak,
+            "decode_GBps_of_weights": n * vb / d / 1e6,
+        }
+    codec.init_caches(w_a)
+    return res
+
+
+def e2e(args, layers, wa, wb, world, rank, barrier):
+    """Same step, but the weights start in pinned host memory and the reconstructed weights end
+    there: every layer goes through ciera_roundtrip_host (H2D copy, encode, transport, decode,
+    D2H copy), two streams so that the copies of neighbouring layers overlap."""
+    import torch
+    import torch.distributed as dist
+
+    host_a = [torch.empty(w.numel(), dtype=torch.uint8, pin_memory=True) for w in wa]
+    host_b = [torch.empty(w.numel(), dtype=torch.uint8, pin_memory=True) for w in wb]
+    host_out = [torch.empty(w.numel(), dtype=torch.uint8, pin_memory=True) for w in wa]
+    wire_host = [torch.empty(len(c.units), dtype=torch.int64, pin_memory=True) for c in layers]
+    for h, w in zip(host_a, wa):
+        h.copy_(w)
+    for h, w in zip(host_b, wb):
+        h.copy_(w)
+    for c, w in zip(layers, wa):
+        c.init_caches(w)
+    staging = [torch.empty_like(wa[0]) for _ in range(2)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+
+    def step(src):
+        for l, c in enumerate(layers):
+            c.step_host(src[l], host_out[l], staging[l % 2], wire_host[l], streams[l % 2])
+
+    steps = max(1, min(args.steps, 3))
+    step(host_b)
+    step(host_a)
+    barrier()
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    cur = torch.cuda.current_stream()
+    t0.record(cur)
+    for s in streams:
+        s.wait_event(t0)
+    for i in range(steps):
+        step(host_b if i % 2 == 0 else host_a)
+    for s in streams:
+        cur.wait_stream(s)
+    t1.record(cur)
+    barrier()
+    ms = t0.elapsed_time(t1) / steps
+    if world > 1:
+        t = torch.tensor([ms], device=wa[0].device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ok = all(torch.equal(o, (host_b if (steps - 1) % 2 == 0 else host_a)[l]) for l, o in enumerate(host_out))
+    nbytes = sum(h.numel() for h in host_a)
+    return {"value": world * nbytes / (ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms, "steps": steps,
+            "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes + 8 * sum(len(c.units) for c in layers),
+            "bit_exact": bool(ok), "api": "ciera_roundtrip_host (pinned host weights in, host weights out)"}
+
+
+if __name__ == "__main__":
+    main()

@@ -130,10 +130,10 @@ CIERA_API int ciera_plan_bind(ciera_plan* plan, void* plan_dev, size_t plan_dev_
 
 /* ---- caches (Algorithm 1: persistent sender / receiver state) ------------------------------ */
 
-/* cache := exponents of `weights_dev`, or all zero if weights_dev == NULL.  The paper starts
- * "after model initialization and warmup" without fixing the first cache state; initialising
- * both sides from the same weights (as if they had been sent uncompressed), or both to zero,
- * keeps them in agreement. */
+/* cache := exponents of `weights_dev`, or all zero if weights_dev == NULL.  The paper switches
+ * its method on once warm-up is over and does not say what the caches hold at that moment;
+ * initialising both sides from the same weights (as if they had been sent uncompressed), or
+ * both to zero, keeps them in agreement. */
 CIERA_API int ciera_cache_init(const ciera_plan* plan, void* cache_dev, const void* weights_dev, void* stream);
 /* cache := exponents of `weights_dev`, unconditionally (e.g. after a checkpoint restore). */
 CIERA_API int ciera_cache_update(const ciera_plan* plan, void* cache_dev, const void* weights_dev, void* stream);
@@ -180,6 +180,32 @@ CIERA_API int ciera_transport(const ciera_plan* plan, const void* src_messages_d
  */
 CIERA_API int ciera_decode(const ciera_plan* plan, const void* messages_dev, void* receiver_cache_dev,
                  void* weights_out_dev, const uint64_t* wire_bytes_dev, int32_t* status_dev, void* stream);
+
+/* ---- whole step with host buffers ---------------------------------------------------------- */
+
+/* Device buffers one ciera_roundtrip_host call works in; all caller-owned, sized as for the
+ * separate calls above (weights_dev / weights_out_dev: weights_bytes each). */
+typedef struct ciera_device_buffers {
+    void* weights_dev;
+    void* sender_cache_dev;
+    void* msg_send_dev;
+    void* msg_recv_dev;
+    void* receiver_cache_dev;
+    void* weights_out_dev;
+    uint64_t* wire_bytes_dev;
+    uint32_t* changed_blocks_dev;
+    void* workspace_dev;
+    int32_t* status_dev;
+} ciera_device_buffers;
+
+/* One sender + receiver step of Algorithm 1 on weights that live in HOST memory:
+ * copy `weights_host` (weights_bytes, ideally pinned) to the device, ciera_encode,
+ * ciera_transport, ciera_decode, copy the reconstructed weights to `weights_out_host` and the
+ * per-unit wire lengths to `wire_bytes_host` ([n_units], may be NULL).  Everything is enqueued on
+ * `stream`; the host buffers must stay valid until the stream has drained. */
+CIERA_API int ciera_roundtrip_host(const ciera_plan* plan, const void* weights_host, size_t weights_bytes,
+                         void* weights_out_host, uint64_t* wire_bytes_host, const ciera_device_buffers* bufs,
+                         void* stream);
 
 /* ---- selective compression: the gain rule of Section 3.2 (host only) ----------------------- */
 

@@ -70,6 +70,7 @@ _SIGS = {
     "ciera_encode": ([_vp] * 9, _i32),
     "ciera_transport": ([_vp] * 5, _i32),
     "ciera_decode": ([_vp] * 7, _i32),
+    "ciera_roundtrip_host": ([_vp, _vp, _sz, _vp, _vp, _vp, _vp], _i32),
     "ciera_should_compress": ([ctypes.POINTER(GainIn), ctypes.POINTER(_dbl), ctypes.POINTER(_i32)], _i32),
     "ciera_last_cuda_error": ([], _i32),
     "ciera_kernel_launch_count": ([], _u64),
@@ -212,6 +213,21 @@ def decode(plan: Plan, messages, receiver_cache, weights_out, wire_bytes=None, s
     _check("ciera_decode",
            _lib.ciera_decode(plan.handle, _ptr(messages), _ptr(receiver_cache), _ptr(weights_out), _ptr(wire_bytes),
                              _ptr(status), _stream(stream)))
+
+
+class DeviceBuffers(ctypes.Structure):
+    _fields_ = [(n, _vp) for n in ("weights_dev", "sender_cache_dev", "msg_send_dev", "msg_recv_dev",
+                                   "receiver_cache_dev", "weights_out_dev", "wire_bytes_dev", "changed_blocks_dev",
+                                   "workspace_dev", "status_dev")]
+
+
+def roundtrip_host(plan: Plan, weights_host: torch.Tensor, weights_out_host: torch.Tensor,
+                   wire_bytes_host: Optional[torch.Tensor], bufs: DeviceBuffers, stream=None) -> None:
+    """Host weights in, host weights out (both CPU tensors, ideally pinned); see ciera.h."""
+    nbytes = weights_host.numel() * weights_host.element_size()
+    _check("ciera_roundtrip_host",
+           _lib.ciera_roundtrip_host(plan.handle, _ptr(weights_host), nbytes, _ptr(weights_out_host),
+                                     _ptr(wire_bytes_host), ctypes.addressof(bufs), _stream(stream)))
 
 
 # ------------------------------------------------------------------------------ gain rule (host)

@@ -491,3 +491,30 @@ extern "C" int ciera_decode(const ciera_plan* p, const void* messages_dev, void*
     count_launch();
     return check_launch();
 }
+
+extern "C" int ciera_roundtrip_host(const ciera_plan* p, const void* weights_host, size_t weights_bytes,
+                                    void* weights_out_host, uint64_t* wire_bytes_host, const ciera_device_buffers* b,
+                                    void* stream) {
+    int rc = check_plan(p);
+    if (rc) return rc;
+    if (!b || !weights_host || !weights_out_host) return CIERA_ERR_INVALID_ARG;
+    if (p->tiles.empty()) return CIERA_OK;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaMemcpyAsync(b->weights_dev, weights_host, weights_bytes, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    rc = ciera_encode(p, b->weights_dev, b->sender_cache_dev, b->msg_send_dev, b->wire_bytes_dev, b->changed_blocks_dev,
+                      b->workspace_dev, b->status_dev, stream);
+    if (rc) return rc;
+    rc = ciera_transport(p, b->msg_send_dev, b->msg_recv_dev, b->wire_bytes_dev, stream);
+    if (rc) return rc;
+    rc = ciera_decode(p, b->msg_recv_dev, b->receiver_cache_dev, b->weights_out_dev, b->wire_bytes_dev, b->status_dev,
+                      stream);
+    if (rc) return rc;
+    e = cudaMemcpyAsync(weights_out_host, b->weights_out_dev, weights_bytes, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    if (wire_bytes_host) {
+        e = cudaMemcpyAsync(wire_bytes_host, b->wire_bytes_dev, sizeof(uint64_t) * p->n_units, cudaMemcpyDeviceToHost, s);
+        if (e != cudaSuccess) return record_cuda_error(e);
+    }
+    return CIERA_OK;
+}

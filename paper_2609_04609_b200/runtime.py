@@ -72,6 +72,25 @@ class LayerCodec:
         self.transport(stream)
         self.decode(weights_out, stream)
 
+    def device_buffers(self, weights_dev: torch.Tensor) -> "ciera.DeviceBuffers":
+        b = ciera.DeviceBuffers()
+        b.weights_dev = weights_dev.data_ptr()
+        b.sender_cache_dev = self.sender_cache.data_ptr()
+        b.msg_send_dev = self.msg_send.data_ptr()
+        b.msg_recv_dev = self.msg_recv.data_ptr()
+        b.receiver_cache_dev = self.receiver_cache.data_ptr()
+        b.weights_out_dev = self.weights_out.data_ptr()
+        b.wire_bytes_dev = self.wire_bytes.data_ptr()
+        b.changed_blocks_dev = self.changed_blocks.data_ptr()
+        b.workspace_dev = self.workspace.data_ptr()
+        b.status_dev = self.status.data_ptr()
+        return b
+
+    def step_host(self, weights_host: torch.Tensor, weights_out_host: torch.Tensor, staging: torch.Tensor,
+                  wire_host: Optional[torch.Tensor] = None, stream=None) -> None:
+        """Whole step on host-resident weights through ``ciera_roundtrip_host``."""
+        ciera.roundtrip_host(self.plan, weights_host, weights_out_host, wire_host, self.device_buffers(staging), stream)
+
     def check_status(self) -> None:
         s = int(self.status.item())
         if s != 0:
