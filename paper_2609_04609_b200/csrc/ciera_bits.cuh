@@ -14,6 +14,25 @@ namespace ciera {
 
 __device__ __forceinline__ uint4 ld_stream16(const void* p) { return __ldcs(reinterpret_cast<const uint4*>(p)); }
 __device__ __forceinline__ void st_stream16(void* p, uint4 v) { __stcs(reinterpret_cast<uint4*>(p), v); }
+__device__ __forceinline__ uint4 ld_shared16(const void* p) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "r"((uint32_t)__cvta_generic_to_shared(p)));
+    return v;
+}
+__device__ __forceinline__ void st_shared16(void* p, uint4 v) {
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"((uint32_t)__cvta_generic_to_shared(p)), "r"(v.x),
+                 "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+// where a group's 16-byte pieces come from: global memory (streaming) or a staged shared-memory tile
+struct FromGlobal {
+    __device__ __forceinline__ uint4 operator()(const uint8_t* p) const { return ld_stream16(p); }
+};
+struct FromShared {
+    __device__ __forceinline__ uint4 operator()(const uint8_t* p) const { return ld_shared16(p); }
+};
 
 // ---- bf16 --------------------------------------------------------------------------------
 // a = v0 | v1 << 16, b = v2 | v3 << 16  ->  e0 | e1<<8 | e2<<16 | e3<<24
@@ -66,8 +85,9 @@ struct Group<CIERA_BF16> {
     uint32_t s[4];  // 16 sm bytes
 
     // 16 values from 32 aligned bytes
-    __device__ __forceinline__ void split_full(const uint8_t* w) {
-        uint4 a = ld_stream16(w), b = ld_stream16(w + 16);
+    template <class Ld = FromGlobal>
+    __device__ __forceinline__ void split_full(const uint8_t* w, Ld ld = Ld()) {
+        uint4 a = ld(w), b = ld(w + 16);
         e[0] = bf16_exp4(a.x, a.y); e[1] = bf16_exp4(a.z, a.w); e[2] = bf16_exp4(b.x, b.y); e[3] = bf16_exp4(b.z, b.w);
         s[0] = bf16_sm4(a.x, a.y);  s[1] = bf16_sm4(a.z, a.w);  s[2] = bf16_sm4(b.x, b.y);  s[3] = bf16_sm4(b.z, b.w);
     }
@@ -92,8 +112,9 @@ struct Group<CIERA_BF16> {
         for (int i = 0; i < 16; ++i)
             if (i < nvalid) dst[i] = (uint8_t)(s[i >> 2] >> (8 * (i & 3)));
     }
-    __device__ __forceinline__ void load_sm_full(const uint8_t* src) {
-        uint4 v = ld_stream16(src);
+    template <class Ld = FromGlobal>
+    __device__ __forceinline__ void load_sm_full(const uint8_t* src, Ld ld = Ld()) {
+        uint4 v = ld(src);
         s[0] = v.x; s[1] = v.y; s[2] = v.z; s[3] = v.w;
     }
     __device__ __forceinline__ void load_sm_partial(const uint8_t* src, int nvalid) {
@@ -134,11 +155,12 @@ struct Group<CIERA_FP32> {
                        s[3 * i], s[3 * i + 1], s[3 * i + 2]);
         }
     }
-    __device__ __forceinline__ void split_full(const uint8_t* w) {
+    template <class Ld = FromGlobal>
+    __device__ __forceinline__ void split_full(const uint8_t* w, Ld ld = Ld()) {
         uint32_t x[16];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            uint4 v = ld_stream16(w + 16 * i);
+            uint4 v = ld(w + 16 * i);
             x[4 * i] = v.x; x[4 * i + 1] = v.y; x[4 * i + 2] = v.z; x[4 * i + 3] = v.w;
         }
         from_words(x);
@@ -159,10 +181,11 @@ struct Group<CIERA_FP32> {
         for (int i = 0; i < 48; ++i)
             if (i < 3 * nvalid) dst[i] = (uint8_t)(s[i >> 2] >> (8 * (i & 3)));
     }
-    __device__ __forceinline__ void load_sm_full(const uint8_t* src) {
+    template <class Ld = FromGlobal>
+    __device__ __forceinline__ void load_sm_full(const uint8_t* src, Ld ld = Ld()) {
 #pragma unroll
         for (int i = 0; i < 3; ++i) {
-            uint4 v = ld_stream16(src + 16 * i);
+            uint4 v = ld(src + 16 * i);
             s[4 * i] = v.x; s[4 * i + 1] = v.y; s[4 * i + 2] = v.z; s[4 * i + 3] = v.w;
         }
     }

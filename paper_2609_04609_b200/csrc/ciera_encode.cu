@@ -1,0 +1,525 @@
+// Sender side (paper Algorithm 1, sender part; Section 3.1) as one persistent sm_100a kernel.
+//
+// Grid = G thread blocks that are all resident at once (cooperative launch); block c works on
+// tiles c, c + G, c + 2G, ... of the plan's tile table, so neighbouring tiles of a unit are worked
+// on by neighbouring blocks at about the same time and the look-back below rarely waits.
+// A thread block has four roles:
+//
+//   producer warp   runs ahead of the others: for each of its tiles it fetches the tile
+//                   descriptor and starts two bulk-async copies into shared memory -- the weights
+//                   tile into a short ring (freed as soon as the consumers have read it) and the
+//                   cached-exponent tile into a longer ring (held until the tile is resolved);
+//   16 consumer     each thread owns 16 consecutive values: split into exponent bytes and
+//   warps           sign-plus-mantissa, compare with the cached exponents, vote (ballot) the
+//                   "my 16 values changed" bit, store sign-plus-mantissa to the message and
+//                   leave the new exponents where the cached ones were staged;
+//   aggregator warp turns the 512 vote bits of a tile into block flags (the unit's bitmap), counts
+//                   the tile's payload bytes and publishes them as the tile's status word;
+//   resolver warps  resolve the tile's exclusive offset in the unit's payload with a single-pass
+//                   look-back over the status words, then send the exponents of changed blocks
+//                   from shared memory to the payload and to the cache, and hand the stage back.
+//
+// Only the resolvers ever wait for another thread block; consumers and aggregator never do, so
+// a tile's status is published as soon as its votes are in.
+#include "ciera_bits.cuh"
+#include "ciera_pipe.cuh"
+
+namespace ciera {
+
+constexpr int kResolvers = 3;                       // resolver warps
+constexpr int kEncodeThreads = kThreads + 64 + 32 * kResolvers;  // consumers + producer + aggregator + resolvers
+constexpr int kProducerWarp = kWarps;               // 16
+constexpr int kAggregatorWarp = kWarps + 1;         // 17
+constexpr int kResolverWarp0 = kWarps + 2;          // 18 ..
+constexpr int kDescRing = 16;                       // > exponent stages + 2
+
+template <int DT>
+struct EncodeCfg;
+template <>
+struct EncodeCfg<CIERA_BF16> {
+    static constexpr int kWStages = 3;  // 3 x 16 KB weights tiles
+    static constexpr int kEStages = 7;  // 7 x  8 KB exponent tiles
+};
+template <>
+struct EncodeCfg<CIERA_FP32> {
+    static constexpr int kWStages = 2;  // 2 x 32 KB
+    static constexpr int kEStages = 5;  // 5 x  8 KB
+};
+
+template <int SW, int SE>
+struct EncodeCtl {
+    uint64_t full_w[SW];   // weights tile landed
+    uint64_t empty_w[SW];  // all 16 consumer warps have read it
+    uint64_t full_e[SE];   // cached-exponent tile landed
+    uint64_t voted[SE];    // all 16 consumer warps have left their exponents there and voted
+    uint64_t summed[SE];   // aggregator has published the tile's status and block flags
+    uint64_t empty_e[SE];  // resolver is done with the tile
+    TileDesc desc[kDescRing];
+    uint32_t tile_idx[kDescRing];  // table index of the tile in desc[]; kNoTile = no more work
+    uint32_t ballot[SE][kWarps];
+    uint32_t bm[SE][kBitmapWords];
+    uint32_t pre[SE][kBitmapWords];
+    unsigned long long agg[SE];
+    int abort;
+    uint32_t issued;  // tiles whose loads have been started (producer)
+    uint32_t seen;    // tiles whose loads the consumers have seen complete
+};
+
+__device__ __forceinline__ unsigned long long ld_status(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_status(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+// Polls a tile status word until its flag is set.  Bounded: after kMaxPolls reads it gives up,
+// raises CIERA_ERR_TIMEOUT and returns "prefix 0" so that the caller finishes (with unspecified
+// output) instead of hanging.
+__device__ __forceinline__ unsigned long long wait_status(const unsigned long long* p, int32_t* status) {
+    unsigned long long st = ld_status(p);
+    uint32_t polls = 0;
+    while ((st >> 62) == 0) {
+        if (++polls > kMaxPolls) {
+            if (status) atomicCAS(status, 0, (int32_t)CIERA_ERR_TIMEOUT);
+            return kFlagPrefix;
+        }
+        if (polls > 16) __nanosleep(polls > 1024 ? 400 : 40);
+        st = ld_status(p);
+    }
+    return st;
+}
+
+__device__ __forceinline__ uint64_t warp_sum_u64(uint64_t v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Block flags of a tile from the per-warp ballots of "my 16 values differ" (one warp).
+// Fills bm (one bit per block of the tile) and pre (set bits before each word); returns the
+// number of changed blocks of the tile.
+__device__ __forceinline__ uint32_t build_block_bitmap(const uint32_t* ballot, uint32_t* bm, uint32_t* pre,
+                                                       uint32_t log2b, uint32_t lane) {
+    const uint32_t gl2 = log2b - 4;             // log2(groups of 16 values per block)
+    const uint32_t nbt = kTileValues >> log2b;  // blocks of a full tile
+    uint32_t run = 0;
+    for (uint32_t base = 0; base < nbt; base += 32) {
+        const uint32_t i = base + lane;
+        bool f = false;
+        if (i < nbt) {
+            const uint32_t g0 = i << gl2;
+            if (gl2 <= 5) {
+                const uint32_t width = 1u << gl2;
+                const uint32_t m = width == 32 ? 0xffffffffu : ((1u << width) - 1u);
+                f = ((ballot[g0 >> 5] >> (g0 & 31)) & m) != 0;
+            } else {
+                const uint32_t nw = 1u << (gl2 - 5);
+                uint32_t acc = 0;
+                for (uint32_t j = 0; j < nw; ++j) acc |= ballot[(g0 >> 5) + j];
+                f = acc != 0;
+            }
+        }
+        const uint32_t word = __ballot_sync(0xffffffffu, f);
+        if (lane == 0) {
+            bm[base >> 5] = word;
+            pre[base >> 5] = run;
+        }
+        run += __popc(word);
+    }
+    __syncwarp();
+    return run;
+}
+
+// Aggregator warp, one tile: block flags, the tile's bitmap bytes, the tile's payload byte count,
+// published at once as the tile's status word so that later tiles never wait for it longer than
+// for the votes themselves.  Waits for nothing outside the thread block.
+template <int DT>
+__device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t tile, uint32_t log2b,
+                                                   const uint32_t* ballot, uint32_t* bm, uint32_t* pre, uint8_t* msgs,
+                                                   unsigned long long* tile_status, uint32_t lane) {
+    const uint64_t N = td.n_unit;
+    const uint32_t B = 1u << log2b;
+    const uint32_t nbt = kTileValues >> log2b;
+    const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
+    const uint32_t nv = (uint32_t)min((uint64_t)kTileValues, N - v0);
+    uint8_t* msg = msgs + td.msg_off;
+
+    const uint32_t run = build_block_bitmap(ballot, bm, pre, log2b, lane);
+
+    // payload bytes of this tile: B per changed block, less for a changed short last block
+    uint64_t agg = (uint64_t)run << log2b;
+    const uint32_t rem = nv & (B - 1u);
+    if (rem) {
+        const uint32_t kb = nv >> log2b;
+        if ((bm[kb >> 5] >> (kb & 31u)) & 1u) agg -= (B - rem);
+    }
+    // a unit's first tile knows its prefix (0) already
+    const uint32_t mybits = nbt < 8 ? bm[0] : 0u;
+    const unsigned long long flag = td.tile_in_unit == 0 ? kFlagPrefix : kFlagAggregate;
+    if (lane == 0) st_status(tile_status + tile, flag | ((unsigned long long)mybits << kBitsShift) | agg);
+
+    // bitmap bytes of this tile (tiles of >= 8 blocks own whole bytes)
+    if (nbt >= 8) {
+        const uint64_t byte0 = (uint64_t)td.tile_in_unit * (nbt >> 3);
+        const uint32_t nbytes = (((nv + B - 1u) >> log2b) + 7u) >> 3;
+        for (uint32_t b = lane; b < nbytes; b += 32) msg[byte0 + b] = (uint8_t)(bm[b >> 2] >> ((b & 3u) * 8u));
+    }
+    return agg;
+}
+
+// Resolver warp, one tile: exclusive prefix of the payload bytes over the earlier tiles of the
+// same unit by a single-pass look-back over the status words, then the duties that need it.
+// Returns the tile's exclusive payload offset inside its unit.
+template <int DT>
+__device__ __forceinline__ uint64_t resolve_tile(const TileDesc& td, uint32_t tile, uint32_t log2b, uint64_t agg,
+                                                 const uint32_t* bm, uint8_t* msgs, unsigned long long* wire_bytes,
+                                                 uint32_t* changed_blocks, unsigned long long* tile_status,
+                                                 int32_t* status, uint32_t lane) {
+    constexpr int SMB = Traits<DT>::kSmBytes;
+    const uint64_t N = td.n_unit;
+    const uint32_t B = 1u << log2b;
+    const uint32_t nbt = kTileValues >> log2b;
+    uint8_t* msg = msgs + td.msg_off;
+    const uint32_t mybits = nbt < 8 ? bm[0] : 0u;
+
+    uint64_t excl = 0;
+    if (td.tile_in_unit != 0) {
+        int64_t hi = (int64_t)tile - 1;
+        while (true) {
+            const int64_t idx = hi - (int64_t)lane;
+            unsigned long long st = kFlagPrefix;  // "prefix 0" stands before the unit's first tile
+            if (idx >= (int64_t)td.first_tile) st = wait_status(tile_status + idx, status);
+            __syncwarp();
+            const uint32_t pmask = __ballot_sync(0xffffffffu, (st >> 62) == 2ull);
+            const uint32_t first = pmask ? (uint32_t)__ffs(pmask) - 1u : 31u;
+            excl += warp_sum_u64(lane <= first ? (st & kValueMask) : 0ull);
+            if (pmask) break;
+            hi -= 32;
+        }
+        if (lane == 0)
+            st_status(tile_status + tile, kFlagPrefix | ((unsigned long long)mybits << kBitsShift) | (excl + agg));
+    }
+
+    // tiles of fewer than 8 blocks share a bitmap byte: the last tile of each byte collects the
+    // bits its predecessors published in their status words
+    if (nbt < 8) {
+        const uint32_t tpb = 8u / nbt;
+        const uint32_t p = td.tile_in_unit & (tpb - 1u);
+        if (p == tpb - 1u || td.tile_in_unit == td.n_tiles_unit - 1u) {
+            uint32_t part = 0;
+            if (lane < p) {
+                unsigned long long st = wait_status(tile_status + (tile - p + lane), status);
+                part = (uint32_t)((st >> kBitsShift) & 0x3Full) << (lane * nbt);
+            }
+            __syncwarp();
+            part = __reduce_or_sync(0xffffffffu, part);
+            if (lane == 0) msg[td.tile_in_unit / tpb] = (uint8_t)(part | (mybits << (p * nbt)));
+        }
+    }
+
+    // the unit's last tile reports the totals and zeroes the two pads
+    if (td.tile_in_unit == td.n_tiles_unit - 1u) {
+        const uint64_t smoff = sm_offset(N, log2b);
+        const uint64_t payoff = smoff + pad16(N * SMB);
+        const uint64_t total = excl + agg;
+        if (lane == 0) {
+            wire_bytes[td.unit] = payoff + total;
+            changed_blocks[td.unit] = (uint32_t)((total + B - 1u) >> log2b);
+        }
+        for (uint64_t b = bitmap_bytes(N, log2b) + lane; b < smoff; b += 32) msg[b] = 0;
+        for (uint64_t b = smoff + N * SMB + lane; b < payoff; b += 32) msg[b] = 0;
+    }
+    return excl;
+}
+
+// payload <- exponents of changed blocks in block order; cache refreshed for the same blocks.
+// One warp walks the tile's 512 groups of 16 values, 32 groups at a time; the exponents were
+// left in the stage's shared-memory tile by the consumers.
+template <int DT>
+__device__ __forceinline__ void write_changed(const TileDesc& td, uint32_t log2b, const uint32_t* bm,
+                                              const uint32_t* pre, uint64_t base, const uint8_t* s_exp,
+                                              uint8_t* cache, uint8_t* msgs, uint32_t lane) {
+    constexpr int SMB = Traits<DT>::kSmBytes;
+    const uint64_t N = td.n_unit;
+    const uint32_t B = 1u << log2b;
+    const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
+    const uint32_t nv = (uint32_t)min((uint64_t)kTileValues, N - v0);
+    const uint64_t payoff = sm_offset(N, log2b) + pad16(N * SMB);
+    uint8_t* pbase = msgs + td.msg_off + payoff + base;
+    uint8_t* cbase = cache + td.c_off;
+    for (uint32_t w0 = 0; w0 < nv; w0 += 512u) {
+        const uint32_t t0 = w0 + lane * kVPT;
+        const uint32_t kb = t0 >> log2b;
+        const uint32_t word = bm[kb >> 5];
+        const bool chg = t0 < nv && ((word >> (kb & 31u)) & 1u);
+        if (!__any_sync(0xffffffffu, chg)) continue;
+        if (chg) {
+            const int nvalid = (int)min(16u, nv - t0);
+            const uint32_t rank = pre[kb >> 5] + __popc(word & ((1u << (kb & 31u)) - 1u));
+            uint8_t* pdst = pbase + ((uint64_t)rank << log2b) + (t0 & (B - 1u));
+            uint8_t* cdst = cbase + t0;
+            const uint4 ev = ld_shared16(s_exp + t0);
+            if (nvalid == 16) {
+                st_stream16(pdst, ev);
+                st_stream16(cdst, ev);
+            } else {
+                const uint32_t e[4] = {ev.x, ev.y, ev.z, ev.w};
+                store_exp_partial(pdst, e, nvalid);
+                store_exp_partial(cdst, e, nvalid);
+            }
+        }
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kEncodeThreads, 2)
+encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log2b, const uint8_t* __restrict__ weights,
+              uint8_t* cache, uint8_t* msgs, unsigned long long* wire_bytes, uint32_t* changed_blocks,
+              unsigned long long* tile_status, int32_t* status) {
+    constexpr int VB = Traits<DT>::kValueBytes;
+    constexpr int SMB = Traits<DT>::kSmBytes;
+    constexpr int SW = EncodeCfg<DT>::kWStages;
+    constexpr int SE = EncodeCfg<DT>::kEStages;
+    constexpr uint32_t kWBytes = kTileValues * VB;
+    constexpr uint32_t kEBytes = kTileValues;
+    extern __shared__ __align__(128) uint8_t smem[];
+    uint8_t* const ring_w = smem;
+    uint8_t* const ring_e = smem + (size_t)SW * kWBytes;
+    EncodeCtl<SW, SE>* ctl = reinterpret_cast<EncodeCtl<SW, SE>*>(ring_e + (size_t)SE * kEBytes);
+
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const uint32_t G = gridDim.x;
+    // tiles of this block: blockIdx.x + k * G for k < my_tiles
+    const uint32_t my_tiles = blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + G - 1u) / G : 0u;
+    volatile int* abort = &ctl->abort;
+
+    if (tid == 0) {
+        for (int s = 0; s < SW; ++s) {
+            mbar_init(&ctl->full_w[s], 1);
+            mbar_init(&ctl->empty_w[s], kWarps);
+        }
+        for (int s = 0; s < SE; ++s) {
+            mbar_init(&ctl->full_e[s], 1);
+            mbar_init(&ctl->voted[s], kWarps);
+            mbar_init(&ctl->summed[s], 1);
+            mbar_init(&ctl->empty_e[s], 1);
+        }
+        ctl->abort = 0;
+        ctl->issued = 0;
+        ctl->seen = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+
+    if (warp == kProducerWarp) {
+        // ---------------------------------------------------------------- producer
+        if (lane == 0 && my_tiles > 0) {
+            TileDesc nxt = load_tile_desc(tiles + blockIdx.x);  // descriptors are fetched one tile ahead
+            for (uint32_t k = 0; k < my_tiles; ++k) {
+                const TileDesc td = nxt;
+                const uint32_t tile = blockIdx.x + k * G;
+                if (k + 1u < my_tiles) nxt = load_tile_desc(tiles + tile + G);
+                const uint32_t sw = k % SW, se = k % SE;
+                if (k >= (uint32_t)SW && !mbar_wait(&ctl->empty_w[sw], ((k / SW) & 1u) ^ 1u, abort, status)) break;
+                if (k >= (uint32_t)SE && !mbar_wait(&ctl->empty_e[se], ((k / SE) & 1u) ^ 1u, abort, status)) break;
+                ctl->desc[k % kDescRing] = td;
+                ctl->tile_idx[k % kDescRing] = tile;
+                const uint64_t left = td.n_unit - (uint64_t)td.tile_in_unit * kTileValues;
+                if (left >= (uint64_t)kTileValues) {
+                    mbar_arrive_expect_tx(&ctl->full_w[sw], kWBytes);
+                    bulk_load(ring_w + (size_t)sw * kWBytes, weights + td.w_off, kWBytes, &ctl->full_w[sw]);
+                    mbar_arrive_expect_tx(&ctl->full_e[se], kEBytes);
+                    bulk_load(ring_e + (size_t)se * kEBytes, cache + td.c_off, kEBytes, &ctl->full_e[se]);
+                } else {
+                    // short tile: consumers read global memory themselves
+                    mbar_arrive(&ctl->full_w[sw]);
+                    mbar_arrive(&ctl->full_e[se]);
+                }
+                ctl->issued = k + 1;
+            }
+        }
+    } else if (warp == kAggregatorWarp) {
+        // ---------------------------------------------------------------- aggregator
+        for (uint32_t k = 0; k < my_tiles; ++k) {
+            const uint32_t se = k % SE;
+            if (!mbar_wait(&ctl->voted[se], (k / SE) & 1u, abort, status)) break;
+            const TileDesc td = ctl->desc[k % kDescRing];
+            const uint64_t agg = aggregate_tile<DT>(td, ctl->tile_idx[k % kDescRing], log2b, ctl->ballot[se], ctl->bm[se],
+                                                    ctl->pre[se], msgs, tile_status, lane);
+            if (lane == 0) ctl->agg[se] = agg;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->summed[se]);
+        }
+    } else if (warp >= kResolverWarp0) {
+        // ---------------------------------------------------------------- resolvers (tiles k = i, i + R, ...)
+        for (uint32_t k = warp - kResolverWarp0; k < my_tiles; k += kResolvers) {
+            const uint32_t se = k % SE;
+            if (!mbar_wait(&ctl->summed[se], (k / SE) & 1u, abort, status)) break;
+            const TileDesc td = ctl->desc[k % kDescRing];
+            const uint64_t excl = resolve_tile<DT>(td, ctl->tile_idx[k % kDescRing], log2b, ctl->agg[se], ctl->bm[se], msgs,
+                                                   wire_bytes, changed_blocks, tile_status, status, lane);
+            write_changed<DT>(td, log2b, ctl->bm[se], ctl->pre[se], excl, ring_e + (size_t)se * kEBytes, cache, msgs, lane);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->empty_e[se]);
+        }
+    } else {
+        // ---------------------------------------------------------------- consumers
+        const uint32_t t0 = tid * kVPT;
+        for (uint32_t k = 0; k < my_tiles; ++k) {
+            const uint32_t sw = k % SW, se = k % SE;
+            if (!mbar_wait(&ctl->full_w[sw], (k / SW) & 1u, abort, status)) break;
+            if (!mbar_wait(&ctl->full_e[se], (k / SE) & 1u, abort, status)) break;
+            if (tid == 0) ctl->seen = k + 1;
+            const TileDesc td = ctl->desc[k % kDescRing];
+            const uint64_t N = td.n_unit;
+            const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
+            const uint32_t nv = (uint32_t)min((uint64_t)kTileValues, N - v0);
+            const int nvalid = t0 >= nv ? 0 : (int)min(16u, nv - t0);
+            uint8_t* const se_ptr = ring_e + (size_t)se * kEBytes + t0;
+
+            // (exp, mant) <- SplitExpMant, and the cached exponents of the same 16 values
+            Group<DT> g;
+            uint32_t c[4];
+            if (nv == (uint32_t)kTileValues) {
+                g.split_full(ring_w + (size_t)sw * kWBytes + (size_t)t0 * VB, FromShared());
+                const uint4 cv = ld_shared16(se_ptr);
+                c[0] = cv.x; c[1] = cv.y; c[2] = cv.z; c[3] = cv.w;
+            } else if (nvalid == 16) {
+                g.split_full(weights + td.w_off + (uint64_t)t0 * VB);
+                const uint4 cv = ld_stream16(cache + td.c_off + t0);
+                c[0] = cv.x; c[1] = cv.y; c[2] = cv.z; c[3] = cv.w;
+            } else {
+                // values past the end of the unit read as exponent 0 against a cached 0: never "changed"
+                g.split_partial(weights + td.w_off + (uint64_t)t0 * VB, nvalid);
+                load_exp_partial(c, cache + td.c_off + t0, nvalid);
+            }
+            // leave the new exponents where the cached ones were staged: a resolver sends the
+            // changed blocks from there once it knows where they go
+            st_shared16(se_ptr, make_uint4(g.e[0], g.e[1], g.e[2], g.e[3]));
+
+            const bool diff = ((g.e[0] ^ c[0]) | (g.e[1] ^ c[1]) | (g.e[2] ^ c[2]) | (g.e[3] ^ c[3])) != 0;
+            const uint32_t bal = __ballot_sync(0xffffffffu, diff);
+            __syncwarp();  // the warp's shared-memory accesses above are ordered before lane 0's arrives
+            if (lane == 0) {
+                mbar_arrive(&ctl->empty_w[sw]);
+                ctl->ballot[se][warp] = bal;
+                mbar_arrive(&ctl->voted[se]);
+            }
+
+            // sign-plus-mantissa of every value
+            uint8_t* smdst = msgs + td.msg_off + sm_offset(N, log2b) + (v0 + t0) * SMB;
+            if (nvalid == 16)
+                g.store_sm_full(smdst);
+            else if (nvalid > 0)
+                g.store_sm_partial(smdst, nvalid);
+        }
+    }
+
+    // leave together; after an aborted run wait (bounded) for bulk copies that are still in flight
+    __syncthreads();
+    if (tid == 0 && ctl->abort) {
+        for (uint32_t k = ctl->seen; k < ctl->issued; ++k) {
+            for (uint32_t i = 0; i < kMaxBarrierPolls; ++i)
+                if (mbar_try_wait(&ctl->full_w[k % SW], (k / SW) & 1u)) break;
+            for (uint32_t i = 0; i < kMaxBarrierPolls; ++i)
+                if (mbar_try_wait(&ctl->full_e[k % SE], (k / SE) & 1u)) break;
+        }
+    }
+}
+
+template <int DT>
+static size_t encode_smem_bytes() {
+    constexpr int SW = EncodeCfg<DT>::kWStages, SE = EncodeCfg<DT>::kEStages;
+    return (size_t)SW * kTileValues * Traits<DT>::kValueBytes + (size_t)SE * kTileValues + sizeof(EncodeCtl<SW, SE>);
+}
+
+// Largest grid whose blocks are all resident at once, per device (0 = not yet known).
+template <int DT>
+static int encode_grid_limit(int* out) {
+    static int cached[64] = {0};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    if (dev < 0 || dev >= 64) return CIERA_ERR_UNSUPPORTED;
+    if (cached[dev] == 0) {
+        const size_t smem = encode_smem_bytes<DT>();
+        e = cudaFuncSetAttribute(encode_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        int per_sm = 0, sms = 0, coop = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, encode_kernel<DT>, kEncodeThreads, smem);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        if (per_sm < 1 || sms < 1 || !coop) return CIERA_ERR_UNSUPPORTED;
+        cached[dev] = per_sm * sms;
+    }
+    *out = cached[dev];
+    return CIERA_OK;
+}
+
+template <int DT>
+static int launch_encode(const ciera_plan* p, uint32_t grid, const void* weights_dev, void* sender_cache_dev,
+                         void* messages_dev, uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* workspace_dev,
+                         int32_t* status_dev, cudaStream_t s) {
+    const TileDesc* tiles = p->tiles_dev;
+    uint32_t nt = (uint32_t)p->tiles.size();
+    uint32_t log2b = p->log2b;
+    const uint8_t* w = (const uint8_t*)weights_dev;
+    uint8_t* c = (uint8_t*)sender_cache_dev;
+    uint8_t* m = (uint8_t*)messages_dev;
+    unsigned long long* wb = (unsigned long long*)wire_bytes_dev;
+    unsigned long long* ts = (unsigned long long*)workspace_dev;
+    void* args[] = {&tiles, &nt, &log2b, &w, &c, &m, &wb, &changed_blocks_dev, &ts, &status_dev};
+    // cooperative launch: the runtime starts the grid only when all of its blocks fit on the GPU
+    // together, which is what the look-back between blocks relies on
+    cudaError_t e = cudaLaunchCooperativeKernel((const void*)encode_kernel<DT>, dim3(grid), dim3(kEncodeThreads), args,
+                                                encode_smem_bytes<DT>(), s);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    count_launch();
+    return CIERA_OK;
+}
+
+}  // namespace ciera
+
+using namespace ciera;
+
+static bool misaligned16(const void* p) { return ((uintptr_t)p & 15u) != 0; }
+
+extern "C" int ciera_encode(const ciera_plan* p, const void* weights_dev, void* sender_cache_dev, void* messages_dev,
+                            uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* workspace_dev,
+                            int32_t* status_dev, void* stream) {
+    if (!p) return CIERA_ERR_INVALID_ARG;
+    if (!p->tiles.empty() && !p->tiles_dev) return CIERA_ERR_NOT_BOUND;
+    if (p->n_units == 0) return CIERA_OK;
+    if (!wire_bytes_dev || !changed_blocks_dev) return CIERA_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    const uint32_t nt = (uint32_t)p->tiles.size();
+    cudaError_t e;
+    if (p->has_empty_units) {  // units without tiles: their outputs are written here
+        e = cudaMemsetAsync(wire_bytes_dev, 0, sizeof(uint64_t) * p->n_units, s);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        e = cudaMemsetAsync(changed_blocks_dev, 0, sizeof(uint32_t) * p->n_units, s);
+        if (e != cudaSuccess) return record_cuda_error(e);
+    }
+    if (nt == 0) return CIERA_OK;
+    if (!weights_dev || !sender_cache_dev || !messages_dev || !workspace_dev) return CIERA_ERR_INVALID_ARG;
+    if (misaligned16(weights_dev) || misaligned16(sender_cache_dev) || misaligned16(messages_dev) ||
+        misaligned16(workspace_dev) || ((uintptr_t)wire_bytes_dev & 7u) || ((uintptr_t)changed_blocks_dev & 3u))
+        return CIERA_ERR_MISALIGNED;
+    int limit = 0;
+    int rc = p->dtype == CIERA_BF16 ? encode_grid_limit<CIERA_BF16>(&limit) : encode_grid_limit<CIERA_FP32>(&limit);
+    if (rc) return rc;
+    const uint32_t grid = nt < (uint32_t)limit ? nt : (uint32_t)limit;
+    // scratch = one look-back status word per tile; all of it starts at zero
+    e = cudaMemsetAsync(workspace_dev, 0, sizeof(unsigned long long) * nt, s);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    if (p->dtype == CIERA_BF16)
+        return launch_encode<CIERA_BF16>(p, grid, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
+                                         changed_blocks_dev, workspace_dev, status_dev, s);
+    return launch_encode<CIERA_FP32>(p, grid, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
+                                     changed_blocks_dev, workspace_dev, status_dev, s);
+}

@@ -129,8 +129,8 @@ extern "C" const void* ciera_plan_host_image(const ciera_plan* p) { return p ? p
 
 extern "C" size_t ciera_plan_workspace_bytes(const ciera_plan* p) {
     if (!p) return 0;
-    size_t b = p->tiles.size() * sizeof(unsigned long long);
-    return b ? b : 16;
+    // one look-back status word per tile + the ticket counter
+    return p->tiles.size() * sizeof(unsigned long long) + 16;
 }
 
 extern "C" int ciera_plan_bind(ciera_plan* p, void* plan_dev, size_t plan_dev_bytes, void* stream) {

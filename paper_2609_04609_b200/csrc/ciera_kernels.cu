@@ -9,222 +9,6 @@
 namespace ciera {
 
 // ------------------------------------------------------------------------------------------
-// helpers
-
-__device__ __forceinline__ unsigned long long ld_status(const unsigned long long* p) {
-    unsigned long long v;
-    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_status(unsigned long long* p, unsigned long long v) {
-    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-
-// Polls a tile status word until its flag is set.  Bounded: after kMaxPolls reads it gives up,
-// raises CIERA_ERR_TIMEOUT in the caller's status word and returns "prefix 0" so that the block
-// finishes (with unspecified output) instead of hanging.
-__device__ __forceinline__ unsigned long long wait_status(const unsigned long long* p, int32_t* status) {
-    unsigned long long st = ld_status(p);
-    uint32_t polls = 0;
-    while ((st >> 62) == 0) {
-        if (++polls > kMaxPolls) {
-            if (status) atomicCAS(status, 0, (int32_t)CIERA_ERR_TIMEOUT);
-            return kFlagPrefix;
-        }
-        if (polls > 32) __nanosleep(polls > 1024 ? 400 : 40);
-        st = ld_status(p);
-    }
-    return st;
-}
-
-__device__ __forceinline__ uint64_t warp_sum_u64(uint64_t v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
-
-// Block flags of a tile from the per-warp ballots of "my 16 values differ".
-// Warp 0 only.  Fills s_bm (one bit per block of the tile) and s_pre (set bits before each word);
-// returns the number of changed blocks of the tile.
-__device__ __forceinline__ uint32_t build_block_bitmap(const uint32_t* s_ballot, uint32_t* s_bm, uint32_t* s_pre,
-                                                       uint32_t log2b, uint32_t lane) {
-    const uint32_t gl2 = log2b - 4;             // log2(groups of 16 values per block)
-    const uint32_t nbt = kTileValues >> log2b;  // blocks of a full tile
-    uint32_t run = 0;
-    for (uint32_t base = 0; base < nbt; base += 32) {
-        const uint32_t i = base + lane;
-        bool f = false;
-        if (i < nbt) {
-            const uint32_t g0 = i << gl2;
-            if (gl2 <= 5) {
-                const uint32_t width = 1u << gl2;
-                const uint32_t m = width == 32 ? 0xffffffffu : ((1u << width) - 1u);
-                f = ((s_ballot[g0 >> 5] >> (g0 & 31)) & m) != 0;
-            } else {
-                const uint32_t nw = 1u << (gl2 - 5);
-                uint32_t acc = 0;
-                for (uint32_t j = 0; j < nw; ++j) acc |= s_ballot[(g0 >> 5) + j];
-                f = acc != 0;
-            }
-        }
-        const uint32_t word = __ballot_sync(0xffffffffu, f);
-        if (lane == 0) {
-            s_bm[base >> 5] = word;
-            s_pre[base >> 5] = run;
-        }
-        run += __popc(word);
-    }
-    __syncwarp();
-    return run;
-}
-
-// ------------------------------------------------------------------------------------------
-// encode: Algorithm 1, sender part
-
-template <int DT>
-__global__ void __launch_bounds__(kThreads)
-encode_kernel(const TileDesc* __restrict__ tiles, uint32_t log2b, const uint8_t* __restrict__ weights,
-              uint8_t* cache, uint8_t* __restrict__ msgs, unsigned long long* __restrict__ wire_bytes,
-              uint32_t* __restrict__ changed_blocks, unsigned long long* tile_status, int32_t* status) {
-    constexpr int VB = Traits<DT>::kValueBytes;
-    constexpr int SMB = Traits<DT>::kSmBytes;
-    __shared__ uint32_t s_ballot[kWarps];
-    __shared__ uint32_t s_bm[kBitmapWords];
-    __shared__ uint32_t s_pre[kBitmapWords];
-    __shared__ unsigned long long s_base;
-
-    const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
-    const TileDesc td = load_tile_desc(tiles + blockIdx.x);
-    const uint64_t N = td.n_unit;
-    const uint32_t B = 1u << log2b;
-    const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
-    const uint32_t nv = (uint32_t)min((uint64_t)kTileValues, N - v0);
-    const uint32_t t0 = tid * kVPT;
-    const int nvalid = t0 >= nv ? 0 : (int)min(16u, nv - t0);
-    const uint64_t smoff = sm_offset(N, log2b);
-    const uint64_t payoff = smoff + pad16(N * SMB);
-    uint8_t* msg = msgs + td.msg_off;
-
-    // (exp, mant) <- SplitExpMant, and the cached exponents of the same 16 values
-    Group<DT> g;
-    uint32_t c[4];
-    if (nvalid == 16) {
-        g.split_full(weights + td.w_off + (uint64_t)t0 * VB);
-        uint4 cv = ld_stream16(cache + td.c_off + t0);
-        c[0] = cv.x; c[1] = cv.y; c[2] = cv.z; c[3] = cv.w;
-    } else {
-        // values past the end of the unit read as exponent 0 against a cached 0: never "changed"
-        g.split_partial(weights + td.w_off + (uint64_t)t0 * VB, nvalid);
-        load_exp_partial(c, cache + td.c_off + t0, nvalid);
-    }
-    const bool diff = ((g.e[0] ^ c[0]) | (g.e[1] ^ c[1]) | (g.e[2] ^ c[2]) | (g.e[3] ^ c[3])) != 0;
-    const uint32_t bal = __ballot_sync(0xffffffffu, diff);
-    if (lane == 0) s_ballot[warp] = bal;
-
-    // sign-plus-mantissa of every value: independent of the change flags, so issue it now
-    if (nvalid == 16)
-        g.store_sm_full(msg + smoff + (v0 + t0) * SMB);
-    else if (nvalid > 0)
-        g.store_sm_partial(msg + smoff + (v0 + t0) * SMB, nvalid);
-    __syncthreads();
-
-    if (warp == 0) {
-        const uint32_t nbt = kTileValues >> log2b;
-        const uint32_t run = build_block_bitmap(s_ballot, s_bm, s_pre, log2b, lane);
-
-        // payload bytes of this tile: B per changed block, less for a changed short last block
-        uint64_t agg = (uint64_t)run << log2b;
-        const uint32_t rem = nv & (B - 1u);
-        if (rem) {
-            const uint32_t kb = nv >> log2b;
-            if ((s_bm[kb >> 5] >> (kb & 31u)) & 1u) agg -= (B - rem);
-        }
-
-        // bitmap bytes of this tile (tiles of >= 8 blocks own whole bytes)
-        if (nbt >= 8) {
-            const uint64_t byte0 = (uint64_t)td.tile_in_unit * (nbt >> 3);
-            const uint32_t nbytes = (((nv + B - 1u) >> log2b) + 7u) >> 3;
-            for (uint32_t b = lane; b < nbytes; b += 32) msg[byte0 + b] = (uint8_t)(s_bm[b >> 2] >> ((b & 3u) * 8u));
-        }
-        const uint32_t mybits = nbt < 8 ? s_bm[0] : 0u;
-        const unsigned long long bits_field = (unsigned long long)mybits << kBitsShift;
-
-        // exclusive prefix of the payload bytes over the earlier tiles of the same unit:
-        // single-pass look-back over the tile status words
-        unsigned long long* my = tile_status + blockIdx.x;
-        uint64_t excl = 0;
-        if (td.tile_in_unit != 0) {
-            if (lane == 0) st_status(my, kFlagAggregate | bits_field | agg);
-            int64_t hi = (int64_t)blockIdx.x - 1;
-            while (true) {
-                const int64_t idx = hi - (int64_t)lane;
-                unsigned long long st = kFlagPrefix;  // "prefix 0" stands before the unit's first tile
-                if (idx >= (int64_t)td.first_tile) st = wait_status(tile_status + idx, status);
-                __syncwarp();
-                const uint32_t pmask = __ballot_sync(0xffffffffu, (st >> 62) == 2ull);
-                const uint32_t first = pmask ? (uint32_t)__ffs(pmask) - 1u : 31u;
-                excl += warp_sum_u64(lane <= first ? (st & kValueMask) : 0ull);
-                if (pmask) break;
-                hi -= 32;
-            }
-        }
-        if (lane == 0) {
-            st_status(my, kFlagPrefix | bits_field | (excl + agg));
-            s_base = excl;
-        }
-
-        // tiles of fewer than 8 blocks share a bitmap byte: the last tile of each byte collects
-        // the bits its predecessors published in their status words
-        if (nbt < 8) {
-            const uint32_t tpb = 8u / nbt;
-            const uint32_t p = td.tile_in_unit & (tpb - 1u);
-            if (p == tpb - 1u || td.tile_in_unit == td.n_tiles_unit - 1u) {
-                uint32_t part = 0;
-                if (lane < p) {
-                    unsigned long long st = wait_status(tile_status + (blockIdx.x - p + lane), status);
-                    part = (uint32_t)((st >> kBitsShift) & 0x3Full) << (lane * nbt);
-                }
-                __syncwarp();
-                part = __reduce_or_sync(0xffffffffu, part);
-                if (lane == 0) msg[td.tile_in_unit / tpb] = (uint8_t)(part | (mybits << (p * nbt)));
-            }
-        }
-
-        // the unit's last tile reports the totals and zeroes the two pads
-        if (td.tile_in_unit == td.n_tiles_unit - 1u) {
-            const uint64_t total = excl + agg;
-            if (lane == 0) {
-                wire_bytes[td.unit] = payoff + total;
-                changed_blocks[td.unit] = (uint32_t)((total + B - 1u) >> log2b);
-            }
-            for (uint64_t b = bitmap_bytes(N, log2b) + lane; b < smoff; b += 32) msg[b] = 0;
-            for (uint64_t b = smoff + N * SMB + lane; b < payoff; b += 32) msg[b] = 0;
-        }
-    }
-    __syncthreads();
-
-    // payload <- exponents of changed blocks, in block order; cache refreshed for the same blocks
-    if (nvalid > 0) {
-        const uint32_t kb = t0 >> log2b;
-        const uint32_t word = s_bm[kb >> 5];
-        if ((word >> (kb & 31u)) & 1u) {
-            const uint32_t rank = s_pre[kb >> 5] + __popc(word & ((1u << (kb & 31u)) - 1u));
-            const uint64_t off = s_base + ((uint64_t)rank << log2b) + (t0 & (B - 1u));
-            uint8_t* pdst = msg + payoff + off;
-            uint8_t* cdst = cache + td.c_off + t0;
-            if (nvalid == 16) {
-                const uint4 ev = make_uint4(g.e[0], g.e[1], g.e[2], g.e[3]);
-                st_stream16(pdst, ev);
-                st_stream16(cdst, ev);
-            } else {
-                store_exp_partial(pdst, g.e, nvalid);
-                store_exp_partial(cdst, g.e, nvalid);
-            }
-        }
-    }
-}
-
-// ------------------------------------------------------------------------------------------
 // decode: Algorithm 1, receiver part
 
 template <int DT>
@@ -418,41 +202,6 @@ extern "C" int ciera_cache_init(const ciera_plan* plan, void* cache_dev, const v
 extern "C" int ciera_cache_update(const ciera_plan* plan, void* cache_dev, const void* weights_dev, void* stream) {
     if (!weights_dev) return CIERA_ERR_INVALID_ARG;
     return cache_fill(plan, cache_dev, weights_dev, stream);
-}
-
-extern "C" int ciera_encode(const ciera_plan* p, const void* weights_dev, void* sender_cache_dev, void* messages_dev,
-                            uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* workspace_dev,
-                            int32_t* status_dev, void* stream) {
-    int rc = check_plan(p);
-    if (rc) return rc;
-    if (p->n_units == 0) return CIERA_OK;
-    if (!wire_bytes_dev || !changed_blocks_dev) return CIERA_ERR_INVALID_ARG;
-    cudaStream_t s = (cudaStream_t)stream;
-    const uint32_t nt = (uint32_t)p->tiles.size();
-    cudaError_t e;
-    if (p->has_empty_units) {  // units without tiles: their outputs are written here
-        e = cudaMemsetAsync(wire_bytes_dev, 0, sizeof(uint64_t) * p->n_units, s);
-        if (e != cudaSuccess) return record_cuda_error(e);
-        e = cudaMemsetAsync(changed_blocks_dev, 0, sizeof(uint32_t) * p->n_units, s);
-        if (e != cudaSuccess) return record_cuda_error(e);
-    }
-    if (nt == 0) return CIERA_OK;
-    if (!weights_dev || !sender_cache_dev || !messages_dev || !workspace_dev) return CIERA_ERR_INVALID_ARG;
-    if (misaligned16(weights_dev) || misaligned16(sender_cache_dev) || misaligned16(messages_dev) ||
-        misaligned16(workspace_dev) || ((uintptr_t)wire_bytes_dev & 7u) || ((uintptr_t)changed_blocks_dev & 3u))
-        return CIERA_ERR_MISALIGNED;
-    e = cudaMemsetAsync(workspace_dev, 0, sizeof(unsigned long long) * nt, s);
-    if (e != cudaSuccess) return record_cuda_error(e);
-    if (p->dtype == CIERA_BF16)
-        encode_kernel<CIERA_BF16><<<nt, kThreads, 0, s>>>(
-            p->tiles_dev, p->log2b, (const uint8_t*)weights_dev, (uint8_t*)sender_cache_dev, (uint8_t*)messages_dev,
-            (unsigned long long*)wire_bytes_dev, changed_blocks_dev, (unsigned long long*)workspace_dev, status_dev);
-    else
-        encode_kernel<CIERA_FP32><<<nt, kThreads, 0, s>>>(
-            p->tiles_dev, p->log2b, (const uint8_t*)weights_dev, (uint8_t*)sender_cache_dev, (uint8_t*)messages_dev,
-            (unsigned long long*)wire_bytes_dev, changed_blocks_dev, (unsigned long long*)workspace_dev, status_dev);
-    count_launch();
-    return check_launch();
 }
 
 extern "C" int ciera_transport(const ciera_plan* p, const void* src_messages_dev, void* dst_messages_dev,
