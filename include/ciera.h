@@ -120,7 +120,7 @@ CIERA_API uint64_t ciera_plan_total_values(const ciera_plan* plan);
 /* Bytes of device memory the table needs (>= 16), and the host image that has to be there. */
 CIERA_API size_t ciera_plan_device_bytes(const ciera_plan* plan);
 CIERA_API const void* ciera_plan_host_image(const ciera_plan* plan);
-/* Bytes of scratch one ciera_encode call needs (tile status words for the look-back). */
+/* Bytes of scratch one ciera_encode or ciera_decode call needs (per-tile words). */
 CIERA_API size_t ciera_plan_workspace_bytes(const ciera_plan* plan);
 
 /* Copies the table into caller-owned device memory `plan_dev` (>= ciera_plan_device_bytes,
@@ -177,9 +177,13 @@ CIERA_API int ciera_transport(const ciera_plan* plan, const void* src_messages_d
  *   wire_bytes_dev      in   optional (may be NULL): lengths as reported by the sender; a unit
  *                            whose bitmap implies a different length raises CIERA_ERR_CORRUPT in
  *                            status_dev (its output is then unspecified)
+ *   workspace_dev       scratch of ciera_plan_workspace_bytes(), 16-byte aligned.  Only used (by a
+ *                            small prefix kernel that runs first) when some unit has more than 4096
+ *                            blocks; may be NULL otherwise.  Not shared by overlapping calls.
  */
 CIERA_API int ciera_decode(const ciera_plan* plan, const void* messages_dev, void* receiver_cache_dev,
-                 void* weights_out_dev, const uint64_t* wire_bytes_dev, int32_t* status_dev, void* stream);
+                 void* weights_out_dev, const uint64_t* wire_bytes_dev, void* workspace_dev, int32_t* status_dev,
+                 void* stream);
 
 /* ---- whole step with host buffers ---------------------------------------------------------- */
 

@@ -69,7 +69,7 @@ _SIGS = {
     "ciera_cache_update": ([_vp, _vp, _vp, _vp], _i32),
     "ciera_encode": ([_vp] * 9, _i32),
     "ciera_transport": ([_vp] * 5, _i32),
-    "ciera_decode": ([_vp] * 7, _i32),
+    "ciera_decode": ([_vp] * 8, _i32),
     "ciera_roundtrip_host": ([_vp, _vp, _sz, _vp, _vp, _vp, _vp], _i32),
     "ciera_should_compress": ([ctypes.POINTER(GainIn), ctypes.POINTER(_dbl), ctypes.POINTER(_i32)], _i32),
     "ciera_last_cuda_error": ([], _i32),
@@ -158,7 +158,7 @@ class Plan:
             self.bind(device)
 
     def host_image(self) -> np.ndarray:
-        n = self.n_tiles * 48
+        n = self.device_bytes
         if n == 0:
             return np.zeros(0, np.uint8)
         buf = (ctypes.c_uint8 * n).from_address(_lib.ciera_plan_host_image(self._h))
@@ -209,10 +209,11 @@ def transport(plan: Plan, src_messages, dst_messages, wire_bytes, stream=None) -
                                 _stream(stream)))
 
 
-def decode(plan: Plan, messages, receiver_cache, weights_out, wire_bytes=None, status=None, stream=None) -> None:
+def decode(plan: Plan, messages, receiver_cache, weights_out, wire_bytes=None, workspace=None, status=None,
+           stream=None) -> None:
     _check("ciera_decode",
            _lib.ciera_decode(plan.handle, _ptr(messages), _ptr(receiver_cache), _ptr(weights_out), _ptr(wire_bytes),
-                             _ptr(status), _stream(stream)))
+                             _ptr(workspace), _ptr(status), _stream(stream)))
 
 
 class DeviceBuffers(ctypes.Structure):

@@ -33,21 +33,33 @@ struct FromGlobal {
 struct FromShared {
     __device__ __forceinline__ uint4 operator()(const uint8_t* p) const { return ld_shared16(p); }
 };
+// ... and where they go
+struct ToGlobal {
+    __device__ __forceinline__ void operator()(uint8_t* p, uint4 v) const { st_stream16(p, v); }
+};
+struct ToShared {
+    __device__ __forceinline__ void operator()(uint8_t* p, uint4 v) const { st_shared16(p, v); }
+};
+
+// (x & mask) | (y & ~mask): one three-input logic operation
+__device__ __forceinline__ uint32_t bitselect(uint32_t mask, uint32_t x, uint32_t y) { return (x & mask) | (y & ~mask); }
 
 // ---- bf16 --------------------------------------------------------------------------------
-// a = v0 | v1 << 16, b = v2 | v3 << 16  ->  e0 | e1<<8 | e2<<16 | e3<<24
-__device__ __forceinline__ uint32_t bf16_exp4(uint32_t a, uint32_t b) { return __byte_perm(a >> 7, b >> 7, 0x6420); }
-__device__ __forceinline__ uint32_t bf16_sm4(uint32_t a, uint32_t b) {
-    uint32_t ya = (a & 0x007F007Fu) | ((a >> 8) & 0x00800080u);
-    uint32_t yb = (b & 0x007F007Fu) | ((b >> 8) & 0x00800080u);
-    return __byte_perm(ya, yb, 0x6420);
+// Four values a = v0 | v1 << 16, b = v2 | v3 << 16.  Gather their low bytes (e0 m6..m0) and high
+// bytes (s e7..e1) with two byte permutes; then
+//   sm byte  = (high & 0x80) | (low & 0x7F)            exponent byte = (high << 1) | (low >> 7)
+// for all four at once (the shifts leak across byte lanes only into bits that are masked off).
+__device__ __forceinline__ void bf16_split4(uint32_t a, uint32_t b, uint32_t& e, uint32_t& sm) {
+    const uint32_t lo = __byte_perm(a, b, 0x6420), hi = __byte_perm(a, b, 0x7531);
+    sm = bitselect(0x7F7F7F7Fu, lo, hi);
+    e = bitselect(0xFEFEFEFEu, hi << 1, lo >> 7);
 }
 // four exponent bytes + four sm bytes -> two words of two bf16 each
-__device__ __forceinline__ void bf16_merge4(uint32_t e, uint32_t s, uint32_t& lo, uint32_t& hi) {
-    uint32_t e01 = __byte_perm(e, 0u, 0x4140), e23 = __byte_perm(e, 0u, 0x4342);
-    uint32_t s01 = __byte_perm(s, 0u, 0x4140), s23 = __byte_perm(s, 0u, 0x4342);
-    lo = ((s01 & 0x00800080u) << 8) | (e01 << 7) | (s01 & 0x007F007Fu);
-    hi = ((s23 & 0x00800080u) << 8) | (e23 << 7) | (s23 & 0x007F007Fu);
+__device__ __forceinline__ void bf16_merge4(uint32_t e, uint32_t s, uint32_t& a, uint32_t& b) {
+    const uint32_t lo = bitselect(0x7F7F7F7Fu, s, e << 7);  // e0 m6..m0
+    const uint32_t hi = bitselect(0x80808080u, s, e >> 1);  // s e7..e1
+    a = __byte_perm(lo, hi, 0x5140);
+    b = __byte_perm(lo, hi, 0x7362);
 }
 
 // ---- fp32 --------------------------------------------------------------------------------
@@ -56,23 +68,26 @@ __device__ __forceinline__ uint32_t fp32_exp4(uint32_t w0, uint32_t w1, uint32_t
     uint32_t t23 = __byte_perm(w2 << 1, w3 << 1, 0x0073);
     return __byte_perm(t01, t23, 0x5410);
 }
-__device__ __forceinline__ uint32_t fp32_sm(uint32_t w) { return ((w >> 8) & 0x00800000u) | (w & 0x007FFFFFu); }
+// sign << 23 | mantissa in bits 23:0 (bits 31:24 are don't-care for the packing below)
+__device__ __forceinline__ uint32_t fp32_sm(uint32_t w) { return bitselect(0x007FFFFFu, w, w >> 8); }
 // four 24-bit sm values -> three little-endian words
 __device__ __forceinline__ void fp32_pack4(uint32_t s0, uint32_t s1, uint32_t s2, uint32_t s3, uint32_t& o0,
                                            uint32_t& o1, uint32_t& o2) {
-    o0 = s0 | (s1 << 24);
-    o1 = (s1 >> 8) | (s2 << 16);
-    o2 = (s2 >> 16) | (s3 << 8);
+    o0 = __byte_perm(s0, s1, 0x4210);
+    o1 = __byte_perm(s1, s2, 0x5421);
+    o2 = __byte_perm(s2, s3, 0x6542);
 }
+// three words -> four sm values in bits 23:0 (bits 31:24 don't-care)
 __device__ __forceinline__ void fp32_unpack4(uint32_t o0, uint32_t o1, uint32_t o2, uint32_t& s0, uint32_t& s1,
                                              uint32_t& s2, uint32_t& s3) {
-    s0 = o0 & 0x00FFFFFFu;
-    s1 = (o0 >> 24) | ((o1 & 0x0000FFFFu) << 8);
-    s2 = (o1 >> 16) | ((o2 & 0x000000FFu) << 16);
+    s0 = o0;
+    s1 = __byte_perm(o0, o1, 0x0543);
+    s2 = __byte_perm(o1, o2, 0x0432);
     s3 = o2 >> 8;
 }
+// exponent in bits 7:0 of e (higher bits don't-care), sm in bits 23:0 of s
 __device__ __forceinline__ uint32_t fp32_merge(uint32_t e, uint32_t s) {
-    return ((s & 0x00800000u) << 8) | (e << 23) | (s & 0x007FFFFFu);
+    return bitselect(0x007FFFFFu, s, bitselect(0x7F800000u, e << 23, s << 8));
 }
 
 // ---- a group in registers ------------------------------------------------------------------
@@ -88,8 +103,10 @@ struct Group<CIERA_BF16> {
     template <class Ld = FromGlobal>
     __device__ __forceinline__ void split_full(const uint8_t* w, Ld ld = Ld()) {
         uint4 a = ld(w), b = ld(w + 16);
-        e[0] = bf16_exp4(a.x, a.y); e[1] = bf16_exp4(a.z, a.w); e[2] = bf16_exp4(b.x, b.y); e[3] = bf16_exp4(b.z, b.w);
-        s[0] = bf16_sm4(a.x, a.y);  s[1] = bf16_sm4(a.z, a.w);  s[2] = bf16_sm4(b.x, b.y);  s[3] = bf16_sm4(b.z, b.w);
+        bf16_split4(a.x, a.y, e[0], s[0]);
+        bf16_split4(a.z, a.w, e[1], s[1]);
+        bf16_split4(b.x, b.y, e[2], s[2]);
+        bf16_split4(b.z, b.w, e[3], s[3]);
     }
     // the first nvalid (< 16) values; the others read as +0.0 (exponent 0)
     __device__ __forceinline__ void split_partial(const uint8_t* w, int nvalid) {
@@ -101,10 +118,7 @@ struct Group<CIERA_BF16> {
         for (int i = 0; i < 16; ++i)
             if (i < nvalid) x[i >> 1] |= (uint32_t)p[i] << (16 * (i & 1));
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            e[i] = bf16_exp4(x[2 * i], x[2 * i + 1]);
-            s[i] = bf16_sm4(x[2 * i], x[2 * i + 1]);
-        }
+        for (int i = 0; i < 4; ++i) bf16_split4(x[2 * i], x[2 * i + 1], e[i], s[i]);
     }
     __device__ __forceinline__ void store_sm_full(uint8_t* dst) const { st_stream16(dst, make_uint4(s[0], s[1], s[2], s[3])); }
     __device__ __forceinline__ void store_sm_partial(uint8_t* dst, int nvalid) const {
@@ -124,12 +138,13 @@ struct Group<CIERA_BF16> {
         for (int i = 0; i < 16; ++i)
             if (i < nvalid) s[i >> 2] |= (uint32_t)src[i] << (8 * (i & 3));
     }
-    __device__ __forceinline__ void merge_store_full(uint8_t* w) const {
+    template <class St = ToGlobal>
+    __device__ __forceinline__ void merge_store_full(uint8_t* w, St st = St()) const {
         uint4 a, b;
         bf16_merge4(e[0], s[0], a.x, a.y); bf16_merge4(e[1], s[1], a.z, a.w);
         bf16_merge4(e[2], s[2], b.x, b.y); bf16_merge4(e[3], s[3], b.z, b.w);
-        st_stream16(w, a);
-        st_stream16(w + 16, b);
+        st(w, a);
+        st(w + 16, b);
     }
     __device__ __forceinline__ void merge_store_partial(uint8_t* w, int nvalid) const {
         uint32_t x[8];
@@ -201,17 +216,18 @@ struct Group<CIERA_FP32> {
         for (int i = 0; i < 4; ++i) {
             uint32_t s0, s1, s2, s3;
             fp32_unpack4(s[3 * i], s[3 * i + 1], s[3 * i + 2], s0, s1, s2, s3);
-            x[4 * i] = fp32_merge(e[i] & 0xFFu, s0);
-            x[4 * i + 1] = fp32_merge((e[i] >> 8) & 0xFFu, s1);
-            x[4 * i + 2] = fp32_merge((e[i] >> 16) & 0xFFu, s2);
+            x[4 * i] = fp32_merge(e[i], s0);
+            x[4 * i + 1] = fp32_merge(e[i] >> 8, s1);
+            x[4 * i + 2] = fp32_merge(e[i] >> 16, s2);
             x[4 * i + 3] = fp32_merge(e[i] >> 24, s3);
         }
     }
-    __device__ __forceinline__ void merge_store_full(uint8_t* w) const {
+    template <class St = ToGlobal>
+    __device__ __forceinline__ void merge_store_full(uint8_t* w, St st = St()) const {
         uint32_t x[16];
         merge_words(x);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) st_stream16(w + 16 * i, make_uint4(x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]));
+        for (int i = 0; i < 4; ++i) st(w + 16 * i, make_uint4(x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]));
     }
     __device__ __forceinline__ void merge_store_partial(uint8_t* w, int nvalid) const {
         uint32_t x[16];

@@ -16,13 +16,17 @@
 //   aggregator warp turns the 512 vote bits of a tile into block flags (the unit's bitmap), counts
 //                   the tile's payload bytes and publishes them as the tile's status word;
 //   resolver warps  resolve the tile's exclusive offset in the unit's payload with a single-pass
-//                   look-back over the status words, then send the exponents of changed blocks
-//                   from shared memory to the payload and to the cache, and hand the stage back.
+//                   look-back over the status words.
+// A few tiles later, when that offset is known, the consumers send the exponents of changed
+// blocks from shared memory to the payload and to the cache and hand the stage back.
 //
-// Only the resolvers ever wait for another thread block; consumers and aggregator never do, so
-// a tile's status is published as soon as its votes are in.
+// Only the resolvers ever wait for another thread block; the aggregator never does, and the
+// consumers only for a resolver that is several tiles late, so a tile's status is published as
+// soon as its votes are in.
 #include "ciera_bits.cuh"
 #include "ciera_pipe.cuh"
+
+CIERA_PROF_READER(enc)
 
 namespace ciera {
 
@@ -32,6 +36,7 @@ constexpr int kProducerWarp = kWarps;               // 16
 constexpr int kAggregatorWarp = kWarps + 1;         // 17
 constexpr int kResolverWarp0 = kWarps + 2;          // 18 ..
 constexpr int kDescRing = 16;                       // > exponent stages + 2
+constexpr int kDefer = 3;                           // consumers send a tile's changed exponents this many tiles later
 
 template <int DT>
 struct EncodeCfg;
@@ -46,6 +51,17 @@ struct EncodeCfg<CIERA_FP32> {
     static constexpr int kEStages = 5;  // 5 x  8 KB
 };
 
+// What the consumers need of a tile, worked out once by the producer thread instead of by each
+// of the 512 consumer threads.
+struct __align__(16) EncodeTileInfo {
+    uint8_t* sm_dst;       // where the tile's sign-plus-mantissa goes
+    uint8_t* pay_dst;      // start of the unit's payload section
+    uint8_t* c_ptr;        // the tile's cached exponents
+    const uint8_t* w_src;  // the tile's weights
+    uint32_t nv;           // values in the tile
+    uint32_t pad[3];
+};
+
 template <int SW, int SE>
 struct EncodeCtl {
     uint64_t full_w[SW];   // weights tile landed
@@ -53,13 +69,16 @@ struct EncodeCtl {
     uint64_t full_e[SE];   // cached-exponent tile landed
     uint64_t voted[SE];    // all 16 consumer warps have left their exponents there and voted
     uint64_t summed[SE];   // aggregator has published the tile's status and block flags
-    uint64_t empty_e[SE];  // resolver is done with the tile
+    uint64_t resolved[SE]; // a resolver knows the tile's offset in the unit's payload
+    uint64_t empty_e[SE];  // all 16 consumer warps have sent the tile's changed exponents
     TileDesc desc[kDescRing];
-    uint32_t tile_idx[kDescRing];  // table index of the tile in desc[]; kNoTile = no more work
+    EncodeTileInfo info[kDescRing];
+    uint32_t tile_idx[kDescRing];  // table index of the tile in desc[]
     uint32_t ballot[SE][kWarps];
     uint32_t bm[SE][kBitmapWords];
     uint32_t pre[SE][kBitmapWords];
     unsigned long long agg[SE];
+    unsigned long long base[SE];
     int abort;
     uint32_t issued;  // tiles whose loads have been started (producer)
     uint32_t seen;    // tiles whose loads the consumers have seen complete
@@ -235,41 +254,26 @@ __device__ __forceinline__ uint64_t resolve_tile(const TileDesc& td, uint32_t ti
 }
 
 // payload <- exponents of changed blocks in block order; cache refreshed for the same blocks.
-// One warp walks the tile's 512 groups of 16 values, 32 groups at a time; the exponents were
-// left in the stage's shared-memory tile by the consumers.
-template <int DT>
-__device__ __forceinline__ void write_changed(const TileDesc& td, uint32_t log2b, const uint32_t* bm,
-                                              const uint32_t* pre, uint64_t base, const uint8_t* s_exp,
-                                              uint8_t* cache, uint8_t* msgs, uint32_t lane) {
-    constexpr int SMB = Traits<DT>::kSmBytes;
-    const uint64_t N = td.n_unit;
-    const uint32_t B = 1u << log2b;
-    const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
-    const uint32_t nv = (uint32_t)min((uint64_t)kTileValues, N - v0);
-    const uint64_t payoff = sm_offset(N, log2b) + pad16(N * SMB);
-    uint8_t* pbase = msgs + td.msg_off + payoff + base;
-    uint8_t* cbase = cache + td.c_off;
-    for (uint32_t w0 = 0; w0 < nv; w0 += 512u) {
-        const uint32_t t0 = w0 + lane * kVPT;
-        const uint32_t kb = t0 >> log2b;
-        const uint32_t word = bm[kb >> 5];
-        const bool chg = t0 < nv && ((word >> (kb & 31u)) & 1u);
-        if (!__any_sync(0xffffffffu, chg)) continue;
-        if (chg) {
-            const int nvalid = (int)min(16u, nv - t0);
-            const uint32_t rank = pre[kb >> 5] + __popc(word & ((1u << (kb & 31u)) - 1u));
-            uint8_t* pdst = pbase + ((uint64_t)rank << log2b) + (t0 & (B - 1u));
-            uint8_t* cdst = cbase + t0;
-            const uint4 ev = ld_shared16(s_exp + t0);
-            if (nvalid == 16) {
-                st_stream16(pdst, ev);
-                st_stream16(cdst, ev);
-            } else {
-                const uint32_t e[4] = {ev.x, ev.y, ev.z, ev.w};
-                store_exp_partial(pdst, e, nvalid);
-                store_exp_partial(cdst, e, nvalid);
-            }
-        }
+// Every consumer thread sends its own 16 exponents (left in the stage's shared-memory tile) if
+// its block changed; `base` is the tile's exclusive offset in the unit's payload.
+__device__ __forceinline__ void write_changed(const EncodeTileInfo& ti, uint32_t log2b, const uint32_t* bm,
+                                              const uint32_t* pre, uint64_t base, const uint8_t* s_exp, uint32_t t0) {
+    if (t0 >= ti.nv) return;
+    const uint32_t kb = t0 >> log2b;
+    const uint32_t word = bm[kb >> 5];
+    if (!((word >> (kb & 31u)) & 1u)) return;
+    const int nvalid = (int)min(16u, ti.nv - t0);
+    const uint32_t rank = pre[kb >> 5] + __popc(word & ((1u << (kb & 31u)) - 1u));
+    uint8_t* pdst = ti.pay_dst + base + ((uint64_t)rank << log2b) + (t0 & ((1u << log2b) - 1u));
+    uint8_t* cdst = ti.c_ptr + t0;
+    const uint4 ev = ld_shared16(s_exp + t0);
+    if (nvalid == 16) {
+        st_stream16(pdst, ev);
+        st_stream16(cdst, ev);
+    } else {
+        const uint32_t e[4] = {ev.x, ev.y, ev.z, ev.w};
+        store_exp_partial(pdst, e, nvalid);
+        store_exp_partial(cdst, e, nvalid);
     }
 }
 
@@ -304,7 +308,8 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
             mbar_init(&ctl->full_e[s], 1);
             mbar_init(&ctl->voted[s], kWarps);
             mbar_init(&ctl->summed[s], 1);
-            mbar_init(&ctl->empty_e[s], 1);
+            mbar_init(&ctl->resolved[s], 1);
+            mbar_init(&ctl->empty_e[s], kWarps);
         }
         ctl->abort = 0;
         ctl->issued = 0;
@@ -317,6 +322,7 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
         // ---------------------------------------------------------------- producer
         if (lane == 0 && my_tiles > 0) {
             TileDesc nxt = load_tile_desc(tiles + blockIdx.x);  // descriptors are fetched one tile ahead
+            PROF_T0;
             for (uint32_t k = 0; k < my_tiles; ++k) {
                 const TileDesc td = nxt;
                 const uint32_t tile = blockIdx.x + k * G;
@@ -324,9 +330,21 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                 const uint32_t sw = k % SW, se = k % SE;
                 if (k >= (uint32_t)SW && !mbar_wait(&ctl->empty_w[sw], ((k / SW) & 1u) ^ 1u, abort, status)) break;
                 if (k >= (uint32_t)SE && !mbar_wait(&ctl->empty_e[se], ((k / SE) & 1u) ^ 1u, abort, status)) break;
+                PROF_ADD(0);
                 ctl->desc[k % kDescRing] = td;
                 ctl->tile_idx[k % kDescRing] = tile;
-                const uint64_t left = td.n_unit - (uint64_t)td.tile_in_unit * kTileValues;
+                const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
+                const uint64_t left = td.n_unit - v0;
+                {
+                    const uint64_t smoff = sm_offset(td.n_unit, log2b);
+                    EncodeTileInfo ti;
+                    ti.sm_dst = msgs + td.msg_off + smoff + v0 * SMB;
+                    ti.pay_dst = msgs + td.msg_off + smoff + pad16(td.n_unit * SMB);
+                    ti.c_ptr = cache + td.c_off;
+                    ti.w_src = weights + td.w_off;
+                    ti.nv = (uint32_t)min((uint64_t)kTileValues, left);
+                    ctl->info[k % kDescRing] = ti;
+                }
                 if (left >= (uint64_t)kTileValues) {
                     mbar_arrive_expect_tx(&ctl->full_w[sw], kWBytes);
                     bulk_load(ring_w + (size_t)sw * kWBytes, weights + td.w_off, kWBytes, &ctl->full_w[sw]);
@@ -338,44 +356,55 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                     mbar_arrive(&ctl->full_e[se]);
                 }
                 ctl->issued = k + 1;
+                PROF_ADD(1);
             }
+            PROF_FLUSH;
         }
     } else if (warp == kAggregatorWarp) {
         // ---------------------------------------------------------------- aggregator
+        PROF_T0;
         for (uint32_t k = 0; k < my_tiles; ++k) {
             const uint32_t se = k % SE;
             if (!mbar_wait(&ctl->voted[se], (k / SE) & 1u, abort, status)) break;
+            PROF_ADD(2);
             const TileDesc td = ctl->desc[k % kDescRing];
             const uint64_t agg = aggregate_tile<DT>(td, ctl->tile_idx[k % kDescRing], log2b, ctl->ballot[se], ctl->bm[se],
                                                     ctl->pre[se], msgs, tile_status, lane);
             if (lane == 0) ctl->agg[se] = agg;
             __syncwarp();
             if (lane == 0) mbar_arrive(&ctl->summed[se]);
+            PROF_ADD(3);
         }
+        PROF_FLUSH;
     } else if (warp >= kResolverWarp0) {
         // ---------------------------------------------------------------- resolvers (tiles k = i, i + R, ...)
+        PROF_T0;
         for (uint32_t k = warp - kResolverWarp0; k < my_tiles; k += kResolvers) {
             const uint32_t se = k % SE;
             if (!mbar_wait(&ctl->summed[se], (k / SE) & 1u, abort, status)) break;
+            PROF_ADD(4);
             const TileDesc td = ctl->desc[k % kDescRing];
             const uint64_t excl = resolve_tile<DT>(td, ctl->tile_idx[k % kDescRing], log2b, ctl->agg[se], ctl->bm[se], msgs,
                                                    wire_bytes, changed_blocks, tile_status, status, lane);
-            write_changed<DT>(td, log2b, ctl->bm[se], ctl->pre[se], excl, ring_e + (size_t)se * kEBytes, cache, msgs, lane);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&ctl->empty_e[se]);
+            PROF_ADD(5);
+            if (lane == 0) {
+                ctl->base[se] = excl;
+                mbar_arrive(&ctl->resolved[se]);
+            }
         }
+        if (warp == kResolverWarp0) PROF_FLUSH;
     } else {
         // ---------------------------------------------------------------- consumers
         const uint32_t t0 = tid * kVPT;
+        PROF_T0;
         for (uint32_t k = 0; k < my_tiles; ++k) {
             const uint32_t sw = k % SW, se = k % SE;
             if (!mbar_wait(&ctl->full_w[sw], (k / SW) & 1u, abort, status)) break;
             if (!mbar_wait(&ctl->full_e[se], (k / SE) & 1u, abort, status)) break;
+            PROF_ADD(7);
             if (tid == 0) ctl->seen = k + 1;
-            const TileDesc td = ctl->desc[k % kDescRing];
-            const uint64_t N = td.n_unit;
-            const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
-            const uint32_t nv = (uint32_t)min((uint64_t)kTileValues, N - v0);
+            const EncodeTileInfo ti = ctl->info[k % kDescRing];
+            const uint32_t nv = ti.nv;
             const int nvalid = t0 >= nv ? 0 : (int)min(16u, nv - t0);
             uint8_t* const se_ptr = ring_e + (size_t)se * kEBytes + t0;
 
@@ -387,13 +416,13 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                 const uint4 cv = ld_shared16(se_ptr);
                 c[0] = cv.x; c[1] = cv.y; c[2] = cv.z; c[3] = cv.w;
             } else if (nvalid == 16) {
-                g.split_full(weights + td.w_off + (uint64_t)t0 * VB);
-                const uint4 cv = ld_stream16(cache + td.c_off + t0);
+                g.split_full(ti.w_src + (size_t)t0 * VB);
+                const uint4 cv = ld_stream16(ti.c_ptr + t0);
                 c[0] = cv.x; c[1] = cv.y; c[2] = cv.z; c[3] = cv.w;
             } else {
                 // values past the end of the unit read as exponent 0 against a cached 0: never "changed"
-                g.split_partial(weights + td.w_off + (uint64_t)t0 * VB, nvalid);
-                load_exp_partial(c, cache + td.c_off + t0, nvalid);
+                g.split_partial(ti.w_src + (size_t)t0 * VB, nvalid);
+                load_exp_partial(c, ti.c_ptr + t0, nvalid);
             }
             // leave the new exponents where the cached ones were staged: a resolver sends the
             // changed blocks from there once it knows where they go
@@ -409,12 +438,36 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
             }
 
             // sign-plus-mantissa of every value
-            uint8_t* smdst = msgs + td.msg_off + sm_offset(N, log2b) + (v0 + t0) * SMB;
+            uint8_t* smdst = ti.sm_dst + (size_t)t0 * SMB;
             if (nvalid == 16)
                 g.store_sm_full(smdst);
             else if (nvalid > 0)
                 g.store_sm_partial(smdst, nvalid);
+            PROF_ADD(8);
+
+            // the changed exponents of the tile handled kDefer tiles ago: its offset is known by now
+            if (k >= (uint32_t)kDefer) {
+                const uint32_t j = k - kDefer, je = j % SE;
+                if (!mbar_wait(&ctl->resolved[je], (j / SE) & 1u, abort, status)) break;
+                PROF_ADD(6);
+                write_changed(ctl->info[j % kDescRing], log2b, ctl->bm[je], ctl->pre[je], ctl->base[je],
+                              ring_e + (size_t)je * kEBytes, t0);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->empty_e[je]);
+                PROF_ADD(9);
+            }
         }
+        if (!*abort) {
+            for (uint32_t j = my_tiles > (uint32_t)kDefer ? my_tiles - kDefer : 0u; j < my_tiles; ++j) {
+                const uint32_t je = j % SE;
+                if (!mbar_wait(&ctl->resolved[je], (j / SE) & 1u, abort, status)) break;
+                write_changed(ctl->info[j % kDescRing], log2b, ctl->bm[je], ctl->pre[je], ctl->base[je],
+                              ring_e + (size_t)je * kEBytes, t0);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->empty_e[je]);
+            }
+        }
+        if (warp == 0) PROF_FLUSH;
     }
 
     // leave together; after an aborted run wait (bounded) for bulk copies that are still in flight

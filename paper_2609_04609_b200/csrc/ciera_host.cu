@@ -1,4 +1,6 @@
 // Host side of libciera: size rules, the plan (tile table), the gain rule, diagnostics.
+#include <string.h>
+
 #include <new>
 
 #include "ciera_internal.cuh"
@@ -108,7 +110,13 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
             t.n_tiles_unit = nt;
             p->tiles.push_back(t);
         }
+        if (nt && (un.n_values + block - 1) / block > kDecodeDirectBlocks) p->long_units.push_back(first);
     }
+    // device image: the tile table, then (16-byte aligned) the list of long units
+    const size_t tb = p->tiles.size() * sizeof(TileDesc);
+    p->image.assign(tb + p->long_units.size() * sizeof(uint32_t) + 16, 0);
+    if (tb) memcpy(p->image.data(), p->tiles.data(), tb);
+    if (!p->long_units.empty()) memcpy(p->image.data() + tb, p->long_units.data(), p->long_units.size() * 4);
     *plan_out = p;
     return CIERA_OK;
 }
@@ -120,12 +128,8 @@ extern "C" uint32_t ciera_plan_n_tiles(const ciera_plan* p) { return p ? (uint32
 extern "C" uint32_t ciera_plan_tile_values(const ciera_plan*) { return kTileValues; }
 extern "C" uint64_t ciera_plan_total_values(const ciera_plan* p) { return p ? p->total_values : 0; }
 
-extern "C" size_t ciera_plan_device_bytes(const ciera_plan* p) {
-    if (!p) return 0;
-    size_t b = p->tiles.size() * sizeof(TileDesc);
-    return b ? b : 16;
-}
-extern "C" const void* ciera_plan_host_image(const ciera_plan* p) { return p ? p->tiles.data() : nullptr; }
+extern "C" size_t ciera_plan_device_bytes(const ciera_plan* p) { return p ? p->image.size() : 0; }
+extern "C" const void* ciera_plan_host_image(const ciera_plan* p) { return p ? p->image.data() : nullptr; }
 
 extern "C" size_t ciera_plan_workspace_bytes(const ciera_plan* p) {
     if (!p) return 0;
@@ -136,16 +140,15 @@ extern "C" size_t ciera_plan_workspace_bytes(const ciera_plan* p) {
 extern "C" int ciera_plan_bind(ciera_plan* p, void* plan_dev, size_t plan_dev_bytes, void* stream) {
     if (!p || !plan_dev) return CIERA_ERR_INVALID_ARG;
     if ((uintptr_t)plan_dev & 15u) return CIERA_ERR_MISALIGNED;
-    size_t need = p->tiles.size() * sizeof(TileDesc);
+    const size_t need = p->image.size();
     if (plan_dev_bytes < need) return CIERA_ERR_CAPACITY;
     cudaStream_t s = (cudaStream_t)stream;
-    if (need) {
-        cudaError_t e = cudaMemcpyAsync(plan_dev, p->tiles.data(), need, cudaMemcpyHostToDevice, s);
-        if (e != cudaSuccess) return record_cuda_error(e);
-        e = cudaStreamSynchronize(s);
-        if (e != cudaSuccess) return record_cuda_error(e);
-    }
+    cudaError_t e = cudaMemcpyAsync(plan_dev, p->image.data(), need, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return record_cuda_error(e);
     p->tiles_dev = (const TileDesc*)plan_dev;
+    p->long_units_dev = (const uint32_t*)((const uint8_t*)plan_dev + p->tiles.size() * sizeof(TileDesc));
     return CIERA_OK;
 }
 

@@ -70,6 +70,10 @@ __host__ __device__ inline uint64_t payload_offset(uint64_t n, uint32_t sm_bytes
     return sm_offset(n, log2b) + pad16(n * sm_bytes_per_value);
 }
 
+// Units with more blocks than this get their per-tile "changed blocks before" counts from a
+// prefix kernel at decode time; shorter ones read them straight from the bitmap.
+constexpr uint32_t kDecodeDirectBlocks = 4096;
+
 // Bytes of a message slot that one tile moves in the transport kernel: slot capacity <= tiles * this.
 __host__ __device__ inline uint64_t transport_chunk_bytes(uint32_t sm_bytes_per_value) {
     return (uint64_t)kTileValues * (sm_bytes_per_value + 1) + 96;
@@ -87,7 +91,10 @@ struct ciera_plan {
     bool has_empty_units = false;
     std::vector<ciera_unit> units;
     std::vector<ciera::TileDesc> tiles;
+    std::vector<uint32_t> long_units;  // first tile of every unit whose decode needs the prefix kernel
+    std::vector<uint8_t> image;        // device image: tiles, then long_units
     const ciera::TileDesc* tiles_dev = nullptr;
+    const uint32_t* long_units_dev = nullptr;
 };
 
 namespace ciera {

@@ -8,6 +8,22 @@
 
 #include "ciera_internal.cuh"
 
+#ifdef CIERA_PROF
+static __device__ unsigned long long g_prof[16];
+#define CIERA_PROF_READER(name) \
+    extern "C" __attribute__((visibility("default"))) int ciera_debug_prof_##name(unsigned long long* out, int reset) { \
+        if (reset) { unsigned long long z[16] = {0}; return (int)cudaMemcpyToSymbol(g_prof, z, sizeof(z)); } \
+        return (int)cudaMemcpyFromSymbol(out, g_prof, sizeof(unsigned long long) * 16); }
+#define PROF_T0 long long _t = clock64(); long long _p[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
+#define PROF_ADD(i) { long long _n = clock64(); _p[i] += _n - _t; _t = _n; }
+#define PROF_FLUSH { if (lane == 0) { _Pragma("unroll") for (int _i = 0; _i < 10; ++_i) if (_p[_i]) atomicAdd(&g_prof[_i], (unsigned long long)_p[_i]); } }
+#else
+#define PROF_T0
+#define PROF_ADD(i)
+#define PROF_FLUSH
+#define CIERA_PROF_READER(name)
+#endif
+
 namespace ciera {
 
 constexpr uint32_t kMaxBarrierPolls = 1u << 22;  // each poll may itself suspend for a short time slice
@@ -73,6 +89,19 @@ template <int N>
 __device__ __forceinline__ void bulk_wait_all() {
     asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
 }
+// per-thread asynchronous global -> shared copies of 4 or 16 bytes (no registers held while in flight)
+__device__ __forceinline__ void cp_async4(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
 // make generic-proxy writes to shared memory visible to the async proxy (before a bulk store)
 __device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 

@@ -65,7 +65,7 @@ class LayerCodec:
     def decode(self, weights_out: Optional[torch.Tensor] = None, stream=None, check_length: bool = True) -> None:
         out = self.weights_out if weights_out is None else weights_out
         ciera.decode(self.plan, self.msg_recv, self.receiver_cache, out,
-                     self.wire_bytes if check_length else None, self.status, stream)
+                     self.wire_bytes if check_length else None, self.workspace, self.status, stream)
 
     def step(self, weights: torch.Tensor, weights_out: Optional[torch.Tensor] = None, stream=None) -> None:
         self.encode(weights, stream)

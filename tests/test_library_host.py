@@ -83,8 +83,8 @@ def test_plan_tile_table(ciera):
     p = ciera.Plan(units, 1, 64)
     want_tiles = sum(-(-n // T) for n in sizes)
     assert (p.n_units, p.n_tiles, p.tile_values, p.total_values) == (len(sizes), want_tiles, T, sum(sizes))
-    assert p.workspace_bytes >= 8 * want_tiles and p.device_bytes == 48 * want_tiles
-    img = p.host_image().view(np.dtype([("w", "<u8"), ("c", "<u8"), ("m", "<u8"), ("n", "<u8"), ("unit", "<u4"),
+    assert p.workspace_bytes >= 8 * want_tiles and p.device_bytes >= 48 * want_tiles
+    img = p.host_image()[: 48 * want_tiles].view(np.dtype([("w", "<u8"), ("c", "<u8"), ("m", "<u8"), ("n", "<u8"), ("unit", "<u4"),
                                         ("j", "<u4"), ("first", "<u4"), ("nt", "<u4")]))
     k = 0
     for ui, u in enumerate(units):
