@@ -1,19 +1,31 @@
-// Per-thread register work: one "group" = 16 consecutive values of one thread.
+// Per-thread register work on "pieces": runs of consecutive values owned by one thread.
 //
 // Split and merge follow the paper's Section 3.1 (a value is sign, exponent and mantissa bits;
 // the exponent travels apart from sign-plus-mantissa) on the IEEE binary32 / bfloat16 layouts:
 //   bf16: bit 15 sign, bits 14:7 exponent, bits 6:0 mantissa  -> sm byte  = sign<<7  | mantissa
 //   fp32: bit 31 sign, bits 30:23 exponent, bits 22:0 mantissa -> sm 24bit = sign<<23 | mantissa
 // Everything is done on packed 32-bit words with shifts, three-input logic and byte permutes,
-// four values at a time, so that a group's 16 exponent bytes end up as one uint4.
+// four values at a time.
+//
+// Thread -> value layout inside a tile of 8192 values (512 consumer threads):
+//   bf16: two pieces of 8 values per thread, piece p of thread t = values [4096 p + 8 t, +8).
+//         Every access of a warp is then one contiguous run: 16 B / lane on the weights,
+//         8 B / lane on the byte-wide streams (exponents, sign-plus-mantissa).
+//   fp32: one piece of 16 values per thread, values [16 t, +16): 64 B of weights, 16 B of
+//         exponents, 48 B of sign-plus-mantissa per lane.
+// A piece never straddles a block (block sizes are multiples of 16), so a piece has one
+// "my exponents changed" bit; the tile has 1024 (bf16) or 512 (fp32) such bits.
 #pragma once
 
 #include "ciera_internal.cuh"
 
 namespace ciera {
 
+// ---- 8- and 16-byte accesses ---------------------------------------------------------------
 __device__ __forceinline__ uint4 ld_stream16(const void* p) { return __ldcs(reinterpret_cast<const uint4*>(p)); }
+__device__ __forceinline__ uint2 ld_stream8(const void* p) { return __ldcs(reinterpret_cast<const uint2*>(p)); }
 __device__ __forceinline__ void st_stream16(void* p, uint4 v) { __stcs(reinterpret_cast<uint4*>(p), v); }
+__device__ __forceinline__ void st_stream8(void* p, uint2 v) { __stcs(reinterpret_cast<uint2*>(p), v); }
 __device__ __forceinline__ uint4 ld_shared16(const void* p) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
@@ -21,24 +33,32 @@ __device__ __forceinline__ uint4 ld_shared16(const void* p) {
                  : "r"((uint32_t)__cvta_generic_to_shared(p)));
     return v;
 }
+__device__ __forceinline__ uint2 ld_shared8(const void* p) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"((uint32_t)__cvta_generic_to_shared(p)));
+    return v;
+}
 __device__ __forceinline__ void st_shared16(void* p, uint4 v) {
     asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"((uint32_t)__cvta_generic_to_shared(p)), "r"(v.x),
                  "r"(v.y), "r"(v.z), "r"(v.w)
                  : "memory");
 }
-// where a group's 16-byte pieces come from: global memory (streaming) or a staged shared-memory tile
-struct FromGlobal {
-    __device__ __forceinline__ uint4 operator()(const uint8_t* p) const { return ld_stream16(p); }
+__device__ __forceinline__ void st_shared8(void* p, uint2 v) {
+    asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"((uint32_t)__cvta_generic_to_shared(p)), "r"(v.x), "r"(v.y)
+                 : "memory");
+}
+// memory spaces a piece is read from / written to
+struct Global {
+    static __device__ __forceinline__ uint4 ld16(const uint8_t* p) { return ld_stream16(p); }
+    static __device__ __forceinline__ uint2 ld8(const uint8_t* p) { return ld_stream8(p); }
+    static __device__ __forceinline__ void st16(uint8_t* p, uint4 v) { st_stream16(p, v); }
+    static __device__ __forceinline__ void st8(uint8_t* p, uint2 v) { st_stream8(p, v); }
 };
-struct FromShared {
-    __device__ __forceinline__ uint4 operator()(const uint8_t* p) const { return ld_shared16(p); }
-};
-// ... and where they go
-struct ToGlobal {
-    __device__ __forceinline__ void operator()(uint8_t* p, uint4 v) const { st_stream16(p, v); }
-};
-struct ToShared {
-    __device__ __forceinline__ void operator()(uint8_t* p, uint4 v) const { st_shared16(p, v); }
+struct Shared {
+    static __device__ __forceinline__ uint4 ld16(const uint8_t* p) { return ld_shared16(p); }
+    static __device__ __forceinline__ uint2 ld8(const uint8_t* p) { return ld_shared8(p); }
+    static __device__ __forceinline__ void st16(uint8_t* p, uint4 v) { st_shared16(p, v); }
+    static __device__ __forceinline__ void st8(uint8_t* p, uint2 v) { st_shared8(p, v); }
 };
 
 // (x & mask) | (y & ~mask): one three-input logic operation
@@ -90,77 +110,107 @@ __device__ __forceinline__ uint32_t fp32_merge(uint32_t e, uint32_t s) {
     return bitselect(0x007FFFFFu, s, bitselect(0x7F800000u, e << 23, s << 8));
 }
 
-// ---- a group in registers ------------------------------------------------------------------
+// ---- byte-granular access to a short run of exponent / sm bytes held in words ---------------
+template <int NB>
+__device__ __forceinline__ void load_bytes_partial(uint32_t* w, const uint8_t* src, int nbytes) {
+#pragma unroll
+    for (int i = 0; i < NB / 4; ++i) w[i] = 0;
+#pragma unroll
+    for (int i = 0; i < NB; ++i)
+        if (i < nbytes) w[i >> 2] |= (uint32_t)src[i] << (8 * (i & 3));
+}
+template <int NB>
+__device__ __forceinline__ void store_bytes_partial(uint8_t* dst, const uint32_t* w, int nbytes) {
+#pragma unroll
+    for (int i = 0; i < NB; ++i)
+        if (i < nbytes) dst[i] = (uint8_t)(w[i >> 2] >> (8 * (i & 3)));
+}
+
+// ---- pieces --------------------------------------------------------------------------------
 template <int DT>
-struct Group;
+struct Piece;
 
+// bf16: 8 values = 16 B of weights, 8 exponent bytes, 8 sm bytes
 template <>
-struct Group<CIERA_BF16> {
-    uint32_t e[4];  // 16 exponent bytes
-    uint32_t s[4];  // 16 sm bytes
+struct Piece<CIERA_BF16> {
+    static constexpr int kValues = 8;
+    static constexpr int kLog2Values = 3;
+    static constexpr int kPerThread = 2;  // pieces per thread
+    static constexpr int kExpWords = 2;
+    static constexpr int kSmWords = 2;
+    // first value (inside the tile) of piece p of consumer thread tid
+    static __device__ __forceinline__ uint32_t start(uint32_t tid, int p) {
+        return (uint32_t)p * (kTileValues / 2) + tid * 8u;
+    }
 
-    // 16 values from 32 aligned bytes
-    template <class Ld = FromGlobal>
-    __device__ __forceinline__ void split_full(const uint8_t* w, Ld ld = Ld()) {
-        uint4 a = ld(w), b = ld(w + 16);
+    uint32_t e[kExpWords];
+    uint32_t s[kSmWords];
+
+    template <class M>
+    __device__ __forceinline__ void split_full(const uint8_t* w) {
+        const uint4 a = M::ld16(w);
         bf16_split4(a.x, a.y, e[0], s[0]);
         bf16_split4(a.z, a.w, e[1], s[1]);
-        bf16_split4(b.x, b.y, e[2], s[2]);
-        bf16_split4(b.z, b.w, e[3], s[3]);
     }
-    // the first nvalid (< 16) values; the others read as +0.0 (exponent 0)
+    // the first nvalid (< 8) values; the others read as +0.0 (exponent 0)
     __device__ __forceinline__ void split_partial(const uint8_t* w, int nvalid) {
-        uint32_t x[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) x[i] = 0;
+        uint32_t x[4] = {0, 0, 0, 0};
         const uint16_t* p = reinterpret_cast<const uint16_t*>(w);
 #pragma unroll
-        for (int i = 0; i < 16; ++i)
+        for (int i = 0; i < 8; ++i)
             if (i < nvalid) x[i >> 1] |= (uint32_t)p[i] << (16 * (i & 1));
-#pragma unroll
-        for (int i = 0; i < 4; ++i) bf16_split4(x[2 * i], x[2 * i + 1], e[i], s[i]);
+        bf16_split4(x[0], x[1], e[0], s[0]);
+        bf16_split4(x[2], x[3], e[1], s[1]);
     }
-    __device__ __forceinline__ void store_sm_full(uint8_t* dst) const { st_stream16(dst, make_uint4(s[0], s[1], s[2], s[3])); }
-    __device__ __forceinline__ void store_sm_partial(uint8_t* dst, int nvalid) const {
-#pragma unroll
-        for (int i = 0; i < 16; ++i)
-            if (i < nvalid) dst[i] = (uint8_t)(s[i >> 2] >> (8 * (i & 3)));
+    template <class M>
+    __device__ __forceinline__ void load_exp_full(const uint8_t* src) {
+        const uint2 v = M::ld8(src);
+        e[0] = v.x; e[1] = v.y;
     }
-    template <class Ld = FromGlobal>
-    __device__ __forceinline__ void load_sm_full(const uint8_t* src, Ld ld = Ld()) {
-        uint4 v = ld(src);
-        s[0] = v.x; s[1] = v.y; s[2] = v.z; s[3] = v.w;
+    template <class M>
+    __device__ __forceinline__ void store_exp_full(uint8_t* dst) const { M::st8(dst, make_uint2(e[0], e[1])); }
+    __device__ __forceinline__ void load_exp_partial(const uint8_t* src, int nvalid) { load_bytes_partial<8>(e, src, nvalid); }
+    __device__ __forceinline__ void store_exp_partial(uint8_t* dst, int nvalid) const { store_bytes_partial<8>(dst, e, nvalid); }
+    template <class M>
+    __device__ __forceinline__ void load_sm_full(const uint8_t* src) {
+        const uint2 v = M::ld8(src);
+        s[0] = v.x; s[1] = v.y;
     }
-    __device__ __forceinline__ void load_sm_partial(const uint8_t* src, int nvalid) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) s[i] = 0;
-#pragma unroll
-        for (int i = 0; i < 16; ++i)
-            if (i < nvalid) s[i >> 2] |= (uint32_t)src[i] << (8 * (i & 3));
-    }
-    template <class St = ToGlobal>
-    __device__ __forceinline__ void merge_store_full(uint8_t* w, St st = St()) const {
-        uint4 a, b;
-        bf16_merge4(e[0], s[0], a.x, a.y); bf16_merge4(e[1], s[1], a.z, a.w);
-        bf16_merge4(e[2], s[2], b.x, b.y); bf16_merge4(e[3], s[3], b.z, b.w);
-        st(w, a);
-        st(w + 16, b);
+    template <class M>
+    __device__ __forceinline__ void store_sm_full(uint8_t* dst) const { M::st8(dst, make_uint2(s[0], s[1])); }
+    __device__ __forceinline__ void load_sm_partial(const uint8_t* src, int nvalid) { load_bytes_partial<8>(s, src, nvalid); }
+    __device__ __forceinline__ void store_sm_partial(uint8_t* dst, int nvalid) const { store_bytes_partial<8>(dst, s, nvalid); }
+    template <class M>
+    __device__ __forceinline__ void merge_store_full(uint8_t* w) const {
+        uint4 a;
+        bf16_merge4(e[0], s[0], a.x, a.y);
+        bf16_merge4(e[1], s[1], a.z, a.w);
+        M::st16(w, a);
     }
     __device__ __forceinline__ void merge_store_partial(uint8_t* w, int nvalid) const {
-        uint32_t x[8];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) bf16_merge4(e[i], s[i], x[2 * i], x[2 * i + 1]);
+        uint32_t x[4];
+        bf16_merge4(e[0], s[0], x[0], x[1]);
+        bf16_merge4(e[1], s[1], x[2], x[3]);
         uint16_t* p = reinterpret_cast<uint16_t*>(w);
 #pragma unroll
-        for (int i = 0; i < 16; ++i)
+        for (int i = 0; i < 8; ++i)
             if (i < nvalid) p[i] = (uint16_t)(x[i >> 1] >> (16 * (i & 1)));
     }
+    __device__ __forceinline__ bool differs(const Piece& o) const { return ((e[0] ^ o.e[0]) | (e[1] ^ o.e[1])) != 0; }
 };
 
+// fp32: 16 values = 64 B of weights, 16 exponent bytes, 48 sm bytes
 template <>
-struct Group<CIERA_FP32> {
-    uint32_t e[4];   // 16 exponent bytes
-    uint32_t s[12];  // 16 x 24-bit sm, packed little-endian
+struct Piece<CIERA_FP32> {
+    static constexpr int kValues = 16;
+    static constexpr int kLog2Values = 4;
+    static constexpr int kPerThread = 1;
+    static constexpr int kExpWords = 4;
+    static constexpr int kSmWords = 12;
+    static __device__ __forceinline__ uint32_t start(uint32_t tid, int) { return tid * 16u; }
+
+    uint32_t e[kExpWords];
+    uint32_t s[kSmWords];
 
     __device__ __forceinline__ void from_words(const uint32_t* x) {
 #pragma unroll
@@ -170,12 +220,12 @@ struct Group<CIERA_FP32> {
                        s[3 * i], s[3 * i + 1], s[3 * i + 2]);
         }
     }
-    template <class Ld = FromGlobal>
-    __device__ __forceinline__ void split_full(const uint8_t* w, Ld ld = Ld()) {
+    template <class M>
+    __device__ __forceinline__ void split_full(const uint8_t* w) {
         uint32_t x[16];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            uint4 v = ld(w + 16 * i);
+            const uint4 v = M::ld16(w + 16 * i);
             x[4 * i] = v.x; x[4 * i + 1] = v.y; x[4 * i + 2] = v.z; x[4 * i + 3] = v.w;
         }
         from_words(x);
@@ -187,30 +237,30 @@ struct Group<CIERA_FP32> {
         for (int i = 0; i < 16; ++i) x[i] = i < nvalid ? p[i] : 0u;
         from_words(x);
     }
-    __device__ __forceinline__ void store_sm_full(uint8_t* dst) const {
-#pragma unroll
-        for (int i = 0; i < 3; ++i) st_stream16(dst + 16 * i, make_uint4(s[4 * i], s[4 * i + 1], s[4 * i + 2], s[4 * i + 3]));
+    template <class M>
+    __device__ __forceinline__ void load_exp_full(const uint8_t* src) {
+        const uint4 v = M::ld16(src);
+        e[0] = v.x; e[1] = v.y; e[2] = v.z; e[3] = v.w;
     }
-    __device__ __forceinline__ void store_sm_partial(uint8_t* dst, int nvalid) const {
-#pragma unroll
-        for (int i = 0; i < 48; ++i)
-            if (i < 3 * nvalid) dst[i] = (uint8_t)(s[i >> 2] >> (8 * (i & 3)));
-    }
-    template <class Ld = FromGlobal>
-    __device__ __forceinline__ void load_sm_full(const uint8_t* src, Ld ld = Ld()) {
+    template <class M>
+    __device__ __forceinline__ void store_exp_full(uint8_t* dst) const { M::st16(dst, make_uint4(e[0], e[1], e[2], e[3])); }
+    __device__ __forceinline__ void load_exp_partial(const uint8_t* src, int nvalid) { load_bytes_partial<16>(e, src, nvalid); }
+    __device__ __forceinline__ void store_exp_partial(uint8_t* dst, int nvalid) const { store_bytes_partial<16>(dst, e, nvalid); }
+    template <class M>
+    __device__ __forceinline__ void load_sm_full(const uint8_t* src) {
 #pragma unroll
         for (int i = 0; i < 3; ++i) {
-            uint4 v = ld(src + 16 * i);
+            const uint4 v = M::ld16(src + 16 * i);
             s[4 * i] = v.x; s[4 * i + 1] = v.y; s[4 * i + 2] = v.z; s[4 * i + 3] = v.w;
         }
     }
-    __device__ __forceinline__ void load_sm_partial(const uint8_t* src, int nvalid) {
+    template <class M>
+    __device__ __forceinline__ void store_sm_full(uint8_t* dst) const {
 #pragma unroll
-        for (int i = 0; i < 12; ++i) s[i] = 0;
-#pragma unroll
-        for (int i = 0; i < 48; ++i)
-            if (i < 3 * nvalid) s[i >> 2] |= (uint32_t)src[i] << (8 * (i & 3));
+        for (int i = 0; i < 3; ++i) M::st16(dst + 16 * i, make_uint4(s[4 * i], s[4 * i + 1], s[4 * i + 2], s[4 * i + 3]));
     }
+    __device__ __forceinline__ void load_sm_partial(const uint8_t* src, int nvalid) { load_bytes_partial<48>(s, src, 3 * nvalid); }
+    __device__ __forceinline__ void store_sm_partial(uint8_t* dst, int nvalid) const { store_bytes_partial<48>(dst, s, 3 * nvalid); }
     __device__ __forceinline__ void merge_words(uint32_t* x) const {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -222,12 +272,12 @@ struct Group<CIERA_FP32> {
             x[4 * i + 3] = fp32_merge(e[i] >> 24, s3);
         }
     }
-    template <class St = ToGlobal>
-    __device__ __forceinline__ void merge_store_full(uint8_t* w, St st = St()) const {
+    template <class M>
+    __device__ __forceinline__ void merge_store_full(uint8_t* w) const {
         uint32_t x[16];
         merge_words(x);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) st(w + 16 * i, make_uint4(x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]));
+        for (int i = 0; i < 4; ++i) M::st16(w + 16 * i, make_uint4(x[4 * i], x[4 * i + 1], x[4 * i + 2], x[4 * i + 3]));
     }
     __device__ __forceinline__ void merge_store_partial(uint8_t* w, int nvalid) const {
         uint32_t x[16];
@@ -237,20 +287,15 @@ struct Group<CIERA_FP32> {
         for (int i = 0; i < 16; ++i)
             if (i < nvalid) p[i] = x[i];
     }
+    __device__ __forceinline__ bool differs(const Piece& o) const {
+        return ((e[0] ^ o.e[0]) | (e[1] ^ o.e[1]) | (e[2] ^ o.e[2]) | (e[3] ^ o.e[3])) != 0;
+    }
 };
 
-// 16 exponent bytes <-> memory
-__device__ __forceinline__ void load_exp_partial(uint32_t* e, const uint8_t* src, int nvalid) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) e[i] = 0;
-#pragma unroll
-    for (int i = 0; i < 16; ++i)
-        if (i < nvalid) e[i >> 2] |= (uint32_t)src[i] << (8 * (i & 3));
-}
-__device__ __forceinline__ void store_exp_partial(uint8_t* dst, const uint32_t* e, int nvalid) {
-#pragma unroll
-    for (int i = 0; i < 16; ++i)
-        if (i < nvalid) dst[i] = (uint8_t)(e[i >> 2] >> (8 * (i & 3)));
+// number of valid values of the piece starting at value `start` in a tile of nv values
+template <int DT>
+__device__ __forceinline__ int piece_valid(uint32_t start, uint32_t nv) {
+    return start >= nv ? 0 : (int)min((uint32_t)Piece<DT>::kValues, nv - start);
 }
 
 __device__ __forceinline__ TileDesc load_tile_desc(const TileDesc* t) {

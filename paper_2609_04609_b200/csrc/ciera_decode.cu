@@ -3,30 +3,31 @@
 // Grid = at most as many thread blocks as fit on the GPU; block c works on tiles c, c + G, ...
 // Tiles are independent here, so no block ever waits for another.  Two roles:
 //
-//   producer warp   runs ahead: for each tile it reads the tile's bits of the unit's bitmap and the
-//                   number of changed blocks before the tile, then assembles the tile's inputs in a
-//                   shared-memory stage with bulk-async copies: the received sign-plus-mantissa
-//                   tile, and the tile's exponents -- every run of unchanged blocks from the
-//                   receiver's cache, every run of changed blocks from the message payload;
-//   16 consumer     each thread merges 16 exponent bytes and 16 sign-plus-mantissa values from the
-//   warps           stage into 16 weights and stores them; threads of changed blocks also store
-//                   the new exponents to the cache (ExpCache[i,k] <- newExp[j]).
+//   producer warps  run ahead, taking the block's tiles in turn: for each tile a producer reads
+//                   the tile's bits of the unit's bitmap and the number of changed blocks before
+//                   the tile, works out the tile's addresses once for everybody, and fills a
+//                   shared-memory stage with three bulk-async copies: the received
+//                   sign-plus-mantissa tile, the span of the receiver's cached exponents that
+//                   covers the tile's unchanged blocks, and the slice of the message payload that
+//                   holds the tile's changed blocks (they are contiguous there, in block order);
+//   16 consumer     each thread merges the exponent bytes (from the cache span, or from the
+//   warps           payload slice if its block changed) and the sign-plus-mantissa of its pieces
+//                   into weights and stores them; threads of changed blocks also store the new
+//                   exponents to the cache (ExpCache[i,k] <- newExp[j]).
 //
 // The number of changed blocks before a tile is the popcount of the bitmap bits before it.  For
-// units of up to kDirectBlocks blocks the producer takes it straight from the bitmap (at most four
+// units of up to kDirectBlocks blocks a producer takes it straight from the bitmap (at most four
 // words per lane, fetched one tile ahead); longer units get it from a small prefix kernel that
 // runs first and writes one count per tile into the caller's scratch.
 #include "ciera_bits.cuh"
 #include "ciera_pipe.cuh"
 
-CIERA_PROF_READER(dec)
-
 namespace ciera {
 
-constexpr int kDecProducers = 2;                             // producer warps, taking tiles in turn
+constexpr int kDecProducers = 2;                               // producer warps, taking tiles in turn
 constexpr int kDecodeThreads = kThreads + 32 * kDecProducers;  // consumers + producers
 constexpr int kDecProducerWarp0 = kWarps;
-constexpr int kDecDescRing = 16;  // > stages + 2 * producers + 1: slots are refilled only after their tile is done
+constexpr int kDecRing = 12;  // > stages + 2 * producers + 1: slots are refilled only after their tile is done
 constexpr uint32_t kDirectWordsPerLane = 4;
 constexpr uint32_t kDirectBlocks = kDecodeDirectBlocks;
 static_assert(kDirectBlocks == 32u * 32u * kDirectWordsPerLane, "one fetch covers the direct range");
@@ -35,43 +36,48 @@ template <int DT>
 struct DecodeCfg;
 template <>
 struct DecodeCfg<CIERA_BF16> {
-    static constexpr int kStages = 5;  // 5 x (8 KB sm + 8 KB exponents)
+    static constexpr int kStages = 4;        // 4 x (8 KB sm + 8 KB cache span + 8 KB payload slice)
+    static constexpr int kBlocksPerSM = 2;
+    static constexpr bool kStageOut = false;  // weights leave as 16 B / lane, contiguous per warp
 };
 template <>
 struct DecodeCfg<CIERA_FP32> {
-    static constexpr int kStages = 2;  // 2 x (24 KB sm + 8 KB exponents)
+    static constexpr int kStages = 4;        // 4 x (24 KB sm + 8 KB + 8 KB)
+    static constexpr int kBlocksPerSM = 1;
+    static constexpr bool kStageOut = true;   // 64 B / lane: staged, then one bulk store per warp
 };
 
 // Per-tile bookkeeping, in a ring that the producers fill ahead of the consumers.
 struct __align__(16) DecodeRing {
-    TileDesc desc;                                  // copied from the plan's table (asynchronously)
+    TileDesc desc;                           // copied from the plan's table (asynchronously)
     // worked out once by a producer for the 512 consumer threads:
-    uint8_t* w_dst;                                 // where the tile's reconstructed weights go
-    uint8_t* c_ptr;                                 // the tile's cached exponents
-    const uint8_t* sm_src;                          // the tile's received sign-plus-mantissa
-    const uint8_t* pay_src;                         // start of the unit's payload section
-    unsigned long long before;                      // changed blocks of the unit before the tile
-    uint32_t nv;                                    // values in the tile
+    uint8_t* w_dst;                          // where the tile's reconstructed weights go
+    uint8_t* c_ptr;                          // the tile's cached exponents
+    const uint8_t* sm_src;                   // the tile's received sign-plus-mantissa
+    const uint8_t* pay_src;                  // the payload slice holding the tile's changed blocks
+    uint32_t nv;                             // values in the tile
     uint32_t pad;
-    uint32_t pre[32 * kDirectWordsPerLane];         // raw bitmap words before the tile
-    uint32_t own[kBitmapWords];                     // raw words holding the tile's own bits
-    uint32_t ws;                                    // count from the scratch (long units)
-    uint32_t bm[kBitmapWords];                      // digested: the tile's block flags
+    uint32_t bm[kBitmapWords];               // the tile's block flags
+    uint32_t pre[kBitmapWords];              // set flags before each word
+    // raw material, fetched asynchronously one tile ahead:
+    uint32_t raw_pre[32 * kDirectWordsPerLane];  // bitmap words before the tile
+    uint32_t raw_own[kBitmapWords];              // words holding the tile's own bits
+    uint32_t ws;                                 // count from the scratch (long units)
 };
 
 template <int S>
 struct DecodeCtl {
-    uint64_t full[S];   // stage assembled (producer arrive + bulk-copy bytes)
+    uint64_t full[S];   // stage filled (producer arrive + bulk-copy bytes)
     uint64_t empty[S];  // all 16 consumer warps have read it
-    DecodeRing ring[kDecDescRing];
+    DecodeRing ring[kDecRing];
     int abort;
     uint32_t issued;
     uint32_t seen;
 };
 
-// Starts the asynchronous fetch of the bitmap words the producer needs for one tile into the
-// ring slot `r`: the unit's words before the tile (direct units) or the tile's count from the
-// scratch (long units), and the tile's own words.  Nothing is held in registers meanwhile.
+// Starts the asynchronous fetch of the bitmap words a producer needs for one tile into the ring
+// slot `r`: the unit's words before the tile (direct units) or the tile's count from the scratch
+// (long units), and the tile's own words.  Nothing is held in registers meanwhile.
 __device__ __forceinline__ void fetch_bitmap(const TileDesc& td, uint32_t tile, uint32_t log2b, const uint8_t* msgs,
                                              const uint32_t* ws_prefix, DecodeRing* r, uint32_t lane) {
     const uint32_t* bm32 = reinterpret_cast<const uint32_t*>(msgs + td.msg_off);
@@ -83,7 +89,7 @@ __device__ __forceinline__ void fetch_bitmap(const TileDesc& td, uint32_t tile, 
 #pragma unroll
         for (uint32_t i = 0; i < kDirectWordsPerLane; ++i) {
             const uint32_t w = lane + 32u * i;
-            if (w < nwords) cp_async4(&r->pre[w], bm32 + w);
+            if (w < nwords) cp_async4(&r->raw_pre[w], bm32 + w);
         }
     } else if (lane == 0) {
         cp_async4(&r->ws, ws_prefix + tile);
@@ -92,12 +98,14 @@ __device__ __forceinline__ void fetch_bitmap(const TileDesc& td, uint32_t tile, 
     const uint32_t own_words = nbt >= 32 ? (nbt >> 5) : 1u;
     if (lane < own_words) {
         const uint64_t w = (kb0 >> 5) + lane;
-        if ((w << 5) < nb) cp_async4(&r->own[lane], bm32 + w);  // never past the bitmap's padded end
+        if ((w << 5) < nb) cp_async4(&r->raw_own[lane], bm32 + w);  // never past the bitmap's padded end
     }
 }
 
-// Turns a completed fetch into (changed blocks before the tile, the tile's block flags in r->bm).
-__device__ __forceinline__ uint64_t digest_bitmap(DecodeRing* r, const TileDesc& td, uint32_t log2b, uint32_t lane) {
+// Turns a completed fetch into the tile's block flags (r->bm, r->pre).  Returns the number of
+// changed blocks before the tile; `own_total` gets the number of changed blocks of the tile.
+__device__ __forceinline__ uint64_t digest_bitmap(DecodeRing* r, const TileDesc& td, uint32_t log2b, uint32_t lane,
+                                                  uint32_t& own_total) {
     const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
     const uint64_t kb0 = v0 >> log2b;
     const uint64_t nb = num_blocks(td.n_unit, log2b);
@@ -111,9 +119,9 @@ __device__ __forceinline__ uint64_t digest_bitmap(DecodeRing* r, const TileDesc&
         for (uint32_t i = 0; i < kDirectWordsPerLane; ++i) {
             const uint32_t w = lane + 32u * i;
             if (w < nfull)
-                cnt += __popc(r->pre[w]);
+                cnt += __popc(r->raw_pre[w]);
             else if (w == nfull && (kb0 & 31u))
-                cnt += __popc(r->pre[w] & ((1u << (kb0 & 31u)) - 1u));
+                cnt += __popc(r->raw_pre[w] & ((1u << (kb0 & 31u)) - 1u));
         }
         cnt = __reduce_add_sync(0xffffffffu, cnt);
     } else {
@@ -122,59 +130,64 @@ __device__ __forceinline__ uint64_t digest_bitmap(DecodeRing* r, const TileDesc&
     uint32_t word = 0;
     if (nbt >= 32) {
         if (lane < (nbt >> 5) && lane * 32u < nblk) {
-            word = r->own[lane];
+            word = r->raw_own[lane];
             const uint32_t left = nblk - lane * 32u;
             if (left < 32u) word &= (1u << left) - 1u;
         }
     } else if (lane == 0) {
-        word = (r->own[0] >> (kb0 & 31u)) & ((1u << nblk) - 1u);
+        word = (r->raw_own[0] >> (kb0 & 31u)) & ((1u << nblk) - 1u);
     }
-    if (lane < kBitmapWords) r->bm[lane] = word;
+    // exclusive popcount prefix over the (at most 16) words
+    const uint32_t pc = __popc(word);
+    uint32_t incl = pc;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+        if ((int)lane >= o) incl += t;
+    }
+    if (lane < kBitmapWords) {
+        r->bm[lane] = word;
+        r->pre[lane] = incl - pc;
+    }
+    own_total = __shfl_sync(0xffffffffu, incl, 31);
     __syncwarp();
     return cnt;
 }
 
-// Starts the bulk copies that assemble the exponent tile of a FULL tile: runs of unchanged blocks
-// come from the cache, runs of changed blocks from the payload.  All 32 lanes take part; every
-// lane owns the blocks lane, lane + 32, ... of each 32-block word.  Total bytes = kTileValues.
-__device__ __forceinline__ void assemble_exponents(uint8_t* s_exp, const uint8_t* cache_tile, const uint8_t* payload,
-                                                   uint64_t before, const uint32_t* bm, uint32_t log2b, uint64_t* bar,
-                                                   uint32_t lane) {
+// First and last unchanged block of a full tile (lo > hi if every block changed).  One warp;
+// lane w looks at word w of the block flags.
+__device__ __forceinline__ void unchanged_span(const uint32_t* bm, uint32_t log2b, uint32_t lane, uint32_t& lo,
+                                               uint32_t& hi) {
     const uint32_t nbt = kTileValues >> log2b;
     const uint32_t nwords = nbt >= 32 ? (nbt >> 5) : 1u;
-    const uint32_t per = nbt >= 32 ? 32u : nbt;  // blocks per word
-    uint32_t rank0 = 0;                          // changed blocks of the tile before this word
-    for (uint32_t w = 0; w < nwords; ++w) {
-        const uint32_t bits = bm[w];
-        if (lane < per) {
-            // a run starts at block 0 of the word and wherever a bit differs from its predecessor
-            const uint32_t starts = (bits ^ (bits << 1)) | 1u;
-            if ((starts >> lane) & 1u) {
-                const uint32_t later = per == 32u ? starts >> 1 >> lane : (starts & ((1u << per) - 1u)) >> 1 >> lane;
-                const uint32_t len = later ? (uint32_t)__ffs(later) : per - lane;  // blocks in the run
-                const uint32_t blk = w * 32u + lane;                                // block index in the tile
-                const bool chg = (bits >> lane) & 1u;
-                const uint32_t rank = rank0 + __popc(bits & ((1u << lane) - 1u));
-                const uint8_t* src = chg ? payload + ((before + rank) << log2b) : cache_tile + ((uint64_t)blk << log2b);
-                bulk_load(s_exp + ((size_t)blk << log2b), src, len << log2b, bar);
-            }
-        }
-        rank0 += __popc(bits);
+    const uint32_t valid = nbt >= 32 ? 0xffffffffu : ((1u << nbt) - 1u);
+    const uint32_t zeros = lane < nwords ? (~bm[lane] & valid) : 0u;
+    const uint32_t have = __ballot_sync(0xffffffffu, zeros != 0);
+    if (!have) {
+        lo = 1;
+        hi = 0;
+        return;
     }
+    const uint32_t wf = (uint32_t)__ffs(have) - 1u, wl = 31u - (uint32_t)__clz(have);
+    const uint32_t zf = __shfl_sync(0xffffffffu, zeros, wf), zl = __shfl_sync(0xffffffffu, zeros, wl);
+    lo = wf * 32u + (uint32_t)__ffs(zf) - 1u;
+    hi = wl * 32u + 31u - (uint32_t)__clz(zl);
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kDecodeThreads, 2)
+__global__ void __launch_bounds__(kDecodeThreads, DecodeCfg<DT>::kBlocksPerSM)
 decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log2b, const uint8_t* msgs, uint8_t* cache,
               uint8_t* __restrict__ weights, const unsigned long long* __restrict__ wire_bytes,
               const uint32_t* __restrict__ ws_prefix, int32_t* status) {
+    using P = Piece<DT>;
     constexpr int VB = Traits<DT>::kValueBytes;
     constexpr int SMB = Traits<DT>::kSmBytes;
     constexpr int S = DecodeCfg<DT>::kStages;
-    constexpr uint32_t kSmBytesTile = kTileValues * SMB;
-    constexpr uint32_t kStageBytes = kSmBytesTile + kTileValues;
-    constexpr uint32_t kOutBytes = kTileValues * VB;       // reconstructed tile, staged for bulk stores
-    constexpr uint32_t kWarpOutBytes = 32 * kVPT * VB;     // one warp's contiguous slice of it
+    constexpr bool kStageOut = DecodeCfg<DT>::kStageOut;
+    constexpr uint32_t kSmTile = kTileValues * SMB;                   // sign-plus-mantissa of a tile
+    constexpr uint32_t kStageBytes = kSmTile + 2u * kTileValues;       // + cache span + payload slice
+    constexpr uint32_t kOutBytes = kStageOut ? kTileValues * VB : 0u;  // reconstructed tile, staged for bulk stores
+    constexpr uint32_t kWarpOutBytes = 32 * P::kValues * VB;           // one warp's contiguous slice of it
     extern __shared__ __align__(128) uint8_t smem[];
     uint8_t* const s_out = smem + (size_t)S * kStageBytes;
     DecodeCtl<S>* ctl = reinterpret_cast<DecodeCtl<S>*>(s_out + kOutBytes);
@@ -198,18 +211,17 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
 
     if (warp >= kDecProducerWarp0) {
         // ---------------------------------------------------------------- producers (all lanes)
-        // producer p handles this block's tiles p, p + P, p + 2P, ... (index k below counts them)
+        // producer p handles this block's tiles p, p + P, p + 2P, ... (jj below counts them)
         const uint32_t pidx = warp - kDecProducerWarp0;
         const uint32_t my_prod = my_tiles > pidx ? (my_tiles - pidx + kDecProducers - 1u) / kDecProducers : 0u;
         if (my_prod > 0) {
             // software pipeline through the ring: descriptor two tiles ahead, bitmap words one tile
             // ahead, both by per-thread asynchronous copies (groups D_j and B_j, committed in the
             // order D_0 D_1 B_0 | D_2 B_1 | D_3 B_2 | ...)
-            // jj counts this producer's tiles; seq(jj) is the tile's place in the block's sequence
-            auto seq = [&](uint32_t jj) { return pidx + jj * kDecProducers; };
+            auto seq = [&](uint32_t jj) { return pidx + jj * kDecProducers; };  // place in the block's sequence
             auto fetch_desc = [&](uint32_t jj) {
                 if (jj < my_prod && lane < 3)
-                    cp_async16(reinterpret_cast<uint8_t*>(&ctl->ring[seq(jj) % kDecDescRing].desc) + 16u * lane,
+                    cp_async16(reinterpret_cast<uint8_t*>(&ctl->ring[seq(jj) % kDecRing].desc) + 16u * lane,
                                reinterpret_cast<const uint8_t*>(tiles + blockIdx.x + (uint64_t)seq(jj) * G) + 16u * lane);
                 cp_async_commit();
             };
@@ -217,155 +229,160 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
             fetch_desc(1);
             cp_async_wait<1>();  // D_0
             __syncwarp();
-            fetch_bitmap(ctl->ring[seq(0) % kDecDescRing].desc, blockIdx.x + seq(0) * G, log2b, msgs, ws_prefix,
-                         &ctl->ring[seq(0) % kDecDescRing], lane);
+            fetch_bitmap(ctl->ring[seq(0) % kDecRing].desc, blockIdx.x + seq(0) * G, log2b, msgs, ws_prefix,
+                         &ctl->ring[seq(0) % kDecRing], lane);
             cp_async_commit();
-            PROF_T0;
             for (uint32_t jj = 0; jj < my_prod; ++jj) {
                 const uint32_t k = seq(jj);
                 fetch_desc(jj + 2u);
                 cp_async_wait<1>();  // everything but D_{jj+2}: D_{jj+1} and B_jj have landed
-                PROF_ADD(0);
                 __syncwarp();
                 if (jj + 1u < my_prod) {
-                    DecodeRing* rn = &ctl->ring[seq(jj + 1u) % kDecDescRing];
+                    DecodeRing* rn = &ctl->ring[seq(jj + 1u) % kDecRing];
                     fetch_bitmap(rn->desc, blockIdx.x + seq(jj + 1u) * G, log2b, msgs, ws_prefix, rn, lane);
                 }
                 cp_async_commit();
-                PROF_ADD(1);
 
                 const uint32_t stage = k % S;
                 bool ok = true;
                 if (k >= (uint32_t)S) ok = mbar_wait(&ctl->empty[stage], ((k / S) & 1u) ^ 1u, abort, status);
                 if (!__all_sync(0xffffffffu, ok)) break;
-                PROF_ADD(2);
 
-                DecodeRing* r = &ctl->ring[k % kDecDescRing];
+                DecodeRing* r = &ctl->ring[k % kDecRing];
                 const TileDesc td = r->desc;
-                const uint64_t before = digest_bitmap(r, td, log2b, lane);
+                uint32_t own = 0;
+                const uint64_t before = digest_bitmap(r, td, log2b, lane, own);
                 const uint64_t N = td.n_unit;
                 const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
                 const uint64_t smoff = sm_offset(N, log2b);
                 const uint64_t payoff = smoff + pad16(N * SMB);
                 const uint8_t* msg = msgs + td.msg_off;
+                const uint8_t* pay = msg + payoff + (before << log2b);  // this tile's slice of the payload
                 uint8_t* st = smem + (size_t)stage * kStageBytes;
+                const bool full_tile = N - v0 >= (uint64_t)kTileValues;
+                uint32_t lo = 1, hi = 0;
+                if (full_tile) unchanged_span(r->bm, log2b, lane, lo, hi);
+
                 if (lane == 0) {
                     r->w_dst = weights + td.w_off;
                     r->c_ptr = cache + td.c_off;
                     r->sm_src = msg + smoff + v0 * SMB;
-                    r->pay_src = msg + payoff;
-                    r->before = before;
+                    r->pay_src = pay;
                     r->nv = (uint32_t)min((uint64_t)kTileValues, N - v0);
-                }
-                PROF_ADD(6);
 
-                // integrity check by the unit's last tile: the bitmap fixes the message length
-                if (wire_bytes != nullptr && status != nullptr && td.tile_in_unit == td.n_tiles_unit - 1u) {
-                    uint32_t own = lane < kBitmapWords ? __popc(r->bm[lane]) : 0u;
-                    own = __reduce_add_sync(0xffffffffu, own);
-                    const uint32_t B = 1u << log2b;
-                    const uint32_t nv = (uint32_t)(N - v0);
-                    uint64_t total = (before + own) << log2b;
-                    const uint32_t rem = nv & (B - 1u);
-                    if (rem) {
-                        const uint32_t kb = nv >> log2b;
-                        if ((r->bm[kb >> 5] >> (kb & 31u)) & 1u) total -= (B - rem);
+                    // integrity check by the unit's last tile: the bitmap fixes the message length
+                    if (wire_bytes != nullptr && status != nullptr && td.tile_in_unit == td.n_tiles_unit - 1u) {
+                        const uint32_t B = 1u << log2b;
+                        const uint32_t nv = (uint32_t)(N - v0);
+                        uint64_t total = (before + own) << log2b;
+                        const uint32_t rem = nv & (B - 1u);
+                        if (rem) {
+                            const uint32_t kb = nv >> log2b;
+                            if ((r->bm[kb >> 5] >> (kb & 31u)) & 1u) total -= (B - rem);
+                        }
+                        if (wire_bytes[td.unit] != payoff + total) atomicCAS(status, 0, (int32_t)CIERA_ERR_CORRUPT);
                     }
-                    if (lane == 0 && wire_bytes[td.unit] != payoff + total)
-                        atomicCAS(status, 0, (int32_t)CIERA_ERR_CORRUPT);
-                }
 
-                PROF_ADD(7);
-                if (N - v0 >= (uint64_t)kTileValues) {
-                    if (lane == 0) {
-                        mbar_arrive_expect_tx(&ctl->full[stage], kStageBytes);
-                        bulk_load(st, msg + smoff + v0 * SMB, kSmBytesTile, &ctl->full[stage]);
+                    if (full_tile) {
+                        const uint32_t span = lo <= hi ? (hi - lo + 1u) << log2b : 0u;
+                        const uint32_t slice = own << log2b;
+                        mbar_arrive_expect_tx(&ctl->full[stage], kSmTile + span + slice);
+                        bulk_load(st, r->sm_src, kSmTile, &ctl->full[stage]);
+                        if (span)
+                            bulk_load(st + kSmTile + ((size_t)lo << log2b), r->c_ptr + ((size_t)lo << log2b), span,
+                                      &ctl->full[stage]);
+                        if (slice) bulk_load(st + kSmTile + kTileValues, pay, slice, &ctl->full[stage]);
+                    } else {
+                        mbar_arrive(&ctl->full[stage]);  // short tile: consumers read global memory themselves
                     }
-                    __syncwarp();
-                    PROF_ADD(8);
-                    assemble_exponents(st + kSmBytesTile, cache + td.c_off, msg + payoff, before, r->bm, log2b,
-                                       &ctl->full[stage], lane);
-                } else {
-                    // short tile: consumers read global memory themselves
-                    if (lane == 0) mbar_arrive(&ctl->full[stage]);
+                    atomicMax(&ctl->issued, k + 1u);
                 }
-                if (lane == 0) atomicMax(&ctl->issued, k + 1u);
-                PROF_ADD(3);
+                __syncwarp();
             }
-            PROF_FLUSH;
             cp_async_wait<0>();
         }
     } else {
         // ---------------------------------------------------------------- consumers
-        const uint32_t t0 = tid * kVPT;
-        PROF_T0;
+        const uint32_t bmask = (1u << log2b) - 1u;
         for (uint32_t k = 0; k < my_tiles; ++k) {
             const uint32_t stage = k % S;
             if (!mbar_wait(&ctl->full[stage], (k / S) & 1u, abort, status)) break;
-            PROF_ADD(4);
             if (tid == 0) ctl->seen = k + 1;
-            const DecodeRing* r = &ctl->ring[k % kDecDescRing];
+            const DecodeRing* r = &ctl->ring[k % kDecRing];
             const uint32_t nv = r->nv;
-            const int nvalid = t0 >= nv ? 0 : (int)min(16u, nv - t0);
-            const uint8_t* st = smem + (size_t)stage * kStageBytes;
-            const uint32_t kb = t0 >> log2b;
-            const uint32_t word = r->bm[kb >> 5];
-            const bool chg = nvalid > 0 && ((word >> (kb & 31u)) & 1u);
-            uint8_t* cptr = r->c_ptr + t0;
+            const uint8_t* const st = smem + (size_t)stage * kStageBytes;
+            uint8_t* const c_ptr = r->c_ptr;
             uint8_t* const w_dst = r->w_dst;
-            uint8_t* wptr = w_dst + (size_t)t0 * VB;
 
-            Group<DT> g;
             if (nv == (uint32_t)kTileValues) {
-                g.load_sm_full(st + (size_t)t0 * SMB, FromShared());
-                const uint4 ev = ld_shared16(st + kSmBytesTile + t0);
-                g.e[0] = ev.x; g.e[1] = ev.y; g.e[2] = ev.z; g.e[3] = ev.w;
-                if (chg) st_stream16(cptr, ev);  // ExpCache[i,k] <- newExp[j]
-                // the warp's 32 x 16 weights are contiguous: stage them and send them with one
-                // bulk store (fully coalesced by the copy engine, no store instructions per lane)
-                if (lane == 0) bulk_wait_read<0>();  // the slice's previous bulk store has been read out
-                __syncwarp();
-                g.merge_store_full(s_out + (size_t)t0 * VB, ToShared());
-                fence_async_shared();
-                __syncwarp();  // every lane has used what it read from the stage and written its part
+                if (kStageOut) {
+                    if (lane == 0) bulk_wait_read<0>();  // the warp's previous bulk store has been read out
+                    __syncwarp();
+                }
+#pragma unroll
+                for (int p = 0; p < P::kPerThread; ++p) {
+                    const uint32_t t0 = P::start(tid, p);
+                    const uint32_t kb = t0 >> log2b;
+                    const uint32_t word = r->bm[kb >> 5];
+                    const bool chg = (word >> (kb & 31u)) & 1u;
+                    // exponents: the cached ones, or -- changed block -- the ones that came in the payload
+                    const uint32_t rank = r->pre[kb >> 5] + __popc(word & ((1u << (kb & 31u)) - 1u));
+                    const uint8_t* esrc = chg ? st + kSmTile + kTileValues + ((size_t)rank << log2b) + (t0 & bmask)
+                                              : st + kSmTile + t0;
+                    P x;
+                    x.template load_sm_full<Shared>(st + (size_t)t0 * SMB);
+                    x.template load_exp_full<Shared>(esrc);
+                    if (chg) x.template store_exp_full<Global>(c_ptr + t0);  // ExpCache[i,k] <- newExp[j]
+                    if (kStageOut)
+                        x.template merge_store_full<Shared>(s_out + (size_t)t0 * VB);
+                    else
+                        x.template merge_store_full<Global>(w_dst + (size_t)t0 * VB);
+                }
+                if (kStageOut) fence_async_shared();
+                __syncwarp();  // every lane has used what it read from the stage (and staged its output)
                 if (lane == 0) {
                     mbar_arrive(&ctl->empty[stage]);
-                    bulk_store(w_dst + (size_t)warp * kWarpOutBytes, s_out + (size_t)warp * kWarpOutBytes, kWarpOutBytes);
-                    bulk_commit();
-                }
-                PROF_ADD(5);
-            } else {
-                const unsigned long long before = r->before;
-                const uint8_t* smsrc = r->sm_src + (size_t)t0 * SMB;
-                const uint8_t* paysrc = r->pay_src;
-                uint32_t rank = __popc(word & ((1u << (kb & 31u)) - 1u));
-                for (uint32_t w = 0; w < (kb >> 5); ++w) rank += __popc(r->bm[w]);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl->empty[stage]);
-                if (nvalid > 0) {
-                    const uint8_t* src = cptr;  // unchanged block: the cached exponents
-                    if (chg)                    // changed block: its exponents are in the payload
-                        src = paysrc + ((before + rank) << log2b) + (t0 & ((1u << log2b) - 1u));
-                    if (nvalid == 16) {
-                        g.load_sm_full(smsrc);
-                        const uint4 ev = ld_stream16(src);
-                        g.e[0] = ev.x; g.e[1] = ev.y; g.e[2] = ev.z; g.e[3] = ev.w;
-                        if (chg) st_stream16(cptr, ev);
-                        g.merge_store_full(wptr);
-                    } else {
-                        g.load_sm_partial(smsrc, nvalid);
-                        load_exp_partial(g.e, src, nvalid);
-                        if (chg) store_exp_partial(cptr, g.e, nvalid);
-                        g.merge_store_partial(wptr, nvalid);
+                    if (kStageOut) {
+                        // the warp's weights are contiguous: one bulk store, coalesced by the copy engine
+                        bulk_store(w_dst + (size_t)warp * kWarpOutBytes, s_out + (size_t)warp * kWarpOutBytes, kWarpOutBytes);
+                        bulk_commit();
                     }
                 }
+            } else {
+                // short tile: straight from global memory
+                const uint8_t* const sm_src = r->sm_src;
+                const uint8_t* const pay_src = r->pay_src;
+#pragma unroll
+                for (int p = 0; p < P::kPerThread; ++p) {
+                    const uint32_t t0 = P::start(tid, p);
+                    const int nvalid = piece_valid<DT>(t0, nv);
+                    if (nvalid == 0) continue;
+                    const uint32_t kb = t0 >> log2b;
+                    const uint32_t word = r->bm[kb >> 5];
+                    const bool chg = (word >> (kb & 31u)) & 1u;
+                    const uint32_t rank = r->pre[kb >> 5] + __popc(word & ((1u << (kb & 31u)) - 1u));
+                    const uint8_t* esrc = chg ? pay_src + ((size_t)rank << log2b) + (t0 & bmask) : c_ptr + t0;
+                    P x;
+                    if (nvalid == P::kValues) {
+                        x.template load_sm_full<Global>(sm_src + (size_t)t0 * SMB);
+                        x.template load_exp_full<Global>(esrc);
+                        if (chg) x.template store_exp_full<Global>(c_ptr + t0);
+                        x.template merge_store_full<Global>(w_dst + (size_t)t0 * VB);
+                    } else {
+                        x.load_sm_partial(sm_src + (size_t)t0 * SMB, nvalid);
+                        x.load_exp_partial(esrc, nvalid);
+                        if (chg) x.store_exp_partial(c_ptr + t0, nvalid);
+                        x.merge_store_partial(w_dst + (size_t)t0 * VB, nvalid);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->empty[stage]);
             }
         }
-        if (warp == 0) PROF_FLUSH;
     }
 
     // bulk stores of this thread (lane 0 of the consumer warps) are complete before the block ends
-    bulk_wait_all<0>();
+    if (kStageOut) bulk_wait_all<0>();
     // leave together; after an aborted run wait (bounded) for bulk copies that are still in flight
     __syncthreads();
     if (tid == 0 && ctl->abort) {
@@ -431,8 +448,9 @@ decode_prefix_kernel(const TileDesc* __restrict__ tiles, const uint32_t* __restr
 template <int DT>
 static size_t decode_smem_bytes() {
     constexpr int S = DecodeCfg<DT>::kStages;
-    return (size_t)S * (kTileValues * Traits<DT>::kSmBytes + kTileValues) + (size_t)kTileValues * Traits<DT>::kValueBytes +
-           sizeof(DecodeCtl<S>);
+    const size_t stage = (size_t)kTileValues * Traits<DT>::kSmBytes + 2u * kTileValues;
+    const size_t out = DecodeCfg<DT>::kStageOut ? (size_t)kTileValues * Traits<DT>::kValueBytes : 0;
+    return (size_t)S * stage + out + sizeof(DecodeCtl<S>);
 }
 
 template <int DT>

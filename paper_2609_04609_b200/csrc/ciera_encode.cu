@@ -2,19 +2,20 @@
 //
 // Grid = G thread blocks that are all resident at once (cooperative launch); block c works on
 // tiles c, c + G, c + 2G, ... of the plan's tile table, so neighbouring tiles of a unit are worked
-// on by neighbouring blocks at about the same time and the look-back below rarely waits.
+// on by neighbouring blocks at about the same time and the look-back below rarely waits long.
 // A thread block has four roles:
 //
 //   producer warp   runs ahead of the others: for each of its tiles it fetches the tile
-//                   descriptor and starts two bulk-async copies into shared memory -- the weights
-//                   tile into a short ring (freed as soon as the consumers have read it) and the
-//                   cached-exponent tile into a longer ring (held until the tile is resolved);
-//   16 consumer     each thread owns 16 consecutive values: split into exponent bytes and
-//   warps           sign-plus-mantissa, compare with the cached exponents, vote (ballot) the
-//                   "my 16 values changed" bit, store sign-plus-mantissa to the message and
-//                   leave the new exponents where the cached ones were staged;
-//   aggregator warp turns the 512 vote bits of a tile into block flags (the unit's bitmap), counts
-//                   the tile's payload bytes and publishes them as the tile's status word;
+//                   descriptor, works out the tile's addresses once for everybody, and starts two
+//                   bulk-async copies into shared memory -- the weights tile into a short ring
+//                   (freed as soon as the consumers have read it) and the cached-exponent tile
+//                   into a longer ring (held until the tile's changed exponents have been sent);
+//   16 consumer     each thread owns one or two pieces of consecutive values: split into exponent
+//   warps           bytes and sign-plus-mantissa, compare with the cached exponents, vote (ballot)
+//                   the "my piece changed" bit, store sign-plus-mantissa to the message and leave
+//                   the new exponents where the cached ones were staged;
+//   aggregator warp turns the vote bits of a tile into block flags (the unit's bitmap), counts the
+//                   tile's payload bytes and publishes them as the tile's status word;
 //   resolver warps  resolve the tile's exclusive offset in the unit's payload with a single-pass
 //                   look-back over the status words.
 // A few tiles later, when that offset is known, the consumers send the exponents of changed
@@ -26,17 +27,16 @@
 #include "ciera_bits.cuh"
 #include "ciera_pipe.cuh"
 
-CIERA_PROF_READER(enc)
-
 namespace ciera {
 
-constexpr int kResolvers = 3;                       // resolver warps
+constexpr int kResolvers = 3;                                    // resolver warps
 constexpr int kEncodeThreads = kThreads + 64 + 32 * kResolvers;  // consumers + producer + aggregator + resolvers
-constexpr int kProducerWarp = kWarps;               // 16
-constexpr int kAggregatorWarp = kWarps + 1;         // 17
-constexpr int kResolverWarp0 = kWarps + 2;          // 18 ..
-constexpr int kDescRing = 16;                       // > exponent stages + 2
-constexpr int kDefer = 3;                           // consumers send a tile's changed exponents this many tiles later
+constexpr int kProducerWarp = kWarps;                            // 16
+constexpr int kAggregatorWarp = kWarps + 1;                      // 17
+constexpr int kResolverWarp0 = kWarps + 2;                       // 18 ..
+constexpr int kDescRing = 16;                                    // > exponent stages + 2
+constexpr int kDefer = 3;       // consumers send a tile's changed exponents this many tiles later
+constexpr int kVoteWords = 32;  // vote bits of a tile: up to 1024 pieces
 
 template <int DT>
 struct EncodeCfg;
@@ -64,17 +64,17 @@ struct __align__(16) EncodeTileInfo {
 
 template <int SW, int SE>
 struct EncodeCtl {
-    uint64_t full_w[SW];   // weights tile landed
-    uint64_t empty_w[SW];  // all 16 consumer warps have read it
-    uint64_t full_e[SE];   // cached-exponent tile landed
-    uint64_t voted[SE];    // all 16 consumer warps have left their exponents there and voted
-    uint64_t summed[SE];   // aggregator has published the tile's status and block flags
-    uint64_t resolved[SE]; // a resolver knows the tile's offset in the unit's payload
-    uint64_t empty_e[SE];  // all 16 consumer warps have sent the tile's changed exponents
+    uint64_t full_w[SW];    // weights tile landed
+    uint64_t empty_w[SW];   // all 16 consumer warps have read it
+    uint64_t full_e[SE];    // cached-exponent tile landed
+    uint64_t voted[SE];     // all 16 consumer warps have left their exponents there and voted
+    uint64_t summed[SE];    // aggregator has published the tile's status and block flags
+    uint64_t resolved[SE];  // a resolver knows the tile's offset in the unit's payload
+    uint64_t empty_e[SE];   // all 16 consumer warps have sent the tile's changed exponents
     TileDesc desc[kDescRing];
     EncodeTileInfo info[kDescRing];
     uint32_t tile_idx[kDescRing];  // table index of the tile in desc[]
-    uint32_t ballot[SE][kWarps];
+    uint32_t ballot[SE][kVoteWords];
     uint32_t bm[SE][kBitmapWords];
     uint32_t pre[SE][kBitmapWords];
     unsigned long long agg[SE];
@@ -116,12 +116,12 @@ __device__ __forceinline__ uint64_t warp_sum_u64(uint64_t v) {
     return v;
 }
 
-// Block flags of a tile from the per-warp ballots of "my 16 values differ" (one warp).
-// Fills bm (one bit per block of the tile) and pre (set bits before each word); returns the
-// number of changed blocks of the tile.
+// Block flags of a tile from the vote bits "my piece differs" (one warp).  `pl2` = log2 of the
+// values per piece.  Fills bm (one bit per block of the tile) and pre (set bits before each word);
+// returns the number of changed blocks of the tile.
 __device__ __forceinline__ uint32_t build_block_bitmap(const uint32_t* ballot, uint32_t* bm, uint32_t* pre,
-                                                       uint32_t log2b, uint32_t lane) {
-    const uint32_t gl2 = log2b - 4;             // log2(groups of 16 values per block)
+                                                       uint32_t log2b, uint32_t pl2, uint32_t lane) {
+    const uint32_t gl2 = log2b - pl2;           // log2(pieces per block)
     const uint32_t nbt = kTileValues >> log2b;  // blocks of a full tile
     uint32_t run = 0;
     for (uint32_t base = 0; base < nbt; base += 32) {
@@ -165,7 +165,7 @@ __device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t 
     const uint32_t nv = (uint32_t)min((uint64_t)kTileValues, N - v0);
     uint8_t* msg = msgs + td.msg_off;
 
-    const uint32_t run = build_block_bitmap(ballot, bm, pre, log2b, lane);
+    const uint32_t run = build_block_bitmap(ballot, bm, pre, log2b, Piece<DT>::kLog2Values, lane);
 
     // payload bytes of this tile: B per changed block, less for a changed short last block
     uint64_t agg = (uint64_t)run << log2b;
@@ -254,26 +254,32 @@ __device__ __forceinline__ uint64_t resolve_tile(const TileDesc& td, uint32_t ti
 }
 
 // payload <- exponents of changed blocks in block order; cache refreshed for the same blocks.
-// Every consumer thread sends its own 16 exponents (left in the stage's shared-memory tile) if
-// its block changed; `base` is the tile's exclusive offset in the unit's payload.
+// Every consumer thread sends the exponents of its own pieces (left in the stage's shared-memory
+// tile) if their block changed; `base` is the tile's exclusive offset in the unit's payload.
+template <int DT>
 __device__ __forceinline__ void write_changed(const EncodeTileInfo& ti, uint32_t log2b, const uint32_t* bm,
-                                              const uint32_t* pre, uint64_t base, const uint8_t* s_exp, uint32_t t0) {
-    if (t0 >= ti.nv) return;
-    const uint32_t kb = t0 >> log2b;
-    const uint32_t word = bm[kb >> 5];
-    if (!((word >> (kb & 31u)) & 1u)) return;
-    const int nvalid = (int)min(16u, ti.nv - t0);
-    const uint32_t rank = pre[kb >> 5] + __popc(word & ((1u << (kb & 31u)) - 1u));
-    uint8_t* pdst = ti.pay_dst + base + ((uint64_t)rank << log2b) + (t0 & ((1u << log2b) - 1u));
-    uint8_t* cdst = ti.c_ptr + t0;
-    const uint4 ev = ld_shared16(s_exp + t0);
-    if (nvalid == 16) {
-        st_stream16(pdst, ev);
-        st_stream16(cdst, ev);
-    } else {
-        const uint32_t e[4] = {ev.x, ev.y, ev.z, ev.w};
-        store_exp_partial(pdst, e, nvalid);
-        store_exp_partial(cdst, e, nvalid);
+                                              const uint32_t* pre, uint64_t base, const uint8_t* s_exp, uint32_t tid) {
+    using P = Piece<DT>;
+#pragma unroll
+    for (int p = 0; p < P::kPerThread; ++p) {
+        const uint32_t t0 = P::start(tid, p);
+        const int nvalid = piece_valid<DT>(t0, ti.nv);
+        if (nvalid == 0) continue;
+        const uint32_t kb = t0 >> log2b;
+        const uint32_t word = bm[kb >> 5];
+        if (!((word >> (kb & 31u)) & 1u)) continue;
+        const uint32_t rank = pre[kb >> 5] + __popc(word & ((1u << (kb & 31u)) - 1u));
+        uint8_t* pdst = ti.pay_dst + base + ((uint64_t)rank << log2b) + (t0 & ((1u << log2b) - 1u));
+        uint8_t* cdst = ti.c_ptr + t0;
+        P x;
+        x.template load_exp_full<Shared>(s_exp + t0);
+        if (nvalid == P::kValues) {
+            x.template store_exp_full<Global>(pdst);
+            x.template store_exp_full<Global>(cdst);
+        } else {
+            x.store_exp_partial(pdst, nvalid);
+            x.store_exp_partial(cdst, nvalid);
+        }
     }
 }
 
@@ -282,6 +288,7 @@ __global__ void __launch_bounds__(kEncodeThreads, 2)
 encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log2b, const uint8_t* __restrict__ weights,
               uint8_t* cache, uint8_t* msgs, unsigned long long* wire_bytes, uint32_t* changed_blocks,
               unsigned long long* tile_status, int32_t* status) {
+    using P = Piece<DT>;
     constexpr int VB = Traits<DT>::kValueBytes;
     constexpr int SMB = Traits<DT>::kSmBytes;
     constexpr int SW = EncodeCfg<DT>::kWStages;
@@ -322,7 +329,6 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
         // ---------------------------------------------------------------- producer
         if (lane == 0 && my_tiles > 0) {
             TileDesc nxt = load_tile_desc(tiles + blockIdx.x);  // descriptors are fetched one tile ahead
-            PROF_T0;
             for (uint32_t k = 0; k < my_tiles; ++k) {
                 const TileDesc td = nxt;
                 const uint32_t tile = blockIdx.x + k * G;
@@ -330,7 +336,6 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                 const uint32_t sw = k % SW, se = k % SE;
                 if (k >= (uint32_t)SW && !mbar_wait(&ctl->empty_w[sw], ((k / SW) & 1u) ^ 1u, abort, status)) break;
                 if (k >= (uint32_t)SE && !mbar_wait(&ctl->empty_e[se], ((k / SE) & 1u) ^ 1u, abort, status)) break;
-                PROF_ADD(0);
                 ctl->desc[k % kDescRing] = td;
                 ctl->tile_idx[k % kDescRing] = tile;
                 const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
@@ -356,118 +361,100 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                     mbar_arrive(&ctl->full_e[se]);
                 }
                 ctl->issued = k + 1;
-                PROF_ADD(1);
             }
-            PROF_FLUSH;
         }
     } else if (warp == kAggregatorWarp) {
         // ---------------------------------------------------------------- aggregator
-        PROF_T0;
         for (uint32_t k = 0; k < my_tiles; ++k) {
             const uint32_t se = k % SE;
             if (!mbar_wait(&ctl->voted[se], (k / SE) & 1u, abort, status)) break;
-            PROF_ADD(2);
             const TileDesc td = ctl->desc[k % kDescRing];
             const uint64_t agg = aggregate_tile<DT>(td, ctl->tile_idx[k % kDescRing], log2b, ctl->ballot[se], ctl->bm[se],
                                                     ctl->pre[se], msgs, tile_status, lane);
             if (lane == 0) ctl->agg[se] = agg;
             __syncwarp();
             if (lane == 0) mbar_arrive(&ctl->summed[se]);
-            PROF_ADD(3);
         }
-        PROF_FLUSH;
     } else if (warp >= kResolverWarp0) {
         // ---------------------------------------------------------------- resolvers (tiles k = i, i + R, ...)
-        PROF_T0;
         for (uint32_t k = warp - kResolverWarp0; k < my_tiles; k += kResolvers) {
             const uint32_t se = k % SE;
             if (!mbar_wait(&ctl->summed[se], (k / SE) & 1u, abort, status)) break;
-            PROF_ADD(4);
             const TileDesc td = ctl->desc[k % kDescRing];
             const uint64_t excl = resolve_tile<DT>(td, ctl->tile_idx[k % kDescRing], log2b, ctl->agg[se], ctl->bm[se], msgs,
                                                    wire_bytes, changed_blocks, tile_status, status, lane);
-            PROF_ADD(5);
             if (lane == 0) {
                 ctl->base[se] = excl;
                 mbar_arrive(&ctl->resolved[se]);
             }
         }
-        if (warp == kResolverWarp0) PROF_FLUSH;
     } else {
         // ---------------------------------------------------------------- consumers
-        const uint32_t t0 = tid * kVPT;
-        PROF_T0;
         for (uint32_t k = 0; k < my_tiles; ++k) {
             const uint32_t sw = k % SW, se = k % SE;
             if (!mbar_wait(&ctl->full_w[sw], (k / SW) & 1u, abort, status)) break;
             if (!mbar_wait(&ctl->full_e[se], (k / SE) & 1u, abort, status)) break;
-            PROF_ADD(7);
             if (tid == 0) ctl->seen = k + 1;
             const EncodeTileInfo ti = ctl->info[k % kDescRing];
             const uint32_t nv = ti.nv;
-            const int nvalid = t0 >= nv ? 0 : (int)min(16u, nv - t0);
-            uint8_t* const se_ptr = ring_e + (size_t)se * kEBytes + t0;
+            const uint8_t* const s_w = ring_w + (size_t)sw * kWBytes;
+            uint8_t* const s_e = ring_e + (size_t)se * kEBytes;
 
-            // (exp, mant) <- SplitExpMant, and the cached exponents of the same 16 values
-            Group<DT> g;
-            uint32_t c[4];
-            if (nv == (uint32_t)kTileValues) {
-                g.split_full(ring_w + (size_t)sw * kWBytes + (size_t)t0 * VB, FromShared());
-                const uint4 cv = ld_shared16(se_ptr);
-                c[0] = cv.x; c[1] = cv.y; c[2] = cv.z; c[3] = cv.w;
-            } else if (nvalid == 16) {
-                g.split_full(ti.w_src + (size_t)t0 * VB);
-                const uint4 cv = ld_stream16(ti.c_ptr + t0);
-                c[0] = cv.x; c[1] = cv.y; c[2] = cv.z; c[3] = cv.w;
-            } else {
-                // values past the end of the unit read as exponent 0 against a cached 0: never "changed"
-                g.split_partial(ti.w_src + (size_t)t0 * VB, nvalid);
-                load_exp_partial(c, ti.c_ptr + t0, nvalid);
+#pragma unroll
+            for (int p = 0; p < P::kPerThread; ++p) {
+                const uint32_t t0 = P::start(tid, p);
+                const int nvalid = piece_valid<DT>(t0, nv);
+                // (exp, mant) <- SplitExpMant, and the cached exponents of the same values
+                P x, c;
+                if (nv == (uint32_t)kTileValues) {
+                    x.template split_full<Shared>(s_w + (size_t)t0 * VB);
+                    c.template load_exp_full<Shared>(s_e + t0);
+                } else if (nvalid == P::kValues) {
+                    x.template split_full<Global>(ti.w_src + (size_t)t0 * VB);
+                    c.template load_exp_full<Global>(ti.c_ptr + t0);
+                } else {
+                    // values past the end of the unit read as exponent 0 against a cached 0: never "changed"
+                    x.split_partial(ti.w_src + (size_t)t0 * VB, nvalid);
+                    c.load_exp_partial(ti.c_ptr + t0, nvalid);
+                }
+                // leave the new exponents where the cached ones were staged: they are sent from
+                // there once the tile's place in the payload is known
+                x.template store_exp_full<Shared>(s_e + t0);
+                const uint32_t bal = __ballot_sync(0xffffffffu, x.differs(c));
+                if (lane == 0) ctl->ballot[se][p * kWarps + warp] = bal;
+                // sign-plus-mantissa of every value
+                uint8_t* smdst = ti.sm_dst + (size_t)t0 * SMB;
+                if (nvalid == P::kValues)
+                    x.template store_sm_full<Global>(smdst);
+                else if (nvalid > 0)
+                    x.store_sm_partial(smdst, nvalid);
             }
-            // leave the new exponents where the cached ones were staged: a resolver sends the
-            // changed blocks from there once it knows where they go
-            st_shared16(se_ptr, make_uint4(g.e[0], g.e[1], g.e[2], g.e[3]));
-
-            const bool diff = ((g.e[0] ^ c[0]) | (g.e[1] ^ c[1]) | (g.e[2] ^ c[2]) | (g.e[3] ^ c[3])) != 0;
-            const uint32_t bal = __ballot_sync(0xffffffffu, diff);
             __syncwarp();  // the warp's shared-memory accesses above are ordered before lane 0's arrives
             if (lane == 0) {
                 mbar_arrive(&ctl->empty_w[sw]);
-                ctl->ballot[se][warp] = bal;
                 mbar_arrive(&ctl->voted[se]);
             }
-
-            // sign-plus-mantissa of every value
-            uint8_t* smdst = ti.sm_dst + (size_t)t0 * SMB;
-            if (nvalid == 16)
-                g.store_sm_full(smdst);
-            else if (nvalid > 0)
-                g.store_sm_partial(smdst, nvalid);
-            PROF_ADD(8);
 
             // the changed exponents of the tile handled kDefer tiles ago: its offset is known by now
             if (k >= (uint32_t)kDefer) {
                 const uint32_t j = k - kDefer, je = j % SE;
                 if (!mbar_wait(&ctl->resolved[je], (j / SE) & 1u, abort, status)) break;
-                PROF_ADD(6);
-                write_changed(ctl->info[j % kDescRing], log2b, ctl->bm[je], ctl->pre[je], ctl->base[je],
-                              ring_e + (size_t)je * kEBytes, t0);
+                write_changed<DT>(ctl->info[j % kDescRing], log2b, ctl->bm[je], ctl->pre[je], ctl->base[je],
+                                  ring_e + (size_t)je * kEBytes, tid);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&ctl->empty_e[je]);
-                PROF_ADD(9);
             }
         }
         if (!*abort) {
             for (uint32_t j = my_tiles > (uint32_t)kDefer ? my_tiles - kDefer : 0u; j < my_tiles; ++j) {
                 const uint32_t je = j % SE;
                 if (!mbar_wait(&ctl->resolved[je], (j / SE) & 1u, abort, status)) break;
-                write_changed(ctl->info[j % kDescRing], log2b, ctl->bm[je], ctl->pre[je], ctl->base[je],
-                              ring_e + (size_t)je * kEBytes, t0);
+                write_changed<DT>(ctl->info[j % kDescRing], log2b, ctl->bm[je], ctl->pre[je], ctl->base[je],
+                                  ring_e + (size_t)je * kEBytes, tid);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&ctl->empty_e[je]);
             }
         }
-        if (warp == 0) PROF_FLUSH;
     }
 
     // leave together; after an aborted run wait (bounded) for bulk copies that are still in flight

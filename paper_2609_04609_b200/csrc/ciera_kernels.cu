@@ -10,25 +10,30 @@ namespace ciera {
 template <int DT>
 __global__ void __launch_bounds__(kThreads)
 cache_fill_kernel(const TileDesc* __restrict__ tiles, const uint8_t* __restrict__ weights, uint8_t* __restrict__ cache) {
+    using P = Piece<DT>;
     constexpr int VB = Traits<DT>::kValueBytes;
     const TileDesc td = load_tile_desc(tiles + blockIdx.x);
     const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
     const uint32_t nv = (uint32_t)min((uint64_t)kTileValues, td.n_unit - v0);
-    const uint32_t t0 = threadIdx.x * kVPT;
-    const int nvalid = t0 >= nv ? 0 : (int)min(16u, nv - t0);
-    if (nvalid == 0) return;
-    Group<DT> g;
-    g.e[0] = g.e[1] = g.e[2] = g.e[3] = 0;
-    if (weights != nullptr) {
-        if (nvalid == 16)
-            g.split_full(weights + td.w_off + (uint64_t)t0 * VB);
+#pragma unroll
+    for (int p = 0; p < P::kPerThread; ++p) {
+        const uint32_t t0 = P::start(threadIdx.x, p);
+        const int nvalid = piece_valid<DT>(t0, nv);
+        if (nvalid == 0) continue;
+        P x;
+#pragma unroll
+        for (int i = 0; i < P::kExpWords; ++i) x.e[i] = 0;
+        if (weights != nullptr) {
+            if (nvalid == P::kValues)
+                x.template split_full<Global>(weights + td.w_off + (uint64_t)t0 * VB);
+            else
+                x.split_partial(weights + td.w_off + (uint64_t)t0 * VB, nvalid);
+        }
+        if (nvalid == P::kValues)
+            x.template store_exp_full<Global>(cache + td.c_off + t0);
         else
-            g.split_partial(weights + td.w_off + (uint64_t)t0 * VB, nvalid);
+            x.store_exp_partial(cache + td.c_off + t0, nvalid);
     }
-    if (nvalid == 16)
-        st_stream16(cache + td.c_off + t0, make_uint4(g.e[0], g.e[1], g.e[2], g.e[3]));
-    else
-        store_exp_partial(cache + td.c_off + t0, g.e, nvalid);
 }
 
 // ------------------------------------------------------------------------------------------
