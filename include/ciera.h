@@ -162,9 +162,9 @@ CIERA_API int ciera_encode(const ciera_plan* plan, const void* weights_dev, void
 
 /* Copies, for every unit, the first wire_bytes_dev[u] bytes of its slot from `src_messages_dev`
  * to the same slot of `dst_messages_dev` (one kernel; the lengths are read on the device).  This
- * stands where the Allgather of the messages would be. */
+ * stands where the Allgather of the messages would be.  status_dev (may be NULL) as above. */
 CIERA_API int ciera_transport(const ciera_plan* plan, const void* src_messages_dev, void* dst_messages_dev,
-                    const uint64_t* wire_bytes_dev, void* stream);
+                    const uint64_t* wire_bytes_dev, int32_t* status_dev, void* stream);
 
 /* ---- receiver: Algorithm 1, receiver part; Section 3.1 ------------------------------------- */
 

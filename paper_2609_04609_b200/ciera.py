@@ -68,7 +68,7 @@ _SIGS = {
     "ciera_cache_init": ([_vp, _vp, _vp, _vp], _i32),
     "ciera_cache_update": ([_vp, _vp, _vp, _vp], _i32),
     "ciera_encode": ([_vp] * 9, _i32),
-    "ciera_transport": ([_vp] * 5, _i32),
+    "ciera_transport": ([_vp] * 6, _i32),
     "ciera_decode": ([_vp] * 8, _i32),
     "ciera_roundtrip_host": ([_vp, _vp, _sz, _vp, _vp, _vp, _vp], _i32),
     "ciera_should_compress": ([ctypes.POINTER(GainIn), ctypes.POINTER(_dbl), ctypes.POINTER(_i32)], _i32),
@@ -203,9 +203,9 @@ def encode(plan: Plan, weights, sender_cache, messages, wire_bytes, changed_bloc
                              _ptr(changed_blocks), _ptr(workspace), _ptr(status), _stream(stream)))
 
 
-def transport(plan: Plan, src_messages, dst_messages, wire_bytes, stream=None) -> None:
+def transport(plan: Plan, src_messages, dst_messages, wire_bytes, status=None, stream=None) -> None:
     _check("ciera_transport",
-           _lib.ciera_transport(plan.handle, _ptr(src_messages), _ptr(dst_messages), _ptr(wire_bytes),
+           _lib.ciera_transport(plan.handle, _ptr(src_messages), _ptr(dst_messages), _ptr(wire_bytes), _ptr(status),
                                 _stream(stream)))
 
 

@@ -1,6 +1,7 @@
 // Auxiliary sm_100a kernels of libciera: cache initialisation, the transport stand-in, and the
 // host-buffer round trip.  (Encode and decode live in ciera_encode.cu / ciera_decode.cu.)
 #include "ciera_bits.cuh"
+#include "ciera_pipe.cuh"
 
 namespace ciera {
 
@@ -38,22 +39,79 @@ cache_fill_kernel(const TileDesc* __restrict__ tiles, const uint8_t* __restrict_
 
 // ------------------------------------------------------------------------------------------
 // transport stand-in: copy the used bytes of every slot
+//
+// A persistent copy kernel in which every warp works on its own: warp w of the grid takes tiles
+// w, w + W, ... of the plan's table; tile j of a unit moves bytes [j * chunk, (j + 1) * chunk) of
+// the unit's slot, cut off at the length the sender reported.  A warp moves 4 KB per step (eight
+// 128-bit loads per lane in flight, then eight stores); the tile descriptor and the reported
+// length of the next tiles are fetched ahead so that no step waits for them.
 
-__global__ void __launch_bounds__(kThreads)
-transport_kernel(const TileDesc* __restrict__ tiles, uint32_t sm_bytes_per_value, const uint8_t* __restrict__ src,
-                 uint8_t* __restrict__ dst, const unsigned long long* __restrict__ wire_bytes) {
-    const TileDesc td = load_tile_desc(tiles + blockIdx.x);
-    const uint64_t used = wire_bytes[td.unit];
+constexpr int kCopyThreads = 256;
+constexpr int kCopyUnroll = 8;
+
+__global__ void __launch_bounds__(kCopyThreads)
+transport_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t sm_bytes_per_value,
+                 const uint8_t* __restrict__ src, uint8_t* __restrict__ dst,
+                 const unsigned long long* __restrict__ wire_bytes) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t warps_per_block = kCopyThreads / 32;
+    const uint32_t W = gridDim.x * warps_per_block;
+    const uint32_t t_first = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
     const uint64_t chunk = transport_chunk_bytes(sm_bytes_per_value);
-    const uint64_t lo = (uint64_t)td.tile_in_unit * chunk;
-    if (lo >= used) return;
-    const uint64_t hi = min(lo + chunk, used);
-    const uint8_t* s = src + td.msg_off + lo;
-    uint8_t* d = dst + td.msg_off + lo;
-    const uint32_t nvec = (uint32_t)((hi - lo) >> 4);
-    for (uint32_t i = threadIdx.x; i < nvec; i += kThreads) st_stream16(d + 16ull * i, ld_stream16(s + 16ull * i));
-    const uint32_t tail = (uint32_t)((hi - lo) & 15ull);
-    if (threadIdx.x < tail) d[16ull * nvec + threadIdx.x] = s[16ull * nvec + threadIdx.x];
+
+    // descriptors two tiles ahead, reported lengths one tile ahead
+    TileDesc td_a, td_b;
+    unsigned long long used_a = 0;
+    if (t_first < n_tiles) {
+        td_a = load_tile_desc(tiles + t_first);
+        used_a = __ldg(wire_bytes + td_a.unit);
+    }
+    if (t_first + W < n_tiles) td_b = load_tile_desc(tiles + t_first + W);
+    for (uint32_t t = t_first; t < n_tiles; t += W) {
+        const TileDesc td = td_a;
+        const uint64_t used = used_a;
+        td_a = td_b;
+        if (t + W < n_tiles) used_a = __ldg(wire_bytes + td_a.unit);
+        if (t + 2ull * W < n_tiles) td_b = load_tile_desc(tiles + t + 2u * W);
+
+        const uint64_t lo = (uint64_t)td.tile_in_unit * chunk;
+        if (lo >= used) continue;
+        const uint64_t hi = lo + chunk < used ? lo + chunk : used;
+        const uint8_t* s = src + td.msg_off + lo;
+        uint8_t* d = dst + td.msg_off + lo;
+        const uint32_t nvec = (uint32_t)((hi - lo) >> 4);  // 16-byte pieces
+        uint32_t i = lane;
+        for (; i + 32u * (kCopyUnroll - 1) < nvec; i += 32u * kCopyUnroll) {
+            uint4 v[kCopyUnroll];
+#pragma unroll
+            for (int u = 0; u < kCopyUnroll; ++u) v[u] = ld_stream16(s + 16ull * (i + 32u * u));
+#pragma unroll
+            for (int u = 0; u < kCopyUnroll; ++u) st_stream16(d + 16ull * (i + 32u * u), v[u]);
+        }
+        for (; i < nvec; i += 32u) st_stream16(d + 16ull * i, ld_stream16(s + 16ull * i));
+        // a ragged end (fewer than 16 bytes; only the last tile of a message can have one)
+        const uint32_t tail = (uint32_t)((hi - lo) & 15ull);
+        if (lane < tail) d[16ull * nvec + lane] = s[16ull * nvec + lane];
+    }
+}
+
+static int transport_grid_limit(int* out) {
+    static int cached[64] = {0};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    if (dev < 0 || dev >= 64) return CIERA_ERR_UNSUPPORTED;
+    if (cached[dev] == 0) {
+        int per_sm = 0, sms = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, transport_kernel, kCopyThreads, 0);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        if (per_sm < 1 || sms < 1) return CIERA_ERR_UNSUPPORTED;
+        cached[dev] = per_sm * sms;
+    }
+    *out = cached[dev];
+    return CIERA_OK;
 }
 
 }  // namespace ciera
@@ -96,15 +154,21 @@ extern "C" int ciera_cache_update(const ciera_plan* plan, void* cache_dev, const
 }
 
 extern "C" int ciera_transport(const ciera_plan* p, const void* src_messages_dev, void* dst_messages_dev,
-                               const uint64_t* wire_bytes_dev, void* stream) {
+                               const uint64_t* wire_bytes_dev, int32_t* status_dev, void* stream) {
     int rc = check_plan(p);
     if (rc) return rc;
     const uint32_t nt = (uint32_t)p->tiles.size();
     if (nt == 0) return CIERA_OK;
     if (!src_messages_dev || !dst_messages_dev || !wire_bytes_dev) return CIERA_ERR_INVALID_ARG;
     if (misaligned16(src_messages_dev) || misaligned16(dst_messages_dev)) return CIERA_ERR_MISALIGNED;
-    transport_kernel<<<nt, kThreads, 0, (cudaStream_t)stream>>>(
-        p->tiles_dev, p->dtype == CIERA_BF16 ? 1u : 3u, (const uint8_t*)src_messages_dev, (uint8_t*)dst_messages_dev,
+    int limit = 0;
+    rc = transport_grid_limit(&limit);
+    if (rc) return rc;
+    const uint32_t want = (nt + kCopyThreads / 32 - 1) / (kCopyThreads / 32);
+    const uint32_t grid = want < (uint32_t)limit ? want : (uint32_t)limit;
+    (void)status_dev;  // this kernel has no waits that could run out
+    transport_kernel<<<grid, kCopyThreads, 0, (cudaStream_t)stream>>>(
+        p->tiles_dev, nt, p->dtype == CIERA_BF16 ? 1u : 3u, (const uint8_t*)src_messages_dev, (uint8_t*)dst_messages_dev,
         (const unsigned long long*)wire_bytes_dev);
     count_launch();
     return check_launch();
@@ -123,7 +187,7 @@ extern "C" int ciera_roundtrip_host(const ciera_plan* p, const void* weights_hos
     rc = ciera_encode(p, b->weights_dev, b->sender_cache_dev, b->msg_send_dev, b->wire_bytes_dev, b->changed_blocks_dev,
                       b->workspace_dev, b->status_dev, stream);
     if (rc) return rc;
-    rc = ciera_transport(p, b->msg_send_dev, b->msg_recv_dev, b->wire_bytes_dev, stream);
+    rc = ciera_transport(p, b->msg_send_dev, b->msg_recv_dev, b->wire_bytes_dev, b->status_dev, stream);
     if (rc) return rc;
     rc = ciera_decode(p, b->msg_recv_dev, b->receiver_cache_dev, b->weights_out_dev, b->wire_bytes_dev,
                       b->workspace_dev, b->status_dev, stream);

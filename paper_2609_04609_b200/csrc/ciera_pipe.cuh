@@ -8,22 +8,6 @@
 
 #include "ciera_internal.cuh"
 
-#ifdef CIERA_PROF
-static __device__ unsigned long long g_prof[16];
-#define CIERA_PROF_READER(name) \
-    extern "C" __attribute__((visibility("default"))) int ciera_debug_prof_##name(unsigned long long* out, int reset) { \
-        if (reset) { unsigned long long z[16] = {0}; return (int)cudaMemcpyToSymbol(g_prof, z, sizeof(z)); } \
-        return (int)cudaMemcpyFromSymbol(out, g_prof, sizeof(unsigned long long) * 16); }
-#define PROF_T0 long long _t = clock64(); long long _p[10] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0}
-#define PROF_ADD(i) { long long _n = clock64(); _p[i] += _n - _t; _t = _n; }
-#define PROF_FLUSH { if (lane == 0) { _Pragma("unroll") for (int _i = 0; _i < 10; ++_i) if (_p[_i]) atomicAdd(&g_prof[_i], (unsigned long long)_p[_i]); } }
-#else
-#define PROF_T0
-#define PROF_ADD(i)
-#define PROF_FLUSH
-#define CIERA_PROF_READER(name)
-#endif
-
 namespace ciera {
 
 constexpr uint32_t kMaxBarrierPolls = 1u << 22;  // each poll may itself suspend for a short time slice
