@@ -35,10 +35,11 @@ METRIC = "encode/decode GB/s of weights"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic of one encode launch per value, from the ncu capture summarised under profiles/
-# (dram__bytes_read.sum + dram__bytes_write.sum of a smaller case, divided by its values); None
-# until a capture exists for the current kernel.
-NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE = None
+# DRAM traffic of one encode launch per value, from the ncu capture summarised in
+# profiles/ncu_full_one_layer_bf16.md: dram__bytes_read.sum + dram__bytes_write.sum of a one-layer
+# case (1.7526 GB) divided by its 402 653 184 values; traffic grows in proportion to the values of
+# a launch, and every launch of the bench workload is one such layer.  bf16, B = 512, q = 0.22 only.
+NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE = 4.353
 
 
 def parse_args():
@@ -371,21 +372,39 @@ def main():
     for c in layers:
         c.check_status()
 
+    # ---- the same K steps once more on ONE stream: kernels do not overlap, so the CUDA events
+    #      around each launch time that kernel alone (used for the roofline entries)
+    serial_timers = []
+    sev0, sev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sev0.record(s_enc)
+    for _ in range(args.steps):
+        run_step(layers, weights_of(step_i), s_enc, s_enc, events, "serial", serial_timers)
+        step_i += 1
+    sev1.record(s_enc)
+    barrier()
+    serial_ms_per_step = sev0.elapsed_time(sev1) / args.steps
+    for c in layers:
+        c.check_status()
+
     # ---- what was moved: change rates and the paper's byte count of the last step
     changed = sum(int(c.changed_blocks.sum().item()) for c in layers)
     blocks = sum(c.n_blocks() for c in layers)
     q = changed / blocks
     paper_bytes = sum(c.paper_bytes() for c in layers)
-    enc_ms = float(np.mean([t[0].elapsed_time(t[1]) for t in timers]))
-    tra_ms = float(np.mean([t[2].elapsed_time(t[3]) for t in timers]))
-    dec_ms = float(np.mean([t[4].elapsed_time(t[5]) for t in timers]))
+    ovl_ms = [float(np.mean([t[2 * i].elapsed_time(t[2 * i + 1]) for t in timers])) for i in range(3)]
+    enc_ms, tra_ms, dec_ms = [float(np.mean([t[2 * i].elapsed_time(t[2 * i + 1]) for t in serial_timers]))
+                              for i in range(3)]
     n_layer = layers[0].plan.total_values
     a_enc, a_tra, a_dec = algorithmic_bytes(n_layer, q, args.dtype)
     enc_gbs = a_enc / (enc_ms * 1e-3) / 1e9
+    dec_gbs = a_dec / (dec_ms * 1e-3) / 1e9
+    tra_gbs = a_tra / (tra_ms * 1e-3) / 1e9
+    path_gbs = len(layers) * (a_enc + a_tra + a_dec) / (ms_per_step * 1e-3) / 1e9
 
     # ---- correctness at full size: exact round trip everywhere, oracle on sampled units
     last_w = weights_of(step_i - 1)
-    prev_w = weights_of(step_i)
+    prev_w = weights_of(step_i)  # the iterate before the last one (the steps alternate)
     verified = all(torch.equal(c.weights_out[: w.numel()], w) for c, w in zip(layers, last_w))
     verified = verified and all(torch.equal(c.sender_cache, c.receiver_cache) for c in layers)
     sampled = 0
@@ -433,14 +452,25 @@ def main():
         "bytes_ratio": paper_bytes / weight_bytes,
         "encode_GBps_of_weights": n_layer * vb / (enc_ms * 1e-3) / 1e9,
         "decode_GBps_of_weights": n_layer * vb / (dec_ms * 1e-3) / 1e9,
-        "transport_GBps": a_tra / (tra_ms * 1e-3) / 1e9,
-        "decode_hbm_GBps": a_dec / (dec_ms * 1e-3) / 1e9,
-        "kernel_ms": {"encode": enc_ms, "transport": tra_ms, "decode": dec_ms, "per": "layer launch, timed region"},
+        "kernel_ms": {"encode": enc_ms, "transport": tra_ms, "decode": dec_ms,
+                      "per": "layer launch; serial re-run of the timed steps on one stream"},
+        "kernel_ms_overlapped": {"encode": ovl_ms[0], "transport": ovl_ms[1], "decode": ovl_ms[2],
+                                 "per": "layer launch inside the two-stream timed region (kernels overlap)"},
+        "serial_ms_per_step": serial_ms_per_step,
         "roofline": {
             "bound": "hbm", "kernel": "encode_kernel", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
             "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBps": enc_gbs / NOMINAL_HBM_GBS,
-            "traffic": (NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE * n_layer if NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE else None),
+            "traffic": (NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE * n_layer
+                        if args.dtype == "bf16" and args.block == 512 and args.update == "clustered" else None),
             "algorithmic_bytes_per_launch": a_enc,
+            "timed": "CUDA events around every encode launch, same K steps re-run on one stream so that "
+                     "no other kernel overlaps it",
+        },
+        "roofline_other": {
+            "decode_kernel": {"achieved": dec_gbs, "frac": dec_gbs / peak, "algorithmic_bytes_per_launch": a_dec},
+            "transport_kernel": {"achieved": tra_gbs, "frac": tra_gbs / peak, "algorithmic_bytes_per_launch": a_tra},
+            "whole_step_pipelined": {"achieved": path_gbs, "frac": path_gbs / peak,
+                                     "note": "algorithmic bytes of all three kernels over the two-stream step time"},
         },
     }
 
