@@ -71,6 +71,31 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+# --------------------------------------------------------------------------------- ranks
+
+
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """Slowest rank's time: every rank gets the maximum (needs an initialised process group when world > 1)."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbps(world: int, bytes_per_rank: int, ms_per_step: float) -> float:
+    """Weak scaling: every rank processes its own stack; the job's throughput is the sum."""
+    return world * bytes_per_rank / (ms_per_step * 1e-3) / 1e9
+
+
+def rank_seed(rank: int) -> int:
+    """Seed base of a rank's synthetic stack (config id 3; ranks get different weights)."""
+    return 1234 + 3 + 1000 * rank
+
+
 # --------------------------------------------------------------------------------- clocks
 
 
@@ -322,7 +347,7 @@ def main():
 
     peak, peak_kind = measured_peak()
     vb = wl.VALUE_BYTES[args.dtype]
-    layers, wa, wb = build_stack(args, device, seed_base=1234 + 3 + 1000 * rank)
+    layers, wa, wb = build_stack(args, device, seed_base=rank_seed(rank))
     n_values = sum(c.plan.total_values for c in layers)
     weight_bytes = n_values * vb
     s_enc, s_dec = torch.cuda.Stream(), torch.cuda.Stream()
@@ -363,11 +388,7 @@ def main():
     barrier()
     clocks = sampler.stop()
     launches = ciera.kernel_launch_count() - launches0
-    ms_total = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([ms_total], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1), world, device)
     ms_per_step = ms_total / args.steps
     for c in layers:
         c.check_status()
@@ -432,7 +453,7 @@ def main():
 
     out = {
         "metric": METRIC,
-        "value": world * weight_bytes / (ms_per_step * 1e-3) / 1e9,
+        "value": whole_job_gbps(world, weight_bytes, ms_per_step),
         "unit": "GB/s",
         "n_gpus": world,
         "steps": args.steps,
@@ -588,14 +609,10 @@ def e2e(args, layers, wa, wb, world, rank, barrier):
         cur.wait_stream(s)
     t1.record(cur)
     barrier()
-    ms = t0.elapsed_time(t1) / steps
-    if world > 1:
-        t = torch.tensor([ms], device=wa[0].device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(t0.elapsed_time(t1) / steps, world, wa[0].device)
     ok = all(torch.equal(o, (host_b if (steps - 1) % 2 == 0 else host_a)[l]) for l, o in enumerate(host_out))
     nbytes = sum(h.numel() for h in host_a)
-    return {"value": world * nbytes / (ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms, "steps": steps,
+    return {"value": whole_job_gbps(world, nbytes, ms), "unit": "GB/s", "ms_per_step": ms, "steps": steps,
             "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes + 8 * sum(len(c.units) for c in layers),
             "bit_exact": bool(ok), "api": "ciera_roundtrip_host (pinned host weights in, host weights out)"}
 
