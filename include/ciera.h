@@ -68,7 +68,8 @@ typedef enum ciera_status {
     CIERA_ERR_CUDA = -5,        /* a CUDA runtime call failed (see ciera_last_cuda_error)       */
     CIERA_ERR_TIMEOUT = -6,     /* device: a bounded wait on another tile ran out               */
     CIERA_ERR_CORRUPT = -7,     /* device: message length disagrees with its bitmap             */
-    CIERA_ERR_NOT_BOUND = -8    /* the plan has no device image yet (ciera_plan_bind)           */
+    CIERA_ERR_NOT_BOUND = -8,   /* the plan has no device image yet (ciera_plan_bind)           */
+    CIERA_ERR_TOO_LARGE = -9    /* more tiles than the built-in scratch of ciera_encode_noalloc */
 } ciera_status;
 
 typedef enum ciera_dtype {
@@ -157,6 +158,37 @@ CIERA_API int ciera_cache_update(const ciera_plan* plan, void* cache_dev, const 
 CIERA_API int ciera_encode(const ciera_plan* plan, const void* weights_dev, void* sender_cache_dev, void* messages_dev,
                  uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* workspace_dev,
                  int32_t* status_dev, void* stream);
+
+/* ---- sender, for callers that cannot supply scratch ---------------------------------------- */
+
+/* Largest plan ciera_encode_noalloc accepts: 65 536 tiles (ciera_plan_n_tiles), i.e. at most
+ * 536 870 912 values per call.  The library keeps 8 bytes per tile = 512 KiB of device memory for it
+ * on every GPU that loads the library, from load until the process exits. */
+#define CIERA_NOALLOC_MAX_TILES 65536u
+
+/*
+ * (This entry point has no counterpart in the paper; it is a convenience of this library.)
+ *
+ * Same work and same outputs as ciera_encode, but without the `workspace_dev` argument: the
+ * look-back scratch is a fixed array inside the library.  It is meant for callers that can pass the
+ * buffers they already own but cannot obtain a fresh device allocation when they call -- a training
+ * runtime whose memory pool already holds the whole GPU, a parameter-gather hook that must not
+ * stall the device (allocating does), a plug-in that was handed pointers but no allocator.  The
+ * call itself allocates nothing, on the host or on the device.
+ *
+ *   - Plans with more than CIERA_NOALLOC_MAX_TILES tiles are refused with CIERA_ERR_TOO_LARGE before
+ *     any device work is enqueued; split the unit table, or use ciera_encode with your own scratch.
+ *   - The first call on each device looks up the array's device address (a CUDA runtime query made
+ *     with that device current).  Make that first call outside of any stream capture.
+ *   - All calls on a device share the one array, which keeps whatever the last call left in it; every
+ *     call therefore clears the part it uses, on `stream`, before its kernel.  Two calls that can
+ *     run on the GPU at the same time (different streams, no ordering between them) race on the
+ *     array and produce garbage: order them, or give all but one of them ciera_encode with scratch
+ *     of its own.
+ */
+CIERA_API int ciera_encode_noalloc(const ciera_plan* plan, const void* weights_dev, void* sender_cache_dev,
+                         void* messages_dev, uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev,
+                         int32_t* status_dev, void* stream);
 
 /* ---- transport stand-in: Send / Recv of Algorithm 1 on one GPU ----------------------------- */
 

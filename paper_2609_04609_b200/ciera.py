@@ -28,6 +28,8 @@ ERR_CUDA = -5
 ERR_TIMEOUT = -6
 ERR_CORRUPT = -7
 ERR_NOT_BOUND = -8
+ERR_TOO_LARGE = -9
+NOALLOC_MAX_TILES = 65536
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libciera.so")
 if not os.path.exists(_LIB_PATH):
@@ -68,6 +70,7 @@ _SIGS = {
     "ciera_cache_init": ([_vp, _vp, _vp, _vp], _i32),
     "ciera_cache_update": ([_vp, _vp, _vp, _vp], _i32),
     "ciera_encode": ([_vp] * 9, _i32),
+    "ciera_encode_noalloc": ([_vp] * 8, _i32),
     "ciera_transport": ([_vp] * 6, _i32),
     "ciera_decode": ([_vp] * 8, _i32),
     "ciera_roundtrip_host": ([_vp, _vp, _sz, _vp, _vp, _vp, _vp], _i32),
@@ -201,6 +204,16 @@ def encode(plan: Plan, weights, sender_cache, messages, wire_bytes, changed_bloc
     _check("ciera_encode",
            _lib.ciera_encode(plan.handle, _ptr(weights), _ptr(sender_cache), _ptr(messages), _ptr(wire_bytes),
                              _ptr(changed_blocks), _ptr(workspace), _ptr(status), _stream(stream)))
+
+
+def encode_noalloc(plan: Plan, weights, sender_cache, messages, wire_bytes, changed_blocks, status=None,
+                   stream=None) -> None:
+    """``ciera_encode`` without a scratch argument: for callers that can pass the buffers they own
+    but cannot allocate one more (see ciera.h).  At most NOALLOC_MAX_TILES tiles per call; calls
+    that may overlap on the GPU must not both use it."""
+    _check("ciera_encode_noalloc",
+           _lib.ciera_encode_noalloc(plan.handle, _ptr(weights), _ptr(sender_cache), _ptr(messages), _ptr(wire_bytes),
+                                     _ptr(changed_blocks), _ptr(status), _stream(stream)))
 
 
 def transport(plan: Plan, src_messages, dst_messages, wire_bytes, status=None, stream=None) -> None:

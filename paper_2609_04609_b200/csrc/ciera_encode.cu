@@ -563,3 +563,78 @@ extern "C" int ciera_encode(const ciera_plan* p, const void* weights_dev, void* 
     return launch_encode<CIERA_FP32>(p, grid, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
                                      changed_blocks_dev, workspace_dev, status_dev, s);
 }
+
+// ------------------------------------------------------------------------------------------
+// Encode for callers that have no scratch buffer to give.
+//
+// Some callers hand this library only the buffers they already own -- parameter shards, caches,
+// communication buffers -- and cannot come up with one more device allocation at the moment of the
+// call: a training runtime whose memory pool has claimed the whole GPU (a fresh allocation would
+// fail or fragment the pool), a gather hook that must not synchronise the device (allocating
+// does), a plug-in that was given pointers but no allocator.  For them the look-back scratch of
+// the encode kernel lives in the library itself: a fixed array in device memory that every GPU
+// loading the library holds from load until the process exits.
+
+static __device__ __align__(256) unsigned long long g_encode_scratch[CIERA_NOALLOC_MAX_TILES];
+
+// Device address of g_encode_scratch on the current device.  In host code the array's name is only
+// a handle for the runtime, not an address a kernel could use, so the address is looked up once
+// per device (with that device current) and kept.
+static int encode_scratch_address(unsigned long long** out) {
+    static std::atomic<unsigned long long*> cached[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    if (dev < 0 || dev >= 64) return CIERA_ERR_UNSUPPORTED;
+    unsigned long long* ptr = cached[dev].load(std::memory_order_acquire);
+    if (ptr == nullptr) {
+        void* q = nullptr;
+        e = cudaGetSymbolAddress(&q, g_encode_scratch);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        if (q == nullptr) return CIERA_ERR_CUDA;
+        ptr = static_cast<unsigned long long*>(q);
+        cached[dev].store(ptr, std::memory_order_release);
+    }
+    *out = ptr;
+    return CIERA_OK;
+}
+
+extern "C" int ciera_encode_noalloc(const ciera_plan* p, const void* weights_dev, void* sender_cache_dev,
+                                    void* messages_dev, uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev,
+                                    int32_t* status_dev, void* stream) {
+    if (!p) return CIERA_ERR_INVALID_ARG;
+    if (!p->tiles.empty() && !p->tiles_dev) return CIERA_ERR_NOT_BOUND;
+    const uint32_t nt = (uint32_t)p->tiles.size();
+    if (nt > CIERA_NOALLOC_MAX_TILES) return CIERA_ERR_TOO_LARGE;
+    if (p->n_units == 0) return CIERA_OK;
+    if (!wire_bytes_dev || !changed_blocks_dev) return CIERA_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e;
+    if (p->has_empty_units) {  // units without tiles: their outputs are written here
+        e = cudaMemsetAsync(wire_bytes_dev, 0, sizeof(uint64_t) * p->n_units, s);
+        if (e != cudaSuccess) return record_cuda_error(e);
+        e = cudaMemsetAsync(changed_blocks_dev, 0, sizeof(uint32_t) * p->n_units, s);
+        if (e != cudaSuccess) return record_cuda_error(e);
+    }
+    if (nt == 0) return CIERA_OK;
+    if (!weights_dev || !sender_cache_dev || !messages_dev) return CIERA_ERR_INVALID_ARG;
+    if (misaligned16(weights_dev) || misaligned16(sender_cache_dev) || misaligned16(messages_dev) ||
+        ((uintptr_t)wire_bytes_dev & 7u) || ((uintptr_t)changed_blocks_dev & 3u))
+        return CIERA_ERR_MISALIGNED;
+    unsigned long long* scratch = nullptr;
+    int rc = encode_scratch_address(&scratch);
+    if (rc) return rc;
+    int limit = 0;
+    rc = p->dtype == CIERA_BF16 ? encode_grid_limit<CIERA_BF16>(&limit) : encode_grid_limit<CIERA_FP32>(&limit);
+    if (rc) return rc;
+    const uint32_t grid = nt < (uint32_t)limit ? nt : (uint32_t)limit;
+    // the array keeps what the previous call left in it: the status words of this call's tiles
+    // have to start at zero
+    e = cudaMemsetAsync(scratch, 0, sizeof(unsigned long long) * nt, s);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    if (p->dtype == CIERA_BF16)
+        return launch_encode<CIERA_BF16>(p, grid, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
+                                         changed_blocks_dev, scratch, status_dev, s);
+    return launch_encode<CIERA_FP32>(p, grid, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
+                                     changed_blocks_dev, scratch, status_dev, s);
+}

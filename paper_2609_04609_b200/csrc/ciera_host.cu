@@ -203,6 +203,7 @@ extern "C" const char* ciera_status_string(int s) {
         case CIERA_ERR_TIMEOUT: return "device wait ran out";
         case CIERA_ERR_CORRUPT: return "message length contradicts its bitmap";
         case CIERA_ERR_NOT_BOUND: return "plan not bound to device memory";
+        case CIERA_ERR_TOO_LARGE: return "plan has more tiles than the built-in scratch of ciera_encode_noalloc holds";
         default: return "unknown status";
     }
 }
