@@ -209,9 +209,10 @@ CIERA_API int ciera_transport(const ciera_plan* plan, const void* src_messages_d
  *   wire_bytes_dev      in   optional (may be NULL): lengths as reported by the sender; a unit
  *                            whose bitmap implies a different length raises CIERA_ERR_CORRUPT in
  *                            status_dev (its output is then unspecified)
- *   workspace_dev       scratch of ciera_plan_workspace_bytes(), 16-byte aligned.  Only used (by a
- *                            small prefix kernel that runs first) when some unit has more than 4096
- *                            blocks; may be NULL otherwise.  Not shared by overlapping calls.
+ *   workspace_dev       scratch of ciera_plan_workspace_bytes(), 16-byte aligned: the counter tiles
+ *                            are handed out from (cleared by the call itself) and, when some unit has
+ *                            more than 4096 blocks, the per-tile counts of a small prefix kernel that
+ *                            runs first.  Must not be shared by calls that can overlap on the GPU.
  */
 CIERA_API int ciera_decode(const ciera_plan* plan, const void* messages_dev, void* receiver_cache_dev,
                  void* weights_out_dev, const uint64_t* wire_bytes_dev, void* workspace_dev, int32_t* status_dev,

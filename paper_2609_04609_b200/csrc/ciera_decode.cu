@@ -1,7 +1,9 @@
 // Receiver side (paper Algorithm 1, receiver part; Section 3.1) as one persistent sm_100a kernel.
 //
-// Grid = at most as many thread blocks as fit on the GPU; block c works on tiles c, c + G, ...
-// Tiles are independent here, so no block ever waits for another.  Two roles:
+// Grid = at most as many thread blocks as fit on the GPU.  Tiles are independent here, so they
+// are handed out dynamically: every producer warp draws the next tile number from a counter in
+// the caller's scratch, which keeps all SMs busy to the end whatever their individual pace.
+// Two roles:
 //
 //   producer warps  run ahead, taking the block's tiles in turn: for each tile a producer reads
 //                   the tile's bits of the unit's bitmap and the number of changed blocks before
@@ -28,6 +30,7 @@ constexpr int kDecProducers = 2;                               // producer warps
 constexpr int kDecodeThreads = kThreads + 32 * kDecProducers;  // consumers + producers
 constexpr int kDecProducerWarp0 = kWarps;
 constexpr int kDecRing = 12;  // > stages + 2 * producers + 1: slots are refilled only after their tile is done
+constexpr uint32_t kNoTile = 0xffffffffu;
 constexpr uint32_t kDirectWordsPerLane = 4;
 constexpr uint32_t kDirectBlocks = kDecodeDirectBlocks;
 static_assert(kDirectBlocks == 32u * 32u * kDirectWordsPerLane, "one fetch covers the direct range");
@@ -56,7 +59,7 @@ struct __align__(16) DecodeRing {
     const uint8_t* sm_src;                   // the tile's received sign-plus-mantissa
     const uint8_t* pay_src;                  // the payload slice holding the tile's changed blocks
     uint32_t nv;                             // values in the tile
-    uint32_t pad;
+    uint32_t tile;                           // the tile's number, or kNoTile: this producer has no more work
     uint32_t bm[kBitmapWords];               // the tile's block flags
     uint32_t pre[kBitmapWords];              // set flags before each word
     // raw material, fetched asynchronously one tile ahead:
@@ -178,11 +181,12 @@ template <int DT>
 __global__ void __launch_bounds__(kDecodeThreads, DecodeCfg<DT>::kBlocksPerSM)
 decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log2b, const uint8_t* msgs, uint8_t* cache,
               uint8_t* __restrict__ weights, const unsigned long long* __restrict__ wire_bytes,
-              const uint32_t* __restrict__ ws_prefix, int32_t* status) {
+              const uint32_t* __restrict__ ws_prefix, unsigned int* ticket, int32_t* status) {
     using P = Piece<DT>;
     constexpr int VB = Traits<DT>::kValueBytes;
     constexpr int SMB = Traits<DT>::kSmBytes;
     constexpr int S = DecodeCfg<DT>::kStages;
+    static_assert(S % kDecProducers == 0, "every producer cycles through stages of its own");
     constexpr bool kStageOut = DecodeCfg<DT>::kStageOut;
     constexpr uint32_t kSmTile = kTileValues * SMB;                   // sign-plus-mantissa of a tile
     constexpr uint32_t kStageBytes = kSmTile + 2u * kTileValues;       // + cache span + payload slice
@@ -193,8 +197,6 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
     DecodeCtl<S>* ctl = reinterpret_cast<DecodeCtl<S>*>(s_out + kOutBytes);
 
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
-    const uint32_t G = gridDim.x;
-    const uint32_t my_tiles = blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + G - 1u) / G : 0u;
     volatile int* abort = &ctl->abort;
 
     if (tid == 0) {
@@ -211,104 +213,125 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
 
     if (warp >= kDecProducerWarp0) {
         // ---------------------------------------------------------------- producers (all lanes)
-        // producer p handles this block's tiles p, p + P, p + 2P, ... (jj below counts them)
+        // producer p fills the slots p, p + P, p + 2P, ... of the block's sequence (jj counts them),
+        // each with the tile whose number it draws from the counter
         const uint32_t pidx = warp - kDecProducerWarp0;
-        const uint32_t my_prod = my_tiles > pidx ? (my_tiles - pidx + kDecProducers - 1u) / kDecProducers : 0u;
-        if (my_prod > 0) {
-            // software pipeline through the ring: descriptor two tiles ahead, bitmap words one tile
-            // ahead, both by per-thread asynchronous copies (groups D_j and B_j, committed in the
-            // order D_0 D_1 B_0 | D_2 B_1 | D_3 B_2 | ...)
-            auto seq = [&](uint32_t jj) { return pidx + jj * kDecProducers; };  // place in the block's sequence
-            auto fetch_desc = [&](uint32_t jj) {
-                if (jj < my_prod && lane < 3)
-                    cp_async16(reinterpret_cast<uint8_t*>(&ctl->ring[seq(jj) % kDecRing].desc) + 16u * lane,
-                               reinterpret_cast<const uint8_t*>(tiles + blockIdx.x + (uint64_t)seq(jj) * G) + 16u * lane);
-                cp_async_commit();
-            };
-            fetch_desc(0);
-            fetch_desc(1);
-            cp_async_wait<1>();  // D_0
-            __syncwarp();
-            fetch_bitmap(ctl->ring[seq(0) % kDecRing].desc, blockIdx.x + seq(0) * G, log2b, msgs, ws_prefix,
-                         &ctl->ring[seq(0) % kDecRing], lane);
+        auto seq = [&](uint32_t jj) { return pidx + jj * kDecProducers; };  // place in the block's sequence
+        auto draw = [&]() {
+            uint32_t t = 0;
+            if (lane == 0) t = atomicAdd(ticket, 1u);
+            t = __shfl_sync(0xffffffffu, t, 0);
+            return t < n_tiles ? t : kNoTile;
+        };
+        // software pipeline through the ring: tile number and descriptor two slots ahead, bitmap
+        // words one slot ahead, both by per-thread asynchronous copies (groups D_j and B_j, committed
+        // in the order D_0 D_1 B_0 | D_2 B_1 | D_3 B_2 | ...)
+        auto fetch_desc = [&](uint32_t jj, uint32_t tile) {
+            DecodeRing* r = &ctl->ring[seq(jj) % kDecRing];
+            if (lane == 0) r->tile = tile;
+            if (tile != kNoTile && lane < 3)
+                cp_async16(reinterpret_cast<uint8_t*>(&r->desc) + 16u * lane,
+                           reinterpret_cast<const uint8_t*>(tiles + tile) + 16u * lane);
             cp_async_commit();
-            for (uint32_t jj = 0; jj < my_prod; ++jj) {
-                const uint32_t k = seq(jj);
-                fetch_desc(jj + 2u);
-                cp_async_wait<1>();  // everything but D_{jj+2}: D_{jj+1} and B_jj have landed
-                __syncwarp();
-                if (jj + 1u < my_prod) {
-                    DecodeRing* rn = &ctl->ring[seq(jj + 1u) % kDecRing];
-                    fetch_bitmap(rn->desc, blockIdx.x + seq(jj + 1u) * G, log2b, msgs, ws_prefix, rn, lane);
-                }
-                cp_async_commit();
-
-                const uint32_t stage = k % S;
-                bool ok = true;
-                if (k >= (uint32_t)S) ok = mbar_wait(&ctl->empty[stage], ((k / S) & 1u) ^ 1u, abort, status);
-                if (!__all_sync(0xffffffffu, ok)) break;
-
-                DecodeRing* r = &ctl->ring[k % kDecRing];
-                const TileDesc td = r->desc;
-                uint32_t own = 0;
-                const uint64_t before = digest_bitmap(r, td, log2b, lane, own);
-                const uint64_t N = td.n_unit;
-                const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
-                const uint64_t smoff = sm_offset(N, log2b);
-                const uint64_t payoff = smoff + pad16(N * SMB);
-                const uint8_t* msg = msgs + td.msg_off;
-                const uint8_t* pay = msg + payoff + (before << log2b);  // this tile's slice of the payload
-                uint8_t* st = smem + (size_t)stage * kStageBytes;
-                const bool full_tile = N - v0 >= (uint64_t)kTileValues;
-                uint32_t lo = 1, hi = 0;
-                if (full_tile) unchanged_span(r->bm, log2b, lane, lo, hi);
-
-                if (lane == 0) {
-                    r->w_dst = weights + td.w_off;
-                    r->c_ptr = cache + td.c_off;
-                    r->sm_src = msg + smoff + v0 * SMB;
-                    r->pay_src = pay;
-                    r->nv = (uint32_t)min((uint64_t)kTileValues, N - v0);
-
-                    // integrity check by the unit's last tile: the bitmap fixes the message length
-                    if (wire_bytes != nullptr && status != nullptr && td.tile_in_unit == td.n_tiles_unit - 1u) {
-                        const uint32_t B = 1u << log2b;
-                        const uint32_t nv = (uint32_t)(N - v0);
-                        uint64_t total = (before + own) << log2b;
-                        const uint32_t rem = nv & (B - 1u);
-                        if (rem) {
-                            const uint32_t kb = nv >> log2b;
-                            if ((r->bm[kb >> 5] >> (kb & 31u)) & 1u) total -= (B - rem);
-                        }
-                        if (wire_bytes[td.unit] != payoff + total) atomicCAS(status, 0, (int32_t)CIERA_ERR_CORRUPT);
-                    }
-
-                    if (full_tile) {
-                        const uint32_t span = lo <= hi ? (hi - lo + 1u) << log2b : 0u;
-                        const uint32_t slice = own << log2b;
-                        mbar_arrive_expect_tx(&ctl->full[stage], kSmTile + span + slice);
-                        bulk_load(st, r->sm_src, kSmTile, &ctl->full[stage]);
-                        if (span)
-                            bulk_load(st + kSmTile + ((size_t)lo << log2b), r->c_ptr + ((size_t)lo << log2b), span,
-                                      &ctl->full[stage]);
-                        if (slice) bulk_load(st + kSmTile + kTileValues, pay, slice, &ctl->full[stage]);
-                    } else {
-                        mbar_arrive(&ctl->full[stage]);  // short tile: consumers read global memory themselves
-                    }
-                    atomicMax(&ctl->issued, k + 1u);
-                }
-                __syncwarp();
+        };
+        uint32_t t_cur = draw(), t_nxt = draw();
+        fetch_desc(0, t_cur);
+        fetch_desc(1, t_nxt);
+        cp_async_wait<1>();  // D_0
+        __syncwarp();
+        if (t_cur != kNoTile)
+            fetch_bitmap(ctl->ring[seq(0) % kDecRing].desc, t_cur, log2b, msgs, ws_prefix, &ctl->ring[seq(0) % kDecRing], lane);
+        cp_async_commit();
+        for (uint32_t jj = 0;; ++jj) {
+            const uint32_t k = seq(jj);
+            const uint32_t stage = k % S;
+            // make sure the slot two ahead is free before refilling it: its previous tile is done once
+            // the stage of slot k is free (slots are used in order, the ring is longer than that)
+            bool ok = true;
+            if (k >= (uint32_t)S) ok = mbar_wait(&ctl->empty[stage], ((k / S) & 1u) ^ 1u, abort, status);
+            if (!__all_sync(0xffffffffu, ok)) break;
+            if (t_cur == kNoTile) {  // no work left: tell the consumers and stop
+                if (lane == 0) mbar_arrive(&ctl->full[stage]);
+                break;
             }
-            cp_async_wait<0>();
+            const uint32_t t_nn = t_nxt != kNoTile ? draw() : kNoTile;
+            fetch_desc(jj + 2u, t_nn);
+            cp_async_wait<1>();  // everything but D_{jj+2}: D_{jj+1} and B_jj have landed
+            __syncwarp();
+            if (t_nxt != kNoTile) {
+                DecodeRing* rn = &ctl->ring[seq(jj + 1u) % kDecRing];
+                fetch_bitmap(rn->desc, t_nxt, log2b, msgs, ws_prefix, rn, lane);
+            }
+            cp_async_commit();
+
+            DecodeRing* r = &ctl->ring[k % kDecRing];
+            const TileDesc td = r->desc;
+            uint32_t own = 0;
+            const uint64_t before = digest_bitmap(r, td, log2b, lane, own);
+            const uint64_t N = td.n_unit;
+            const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
+            const uint64_t smoff = sm_offset(N, log2b);
+            const uint64_t payoff = smoff + pad16(N * SMB);
+            const uint8_t* msg = msgs + td.msg_off;
+            const uint8_t* pay = msg + payoff + (before << log2b);  // this tile's slice of the payload
+            uint8_t* st = smem + (size_t)stage * kStageBytes;
+            const bool full_tile = N - v0 >= (uint64_t)kTileValues;
+            uint32_t lo = 1, hi = 0;
+            if (full_tile) unchanged_span(r->bm, log2b, lane, lo, hi);
+
+            if (lane == 0) {
+                r->w_dst = weights + td.w_off;
+                r->c_ptr = cache + td.c_off;
+                r->sm_src = msg + smoff + v0 * SMB;
+                r->pay_src = pay;
+                r->nv = (uint32_t)min((uint64_t)kTileValues, N - v0);
+
+                // integrity check by the unit's last tile: the bitmap fixes the message length
+                if (wire_bytes != nullptr && status != nullptr && td.tile_in_unit == td.n_tiles_unit - 1u) {
+                    const uint32_t B = 1u << log2b;
+                    const uint32_t nv = (uint32_t)(N - v0);
+                    uint64_t total = (before + own) << log2b;
+                    const uint32_t rem = nv & (B - 1u);
+                    if (rem) {
+                        const uint32_t kb = nv >> log2b;
+                        if ((r->bm[kb >> 5] >> (kb & 31u)) & 1u) total -= (B - rem);
+                    }
+                    if (wire_bytes[td.unit] != payoff + total) atomicCAS(status, 0, (int32_t)CIERA_ERR_CORRUPT);
+                }
+
+                if (full_tile) {
+                    const uint32_t span = lo <= hi ? (hi - lo + 1u) << log2b : 0u;
+                    const uint32_t slice = own << log2b;
+                    mbar_arrive_expect_tx(&ctl->full[stage], kSmTile + span + slice);
+                    bulk_load(st, r->sm_src, kSmTile, &ctl->full[stage]);
+                    if (span)
+                        bulk_load(st + kSmTile + ((size_t)lo << log2b), r->c_ptr + ((size_t)lo << log2b), span,
+                                  &ctl->full[stage]);
+                    if (slice) bulk_load(st + kSmTile + kTileValues, pay, slice, &ctl->full[stage]);
+                } else {
+                    mbar_arrive(&ctl->full[stage]);  // short tile: consumers read global memory themselves
+                }
+                atomicMax(&ctl->issued, k + 1u);
+            }
+            __syncwarp();
+            t_cur = t_nxt;
+            t_nxt = t_nn;
         }
+        cp_async_wait<0>();
     } else {
         // ---------------------------------------------------------------- consumers
         const uint32_t bmask = (1u << log2b) - 1u;
-        for (uint32_t k = 0; k < my_tiles; ++k) {
+        uint32_t live = (1u << kDecProducers) - 1u;  // producers that have not sent their end marker
+        for (uint32_t k = 0; live != 0; ++k) {
+            if (!((live >> (k % kDecProducers)) & 1u)) continue;  // that producer's slots are over
             const uint32_t stage = k % S;
             if (!mbar_wait(&ctl->full[stage], (k / S) & 1u, abort, status)) break;
             if (tid == 0) ctl->seen = k + 1;
             const DecodeRing* r = &ctl->ring[k % kDecRing];
+            if (r->tile == kNoTile) {
+                live &= ~(1u << (k % kDecProducers));
+                continue;
+            }
             const uint32_t nv = r->nv;
             const uint8_t* const st = smem + (size_t)stage * kStageBytes;
             uint8_t* const c_ptr = r->c_ptr;
@@ -489,14 +512,18 @@ extern "C" int ciera_decode(const ciera_plan* p, const void* messages_dev, void*
     if (!p->tiles.empty() && !p->tiles_dev) return CIERA_ERR_NOT_BOUND;
     const uint32_t nt = (uint32_t)p->tiles.size();
     if (nt == 0) return CIERA_OK;
-    if (!messages_dev || !receiver_cache_dev || !weights_out_dev) return CIERA_ERR_INVALID_ARG;
+    if (!messages_dev || !receiver_cache_dev || !weights_out_dev || !workspace_dev) return CIERA_ERR_INVALID_ARG;
     if (misaligned16(messages_dev) || misaligned16(receiver_cache_dev) || misaligned16(weights_out_dev) ||
         misaligned16(workspace_dev))
         return CIERA_ERR_MISALIGNED;
     cudaStream_t s = (cudaStream_t)stream;
+    // scratch = per-tile counts for long units (4 bytes per tile), then, past 8 bytes per tile, the
+    // tile counter, which starts at zero
+    unsigned int* ticket = (unsigned int*)((unsigned long long*)workspace_dev + nt);
+    cudaError_t me = cudaMemsetAsync(ticket, 0, 16, s);
+    if (me != cudaSuccess) return record_cuda_error(me);
     const uint32_t n_long = (uint32_t)p->long_units.size();
     if (n_long) {
-        if (!workspace_dev) return CIERA_ERR_INVALID_ARG;
         decode_prefix_kernel<<<n_long, 256, 0, s>>>(p->tiles_dev, p->long_units_dev, p->log2b,
                                                     (const uint8_t*)messages_dev, (uint32_t*)workspace_dev);
         count_launch();
@@ -510,12 +537,12 @@ extern "C" int ciera_decode(const ciera_plan* p, const void* messages_dev, void*
     if (p->dtype == CIERA_BF16)
         decode_kernel<CIERA_BF16><<<grid, kDecodeThreads, decode_smem_bytes<CIERA_BF16>(), s>>>(
             p->tiles_dev, nt, p->log2b, (const uint8_t*)messages_dev, (uint8_t*)receiver_cache_dev,
-            (uint8_t*)weights_out_dev, (const unsigned long long*)wire_bytes_dev, (const uint32_t*)workspace_dev,
+            (uint8_t*)weights_out_dev, (const unsigned long long*)wire_bytes_dev, (const uint32_t*)workspace_dev, ticket,
             status_dev);
     else
         decode_kernel<CIERA_FP32><<<grid, kDecodeThreads, decode_smem_bytes<CIERA_FP32>(), s>>>(
             p->tiles_dev, nt, p->log2b, (const uint8_t*)messages_dev, (uint8_t*)receiver_cache_dev,
-            (uint8_t*)weights_out_dev, (const unsigned long long*)wire_bytes_dev, (const uint32_t*)workspace_dev,
+            (uint8_t*)weights_out_dev, (const unsigned long long*)wire_bytes_dev, (const uint32_t*)workspace_dev, ticket,
             status_dev);
     count_launch();
     return check_launch();

@@ -1,8 +1,13 @@
 // Sender side (paper Algorithm 1, sender part; Section 3.1) as one persistent sm_100a kernel.
 //
-// Grid = G thread blocks that are all resident at once (cooperative launch); block c works on
-// tiles c, c + G, c + 2G, ... of the plan's tile table, so neighbouring tiles of a unit are worked
-// on by neighbouring blocks at about the same time and the look-back below rarely waits long.
+// Grid = G thread blocks that are all resident at once (cooperative launch).  The plan lists the
+// tiles of short units (up to 32 tiles) first.  A block first works through whole short units, tile
+// after tile -- units c, c + G, ... of that list, as long as a full round of G units is left -- so
+// that a tile's place in its unit's payload is a running sum inside the block and nothing waits
+// for another block.  All remaining tiles (the last, partial round of short units and every longer
+// unit) are spread tile by tile over the blocks, block c taking tiles T0 + c, T0 + c + G, ...:
+// neighbouring tiles of a unit are then worked on by neighbouring blocks at about the same time,
+// and their payload offsets come from a single-pass look-back over per-tile status words.
 // A thread block has four roles:
 //
 //   producer warp   runs ahead of the others: for each of its tiles it fetches the tile
@@ -14,10 +19,12 @@
 //   warps           bytes and sign-plus-mantissa, compare with the cached exponents, vote (ballot)
 //                   the "my piece changed" bit, store sign-plus-mantissa to the message and leave
 //                   the new exponents where the cached ones were staged;
-//   aggregator warp turns the vote bits of a tile into block flags (the unit's bitmap), counts the
-//                   tile's payload bytes and publishes them as the tile's status word;
-//   resolver warps  resolve the tile's exclusive offset in the unit's payload with a single-pass
-//                   look-back over the status words.
+//   aggregator warp turns the vote bits of a tile into block flags (the unit's bitmap) and counts
+//                   the tile's payload bytes; for a tile of a unit that this block works through
+//                   alone it also keeps the running offset, otherwise it publishes the count as
+//                   the tile's status word;
+//   resolver warps  (spread tiles only) resolve the tile's exclusive offset in the unit's payload
+//                   with a single-pass look-back over the status words.
 // A few tiles later, when that offset is known, the consumers send the exponents of changed
 // blocks from shared memory to the payload and to the cache and hand the stage back.
 //
@@ -74,14 +81,56 @@ struct EncodeCtl {
     TileDesc desc[kDescRing];
     EncodeTileInfo info[kDescRing];
     uint32_t tile_idx[kDescRing];  // table index of the tile in desc[]
+    uint32_t seq[kDescRing];       // 1: tile of a unit this block works through alone
     uint32_t ballot[SE][kVoteWords];
     uint32_t bm[SE][kBitmapWords];
     uint32_t pre[SE][kBitmapWords];
     unsigned long long agg[SE];
     unsigned long long base[SE];
     int abort;
-    uint32_t issued;  // tiles whose loads have been started (producer)
-    uint32_t seen;    // tiles whose loads the consumers have seen complete
+    uint32_t issued;    // tiles whose loads have been started (producer)
+    uint32_t seen;      // tiles whose loads the consumers have seen complete
+    uint32_t my_tiles;  // tiles of this block
+};
+
+// The sequence of tiles of one thread block (see the head of this file).
+struct TileWalk {
+    const uint32_t* seq_first;
+    uint32_t n_tiles, G, c, R, T0;
+    uint32_t r, tile, end;  // walking state
+    bool spread;
+
+    __device__ TileWalk(const uint32_t* sf, uint32_t n_short, uint32_t nt, uint32_t grid, uint32_t block)
+        : seq_first(sf), n_tiles(nt), G(grid), c(block), R(n_short / grid), r(0), tile(0), end(0), spread(false) {
+        T0 = __ldg(sf + (size_t)R * G);
+    }
+    // number of tiles of the block
+    __device__ uint32_t count() const {
+        uint32_t n = 0;
+        for (uint32_t i = 0; i < R; ++i) n += __ldg(seq_first + (size_t)i * G + c + 1) - __ldg(seq_first + (size_t)i * G + c);
+        if (T0 + c < n_tiles) n += (n_tiles - T0 - c + G - 1u) / G;
+        return n;
+    }
+    // next tile; `seq` tells whether it belongs to a unit the block works through alone
+    __device__ uint32_t next(bool& seq) {
+        if (!spread) {
+            while (tile == end && r < R) {
+                tile = __ldg(seq_first + (size_t)r * G + c);
+                end = __ldg(seq_first + (size_t)r * G + c + 1);
+                ++r;
+            }
+            if (tile != end) {
+                seq = true;
+                return tile++;
+            }
+            spread = true;
+            tile = T0 + c;
+        }
+        seq = false;
+        const uint32_t t = tile;
+        tile += G;
+        return t;
+    }
 };
 
 __device__ __forceinline__ unsigned long long ld_status(const unsigned long long* p) {
@@ -151,11 +200,11 @@ __device__ __forceinline__ uint32_t build_block_bitmap(const uint32_t* ballot, u
     return run;
 }
 
-// Aggregator warp, one tile: block flags, the tile's bitmap bytes, the tile's payload byte count,
-// published at once as the tile's status word so that later tiles never wait for it longer than
-// for the votes themselves.  Waits for nothing outside the thread block.
+// Aggregator warp, one tile: block flags, the tile's bitmap bytes, the tile's payload byte count.
+// With `publish` the count goes out at once as the tile's status word, so that later tiles never
+// wait for it longer than for the votes themselves.  Waits for nothing outside the thread block.
 template <int DT>
-__device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t tile, uint32_t log2b,
+__device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t tile, uint32_t log2b, bool publish,
                                                    const uint32_t* ballot, uint32_t* bm, uint32_t* pre, uint8_t* msgs,
                                                    unsigned long long* tile_status, uint32_t lane) {
     const uint64_t N = td.n_unit;
@@ -174,11 +223,12 @@ __device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t 
         const uint32_t kb = nv >> log2b;
         if ((bm[kb >> 5] >> (kb & 31u)) & 1u) agg -= (B - rem);
     }
-    // a unit's first tile knows its prefix (0) already
-    const uint32_t mybits = nbt < 8 ? bm[0] : 0u;
-    const unsigned long long flag = td.tile_in_unit == 0 ? kFlagPrefix : kFlagAggregate;
-    if (lane == 0) st_status(tile_status + tile, flag | ((unsigned long long)mybits << kBitsShift) | agg);
-
+    if (publish) {
+        // a unit's first tile knows its prefix (0) already
+        const uint32_t mybits = nbt < 8 ? bm[0] : 0u;
+        const unsigned long long flag = td.tile_in_unit == 0 ? kFlagPrefix : kFlagAggregate;
+        if (lane == 0) st_status(tile_status + tile, flag | ((unsigned long long)mybits << kBitsShift) | agg);
+    }
     // bitmap bytes of this tile (tiles of >= 8 blocks own whole bytes)
     if (nbt >= 8) {
         const uint64_t byte0 = (uint64_t)td.tile_in_unit * (nbt >> 3);
@@ -188,17 +238,32 @@ __device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t 
     return agg;
 }
 
-// Resolver warp, one tile: exclusive prefix of the payload bytes over the earlier tiles of the
-// same unit by a single-pass look-back over the status words, then the duties that need it.
+// The unit's last tile reports the totals and zeroes the two pads (one warp).
+template <int DT>
+__device__ __forceinline__ void finish_unit(const TileDesc& td, uint32_t log2b, uint64_t total, uint8_t* msgs,
+                                            unsigned long long* wire_bytes, uint32_t* changed_blocks, uint32_t lane) {
+    constexpr int SMB = Traits<DT>::kSmBytes;
+    const uint64_t N = td.n_unit;
+    const uint32_t B = 1u << log2b;
+    uint8_t* msg = msgs + td.msg_off;
+    const uint64_t smoff = sm_offset(N, log2b);
+    const uint64_t payoff = smoff + pad16(N * SMB);
+    if (lane == 0) {
+        wire_bytes[td.unit] = payoff + total;
+        changed_blocks[td.unit] = (uint32_t)((total + B - 1u) >> log2b);
+    }
+    for (uint64_t b = bitmap_bytes(N, log2b) + lane; b < smoff; b += 32) msg[b] = 0;
+    for (uint64_t b = smoff + N * SMB + lane; b < payoff; b += 32) msg[b] = 0;
+}
+
+// Resolver warp, one spread tile: exclusive prefix of the payload bytes over the earlier tiles of
+// the same unit by a single-pass look-back over the status words, then the duties that need it.
 // Returns the tile's exclusive payload offset inside its unit.
 template <int DT>
 __device__ __forceinline__ uint64_t resolve_tile(const TileDesc& td, uint32_t tile, uint32_t log2b, uint64_t agg,
                                                  const uint32_t* bm, uint8_t* msgs, unsigned long long* wire_bytes,
                                                  uint32_t* changed_blocks, unsigned long long* tile_status,
                                                  int32_t* status, uint32_t lane) {
-    constexpr int SMB = Traits<DT>::kSmBytes;
-    const uint64_t N = td.n_unit;
-    const uint32_t B = 1u << log2b;
     const uint32_t nbt = kTileValues >> log2b;
     uint8_t* msg = msgs + td.msg_off;
     const uint32_t mybits = nbt < 8 ? bm[0] : 0u;
@@ -237,19 +302,8 @@ __device__ __forceinline__ uint64_t resolve_tile(const TileDesc& td, uint32_t ti
             if (lane == 0) msg[td.tile_in_unit / tpb] = (uint8_t)(part | (mybits << (p * nbt)));
         }
     }
-
-    // the unit's last tile reports the totals and zeroes the two pads
-    if (td.tile_in_unit == td.n_tiles_unit - 1u) {
-        const uint64_t smoff = sm_offset(N, log2b);
-        const uint64_t payoff = smoff + pad16(N * SMB);
-        const uint64_t total = excl + agg;
-        if (lane == 0) {
-            wire_bytes[td.unit] = payoff + total;
-            changed_blocks[td.unit] = (uint32_t)((total + B - 1u) >> log2b);
-        }
-        for (uint64_t b = bitmap_bytes(N, log2b) + lane; b < smoff; b += 32) msg[b] = 0;
-        for (uint64_t b = smoff + N * SMB + lane; b < payoff; b += 32) msg[b] = 0;
-    }
+    if (td.tile_in_unit == td.n_tiles_unit - 1u)
+        finish_unit<DT>(td, log2b, excl + agg, msgs, wire_bytes, changed_blocks, lane);
     return excl;
 }
 
@@ -285,9 +339,10 @@ __device__ __forceinline__ void write_changed(const EncodeTileInfo& ti, uint32_t
 
 template <int DT>
 __global__ void __launch_bounds__(kEncodeThreads, 2)
-encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log2b, const uint8_t* __restrict__ weights,
-              uint8_t* cache, uint8_t* msgs, unsigned long long* wire_bytes, uint32_t* changed_blocks,
-              unsigned long long* tile_status, int32_t* status) {
+encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32_t* __restrict__ seq_first,
+              uint32_t n_short, uint32_t log2b, const uint8_t* __restrict__ weights, uint8_t* cache, uint8_t* msgs,
+              unsigned long long* wire_bytes, uint32_t* changed_blocks, unsigned long long* tile_status,
+              int32_t* status) {
     using P = Piece<DT>;
     constexpr int VB = Traits<DT>::kValueBytes;
     constexpr int SMB = Traits<DT>::kSmBytes;
@@ -301,9 +356,6 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
     EncodeCtl<SW, SE>* ctl = reinterpret_cast<EncodeCtl<SW, SE>*>(ring_e + (size_t)SE * kEBytes);
 
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
-    const uint32_t G = gridDim.x;
-    // tiles of this block: blockIdx.x + k * G for k < my_tiles
-    const uint32_t my_tiles = blockIdx.x < n_tiles ? (n_tiles - blockIdx.x + G - 1u) / G : 0u;
     volatile int* abort = &ctl->abort;
 
     if (tid == 0) {
@@ -321,23 +373,33 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
         ctl->abort = 0;
         ctl->issued = 0;
         ctl->seen = 0;
+        ctl->my_tiles = TileWalk(seq_first, n_short, n_tiles, gridDim.x, blockIdx.x).count();
         mbar_fence_init();
     }
     __syncthreads();
+    const uint32_t my_tiles = ctl->my_tiles;
 
     if (warp == kProducerWarp) {
         // ---------------------------------------------------------------- producer
         if (lane == 0 && my_tiles > 0) {
-            TileDesc nxt = load_tile_desc(tiles + blockIdx.x);  // descriptors are fetched one tile ahead
+            TileWalk walk(seq_first, n_short, n_tiles, gridDim.x, blockIdx.x);
+            bool seq_nxt = false;
+            uint32_t tile_nxt = walk.next(seq_nxt);
+            TileDesc nxt = load_tile_desc(tiles + tile_nxt);  // descriptors are fetched one tile ahead
             for (uint32_t k = 0; k < my_tiles; ++k) {
                 const TileDesc td = nxt;
-                const uint32_t tile = blockIdx.x + k * G;
-                if (k + 1u < my_tiles) nxt = load_tile_desc(tiles + tile + G);
+                const uint32_t tile = tile_nxt;
+                const bool seq = seq_nxt;
+                if (k + 1u < my_tiles) {
+                    tile_nxt = walk.next(seq_nxt);
+                    nxt = load_tile_desc(tiles + tile_nxt);
+                }
                 const uint32_t sw = k % SW, se = k % SE;
                 if (k >= (uint32_t)SW && !mbar_wait(&ctl->empty_w[sw], ((k / SW) & 1u) ^ 1u, abort, status)) break;
                 if (k >= (uint32_t)SE && !mbar_wait(&ctl->empty_e[se], ((k / SE) & 1u) ^ 1u, abort, status)) break;
                 ctl->desc[k % kDescRing] = td;
                 ctl->tile_idx[k % kDescRing] = tile;
+                ctl->seq[k % kDescRing] = seq ? 1u : 0u;
                 const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
                 const uint64_t left = td.n_unit - v0;
                 {
@@ -365,21 +427,43 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
         }
     } else if (warp == kAggregatorWarp) {
         // ---------------------------------------------------------------- aggregator
+        uint64_t run_incl = 0;  // payload bytes of the current alone-worked unit up to the last tile
+        uint32_t byte_acc = 0;  // its bitmap byte in the making (tiles of fewer than 8 blocks)
         for (uint32_t k = 0; k < my_tiles; ++k) {
             const uint32_t se = k % SE;
             if (!mbar_wait(&ctl->voted[se], (k / SE) & 1u, abort, status)) break;
             const TileDesc td = ctl->desc[k % kDescRing];
-            const uint64_t agg = aggregate_tile<DT>(td, ctl->tile_idx[k % kDescRing], log2b, ctl->ballot[se], ctl->bm[se],
-                                                    ctl->pre[se], msgs, tile_status, lane);
-            if (lane == 0) ctl->agg[se] = agg;
+            const bool seq = ctl->seq[k % kDescRing] != 0;
+            const uint64_t agg = aggregate_tile<DT>(td, ctl->tile_idx[k % kDescRing], log2b, !seq, ctl->ballot[se],
+                                                    ctl->bm[se], ctl->pre[se], msgs, tile_status, lane);
+            if (seq) {
+                // the whole unit is this block's: the tile's offset is the running sum
+                const uint64_t excl = td.tile_in_unit == 0 ? 0ull : run_incl;
+                run_incl = excl + agg;
+                const uint32_t nbt = kTileValues >> log2b;
+                const bool last = td.tile_in_unit == td.n_tiles_unit - 1u;
+                if (nbt < 8) {
+                    const uint32_t tpb = 8u / nbt, p = td.tile_in_unit & (tpb - 1u);
+                    byte_acc = (p == 0 ? 0u : byte_acc) | (ctl->bm[se][0] << (p * nbt));
+                    if ((p == tpb - 1u || last) && lane == 0) msgs[td.msg_off + td.tile_in_unit / tpb] = (uint8_t)byte_acc;
+                }
+                if (last) finish_unit<DT>(td, log2b, run_incl, msgs, wire_bytes, changed_blocks, lane);
+                if (lane == 0) ctl->base[se] = excl;
+            } else if (lane == 0) {
+                ctl->agg[se] = agg;
+            }
             __syncwarp();
-            if (lane == 0) mbar_arrive(&ctl->summed[se]);
+            if (lane == 0) {
+                mbar_arrive(&ctl->summed[se]);
+                if (seq) mbar_arrive(&ctl->resolved[se]);
+            }
         }
     } else if (warp >= kResolverWarp0) {
         // ---------------------------------------------------------------- resolvers (tiles k = i, i + R, ...)
         for (uint32_t k = warp - kResolverWarp0; k < my_tiles; k += kResolvers) {
             const uint32_t se = k % SE;
             if (!mbar_wait(&ctl->summed[se], (k / SE) & 1u, abort, status)) break;
+            if (ctl->seq[k % kDescRing] != 0) continue;  // the aggregator has done it all
             const TileDesc td = ctl->desc[k % kDescRing];
             const uint64_t excl = resolve_tile<DT>(td, ctl->tile_idx[k % kDescRing], log2b, ctl->agg[se], ctl->bm[se], msgs,
                                                    wire_bytes, changed_blocks, tile_status, status, lane);
@@ -507,13 +591,15 @@ static int launch_encode(const ciera_plan* p, uint32_t grid, const void* weights
                          int32_t* status_dev, cudaStream_t s) {
     const TileDesc* tiles = p->tiles_dev;
     uint32_t nt = (uint32_t)p->tiles.size();
+    const uint32_t* seq_first = p->seq_first_dev;
+    uint32_t n_short = (uint32_t)p->seq_first.size() - 1u;
     uint32_t log2b = p->log2b;
     const uint8_t* w = (const uint8_t*)weights_dev;
     uint8_t* c = (uint8_t*)sender_cache_dev;
     uint8_t* m = (uint8_t*)messages_dev;
     unsigned long long* wb = (unsigned long long*)wire_bytes_dev;
     unsigned long long* ts = (unsigned long long*)workspace_dev;
-    void* args[] = {&tiles, &nt, &log2b, &w, &c, &m, &wb, &changed_blocks_dev, &ts, &status_dev};
+    void* args[] = {&tiles, &nt, &seq_first, &n_short, &log2b, &w, &c, &m, &wb, &changed_blocks_dev, &ts, &status_dev};
     // cooperative launch: the runtime starts the grid only when all of its blocks fit on the GPU
     // together, which is what the look-back between blocks relies on
     cudaError_t e = cudaLaunchCooperativeKernel((const void*)encode_kernel<DT>, dim3(grid), dim3(kEncodeThreads), args,

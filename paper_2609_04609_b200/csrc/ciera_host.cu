@@ -1,6 +1,7 @@
 // Host side of libciera: size rules, the plan (tile table), the gain rule, diagnostics.
 #include <string.h>
 
+#include <algorithm>
 #include <new>
 
 #include "ciera_internal.cuh"
@@ -94,10 +95,19 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
     p->units.assign(units_host, units_host + n_units);
     p->tiles.reserve((size_t)n_tiles);
     const uint32_t vb = value_bytes_of(dtype);
+    // processing order: short units by descending tile count (ties in table order), then the rest
+    auto tiles_of = [&](uint32_t u) { return (uint32_t)((units_host[u].n_values + kTileValues - 1) / kTileValues); };
+    std::vector<uint32_t> shorts, longs;
     for (uint32_t u = 0; u < n_units; ++u) {
+        const uint32_t nt = tiles_of(u);
+        if (nt == 0) continue;
+        (nt <= kSeqMaxTiles ? shorts : longs).push_back(u);
+    }
+    std::stable_sort(shorts.begin(), shorts.end(), [&](uint32_t a, uint32_t b) { return tiles_of(a) > tiles_of(b); });
+    auto emit = [&](uint32_t u) {
         const ciera_unit& un = units_host[u];
-        uint32_t nt = (uint32_t)((un.n_values + kTileValues - 1) / kTileValues);
-        uint32_t first = (uint32_t)p->tiles.size();
+        const uint32_t nt = tiles_of(u);
+        const uint32_t first = (uint32_t)p->tiles.size();
         for (uint32_t j = 0; j < nt; ++j) {
             TileDesc t;
             t.w_off = un.weights_off + (uint64_t)j * kTileValues * vb;
@@ -110,13 +120,22 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
             t.n_tiles_unit = nt;
             p->tiles.push_back(t);
         }
-        if (nt && (un.n_values + block - 1) / block > kDecodeDirectBlocks) p->long_units.push_back(first);
+        if ((un.n_values + block - 1) / block > kDecodeDirectBlocks) p->long_units.push_back(first);
+    };
+    for (uint32_t u : shorts) {
+        p->seq_first.push_back((uint32_t)p->tiles.size());
+        emit(u);
     }
-    // device image: the tile table, then (16-byte aligned) the list of long units
+    p->seq_first.push_back((uint32_t)p->tiles.size());
+    for (uint32_t u : longs) emit(u);
+    // device image: the tile table, then (16-byte aligned) the two index lists
     const size_t tb = p->tiles.size() * sizeof(TileDesc);
-    p->image.assign(tb + p->long_units.size() * sizeof(uint32_t) + 16, 0);
+    const size_t lb = (p->long_units.size() * sizeof(uint32_t) + 15) / 16 * 16;
+    const size_t sb = p->seq_first.size() * sizeof(uint32_t);
+    p->image.assign(tb + lb + sb + 16, 0);
     if (tb) memcpy(p->image.data(), p->tiles.data(), tb);
     if (!p->long_units.empty()) memcpy(p->image.data() + tb, p->long_units.data(), p->long_units.size() * 4);
+    memcpy(p->image.data() + tb + lb, p->seq_first.data(), sb);
     *plan_out = p;
     return CIERA_OK;
 }
@@ -148,7 +167,10 @@ extern "C" int ciera_plan_bind(ciera_plan* p, void* plan_dev, size_t plan_dev_by
     e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return record_cuda_error(e);
     p->tiles_dev = (const TileDesc*)plan_dev;
-    p->long_units_dev = (const uint32_t*)((const uint8_t*)plan_dev + p->tiles.size() * sizeof(TileDesc));
+    const size_t tb = p->tiles.size() * sizeof(TileDesc);
+    const size_t lb = (p->long_units.size() * sizeof(uint32_t) + 15) / 16 * 16;
+    p->long_units_dev = (const uint32_t*)((const uint8_t*)plan_dev + tb);
+    p->seq_first_dev = (const uint32_t*)((const uint8_t*)plan_dev + tb + lb);
     return CIERA_OK;
 }
 

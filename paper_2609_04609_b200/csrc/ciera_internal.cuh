@@ -74,6 +74,12 @@ __host__ __device__ inline uint64_t payload_offset(uint64_t n, uint32_t sm_bytes
 // prefix kernel at decode time; shorter ones read them straight from the bitmap.
 constexpr uint32_t kDecodeDirectBlocks = 4096;
 
+// The tile table lists the tiles of "short" units (up to this many tiles) first, longest units
+// first, then the tiles of the longer units.  The encode kernel lets one thread block work through
+// a short unit tile after tile (the tile's place in the payload is then a running sum inside the
+// block) and spreads everything else tile by tile over all blocks.
+constexpr uint32_t kSeqMaxTiles = 32;
+
 // Bytes of a message slot that one tile moves in the transport kernel: slot capacity <= tiles * this.
 __host__ __device__ inline uint64_t transport_chunk_bytes(uint32_t sm_bytes_per_value) {
     return (uint64_t)kTileValues * (sm_bytes_per_value + 1) + 96;
@@ -92,9 +98,11 @@ struct ciera_plan {
     std::vector<ciera_unit> units;
     std::vector<ciera::TileDesc> tiles;
     std::vector<uint32_t> long_units;  // first tile of every unit whose decode needs the prefix kernel
-    std::vector<uint8_t> image;        // device image: tiles, then long_units
+    std::vector<uint32_t> seq_first;   // first tile of every short unit, in table order, + end marker
+    std::vector<uint8_t> image;        // device image: tiles, then long_units, then seq_first
     const ciera::TileDesc* tiles_dev = nullptr;
     const uint32_t* long_units_dev = nullptr;
+    const uint32_t* seq_first_dev = nullptr;
 };
 
 namespace ciera {

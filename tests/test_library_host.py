@@ -77,21 +77,26 @@ def test_plan_validation(ciera):
 
 
 def test_plan_tile_table(ciera):
+    """Every unit is cut into tiles of 8192 values; the table lists short units (<= 32 tiles) first, longest
+    first and otherwise in table order, then the longer units; empty units have no tiles."""
     T = 8192
-    sizes = [0, 5, T, T + 1, 3 * T + 17, 0, 40000]
+    sizes = [0, 5, T, T + 1, 3 * T + 17, 0, 40000, 40 * T + 3, 33 * T]
     units, wb, cb, mb = layout_units(sizes, 1, 4, lambda n: ciera.message_capacity(n, 1, 64))
     p = ciera.Plan(units, 1, 64)
-    want_tiles = sum(-(-n // T) for n in sizes)
+    ntiles = [-(-n // T) for n in sizes]
+    want_tiles = sum(ntiles)
     assert (p.n_units, p.n_tiles, p.tile_values, p.total_values) == (len(sizes), want_tiles, T, sum(sizes))
     assert p.workspace_bytes >= 8 * want_tiles and p.device_bytes >= 48 * want_tiles
-    img = p.host_image()[: 48 * want_tiles].view(np.dtype([("w", "<u8"), ("c", "<u8"), ("m", "<u8"), ("n", "<u8"), ("unit", "<u4"),
-                                        ("j", "<u4"), ("first", "<u4"), ("nt", "<u4")]))
+    img = p.host_image()[: 48 * want_tiles].view(np.dtype([("w", "<u8"), ("c", "<u8"), ("m", "<u8"), ("n", "<u8"),
+                                                          ("unit", "<u4"), ("j", "<u4"), ("first", "<u4"), ("nt", "<u4")]))
+    short = sorted([u for u in range(len(sizes)) if 1 <= ntiles[u] <= 32], key=lambda u: -ntiles[u])
+    long_ = [u for u in range(len(sizes)) if ntiles[u] > 32]
     k = 0
-    for ui, u in enumerate(units):
-        nt = -(-int(u["n_values"]) // T)
-        for j in range(nt):
+    for ui in short + long_:
+        u = units[ui]
+        for j in range(ntiles[ui]):
             t = img[k]
-            assert (t["unit"], t["j"], t["first"], t["nt"], t["n"]) == (ui, j, k - j, nt, u["n_values"])
+            assert (t["unit"], t["j"], t["first"], t["nt"], t["n"]) == (ui, j, k - j, ntiles[ui], u["n_values"])
             assert t["w"] == u["weights_off"] + j * T * 4 and t["c"] == u["cache_off"] + j * T
             assert t["m"] == u["msg_off"]
             k += 1
