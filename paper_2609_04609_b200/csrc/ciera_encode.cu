@@ -1,13 +1,14 @@
 // Sender side (paper Algorithm 1, sender part; Section 3.1) as one persistent sm_100a kernel.
 //
-// Grid = G thread blocks that are all resident at once (cooperative launch).  The plan lists the
-// tiles of short units (up to 32 tiles) first.  A block first works through whole short units, tile
-// after tile -- units c, c + G, ... of that list, as long as a full round of G units is left -- so
-// that a tile's place in its unit's payload is a running sum inside the block and nothing waits
-// for another block.  All remaining tiles (the last, partial round of short units and every longer
-// unit) are spread tile by tile over the blocks, block c taking tiles T0 + c, T0 + c + G, ...:
-// neighbouring tiles of a unit are then worked on by neighbouring blocks at about the same time,
-// and their payload offsets come from a single-pass look-back over per-tile status words.
+// Grid = G persistent thread blocks.  The plan lists the tiles of short units (up to 32 tiles)
+// first.  A block first takes its share of the tiles of the longer units, spread tile by tile over
+// the blocks (block c takes tiles T0 + c, T0 + c + G, ...; neighbouring tiles of a unit are then
+// worked on by neighbouring blocks at about the same time, and their payload offsets come from a
+// single-pass look-back over per-tile status words; this part needs all blocks resident, so a
+// plan with longer units is launched cooperatively).  Then it works through whole short units,
+// tile after tile, drawing the next unit's number from a counter in the scratch: a tile's place in
+// its unit's payload is then a running sum inside the block, nothing waits for another block, and
+// all SMs stay busy to the end whatever their individual pace.
 // A thread block has four roles:
 //
 //   producer warp   runs ahead of the others: for each of its tiles it fetches the tile
@@ -80,7 +81,7 @@ struct EncodeCtl {
     uint64_t empty_e[SE];   // all 16 consumer warps have sent the tile's changed exponents
     TileDesc desc[kDescRing];
     EncodeTileInfo info[kDescRing];
-    uint32_t tile_idx[kDescRing];  // table index of the tile in desc[]
+    uint32_t tile_idx[kDescRing];  // table index of the tile in desc[]; kNoTile = end marker
     uint32_t seq[kDescRing];       // 1: tile of a unit this block works through alone
     uint32_t ballot[SE][kVoteWords];
     uint32_t bm[SE][kBitmapWords];
@@ -88,48 +89,47 @@ struct EncodeCtl {
     unsigned long long agg[SE];
     unsigned long long base[SE];
     int abort;
-    uint32_t issued;    // tiles whose loads have been started (producer)
-    uint32_t seen;      // tiles whose loads the consumers have seen complete
-    uint32_t my_tiles;  // tiles of this block
+    uint32_t issued;  // tiles whose loads have been started (producer)
+    uint32_t seen;    // tiles whose loads the consumers have seen complete
 };
 
-// The sequence of tiles of one thread block (see the head of this file).
+constexpr uint32_t kNoTile = 0xffffffffu;
+
+// The sequence of tiles of one thread block (see the head of this file); used by the producer.
 struct TileWalk {
     const uint32_t* seq_first;
-    uint32_t n_tiles, G, c, R, T0;
-    uint32_t r, tile, end;  // walking state
+    unsigned int* unit_ticket;
+    uint32_t n_tiles, n_short, G;
+    uint32_t tile, end;      // current short unit: next tile, one past its last tile
+    uint32_t next_unit;      // the unit drawn ahead (its number arrives while the current one is worked on)
+    uint32_t spread_tile;    // next spread tile of this block
     bool spread;
 
-    __device__ TileWalk(const uint32_t* sf, uint32_t n_short, uint32_t nt, uint32_t grid, uint32_t block)
-        : seq_first(sf), n_tiles(nt), G(grid), c(block), R(n_short / grid), r(0), tile(0), end(0), spread(false) {
-        T0 = __ldg(sf + (size_t)R * G);
+    __device__ TileWalk(const uint32_t* sf, unsigned int* ticket, uint32_t nshort, uint32_t nt, uint32_t grid, uint32_t block)
+        : seq_first(sf), unit_ticket(ticket), n_tiles(nt), n_short(nshort), G(grid), tile(0), end(0), spread(true) {
+        spread_tile = __ldg(sf + nshort) + block;  // tiles of longer units start after the short units' tiles
+        next_unit = nshort ? atomicAdd(ticket, 1u) : kNoTile;
     }
-    // number of tiles of the block
-    __device__ uint32_t count() const {
-        uint32_t n = 0;
-        for (uint32_t i = 0; i < R; ++i) n += __ldg(seq_first + (size_t)i * G + c + 1) - __ldg(seq_first + (size_t)i * G + c);
-        if (T0 + c < n_tiles) n += (n_tiles - T0 - c + G - 1u) / G;
-        return n;
-    }
-    // next tile; `seq` tells whether it belongs to a unit the block works through alone
+    // next tile, or kNoTile; `seq` tells whether it belongs to a unit the block works through alone
     __device__ uint32_t next(bool& seq) {
-        if (!spread) {
-            while (tile == end && r < R) {
-                tile = __ldg(seq_first + (size_t)r * G + c);
-                end = __ldg(seq_first + (size_t)r * G + c + 1);
-                ++r;
+        if (spread) {
+            if (spread_tile < n_tiles) {
+                seq = false;
+                const uint32_t t = spread_tile;
+                spread_tile += G;
+                return t;
             }
-            if (tile != end) {
-                seq = true;
-                return tile++;
-            }
-            spread = true;
-            tile = T0 + c;
+            spread = false;
         }
-        seq = false;
-        const uint32_t t = tile;
-        tile += G;
-        return t;
+        seq = true;
+        while (tile == end) {
+            const uint32_t u = next_unit;
+            if (u >= n_short) return kNoTile;
+            next_unit = atomicAdd(unit_ticket, 1u);
+            tile = __ldg(seq_first + u);
+            end = __ldg(seq_first + u + 1);
+        }
+        return tile++;
     }
 };
 
@@ -342,7 +342,7 @@ __global__ void __launch_bounds__(kEncodeThreads, 2)
 encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32_t* __restrict__ seq_first,
               uint32_t n_short, uint32_t log2b, const uint8_t* __restrict__ weights, uint8_t* cache, uint8_t* msgs,
               unsigned long long* wire_bytes, uint32_t* changed_blocks, unsigned long long* tile_status,
-              int32_t* status) {
+              unsigned int* unit_ticket, int32_t* status) {
     using P = Piece<DT>;
     constexpr int VB = Traits<DT>::kValueBytes;
     constexpr int SMB = Traits<DT>::kSmBytes;
@@ -373,32 +373,41 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
         ctl->abort = 0;
         ctl->issued = 0;
         ctl->seen = 0;
-        ctl->my_tiles = TileWalk(seq_first, n_short, n_tiles, gridDim.x, blockIdx.x).count();
         mbar_fence_init();
     }
     __syncthreads();
-    const uint32_t my_tiles = ctl->my_tiles;
 
+    // The block's tiles form a sequence k = 0, 1, 2, ... that only the producer knows in advance;
+    // it closes the sequence with kResolvers end markers (one for each resolver warp), which the
+    // other roles pass on to each other through the same barriers as real tiles.
     if (warp == kProducerWarp) {
         // ---------------------------------------------------------------- producer
-        if (lane == 0 && my_tiles > 0) {
-            TileWalk walk(seq_first, n_short, n_tiles, gridDim.x, blockIdx.x);
+        if (lane == 0) {
+            TileWalk walk(seq_first, unit_ticket, n_short, n_tiles, gridDim.x, blockIdx.x);
             bool seq_nxt = false;
             uint32_t tile_nxt = walk.next(seq_nxt);
-            TileDesc nxt = load_tile_desc(tiles + tile_nxt);  // descriptors are fetched one tile ahead
-            for (uint32_t k = 0; k < my_tiles; ++k) {
+            TileDesc nxt;
+            if (tile_nxt != kNoTile) nxt = load_tile_desc(tiles + tile_nxt);  // descriptors are fetched one tile ahead
+            uint32_t markers = 0;
+            for (uint32_t k = 0;; ++k) {
                 const TileDesc td = nxt;
                 const uint32_t tile = tile_nxt;
                 const bool seq = seq_nxt;
-                if (k + 1u < my_tiles) {
+                if (tile != kNoTile) {
                     tile_nxt = walk.next(seq_nxt);
-                    nxt = load_tile_desc(tiles + tile_nxt);
+                    if (tile_nxt != kNoTile) nxt = load_tile_desc(tiles + tile_nxt);
                 }
                 const uint32_t sw = k % SW, se = k % SE;
                 if (k >= (uint32_t)SW && !mbar_wait(&ctl->empty_w[sw], ((k / SW) & 1u) ^ 1u, abort, status)) break;
                 if (k >= (uint32_t)SE && !mbar_wait(&ctl->empty_e[se], ((k / SE) & 1u) ^ 1u, abort, status)) break;
-                ctl->desc[k % kDescRing] = td;
                 ctl->tile_idx[k % kDescRing] = tile;
+                if (tile == kNoTile) {  // end marker
+                    mbar_arrive(&ctl->full_w[sw]);
+                    mbar_arrive(&ctl->full_e[se]);
+                    if (++markers == (uint32_t)kResolvers) break;
+                    continue;
+                }
+                ctl->desc[k % kDescRing] = td;
                 ctl->seq[k % kDescRing] = seq ? 1u : 0u;
                 const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
                 const uint64_t left = td.n_unit - v0;
@@ -429,13 +438,20 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
         // ---------------------------------------------------------------- aggregator
         uint64_t run_incl = 0;  // payload bytes of the current alone-worked unit up to the last tile
         uint32_t byte_acc = 0;  // its bitmap byte in the making (tiles of fewer than 8 blocks)
-        for (uint32_t k = 0; k < my_tiles; ++k) {
+        uint32_t markers = 0;
+        for (uint32_t k = 0;; ++k) {
             const uint32_t se = k % SE;
             if (!mbar_wait(&ctl->voted[se], (k / SE) & 1u, abort, status)) break;
+            const uint32_t tile = ctl->tile_idx[k % kDescRing];
+            if (tile == kNoTile) {  // pass the end marker on to the resolver in charge of slot k
+                if (lane == 0) mbar_arrive(&ctl->summed[se]);
+                if (++markers == (uint32_t)kResolvers) break;
+                continue;
+            }
             const TileDesc td = ctl->desc[k % kDescRing];
             const bool seq = ctl->seq[k % kDescRing] != 0;
-            const uint64_t agg = aggregate_tile<DT>(td, ctl->tile_idx[k % kDescRing], log2b, !seq, ctl->ballot[se],
-                                                    ctl->bm[se], ctl->pre[se], msgs, tile_status, lane);
+            const uint64_t agg = aggregate_tile<DT>(td, tile, log2b, !seq, ctl->ballot[se], ctl->bm[se], ctl->pre[se], msgs,
+                                                    tile_status, lane);
             if (seq) {
                 // the whole unit is this block's: the tile's offset is the running sum
                 const uint64_t excl = td.tile_in_unit == 0 ? 0ull : run_incl;
@@ -459,14 +475,16 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
             }
         }
     } else if (warp >= kResolverWarp0) {
-        // ---------------------------------------------------------------- resolvers (tiles k = i, i + R, ...)
-        for (uint32_t k = warp - kResolverWarp0; k < my_tiles; k += kResolvers) {
+        // ---------------------------------------------------------------- resolvers (slots k = i, i + R, ...)
+        for (uint32_t k = warp - kResolverWarp0;; k += kResolvers) {
             const uint32_t se = k % SE;
             if (!mbar_wait(&ctl->summed[se], (k / SE) & 1u, abort, status)) break;
+            const uint32_t tile = ctl->tile_idx[k % kDescRing];
+            if (tile == kNoTile) break;
             if (ctl->seq[k % kDescRing] != 0) continue;  // the aggregator has done it all
             const TileDesc td = ctl->desc[k % kDescRing];
-            const uint64_t excl = resolve_tile<DT>(td, ctl->tile_idx[k % kDescRing], log2b, ctl->agg[se], ctl->bm[se], msgs,
-                                                   wire_bytes, changed_blocks, tile_status, status, lane);
+            const uint64_t excl = resolve_tile<DT>(td, tile, log2b, ctl->agg[se], ctl->bm[se], msgs, wire_bytes,
+                                                   changed_blocks, tile_status, status, lane);
             if (lane == 0) {
                 ctl->base[se] = excl;
                 mbar_arrive(&ctl->resolved[se]);
@@ -474,53 +492,65 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
         }
     } else {
         // ---------------------------------------------------------------- consumers
-        for (uint32_t k = 0; k < my_tiles; ++k) {
+        uint32_t k_end = kNoTile;  // slot of the first end marker, once seen
+        uint32_t k = 0;
+        for (;; ++k) {
             const uint32_t sw = k % SW, se = k % SE;
             if (!mbar_wait(&ctl->full_w[sw], (k / SW) & 1u, abort, status)) break;
             if (!mbar_wait(&ctl->full_e[se], (k / SE) & 1u, abort, status)) break;
             if (tid == 0) ctl->seen = k + 1;
-            const EncodeTileInfo ti = ctl->info[k % kDescRing];
-            const uint32_t nv = ti.nv;
-            const uint8_t* const s_w = ring_w + (size_t)sw * kWBytes;
-            uint8_t* const s_e = ring_e + (size_t)se * kEBytes;
-
-#pragma unroll
-            for (int p = 0; p < P::kPerThread; ++p) {
-                const uint32_t t0 = P::start(tid, p);
-                const int nvalid = piece_valid<DT>(t0, nv);
-                // (exp, mant) <- SplitExpMant, and the cached exponents of the same values
-                P x, c;
-                if (nv == (uint32_t)kTileValues) {
-                    x.template split_full<Shared>(s_w + (size_t)t0 * VB);
-                    c.template load_exp_full<Shared>(s_e + t0);
-                } else if (nvalid == P::kValues) {
-                    x.template split_full<Global>(ti.w_src + (size_t)t0 * VB);
-                    c.template load_exp_full<Global>(ti.c_ptr + t0);
-                } else {
-                    // values past the end of the unit read as exponent 0 against a cached 0: never "changed"
-                    x.split_partial(ti.w_src + (size_t)t0 * VB, nvalid);
-                    c.load_exp_partial(ti.c_ptr + t0, nvalid);
+            const bool marker = ctl->tile_idx[k % kDescRing] == kNoTile;
+            if (marker) {
+                if (k_end == kNoTile) k_end = k;
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(&ctl->voted[se]);  // pass the end marker on to the aggregator
+                    mbar_arrive(&ctl->empty_w[sw]);  // and hand the marker's (unused) stages back
+                    mbar_arrive(&ctl->empty_e[se]);
                 }
-                // leave the new exponents where the cached ones were staged: they are sent from
-                // there once the tile's place in the payload is known
-                x.template store_exp_full<Shared>(s_e + t0);
-                const uint32_t bal = __ballot_sync(0xffffffffu, x.differs(c));
-                if (lane == 0) ctl->ballot[se][p * kWarps + warp] = bal;
-                // sign-plus-mantissa of every value
-                uint8_t* smdst = ti.sm_dst + (size_t)t0 * SMB;
-                if (nvalid == P::kValues)
-                    x.template store_sm_full<Global>(smdst);
-                else if (nvalid > 0)
-                    x.store_sm_partial(smdst, nvalid);
-            }
-            __syncwarp();  // the warp's shared-memory accesses above are ordered before lane 0's arrives
-            if (lane == 0) {
-                mbar_arrive(&ctl->empty_w[sw]);
-                mbar_arrive(&ctl->voted[se]);
+            } else {
+                const EncodeTileInfo ti = ctl->info[k % kDescRing];
+                const uint32_t nv = ti.nv;
+                const uint8_t* const s_w = ring_w + (size_t)sw * kWBytes;
+                uint8_t* const s_e = ring_e + (size_t)se * kEBytes;
+#pragma unroll
+                for (int p = 0; p < P::kPerThread; ++p) {
+                    const uint32_t t0 = P::start(tid, p);
+                    const int nvalid = piece_valid<DT>(t0, nv);
+                    // (exp, mant) <- SplitExpMant, and the cached exponents of the same values
+                    P x, c;
+                    if (nv == (uint32_t)kTileValues) {
+                        x.template split_full<Shared>(s_w + (size_t)t0 * VB);
+                        c.template load_exp_full<Shared>(s_e + t0);
+                    } else if (nvalid == P::kValues) {
+                        x.template split_full<Global>(ti.w_src + (size_t)t0 * VB);
+                        c.template load_exp_full<Global>(ti.c_ptr + t0);
+                    } else {
+                        // values past the end of the unit read as exponent 0 against a cached 0: never "changed"
+                        x.split_partial(ti.w_src + (size_t)t0 * VB, nvalid);
+                        c.load_exp_partial(ti.c_ptr + t0, nvalid);
+                    }
+                    // leave the new exponents where the cached ones were staged: they are sent from
+                    // there once the tile's place in the payload is known
+                    x.template store_exp_full<Shared>(s_e + t0);
+                    const uint32_t bal = __ballot_sync(0xffffffffu, x.differs(c));
+                    if (lane == 0) ctl->ballot[se][p * kWarps + warp] = bal;
+                    // sign-plus-mantissa of every value
+                    uint8_t* smdst = ti.sm_dst + (size_t)t0 * SMB;
+                    if (nvalid == P::kValues)
+                        x.template store_sm_full<Global>(smdst);
+                    else if (nvalid > 0)
+                        x.store_sm_partial(smdst, nvalid);
+                }
+                __syncwarp();  // the warp's shared-memory accesses above are ordered before lane 0's arrives
+                if (lane == 0) {
+                    mbar_arrive(&ctl->empty_w[sw]);
+                    mbar_arrive(&ctl->voted[se]);
+                }
             }
 
-            // the changed exponents of the tile handled kDefer tiles ago: its offset is known by now
-            if (k >= (uint32_t)kDefer) {
+            // the changed exponents of the tile handled kDefer slots ago: its offset is known by now
+            if (k >= (uint32_t)kDefer && k - kDefer < k_end) {
                 const uint32_t j = k - kDefer, je = j % SE;
                 if (!mbar_wait(&ctl->resolved[je], (j / SE) & 1u, abort, status)) break;
                 write_changed<DT>(ctl->info[j % kDescRing], log2b, ctl->bm[je], ctl->pre[je], ctl->base[je],
@@ -528,9 +558,11 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&ctl->empty_e[je]);
             }
+            if (marker && k + 1u == k_end + (uint32_t)kResolvers) break;  // that was the last end marker
         }
-        if (!*abort) {
-            for (uint32_t j = my_tiles > (uint32_t)kDefer ? my_tiles - kDefer : 0u; j < my_tiles; ++j) {
+        // tiles whose changed exponents are still to be sent (when kDefer > kResolvers)
+        if (!*abort && k_end != kNoTile) {
+            for (uint32_t j = k + 1u >= (uint32_t)kDefer ? k + 1u - kDefer : 0u; j < k_end; ++j) {
                 const uint32_t je = j % SE;
                 if (!mbar_wait(&ctl->resolved[je], (j / SE) & 1u, abort, status)) break;
                 write_changed<DT>(ctl->info[j % kDescRing], log2b, ctl->bm[je], ctl->pre[je], ctl->base[je],
@@ -585,9 +617,10 @@ static int encode_grid_limit(int* out) {
     return CIERA_OK;
 }
 
+// `scratch`: one status word per tile, then the unit counter; all zero at kernel start.
 template <int DT>
 static int launch_encode(const ciera_plan* p, uint32_t grid, const void* weights_dev, void* sender_cache_dev,
-                         void* messages_dev, uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* workspace_dev,
+                         void* messages_dev, uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* scratch,
                          int32_t* status_dev, cudaStream_t s) {
     const TileDesc* tiles = p->tiles_dev;
     uint32_t nt = (uint32_t)p->tiles.size();
@@ -598,12 +631,22 @@ static int launch_encode(const ciera_plan* p, uint32_t grid, const void* weights
     uint8_t* c = (uint8_t*)sender_cache_dev;
     uint8_t* m = (uint8_t*)messages_dev;
     unsigned long long* wb = (unsigned long long*)wire_bytes_dev;
-    unsigned long long* ts = (unsigned long long*)workspace_dev;
-    void* args[] = {&tiles, &nt, &seq_first, &n_short, &log2b, &w, &c, &m, &wb, &changed_blocks_dev, &ts, &status_dev};
-    // cooperative launch: the runtime starts the grid only when all of its blocks fit on the GPU
-    // together, which is what the look-back between blocks relies on
-    cudaError_t e = cudaLaunchCooperativeKernel((const void*)encode_kernel<DT>, dim3(grid), dim3(kEncodeThreads), args,
-                                                encode_smem_bytes<DT>(), s);
+    unsigned long long* ts = (unsigned long long*)scratch;
+    unsigned int* ticket = (unsigned int*)(ts + nt);
+    const bool has_spread = p->seq_first.back() < nt;  // tiles of longer units: look-back between blocks
+    cudaError_t e;
+    if (has_spread) {
+        // cooperative launch: the runtime starts the grid only when all of its blocks fit on the
+        // GPU together, which is what the look-back between blocks relies on
+        void* args[] = {&tiles, &nt, &seq_first, &n_short, &log2b, &w, &c, &m, &wb, &changed_blocks_dev, &ts, &ticket,
+                        &status_dev};
+        e = cudaLaunchCooperativeKernel((const void*)encode_kernel<DT>, dim3(grid), dim3(kEncodeThreads), args,
+                                        encode_smem_bytes<DT>(), s);
+    } else {
+        encode_kernel<DT><<<grid, kEncodeThreads, encode_smem_bytes<DT>(), s>>>(tiles, nt, seq_first, n_short, log2b, w, c, m,
+                                                                               wb, changed_blocks_dev, ts, ticket, status_dev);
+        e = cudaGetLastError();
+    }
     if (e != cudaSuccess) return record_cuda_error(e);
     count_launch();
     return CIERA_OK;
@@ -640,8 +683,8 @@ extern "C" int ciera_encode(const ciera_plan* p, const void* weights_dev, void* 
     int rc = p->dtype == CIERA_BF16 ? encode_grid_limit<CIERA_BF16>(&limit) : encode_grid_limit<CIERA_FP32>(&limit);
     if (rc) return rc;
     const uint32_t grid = nt < (uint32_t)limit ? nt : (uint32_t)limit;
-    // scratch = one look-back status word per tile; all of it starts at zero
-    e = cudaMemsetAsync(workspace_dev, 0, sizeof(unsigned long long) * nt, s);
+    // scratch = one look-back status word per tile, then the unit counter; all of it starts at zero
+    e = cudaMemsetAsync(workspace_dev, 0, sizeof(unsigned long long) * nt + 16, s);
     if (e != cudaSuccess) return record_cuda_error(e);
     if (p->dtype == CIERA_BF16)
         return launch_encode<CIERA_BF16>(p, grid, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
@@ -661,7 +704,7 @@ extern "C" int ciera_encode(const ciera_plan* p, const void* weights_dev, void* 
 // the encode kernel lives in the library itself: a fixed array in device memory that every GPU
 // loading the library holds from load until the process exits.
 
-static __device__ __align__(256) unsigned long long g_encode_scratch[CIERA_NOALLOC_MAX_TILES];
+static __device__ __align__(256) unsigned long long g_encode_scratch[CIERA_NOALLOC_MAX_TILES + 2];
 
 // Device address of g_encode_scratch on the current device.  In host code the array's name is only
 // a handle for the runtime, not an address a kernel could use, so the address is looked up once
@@ -714,9 +757,9 @@ extern "C" int ciera_encode_noalloc(const ciera_plan* p, const void* weights_dev
     rc = p->dtype == CIERA_BF16 ? encode_grid_limit<CIERA_BF16>(&limit) : encode_grid_limit<CIERA_FP32>(&limit);
     if (rc) return rc;
     const uint32_t grid = nt < (uint32_t)limit ? nt : (uint32_t)limit;
-    // the array keeps what the previous call left in it: the status words of this call's tiles
-    // have to start at zero
-    e = cudaMemsetAsync(scratch, 0, sizeof(unsigned long long) * nt, s);
+    // the array keeps what the previous call left in it: the status words of this call's tiles and
+    // the unit counter behind them have to start at zero
+    e = cudaMemsetAsync(scratch, 0, sizeof(unsigned long long) * nt + 16, s);
     if (e != cudaSuccess) return record_cuda_error(e);
     if (p->dtype == CIERA_BF16)
         return launch_encode<CIERA_BF16>(p, grid, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
