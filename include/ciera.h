@@ -121,7 +121,8 @@ CIERA_API uint64_t ciera_plan_total_values(const ciera_plan* plan);
 /* Bytes of device memory the table needs (>= 16), and the host image that has to be there. */
 CIERA_API size_t ciera_plan_device_bytes(const ciera_plan* plan);
 CIERA_API const void* ciera_plan_host_image(const ciera_plan* plan);
-/* Bytes of scratch one ciera_encode or ciera_decode call needs (per-tile words). */
+/* Bytes of scratch one ciera_encode, ciera_transport or ciera_decode call needs (per-tile words
+ * and a work counter). */
 CIERA_API size_t ciera_plan_workspace_bytes(const ciera_plan* plan);
 
 /* Copies the table into caller-owned device memory `plan_dev` (>= ciera_plan_device_bytes,
@@ -150,8 +151,9 @@ CIERA_API int ciera_cache_update(const ciera_plan* plan, void* cache_dev, const 
  *   wire_bytes_dev      out  [n_units] bytes that have to travel (payload offset + payload bytes;
  *                            0 for an empty unit)
  *   changed_blocks_dev  out  [n_units] number of set bitmap bits
- *   workspace_dev       scratch of ciera_plan_workspace_bytes(), 16-byte aligned; cleared by the
- *                            call itself; must not be shared by calls that can overlap on the GPU
+ *   workspace_dev       scratch of ciera_plan_workspace_bytes(), 16-byte aligned (look-back status
+ *                            words and the counter units are handed out from); cleared by the call
+ *                            itself; must not be shared by calls that can overlap on the GPU
  *   status_dev          i/o  device error word (may be NULL)
  * One kernel launch (plus one memset of the scratch) for the whole table.
  */
@@ -162,8 +164,8 @@ CIERA_API int ciera_encode(const ciera_plan* plan, const void* weights_dev, void
 /* ---- sender, for callers that cannot supply scratch ---------------------------------------- */
 
 /* Largest plan ciera_encode_noalloc accepts: 65 536 tiles (ciera_plan_n_tiles), i.e. at most
- * 536 870 912 values per call.  The library keeps 8 bytes per tile = 512 KiB of device memory for it
- * on every GPU that loads the library, from load until the process exits. */
+ * 536 870 912 values per call.  The library keeps 8 bytes per tile (+ 16) = 512 KiB of device memory
+ * for it on every GPU that loads the library, from load until the process exits. */
 #define CIERA_NOALLOC_MAX_TILES 65536u
 
 /*
@@ -194,9 +196,11 @@ CIERA_API int ciera_encode_noalloc(const ciera_plan* plan, const void* weights_d
 
 /* Copies, for every unit, the first wire_bytes_dev[u] bytes of its slot from `src_messages_dev`
  * to the same slot of `dst_messages_dev` (one kernel; the lengths are read on the device).  This
- * stands where the Allgather of the messages would be.  status_dev (may be NULL) as above. */
+ * stands where the Allgather of the messages would be.  `workspace_dev`: scratch of
+ * ciera_plan_workspace_bytes() (holds the counter tiles are handed out from; cleared by the call;
+ * not to be shared by calls that can overlap on the GPU). */
 CIERA_API int ciera_transport(const ciera_plan* plan, const void* src_messages_dev, void* dst_messages_dev,
-                    const uint64_t* wire_bytes_dev, int32_t* status_dev, void* stream);
+                    const uint64_t* wire_bytes_dev, void* workspace_dev, void* stream);
 
 /* ---- receiver: Algorithm 1, receiver part; Section 3.1 ------------------------------------- */
 

@@ -216,10 +216,10 @@ def encode_noalloc(plan: Plan, weights, sender_cache, messages, wire_bytes, chan
                                      _ptr(changed_blocks), _ptr(status), _stream(stream)))
 
 
-def transport(plan: Plan, src_messages, dst_messages, wire_bytes, status=None, stream=None) -> None:
+def transport(plan: Plan, src_messages, dst_messages, wire_bytes, workspace, stream=None) -> None:
     _check("ciera_transport",
-           _lib.ciera_transport(plan.handle, _ptr(src_messages), _ptr(dst_messages), _ptr(wire_bytes), _ptr(status),
-                                _stream(stream)))
+           _lib.ciera_transport(plan.handle, _ptr(src_messages), _ptr(dst_messages), _ptr(wire_bytes),
+                                _ptr(workspace), _stream(stream)))
 
 
 def decode(plan: Plan, messages, receiver_cache, weights_out, wire_bytes=None, workspace=None, status=None,

@@ -40,11 +40,12 @@ cache_fill_kernel(const TileDesc* __restrict__ tiles, const uint8_t* __restrict_
 // ------------------------------------------------------------------------------------------
 // transport stand-in: copy the used bytes of every slot
 //
-// A persistent copy kernel in which every warp works on its own: warp w of the grid takes tiles
-// w, w + W, ... of the plan's table; tile j of a unit moves bytes [j * chunk, (j + 1) * chunk) of
-// the unit's slot, cut off at the length the sender reported.  A warp moves 4 KB per step (eight
-// 128-bit loads per lane in flight, then eight stores); the tile descriptor and the reported
-// length of the next tiles are fetched ahead so that no step waits for them.
+// A persistent copy kernel in which every warp works on its own: it draws tile numbers from a
+// counter in the caller's scratch (so all SMs stay busy to the end whatever their pace); tile j of
+// a unit moves bytes [j * chunk, (j + 1) * chunk) of the unit's slot, cut off at the length the
+// sender reported.  A warp moves 4 KB per step (eight 128-bit loads per lane in flight, then eight
+// stores); tile numbers, descriptors and reported lengths are fetched three, two and one tile
+// ahead, so that no step waits for them.
 
 constexpr int kCopyThreads = 256;
 constexpr int kCopyUnroll = 8;
@@ -52,27 +53,35 @@ constexpr int kCopyUnroll = 8;
 __global__ void __launch_bounds__(kCopyThreads)
 transport_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t sm_bytes_per_value,
                  const uint8_t* __restrict__ src, uint8_t* __restrict__ dst,
-                 const unsigned long long* __restrict__ wire_bytes) {
+                 const unsigned long long* __restrict__ wire_bytes, unsigned int* ticket) {
     const uint32_t lane = threadIdx.x & 31u;
-    const uint32_t warps_per_block = kCopyThreads / 32;
-    const uint32_t W = gridDim.x * warps_per_block;
-    const uint32_t t_first = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
     const uint64_t chunk = transport_chunk_bytes(sm_bytes_per_value);
-
-    // descriptors two tiles ahead, reported lengths one tile ahead
+    auto draw = [&]() {
+        uint32_t t = 0;
+        if (lane == 0) t = atomicAdd(ticket, 1u);
+        return __shfl_sync(0xffffffffu, t, 0);
+    };
+    // three-deep software pipeline: tile number drawn (t_c), descriptor loaded (t_b, td_b), reported
+    // length loaded (t_a, td_a, used_a)
+    uint32_t t_a = draw(), t_b = draw(), t_c = draw();
     TileDesc td_a, td_b;
     unsigned long long used_a = 0;
-    if (t_first < n_tiles) {
-        td_a = load_tile_desc(tiles + t_first);
+    if (t_a < n_tiles) {
+        td_a = load_tile_desc(tiles + t_a);
         used_a = __ldg(wire_bytes + td_a.unit);
     }
-    if (t_first + W < n_tiles) td_b = load_tile_desc(tiles + t_first + W);
-    for (uint32_t t = t_first; t < n_tiles; t += W) {
+    if (t_b < n_tiles) td_b = load_tile_desc(tiles + t_b);
+    while (t_a < n_tiles) {
         const TileDesc td = td_a;
         const uint64_t used = used_a;
+        // advance the pipeline; none of these loads is needed before the next iteration
+        const uint32_t t_d = t_c < n_tiles ? draw() : n_tiles;
         td_a = td_b;
-        if (t + W < n_tiles) used_a = __ldg(wire_bytes + td_a.unit);
-        if (t + 2ull * W < n_tiles) td_b = load_tile_desc(tiles + t + 2u * W);
+        if (t_b < n_tiles) used_a = __ldg(wire_bytes + td_a.unit);
+        if (t_c < n_tiles) td_b = load_tile_desc(tiles + t_c);
+        t_a = t_b;
+        t_b = t_c;
+        t_c = t_d;
 
         const uint64_t lo = (uint64_t)td.tile_in_unit * chunk;
         if (lo >= used) continue;
@@ -154,22 +163,26 @@ extern "C" int ciera_cache_update(const ciera_plan* plan, void* cache_dev, const
 }
 
 extern "C" int ciera_transport(const ciera_plan* p, const void* src_messages_dev, void* dst_messages_dev,
-                               const uint64_t* wire_bytes_dev, int32_t* status_dev, void* stream) {
+                               const uint64_t* wire_bytes_dev, void* workspace_dev, void* stream) {
     int rc = check_plan(p);
     if (rc) return rc;
     const uint32_t nt = (uint32_t)p->tiles.size();
     if (nt == 0) return CIERA_OK;
-    if (!src_messages_dev || !dst_messages_dev || !wire_bytes_dev) return CIERA_ERR_INVALID_ARG;
-    if (misaligned16(src_messages_dev) || misaligned16(dst_messages_dev)) return CIERA_ERR_MISALIGNED;
+    if (!src_messages_dev || !dst_messages_dev || !wire_bytes_dev || !workspace_dev) return CIERA_ERR_INVALID_ARG;
+    if (misaligned16(src_messages_dev) || misaligned16(dst_messages_dev) || misaligned16(workspace_dev))
+        return CIERA_ERR_MISALIGNED;
+    // the tile counter sits past the per-tile words of the scratch and starts at zero
+    unsigned int* ticket = (unsigned int*)((unsigned long long*)workspace_dev + nt);
+    cudaError_t me = cudaMemsetAsync(ticket, 0, 16, (cudaStream_t)stream);
+    if (me != cudaSuccess) return record_cuda_error(me);
     int limit = 0;
     rc = transport_grid_limit(&limit);
     if (rc) return rc;
     const uint32_t want = (nt + kCopyThreads / 32 - 1) / (kCopyThreads / 32);
     const uint32_t grid = want < (uint32_t)limit ? want : (uint32_t)limit;
-    (void)status_dev;  // this kernel has no waits that could run out
     transport_kernel<<<grid, kCopyThreads, 0, (cudaStream_t)stream>>>(
         p->tiles_dev, nt, p->dtype == CIERA_BF16 ? 1u : 3u, (const uint8_t*)src_messages_dev, (uint8_t*)dst_messages_dev,
-        (const unsigned long long*)wire_bytes_dev);
+        (const unsigned long long*)wire_bytes_dev, ticket);
     count_launch();
     return check_launch();
 }
@@ -187,7 +200,7 @@ extern "C" int ciera_roundtrip_host(const ciera_plan* p, const void* weights_hos
     rc = ciera_encode(p, b->weights_dev, b->sender_cache_dev, b->msg_send_dev, b->wire_bytes_dev, b->changed_blocks_dev,
                       b->workspace_dev, b->status_dev, stream);
     if (rc) return rc;
-    rc = ciera_transport(p, b->msg_send_dev, b->msg_recv_dev, b->wire_bytes_dev, b->status_dev, stream);
+    rc = ciera_transport(p, b->msg_send_dev, b->msg_recv_dev, b->wire_bytes_dev, b->workspace_dev, stream);
     if (rc) return rc;
     rc = ciera_decode(p, b->msg_recv_dev, b->receiver_cache_dev, b->weights_out_dev, b->wire_bytes_dev,
                       b->workspace_dev, b->status_dev, stream);
