@@ -80,9 +80,11 @@ constexpr uint32_t kDecodeDirectBlocks = 4096;
 // block) and spreads everything else tile by tile over all blocks.
 constexpr uint32_t kSeqMaxTiles = 32;
 
-// Bytes of a message slot that one tile moves in the transport kernel: slot capacity <= tiles * this.
+// Bytes of a message slot that tile j of a unit moves in the transport kernel: [j * chunk,
+// (j + 1) * chunk); the unit's last tile also moves whatever lies beyond (bitmap and pads: the slot
+// capacity exceeds tiles * chunk by less than 100 bytes per unit plus one bitmap byte per 8 blocks).
 __host__ __device__ inline uint64_t transport_chunk_bytes(uint32_t sm_bytes_per_value) {
-    return (uint64_t)kTileValues * (sm_bytes_per_value + 1) + 96;
+    return (uint64_t)kTileValues * (sm_bytes_per_value + 1);
 }
 
 }  // namespace ciera

@@ -42,13 +42,35 @@ cache_fill_kernel(const TileDesc* __restrict__ tiles, const uint8_t* __restrict_
 //
 // A persistent copy kernel in which every warp works on its own: it draws tile numbers from a
 // counter in the caller's scratch (so all SMs stay busy to the end whatever their pace); tile j of
-// a unit moves bytes [j * chunk, (j + 1) * chunk) of the unit's slot, cut off at the length the
-// sender reported.  A warp moves 4 KB per step (eight 128-bit loads per lane in flight, then eight
+// a unit moves bytes [j * chunk, (j + 1) * chunk) of the unit's slot (chunk = 16 KB for bf16, 32 KB
+// for fp32), the last tile also what lies beyond, cut off at the length the sender reported.  A warp moves 4 KB per step (eight 128-bit loads per lane in flight, then eight
 // stores); tile numbers, descriptors and reported lengths are fetched three, two and one tile
 // ahead, so that no step waits for them.
 
-constexpr int kCopyThreads = 256;
-constexpr int kCopyUnroll = 8;
+#ifndef CIERA_COPY_THREADS
+#define CIERA_COPY_THREADS 256
+#endif
+#ifndef CIERA_COPY_UNROLL
+#define CIERA_COPY_UNROLL 8
+#endif
+constexpr int kCopyThreads = CIERA_COPY_THREADS;
+constexpr int kCopyUnroll = CIERA_COPY_UNROLL;
+
+// the part of a tile descriptor the copy needs (keeps the prefetched copies small in registers)
+struct CopyDesc {
+    uint64_t msg_off;
+    uint32_t unit, tile_in_unit, n_tiles_unit;
+};
+__device__ __forceinline__ CopyDesc load_copy_desc(const TileDesc* t) {
+    const uint4* p = reinterpret_cast<const uint4*>(t);
+    const uint4 b = __ldg(p + 1), c = __ldg(p + 2);
+    CopyDesc d;
+    d.msg_off = (uint64_t)b.x | ((uint64_t)b.y << 32);
+    d.unit = c.x;
+    d.tile_in_unit = c.y;
+    d.n_tiles_unit = c.w;
+    return d;
+}
 
 __global__ void __launch_bounds__(kCopyThreads)
 transport_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t sm_bytes_per_value,
@@ -64,28 +86,30 @@ transport_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t 
     // three-deep software pipeline: tile number drawn (t_c), descriptor loaded (t_b, td_b), reported
     // length loaded (t_a, td_a, used_a)
     uint32_t t_a = draw(), t_b = draw(), t_c = draw();
-    TileDesc td_a, td_b;
+    CopyDesc td_a, td_b;
     unsigned long long used_a = 0;
     if (t_a < n_tiles) {
-        td_a = load_tile_desc(tiles + t_a);
+        td_a = load_copy_desc(tiles + t_a);
         used_a = __ldg(wire_bytes + td_a.unit);
     }
-    if (t_b < n_tiles) td_b = load_tile_desc(tiles + t_b);
+    if (t_b < n_tiles) td_b = load_copy_desc(tiles + t_b);
     while (t_a < n_tiles) {
-        const TileDesc td = td_a;
+        const CopyDesc td = td_a;
         const uint64_t used = used_a;
         // advance the pipeline; none of these loads is needed before the next iteration
         const uint32_t t_d = t_c < n_tiles ? draw() : n_tiles;
         td_a = td_b;
         if (t_b < n_tiles) used_a = __ldg(wire_bytes + td_a.unit);
-        if (t_c < n_tiles) td_b = load_tile_desc(tiles + t_c);
+        if (t_c < n_tiles) td_b = load_copy_desc(tiles + t_c);
         t_a = t_b;
         t_b = t_c;
         t_c = t_d;
 
         const uint64_t lo = (uint64_t)td.tile_in_unit * chunk;
         if (lo >= used) continue;
-        const uint64_t hi = lo + chunk < used ? lo + chunk : used;
+        // the unit's last tile also takes what lies beyond tiles * chunk
+        const bool last = td.tile_in_unit == td.n_tiles_unit - 1u;
+        const uint64_t hi = (last || lo + chunk >= used) ? used : lo + chunk;
         const uint8_t* s = src + td.msg_off + lo;
         uint8_t* d = dst + td.msg_off + lo;
         const uint32_t nvec = (uint32_t)((hi - lo) >> 4);  // 16-byte pieces

@@ -241,3 +241,49 @@ def test_pipelined_stack_equals_serial(rt):
     for a, b in zip(*results):
         for x, y in zip(a, b):
             assert torch.equal(x, y)
+
+
+@pytest.mark.parametrize("dtype,block", [(0, 512), (1, 512), (0, 64)])
+def test_full_size_layer_sampled_units(rt, dtype, block):
+    """One full OLMoE-shaped layer (64 experts x 3 matrices, 16 shards: 3072 units, 402 653 184 values) in the
+    launch configuration the benchmark times, generated on the device.  The round trip is checked everywhere
+    (device-side comparison); messages, lengths, counts and caches of sampled units are checked against the
+    oracle, which gets the units' weights before and after the step."""
+    ciera, runtime = rt
+    from oracle import ciera_oracle as ora
+
+    name = NAME[dtype]
+    vb = wl.VALUE_BYTES[name]
+    shapes = [r * c for r, c in wl.olmoe_layer_shapes(64)]
+    codec = runtime.LayerCodec.from_tensors(shapes, 16, name, block, DEV)
+    n = codec.weights_bytes // vb
+    gen = wl.make_generator(2024 + dtype, DEV)
+    w0 = wl.init_weights(n, name, gen)
+    w1 = wl.step_clustered(w0, gen, f=0.22)
+    w2 = wl.step_adam_like(w1, gen)  # second step: every block changes
+    b0, b1, b2 = (w.view(torch.uint8) for w in (w0, w1, w2))
+    codec.init_caches(b0)
+    rng = np.random.default_rng(5)
+    picks = sorted(set(rng.integers(0, len(codec.units), 12).tolist()) | {0, len(codec.units) - 1})
+    wdt = WDT[dtype]
+    prev = b0
+    for cur in (b1, b2):
+        codec.step(cur)
+        torch.cuda.synchronize()
+        codec.check_status()
+        assert torch.equal(codec.weights_out[: cur.numel()], cur), "round trip is not bit-exact"
+        assert torch.equal(codec.sender_cache, codec.receiver_cache)
+        for ui in picks:
+            u = codec.units[ui]
+            lo, nn, mo, co = int(u["weights_off"]), int(u["n_values"]), int(u["msg_off"]), int(u["cache_off"])
+            wp = prev[lo : lo + nn * vb].cpu().numpy().view(wdt)
+            wc = cur[lo : lo + nn * vb].cpu().numpy().view(wdt)
+            cache = ora.cache_init(wp, nn, dtype)
+            m, wbytes, pay, cb = ora.encode(wc, cache, dtype, block)
+            assert int(codec.wire_bytes[ui].item()) == wbytes and int(codec.changed_blocks[ui].item()) == cb
+            assert np.array_equal(codec.msg_send[mo : mo + wbytes].cpu().numpy(), m), f"message of unit {ui}"
+            assert np.array_equal(codec.msg_recv[mo : mo + wbytes].cpu().numpy(), m), f"transported message {ui}"
+            assert np.array_equal(codec.sender_cache[co : co + nn].cpu().numpy(), cache)
+        prev = cur
+    q = int(codec.changed_blocks.sum().item()) / codec.n_blocks()
+    assert q > (0.99 if block >= 256 else 0.8)  # the i.i.d. step changes (nearly) every block
