@@ -53,7 +53,11 @@ def parse_args():
     ap.add_argument("--shards", type=int, default=16)
     ap.add_argument("--block", type=int, default=512)
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
-    ap.add_argument("--update", default="clustered", choices=["clustered", "adam"])
+    ap.add_argument("--update", default="clustered", choices=["clustered", "adam", "inject"])
+    ap.add_argument("--inject", type=float, default=0.01, help="exponent change rate of the 'inject' update model")
+    ap.add_argument("--shapes", default="olmoe", choices=["olmoe", "mixed"],
+                    help="olmoe: 64 experts x 3 matrices per layer; mixed: 256 fine-grained experts (2048x512, "
+                         "2048x512, 512x2048) plus dense tensors of 4 KB ... 256 MB (the mixed-shape sweep)")
     ap.add_argument("--f", type=float, default=0.22, help="fraction of segments updated (clustered model)")
     ap.add_argument("--schedule", default="pipelined", choices=["pipelined", "serial"])
     ap.add_argument("--no-e2e", action="store_true")
@@ -167,15 +171,19 @@ def build_stack(args, device, seed_base):
     from paper_2609_04609_b200 import runtime
     from paper_2609_04609_b200 import workloads as wl
 
-    shapes = [r * c for r, c in wl.olmoe_layer_shapes(args.experts)]
+    shapes = layer_numels(args)
     layers, wa, wb = [], [], []
     for l in range(args.layers):
         codec = runtime.LayerCodec.from_tensors(shapes, args.shards, args.dtype, args.block, device)
         n = codec.weights_bytes // wl.VALUE_BYTES[args.dtype]
         gen = wl.make_generator(seed_base + l, device)
         w = wl.init_weights(n, args.dtype, gen)
-        step = (lambda x: wl.step_clustered(x, gen, f=args.f, seg=512)) if args.update == "clustered" else (
-            lambda x: wl.step_adam_like(x, gen))
+        if args.update == "clustered":
+            step = lambda x: wl.step_clustered(x, gen, f=args.f, seg=512)
+        elif args.update == "adam":
+            step = lambda x: wl.step_adam_like(x, gen)
+        else:
+            step = lambda x: wl.inject_exponent_changes(x, gen, args.inject)
         for _ in range(4):  # iterations 1..4 of the trajectory
             w = step(w)
         w5 = step(w)  # iteration 5
@@ -187,6 +195,14 @@ def build_stack(args, device, seed_base):
     return layers, wa, wb
 
 
+def layer_numels(args):
+    from paper_2609_04609_b200 import workloads as wl
+
+    if args.shapes == "mixed":
+        return [r * c for r, c in wl.fine_grained_layer_shapes(256)] + wl.dense_tensor_sizes()
+    return [r * c for r, c in wl.olmoe_layer_shapes(args.experts)]
+
+
 def algorithmic_bytes(n_values, q, dtype):
     """HBM bytes per launch the method needs: (encode, transport, decode)."""
     vb, smb = (2, 1) if dtype == "bf16" else (4, 3)
@@ -196,11 +212,15 @@ def algorithmic_bytes(n_values, q, dtype):
     return enc, tra, dec
 
 
-def run_step(layers, weights, s_enc, s_dec, events, schedule, timers=None):
-    """encode+transport of layer l on s_enc, decode of layer l on s_dec (same stream if serial)."""
+def run_step(layers, weights, s_enc, s_dec, events, schedule, timers=None, decoded=None):
+    """encode+transport of layer l on s_enc, decode of layer l on s_dec (same stream if serial).
+    `decoded[l]`: event recorded after the previous decode of layer l; the sender side of the next
+    step waits for it before it overwrites the layer's message buffers."""
     import torch
 
     for l, (codec, w) in enumerate(zip(layers, weights)):
+        if schedule == "pipelined" and decoded is not None:
+            s_enc.wait_event(decoded[l])
         if timers is not None:
             t = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
             t[0].record(s_enc)
@@ -217,6 +237,8 @@ def run_step(layers, weights, s_enc, s_dec, events, schedule, timers=None):
         if timers is not None:
             t[4].record(s_dec)
         codec.decode(None, s_dec)
+        if schedule == "pipelined" and decoded is not None:
+            decoded[l].record(s_dec)
         if timers is not None:
             t[5].record(s_dec)
             timers.append(t)
@@ -269,16 +291,19 @@ def run_reference(args):
     ora.build()
     code = 0 if args.dtype == "bf16" else 1
     vb = wl.VALUE_BYTES[args.dtype]
-    shapes = [r * c for r, c in wl.olmoe_layer_shapes(args.experts)]
+    shapes = layer_numels(args)
     n_units = min(args.cpu_sample_units, len(shapes) * args.shards)
     units, wbytes, _, _ = wl.layout_units(shapes, args.shards, vb, lambda n: ora.message_capacity(n, code, args.block))
     units = units[:n_units]
     n = int(units[-1]["weights_off"]) // vb + int(units[-1]["n_values"])
     gen = wl.make_generator(1234 + 3)
     w = wl.init_weights(n, args.dtype, gen)
-    step = (lambda x: wl.step_clustered(x, gen, f=args.f, seg=512)) if args.update == "clustered" else (
-        lambda x: wl.step_adam_like(x, gen))
-    w1 = step(w)
+    if args.update == "clustered":
+        w1 = wl.step_clustered(w, gen, f=args.f, seg=512)
+    elif args.update == "adam":
+        w1 = wl.step_adam_like(w, gen)
+    else:
+        w1 = wl.inject_exponent_changes(w, gen, args.inject)
     a = wl.as_bits(w).view(np.uint8)
     b = wl.as_bits(w1).view(np.uint8)
     threads = os.cpu_count() or 1
@@ -303,12 +328,18 @@ def run_reference(args):
 
 
 def workload_config(args):
-    full = args.layers == 16 and args.experts == 64
-    name = ("config3: full OLMoE-1B-7B expert stack" if full else "reduced OLMoE expert stack")
+    full = args.layers == 16 and args.experts == 64 and args.shapes == "olmoe"
+    upd = f"update model {args.update}" + (f" f={args.f}" if args.update == "clustered" else "") + (
+        f" c={args.inject}" if args.update == "inject" else "")
+    if args.shapes == "mixed":
+        what = (f"mixed-shape sweep (config 5), {args.layers} x [256 fine-grained experts x (2048x512, 2048x512, "
+                f"512x2048) + dense tensors 4 KB..256 MB] {args.dtype}")
+    else:
+        name = "config3: full OLMoE-1B-7B expert stack" if full else "reduced OLMoE expert stack"
+        what = (f"{name}, {args.layers} layers x {args.experts} experts x 3 matrices (2048x1024, 2048x1024, "
+                f"1024x2048) {args.dtype}")
     return {
-        "workload": f"{name}, {args.layers} layers x {args.experts} experts x 3 matrices (2048x1024, 2048x1024, "
-                    f"1024x2048) {args.dtype}, {args.shards} simulated shards per matrix, block {args.block}, "
-                    f"update model {args.update}" + (f" f={args.f}" if args.update == "clustered" else ""),
+        "workload": f"{what}, {args.shards} simulated shards per matrix, block {args.block}, {upd}",
         "l2": "inputs larger than L2 (no flush needed)",
         "schedule": args.schedule,
         "round_trip": "encode + device-to-device transport + decode",
@@ -354,13 +385,16 @@ def main():
     if args.schedule == "serial":
         s_dec = s_enc
     events = [torch.cuda.Event() for _ in layers]
+    decoded = [torch.cuda.Event() for _ in layers]
+    for ev in decoded:
+        ev.record(torch.cuda.current_stream())
 
     def weights_of(i):
         return wb if i % 2 == 0 else wa
 
     step_i = 0
     for _ in range(max(args.warmup, 3)):
-        run_step(layers, weights_of(step_i), s_enc, s_dec, events, args.schedule)
+        run_step(layers, weights_of(step_i), s_enc, s_dec, events, args.schedule, None, decoded)
         step_i += 1
     barrier()
 
@@ -380,7 +414,7 @@ def main():
     s_enc.wait_event(ev0)
     s_dec.wait_event(ev0)
     for _ in range(args.steps):
-        run_step(layers, weights_of(step_i), s_enc, s_dec, events, args.schedule, timers)
+        run_step(layers, weights_of(step_i), s_enc, s_dec, events, args.schedule, timers, decoded)
         step_i += 1
     cur.wait_stream(s_enc)
     cur.wait_stream(s_dec)
@@ -426,7 +460,17 @@ def main():
     # ---- correctness at full size: exact round trip everywhere, oracle on sampled units
     last_w = weights_of(step_i - 1)
     prev_w = weights_of(step_i)  # the iterate before the last one (the steps alternate)
-    verified = all(torch.equal(c.weights_out[: w.numel()], w) for c, w in zip(layers, last_w))
+    def same_weights(c, w):
+        """Exact comparison over the units' own bytes (alignment gaps between units carry nothing)."""
+        if int(c.units["n_values"].sum()) * vb == w.numel():
+            return torch.equal(c.weights_out[: w.numel()], w)
+        keep = np.zeros(w.numel(), dtype=bool)
+        for u in c.units:
+            keep[int(u["weights_off"]) : int(u["weights_off"]) + int(u["n_values"]) * vb] = True
+        keep = torch.from_numpy(keep).to(w.device)
+        return torch.equal(c.weights_out[: w.numel()][keep], w[keep])
+
+    verified = all(same_weights(c, w) for c, w in zip(layers, last_w))
     verified = verified and all(torch.equal(c.sender_cache, c.receiver_cache) for c in layers)
     sampled = 0
     if rank == 0:

@@ -119,7 +119,9 @@ def pipelined_step(layers: List[LayerCodec], weights: List[torch.Tensor], outs: 
     """One iteration over a stack of layers on two streams: the sender-side work of layer l+1
     (encode, then the transport of its message) runs on ``s_enc`` while the receiver-side
     decode of layer l runs on ``s_dec`` -- the shape of the paper's computation-communication
-    pipelining, where only the decompression of layer l stays on the critical path."""
+    pipelining, where only the decompression of layer l stays on the critical path.  A caller that
+    runs several iterations back to back must make the next iteration's sender side of a layer wait
+    for this iteration's decode of that layer (they share the layer's message buffers)."""
     n = len(layers)
     if events is None:
         events = [torch.cuda.Event() for _ in range(n)]
