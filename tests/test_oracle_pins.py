@@ -52,7 +52,8 @@ def test_split_fp32_random_and_special_patterns_match_ieee_definition(oracle):
 # ------------------------------------------------------------------ hand-worked fixtures
 
 
-@pytest.mark.parametrize("name", ["bf16_worked_example.txt", "fp32_worked_example.txt"])
+@pytest.mark.parametrize("name", ["bf16_worked_example.txt", "fp32_worked_example.txt",
+                                  "small_block_worked_example.txt"])
 def test_hand_worked_examples(oracle, name):
     for st in parse_golden(os.path.join(GOLDEN, name)):
         dtype = BF16 if st["dtype"][0] == "bf16" else FP32
@@ -123,7 +124,8 @@ def test_transmitted_bytes_formula_and_shadow_bookkeeping(oracle, dtype):
     rng = np.random.default_rng(11 + dtype)
     m_bytes = 1 if dtype == BF16 else 3
     for n, block in [(1, 64), (5, 2), (63, 64), (64, 64), (65, 64), (1000, 128), (4097, 512), (12345, 4096),
-                     (70000, 512), (33, 1), (1024, 16), (2049, 1024)]:
+                     (70000, 512), (33, 1), (1024, 16), (2049, 1024), (8193, 1), (10001, 2), (9003, 4),
+                     (20001, 8)]:
         hi = 1 << (16 if dtype == BF16 else 32)
         w_prev = rng.integers(0, hi, size=n, dtype=np.uint64).astype(np.uint16 if dtype == BF16 else np.uint32)
         w = w_prev.copy()
