@@ -89,8 +89,11 @@ typedef struct ciera_unit {
 
 /* ---- sizes (host, pure functions; Section 3.2) ------------------------------------------- */
 
-/* Smallest and largest supported block size B (a power of two in this range). */
-#define CIERA_MIN_BLOCK 16u
+/* Smallest and largest supported block size B (a power of two in this range).  B = 1 is change
+ * detection per value: the bitmap has one bit per value and the payload holds exactly the exponents
+ * that changed (Section 2.3: a block stays reusable with probability (1-c)^B, so finer blocks are
+ * reused more often, at the price of a longer bitmap). */
+#define CIERA_MIN_BLOCK 1u
 #define CIERA_MAX_BLOCK 4096u
 
 /* Slot size that always suffices: every block changed (payload = N exponent bytes). */

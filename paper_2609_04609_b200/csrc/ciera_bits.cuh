@@ -13,8 +13,9 @@
 //         8 B / lane on the byte-wide streams (exponents, sign-plus-mantissa).
 //   fp32: one piece of 16 values per thread, values [16 t, +16): 64 B of weights, 16 B of
 //         exponents, 48 B of sign-plus-mantissa per lane.
-// A piece never straddles a block (block sizes are multiples of 16), so a piece has one
-// "my exponents changed" bit; the tile has 1024 (bf16) or 512 (fp32) such bits.
+// With blocks of 16 values and more a piece never straddles a block, so a piece has one "my
+// exponents changed" bit; the tile has 1024 (bf16) or 512 (fp32) such bits.  With smaller blocks
+// a piece holds 1 to 16 whole blocks and has one bit for each.
 #pragma once
 
 #include "ciera_internal.cuh"
@@ -53,12 +54,18 @@ struct Global {
     static __device__ __forceinline__ uint2 ld8(const uint8_t* p) { return ld_stream8(p); }
     static __device__ __forceinline__ void st16(uint8_t* p, uint4 v) { st_stream16(p, v); }
     static __device__ __forceinline__ void st8(uint8_t* p, uint2 v) { st_stream8(p, v); }
+    static __device__ __forceinline__ uint32_t ld1(const uint8_t* p) { return __ldcs(p); }
 };
 struct Shared {
     static __device__ __forceinline__ uint4 ld16(const uint8_t* p) { return ld_shared16(p); }
     static __device__ __forceinline__ uint2 ld8(const uint8_t* p) { return ld_shared8(p); }
     static __device__ __forceinline__ void st16(uint8_t* p, uint4 v) { st_shared16(p, v); }
     static __device__ __forceinline__ void st8(uint8_t* p, uint2 v) { st_shared8(p, v); }
+    static __device__ __forceinline__ uint32_t ld1(const uint8_t* p) {
+        uint32_t v;
+        asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"((uint32_t)__cvta_generic_to_shared(p)));
+        return v;
+    }
 };
 
 // (x & mask) | (y & ~mask): one three-input logic operation
@@ -124,6 +131,20 @@ __device__ __forceinline__ void store_bytes_partial(uint8_t* dst, const uint32_t
 #pragma unroll
     for (int i = 0; i < NB; ++i)
         if (i < nbytes) dst[i] = (uint8_t)(w[i >> 2] >> (8 * (i & 3)));
+}
+
+
+// ---- flags of fine blocks ------------------------------------------------------------------
+// d = new exponents ^ cached exponents of four consecutive values (one byte each).  Returns one
+// flag per block of 2^log2b values (log2b = 0, 1, 2: four, two, one flag), lowest value first.
+__device__ __forceinline__ uint32_t word_block_flags(uint32_t d, uint32_t log2b) {
+    if (log2b == 0) {
+        // bytes that differ -> bits 0, 8, 16, 24 -> gathered into bits 24..27 by one multiply
+        // (the partial products land on distinct bit positions, so nothing carries)
+        return (((__vcmpne4(d, 0u) & 0x01010101u) * 0x01020408u) >> 24) & 0xFu;
+    }
+    if (log2b == 1) return ((d & 0xFFFFu) != 0u ? 1u : 0u) | ((d >> 16) != 0u ? 2u : 0u);
+    return d != 0u ? 1u : 0u;
 }
 
 // ---- pieces --------------------------------------------------------------------------------
@@ -197,6 +218,12 @@ struct Piece<CIERA_BF16> {
             if (i < nvalid) p[i] = (uint16_t)(x[i >> 1] >> (16 * (i & 1)));
     }
     __device__ __forceinline__ bool differs(const Piece& o) const { return ((e[0] ^ o.e[0]) | (e[1] ^ o.e[1])) != 0; }
+    // one flag per block of 2^log2b values (log2b <= 3), lowest block first
+    __device__ __forceinline__ uint32_t block_flags(const Piece& o, uint32_t log2b) const {
+        if (log2b >= 3) return differs(o) ? 1u : 0u;
+        const uint32_t per_word = 4u >> log2b;
+        return word_block_flags(e[0] ^ o.e[0], log2b) | (word_block_flags(e[1] ^ o.e[1], log2b) << per_word);
+    }
 };
 
 // fp32: 16 values = 64 B of weights, 16 exponent bytes, 48 sm bytes
@@ -289,6 +316,16 @@ struct Piece<CIERA_FP32> {
     }
     __device__ __forceinline__ bool differs(const Piece& o) const {
         return ((e[0] ^ o.e[0]) | (e[1] ^ o.e[1]) | (e[2] ^ o.e[2]) | (e[3] ^ o.e[3])) != 0;
+    }
+    // one flag per block of 2^log2b values (log2b <= 3), lowest block first
+    __device__ __forceinline__ uint32_t block_flags(const Piece& o, uint32_t log2b) const {
+        if (log2b >= 3)
+            return (((e[0] ^ o.e[0]) | (e[1] ^ o.e[1])) != 0 ? 1u : 0u) | (((e[2] ^ o.e[2]) | (e[3] ^ o.e[3])) != 0 ? 2u : 0u);
+        const uint32_t per_word = 4u >> log2b;
+        uint32_t f = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) f |= word_block_flags(e[i] ^ o.e[i], log2b) << (per_word * i);
+        return f;
     }
 };
 

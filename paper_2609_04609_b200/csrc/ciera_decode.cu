@@ -29,30 +29,52 @@ namespace ciera {
 constexpr int kDecProducers = 2;                               // producer warps, taking tiles in turn
 constexpr int kDecodeThreads = kThreads + 32 * kDecProducers;  // consumers + producers
 constexpr int kDecProducerWarp0 = kWarps;
-constexpr int kDecRing = 12;  // > stages + 2 * producers + 1: slots are refilled only after their tile is done
 constexpr uint32_t kNoTile = 0xffffffffu;
 constexpr uint32_t kDirectWordsPerLane = 4;
 constexpr uint32_t kDirectBlocks = kDecodeDirectBlocks;
 static_assert(kDirectBlocks == 32u * 32u * kDirectWordsPerLane, "one fetch covers the direct range");
 
-template <int DT>
+// kRing: slots of per-tile bookkeeping; > stages + 2 * producers + 1, since a slot is refilled
+// only after its tile is done.  With fine blocks (see ciera_internal.cuh) a slot holds up to 8192
+// block flags instead of 512.
+template <int DT, bool FINE>
 struct DecodeCfg;
 template <>
-struct DecodeCfg<CIERA_BF16> {
+struct DecodeCfg<CIERA_BF16, false> {
     static constexpr int kStages = 4;        // 4 x (8 KB sm + 8 KB cache span + 8 KB payload slice)
     static constexpr int kBlocksPerSM = 2;
     static constexpr bool kStageOut = false;  // weights leave as 16 B / lane, contiguous per warp
+    static constexpr int kRing = 12;
 };
 template <>
-struct DecodeCfg<CIERA_FP32> {
+struct DecodeCfg<CIERA_FP32, false> {
     static constexpr int kStages = 4;        // 4 x (24 KB sm + 8 KB + 8 KB)
     static constexpr int kBlocksPerSM = 1;
     static constexpr bool kStageOut = true;   // 64 B / lane: staged, then one bulk store per warp
+    static constexpr int kRing = 12;
+};
+template <>
+struct DecodeCfg<CIERA_BF16, true> {
+    static constexpr int kStages = 4;
+    static constexpr int kBlocksPerSM = 2;
+    static constexpr bool kStageOut = false;
+    static constexpr int kRing = 10;
+};
+template <>
+struct DecodeCfg<CIERA_FP32, true> {
+    static constexpr int kStages = 4;
+    static constexpr int kBlocksPerSM = 1;
+    static constexpr bool kStageOut = true;
+    static constexpr int kRing = 12;
 };
 
 // Per-tile bookkeeping, in a ring that the producers fill ahead of the consumers.
+template <bool FINE>
 struct __align__(16) DecodeRing {
+    static constexpr int kBm = FINE ? kFineBitmapWords : kBitmapWords;
     TileDesc desc;                           // copied from the plan's table (asynchronously)
+    // the tile's block flags; with fine blocks they are fetched straight into this array
+    uint32_t bm[kBm];
     // worked out once by a producer for the 512 consumer threads:
     uint8_t* w_dst;                          // where the tile's reconstructed weights go
     uint8_t* c_ptr;                          // the tile's cached exponents
@@ -60,19 +82,19 @@ struct __align__(16) DecodeRing {
     const uint8_t* pay_src;                  // the payload slice holding the tile's changed blocks
     uint32_t nv;                             // values in the tile
     uint32_t tile;                           // the tile's number, or kNoTile: this producer has no more work
-    uint32_t bm[kBitmapWords];               // the tile's block flags
-    uint32_t pre[kBitmapWords];              // set flags before each word
-    // raw material, fetched asynchronously one tile ahead:
-    uint32_t raw_pre[32 * kDirectWordsPerLane];  // bitmap words before the tile
-    uint32_t raw_own[kBitmapWords];              // words holding the tile's own bits
-    uint32_t ws;                                 // count from the scratch (long units)
+    uint32_t pay_skew;                       // fine: bytes in front of the slice in its stage (0 .. 15)
+    uint32_t ws;                             // count from the scratch (units that went through the prefix kernel)
+    uint16_t pre[kBm];                       // set flags before each word
+    // raw material of coarse blocks, fetched asynchronously one tile ahead:
+    uint32_t raw_pre[FINE ? 4 : 32 * kDirectWordsPerLane];  // bitmap words before the tile
+    uint32_t raw_own[FINE ? 4 : kBitmapWords];               // words holding the tile's own bits
 };
 
-template <int S>
+template <int S, int R, bool FINE>
 struct DecodeCtl {
     uint64_t full[S];   // stage filled (producer arrive + bulk-copy bytes)
     uint64_t empty[S];  // all 16 consumer warps have read it
-    DecodeRing ring[kDecRing];
+    DecodeRing<FINE> ring[R];
     int abort;
     uint32_t issued;
     uint32_t seen;
@@ -81,12 +103,25 @@ struct DecodeCtl {
 // Starts the asynchronous fetch of the bitmap words a producer needs for one tile into the ring
 // slot `r`: the unit's words before the tile (direct units) or the tile's count from the scratch
 // (long units), and the tile's own words.  Nothing is held in registers meanwhile.
+template <bool FINE>
 __device__ __forceinline__ void fetch_bitmap(const TileDesc& td, uint32_t tile, uint32_t log2b, const uint8_t* msgs,
-                                             const uint32_t* ws_prefix, DecodeRing* r, uint32_t lane) {
+                                             const uint32_t* ws_prefix, DecodeRing<FINE>* r, uint32_t lane) {
     const uint32_t* bm32 = reinterpret_cast<const uint32_t*>(msgs + td.msg_off);
     const uint64_t kb0 = ((uint64_t)td.tile_in_unit * kTileValues) >> log2b;  // first block of the tile
     const uint64_t nb = num_blocks(td.n_unit, log2b);
     const uint32_t nbt = kTileValues >> log2b;
+    if (FINE) {
+        // every unit of more than one tile has its counts in the scratch; the tile's own flags are
+        // 128 to 1024 bytes that start on a 128-byte boundary of the slot: 16 bytes per copy,
+        // never past the bitmap's padded end
+        if (td.tile_in_unit != 0 && lane == 0) cp_async4(&r->ws, ws_prefix + tile);
+        const uint32_t chunks = nbt >> 7;  // 8 .. 64 copies of four words
+        for (uint32_t c = lane; c < chunks; c += 32) {
+            const uint64_t w = (kb0 >> 5) + 4ull * c;
+            if ((w << 5) < nb) cp_async16(&r->bm[4u * c], bm32 + w);
+        }
+        return;
+    }
     if (nb <= kDirectBlocks) {
         const uint32_t nwords = (uint32_t)((kb0 + 31) >> 5);  // words holding bits before kb0
 #pragma unroll
@@ -107,7 +142,8 @@ __device__ __forceinline__ void fetch_bitmap(const TileDesc& td, uint32_t tile, 
 
 // Turns a completed fetch into the tile's block flags (r->bm, r->pre).  Returns the number of
 // changed blocks before the tile; `own_total` gets the number of changed blocks of the tile.
-__device__ __forceinline__ uint64_t digest_bitmap(DecodeRing* r, const TileDesc& td, uint32_t log2b, uint32_t lane,
+template <bool FINE>
+__device__ __forceinline__ uint64_t digest_bitmap(DecodeRing<FINE>* r, const TileDesc& td, uint32_t log2b, uint32_t lane,
                                                   uint32_t& own_total) {
     const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
     const uint64_t kb0 = v0 >> log2b;
@@ -116,6 +152,32 @@ __device__ __forceinline__ uint64_t digest_bitmap(DecodeRing* r, const TileDesc&
     const uint32_t nv = (uint32_t)min((uint64_t)kTileValues, td.n_unit - v0);
     const uint32_t nblk = (nv + (1u << log2b) - 1u) >> log2b;  // valid blocks of this tile
     uint32_t cnt = 0;
+    if (FINE) {
+        // flags past the tile's last block are dropped (words past the bitmap's end were not fetched)
+        uint32_t run = 0;
+        for (uint32_t base = 0; base < (nbt >> 5); base += 32) {
+            const uint32_t w = base + lane;
+            uint32_t word = 0;
+            if (w * 32u < nblk) {
+                word = r->bm[w];
+                const uint32_t left = nblk - w * 32u;
+                if (left < 32u) word &= (1u << left) - 1u;
+            }
+            const uint32_t pc = __popc(word);
+            uint32_t incl = pc;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+                if ((int)lane >= o) incl += t;
+            }
+            r->bm[w] = word;
+            r->pre[w] = (uint16_t)(run + incl - pc);
+            run += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        own_total = run;
+        __syncwarp();
+        return td.tile_in_unit != 0 ? r->ws : 0u;
+    }
     if (nb <= kDirectBlocks) {
         const uint32_t nfull = (uint32_t)(kb0 >> 5);
 #pragma unroll
@@ -150,7 +212,7 @@ __device__ __forceinline__ uint64_t digest_bitmap(DecodeRing* r, const TileDesc&
     }
     if (lane < kBitmapWords) {
         r->bm[lane] = word;
-        r->pre[lane] = incl - pc;
+        r->pre[lane] = (uint16_t)(incl - pc);
     }
     own_total = __shfl_sync(0xffffffffu, incl, 31);
     __syncwarp();
@@ -177,24 +239,73 @@ __device__ __forceinline__ void unchanged_span(const uint32_t* bm, uint32_t log2
     hi = wl * 32u + 31u - (uint32_t)__clz(zl);
 }
 
-template <int DT>
-__global__ void __launch_bounds__(kDecodeThreads, DecodeCfg<DT>::kBlocksPerSM)
+// The same for fine blocks (32 to 256 words of flags; lane l looks at words l, l + 32, ...).
+__device__ __forceinline__ void unchanged_span_fine(const uint32_t* bm, uint32_t log2b, uint32_t lane, uint32_t& lo,
+                                                    uint32_t& hi) {
+    const uint32_t nwords = kTileValues >> (log2b + 5);
+    uint32_t first = 0xffffffffu, last = 0;
+    bool any = false;
+    for (uint32_t w = lane; w < nwords; w += 32) {
+        const uint32_t zeros = ~bm[w];
+        if (zeros) {
+            if (!any) first = w * 32u + (uint32_t)__ffs(zeros) - 1u;
+            last = w * 32u + 31u - (uint32_t)__clz(zeros);
+            any = true;
+        }
+    }
+    if (!__any_sync(0xffffffffu, any)) {
+        lo = 1;
+        hi = 0;
+        return;
+    }
+    lo = __reduce_min_sync(0xffffffffu, first);
+    hi = __reduce_max_sync(0xffffffffu, last);
+}
+
+// Exponents of the changed blocks of one piece, fine blocks: `km` holds the piece's block flags,
+// `src` points at the exponents of its first changed block; they replace the cached exponents in
+// x.e value by value.  Only the first nvalid values exist.
+template <int DT, class M>
+__device__ __forceinline__ void gather_changed(Piece<DT>& x, uint32_t km, uint32_t log2b, const uint8_t* src, int nvalid) {
+    uint32_t cnt = 0;
+#pragma unroll
+    for (int i = 0; i < Piece<DT>::kValues; ++i) {
+        if ((km >> ((uint32_t)i >> log2b)) & 1u) {
+            if (i < nvalid) {
+                const uint32_t b = M::ld1(src + cnt);
+                // byte (i & 3) of the word <- b
+                const uint32_t sel = (i & 3) == 0 ? 0x3214u : (i & 3) == 1 ? 0x3240u : (i & 3) == 2 ? 0x3410u : 0x4210u;
+                x.e[i >> 2] = __byte_perm(x.e[i >> 2], b, sel);
+            }
+            ++cnt;
+        }
+    }
+}
+
+template <int DT, bool FINE>
+__global__ void __launch_bounds__(kDecodeThreads, DecodeCfg<DT, FINE>::kBlocksPerSM)
 decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log2b, const uint8_t* msgs, uint8_t* cache,
               uint8_t* __restrict__ weights, const unsigned long long* __restrict__ wire_bytes,
               const uint32_t* __restrict__ ws_prefix, unsigned int* ticket, int32_t* status) {
     using P = Piece<DT>;
     constexpr int VB = Traits<DT>::kValueBytes;
     constexpr int SMB = Traits<DT>::kSmBytes;
-    constexpr int S = DecodeCfg<DT>::kStages;
+    using Cfg = DecodeCfg<DT, FINE>;
+    constexpr int S = Cfg::kStages;
+    constexpr int kDecRing = Cfg::kRing;
     static_assert(S % kDecProducers == 0, "every producer cycles through stages of its own");
-    constexpr bool kStageOut = DecodeCfg<DT>::kStageOut;
+    static_assert(kDecRing > S + 2 * kDecProducers + 1, "a slot is refilled only after its tile is done");
+    constexpr bool kStageOut = Cfg::kStageOut;
     constexpr uint32_t kSmTile = kTileValues * SMB;                   // sign-plus-mantissa of a tile
-    constexpr uint32_t kStageBytes = kSmTile + 2u * kTileValues;       // + cache span + payload slice
+    // + cache span + payload slice (which, with fine blocks, need not start on a 16-byte boundary)
+    constexpr uint32_t kStageBytes = kSmTile + 2u * kTileValues + (FINE ? 16u : 0u);
     constexpr uint32_t kOutBytes = kStageOut ? kTileValues * VB : 0u;  // reconstructed tile, staged for bulk stores
     constexpr uint32_t kWarpOutBytes = 32 * P::kValues * VB;           // one warp's contiguous slice of it
     extern __shared__ __align__(128) uint8_t smem[];
     uint8_t* const s_out = smem + (size_t)S * kStageBytes;
-    DecodeCtl<S>* ctl = reinterpret_cast<DecodeCtl<S>*>(s_out + kOutBytes);
+    using Ring = DecodeRing<FINE>;
+    using Ctl = DecodeCtl<S, kDecRing, FINE>;
+    Ctl* ctl = reinterpret_cast<Ctl*>(s_out + kOutBytes);
 
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     volatile int* abort = &ctl->abort;
@@ -227,7 +338,7 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
         // words one slot ahead, both by per-thread asynchronous copies (groups D_j and B_j, committed
         // in the order D_0 D_1 B_0 | D_2 B_1 | D_3 B_2 | ...)
         auto fetch_desc = [&](uint32_t jj, uint32_t tile) {
-            DecodeRing* r = &ctl->ring[seq(jj) % kDecRing];
+            Ring* r = &ctl->ring[seq(jj) % kDecRing];
             if (lane == 0) r->tile = tile;
             if (tile != kNoTile && lane < 3)
                 cp_async16(reinterpret_cast<uint8_t*>(&r->desc) + 16u * lane,
@@ -259,12 +370,12 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
             cp_async_wait<1>();  // everything but D_{jj+2}: D_{jj+1} and B_jj have landed
             __syncwarp();
             if (t_nxt != kNoTile) {
-                DecodeRing* rn = &ctl->ring[seq(jj + 1u) % kDecRing];
+                Ring* rn = &ctl->ring[seq(jj + 1u) % kDecRing];
                 fetch_bitmap(rn->desc, t_nxt, log2b, msgs, ws_prefix, rn, lane);
             }
             cp_async_commit();
 
-            DecodeRing* r = &ctl->ring[k % kDecRing];
+            Ring* r = &ctl->ring[k % kDecRing];
             const TileDesc td = r->desc;
             uint32_t own = 0;
             const uint64_t before = digest_bitmap(r, td, log2b, lane, own);
@@ -277,7 +388,12 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
             uint8_t* st = smem + (size_t)stage * kStageBytes;
             const bool full_tile = N - v0 >= (uint64_t)kTileValues;
             uint32_t lo = 1, hi = 0;
-            if (full_tile) unchanged_span(r->bm, log2b, lane, lo, hi);
+            if (full_tile) {
+                if (FINE)
+                    unchanged_span_fine(r->bm, log2b, lane, lo, hi);
+                else
+                    unchanged_span(r->bm, log2b, lane, lo, hi);
+            }
 
             if (lane == 0) {
                 r->w_dst = weights + td.w_off;
@@ -300,14 +416,28 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                 }
 
                 if (full_tile) {
-                    const uint32_t span = lo <= hi ? (hi - lo + 1u) << log2b : 0u;
-                    const uint32_t slice = own << log2b;
+                    // bulk copies move whole 16-byte pieces: with fine blocks the span of cached
+                    // exponents and the payload slice are widened to such boundaries (the tile's
+                    // cache is 16-byte aligned; the slice stays inside the unit's payload section,
+                    // which holds at least the values up to the end of this full tile)
+                    uint32_t span0 = lo << log2b, span = lo <= hi ? (hi - lo + 1u) << log2b : 0u;
+                    uint32_t skew = 0, slice = own << log2b;
+                    if (FINE) {
+                        if (span) {
+                            const uint32_t end = (span0 + span + 15u) & ~15u;
+                            span0 &= ~15u;
+                            span = end - span0;
+                        }
+                        if (slice) {
+                            skew = (uint32_t)((before << log2b) & 15ull);
+                            slice = (skew + slice + 15u) & ~15u;
+                        }
+                        r->pay_skew = skew;
+                    }
                     mbar_arrive_expect_tx(&ctl->full[stage], kSmTile + span + slice);
                     bulk_load(st, r->sm_src, kSmTile, &ctl->full[stage]);
-                    if (span)
-                        bulk_load(st + kSmTile + ((size_t)lo << log2b), r->c_ptr + ((size_t)lo << log2b), span,
-                                  &ctl->full[stage]);
-                    if (slice) bulk_load(st + kSmTile + kTileValues, pay, slice, &ctl->full[stage]);
+                    if (span) bulk_load(st + kSmTile + span0, r->c_ptr + span0, span, &ctl->full[stage]);
+                    if (slice) bulk_load(st + kSmTile + kTileValues, pay - skew, slice, &ctl->full[stage]);
                 } else {
                     mbar_arrive(&ctl->full[stage]);  // short tile: consumers read global memory themselves
                 }
@@ -327,7 +457,7 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
             const uint32_t stage = k % S;
             if (!mbar_wait(&ctl->full[stage], (k / S) & 1u, abort, status)) break;
             if (tid == 0) ctl->seen = k + 1;
-            const DecodeRing* r = &ctl->ring[k % kDecRing];
+            const Ring* r = &ctl->ring[k % kDecRing];
             if (r->tile == kNoTile) {
                 live &= ~(1u << (k % kDecProducers));
                 continue;
@@ -347,14 +477,26 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                     const uint32_t t0 = P::start(tid, p);
                     const uint32_t kb = t0 >> log2b;
                     const uint32_t word = r->bm[kb >> 5];
-                    const bool chg = (word >> (kb & 31u)) & 1u;
                     // exponents: the cached ones, or -- changed block -- the ones that came in the payload
                     const uint32_t rank = r->pre[kb >> 5] + __popc(word & ((1u << (kb & 31u)) - 1u));
-                    const uint8_t* esrc = chg ? st + kSmTile + kTileValues + ((size_t)rank << log2b) + (t0 & bmask)
-                                              : st + kSmTile + t0;
                     P x;
                     x.template load_sm_full<Shared>(st + (size_t)t0 * SMB);
-                    x.template load_exp_full<Shared>(esrc);
+                    bool chg;
+                    if (!FINE) {
+                        chg = (word >> (kb & 31u)) & 1u;
+                        const uint8_t* esrc = chg ? st + kSmTile + kTileValues + ((size_t)rank << log2b) + (t0 & bmask)
+                                                  : st + kSmTile + t0;
+                        x.template load_exp_full<Shared>(esrc);
+                    } else {
+                        // the piece's flags (they never straddle a word) pick, block by block
+                        const uint32_t km = (word >> (kb & 31u)) & ((1u << (P::kValues >> log2b)) - 1u);
+                        chg = km != 0;
+                        x.template load_exp_full<Shared>(st + kSmTile + t0);
+                        if (chg)
+                            gather_changed<DT, Shared>(x, km, log2b,
+                                                       st + kSmTile + kTileValues + r->pay_skew + ((size_t)rank << log2b),
+                                                       P::kValues);
+                    }
                     if (chg) x.template store_exp_full<Global>(c_ptr + t0);  // ExpCache[i,k] <- newExp[j]
                     if (kStageOut)
                         x.template merge_store_full<Shared>(s_out + (size_t)t0 * VB);
@@ -382,18 +524,23 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                     if (nvalid == 0) continue;
                     const uint32_t kb = t0 >> log2b;
                     const uint32_t word = r->bm[kb >> 5];
-                    const bool chg = (word >> (kb & 31u)) & 1u;
                     const uint32_t rank = r->pre[kb >> 5] + __popc(word & ((1u << (kb & 31u)) - 1u));
-                    const uint8_t* esrc = chg ? pay_src + ((size_t)rank << log2b) + (t0 & bmask) : c_ptr + t0;
+                    // coarse: the piece's block; fine: the piece's blocks, picked one by one below
+                    const uint32_t km = FINE ? (word >> (kb & 31u)) & ((1u << (P::kValues >> log2b)) - 1u)
+                                             : (word >> (kb & 31u)) & 1u;
+                    const bool chg = km != 0;
+                    const uint8_t* esrc = (chg && !FINE) ? pay_src + ((size_t)rank << log2b) + (t0 & bmask) : c_ptr + t0;
                     P x;
                     if (nvalid == P::kValues) {
                         x.template load_sm_full<Global>(sm_src + (size_t)t0 * SMB);
                         x.template load_exp_full<Global>(esrc);
+                        if (FINE && chg) gather_changed<DT, Global>(x, km, log2b, pay_src + ((size_t)rank << log2b), nvalid);
                         if (chg) x.template store_exp_full<Global>(c_ptr + t0);
                         x.template merge_store_full<Global>(w_dst + (size_t)t0 * VB);
                     } else {
                         x.load_sm_partial(sm_src + (size_t)t0 * SMB, nvalid);
                         x.load_exp_partial(esrc, nvalid);
+                        if (FINE && chg) gather_changed<DT, Global>(x, km, log2b, pay_src + ((size_t)rank << log2b), nvalid);
                         if (chg) x.store_exp_partial(c_ptr + t0, nvalid);
                         x.merge_store_partial(w_dst + (size_t)t0 * VB, nvalid);
                     }
@@ -468,15 +615,16 @@ decode_prefix_kernel(const TileDesc* __restrict__ tiles, const uint32_t* __restr
     }
 }
 
-template <int DT>
+template <int DT, bool FINE>
 static size_t decode_smem_bytes() {
-    constexpr int S = DecodeCfg<DT>::kStages;
-    const size_t stage = (size_t)kTileValues * Traits<DT>::kSmBytes + 2u * kTileValues;
-    const size_t out = DecodeCfg<DT>::kStageOut ? (size_t)kTileValues * Traits<DT>::kValueBytes : 0;
-    return (size_t)S * stage + out + sizeof(DecodeCtl<S>);
+    using Cfg = DecodeCfg<DT, FINE>;
+    constexpr int S = Cfg::kStages;
+    const size_t stage = (size_t)kTileValues * Traits<DT>::kSmBytes + 2u * kTileValues + (FINE ? 16u : 0u);
+    const size_t out = Cfg::kStageOut ? (size_t)kTileValues * Traits<DT>::kValueBytes : 0;
+    return (size_t)S * stage + out + sizeof(DecodeCtl<S, Cfg::kRing, FINE>);
 }
 
-template <int DT>
+template <int DT, bool FINE>
 static int decode_grid_limit(int* out) {
     static int cached[64] = {0};
     int dev = 0;
@@ -484,11 +632,11 @@ static int decode_grid_limit(int* out) {
     if (e != cudaSuccess) return record_cuda_error(e);
     if (dev < 0 || dev >= 64) return CIERA_ERR_UNSUPPORTED;
     if (cached[dev] == 0) {
-        const size_t smem = decode_smem_bytes<DT>();
-        e = cudaFuncSetAttribute(decode_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        const size_t smem = decode_smem_bytes<DT, FINE>();
+        e = cudaFuncSetAttribute(decode_kernel<DT, FINE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return record_cuda_error(e);
         int per_sm = 0, sms = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_kernel<DT>, kDecodeThreads, smem);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_kernel<DT, FINE>, kDecodeThreads, smem);
         if (e != cudaSuccess) return record_cuda_error(e);
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return record_cuda_error(e);
@@ -497,6 +645,22 @@ static int decode_grid_limit(int* out) {
     }
     *out = cached[dev];
     return CIERA_OK;
+}
+
+template <int DT, bool FINE>
+static int launch_decode(const ciera_plan* p, const void* messages_dev, void* receiver_cache_dev, void* weights_out_dev,
+                         const uint64_t* wire_bytes_dev, void* workspace_dev, unsigned int* ticket, int32_t* status_dev,
+                         cudaStream_t s) {
+    int limit = 0;
+    const int rc = decode_grid_limit<DT, FINE>(&limit);
+    if (rc) return rc;
+    const uint32_t nt = (uint32_t)p->tiles.size();
+    const uint32_t grid = nt < (uint32_t)limit ? nt : (uint32_t)limit;
+    decode_kernel<DT, FINE><<<grid, kDecodeThreads, decode_smem_bytes<DT, FINE>(), s>>>(
+        p->tiles_dev, nt, p->log2b, (const uint8_t*)messages_dev, (uint8_t*)receiver_cache_dev, (uint8_t*)weights_out_dev,
+        (const unsigned long long*)wire_bytes_dev, (const uint32_t*)workspace_dev, ticket, status_dev);
+    count_launch();
+    return check_launch();
 }
 
 }  // namespace ciera
@@ -530,20 +694,14 @@ extern "C" int ciera_decode(const ciera_plan* p, const void* messages_dev, void*
         int rc = check_launch();
         if (rc) return rc;
     }
-    int limit = 0;
-    int rc = p->dtype == CIERA_BF16 ? decode_grid_limit<CIERA_BF16>(&limit) : decode_grid_limit<CIERA_FP32>(&limit);
-    if (rc) return rc;
-    const uint32_t grid = nt < (uint32_t)limit ? nt : (uint32_t)limit;
+    const bool fine = is_fine(p->log2b);
     if (p->dtype == CIERA_BF16)
-        decode_kernel<CIERA_BF16><<<grid, kDecodeThreads, decode_smem_bytes<CIERA_BF16>(), s>>>(
-            p->tiles_dev, nt, p->log2b, (const uint8_t*)messages_dev, (uint8_t*)receiver_cache_dev,
-            (uint8_t*)weights_out_dev, (const unsigned long long*)wire_bytes_dev, (const uint32_t*)workspace_dev, ticket,
-            status_dev);
-    else
-        decode_kernel<CIERA_FP32><<<grid, kDecodeThreads, decode_smem_bytes<CIERA_FP32>(), s>>>(
-            p->tiles_dev, nt, p->log2b, (const uint8_t*)messages_dev, (uint8_t*)receiver_cache_dev,
-            (uint8_t*)weights_out_dev, (const unsigned long long*)wire_bytes_dev, (const uint32_t*)workspace_dev, ticket,
-            status_dev);
-    count_launch();
-    return check_launch();
+        return fine ? launch_decode<CIERA_BF16, true>(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,
+                                                      workspace_dev, ticket, status_dev, s)
+                    : launch_decode<CIERA_BF16, false>(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,
+                                                       workspace_dev, ticket, status_dev, s);
+    return fine ? launch_decode<CIERA_FP32, true>(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,
+                                                  workspace_dev, ticket, status_dev, s)
+                : launch_decode<CIERA_FP32, false>(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,
+                                                   workspace_dev, ticket, status_dev, s);
 }

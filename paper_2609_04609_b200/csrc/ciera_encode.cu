@@ -43,20 +43,40 @@ constexpr int kProducerWarp = kWarps;                            // 16
 constexpr int kAggregatorWarp = kWarps + 1;                      // 17
 constexpr int kResolverWarp0 = kWarps + 2;                       // 18 ..
 constexpr int kDescRing = 16;                                    // > exponent stages + 2
-constexpr int kDefer = 3;       // consumers send a tile's changed exponents this many tiles later
 constexpr int kVoteWords = 32;  // vote bits of a tile: up to 1024 pieces
 
-template <int DT>
+// Ring depths; kDefer = consumers send a tile's changed exponents this many tiles later.  With
+// fine blocks (see ciera_internal.cuh) a tile has up to 8192 block flags instead of 512, and the
+// exponent ring gives up a stage to make room for them (two thread blocks share an SM).
+template <int DT, bool FINE>
 struct EncodeCfg;
 template <>
-struct EncodeCfg<CIERA_BF16> {
+struct EncodeCfg<CIERA_BF16, false> {
     static constexpr int kWStages = 3;  // 3 x 16 KB weights tiles
     static constexpr int kEStages = 7;  // 7 x  8 KB exponent tiles
+    static constexpr int kDefer = 3;
+    static constexpr int kBmWords = kBitmapWords;
 };
 template <>
-struct EncodeCfg<CIERA_FP32> {
+struct EncodeCfg<CIERA_FP32, false> {
     static constexpr int kWStages = 2;  // 2 x 32 KB
     static constexpr int kEStages = 5;  // 5 x  8 KB
+    static constexpr int kDefer = 3;
+    static constexpr int kBmWords = kBitmapWords;
+};
+template <>
+struct EncodeCfg<CIERA_BF16, true> {
+    static constexpr int kWStages = 3;
+    static constexpr int kEStages = 6;
+    static constexpr int kDefer = 3;
+    static constexpr int kBmWords = kFineBitmapWords;
+};
+template <>
+struct EncodeCfg<CIERA_FP32, true> {
+    static constexpr int kWStages = 2;
+    static constexpr int kEStages = 4;
+    static constexpr int kDefer = 2;
+    static constexpr int kBmWords = kFineBitmapWords;
 };
 
 // What the consumers need of a tile, worked out once by the producer thread instead of by each
@@ -70,7 +90,7 @@ struct __align__(16) EncodeTileInfo {
     uint32_t pad[3];
 };
 
-template <int SW, int SE>
+template <int SW, int SE, int BW>
 struct EncodeCtl {
     uint64_t full_w[SW];    // weights tile landed
     uint64_t empty_w[SW];   // all 16 consumer warps have read it
@@ -83,9 +103,9 @@ struct EncodeCtl {
     EncodeTileInfo info[kDescRing];
     uint32_t tile_idx[kDescRing];  // table index of the tile in desc[]; kNoTile = end marker
     uint32_t seq[kDescRing];       // 1: tile of a unit this block works through alone
-    uint32_t ballot[SE][kVoteWords];
-    uint32_t bm[SE][kBitmapWords];
-    uint32_t pre[SE][kBitmapWords];
+    uint32_t ballot[SE][kVoteWords];  // coarse blocks: "my piece differs" votes
+    uint32_t bm[SE][BW];              // block flags of the tile
+    uint16_t pre[SE][BW];             // set flags before each word of bm
     unsigned long long agg[SE];
     unsigned long long base[SE];
     int abort;
@@ -168,7 +188,7 @@ __device__ __forceinline__ uint64_t warp_sum_u64(uint64_t v) {
 // Block flags of a tile from the vote bits "my piece differs" (one warp).  `pl2` = log2 of the
 // values per piece.  Fills bm (one bit per block of the tile) and pre (set bits before each word);
 // returns the number of changed blocks of the tile.
-__device__ __forceinline__ uint32_t build_block_bitmap(const uint32_t* ballot, uint32_t* bm, uint32_t* pre,
+__device__ __forceinline__ uint32_t build_block_bitmap(const uint32_t* ballot, uint32_t* bm, uint16_t* pre,
                                                        uint32_t log2b, uint32_t pl2, uint32_t lane) {
     const uint32_t gl2 = log2b - pl2;           // log2(pieces per block)
     const uint32_t nbt = kTileValues >> log2b;  // blocks of a full tile
@@ -192,9 +212,29 @@ __device__ __forceinline__ uint32_t build_block_bitmap(const uint32_t* ballot, u
         const uint32_t word = __ballot_sync(0xffffffffu, f);
         if (lane == 0) {
             bm[base >> 5] = word;
-            pre[base >> 5] = run;
+            pre[base >> 5] = (uint16_t)run;
         }
         run += __popc(word);
+    }
+    __syncwarp();
+    return run;
+}
+
+// Fine blocks: the consumers have written the block flags themselves; fills pre (set bits before
+// each word) and returns the number of changed blocks of the tile (one warp).
+__device__ __forceinline__ uint32_t scan_block_bitmap(const uint32_t* bm, uint16_t* pre, uint32_t log2b, uint32_t lane) {
+    const uint32_t nwords = kTileValues >> (log2b + 5);  // 32 .. 256
+    uint32_t run = 0;
+    for (uint32_t base = 0; base < nwords; base += 32) {
+        const uint32_t pc = __popc(bm[base + lane]);
+        uint32_t incl = pc;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+            if ((int)lane >= o) incl += t;
+        }
+        pre[base + lane] = (uint16_t)(run + incl - pc);
+        run += __shfl_sync(0xffffffffu, incl, 31);
     }
     __syncwarp();
     return run;
@@ -203,9 +243,9 @@ __device__ __forceinline__ uint32_t build_block_bitmap(const uint32_t* ballot, u
 // Aggregator warp, one tile: block flags, the tile's bitmap bytes, the tile's payload byte count.
 // With `publish` the count goes out at once as the tile's status word, so that later tiles never
 // wait for it longer than for the votes themselves.  Waits for nothing outside the thread block.
-template <int DT>
+template <int DT, bool FINE>
 __device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t tile, uint32_t log2b, bool publish,
-                                                   const uint32_t* ballot, uint32_t* bm, uint32_t* pre, uint8_t* msgs,
+                                                   const uint32_t* ballot, uint32_t* bm, uint16_t* pre, uint8_t* msgs,
                                                    unsigned long long* tile_status, uint32_t lane) {
     const uint64_t N = td.n_unit;
     const uint32_t B = 1u << log2b;
@@ -214,7 +254,8 @@ __device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t 
     const uint32_t nv = (uint32_t)min((uint64_t)kTileValues, N - v0);
     uint8_t* msg = msgs + td.msg_off;
 
-    const uint32_t run = build_block_bitmap(ballot, bm, pre, log2b, Piece<DT>::kLog2Values, lane);
+    const uint32_t run = FINE ? scan_block_bitmap(bm, pre, log2b, lane)
+                              : build_block_bitmap(ballot, bm, pre, log2b, Piece<DT>::kLog2Values, lane);
 
     // payload bytes of this tile: B per changed block, less for a changed short last block
     uint64_t agg = (uint64_t)run << log2b;
@@ -230,7 +271,15 @@ __device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t 
         if (lane == 0) st_status(tile_status + tile, flag | ((unsigned long long)mybits << kBitsShift) | agg);
     }
     // bitmap bytes of this tile (tiles of >= 8 blocks own whole bytes)
-    if (nbt >= 8) {
+    if (FINE) {
+        // at least 128 bytes per full tile, starting on a 128-byte boundary of the (16-byte aligned) slot
+        const uint64_t byte0 = (uint64_t)td.tile_in_unit * (nbt >> 3);
+        const uint32_t nbytes = (((nv + B - 1u) >> log2b) + 7u) >> 3;
+        uint32_t* dst32 = reinterpret_cast<uint32_t*>(msg + byte0);
+        for (uint32_t w = lane; w < (nbytes >> 2); w += 32) dst32[w] = bm[w];
+        const uint32_t done = nbytes & ~3u;
+        if (lane < nbytes - done) msg[byte0 + done + lane] = (uint8_t)(bm[done >> 2] >> (lane * 8u));
+    } else if (nbt >= 8) {
         const uint64_t byte0 = (uint64_t)td.tile_in_unit * (nbt >> 3);
         const uint32_t nbytes = (((nv + B - 1u) >> log2b) + 7u) >> 3;
         for (uint32_t b = lane; b < nbytes; b += 32) msg[byte0 + b] = (uint8_t)(bm[b >> 2] >> ((b & 3u) * 8u));
@@ -312,7 +361,7 @@ __device__ __forceinline__ uint64_t resolve_tile(const TileDesc& td, uint32_t ti
 // tile) if their block changed; `base` is the tile's exclusive offset in the unit's payload.
 template <int DT>
 __device__ __forceinline__ void write_changed(const EncodeTileInfo& ti, uint32_t log2b, const uint32_t* bm,
-                                              const uint32_t* pre, uint64_t base, const uint8_t* s_exp, uint32_t tid) {
+                                              const uint16_t* pre, uint64_t base, const uint8_t* s_exp, uint32_t tid) {
     using P = Piece<DT>;
 #pragma unroll
     for (int p = 0; p < P::kPerThread; ++p) {
@@ -337,7 +386,84 @@ __device__ __forceinline__ void write_changed(const EncodeTileInfo& ti, uint32_t
     }
 }
 
-template <int DT>
+// One block of B = 2^LB (fine) exponent bytes, shared -> global; both addresses are B-aligned.
+template <int LB>
+__device__ __forceinline__ void copy_block(uint8_t* dst, const uint8_t* s_src) {
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(s_src);
+    if (LB == 0) {
+        uint32_t v;
+        asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(a));
+        __stcs(dst, (uint8_t)v);
+    } else if (LB == 1) {
+        uint16_t v;
+        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
+        __stcs(reinterpret_cast<uint16_t*>(dst), v);
+    } else if (LB == 2) {
+        uint32_t v;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+        __stcs(reinterpret_cast<uint32_t*>(dst), v);
+    } else {
+        st_stream8(dst, ld_shared8(s_src));
+    }
+}
+
+// The same duty with fine blocks: a piece holds K = values-per-piece / B blocks with one flag each;
+// the exponents of its changed blocks lie next to each other in the payload, starting at the rank
+// of the piece's first changed block.
+template <int DT, int LB>
+__device__ __forceinline__ void write_changed_fine(const EncodeTileInfo& ti, const uint32_t* bm, const uint16_t* pre,
+                                                   uint64_t base, const uint8_t* s_exp, uint32_t tid) {
+    using P = Piece<DT>;
+    constexpr uint32_t K = (uint32_t)P::kValues >> LB;  // 1 .. 16 blocks per piece
+    constexpr uint32_t B = 1u << LB;
+#pragma unroll
+    for (int p = 0; p < P::kPerThread; ++p) {
+        const uint32_t t0 = P::start(tid, p);
+        const int nvalid = piece_valid<DT>(t0, ti.nv);
+        if (nvalid == 0) continue;
+        const uint32_t kb = t0 >> LB;
+        const uint32_t word = bm[kb >> 5], sh = kb & 31u;
+        const uint32_t km = (word >> sh) & ((1u << K) - 1u);  // the piece's flags (they never straddle a word)
+        if (km == 0) continue;
+        const uint32_t rank = (uint32_t)pre[kb >> 5] + __popc(word & ((1u << sh) - 1u));
+        uint8_t* pdst = ti.pay_dst + base + ((uint64_t)rank << LB);
+#pragma unroll
+        for (uint32_t j = 0; j < K; ++j) {
+            if (!((km >> j) & 1u)) continue;
+            const int left = nvalid - (int)(j << LB);  // > 0: blocks past the unit's end are never flagged
+            if (left >= (int)B) {
+                copy_block<LB>(pdst, s_exp + t0 + (j << LB));
+            } else {
+                for (int i = 0; i < left; ++i) pdst[i] = s_exp[t0 + (j << LB) + i];  // the unit's short last block
+            }
+            pdst += B;
+        }
+        // unchanged blocks of the piece hold what the cache holds already: refresh the whole piece
+        P x;
+        x.template load_exp_full<Shared>(s_exp + t0);
+        if (nvalid == P::kValues)
+            x.template store_exp_full<Global>(ti.c_ptr + t0);
+        else
+            x.store_exp_partial(ti.c_ptr + t0, nvalid);
+    }
+}
+
+template <int DT, bool FINE>
+__device__ __forceinline__ void send_changed(const EncodeTileInfo& ti, uint32_t log2b, const uint32_t* bm,
+                                             const uint16_t* pre, uint64_t base, const uint8_t* s_exp, uint32_t tid) {
+    if (!FINE) {
+        write_changed<DT>(ti, log2b, bm, pre, base, s_exp, tid);
+    } else {
+        switch (log2b) {
+            case 0: write_changed_fine<DT, 0>(ti, bm, pre, base, s_exp, tid); break;
+            case 1: write_changed_fine<DT, 1>(ti, bm, pre, base, s_exp, tid); break;
+            case 2: write_changed_fine<DT, 2>(ti, bm, pre, base, s_exp, tid); break;
+            default: write_changed_fine<DT, 3>(ti, bm, pre, base, s_exp, tid); break;
+        }
+    }
+}
+
+template <int DT, bool FINE>
 __global__ void __launch_bounds__(kEncodeThreads, 2)
 encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32_t* __restrict__ seq_first,
               uint32_t n_short, uint32_t log2b, const uint8_t* __restrict__ weights, uint8_t* cache, uint8_t* msgs,
@@ -346,14 +472,18 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
     using P = Piece<DT>;
     constexpr int VB = Traits<DT>::kValueBytes;
     constexpr int SMB = Traits<DT>::kSmBytes;
-    constexpr int SW = EncodeCfg<DT>::kWStages;
-    constexpr int SE = EncodeCfg<DT>::kEStages;
+    using Cfg = EncodeCfg<DT, FINE>;
+    constexpr int SW = Cfg::kWStages;
+    constexpr int SE = Cfg::kEStages;
+    constexpr int kDefer = Cfg::kDefer;
+    static_assert(kDescRing > SE + 2 && SE > kDefer, "ring depths");
     constexpr uint32_t kWBytes = kTileValues * VB;
     constexpr uint32_t kEBytes = kTileValues;
     extern __shared__ __align__(128) uint8_t smem[];
     uint8_t* const ring_w = smem;
     uint8_t* const ring_e = smem + (size_t)SW * kWBytes;
-    EncodeCtl<SW, SE>* ctl = reinterpret_cast<EncodeCtl<SW, SE>*>(ring_e + (size_t)SE * kEBytes);
+    using Ctl = EncodeCtl<SW, SE, Cfg::kBmWords>;
+    Ctl* ctl = reinterpret_cast<Ctl*>(ring_e + (size_t)SE * kEBytes);
 
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     volatile int* abort = &ctl->abort;
@@ -450,7 +580,7 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
             }
             const TileDesc td = ctl->desc[k % kDescRing];
             const bool seq = ctl->seq[k % kDescRing] != 0;
-            const uint64_t agg = aggregate_tile<DT>(td, tile, log2b, !seq, ctl->ballot[se], ctl->bm[se], ctl->pre[se], msgs,
+            const uint64_t agg = aggregate_tile<DT, FINE>(td, tile, log2b, !seq, ctl->ballot[se], ctl->bm[se], ctl->pre[se], msgs,
                                                     tile_status, lane);
             if (seq) {
                 // the whole unit is this block's: the tile's offset is the running sum
@@ -533,8 +663,18 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
                     // leave the new exponents where the cached ones were staged: they are sent from
                     // there once the tile's place in the payload is known
                     x.template store_exp_full<Shared>(s_e + t0);
-                    const uint32_t bal = __ballot_sync(0xffffffffu, x.differs(c));
-                    if (lane == 0) ctl->ballot[se][p * kWarps + warp] = bal;
+                    if (!FINE) {
+                        const uint32_t bal = __ballot_sync(0xffffffffu, x.differs(c));
+                        if (lane == 0) ctl->ballot[se][p * kWarps + warp] = bal;
+                    } else {
+                        // K = values-per-piece / B flags per piece; the warp's 32 pieces fill K whole
+                        // words of the tile's block flags, 32 / K lanes to a word
+                        const uint32_t k_l2 = (uint32_t)P::kLog2Values - log2b;  // log2 K, 0 .. 4
+                        uint32_t v = x.block_flags(c, log2b) << ((lane << k_l2) & 31u);
+                        for (uint32_t o = 1; o < (32u >> k_l2); o <<= 1) v |= __shfl_xor_sync(0xffffffffu, v, o);
+                        if ((lane & ((32u >> k_l2) - 1u)) == 0)
+                            ctl->bm[se][((p * kWarps + warp) << k_l2) + (lane >> (5u - k_l2))] = v;
+                    }
                     // sign-plus-mantissa of every value
                     uint8_t* smdst = ti.sm_dst + (size_t)t0 * SMB;
                     if (nvalid == P::kValues)
@@ -553,8 +693,8 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
             if (k >= (uint32_t)kDefer && k - kDefer < k_end) {
                 const uint32_t j = k - kDefer, je = j % SE;
                 if (!mbar_wait(&ctl->resolved[je], (j / SE) & 1u, abort, status)) break;
-                write_changed<DT>(ctl->info[j % kDescRing], log2b, ctl->bm[je], ctl->pre[je], ctl->base[je],
-                                  ring_e + (size_t)je * kEBytes, tid);
+                send_changed<DT, FINE>(ctl->info[j % kDescRing], log2b, ctl->bm[je], ctl->pre[je], ctl->base[je],
+                                       ring_e + (size_t)je * kEBytes, tid);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&ctl->empty_e[je]);
             }
@@ -565,8 +705,8 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
             for (uint32_t j = k + 1u >= (uint32_t)kDefer ? k + 1u - kDefer : 0u; j < k_end; ++j) {
                 const uint32_t je = j % SE;
                 if (!mbar_wait(&ctl->resolved[je], (j / SE) & 1u, abort, status)) break;
-                write_changed<DT>(ctl->info[j % kDescRing], log2b, ctl->bm[je], ctl->pre[je], ctl->base[je],
-                                  ring_e + (size_t)je * kEBytes, tid);
+                send_changed<DT, FINE>(ctl->info[j % kDescRing], log2b, ctl->bm[je], ctl->pre[je], ctl->base[je],
+                                       ring_e + (size_t)je * kEBytes, tid);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&ctl->empty_e[je]);
             }
@@ -585,14 +725,16 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
     }
 }
 
-template <int DT>
+template <int DT, bool FINE>
 static size_t encode_smem_bytes() {
-    constexpr int SW = EncodeCfg<DT>::kWStages, SE = EncodeCfg<DT>::kEStages;
-    return (size_t)SW * kTileValues * Traits<DT>::kValueBytes + (size_t)SE * kTileValues + sizeof(EncodeCtl<SW, SE>);
+    using Cfg = EncodeCfg<DT, FINE>;
+    constexpr int SW = Cfg::kWStages, SE = Cfg::kEStages;
+    return (size_t)SW * kTileValues * Traits<DT>::kValueBytes + (size_t)SE * kTileValues +
+           sizeof(EncodeCtl<SW, SE, Cfg::kBmWords>);
 }
 
 // Largest grid whose blocks are all resident at once, per device (0 = not yet known).
-template <int DT>
+template <int DT, bool FINE>
 static int encode_grid_limit(int* out) {
     static int cached[64] = {0};
     int dev = 0;
@@ -600,11 +742,11 @@ static int encode_grid_limit(int* out) {
     if (e != cudaSuccess) return record_cuda_error(e);
     if (dev < 0 || dev >= 64) return CIERA_ERR_UNSUPPORTED;
     if (cached[dev] == 0) {
-        const size_t smem = encode_smem_bytes<DT>();
-        e = cudaFuncSetAttribute(encode_kernel<DT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        const size_t smem = encode_smem_bytes<DT, FINE>();
+        e = cudaFuncSetAttribute(encode_kernel<DT, FINE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return record_cuda_error(e);
         int per_sm = 0, sms = 0, coop = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, encode_kernel<DT>, kEncodeThreads, smem);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, encode_kernel<DT, FINE>, kEncodeThreads, smem);
         if (e != cudaSuccess) return record_cuda_error(e);
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return record_cuda_error(e);
@@ -618,12 +760,16 @@ static int encode_grid_limit(int* out) {
 }
 
 // `scratch`: one status word per tile, then the unit counter; all zero at kernel start.
-template <int DT>
-static int launch_encode(const ciera_plan* p, uint32_t grid, const void* weights_dev, void* sender_cache_dev,
-                         void* messages_dev, uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* scratch,
-                         int32_t* status_dev, cudaStream_t s) {
+template <int DT, bool FINE>
+static int launch_encode(const ciera_plan* p, const void* weights_dev, void* sender_cache_dev, void* messages_dev,
+                         uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* scratch, int32_t* status_dev,
+                         cudaStream_t s) {
+    int limit = 0;
+    const int rc = encode_grid_limit<DT, FINE>(&limit);
+    if (rc) return rc;
     const TileDesc* tiles = p->tiles_dev;
     uint32_t nt = (uint32_t)p->tiles.size();
+    const uint32_t grid = nt < (uint32_t)limit ? nt : (uint32_t)limit;
     const uint32_t* seq_first = p->seq_first_dev;
     uint32_t n_short = (uint32_t)p->seq_first.size() - 1u;
     uint32_t log2b = p->log2b;
@@ -640,16 +786,32 @@ static int launch_encode(const ciera_plan* p, uint32_t grid, const void* weights
         // GPU together, which is what the look-back between blocks relies on
         void* args[] = {&tiles, &nt, &seq_first, &n_short, &log2b, &w, &c, &m, &wb, &changed_blocks_dev, &ts, &ticket,
                         &status_dev};
-        e = cudaLaunchCooperativeKernel((const void*)encode_kernel<DT>, dim3(grid), dim3(kEncodeThreads), args,
-                                        encode_smem_bytes<DT>(), s);
+        e = cudaLaunchCooperativeKernel((const void*)encode_kernel<DT, FINE>, dim3(grid), dim3(kEncodeThreads), args,
+                                        encode_smem_bytes<DT, FINE>(), s);
     } else {
-        encode_kernel<DT><<<grid, kEncodeThreads, encode_smem_bytes<DT>(), s>>>(tiles, nt, seq_first, n_short, log2b, w, c, m,
-                                                                               wb, changed_blocks_dev, ts, ticket, status_dev);
+        encode_kernel<DT, FINE><<<grid, kEncodeThreads, encode_smem_bytes<DT, FINE>(), s>>>(
+            tiles, nt, seq_first, n_short, log2b, w, c, m, wb, changed_blocks_dev, ts, ticket, status_dev);
         e = cudaGetLastError();
     }
     if (e != cudaSuccess) return record_cuda_error(e);
     count_launch();
     return CIERA_OK;
+}
+
+// picks the kernel for the plan's precision and block class
+static int launch_encode_any(const ciera_plan* p, const void* weights_dev, void* sender_cache_dev, void* messages_dev,
+                             uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* scratch, int32_t* status_dev,
+                             cudaStream_t s) {
+    const bool fine = is_fine(p->log2b);
+    if (p->dtype == CIERA_BF16)
+        return fine ? launch_encode<CIERA_BF16, true>(p, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
+                                                      changed_blocks_dev, scratch, status_dev, s)
+                    : launch_encode<CIERA_BF16, false>(p, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
+                                                       changed_blocks_dev, scratch, status_dev, s);
+    return fine ? launch_encode<CIERA_FP32, true>(p, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
+                                                  changed_blocks_dev, scratch, status_dev, s)
+                : launch_encode<CIERA_FP32, false>(p, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
+                                                   changed_blocks_dev, scratch, status_dev, s);
 }
 
 }  // namespace ciera
@@ -679,18 +841,11 @@ extern "C" int ciera_encode(const ciera_plan* p, const void* weights_dev, void* 
     if (misaligned16(weights_dev) || misaligned16(sender_cache_dev) || misaligned16(messages_dev) ||
         misaligned16(workspace_dev) || ((uintptr_t)wire_bytes_dev & 7u) || ((uintptr_t)changed_blocks_dev & 3u))
         return CIERA_ERR_MISALIGNED;
-    int limit = 0;
-    int rc = p->dtype == CIERA_BF16 ? encode_grid_limit<CIERA_BF16>(&limit) : encode_grid_limit<CIERA_FP32>(&limit);
-    if (rc) return rc;
-    const uint32_t grid = nt < (uint32_t)limit ? nt : (uint32_t)limit;
     // scratch = one look-back status word per tile, then the unit counter; all of it starts at zero
     e = cudaMemsetAsync(workspace_dev, 0, sizeof(unsigned long long) * nt + 16, s);
     if (e != cudaSuccess) return record_cuda_error(e);
-    if (p->dtype == CIERA_BF16)
-        return launch_encode<CIERA_BF16>(p, grid, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
-                                         changed_blocks_dev, workspace_dev, status_dev, s);
-    return launch_encode<CIERA_FP32>(p, grid, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
-                                     changed_blocks_dev, workspace_dev, status_dev, s);
+    return launch_encode_any(p, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev, changed_blocks_dev,
+                             workspace_dev, status_dev, s);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -753,17 +908,10 @@ extern "C" int ciera_encode_noalloc(const ciera_plan* p, const void* weights_dev
     unsigned long long* scratch = nullptr;
     int rc = encode_scratch_address(&scratch);
     if (rc) return rc;
-    int limit = 0;
-    rc = p->dtype == CIERA_BF16 ? encode_grid_limit<CIERA_BF16>(&limit) : encode_grid_limit<CIERA_FP32>(&limit);
-    if (rc) return rc;
-    const uint32_t grid = nt < (uint32_t)limit ? nt : (uint32_t)limit;
     // the array keeps what the previous call left in it: the status words of this call's tiles and
     // the unit counter behind them have to start at zero
     e = cudaMemsetAsync(scratch, 0, sizeof(unsigned long long) * nt + 16, s);
     if (e != cudaSuccess) return record_cuda_error(e);
-    if (p->dtype == CIERA_BF16)
-        return launch_encode<CIERA_BF16>(p, grid, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
-                                         changed_blocks_dev, scratch, status_dev, s);
-    return launch_encode<CIERA_FP32>(p, grid, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
-                                     changed_blocks_dev, scratch, status_dev, s);
+    return launch_encode_any(p, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev, changed_blocks_dev, scratch,
+                             status_dev, s);
 }

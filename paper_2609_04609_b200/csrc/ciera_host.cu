@@ -120,7 +120,8 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
             t.n_tiles_unit = nt;
             p->tiles.push_back(t);
         }
-        if ((un.n_values + block - 1) / block > kDecodeDirectBlocks) p->long_units.push_back(first);
+        const bool needs_prefix = is_fine(p->log2b) ? nt > 1 : (un.n_values + block - 1) / block > kDecodeDirectBlocks;
+        if (needs_prefix) p->long_units.push_back(first);
     };
     for (uint32_t u : shorts) {
         p->seq_first.push_back((uint32_t)p->tiles.size());

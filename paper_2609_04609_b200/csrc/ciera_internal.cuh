@@ -18,8 +18,13 @@ constexpr int kThreads = 512;
 constexpr int kVPT = 16;
 constexpr int kTileValues = kThreads * kVPT;  // 8192
 constexpr int kWarps = kThreads / 32;
-constexpr int kMaxBlocksPerTile = kTileValues / CIERA_MIN_BLOCK;  // 512
-constexpr int kBitmapWords = kMaxBlocksPerTile / 32;              // 16
+// Block sizes come in two classes.  "Coarse" blocks (16 values and more) hold whole pieces, so a
+// piece has one flag and a tile at most 512 blocks; "fine" blocks (1, 2, 4 or 8 values) are
+// smaller than (or as large as) a piece, a piece has several flags and a tile up to 8192 blocks.
+constexpr uint32_t kFineLog2 = 4;                    // log2b < kFineLog2: fine
+constexpr int kBitmapWords = kTileValues / 16 / 32;  // 16: words of block flags of a tile, coarse
+constexpr int kFineBitmapWords = kTileValues / 32;   // 256: the same, fine
+__host__ __device__ inline bool is_fine(uint32_t log2b) { return log2b < kFineLog2; }
 
 // Device-side tile descriptor: everything a thread block needs, in one 48-byte record so that
 // a single dependent load stands between block start and the first data load.
@@ -71,7 +76,8 @@ __host__ __device__ inline uint64_t payload_offset(uint64_t n, uint32_t sm_bytes
 }
 
 // Units with more blocks than this get their per-tile "changed blocks before" counts from a
-// prefix kernel at decode time; shorter ones read them straight from the bitmap.
+// prefix kernel at decode time; shorter ones read them straight from the bitmap.  With fine
+// blocks every unit of more than one tile goes through the prefix kernel.
 constexpr uint32_t kDecodeDirectBlocks = 4096;
 
 // The tile table lists the tiles of "short" units (up to this many tiles) first, longest units
@@ -81,10 +87,12 @@ constexpr uint32_t kDecodeDirectBlocks = 4096;
 constexpr uint32_t kSeqMaxTiles = 32;
 
 // Bytes of a message slot that tile j of a unit moves in the transport kernel: [j * chunk,
-// (j + 1) * chunk); the unit's last tile also moves whatever lies beyond (bitmap and pads: the slot
-// capacity exceeds tiles * chunk by less than 100 bytes per unit plus one bitmap byte per 8 blocks).
-__host__ __device__ inline uint64_t transport_chunk_bytes(uint32_t sm_bytes_per_value) {
-    return (uint64_t)kTileValues * (sm_bytes_per_value + 1);
+// (j + 1) * chunk); the unit's last tile also moves whatever lies beyond (pads and, for coarse
+// blocks, the bitmap: less than 100 bytes per unit plus one bitmap byte per 8 blocks).  With fine
+// blocks the bitmap is a sizeable part of the message, so the chunk grows by a tile's share of it.
+__host__ __device__ inline uint64_t transport_chunk_bytes(uint32_t sm_bytes_per_value, uint32_t log2b) {
+    const uint64_t bitmap_share = is_fine(log2b) ? pad16((uint64_t)kTileValues >> (log2b + 3)) : 0;
+    return (uint64_t)kTileValues * (sm_bytes_per_value + 1) + bitmap_share;
 }
 
 }  // namespace ciera

@@ -43,7 +43,7 @@ cache_fill_kernel(const TileDesc* __restrict__ tiles, const uint8_t* __restrict_
 // A persistent copy kernel in which every warp works on its own: it draws tile numbers from a
 // counter in the caller's scratch (so all SMs stay busy to the end whatever their pace); tile j of
 // a unit moves bytes [j * chunk, (j + 1) * chunk) of the unit's slot (chunk = 16 KB for bf16, 32 KB
-// for fp32), the last tile also what lies beyond, cut off at the length the sender reported.  A warp moves 4 KB per step (eight 128-bit loads per lane in flight, then eight
+// for fp32, plus a tile's share of the bitmap when blocks are fine), the last tile also what lies beyond, cut off at the length the sender reported.  A warp moves 4 KB per step (eight 128-bit loads per lane in flight, then eight
 // stores); tile numbers, descriptors and reported lengths are fetched three, two and one tile
 // ahead, so that no step waits for them.
 
@@ -73,11 +73,10 @@ __device__ __forceinline__ CopyDesc load_copy_desc(const TileDesc* t) {
 }
 
 __global__ void __launch_bounds__(kCopyThreads)
-transport_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t sm_bytes_per_value,
+transport_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint64_t chunk,
                  const uint8_t* __restrict__ src, uint8_t* __restrict__ dst,
                  const unsigned long long* __restrict__ wire_bytes, unsigned int* ticket) {
     const uint32_t lane = threadIdx.x & 31u;
-    const uint64_t chunk = transport_chunk_bytes(sm_bytes_per_value);
     auto draw = [&]() {
         uint32_t t = 0;
         if (lane == 0) t = atomicAdd(ticket, 1u);
@@ -205,7 +204,7 @@ extern "C" int ciera_transport(const ciera_plan* p, const void* src_messages_dev
     const uint32_t want = (nt + kCopyThreads / 32 - 1) / (kCopyThreads / 32);
     const uint32_t grid = want < (uint32_t)limit ? want : (uint32_t)limit;
     transport_kernel<<<grid, kCopyThreads, 0, (cudaStream_t)stream>>>(
-        p->tiles_dev, nt, p->dtype == CIERA_BF16 ? 1u : 3u, (const uint8_t*)src_messages_dev, (uint8_t*)dst_messages_dev,
+        p->tiles_dev, nt, transport_chunk_bytes(p->dtype == CIERA_BF16 ? 1u : 3u, p->log2b), (const uint8_t*)src_messages_dev, (uint8_t*)dst_messages_dev,
         (const unsigned long long*)wire_bytes_dev, ticket);
     count_launch();
     return check_launch();

@@ -85,7 +85,7 @@ RAGGED = [0, 1, 15, 16, 17, 31, 33, 511, 512, 513, 1000, 4095, 4097, 8191, 8192,
 
 
 @pytest.mark.parametrize("dtype", [0, 1])
-@pytest.mark.parametrize("block", [16, 32, 64, 128, 256, 512, 1024, 2048, 4096])
+@pytest.mark.parametrize("block", [1, 2, 4, 8, 16, 32, 64, 128, 256, 512, 1024, 2048, 4096])
 def test_ragged_units_every_block_size(rt, dtype, block):
     """Units shorter than a block, not multiples of 16 / of the block / of the tile, empty units;
     random bit patterns (NaN, Inf, subnormals, both zeros included)."""
@@ -109,7 +109,8 @@ def test_zero_initialised_caches(rt, dtype):
 
 
 @pytest.mark.parametrize("block,c,seg", [(512, 0.001, 0), (64, 0.01, 0), (4096, 0.3, 4096), (2048, 0.0005, 0),
-                                         (1024, 0.5, 0), (16, 0.05, 0)])
+                                         (1024, 0.5, 0), (16, 0.05, 0), (1, 0.03, 0), (2, 0.0005, 0), (4, 0.4, 0),
+                                         (8, 0.01, 0), (1, 0.6, 0)])
 def test_long_units_look_back_over_many_tiles(rt, block, c, seg):
     """One unit of ~3 M values = 367 tiles (more than ten look-back windows) and a second,
     shorter one; exponent changes injected at an exact rate."""
@@ -119,6 +120,20 @@ def test_long_units_look_back_over_many_tiles(rt, block, c, seg):
     w1 = wl.inject_exponent_changes(w0, gen, c, seg)
     w2 = wl.inject_exponent_changes(w1, gen, c, seg)
     _run_trajectory(rt, codec, table, [wl.as_bits(w) for w in (w0, w1, w2)], 0, label=f"long-B{block}")
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("block", [1, 2, 4, 8])
+def test_small_blocks_on_a_reduced_moe_layer(rt, dtype, block):
+    """Blocks of 1 to 8 values (B = 1: one bitmap bit per value, the payload holds exactly the
+    exponents that changed) on 2 experts x 3 matrices x 4 shards plus ragged dense tensors, under the
+    Adam-like update (a few per cent of the exponents change) and from zero caches."""
+    sizes = [r * c for r, c in wl.olmoe_layer_shapes(2)] + [70_001, 8192, 8191, 17, 0, 40_000]
+    codec, table, n = _make(rt, sizes, 4, dtype, block)
+    traj = [wl.as_bits(w) for w in wl.trajectory(n, NAME[dtype], 500 + block, 3, "adam")]
+    stats = _run_trajectory(rt, codec, table, traj, dtype, label=f"small-{NAME[dtype]}-B{block}")
+    assert 0 < stats[-1][0] < stats[-1][1]
+    _run_trajectory(rt, codec, table, traj[:2], dtype, zero_cache=True, label=f"small-zero-{NAME[dtype]}-B{block}")
 
 
 def test_change_rate_sweep_mixed_shapes(rt):

@@ -58,7 +58,9 @@ def test_plan_validation(ciera):
     cap = ciera.message_capacity(1000, 0, 512)
     good = _units([(1000, 0, 0, 0, cap)])
     assert ciera.Plan(good, 0, 512).n_tiles == 1
-    for block in (0, 3, 8, 100, 8192):
+    for block in (1, 2, 4, 8, 16, 4096):
+        assert ciera.Plan(_units([(1000, 0, 0, 0, ciera.message_capacity(1000, 0, block))]), 0, block).n_tiles == 1
+    for block in (0, 3, 100, 8192):
         with pytest.raises(ciera.CieraError) as e:
             ciera.Plan(good, 0, block)
         assert e.value.status in (ciera.ERR_INVALID_ARG, ciera.ERR_UNSUPPORTED)
