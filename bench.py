@@ -203,12 +203,14 @@ def layer_numels(args):
     return [r * c for r, c in wl.olmoe_layer_shapes(args.experts)]
 
 
-def algorithmic_bytes(n_values, q, dtype):
-    """HBM bytes per launch the method needs: (encode, transport, decode)."""
+def algorithmic_bytes(n_values, q, dtype, block):
+    """HBM bytes per launch the method needs: (encode, transport, decode).  q = share of the
+    exponent bytes that travel (changed blocks); the bitmap is one bit per block."""
     vb, smb = (2, 1) if dtype == "bf16" else (4, 3)
-    enc = n_values * (vb + 1 + smb + 2 * q)
-    tra = 2 * n_values * (smb + q)
-    dec = n_values * (smb + (1 - q) + q + vb + q)
+    bm = 1.0 / (8 * block)
+    enc = n_values * (vb + 1 + smb + bm + 2 * q)
+    tra = 2 * n_values * (smb + bm + q)
+    dec = n_values * (smb + bm + (1 - q) + q + vb + q)
     return enc, tra, dec
 
 
@@ -451,7 +453,7 @@ def main():
     enc_ms, tra_ms, dec_ms = [float(np.mean([t[2 * i].elapsed_time(t[2 * i + 1]) for t in serial_timers]))
                               for i in range(3)]
     n_layer = layers[0].plan.total_values
-    a_enc, a_tra, a_dec = algorithmic_bytes(n_layer, q, args.dtype)
+    a_enc, a_tra, a_dec = algorithmic_bytes(n_layer, q, args.dtype, args.block)
     enc_gbs = a_enc / (enc_ms * 1e-3) / 1e9
     dec_gbs = a_dec / (dec_ms * 1e-3) / 1e9
     tra_gbs = a_tra / (tra_ms * 1e-3) / 1e9
@@ -598,7 +600,7 @@ def kernels_alone(args, codec, w_a, w_b, peak):
             tra.append(timed(lambda: codec.transport(), 1))
             dec.append(timed(lambda: codec.decode(), 1))
         q = int(codec.changed_blocks.sum().item()) / codec.n_blocks()
-        a_enc, a_tra, a_dec = algorithmic_bytes(n, q, args.dtype)
+        a_enc, a_tra, a_dec = algorithmic_bytes(n, q, args.dtype, args.block)
         e, t, d = float(np.median(enc)), float(np.median(tra)), float(np.median(dec))
         res[name] = {
             "q": q,

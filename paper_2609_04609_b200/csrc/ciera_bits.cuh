@@ -135,14 +135,20 @@ __device__ __forceinline__ void store_bytes_partial(uint8_t* dst, const uint32_t
 
 
 // ---- flags of fine blocks ------------------------------------------------------------------
-// d = new exponents ^ cached exponents of four consecutive values (one byte each).  Returns one
-// flag per block of 2^log2b values (log2b = 0, 1, 2: four, two, one flag), lowest value first.
+// bit 7 of every byte of the result tells whether that byte of d is non-zero
+__device__ __forceinline__ uint32_t nonzero_bytes(uint32_t d) {
+    return (((d & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | d) & 0x80808080u;
+}
+// d0, d1 = new exponents ^ cached exponents of eight consecutive values (one byte each): one flag
+// per value, value 0 in bit 0.  The non-zero marks of d0 go to bits 0, 8, 16, 24 and those of d1 to
+// bits 4, 12, 20, 28; one multiply then gathers bit 8i into bit 24 + i and bit 8i + 4 into bit
+// 28 + i (all partial products land on distinct bits below 32, so nothing carries).
+__device__ __forceinline__ uint32_t value_flags8(uint32_t d0, uint32_t d1) {
+    const uint32_t t = (nonzero_bytes(d0) >> 7) | (nonzero_bytes(d1) >> 3);
+    return (t * 0x01020408u) >> 24;
+}
+// d = the same for four values: one flag per block of 2^log2b values (log2b = 1, 2: two, one flag)
 __device__ __forceinline__ uint32_t word_block_flags(uint32_t d, uint32_t log2b) {
-    if (log2b == 0) {
-        // bytes that differ -> bits 0, 8, 16, 24 -> gathered into bits 24..27 by one multiply
-        // (the partial products land on distinct bit positions, so nothing carries)
-        return (((__vcmpne4(d, 0u) & 0x01010101u) * 0x01020408u) >> 24) & 0xFu;
-    }
     if (log2b == 1) return ((d & 0xFFFFu) != 0u ? 1u : 0u) | ((d >> 16) != 0u ? 2u : 0u);
     return d != 0u ? 1u : 0u;
 }
@@ -221,6 +227,7 @@ struct Piece<CIERA_BF16> {
     // one flag per block of 2^log2b values (log2b <= 3), lowest block first
     __device__ __forceinline__ uint32_t block_flags(const Piece& o, uint32_t log2b) const {
         if (log2b >= 3) return differs(o) ? 1u : 0u;
+        if (log2b == 0) return value_flags8(e[0] ^ o.e[0], e[1] ^ o.e[1]);
         const uint32_t per_word = 4u >> log2b;
         return word_block_flags(e[0] ^ o.e[0], log2b) | (word_block_flags(e[1] ^ o.e[1], log2b) << per_word);
     }
@@ -321,6 +328,8 @@ struct Piece<CIERA_FP32> {
     __device__ __forceinline__ uint32_t block_flags(const Piece& o, uint32_t log2b) const {
         if (log2b >= 3)
             return (((e[0] ^ o.e[0]) | (e[1] ^ o.e[1])) != 0 ? 1u : 0u) | (((e[2] ^ o.e[2]) | (e[3] ^ o.e[3])) != 0 ? 2u : 0u);
+        if (log2b == 0)
+            return value_flags8(e[0] ^ o.e[0], e[1] ^ o.e[1]) | (value_flags8(e[2] ^ o.e[2], e[3] ^ o.e[3]) << 8);
         const uint32_t per_word = 4u >> log2b;
         uint32_t f = 0;
 #pragma unroll

@@ -615,6 +615,59 @@ decode_prefix_kernel(const TileDesc* __restrict__ tiles, const uint32_t* __restr
     }
 }
 
+// The same for fine blocks, where every unit of more than one tile comes here and a tile has 32 to
+// 256 words of flags: the warps take the unit's tiles in turn and each counts a tile's flags with
+// all its lanes (consecutive words, coalesced), then the counts are scanned as above.
+__global__ void __launch_bounds__(256)
+decode_prefix_fine_kernel(const TileDesc* __restrict__ tiles, const uint32_t* __restrict__ long_first_tiles,
+                          uint32_t log2b, const uint8_t* __restrict__ msgs, uint32_t* __restrict__ ws_prefix) {
+    __shared__ uint32_t s_cnt[256];
+    __shared__ uint32_t s_warp[8];
+    __shared__ uint32_t s_carry;
+    const uint32_t first = long_first_tiles[blockIdx.x];
+    const TileDesc td0 = load_tile_desc(tiles + first);
+    const uint32_t* bm32 = reinterpret_cast<const uint32_t*>(msgs + td0.msg_off);
+    const uint64_t nb = num_blocks(td0.n_unit, log2b);
+    const uint32_t words = kTileValues >> (log2b + 5);  // words of flags per tile
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    if (tid == 0) s_carry = 0;
+    __syncthreads();
+    for (uint32_t j0 = 0; j0 < td0.n_tiles_unit; j0 += 256u) {
+        for (uint32_t t = warp; t < 256u && j0 + t < td0.n_tiles_unit; t += 8u) {
+            const uint64_t w0 = (uint64_t)(j0 + t) * words;
+            uint32_t c = 0;
+            for (uint32_t m = lane; m < words; m += 32u) {
+                const uint64_t b0 = (w0 + m) << 5;
+                if (b0 < nb) {
+                    uint32_t word = __ldg(bm32 + w0 + m);
+                    if (nb - b0 < 32) word &= (1u << (uint32_t)(nb - b0)) - 1u;
+                    c += __popc(word);
+                }
+            }
+            c = __reduce_add_sync(0xffffffffu, c);
+            if (lane == 0) s_cnt[t] = c;
+        }
+        __syncthreads();
+        const uint32_t j = j0 + tid;
+        const uint32_t cnt = j < td0.n_tiles_unit ? s_cnt[tid] : 0u;
+        uint32_t incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+            if ((int)lane >= o) incl += v;
+        }
+        if (lane == 31) s_warp[warp] = incl;
+        __syncthreads();
+        uint32_t wbase = 0;
+        for (uint32_t w = 0; w < warp; ++w) wbase += s_warp[w];
+        const uint32_t carry = s_carry;
+        if (j < td0.n_tiles_unit) ws_prefix[first + j] = carry + wbase + incl - cnt;
+        __syncthreads();
+        if (tid == 255) s_carry = carry + wbase + incl;
+        __syncthreads();
+    }
+}
+
 template <int DT, bool FINE>
 static size_t decode_smem_bytes() {
     using Cfg = DecodeCfg<DT, FINE>;
@@ -688,8 +741,12 @@ extern "C" int ciera_decode(const ciera_plan* p, const void* messages_dev, void*
     if (me != cudaSuccess) return record_cuda_error(me);
     const uint32_t n_long = (uint32_t)p->long_units.size();
     if (n_long) {
-        decode_prefix_kernel<<<n_long, 256, 0, s>>>(p->tiles_dev, p->long_units_dev, p->log2b,
-                                                    (const uint8_t*)messages_dev, (uint32_t*)workspace_dev);
+        if (is_fine(p->log2b))
+            decode_prefix_fine_kernel<<<n_long, 256, 0, s>>>(p->tiles_dev, p->long_units_dev, p->log2b,
+                                                             (const uint8_t*)messages_dev, (uint32_t*)workspace_dev);
+        else
+            decode_prefix_kernel<<<n_long, 256, 0, s>>>(p->tiles_dev, p->long_units_dev, p->log2b,
+                                                        (const uint8_t*)messages_dev, (uint32_t*)workspace_dev);
         count_launch();
         int rc = check_launch();
         if (rc) return rc;

@@ -386,65 +386,61 @@ __device__ __forceinline__ void write_changed(const EncodeTileInfo& ti, uint32_t
     }
 }
 
-// One block of B = 2^LB (fine) exponent bytes, shared -> global; both addresses are B-aligned.
+// One block of B = 2^LB (fine) exponent bytes from shared memory to two places in global memory;
+// all three addresses are B-aligned.
 template <int LB>
-__device__ __forceinline__ void copy_block(uint8_t* dst, const uint8_t* s_src) {
+__device__ __forceinline__ void copy_block2(uint8_t* dst_a, uint8_t* dst_b, const uint8_t* s_src) {
     const uint32_t a = (uint32_t)__cvta_generic_to_shared(s_src);
     if (LB == 0) {
         uint32_t v;
         asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(a));
-        __stcs(dst, (uint8_t)v);
+        __stcs(dst_a, (uint8_t)v);
+        __stcs(dst_b, (uint8_t)v);
     } else if (LB == 1) {
         uint16_t v;
         asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
-        __stcs(reinterpret_cast<uint16_t*>(dst), v);
+        __stcs(reinterpret_cast<uint16_t*>(dst_a), v);
+        __stcs(reinterpret_cast<uint16_t*>(dst_b), v);
     } else if (LB == 2) {
         uint32_t v;
         asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
-        __stcs(reinterpret_cast<uint32_t*>(dst), v);
+        __stcs(reinterpret_cast<uint32_t*>(dst_a), v);
+        __stcs(reinterpret_cast<uint32_t*>(dst_b), v);
     } else {
-        st_stream8(dst, ld_shared8(s_src));
+        const uint2 v = ld_shared8(s_src);
+        st_stream8(dst_a, v);
+        st_stream8(dst_b, v);
     }
 }
 
-// The same duty with fine blocks: a piece holds K = values-per-piece / B blocks with one flag each;
-// the exponents of its changed blocks lie next to each other in the payload, starting at the rank
-// of the piece's first changed block.
-template <int DT, int LB>
+// The same duty with fine blocks.  Here the work is split evenly over the tile's block flags
+// rather than by pieces: thread t takes the flags of values [16 t, 16 t + 16) (16, 8, 4 or 2
+// flags), walks the set ones and sends each flagged block's exponents to the payload (its rank
+// = flags set before it in the tile) and to the cache.
+template <int LB>
 __device__ __forceinline__ void write_changed_fine(const EncodeTileInfo& ti, const uint32_t* bm, const uint16_t* pre,
                                                    uint64_t base, const uint8_t* s_exp, uint32_t tid) {
-    using P = Piece<DT>;
-    constexpr uint32_t K = (uint32_t)P::kValues >> LB;  // 1 .. 16 blocks per piece
     constexpr uint32_t B = 1u << LB;
-#pragma unroll
-    for (int p = 0; p < P::kPerThread; ++p) {
-        const uint32_t t0 = P::start(tid, p);
-        const int nvalid = piece_valid<DT>(t0, ti.nv);
-        if (nvalid == 0) continue;
-        const uint32_t kb = t0 >> LB;
-        const uint32_t word = bm[kb >> 5], sh = kb & 31u;
-        const uint32_t km = (word >> sh) & ((1u << K) - 1u);  // the piece's flags (they never straddle a word)
-        if (km == 0) continue;
-        const uint32_t rank = (uint32_t)pre[kb >> 5] + __popc(word & ((1u << sh) - 1u));
-        uint8_t* pdst = ti.pay_dst + base + ((uint64_t)rank << LB);
-#pragma unroll
-        for (uint32_t j = 0; j < K; ++j) {
-            if (!((km >> j) & 1u)) continue;
-            const int left = nvalid - (int)(j << LB);  // > 0: blocks past the unit's end are never flagged
-            if (left >= (int)B) {
-                copy_block<LB>(pdst, s_exp + t0 + (j << LB));
-            } else {
-                for (int i = 0; i < left; ++i) pdst[i] = s_exp[t0 + (j << LB) + i];  // the unit's short last block
+    constexpr uint32_t kFlags = 16u >> LB;  // flags per thread
+    const uint32_t bit0 = tid * kFlags;
+    const uint32_t word = bm[bit0 >> 5], sh = bit0 & 31u;
+    uint32_t bits = (word >> sh) & ((1u << kFlags) - 1u);  // never straddles a word
+    if (bits == 0) return;
+    const uint32_t rank = (uint32_t)pre[bit0 >> 5] + __popc(word & ((1u << sh) - 1u));
+    uint8_t* pdst = ti.pay_dst + base + ((uint64_t)rank << LB);
+    while (bits) {
+        const uint32_t j = (uint32_t)__ffs(bits) - 1u;
+        bits &= bits - 1u;
+        const uint32_t v = (bit0 + j) << LB;  // the block's first value; < nv, since blocks past the end are never flagged
+        if (ti.nv - v >= B) {
+            copy_block2<LB>(pdst, ti.c_ptr + v, s_exp + v);
+        } else {
+            for (uint32_t i = 0; i < ti.nv - v; ++i) {  // the unit's short last block
+                pdst[i] = s_exp[v + i];
+                ti.c_ptr[v + i] = s_exp[v + i];
             }
-            pdst += B;
         }
-        // unchanged blocks of the piece hold what the cache holds already: refresh the whole piece
-        P x;
-        x.template load_exp_full<Shared>(s_exp + t0);
-        if (nvalid == P::kValues)
-            x.template store_exp_full<Global>(ti.c_ptr + t0);
-        else
-            x.store_exp_partial(ti.c_ptr + t0, nvalid);
+        pdst += B;
     }
 }
 
@@ -455,10 +451,10 @@ __device__ __forceinline__ void send_changed(const EncodeTileInfo& ti, uint32_t 
         write_changed<DT>(ti, log2b, bm, pre, base, s_exp, tid);
     } else {
         switch (log2b) {
-            case 0: write_changed_fine<DT, 0>(ti, bm, pre, base, s_exp, tid); break;
-            case 1: write_changed_fine<DT, 1>(ti, bm, pre, base, s_exp, tid); break;
-            case 2: write_changed_fine<DT, 2>(ti, bm, pre, base, s_exp, tid); break;
-            default: write_changed_fine<DT, 3>(ti, bm, pre, base, s_exp, tid); break;
+            case 0: write_changed_fine<0>(ti, bm, pre, base, s_exp, tid); break;
+            case 1: write_changed_fine<1>(ti, bm, pre, base, s_exp, tid); break;
+            case 2: write_changed_fine<2>(ti, bm, pre, base, s_exp, tid); break;
+            default: write_changed_fine<3>(ti, bm, pre, base, s_exp, tid); break;
         }
     }
 }
