@@ -203,6 +203,33 @@ def layer_numels(args):
     return [r * c for r, c in wl.olmoe_layer_shapes(args.experts)]
 
 
+def selection_report(args, ciera, codec, enc_ms, dec_ms, alpha=20e-6, beta=8e9):
+    """Every unit of one layer as a shard of the selection rule.  q_i comes from the last encode,
+    T_cmp and T_decmp are the layer's measured kernel times shared out by size (the sender side is
+    taken as overlapped), Comm(S) = alpha + (W - 1) S / beta with synthetic link parameters
+    (W = the simulated shard count), and the budget is half of what caching every unit would take."""
+    n = codec.units["n_values"].astype(np.int64)
+    changed = codec.changed_blocks.cpu().numpy().astype(np.int64)
+    blocks = np.maximum(-(-n // args.block), 1)
+    total = max(int(n.sum()), 1)
+    code = ciera.DTYPE_CODES[args.dtype]
+    shards = [dict(n_values=int(ni), dtype=code, block=args.block, q=float(min(ci / bi, 1.0)), world_size=args.shards,
+                   alpha=alpha, beta=beta, t_cmp=enc_ms * 1e-3 * ni / total, t_decmp=dec_ms * 1e-3 * ni / total,
+                   overlapped=True) for ni, ci, bi in zip(n, changed, blocks)]
+    everything = ciera.select_shards(shards, 1 << 62, True)
+    budget = sum(everything["footprints"]) // 2
+    got = ciera.select_shards(shards, budget, True)
+    gains = np.array(got["gains"])
+    sel = np.array(got["selected"], bool)
+    return {
+        "rule": "g_i > 0, ranked by g_i / M_i, greedy prefix under the budget (ciera_select_shards)",
+        "comm_model": {"alpha_s": alpha, "beta_Bps": beta, "world_size": args.shards, "kind": "synthetic"},
+        "units": int(n.size), "positive_gain": int((gains > 0).sum()), "selected": int(sel.sum()),
+        "budget_bytes": int(budget), "used_bytes": int(got["used"]),
+        "gain_ms_selected": float(gains[sel].sum() * 1e3), "gain_ms_all_positive": float(gains[gains > 0].sum() * 1e3),
+    }
+
+
 def algorithmic_bytes(n_values, q, dtype, block):
     """HBM bytes per launch the method needs: (encode, transport, decode).  q = share of the
     exponent bytes that travel (changed blocks); the bitmap is one bit per block."""
@@ -540,6 +567,11 @@ def main():
                                      "note": "algorithmic bytes of all three kernels over the two-stream step time"},
         },
     }
+
+    # ---- which shards would be compressed: the gain rule and the selection under a cache budget,
+    #      fed with this run's measured change rates and kernel times (host arithmetic only)
+    if rank == 0:
+        out["selection"] = selection_report(args, ciera, layers[-1], enc_ms, dec_ms)
 
     # ---- per-kernel numbers with each kernel alone on the GPU, three change regimes (one layer)
     if not args.no_regimes and rank == 0:

@@ -275,6 +275,23 @@ typedef struct ciera_gain_in {
  * "compress iff g > 0".  Either output pointer may be NULL. */
 CIERA_API int ciera_should_compress(const ciera_gain_in* in, double* gain_seconds_out, int* decision_out);
 
+/* Shard selection under a cache budget (Section 3.2, last paragraph): shard i costs
+ * M_i = (W - 1) * S_e^i bytes of exponent cache per GPU (S_e^i = one byte per value); shards with
+ * positive gain are ranked in descending order of g_i / M_i and selected down the ranking until the
+ * first one that no longer fits into cache_budget_bytes (ties keep the input order; shards without
+ * values are never selected).  with_sender_cache != 0 counts W * S_e^i instead, i.e. also the
+ * sender-side exponent cache this library compares against.
+ *   shards          host, n_shards entries (q_i, sizes, Comm() model and kernel times per shard)
+ *   ranking_out     host, n_shards indices: the ranked positive-gain shards, then the others in
+ *                   input order; may be NULL
+ *   selected_out    host, n_shards flags (1 = compress this shard)
+ *   gains_out, footprints_out   host, n_shards values g_i (seconds) and M_i (bytes); may be NULL
+ *   used_bytes_out  host, sum of M_i over the selected shards; may be NULL
+ * Returns CIERA_ERR_INVALID_ARG for a shard that ciera_should_compress would reject. */
+CIERA_API int ciera_select_shards(const ciera_gain_in* shards, uint32_t n_shards, uint64_t cache_budget_bytes,
+                                  int with_sender_cache, uint32_t* ranking_out, uint8_t* selected_out,
+                                  double* gains_out, uint64_t* footprints_out, uint64_t* used_bytes_out);
+
 /* ---- diagnostics ---------------------------------------------------------------------------- */
 
 /* cudaError_t of the last failing runtime call made by the calling thread inside this library. */

@@ -75,6 +75,7 @@ _SIGS = {
     "ciera_decode": ([_vp] * 8, _i32),
     "ciera_roundtrip_host": ([_vp, _vp, _sz, _vp, _vp, _vp, _vp], _i32),
     "ciera_should_compress": ([ctypes.POINTER(GainIn), ctypes.POINTER(_dbl), ctypes.POINTER(_i32)], _i32),
+    "ciera_select_shards": ([ctypes.POINTER(GainIn), _u32, _u64, _i32, _vp, _vp, _vp, _vp, _vp], _i32),
     "ciera_last_cuda_error": ([], _i32),
     "ciera_kernel_launch_count": ([], _u64),
     "ciera_status_string": ([_i32], ctypes.c_char_p),
@@ -247,22 +248,49 @@ def roundtrip_host(plan: Plan, weights_host: torch.Tensor, weights_out_host: tor
 # ------------------------------------------------------------------------------ gain rule (host)
 
 
+def _fill_gain_in(gi, keep, n_values, dtype, block, q, world_size=2, alpha=0.0, beta=1.0, table=None, t_hash=0.0,
+                  t_cmp=0.0, t_decmp=0.0, overlapped=False):
+    gi.n_values, gi.dtype, gi.block, gi.q = n_values, dtype, block, q
+    gi.world_size, gi.overlapped, gi.alpha, gi.beta = world_size, int(overlapped), alpha, beta
+    gi.t_hash, gi.t_cmp, gi.t_decmp = t_hash, t_cmp, t_decmp
+    if table:
+        tb = (_dbl * len(table))(*[float(p[0]) for p in table])
+        ts = (_dbl * len(table))(*[float(p[1]) for p in table])
+        keep.append((tb, ts))  # the arrays must outlive the call
+        gi.table_bytes, gi.table_secs, gi.n_points = tb, ts, len(table)
+    else:
+        gi.n_points = 0
+
+
+def select_shards(shards, cache_budget_bytes: int, with_sender_cache: bool = False):
+    """``shards``: a list of dicts with the keyword arguments of ``should_compress``.  Returns a dict with
+    ``ranking``, ``selected``, ``gains``, ``footprints`` (lists) and ``used`` (bytes)."""
+    n = len(shards)
+    arr = (GainIn * max(n, 1))()
+    keep = []
+    for gi, sh in zip(arr, shards):
+        _fill_gain_in(gi, keep, **sh)
+    ranking = (_u32 * max(n, 1))()
+    selected = (ctypes.c_uint8 * max(n, 1))()
+    gains = (_dbl * max(n, 1))()
+    fps = (_u64 * max(n, 1))()
+    used = _u64(0)
+    _check("ciera_select_shards",
+           _lib.ciera_select_shards(arr, n, int(cache_budget_bytes), int(with_sender_cache),
+                                    ctypes.cast(ranking, _vp), ctypes.cast(selected, _vp), ctypes.cast(gains, _vp),
+                                    ctypes.cast(fps, _vp), ctypes.cast(ctypes.pointer(used), _vp)))
+    del keep
+    return {"ranking": list(ranking)[:n], "selected": [bool(x) for x in list(selected)[:n]],
+            "gains": list(gains)[:n], "footprints": list(fps)[:n], "used": int(used.value)}
+
+
 def should_compress(n_values: int, dtype: int, block: int, q: float, world_size: int = 2, alpha: float = 0.0,
                     beta: float = 1.0, table=None, t_hash: float = 0.0, t_cmp: float = 0.0, t_decmp: float = 0.0,
                     overlapped: bool = False):
     """Returns (gain_seconds, decision)."""
     gi = GainIn()
-    gi.n_values, gi.dtype, gi.block, gi.q = n_values, dtype, block, q
-    gi.world_size, gi.overlapped, gi.alpha, gi.beta = world_size, int(overlapped), alpha, beta
-    gi.t_hash, gi.t_cmp, gi.t_decmp = t_hash, t_cmp, t_decmp
-    keep = None
-    if table:
-        tb = (_dbl * len(table))(*[float(p[0]) for p in table])
-        ts = (_dbl * len(table))(*[float(p[1]) for p in table])
-        keep = (tb, ts)
-        gi.table_bytes, gi.table_secs, gi.n_points = tb, ts, len(table)
-    else:
-        gi.n_points = 0
+    keep = []
+    _fill_gain_in(gi, keep, n_values, dtype, block, q, world_size, alpha, beta, table, t_hash, t_cmp, t_decmp, overlapped)
     g = _dbl(0.0)
     d = _i32(0)
     _check("ciera_should_compress", _lib.ciera_should_compress(ctypes.byref(gi), ctypes.byref(g), ctypes.byref(d)))

@@ -187,7 +187,18 @@ static double comm_seconds(const ciera_gain_in* in, double bytes) {
     return y0 + (bytes - x0) * (y1 - y0) / (x1 - x0);
 }
 
+static int gain_of(const ciera_gain_in* in, double* g_out);
+
 extern "C" int ciera_should_compress(const ciera_gain_in* in, double* gain_seconds_out, int* decision_out) {
+    double g = 0.0;
+    const int rc = gain_of(in, &g);
+    if (rc) return rc;
+    if (gain_seconds_out) *gain_seconds_out = g;
+    if (decision_out) *decision_out = g > 0.0 ? 1 : 0;
+    return CIERA_OK;
+}
+
+static int gain_of(const ciera_gain_in* in, double* g_out) {
     if (!in || !valid_dtype(in->dtype) || in->block == 0) return CIERA_ERR_INVALID_ARG;
     if (!(in->q >= 0.0 && in->q <= 1.0)) return CIERA_ERR_INVALID_ARG;
     if (in->n_points >= 2 && in->table_bytes && in->table_secs) {
@@ -204,9 +215,48 @@ extern "C" int ciera_should_compress(const ciera_gain_in* in, double* gain_secon
     const double s_bm = (double)((blocks + 7) / 8);
     const double sent = s_sm + s_bm + in->q * s_exp;
     const double sender = in->overlapped ? 0.0 : in->t_hash + in->t_cmp;
-    const double g = comm_seconds(in, s_full) - (comm_seconds(in, sent) + sender + in->t_decmp);
-    if (gain_seconds_out) *gain_seconds_out = g;
-    if (decision_out) *decision_out = g > 0.0 ? 1 : 0;
+    *g_out = comm_seconds(in, s_full) - (comm_seconds(in, sent) + sender + in->t_decmp);
+    return CIERA_OK;
+}
+
+// ---------------------------------------------------------------------------------- selection
+
+extern "C" int ciera_select_shards(const ciera_gain_in* shards, uint32_t n_shards, uint64_t cache_budget_bytes,
+                                   int with_sender_cache, uint32_t* ranking_out, uint8_t* selected_out,
+                                   double* gains_out, uint64_t* footprints_out, uint64_t* used_bytes_out) {
+    if ((!shards && n_shards) || (!selected_out && n_shards)) return CIERA_ERR_INVALID_ARG;
+    std::vector<double> g(n_shards);
+    std::vector<uint64_t> m(n_shards);
+    for (uint32_t i = 0; i < n_shards; ++i) {
+        const int rc = gain_of(&shards[i], &g[i]);
+        if (rc) return rc;
+        if (shards[i].world_size < 1) return CIERA_ERR_INVALID_ARG;
+        // M_i = (W - 1) S_e^i per GPU, S_e^i = one exponent byte per value (+ S_e^i for this
+        // library's sender-side exponent cache when asked for)
+        m[i] = (uint64_t)(shards[i].world_size - 1 + (with_sender_cache ? 1 : 0)) * shards[i].n_values;
+    }
+    // positive gains in descending order of g_i / M_i (ties: original order), then the rest
+    std::vector<uint32_t> cand, rest;
+    for (uint32_t i = 0; i < n_shards; ++i) ((g[i] > 0.0 && m[i] > 0) ? cand : rest).push_back(i);
+    std::stable_sort(cand.begin(), cand.end(),
+                     [&](uint32_t a, uint32_t b) { return g[a] / (double)m[a] > g[b] / (double)m[b]; });
+    for (uint32_t i = 0; i < n_shards; ++i) selected_out[i] = 0;
+    uint64_t used = 0;
+    for (uint32_t i : cand) {  // until the budget is exhausted: stop at the first shard that does not fit
+        if (m[i] > cache_budget_bytes - used) break;
+        selected_out[i] = 1;
+        used += m[i];
+    }
+    if (ranking_out) {
+        uint32_t k = 0;
+        for (uint32_t i : cand) ranking_out[k++] = i;
+        for (uint32_t i : rest) ranking_out[k++] = i;
+    }
+    for (uint32_t i = 0; i < n_shards; ++i) {
+        if (gains_out) gains_out[i] = g[i];
+        if (footprints_out) footprints_out[i] = m[i];
+    }
+    if (used_bytes_out) *used_bytes_out = used;
     return CIERA_OK;
 }
 
