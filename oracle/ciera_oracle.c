@@ -32,8 +32,11 @@
  *
  * Pins: tests/test_oracle_*.py (IEEE field definition through frexp, exhaustive
  * bf16 x cache sweep, hand-worked fixtures, byte formula, closed forms (1-c)^B,
- * special cases, hand-computed gains).  ANS coding and the 128-bit hash are not
- * built: parity unpinned for those two, by construction absent here.
+ * special cases, hand-computed gains).  ANS coding is not built ("parity unpinned", absent
+ * here).  The hash-based sender (ora_encode_hashed) is pinned as a change detector (published
+ * SplitMix64 streams, equality with the exact-comparison sender, certain detection of single-word
+ * changes); the 128-bit hash VALUES follow a construction the paper does not print, so for them:
+ * parity unpinned.
  */
 #include <stddef.h>
 #include <stdint.h>
@@ -203,6 +206,145 @@ int ora_encode(const void* w, uint8_t* cache_s, uint64_t n, int dtype, uint32_t 
         ++nchg;
     }
 
+    *payload_bytes = plen;
+    *changed_blocks = nchg;
+    *wire_bytes = pay_off + plen;
+    free(exp);
+    free(sm);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Sender side with hash-based change detection (Section 3.1; Algorithm 1 as printed: the sender
+ * keeps HashCache[i,k], a 128-bit hash per block, not the exponents themselves).
+ *
+ * The paper fixes only this much: the hash has 128 bits and is built from two independent 64-bit
+ * SplitMix64 hashes.  The construction used here (a reading; the paper prints none):
+ *   mix(z)  = the SplitMix64 output function: z ^= z >> 30; z *= 0xBF58476D1CE4E5B9;
+ *             z ^= z >> 27; z *= 0x94D049BB133111EB; z ^= z >> 31
+ *   gamma   = 0x9E3779B97F4A7C15 (the SplitMix64 increment)
+ *   a block of L exponent bytes is read as m = ceil(L / 8) little-endian 64-bit words x_0..x_{m-1}
+ *   (the last one zero-padded);
+ *   H_s     = mix( L + sum_j mix(s + (j + 1) * gamma + x_j) )      (all arithmetic mod 2^64)
+ *   Hash128 = (H_s1, H_s2), s1 = 0, s2 = 0x6A09E667F3BCC908.
+ * mix(s + (j + 1) * gamma) is the j-th output of the SplitMix64 generator seeded with s, so each
+ * word is added to the generator's state before the output function; summing the per-word terms
+ * makes the hash independent of the order in which the words are visited.
+ */
+#define ORA_GAMMA 0x9E3779B97F4A7C15ull
+#define ORA_SEED1 0x0000000000000000ull
+#define ORA_SEED2 0x6A09E667F3BCC908ull
+
+uint64_t ora_splitmix64_mix(uint64_t z) {
+    z ^= z >> 30;
+    z *= 0xBF58476D1CE4E5B9ull;
+    z ^= z >> 27;
+    z *= 0x94D049BB133111EBull;
+    z ^= z >> 31;
+    return z;
+}
+
+/* next output of the SplitMix64 generator; *state is advanced (used by the pins only) */
+uint64_t ora_splitmix64_next(uint64_t* state) {
+    *state += ORA_GAMMA;
+    return ora_splitmix64_mix(*state);
+}
+
+void ora_hash128(const uint8_t* exp, uint64_t len, uint64_t out[2]) {
+    const uint64_t seeds[2] = {ORA_SEED1, ORA_SEED2};
+    for (int h = 0; h < 2; ++h) {
+        uint64_t acc = 0;
+        for (uint64_t j = 0; 8 * j < len; ++j) {
+            uint64_t x = 0;
+            for (uint64_t i = 0; i < 8 && 8 * j + i < len; ++i) x |= (uint64_t)exp[8 * j + i] << (8 * i);
+            acc += ora_splitmix64_mix(seeds[h] + (j + 1) * ORA_GAMMA + x);
+        }
+        out[h] = ora_splitmix64_mix(acc + len);
+    }
+}
+
+/* HashCache := Hash128 of every block of exponents(w); of all-zero exponents when w == NULL.
+ * hash_cache holds 2 * S_b words: (H_s1, H_s2) of block 0, of block 1, ... */
+int ora_hash_cache_init(const void* w, uint64_t n, int dtype, uint32_t block, uint64_t* hash_cache) {
+    if (n == 0) return 0;
+    uint8_t* exp = (uint8_t*)calloc(n, 1);
+    uint32_t* sm = (uint32_t*)malloc(n * sizeof(uint32_t));
+    if (!exp || !sm) {
+        free(exp);
+        free(sm);
+        return -1;
+    }
+    if (w) ora_split(w, n, dtype, exp, sm);
+    uint64_t nb = ora_num_blocks(n, block);
+    for (uint64_t k = 0; k < nb; ++k) {
+        uint64_t lo = k * block;
+        uint64_t hi = lo + block < n ? lo + block : n;
+        ora_hash128(exp + lo, hi - lo, hash_cache + 2 * k);
+    }
+    free(exp);
+    free(sm);
+    return 0;
+}
+
+/* Same message layout and outputs as ora_encode; hash_cache (2 * S_b words) is in/out. */
+int ora_encode_hashed(const void* w, uint64_t* hash_cache, uint64_t n, int dtype, uint32_t block, uint8_t* msg,
+                      uint64_t msg_capacity, uint64_t* wire_bytes, uint64_t* payload_bytes,
+                      uint32_t* changed_blocks) {
+    *wire_bytes = 0;
+    *payload_bytes = 0;
+    *changed_blocks = 0;
+    if (n == 0) return 0;
+    if (msg_capacity < ora_message_capacity(n, dtype, block)) return -2;
+
+    int m = ora_m(dtype);
+    uint64_t nb = ora_num_blocks(n, block);
+    uint64_t sm_off = ora_sm_offset(n, block);
+    uint64_t pay_off = ora_payload_offset(n, dtype, block);
+
+    /* (exp, mant) <- SplitExpMant(shard) */
+    uint8_t* exp = (uint8_t*)malloc(n);
+    uint32_t* sm = (uint32_t*)malloc(n * sizeof(uint32_t));
+    if (!exp || !sm) {
+        free(exp);
+        free(sm);
+        return -1;
+    }
+    ora_split(w, n, dtype, exp, sm);
+    memset(msg, 0, pay_off);
+
+    /* for k = 1..S_b: h <- Hash128(exp[k]); if h != HashCache[k]: bitmap[k] <- 1, HashCache[k] <- h */
+    for (uint64_t k = 0; k < nb; ++k) {
+        uint64_t lo = k * block;
+        uint64_t hi = lo + block < n ? lo + block : n;
+        uint64_t h[2];
+        ora_hash128(exp + lo, hi - lo, h);
+        if (h[0] != hash_cache[2 * k] || h[1] != hash_cache[2 * k + 1]) {
+            msg[k >> 3] |= (uint8_t)(1u << (k & 7));
+            hash_cache[2 * k] = h[0];
+            hash_cache[2 * k + 1] = h[1];
+        }
+    }
+
+    for (uint64_t j = 0; j < n; ++j) {
+        if (m == 8) {
+            msg[sm_off + j] = (uint8_t)sm[j];
+        } else {
+            msg[sm_off + 3 * j + 0] = (uint8_t)(sm[j] & 0xFF);
+            msg[sm_off + 3 * j + 1] = (uint8_t)((sm[j] >> 8) & 0xFF);
+            msg[sm_off + 3 * j + 2] = (uint8_t)((sm[j] >> 16) & 0xFF);
+        }
+    }
+
+    /* payload <- { exp[k] | bitmap[k] = 1 } in block order (no entropy stage, as in ora_encode) */
+    uint64_t plen = 0;
+    uint32_t nchg = 0;
+    for (uint64_t k = 0; k < nb; ++k) {
+        if (!((msg[k >> 3] >> (k & 7)) & 1u)) continue;
+        uint64_t lo = k * block;
+        uint64_t hi = lo + block < n ? lo + block : n;
+        for (uint64_t j = lo; j < hi; ++j) msg[pay_off + plen++] = exp[j];
+        ++nchg;
+    }
     *payload_bytes = plen;
     *changed_blocks = nchg;
     *wire_bytes = pay_off + plen;

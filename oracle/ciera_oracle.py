@@ -55,6 +55,12 @@ def lib() -> ctypes.CDLL:
         L.ora_encode.argtypes = [vp, vp, u64, i32, u32, vp, u64, vp, vp, vp]
         L.ora_encode.restype = i32
         L.ora_decode.argtypes, L.ora_decode.restype = [vp, vp, u64, i32, u32, vp], i32
+        L.ora_splitmix64_mix.argtypes, L.ora_splitmix64_mix.restype = [u64], u64
+        L.ora_splitmix64_next.argtypes, L.ora_splitmix64_next.restype = [vp], u64
+        L.ora_hash128.argtypes, L.ora_hash128.restype = [vp, u64, vp], None
+        L.ora_hash_cache_init.argtypes, L.ora_hash_cache_init.restype = [vp, u64, i32, u32, vp], i32
+        L.ora_encode_hashed.argtypes = [vp, vp, u64, i32, u32, vp, u64, vp, vp, vp]
+        L.ora_encode_hashed.restype = i32
         L.ora_gain.argtypes = [u64, i32, u32, dbl, i32, dbl, dbl, vp, vp, i32, dbl, dbl, dbl, i32]
         L.ora_gain.restype = dbl
         _lib = L
@@ -170,3 +176,53 @@ def gain(n, dtype, block, q, world, alpha=0.0, beta=1.0, table=None, t_hash=0.0,
                                     t_hash, t_cmp, t_decmp, int(overlapped)))
     return float(lib().ora_gain(n, dtype, block, q, world, alpha, beta, None, None, 0,
                                 t_hash, t_cmp, t_decmp, int(overlapped)))
+
+
+# ------------------------------------------------------------------ hash-based change detection
+
+
+def splitmix64_stream(seed: int, count: int):
+    """First ``count`` outputs of the SplitMix64 generator seeded with ``seed``."""
+    state = ctypes.c_uint64(seed)
+    return [int(lib().ora_splitmix64_next(ctypes.addressof(state))) for _ in range(count)]
+
+
+def splitmix64_mix(z: int) -> int:
+    return int(lib().ora_splitmix64_mix(z))
+
+
+def hash128(exp: np.ndarray):
+    """Hash128 of one block of exponent bytes: (H_s1, H_s2)."""
+    exp = np.ascontiguousarray(exp, np.uint8)
+    out = np.zeros(2, np.uint64)
+    lib().ora_hash128(_ptr(exp) if exp.size else None, exp.size, _ptr(out))
+    return int(out[0]), int(out[1])
+
+
+def hash_cache_init(w_bits, n: int, dtype: int, block: int) -> np.ndarray:
+    """HashCache of one unit: uint64[2 * S_b]; of all-zero exponents when ``w_bits`` is None."""
+    hc = np.zeros(2 * num_blocks(n, block), np.uint64)
+    if n == 0:
+        return hc
+    if w_bits is None:
+        rc = lib().ora_hash_cache_init(None, n, dtype, block, _ptr(hc))
+    else:
+        w_bits = np.ascontiguousarray(w_bits, dtype=_wdtype(dtype))
+        assert w_bits.size == n
+        rc = lib().ora_hash_cache_init(_ptr(w_bits), n, dtype, block, _ptr(hc))
+    assert rc == 0
+    return hc
+
+
+def encode_hashed(w_bits: np.ndarray, hash_cache: np.ndarray, dtype: int, block: int):
+    """Like ``encode`` but with HashCache (uint64[2 * S_b], updated in place) on the sender."""
+    w_bits = np.ascontiguousarray(w_bits, dtype=_wdtype(dtype))
+    n = w_bits.size
+    assert hash_cache.dtype == np.uint64 and hash_cache.size == 2 * num_blocks(n, block)
+    cap = message_capacity(n, dtype, block)
+    msg = np.zeros(max(cap, 1), np.uint8)
+    wire, pay, chg = ctypes.c_uint64(0), ctypes.c_uint64(0), ctypes.c_uint32(0)
+    rc = lib().ora_encode_hashed(_ptr(w_bits) if n else None, _ptr(hash_cache) if n else None, n, dtype, block, _ptr(msg), cap,
+                                 ctypes.addressof(wire), ctypes.addressof(pay), ctypes.addressof(chg))
+    assert rc == 0, rc
+    return msg[: wire.value].copy(), int(wire.value), int(pay.value), int(chg.value)
