@@ -195,6 +195,37 @@ CIERA_API int ciera_encode_noalloc(const ciera_plan* plan, const void* weights_d
                          void* messages_dev, uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev,
                          int32_t* status_dev, void* stream);
 
+/* ---- sender with hash-based change detection (Section 3.1; Algorithm 1, sender, as printed) ---
+ *
+ * Instead of the previous exponents the sender keeps HashCache: one 128-bit hash per block, built
+ * from two independent 64-bit SplitMix64 hashes of the block's exponents.  A block travels iff its
+ * hash differs from the cached one; the cached hash is then replaced.  The message is the same as
+ * ciera_encode's (a collision, probability about 2^-128 per comparison, would leave a changed
+ * block unsent).  The construction (the paper prints none): with mix() the SplitMix64 output
+ * function and gamma its increment, a block of L exponent bytes read as little-endian 64-bit words
+ * x_j (the last one zero-padded),  H_s = mix(L + sum_j mix(s + (j + 1) * gamma + x_j)) mod 2^64,
+ * Hash128 = (H_0, H_0x6A09E667F3BCC908), stored as two little-endian 64-bit words per block.
+ * Blocks of 16 values and more only (CIERA_ERR_UNSUPPORTED otherwise). */
+
+/* Bytes of a HashCache for the whole plan (16 per block; units in table order), the offset of a
+ * unit's first block in it, and the scratch ciera_encode_hashed needs (72 bytes per tile + 16). */
+CIERA_API size_t ciera_plan_hash_cache_bytes(const ciera_plan* plan);
+CIERA_API size_t ciera_plan_unit_hash_offset(const ciera_plan* plan, uint32_t unit);
+CIERA_API size_t ciera_plan_hashed_workspace_bytes(const ciera_plan* plan);
+
+/* HashCache := Hash128 of every block of exponents(weights); of all-zero exponents when
+ * weights_dev is NULL (the counterpart of a zero-initialised exponent cache).  Device pointers,
+ * 16-byte aligned.  Asynchronous on `stream`. */
+CIERA_API int ciera_hash_cache_init(const ciera_plan* plan, void* hash_cache_dev, const void* weights_dev, void* stream);
+
+/* Sender step with HashCache.  Arguments as for ciera_encode, with hash_cache_dev (in/out,
+ * ciera_plan_hash_cache_bytes) in place of the exponent cache and a scratch of
+ * ciera_plan_hashed_workspace_bytes (contents need not be initialised).  Three kernel launches on
+ * `stream`; nothing waits inside the kernels, so there is no status word. */
+CIERA_API int ciera_encode_hashed(const ciera_plan* plan, const void* weights_dev, void* hash_cache_dev,
+                                  void* messages_dev, uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev,
+                                  void* workspace_dev, void* stream);
+
 /* ---- transport stand-in: Send / Recv of Algorithm 1 on one GPU ----------------------------- */
 
 /* Copies, for every unit, the first wire_bytes_dev[u] bytes of its slot from `src_messages_dev`

@@ -71,6 +71,11 @@ _SIGS = {
     "ciera_cache_update": ([_vp, _vp, _vp, _vp], _i32),
     "ciera_encode": ([_vp] * 9, _i32),
     "ciera_encode_noalloc": ([_vp] * 8, _i32),
+    "ciera_plan_hash_cache_bytes": ([_vp], _sz),
+    "ciera_plan_unit_hash_offset": ([_vp, _u32], _sz),
+    "ciera_plan_hashed_workspace_bytes": ([_vp], _sz),
+    "ciera_hash_cache_init": ([_vp] * 4, _i32),
+    "ciera_encode_hashed": ([_vp] * 8, _i32),
     "ciera_transport": ([_vp] * 6, _i32),
     "ciera_decode": ([_vp] * 8, _i32),
     "ciera_roundtrip_host": ([_vp, _vp, _sz, _vp, _vp, _vp, _vp], _i32),
@@ -157,6 +162,8 @@ class Plan:
         self.total_values = int(_lib.ciera_plan_total_values(h))
         self.device_bytes = int(_lib.ciera_plan_device_bytes(h))
         self.workspace_bytes = int(_lib.ciera_plan_workspace_bytes(h))
+        self.hash_cache_bytes = int(_lib.ciera_plan_hash_cache_bytes(h))
+        self.hashed_workspace_bytes = int(_lib.ciera_plan_hashed_workspace_bytes(h))
         self.table = None
         if device is not None:
             self.bind(device)
@@ -215,6 +222,24 @@ def encode_noalloc(plan: Plan, weights, sender_cache, messages, wire_bytes, chan
     _check("ciera_encode_noalloc",
            _lib.ciera_encode_noalloc(plan.handle, _ptr(weights), _ptr(sender_cache), _ptr(messages), _ptr(wire_bytes),
                                      _ptr(changed_blocks), _ptr(status), _stream(stream)))
+
+
+def unit_hash_offset(plan: Plan, unit: int) -> int:
+    """Byte offset of the unit's first block in the plan's HashCache."""
+    return int(_lib.ciera_plan_unit_hash_offset(plan.handle, unit))
+
+
+def hash_cache_init(plan: Plan, hash_cache: torch.Tensor, weights: Optional[torch.Tensor], stream=None) -> None:
+    _check("ciera_hash_cache_init",
+           _lib.ciera_hash_cache_init(plan.handle, _ptr(hash_cache), _ptr(weights), _stream(stream)))
+
+
+def encode_hashed(plan: Plan, weights, hash_cache, messages, wire_bytes, changed_blocks, workspace, stream=None) -> None:
+    """Sender step with a 128-bit hash per block in place of the exponent cache (blocks of 16 values
+    and more); ``workspace`` holds ``plan.hashed_workspace_bytes``."""
+    _check("ciera_encode_hashed",
+           _lib.ciera_encode_hashed(plan.handle, _ptr(weights), _ptr(hash_cache), _ptr(messages), _ptr(wire_bytes),
+                                    _ptr(changed_blocks), _ptr(workspace), _stream(stream)))
 
 
 def transport(plan: Plan, src_messages, dst_messages, wire_bytes, workspace, stream=None) -> None:

@@ -1,0 +1,362 @@
+// Sender side with hash-based change detection (paper Section 3.1 and Algorithm 1 as printed: the
+// sender keeps HashCache[i,k], a 128-bit hash per block, instead of the previous exponents).
+//
+// The paper fixes only that the hash has 128 bits and is built from two independent 64-bit
+// SplitMix64 hashes.  The construction used here:
+//   mix(z)  = the SplitMix64 output function, gamma = its increment 0x9E3779B97F4A7C15;
+//   a block of L exponent bytes is read as ceil(L / 8) little-endian 64-bit words x_j (the last
+//   one zero-padded);  H_s = mix(L + sum_j mix(s + (j + 1) * gamma + x_j))  (mod 2^64);
+//   Hash128 = (H_s1, H_s2) with s1 = 0 and s2 = 0x6A09E667F3BCC908.
+// The per-word terms are summed, so the threads holding a block's words can be combined in any
+// order: a shuffle reduction inside the warp, then a shared-memory atomic per warp and block.
+//
+// Three plain launches per call (no waiting between thread blocks anywhere):
+//   scan     one thread block per tile: split, sign-plus-mantissa out, block hashes, compare with
+//            HashCache and refresh it; leaves the tile's block flags and their count in the scratch;
+//   unit     one thread block per unit: per-tile payload offsets (running count over the unit's
+//            tiles), the unit's bitmap bytes, pads, reported length and changed-block count;
+//   payload  one thread block per tile: the exponents of the flagged blocks (their weights are read
+//            a second time) go to their place in the payload.
+// HBM bytes per value: 2 + 1 (scan) and 3 q (payload) for bf16, against 4 + 2 q with the exponent
+// cache, plus 16 bytes per block of HashCache traffic; the price is about 40 integer instructions
+// per 8 values for the two hashes.
+#include "ciera_bits.cuh"
+
+namespace ciera {
+
+constexpr uint64_t kGamma = 0x9E3779B97F4A7C15ull;
+constexpr uint64_t kSeed1 = 0x0000000000000000ull;
+constexpr uint64_t kSeed2 = 0x6A09E667F3BCC908ull;
+constexpr uint32_t kFlagWords = kBitmapWords;  // 16 words of block flags per tile in the scratch
+
+__device__ __forceinline__ uint64_t mix64(uint64_t z) {
+    z ^= z >> 30;
+    z *= 0xBF58476D1CE4E5B9ull;
+    z ^= z >> 27;
+    z *= 0x94D049BB133111EBull;
+    z ^= z >> 31;
+    return z;
+}
+
+// Adds the terms of one 64-bit word of exponents (at value offset v of the tile) to the sums of
+// its block.  `lanes` = lanes of this warp that hold words of the same block (a power of two,
+// aligned); lanes whose word does not exist pass valid = false and still take part.
+__device__ __forceinline__ void add_word_terms(unsigned long long (*sums)[2], uint32_t log2b, uint32_t lanes, uint32_t v,
+                                               uint64_t x, bool valid, uint32_t lane) {
+    const uint32_t j = (v & ((1u << log2b) - 1u)) >> 3;
+    uint64_t a = valid ? mix64(kSeed1 + (uint64_t)(j + 1u) * kGamma + x) : 0ull;
+    uint64_t b = valid ? mix64(kSeed2 + (uint64_t)(j + 1u) * kGamma + x) : 0ull;
+    for (uint32_t o = 1; o < lanes; o <<= 1) {
+        a += __shfl_xor_sync(0xffffffffu, a, o);
+        b += __shfl_xor_sync(0xffffffffu, b, o);
+    }
+    if ((lane & (lanes - 1u)) == 0 && valid) {  // a group's first lane holds the block's lowest word: valid if any is
+        atomicAdd(&sums[v >> log2b][0], (unsigned long long)a);
+        atomicAdd(&sums[v >> log2b][1], (unsigned long long)b);
+    }
+}
+
+// Hashes of the blocks of one tile.  INIT: HashCache := hashes (weights may be null: exponents
+// all zero).  Otherwise the scan pass described at the head of this file.
+template <int DT, bool INIT>
+__global__ void __launch_bounds__(kThreads)
+hashed_scan_kernel(const TileDesc* __restrict__ tiles, const unsigned long long* __restrict__ hash_base, uint32_t log2b,
+                   const uint8_t* __restrict__ weights, ulonglong2* hash_cache, uint8_t* msgs, uint32_t* ws_flags,
+                   uint32_t* ws_count) {
+    using P = Piece<DT>;
+    constexpr int VB = Traits<DT>::kValueBytes;
+    constexpr int SMB = Traits<DT>::kSmBytes;
+    __shared__ unsigned long long sums[kTileValues / 16][2];  // up to 512 blocks per tile
+    __shared__ uint32_t s_count;
+    const uint32_t tile = blockIdx.x, tid = threadIdx.x, lane = tid & 31u;
+    const TileDesc td = load_tile_desc(tiles + tile);
+    const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
+    const uint32_t nv = (uint32_t)min((uint64_t)kTileValues, td.n_unit - v0);
+    const uint32_t B = 1u << log2b;
+    const uint32_t nbt = kTileValues >> log2b;
+    const uint32_t nblk = (nv + B - 1u) >> log2b;
+
+    for (uint32_t b = tid; b < nbt; b += kThreads) sums[b][0] = sums[b][1] = 0ull;
+    if (tid == 0) s_count = 0;
+    __syncthreads();
+
+    uint8_t* sm_dst = INIT ? nullptr : msgs + td.msg_off + sm_offset(td.n_unit, log2b) + v0 * SMB;
+    // lanes of a warp that share a block: a lane holds P::kValues consecutive values
+    const uint32_t lanes = min(32u, B >> P::kLog2Values);
+#pragma unroll
+    for (int p = 0; p < P::kPerThread; ++p) {
+        const uint32_t t0 = P::start(tid, p);
+        const int nvalid = piece_valid<DT>(t0, nv);
+        P x;
+#pragma unroll
+        for (int i = 0; i < P::kExpWords; ++i) x.e[i] = 0;
+        if (nvalid > 0 && weights != nullptr) {
+            if (nvalid == P::kValues)
+                x.template split_full<Global>(weights + td.w_off + (uint64_t)t0 * VB);
+            else
+                x.split_partial(weights + td.w_off + (uint64_t)t0 * VB, nvalid);
+            if (!INIT) {
+                if (nvalid == P::kValues)
+                    x.template store_sm_full<Global>(sm_dst + (size_t)t0 * SMB);
+                else
+                    x.store_sm_partial(sm_dst + (size_t)t0 * SMB, nvalid);
+            }
+        }
+#pragma unroll
+        for (int w = 0; w < P::kExpWords / 2; ++w) {
+            const uint64_t word = (uint64_t)x.e[2 * w] | ((uint64_t)x.e[2 * w + 1] << 32);
+            add_word_terms(sums, log2b, lanes, t0 + 8u * w, word, nvalid > 8 * w, lane);
+        }
+    }
+    __syncthreads();
+
+    // one thread per block: finish the two hashes and compare with HashCache
+    const unsigned long long kglob = hash_base[td.unit] + (unsigned long long)td.tile_in_unit * nbt;
+    for (uint32_t b0 = 0; b0 < nbt; b0 += kThreads) {  // nbt <= 512: a single round
+        const uint32_t b = b0 + tid;
+        bool changed = false;
+        if (b < nblk) {
+            const uint32_t L = min(B, nv - (b << log2b));
+            ulonglong2 h;
+            h.x = mix64(sums[b][0] + L);
+            h.y = mix64(sums[b][1] + L);
+            if (INIT) {
+                hash_cache[kglob + b] = h;
+            } else {
+                const ulonglong2 old = hash_cache[kglob + b];
+                changed = old.x != h.x || old.y != h.y;
+                if (changed) hash_cache[kglob + b] = h;  // HashCache[i,k] <- h
+            }
+        }
+        if (!INIT) {
+            const uint32_t flags = __ballot_sync(0xffffffffu, changed);
+            if (lane == 0 && (b >> 5) < kFlagWords) {
+                ws_flags[(size_t)tile * kFlagWords + (b >> 5)] = flags;
+                if (flags) atomicAdd(&s_count, (uint32_t)__popc(flags));
+            }
+        }
+    }
+    if (!INIT) {
+        __syncthreads();
+        if (tid == 0) ws_count[tile] = s_count;
+    }
+}
+
+__device__ __forceinline__ uint32_t block_flag(const uint32_t* ws_flags, uint32_t first_tile, uint32_t log2b, uint64_t k) {
+    const uint32_t nbt = kTileValues >> log2b;
+    const uint64_t t = k / nbt;
+    const uint32_t r = (uint32_t)(k % nbt);
+    return (ws_flags[(size_t)(first_tile + t) * kFlagWords + (r >> 5)] >> (r & 31u)) & 1u;
+}
+
+// One thread block per unit: payload offset of every tile, bitmap bytes, pads, reported totals.
+__global__ void __launch_bounds__(256)
+hashed_unit_kernel(const TileDesc* __restrict__ tiles, const uint32_t* __restrict__ unit_first, uint32_t log2b,
+                   uint32_t sm_bytes_per_value, uint8_t* msgs, const uint32_t* __restrict__ ws_flags,
+                   const uint32_t* __restrict__ ws_count, uint32_t* __restrict__ ws_prefix,
+                   unsigned long long* __restrict__ wire_bytes, uint32_t* __restrict__ changed_blocks) {
+    __shared__ uint32_t s_warp[8];
+    __shared__ uint32_t s_carry;
+    const uint32_t unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const uint32_t first = unit_first[unit];
+    if (first == 0xffffffffu) {  // a unit without values
+        if (tid == 0) {
+            wire_bytes[unit] = 0;
+            changed_blocks[unit] = 0;
+        }
+        return;
+    }
+    const TileDesc td0 = load_tile_desc(tiles + first);
+    const uint64_t N = td0.n_unit;
+    const uint32_t B = 1u << log2b;
+    const uint32_t nbt = kTileValues >> log2b;
+    const uint64_t nb = num_blocks(N, log2b);
+    uint8_t* msg = msgs + td0.msg_off;
+    if (tid == 0) s_carry = 0;
+    __syncthreads();
+    for (uint32_t j0 = 0; j0 < td0.n_tiles_unit; j0 += 256u) {
+        const uint32_t j = j0 + tid;
+        const uint32_t cnt = j < td0.n_tiles_unit ? ws_count[first + j] : 0u;
+        uint32_t incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+            if ((int)lane >= o) incl += t;
+        }
+        if (lane == 31) s_warp[warp] = incl;
+        __syncthreads();
+        uint32_t wbase = 0;
+        for (uint32_t w = 0; w < warp; ++w) wbase += s_warp[w];
+        const uint32_t carry = s_carry;
+        if (j < td0.n_tiles_unit) ws_prefix[first + j] = carry + wbase + incl - cnt;
+        __syncthreads();
+        if (tid == 255) s_carry = carry + wbase + incl;
+        __syncthreads();
+    }
+    const uint64_t smoff = sm_offset(N, log2b);
+    const uint64_t payoff = smoff + pad16(N * sm_bytes_per_value);
+    if (tid == 0) {
+        const uint32_t total = s_carry;  // changed blocks of the unit
+        uint64_t bytes = (uint64_t)total << log2b;
+        const uint32_t rem = (uint32_t)(N & (B - 1u));
+        if (rem && block_flag(ws_flags, first, log2b, nb - 1)) bytes -= (B - rem);  // a changed short last block
+        wire_bytes[unit] = payoff + bytes;
+        changed_blocks[unit] = total;
+    }
+    // bitmap bytes (bit k of the unit = block k, LSB first), then the two pads
+    const uint64_t bm_bytes = bitmap_bytes(N, log2b);
+    for (uint64_t i = tid; i < bm_bytes; i += 256u) {
+        uint32_t byte = 0;
+        if (nbt >= 32) {  // the byte's eight flags lie in one word of one tile
+            const uint64_t k = 8 * i;
+            const uint32_t r = (uint32_t)(k % nbt);
+            byte = (ws_flags[(size_t)(first + k / nbt) * kFlagWords + (r >> 5)] >> (r & 31u)) & 0xFFu;
+        } else {
+            for (uint32_t r = 0; r < 8; ++r)
+                if (8 * i + r < nb) byte |= block_flag(ws_flags, first, log2b, 8 * i + r) << r;
+        }
+        msg[i] = (uint8_t)byte;
+    }
+    for (uint64_t b = bm_bytes + tid; b < smoff; b += 256u) msg[b] = 0;
+    for (uint64_t b = smoff + N * sm_bytes_per_value + tid; b < payoff; b += 256u) msg[b] = 0;
+}
+
+// One thread block per tile: exponents of the flagged blocks to the payload.
+template <int DT>
+__global__ void __launch_bounds__(kThreads)
+hashed_payload_kernel(const TileDesc* __restrict__ tiles, uint32_t log2b, const uint8_t* __restrict__ weights,
+                      uint8_t* msgs, const uint32_t* __restrict__ ws_flags, const uint32_t* __restrict__ ws_count,
+                      const uint32_t* __restrict__ ws_prefix) {
+    using P = Piece<DT>;
+    constexpr int VB = Traits<DT>::kValueBytes;
+    constexpr int SMB = Traits<DT>::kSmBytes;
+    __shared__ uint32_t bm[kFlagWords];
+    __shared__ uint32_t pre[kFlagWords];
+    const uint32_t tile = blockIdx.x, tid = threadIdx.x, lane = tid & 31u;
+    if (ws_count[tile] == 0) return;
+    if (tid < 32) {
+        const uint32_t word = lane < kFlagWords ? ws_flags[(size_t)tile * kFlagWords + lane] : 0u;
+        const uint32_t pc = __popc(word);
+        uint32_t incl = pc;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+            if ((int)lane >= o) incl += t;
+        }
+        if (lane < kFlagWords) {
+            bm[lane] = word;
+            pre[lane] = incl - pc;
+        }
+    }
+    __syncthreads();
+    const TileDesc td = load_tile_desc(tiles + tile);
+    const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
+    const uint32_t nv = (uint32_t)min((uint64_t)kTileValues, td.n_unit - v0);
+    uint8_t* pay = msgs + td.msg_off + payload_offset(td.n_unit, SMB, log2b) + ((uint64_t)ws_prefix[tile] << log2b);
+#pragma unroll
+    for (int p = 0; p < P::kPerThread; ++p) {
+        const uint32_t t0 = P::start(tid, p);
+        const int nvalid = piece_valid<DT>(t0, nv);
+        if (nvalid == 0) continue;
+        const uint32_t kb = t0 >> log2b;
+        const uint32_t word = bm[kb >> 5];
+        if (!((word >> (kb & 31u)) & 1u)) continue;
+        const uint32_t rank = pre[kb >> 5] + __popc(word & ((1u << (kb & 31u)) - 1u));
+        uint8_t* dst = pay + ((uint64_t)rank << log2b) + (t0 & ((1u << log2b) - 1u));
+        P x;
+        if (nvalid == P::kValues) {
+            x.template split_full<Global>(weights + td.w_off + (uint64_t)t0 * VB);
+            x.template store_exp_full<Global>(dst);
+        } else {
+            x.split_partial(weights + td.w_off + (uint64_t)t0 * VB, nvalid);
+            x.store_exp_partial(dst, nvalid);
+        }
+    }
+}
+
+}  // namespace ciera
+
+using namespace ciera;
+
+static bool misaligned16(const void* p) { return ((uintptr_t)p & 15u) != 0; }
+
+static int check_hashed_plan(const ciera_plan* p) {
+    if (!p) return CIERA_ERR_INVALID_ARG;
+    if (!p->tiles.empty() && !p->tiles_dev) return CIERA_ERR_NOT_BOUND;
+    if (is_fine(p->log2b)) return CIERA_ERR_UNSUPPORTED;  // blocks of fewer than 16 values: exact comparison only
+    return CIERA_OK;
+}
+
+extern "C" int ciera_hash_cache_init(const ciera_plan* p, void* hash_cache_dev, const void* weights_dev, void* stream) {
+    int rc = check_hashed_plan(p);
+    if (rc) return rc;
+    const uint32_t nt = (uint32_t)p->tiles.size();
+    if (nt == 0) return CIERA_OK;
+    if (!hash_cache_dev) return CIERA_ERR_INVALID_ARG;
+    if (misaligned16(hash_cache_dev) || misaligned16(weights_dev)) return CIERA_ERR_MISALIGNED;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (p->dtype == CIERA_BF16)
+        hashed_scan_kernel<CIERA_BF16, true><<<nt, kThreads, 0, s>>>(p->tiles_dev, p->hash_base_dev, p->log2b,
+                                                                     (const uint8_t*)weights_dev, (ulonglong2*)hash_cache_dev,
+                                                                     nullptr, nullptr, nullptr);
+    else
+        hashed_scan_kernel<CIERA_FP32, true><<<nt, kThreads, 0, s>>>(p->tiles_dev, p->hash_base_dev, p->log2b,
+                                                                     (const uint8_t*)weights_dev, (ulonglong2*)hash_cache_dev,
+                                                                     nullptr, nullptr, nullptr);
+    count_launch();
+    return check_launch();
+}
+
+extern "C" int ciera_encode_hashed(const ciera_plan* p, const void* weights_dev, void* hash_cache_dev, void* messages_dev,
+                                   uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* workspace_dev,
+                                   void* stream) {
+    int rc = check_hashed_plan(p);
+    if (rc) return rc;
+    if (p->n_units == 0) return CIERA_OK;
+    if (!wire_bytes_dev || !changed_blocks_dev) return CIERA_ERR_INVALID_ARG;
+    const uint32_t nt = (uint32_t)p->tiles.size();
+    cudaStream_t s = (cudaStream_t)stream;
+    if (nt != 0) {
+        if (!weights_dev || !hash_cache_dev || !messages_dev || !workspace_dev) return CIERA_ERR_INVALID_ARG;
+        if (misaligned16(weights_dev) || misaligned16(hash_cache_dev) || misaligned16(messages_dev) ||
+            misaligned16(workspace_dev))
+            return CIERA_ERR_MISALIGNED;
+    }
+    if (((uintptr_t)wire_bytes_dev & 7u) || ((uintptr_t)changed_blocks_dev & 3u)) return CIERA_ERR_MISALIGNED;
+    // scratch: 16 words of block flags per tile, then one count and one payload offset per tile;
+    // the scan pass writes all flags and counts, the unit pass all offsets
+    uint32_t* ws_flags = (uint32_t*)workspace_dev;
+    uint32_t* ws_count = ws_flags + (size_t)nt * kFlagWords;
+    uint32_t* ws_prefix = ws_count + nt;
+    const uint32_t smb = p->dtype == CIERA_BF16 ? 1u : 3u;
+    if (nt != 0) {
+        if (p->dtype == CIERA_BF16)
+            hashed_scan_kernel<CIERA_BF16, false><<<nt, kThreads, 0, s>>>(
+                p->tiles_dev, p->hash_base_dev, p->log2b, (const uint8_t*)weights_dev, (ulonglong2*)hash_cache_dev,
+                (uint8_t*)messages_dev, ws_flags, ws_count);
+        else
+            hashed_scan_kernel<CIERA_FP32, false><<<nt, kThreads, 0, s>>>(
+                p->tiles_dev, p->hash_base_dev, p->log2b, (const uint8_t*)weights_dev, (ulonglong2*)hash_cache_dev,
+                (uint8_t*)messages_dev, ws_flags, ws_count);
+        count_launch();
+        rc = check_launch();
+        if (rc) return rc;
+    }
+    hashed_unit_kernel<<<p->n_units, 256, 0, s>>>(p->tiles_dev, p->unit_first_dev, p->log2b, smb, (uint8_t*)messages_dev,
+                                                  ws_flags, ws_count, ws_prefix, (unsigned long long*)wire_bytes_dev,
+                                                  changed_blocks_dev);
+    count_launch();
+    rc = check_launch();
+    if (rc) return rc;
+    if (nt != 0) {
+        if (p->dtype == CIERA_BF16)
+            hashed_payload_kernel<CIERA_BF16><<<nt, kThreads, 0, s>>>(p->tiles_dev, p->log2b, (const uint8_t*)weights_dev,
+                                                                      (uint8_t*)messages_dev, ws_flags, ws_count, ws_prefix);
+        else
+            hashed_payload_kernel<CIERA_FP32><<<nt, kThreads, 0, s>>>(p->tiles_dev, p->log2b, (const uint8_t*)weights_dev,
+                                                                      (uint8_t*)messages_dev, ws_flags, ws_count, ws_prefix);
+        count_launch();
+        rc = check_launch();
+    }
+    return rc;
+}

@@ -64,6 +64,23 @@ extern "C" size_t ciera_message_bytes(uint64_t n, int dtype, uint32_t block, uin
 
 // ---------------------------------------------------------------------------------- plan
 
+namespace {
+struct ImageLayout {
+    size_t tiles, long_off, seq_off, hash_off, first_off, total;
+};
+size_t up16(size_t x) { return (x + 15) / 16 * 16; }
+ImageLayout image_layout(const ciera_plan* p) {
+    ImageLayout L;
+    L.tiles = p->tiles.size() * sizeof(TileDesc);
+    L.long_off = L.tiles;
+    L.seq_off = L.long_off + up16(p->long_units.size() * sizeof(uint32_t));
+    L.hash_off = L.seq_off + up16(p->seq_first.size() * sizeof(uint32_t));
+    L.first_off = L.hash_off + up16((size_t)p->n_units * sizeof(uint64_t));
+    L.total = L.first_off + up16((size_t)p->n_units * sizeof(uint32_t)) + 16;
+    return L;
+}
+}  // namespace
+
 extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units, int dtype, uint32_t block,
                                  ciera_plan** plan_out) {
     if (!plan_out) return CIERA_ERR_INVALID_ARG;
@@ -129,14 +146,25 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
     }
     p->seq_first.push_back((uint32_t)p->tiles.size());
     for (uint32_t u : longs) emit(u);
-    // device image: the tile table, then (16-byte aligned) the two index lists
-    const size_t tb = p->tiles.size() * sizeof(TileDesc);
-    const size_t lb = (p->long_units.size() * sizeof(uint32_t) + 15) / 16 * 16;
-    const size_t sb = p->seq_first.size() * sizeof(uint32_t);
-    p->image.assign(tb + lb + sb + 16, 0);
-    if (tb) memcpy(p->image.data(), p->tiles.data(), tb);
-    if (!p->long_units.empty()) memcpy(p->image.data() + tb, p->long_units.data(), p->long_units.size() * 4);
-    memcpy(p->image.data() + tb + lb, p->seq_first.data(), sb);
+    // per unit, in table order: where its tiles start and where its blocks start in a hash cache
+    p->unit_first.assign(n_units, 0xffffffffu);
+    for (size_t t = 0; t < p->tiles.size(); ++t)
+        if (p->tiles[t].tile_in_unit == 0) p->unit_first[p->tiles[t].unit] = (uint32_t)t;
+    p->hash_base.resize(n_units);
+    for (uint32_t u = 0; u < n_units; ++u) {
+        p->hash_base[u] = p->total_blocks;
+        p->total_blocks += (units_host[u].n_values + block - 1) / block;
+    }
+    // device image: the tile table, then (each 16-byte aligned) the index lists
+    const ImageLayout L = image_layout(p);
+    p->image.assign(L.total, 0);
+    if (L.tiles) memcpy(p->image.data(), p->tiles.data(), L.tiles);
+    if (!p->long_units.empty()) memcpy(p->image.data() + L.long_off, p->long_units.data(), p->long_units.size() * 4);
+    memcpy(p->image.data() + L.seq_off, p->seq_first.data(), p->seq_first.size() * 4);
+    if (n_units) {
+        memcpy(p->image.data() + L.hash_off, p->hash_base.data(), (size_t)n_units * 8);
+        memcpy(p->image.data() + L.first_off, p->unit_first.data(), (size_t)n_units * 4);
+    }
     *plan_out = p;
     return CIERA_OK;
 }
@@ -157,6 +185,16 @@ extern "C" size_t ciera_plan_workspace_bytes(const ciera_plan* p) {
     return p->tiles.size() * sizeof(unsigned long long) + 16;
 }
 
+extern "C" size_t ciera_plan_hash_cache_bytes(const ciera_plan* p) { return p ? (size_t)p->total_blocks * 16 : 0; }
+extern "C" size_t ciera_plan_unit_hash_offset(const ciera_plan* p, uint32_t unit) {
+    return (p && unit < p->n_units) ? (size_t)p->hash_base[unit] * 16 : 0;
+}
+extern "C" size_t ciera_plan_hashed_workspace_bytes(const ciera_plan* p) {
+    if (!p) return 0;
+    // 16 words of block flags, a count and a payload offset per tile
+    return p->tiles.size() * (16 + 2) * sizeof(uint32_t) + 16;
+}
+
 extern "C" int ciera_plan_bind(ciera_plan* p, void* plan_dev, size_t plan_dev_bytes, void* stream) {
     if (!p || !plan_dev) return CIERA_ERR_INVALID_ARG;
     if ((uintptr_t)plan_dev & 15u) return CIERA_ERR_MISALIGNED;
@@ -168,10 +206,12 @@ extern "C" int ciera_plan_bind(ciera_plan* p, void* plan_dev, size_t plan_dev_by
     e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return record_cuda_error(e);
     p->tiles_dev = (const TileDesc*)plan_dev;
-    const size_t tb = p->tiles.size() * sizeof(TileDesc);
-    const size_t lb = (p->long_units.size() * sizeof(uint32_t) + 15) / 16 * 16;
-    p->long_units_dev = (const uint32_t*)((const uint8_t*)plan_dev + tb);
-    p->seq_first_dev = (const uint32_t*)((const uint8_t*)plan_dev + tb + lb);
+    const ImageLayout L = image_layout(p);
+    const uint8_t* base = (const uint8_t*)plan_dev;
+    p->long_units_dev = (const uint32_t*)(base + L.long_off);
+    p->seq_first_dev = (const uint32_t*)(base + L.seq_off);
+    p->hash_base_dev = (const unsigned long long*)(base + L.hash_off);
+    p->unit_first_dev = (const uint32_t*)(base + L.first_off);
     return CIERA_OK;
 }
 

@@ -109,10 +109,15 @@ struct ciera_plan {
     std::vector<ciera::TileDesc> tiles;
     std::vector<uint32_t> long_units;  // first tile of every unit whose decode needs the prefix kernel
     std::vector<uint32_t> seq_first;   // first tile of every short unit, in table order, + end marker
-    std::vector<uint8_t> image;        // device image: tiles, then long_units, then seq_first
+    std::vector<uint32_t> unit_first;  // first tile of every unit (0xffffffff: a unit without values)
+    std::vector<uint64_t> hash_base;   // index of every unit's first block in a per-block hash cache
+    uint64_t total_blocks = 0;
+    std::vector<uint8_t> image;        // device image: tiles, long_units, seq_first, hash_base, unit_first
     const ciera::TileDesc* tiles_dev = nullptr;
     const uint32_t* long_units_dev = nullptr;
     const uint32_t* seq_first_dev = nullptr;
+    const unsigned long long* hash_base_dev = nullptr;
+    const uint32_t* unit_first_dev = nullptr;
 };
 
 namespace ciera {

@@ -54,6 +54,19 @@ class LayerCodec:
         ciera.cache_init(self.plan, self.sender_cache, weights, stream)
         ciera.cache_init(self.plan, self.receiver_cache, weights, stream)
 
+    # -- sender with a hash per block instead of the exponent cache -------------------------------
+    def init_hash_cache(self, weights: Optional[torch.Tensor], stream=None) -> None:
+        """Allocates (once) and fills the sender's HashCache and the scratch of the hashed encode."""
+        if getattr(self, "hash_cache", None) is None:
+            self.hash_cache = torch.zeros(max(self.plan.hash_cache_bytes, 16), dtype=torch.uint8, device=self.device)
+            self.hashed_workspace = torch.empty(max(self.plan.hashed_workspace_bytes, 16), dtype=torch.uint8,
+                                                device=self.device)
+        ciera.hash_cache_init(self.plan, self.hash_cache, weights, stream)
+
+    def encode_hashed(self, weights: torch.Tensor, stream=None) -> None:
+        ciera.encode_hashed(self.plan, weights, self.hash_cache, self.msg_send, self.wire_bytes, self.changed_blocks,
+                            self.hashed_workspace, stream)
+
     # -- the three stages -----------------------------------------------------------------------
     def encode(self, weights: torch.Tensor, stream=None) -> None:
         ciera.encode(self.plan, weights, self.sender_cache, self.msg_send, self.wire_bytes, self.changed_blocks,
