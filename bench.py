@@ -58,6 +58,9 @@ def parse_args():
     ap.add_argument("--shapes", default="olmoe", choices=["olmoe", "mixed"],
                     help="olmoe: 64 experts x 3 matrices per layer; mixed: 256 fine-grained experts (2048x512, "
                          "2048x512, 512x2048) plus dense tensors of 4 KB ... 256 MB (the mixed-shape sweep)")
+    ap.add_argument("--detect", default="compare", choices=["compare", "hash"],
+                    help="sender-side change detection: exact comparison with an exponent cache, or a 128-bit "
+                         "hash per block (ciera_encode_hashed)")
     ap.add_argument("--f", type=float, default=0.22, help="fraction of segments updated (clustered model)")
     ap.add_argument("--schedule", default="pipelined", choices=["pipelined", "serial"])
     ap.add_argument("--no-e2e", action="store_true")
@@ -191,6 +194,8 @@ def build_stack(args, device, seed_base):
         wa.append(w.view(torch.uint8))
         wb.append(w5.view(torch.uint8))
         codec.init_caches(wa[-1])
+        if args.detect == "hash":
+            codec.init_hash_cache(wa[-1])
     torch.cuda.synchronize()
     return layers, wa, wb
 
@@ -230,12 +235,16 @@ def selection_report(args, ciera, codec, enc_ms, dec_ms, alpha=20e-6, beta=8e9):
     }
 
 
-def algorithmic_bytes(n_values, q, dtype, block):
+def algorithmic_bytes(n_values, q, dtype, block, detect="compare"):
     """HBM bytes per launch the method needs: (encode, transport, decode).  q = share of the
-    exponent bytes that travel (changed blocks); the bitmap is one bit per block."""
+    exponent bytes that travel (changed blocks); the bitmap is one bit per block.  The hashed sender
+    reads no exponent cache but reads the weights of changed blocks twice and keeps 16 bytes per block."""
     vb, smb = (2, 1) if dtype == "bf16" else (4, 3)
     bm = 1.0 / (8 * block)
-    enc = n_values * (vb + 1 + smb + bm + 2 * q)
+    if detect == "hash":
+        enc = n_values * (vb + smb + bm + q * (vb + 1) + 16.0 * (1 + q) / block)
+    else:
+        enc = n_values * (vb + 1 + smb + bm + 2 * q)
     tra = 2 * n_values * (smb + bm + q)
     dec = n_values * (smb + bm + (1 - q) + q + vb + q)
     return enc, tra, dec
@@ -253,7 +262,10 @@ def run_step(layers, weights, s_enc, s_dec, events, schedule, timers=None, decod
         if timers is not None:
             t = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
             t[0].record(s_enc)
-        codec.encode(w, s_enc)
+        if getattr(codec, "hash_cache", None) is not None:
+            codec.encode_hashed(w, s_enc)
+        else:
+            codec.encode(w, s_enc)
         if timers is not None:
             t[1].record(s_enc)
             t[2].record(s_enc)
@@ -372,6 +384,8 @@ def workload_config(args):
         "l2": "inputs larger than L2 (no flush needed)",
         "schedule": args.schedule,
         "round_trip": "encode + device-to-device transport + decode",
+        "change_detection": "exact comparison with a sender-side exponent cache" if args.detect == "compare"
+                            else "128-bit hash per block (HashCache), three launches per encode",
     }
 
 
@@ -480,7 +494,7 @@ def main():
     enc_ms, tra_ms, dec_ms = [float(np.mean([t[2 * i].elapsed_time(t[2 * i + 1]) for t in serial_timers]))
                               for i in range(3)]
     n_layer = layers[0].plan.total_values
-    a_enc, a_tra, a_dec = algorithmic_bytes(n_layer, q, args.dtype, args.block)
+    a_enc, a_tra, a_dec = algorithmic_bytes(n_layer, q, args.dtype, args.block, args.detect)
     enc_gbs = a_enc / (enc_ms * 1e-3) / 1e9
     dec_gbs = a_dec / (dec_ms * 1e-3) / 1e9
     tra_gbs = a_tra / (tra_ms * 1e-3) / 1e9
@@ -500,7 +514,8 @@ def main():
         return torch.equal(c.weights_out[: w.numel()][keep], w[keep])
 
     verified = all(same_weights(c, w) for c, w in zip(layers, last_w))
-    verified = verified and all(torch.equal(c.sender_cache, c.receiver_cache) for c in layers)
+    if args.detect == "compare":
+        verified = verified and all(torch.equal(c.sender_cache, c.receiver_cache) for c in layers)
     sampled = 0
     if rank == 0:
         from oracle import ciera_oracle as ora
@@ -521,7 +536,7 @@ def main():
                 got = c.msg_recv[mo : mo + wbytes].cpu().numpy()
                 verified = verified and int(c.wire_bytes[ui].item()) == wbytes and np.array_equal(got, m)
                 verified = verified and int(c.changed_blocks[ui].item()) == cb
-                verified = verified and np.array_equal(c.sender_cache[co : co + n].cpu().numpy(), cache)
+                verified = verified and np.array_equal(c.receiver_cache[co : co + n].cpu().numpy(), cache)
                 sampled += 1
 
     out = {
@@ -552,7 +567,7 @@ def main():
                                  "per": "layer launch inside the two-stream timed region (kernels overlap)"},
         "serial_ms_per_step": serial_ms_per_step,
         "roofline": {
-            "bound": "hbm", "kernel": "encode_kernel", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
+            "bound": "hbm", "kernel": "encode_kernel" if args.detect == "compare" else "hashed encode (scan + unit + payload launches)", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
             "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBps": enc_gbs / NOMINAL_HBM_GBS,
             "traffic": (NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE * n_layer
                         if args.dtype == "bf16" and args.block == 512 and args.update == "clustered" else None),
@@ -574,7 +589,7 @@ def main():
         out["selection"] = selection_report(args, ciera, layers[-1], enc_ms, dec_ms)
 
     # ---- per-kernel numbers with each kernel alone on the GPU, three change regimes (one layer)
-    if not args.no_regimes and rank == 0:
+    if not args.no_regimes and rank == 0 and args.detect == "compare":
         out["kernels_alone"] = kernels_alone(args, layers[0], wa[0], wb[0], peak)
 
     # ---- end to end through the host-buffer entry point (weights start and end in host memory)

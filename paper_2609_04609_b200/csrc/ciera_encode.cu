@@ -33,6 +33,7 @@
 // consumers only for a resolver that is several tiles late, so a tile's status is published as
 // soon as its votes are in.
 #include "ciera_bits.cuh"
+#include "ciera_lookback.cuh"
 #include "ciera_pipe.cuh"
 
 namespace ciera {
@@ -153,38 +154,6 @@ struct TileWalk {
     }
 };
 
-__device__ __forceinline__ unsigned long long ld_status(const unsigned long long* p) {
-    unsigned long long v;
-    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_status(unsigned long long* p, unsigned long long v) {
-    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
-}
-
-// Polls a tile status word until its flag is set.  Bounded: after kMaxPolls reads it gives up,
-// raises CIERA_ERR_TIMEOUT and returns "prefix 0" so that the caller finishes (with unspecified
-// output) instead of hanging.
-__device__ __forceinline__ unsigned long long wait_status(const unsigned long long* p, int32_t* status) {
-    unsigned long long st = ld_status(p);
-    uint32_t polls = 0;
-    while ((st >> 62) == 0) {
-        if (++polls > kMaxPolls) {
-            if (status) atomicCAS(status, 0, (int32_t)CIERA_ERR_TIMEOUT);
-            return kFlagPrefix;
-        }
-        if (polls > 16) __nanosleep(polls > 1024 ? 400 : 40);
-        st = ld_status(p);
-    }
-    return st;
-}
-
-__device__ __forceinline__ uint64_t warp_sum_u64(uint64_t v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
-
 // Block flags of a tile from the vote bits "my piece differs" (one warp).  `pl2` = log2 of the
 // values per piece.  Fills bm (one bit per block of the tile) and pre (set bits before each word);
 // returns the number of changed blocks of the tile.
@@ -285,75 +254,6 @@ __device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t 
         for (uint32_t b = lane; b < nbytes; b += 32) msg[byte0 + b] = (uint8_t)(bm[b >> 2] >> ((b & 3u) * 8u));
     }
     return agg;
-}
-
-// The unit's last tile reports the totals and zeroes the two pads (one warp).
-template <int DT>
-__device__ __forceinline__ void finish_unit(const TileDesc& td, uint32_t log2b, uint64_t total, uint8_t* msgs,
-                                            unsigned long long* wire_bytes, uint32_t* changed_blocks, uint32_t lane) {
-    constexpr int SMB = Traits<DT>::kSmBytes;
-    const uint64_t N = td.n_unit;
-    const uint32_t B = 1u << log2b;
-    uint8_t* msg = msgs + td.msg_off;
-    const uint64_t smoff = sm_offset(N, log2b);
-    const uint64_t payoff = smoff + pad16(N * SMB);
-    if (lane == 0) {
-        wire_bytes[td.unit] = payoff + total;
-        changed_blocks[td.unit] = (uint32_t)((total + B - 1u) >> log2b);
-    }
-    for (uint64_t b = bitmap_bytes(N, log2b) + lane; b < smoff; b += 32) msg[b] = 0;
-    for (uint64_t b = smoff + N * SMB + lane; b < payoff; b += 32) msg[b] = 0;
-}
-
-// Resolver warp, one spread tile: exclusive prefix of the payload bytes over the earlier tiles of
-// the same unit by a single-pass look-back over the status words, then the duties that need it.
-// Returns the tile's exclusive payload offset inside its unit.
-template <int DT>
-__device__ __forceinline__ uint64_t resolve_tile(const TileDesc& td, uint32_t tile, uint32_t log2b, uint64_t agg,
-                                                 const uint32_t* bm, uint8_t* msgs, unsigned long long* wire_bytes,
-                                                 uint32_t* changed_blocks, unsigned long long* tile_status,
-                                                 int32_t* status, uint32_t lane) {
-    const uint32_t nbt = kTileValues >> log2b;
-    uint8_t* msg = msgs + td.msg_off;
-    const uint32_t mybits = nbt < 8 ? bm[0] : 0u;
-
-    uint64_t excl = 0;
-    if (td.tile_in_unit != 0) {
-        int64_t hi = (int64_t)tile - 1;
-        while (true) {
-            const int64_t idx = hi - (int64_t)lane;
-            unsigned long long st = kFlagPrefix;  // "prefix 0" stands before the unit's first tile
-            if (idx >= (int64_t)td.first_tile) st = wait_status(tile_status + idx, status);
-            __syncwarp();
-            const uint32_t pmask = __ballot_sync(0xffffffffu, (st >> 62) == 2ull);
-            const uint32_t first = pmask ? (uint32_t)__ffs(pmask) - 1u : 31u;
-            excl += warp_sum_u64(lane <= first ? (st & kValueMask) : 0ull);
-            if (pmask) break;
-            hi -= 32;
-        }
-        if (lane == 0)
-            st_status(tile_status + tile, kFlagPrefix | ((unsigned long long)mybits << kBitsShift) | (excl + agg));
-    }
-
-    // tiles of fewer than 8 blocks share a bitmap byte: the last tile of each byte collects the
-    // bits its predecessors published in their status words
-    if (nbt < 8) {
-        const uint32_t tpb = 8u / nbt;
-        const uint32_t p = td.tile_in_unit & (tpb - 1u);
-        if (p == tpb - 1u || td.tile_in_unit == td.n_tiles_unit - 1u) {
-            uint32_t part = 0;
-            if (lane < p) {
-                unsigned long long st = wait_status(tile_status + (tile - p + lane), status);
-                part = (uint32_t)((st >> kBitsShift) & 0x3Full) << (lane * nbt);
-            }
-            __syncwarp();
-            part = __reduce_or_sync(0xffffffffu, part);
-            if (lane == 0) msg[td.tile_in_unit / tpb] = (uint8_t)(part | (mybits << (p * nbt)));
-        }
-    }
-    if (td.tile_in_unit == td.n_tiles_unit - 1u)
-        finish_unit<DT>(td, log2b, excl + agg, msgs, wire_bytes, changed_blocks, lane);
-    return excl;
 }
 
 // payload <- exponents of changed blocks in block order; cache refreshed for the same blocks.

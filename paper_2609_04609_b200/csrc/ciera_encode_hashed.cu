@@ -27,7 +27,10 @@ namespace ciera {
 constexpr uint64_t kGamma = 0x9E3779B97F4A7C15ull;
 constexpr uint64_t kSeed1 = 0x0000000000000000ull;
 constexpr uint64_t kSeed2 = 0x6A09E667F3BCC908ull;
-constexpr uint32_t kFlagWords = kBitmapWords;  // 16 words of block flags per tile in the scratch
+// Scratch record of a tile: 16 words of block flags, the number of set flags, and the number of
+// set flags in the unit's earlier tiles.
+constexpr uint32_t kFlagWords = kBitmapWords;
+constexpr uint32_t kRecCount = kFlagWords, kRecPrefix = kFlagWords + 1, kRecWords = kFlagWords + 2;
 
 __device__ __forceinline__ uint64_t mix64(uint64_t z) {
     z ^= z >> 30;
@@ -61,8 +64,7 @@ __device__ __forceinline__ void add_word_terms(unsigned long long (*sums)[2], ui
 template <int DT, bool INIT>
 __global__ void __launch_bounds__(kThreads)
 hashed_scan_kernel(const TileDesc* __restrict__ tiles, const unsigned long long* __restrict__ hash_base, uint32_t log2b,
-                   const uint8_t* __restrict__ weights, ulonglong2* hash_cache, uint8_t* msgs, uint32_t* ws_flags,
-                   uint32_t* ws_count) {
+                   const uint8_t* __restrict__ weights, ulonglong2* hash_cache, uint8_t* msgs, uint32_t* ws) {
     using P = Piece<DT>;
     constexpr int VB = Traits<DT>::kValueBytes;
     constexpr int SMB = Traits<DT>::kSmBytes;
@@ -76,6 +78,11 @@ hashed_scan_kernel(const TileDesc* __restrict__ tiles, const unsigned long long*
     const uint32_t nbt = kTileValues >> log2b;
     const uint32_t nblk = (nv + B - 1u) >> log2b;
 
+    // the cached hash of "my" block (thread b takes block b, nbt <= 512) is fetched first, so that
+    // its latency passes while the tile is hashed
+    const unsigned long long kglob = hash_base[td.unit] + (unsigned long long)td.tile_in_unit * nbt;
+    ulonglong2 old = make_ulonglong2(0ull, 0ull);
+    if (!INIT && tid < nblk) old = hash_cache[kglob + tid];
     for (uint32_t b = tid; b < nbt; b += kThreads) sums[b][0] = sums[b][1] = 0ull;
     if (tid == 0) s_count = 0;
     __syncthreads();
@@ -111,49 +118,36 @@ hashed_scan_kernel(const TileDesc* __restrict__ tiles, const unsigned long long*
     __syncthreads();
 
     // one thread per block: finish the two hashes and compare with HashCache
-    const unsigned long long kglob = hash_base[td.unit] + (unsigned long long)td.tile_in_unit * nbt;
-    for (uint32_t b0 = 0; b0 < nbt; b0 += kThreads) {  // nbt <= 512: a single round
-        const uint32_t b = b0 + tid;
-        bool changed = false;
-        if (b < nblk) {
-            const uint32_t L = min(B, nv - (b << log2b));
-            ulonglong2 h;
-            h.x = mix64(sums[b][0] + L);
-            h.y = mix64(sums[b][1] + L);
-            if (INIT) {
-                hash_cache[kglob + b] = h;
-            } else {
-                const ulonglong2 old = hash_cache[kglob + b];
-                changed = old.x != h.x || old.y != h.y;
-                if (changed) hash_cache[kglob + b] = h;  // HashCache[i,k] <- h
-            }
-        }
-        if (!INIT) {
-            const uint32_t flags = __ballot_sync(0xffffffffu, changed);
-            if (lane == 0 && (b >> 5) < kFlagWords) {
-                ws_flags[(size_t)tile * kFlagWords + (b >> 5)] = flags;
-                if (flags) atomicAdd(&s_count, (uint32_t)__popc(flags));
-            }
-        }
+    bool changed = false;
+    if (tid < nblk) {
+        const uint32_t L = min(B, nv - (tid << log2b));
+        ulonglong2 h;
+        h.x = mix64(sums[tid][0] + L);
+        h.y = mix64(sums[tid][1] + L);
+        changed = old.x != h.x || old.y != h.y;
+        if (INIT || changed) hash_cache[kglob + tid] = h;  // HashCache[i,k] <- h
     }
-    if (!INIT) {
-        __syncthreads();
-        if (tid == 0) ws_count[tile] = s_count;
+    if (INIT) return;
+    const uint32_t flags = __ballot_sync(0xffffffffu, changed);
+    if (lane == 0) {  // 16 warps write the tile's 16 flag words
+        ws[(size_t)tile * kRecWords + (tid >> 5)] = flags;
+        if (flags) atomicAdd(&s_count, (uint32_t)__popc(flags));
     }
+    __syncthreads();
+    if (tid == 0) ws[(size_t)tile * kRecWords + kRecCount] = s_count;
 }
 
-__device__ __forceinline__ uint32_t block_flag(const uint32_t* ws_flags, uint32_t first_tile, uint32_t log2b, uint64_t k) {
+__device__ __forceinline__ uint32_t block_flag(const uint32_t* ws, uint32_t first_tile, uint32_t log2b, uint64_t k) {
     const uint32_t nbt = kTileValues >> log2b;
     const uint64_t t = k / nbt;
     const uint32_t r = (uint32_t)(k % nbt);
-    return (ws_flags[(size_t)(first_tile + t) * kFlagWords + (r >> 5)] >> (r & 31u)) & 1u;
+    return (ws[(size_t)(first_tile + t) * kRecWords + (r >> 5)] >> (r & 31u)) & 1u;
 }
 
 // One thread block per unit: payload offset of every tile, bitmap bytes, pads, reported totals.
 __global__ void __launch_bounds__(256)
 hashed_unit_kernel(const TileDesc* __restrict__ tiles, const uint32_t* __restrict__ unit_first, uint32_t log2b,
-                   uint32_t sm_bytes_per_value, uint8_t* msgs, const uint32_t* __restrict__ ws_flags,
-                   const uint32_t* __restrict__ ws_count, uint32_t* __restrict__ ws_prefix,
+                   uint32_t sm_bytes_per_value, uint8_t* msgs, uint32_t* ws,
                    unsigned long long* __restrict__ wire_bytes, uint32_t* __restrict__ changed_blocks) {
     __shared__ uint32_t s_warp[8];
     __shared__ uint32_t s_carry;
@@ -176,7 +170,7 @@ hashed_unit_kernel(const TileDesc* __restrict__ tiles, const uint32_t* __restric
     __syncthreads();
     for (uint32_t j0 = 0; j0 < td0.n_tiles_unit; j0 += 256u) {
         const uint32_t j = j0 + tid;
-        const uint32_t cnt = j < td0.n_tiles_unit ? ws_count[first + j] : 0u;
+        const uint32_t cnt = j < td0.n_tiles_unit ? ws[(size_t)(first + j) * kRecWords + kRecCount] : 0u;
         uint32_t incl = cnt;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -188,7 +182,7 @@ hashed_unit_kernel(const TileDesc* __restrict__ tiles, const uint32_t* __restric
         uint32_t wbase = 0;
         for (uint32_t w = 0; w < warp; ++w) wbase += s_warp[w];
         const uint32_t carry = s_carry;
-        if (j < td0.n_tiles_unit) ws_prefix[first + j] = carry + wbase + incl - cnt;
+        if (j < td0.n_tiles_unit) ws[(size_t)(first + j) * kRecWords + kRecPrefix] = carry + wbase + incl - cnt;
         __syncthreads();
         if (tid == 255) s_carry = carry + wbase + incl;
         __syncthreads();
@@ -199,7 +193,7 @@ hashed_unit_kernel(const TileDesc* __restrict__ tiles, const uint32_t* __restric
         const uint32_t total = s_carry;  // changed blocks of the unit
         uint64_t bytes = (uint64_t)total << log2b;
         const uint32_t rem = (uint32_t)(N & (B - 1u));
-        if (rem && block_flag(ws_flags, first, log2b, nb - 1)) bytes -= (B - rem);  // a changed short last block
+        if (rem && block_flag(ws, first, log2b, nb - 1)) bytes -= (B - rem);  // a changed short last block
         wire_bytes[unit] = payoff + bytes;
         changed_blocks[unit] = total;
     }
@@ -210,10 +204,10 @@ hashed_unit_kernel(const TileDesc* __restrict__ tiles, const uint32_t* __restric
         if (nbt >= 32) {  // the byte's eight flags lie in one word of one tile
             const uint64_t k = 8 * i;
             const uint32_t r = (uint32_t)(k % nbt);
-            byte = (ws_flags[(size_t)(first + k / nbt) * kFlagWords + (r >> 5)] >> (r & 31u)) & 0xFFu;
+            byte = (ws[(size_t)(first + k / nbt) * kRecWords + (r >> 5)] >> (r & 31u)) & 0xFFu;
         } else {
             for (uint32_t r = 0; r < 8; ++r)
-                if (8 * i + r < nb) byte |= block_flag(ws_flags, first, log2b, 8 * i + r) << r;
+                if (8 * i + r < nb) byte |= block_flag(ws, first, log2b, 8 * i + r) << r;
         }
         msg[i] = (uint8_t)byte;
     }
@@ -221,48 +215,59 @@ hashed_unit_kernel(const TileDesc* __restrict__ tiles, const uint32_t* __restric
     for (uint64_t b = smoff + N * sm_bytes_per_value + tid; b < payoff; b += 256u) msg[b] = 0;
 }
 
-// One thread block per tile: exponents of the flagged blocks to the payload.
+// One thread block per tile, every warp on its own (no barrier): exponents of the flagged blocks to
+// the payload.  A warp first looks at the flags of its own pieces and leaves if none is set;
+// otherwise it works out the ranks from the tile's scratch record with shuffles and fetches the
+// weights of its flagged pieces a second time.
 template <int DT>
 __global__ void __launch_bounds__(kThreads)
 hashed_payload_kernel(const TileDesc* __restrict__ tiles, uint32_t log2b, const uint8_t* __restrict__ weights,
-                      uint8_t* msgs, const uint32_t* __restrict__ ws_flags, const uint32_t* __restrict__ ws_count,
-                      const uint32_t* __restrict__ ws_prefix) {
+                      uint8_t* msgs, const uint32_t* __restrict__ ws) {
     using P = Piece<DT>;
     constexpr int VB = Traits<DT>::kValueBytes;
     constexpr int SMB = Traits<DT>::kSmBytes;
-    __shared__ uint32_t bm[kFlagWords];
-    __shared__ uint32_t pre[kFlagWords];
     const uint32_t tile = blockIdx.x, tid = threadIdx.x, lane = tid & 31u;
-    if (ws_count[tile] == 0) return;
-    if (tid < 32) {
-        const uint32_t word = lane < kFlagWords ? ws_flags[(size_t)tile * kFlagWords + lane] : 0u;
-        const uint32_t pc = __popc(word);
-        uint32_t incl = pc;
+    const uint32_t* rec = ws + (size_t)tile * kRecWords;
+    // which of this lane's pieces are flagged; most warps leave here
+    uint32_t word[P::kPerThread];
+    bool flagged[P::kPerThread];
+    bool any = false;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
-            if ((int)lane >= o) incl += t;
-        }
-        if (lane < kFlagWords) {
-            bm[lane] = word;
-            pre[lane] = incl - pc;
-        }
+    for (int p = 0; p < P::kPerThread; ++p) {
+        const uint32_t kb = P::start(tid, p) >> log2b;
+        word[p] = __ldg(rec + (kb >> 5));
+        flagged[p] = (word[p] >> (kb & 31u)) & 1u;
+        any |= flagged[p];
     }
-    __syncthreads();
+    if (!__any_sync(0xffffffffu, any)) return;
+    // ranks: set flags before each word of the record (every lane of the warp takes part)
+    const uint32_t word_l = lane < kFlagWords ? __ldg(rec + lane) : 0u;
+    const uint32_t prefix = __ldg(rec + kRecPrefix);
+    const uint32_t pc = __popc(word_l);
+    uint32_t incl = pc;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+        if ((int)lane >= o) incl += t;
+    }
+    const uint32_t pre_l = incl - pc;
+    uint32_t rank[P::kPerThread];
+#pragma unroll
+    for (int p = 0; p < P::kPerThread; ++p) {
+        const uint32_t kb = P::start(tid, p) >> log2b;
+        rank[p] = __shfl_sync(0xffffffffu, pre_l, kb >> 5) + __popc(word[p] & ((1u << (kb & 31u)) - 1u));
+    }
+    if (!any) return;
     const TileDesc td = load_tile_desc(tiles + tile);
     const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
     const uint32_t nv = (uint32_t)min((uint64_t)kTileValues, td.n_unit - v0);
-    uint8_t* pay = msgs + td.msg_off + payload_offset(td.n_unit, SMB, log2b) + ((uint64_t)ws_prefix[tile] << log2b);
+    uint8_t* pay = msgs + td.msg_off + payload_offset(td.n_unit, SMB, log2b) + ((uint64_t)prefix << log2b);
 #pragma unroll
     for (int p = 0; p < P::kPerThread; ++p) {
         const uint32_t t0 = P::start(tid, p);
         const int nvalid = piece_valid<DT>(t0, nv);
-        if (nvalid == 0) continue;
-        const uint32_t kb = t0 >> log2b;
-        const uint32_t word = bm[kb >> 5];
-        if (!((word >> (kb & 31u)) & 1u)) continue;
-        const uint32_t rank = pre[kb >> 5] + __popc(word & ((1u << (kb & 31u)) - 1u));
-        uint8_t* dst = pay + ((uint64_t)rank << log2b) + (t0 & ((1u << log2b) - 1u));
+        if (!flagged[p] || nvalid == 0) continue;
+        uint8_t* dst = pay + ((uint64_t)rank[p] << log2b) + (t0 & ((1u << log2b) - 1u));
         P x;
         if (nvalid == P::kValues) {
             x.template split_full<Global>(weights + td.w_off + (uint64_t)t0 * VB);
@@ -298,11 +303,11 @@ extern "C" int ciera_hash_cache_init(const ciera_plan* p, void* hash_cache_dev, 
     if (p->dtype == CIERA_BF16)
         hashed_scan_kernel<CIERA_BF16, true><<<nt, kThreads, 0, s>>>(p->tiles_dev, p->hash_base_dev, p->log2b,
                                                                      (const uint8_t*)weights_dev, (ulonglong2*)hash_cache_dev,
-                                                                     nullptr, nullptr, nullptr);
+                                                                     nullptr, nullptr);
     else
         hashed_scan_kernel<CIERA_FP32, true><<<nt, kThreads, 0, s>>>(p->tiles_dev, p->hash_base_dev, p->log2b,
                                                                      (const uint8_t*)weights_dev, (ulonglong2*)hash_cache_dev,
-                                                                     nullptr, nullptr, nullptr);
+                                                                     nullptr, nullptr);
     count_launch();
     return check_launch();
 }
@@ -323,38 +328,35 @@ extern "C" int ciera_encode_hashed(const ciera_plan* p, const void* weights_dev,
             return CIERA_ERR_MISALIGNED;
     }
     if (((uintptr_t)wire_bytes_dev & 7u) || ((uintptr_t)changed_blocks_dev & 3u)) return CIERA_ERR_MISALIGNED;
-    // scratch: 16 words of block flags per tile, then one count and one payload offset per tile;
-    // the scan pass writes all flags and counts, the unit pass all offsets
-    uint32_t* ws_flags = (uint32_t*)workspace_dev;
-    uint32_t* ws_count = ws_flags + (size_t)nt * kFlagWords;
-    uint32_t* ws_prefix = ws_count + nt;
+    // scratch: one record of 18 words per tile; the scan pass writes every record's flags and count,
+    // the unit pass its payload offset
+    uint32_t* ws = (uint32_t*)workspace_dev;
     const uint32_t smb = p->dtype == CIERA_BF16 ? 1u : 3u;
     if (nt != 0) {
         if (p->dtype == CIERA_BF16)
             hashed_scan_kernel<CIERA_BF16, false><<<nt, kThreads, 0, s>>>(
                 p->tiles_dev, p->hash_base_dev, p->log2b, (const uint8_t*)weights_dev, (ulonglong2*)hash_cache_dev,
-                (uint8_t*)messages_dev, ws_flags, ws_count);
+                (uint8_t*)messages_dev, ws);
         else
             hashed_scan_kernel<CIERA_FP32, false><<<nt, kThreads, 0, s>>>(
                 p->tiles_dev, p->hash_base_dev, p->log2b, (const uint8_t*)weights_dev, (ulonglong2*)hash_cache_dev,
-                (uint8_t*)messages_dev, ws_flags, ws_count);
+                (uint8_t*)messages_dev, ws);
         count_launch();
         rc = check_launch();
         if (rc) return rc;
     }
     hashed_unit_kernel<<<p->n_units, 256, 0, s>>>(p->tiles_dev, p->unit_first_dev, p->log2b, smb, (uint8_t*)messages_dev,
-                                                  ws_flags, ws_count, ws_prefix, (unsigned long long*)wire_bytes_dev,
-                                                  changed_blocks_dev);
+                                                  ws, (unsigned long long*)wire_bytes_dev, changed_blocks_dev);
     count_launch();
     rc = check_launch();
     if (rc) return rc;
     if (nt != 0) {
         if (p->dtype == CIERA_BF16)
             hashed_payload_kernel<CIERA_BF16><<<nt, kThreads, 0, s>>>(p->tiles_dev, p->log2b, (const uint8_t*)weights_dev,
-                                                                      (uint8_t*)messages_dev, ws_flags, ws_count, ws_prefix);
+                                                                      (uint8_t*)messages_dev, ws);
         else
             hashed_payload_kernel<CIERA_FP32><<<nt, kThreads, 0, s>>>(p->tiles_dev, p->log2b, (const uint8_t*)weights_dev,
-                                                                      (uint8_t*)messages_dev, ws_flags, ws_count, ws_prefix);
+                                                                      (uint8_t*)messages_dev, ws);
         count_launch();
         rc = check_launch();
     }
