@@ -250,41 +250,6 @@ def algorithmic_bytes(n_values, q, dtype, block, detect="compare"):
     return enc, tra, dec
 
 
-def run_step(layers, weights, s_enc, s_dec, events, schedule, timers=None, decoded=None):
-    """encode+transport of layer l on s_enc, decode of layer l on s_dec (same stream if serial).
-    `decoded[l]`: event recorded after the previous decode of layer l; the sender side of the next
-    step waits for it before it overwrites the layer's message buffers."""
-    import torch
-
-    for l, (codec, w) in enumerate(zip(layers, weights)):
-        if schedule == "pipelined" and decoded is not None:
-            s_enc.wait_event(decoded[l])
-        if timers is not None:
-            t = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
-            t[0].record(s_enc)
-        if getattr(codec, "hash_cache", None) is not None:
-            codec.encode_hashed(w, s_enc)
-        else:
-            codec.encode(w, s_enc)
-        if timers is not None:
-            t[1].record(s_enc)
-            t[2].record(s_enc)
-        codec.transport(s_enc)
-        if timers is not None:
-            t[3].record(s_enc)
-        if schedule == "pipelined":
-            events[l].record(s_enc)
-            s_dec.wait_event(events[l])
-        if timers is not None:
-            t[4].record(s_dec)
-        codec.decode(None, s_dec)
-        if schedule == "pipelined" and decoded is not None:
-            decoded[l].record(s_dec)
-        if timers is not None:
-            t[5].record(s_dec)
-            timers.append(t)
-
-
 def oracle_roundtrip_units(units, w_prev, w_cur, dtype_code, block, vb, threads):
     """CPU oracle (as it stands) on a list of units: cache init from w_prev, encode + decode of
     w_cur.  Returns seconds of wall time with ``threads`` host threads."""
@@ -424,20 +389,17 @@ def main():
     layers, wa, wb = build_stack(args, device, seed_base=rank_seed(rank))
     n_values = sum(c.plan.total_values for c in layers)
     weight_bytes = n_values * vb
-    s_enc, s_dec = torch.cuda.Stream(), torch.cuda.Stream()
-    if args.schedule == "serial":
-        s_dec = s_enc
-    events = [torch.cuda.Event() for _ in layers]
-    decoded = [torch.cuda.Event() for _ in layers]
-    for ev in decoded:
-        ev.record(torch.cuda.current_stream())
+    s_enc = torch.cuda.Stream()
+    s_dec = s_enc if args.schedule == "serial" else torch.cuda.Stream()
+    pipe = runtime.LayerPipeline(layers, s_enc, s_dec)
+    serial_pipe = runtime.LayerPipeline(layers, s_enc, s_enc)
 
     def weights_of(i):
         return wb if i % 2 == 0 else wa
 
     step_i = 0
     for _ in range(max(args.warmup, 3)):
-        run_step(layers, weights_of(step_i), s_enc, s_dec, events, args.schedule, None, decoded)
+        pipe.step(weights_of(step_i))
         step_i += 1
     barrier()
 
@@ -457,7 +419,7 @@ def main():
     s_enc.wait_event(ev0)
     s_dec.wait_event(ev0)
     for _ in range(args.steps):
-        run_step(layers, weights_of(step_i), s_enc, s_dec, events, args.schedule, timers, decoded)
+        pipe.step(weights_of(step_i), None, timers)
         step_i += 1
     cur.wait_stream(s_enc)
     cur.wait_stream(s_dec)
@@ -477,7 +439,7 @@ def main():
     barrier()
     sev0.record(s_enc)
     for _ in range(args.steps):
-        run_step(layers, weights_of(step_i), s_enc, s_enc, events, "serial", serial_timers)
+        serial_pipe.step(weights_of(step_i), None, serial_timers)
         step_i += 1
     sev1.record(s_enc)
     barrier()

@@ -144,3 +144,61 @@ def pipelined_step(layers: List[LayerCodec], weights: List[torch.Tensor], outs: 
         events[l].record(s_enc)
         s_dec.wait_event(events[l])
         layers[l].decode(outs[l], s_dec)
+
+
+class LayerPipeline:
+    """A stack of layers stepped repeatedly on two streams (see ``pipelined_step``).
+
+    Across iterations it keeps the dependency that the layers' buffers impose: the sender side of
+    layer l in iteration i+1 (it overwrites the layer's messages, lengths and scratch) starts only
+    after the decode of layer l in iteration i has finished.  ``timers``, if given, collects six CUDA
+    events per layer and step: around encode, transport (both on the sender stream) and decode."""
+
+    def __init__(self, layers: List[LayerCodec], s_enc: Optional[torch.cuda.Stream] = None,
+                 s_dec: Optional[torch.cuda.Stream] = None):
+        self.layers = layers
+        self.s_enc = s_enc if s_enc is not None else torch.cuda.Stream()
+        self.s_dec = s_dec if s_dec is not None else torch.cuda.Stream()
+        self.serial = self.s_enc == self.s_dec
+        self.sent = [torch.cuda.Event() for _ in layers]
+        self.decoded = [torch.cuda.Event() for _ in layers]
+        cur = torch.cuda.current_stream()
+        for ev in self.decoded:
+            ev.record(cur)
+
+    def step(self, weights: List[torch.Tensor], outs: Optional[List[Optional[torch.Tensor]]] = None,
+             timers: Optional[list] = None) -> None:
+        s_enc, s_dec = self.s_enc, self.s_dec
+        for l, (codec, w) in enumerate(zip(self.layers, weights)):
+            if not self.serial:
+                s_enc.wait_event(self.decoded[l])
+            t = [torch.cuda.Event(enable_timing=True) for _ in range(6)] if timers is not None else None
+            if t:
+                t[0].record(s_enc)
+            if getattr(codec, "hash_cache", None) is not None:
+                codec.encode_hashed(w, s_enc)
+            else:
+                codec.encode(w, s_enc)
+            if t:
+                t[1].record(s_enc)
+                t[2].record(s_enc)
+            codec.transport(s_enc)
+            if t:
+                t[3].record(s_enc)
+            if not self.serial:
+                self.sent[l].record(s_enc)
+                s_dec.wait_event(self.sent[l])
+            if t:
+                t[4].record(s_dec)
+            codec.decode(None if outs is None else outs[l], s_dec)
+            if not self.serial:
+                self.decoded[l].record(s_dec)
+            if t:
+                t[5].record(s_dec)
+                timers.append(t)
+
+    def wait(self) -> None:
+        """Makes the current stream wait for everything queued so far."""
+        cur = torch.cuda.current_stream()
+        cur.wait_stream(self.s_enc)
+        cur.wait_stream(self.s_dec)

@@ -258,6 +258,39 @@ def test_pipelined_stack_equals_serial(rt):
             assert torch.equal(x, y)
 
 
+@pytest.mark.parametrize("n_layers", [1, 3])
+def test_pipeline_of_many_iterations_reuses_layer_buffers_safely(rt, n_layers):
+    """Many iterations back to back on two streams, alternating between two iterates: with a single
+    layer the next iteration's sender side would overwrite the message that is still being decoded
+    unless it waits for that decode.  Every iteration must come out exact and with a clean status."""
+    ciera, runtime = rt
+    shapes = [r * c for r, c in wl.olmoe_layer_shapes(8)]
+    layers, wa, wb = [], [], []
+    for l in range(n_layers):
+        codec = runtime.LayerCodec.from_tensors(shapes, 16, "bf16", 512, DEV)
+        n = codec.weights_bytes // 2
+        gen = wl.make_generator(700 + l)
+        w0 = wl.init_weights(n, "bf16", gen)
+        w1 = wl.step_clustered(w0, gen, f=0.3)
+        layers.append(codec)
+        wa.append(to_dev_bytes(wl.as_bits(w0), DEV))
+        wb.append(to_dev_bytes(wl.as_bits(w1), DEV))
+        codec.init_caches(wa[-1])
+    outs = [[torch.empty_like(c.weights_out) for c in layers] for _ in range(8)]
+    pipe = runtime.LayerPipeline(layers)
+    torch.cuda.synchronize()
+    for i in range(8):
+        pipe.step(wb if i % 2 == 0 else wa, outs[i])
+    pipe.wait()
+    torch.cuda.synchronize()
+    for c in layers:
+        c.check_status()
+    for i in range(8):
+        want = wb if i % 2 == 0 else wa
+        for l in range(n_layers):
+            assert torch.equal(outs[i][l][: want[l].numel()], want[l]), f"iteration {i}, layer {l}"
+
+
 @pytest.mark.parametrize("dtype,block", [(0, 512), (1, 512), (0, 64)])
 def test_full_size_layer_sampled_units(rt, dtype, block):
     """One full OLMoE-shaped layer (64 experts x 3 matrices, 16 shards: 3072 units, 402 653 184 values) in the
