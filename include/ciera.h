@@ -282,6 +282,32 @@ CIERA_API int ciera_roundtrip_host(const ciera_plan* plan, const void* weights_h
                          void* weights_out_host, uint64_t* wire_bytes_host, const ciera_device_buffers* bufs,
                          void* stream);
 
+/* ---- entropy stage (Section 3.1; Algorithm 1: ANSEncode on the sender, ANSDecode on the receiver) ---
+ *
+ * Between ciera_encode (or ciera_encode_hashed) and the transport, ciera_entropy_encode replaces the
+ * payload of every message -- the exponents of the changed blocks -- by its rANS-coded form if that
+ * is strictly shorter, and lowers the unit's wire_bytes accordingly; bitmap and sign-plus-mantissa
+ * stay as they are.  Between the transport and ciera_decode, ciera_entropy_decode restores the raw
+ * payload in place (the receiver knows the raw length from the bitmap: a message of exactly that
+ * length carries the raw form) and sets wire_bytes back to the raw length, so that ciera_decode
+ * sees what the sender step had written.  The paper names a vendor library whose format is not
+ * public; coder and layout are this library's own: static model per unit (256 symbols,
+ * probabilities in 1/4096), 32-bit rANS states with 16-bit words, segments of 4096 payload bytes
+ * coded by 32 interleaved coders each; coded section = [256 x u16 frequencies][per segment a u32
+ * word count][segments: 32 x u32 final states, the words, 2 zero bytes if their number is odd].
+ *   messages_dev    device, in/out
+ *   wire_bytes_dev  device, n_units x uint64, in/out
+ *   scratch_dev     device, ciera_plan_entropy_scratch_bytes(plan) bytes, 16-byte aligned; contents
+ *                   need not be initialised
+ *   status_dev      device int32 or NULL: CIERA_ERR_CORRUPT if a coded section is inconsistent
+ *                   (that unit's payload is then left as received)
+ * One launch each, one thread block per unit; nothing waits inside the kernels. */
+CIERA_API size_t ciera_plan_entropy_scratch_bytes(const ciera_plan* plan);
+CIERA_API int ciera_entropy_encode(const ciera_plan* plan, void* messages_dev, uint64_t* wire_bytes_dev, void* scratch_dev,
+                                   void* stream);
+CIERA_API int ciera_entropy_decode(const ciera_plan* plan, void* messages_dev, uint64_t* wire_bytes_dev, void* scratch_dev,
+                                   int32_t* status_dev, void* stream);
+
 /* ---- selective compression: the gain rule of Section 3.2 (host only) ----------------------- */
 
 typedef struct ciera_gain_in {

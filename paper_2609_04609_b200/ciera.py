@@ -76,6 +76,9 @@ _SIGS = {
     "ciera_plan_hashed_workspace_bytes": ([_vp], _sz),
     "ciera_hash_cache_init": ([_vp] * 4, _i32),
     "ciera_encode_hashed": ([_vp] * 8, _i32),
+    "ciera_plan_entropy_scratch_bytes": ([_vp], _sz),
+    "ciera_entropy_encode": ([_vp] * 5, _i32),
+    "ciera_entropy_decode": ([_vp] * 6, _i32),
     "ciera_transport": ([_vp] * 6, _i32),
     "ciera_decode": ([_vp] * 8, _i32),
     "ciera_roundtrip_host": ([_vp, _vp, _sz, _vp, _vp, _vp, _vp], _i32),
@@ -163,6 +166,7 @@ class Plan:
         self.device_bytes = int(_lib.ciera_plan_device_bytes(h))
         self.workspace_bytes = int(_lib.ciera_plan_workspace_bytes(h))
         self.hash_cache_bytes = int(_lib.ciera_plan_hash_cache_bytes(h))
+        self.entropy_scratch_bytes = int(_lib.ciera_plan_entropy_scratch_bytes(h))
         self.hashed_workspace_bytes = int(_lib.ciera_plan_hashed_workspace_bytes(h))
         self.table = None
         if device is not None:
@@ -240,6 +244,19 @@ def encode_hashed(plan: Plan, weights, hash_cache, messages, wire_bytes, changed
     _check("ciera_encode_hashed",
            _lib.ciera_encode_hashed(plan.handle, _ptr(weights), _ptr(hash_cache), _ptr(messages), _ptr(wire_bytes),
                                     _ptr(changed_blocks), _ptr(workspace), _stream(stream)))
+
+
+def entropy_encode(plan: Plan, messages, wire_bytes, scratch, stream=None) -> None:
+    """rANS-codes the payload of every message in place where that shortens it (after encode)."""
+    _check("ciera_entropy_encode",
+           _lib.ciera_entropy_encode(plan.handle, _ptr(messages), _ptr(wire_bytes), _ptr(scratch), _stream(stream)))
+
+
+def entropy_decode(plan: Plan, messages, wire_bytes, scratch, status=None, stream=None) -> None:
+    """Restores the raw payload of every message in place (before decode)."""
+    _check("ciera_entropy_decode",
+           _lib.ciera_entropy_decode(plan.handle, _ptr(messages), _ptr(wire_bytes), _ptr(scratch), _ptr(status),
+                                     _stream(stream)))
 
 
 def transport(plan: Plan, src_messages, dst_messages, wire_bytes, workspace, stream=None) -> None:

@@ -66,7 +66,7 @@ extern "C" size_t ciera_message_bytes(uint64_t n, int dtype, uint32_t block, uin
 
 namespace {
 struct ImageLayout {
-    size_t tiles, long_off, seq_off, hash_off, first_off, total;
+    size_t tiles, long_off, seq_off, hash_off, first_off, seg_off, units_off, total;
 };
 size_t up16(size_t x) { return (x + 15) / 16 * 16; }
 ImageLayout image_layout(const ciera_plan* p) {
@@ -76,7 +76,9 @@ ImageLayout image_layout(const ciera_plan* p) {
     L.seq_off = L.long_off + up16(p->long_units.size() * sizeof(uint32_t));
     L.hash_off = L.seq_off + up16(p->seq_first.size() * sizeof(uint32_t));
     L.first_off = L.hash_off + up16((size_t)p->n_units * sizeof(uint64_t));
-    L.total = L.first_off + up16((size_t)p->n_units * sizeof(uint32_t)) + 16;
+    L.seg_off = L.first_off + up16((size_t)p->n_units * sizeof(uint32_t));
+    L.units_off = L.seg_off + up16((size_t)p->n_units * sizeof(uint64_t));
+    L.total = L.units_off + up16((size_t)p->n_units * sizeof(ciera_unit)) + 16;
     return L;
 }
 }  // namespace
@@ -151,9 +153,14 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
     for (size_t t = 0; t < p->tiles.size(); ++t)
         if (p->tiles[t].tile_in_unit == 0) p->unit_first[p->tiles[t].unit] = (uint32_t)t;
     p->hash_base.resize(n_units);
+    p->seg_base.resize(n_units);
     for (uint32_t u = 0; u < n_units; ++u) {
         p->hash_base[u] = p->total_blocks;
         p->total_blocks += (units_host[u].n_values + block - 1) / block;
+        // the payload of a unit has at most n_values bytes: that many 4096-byte segments
+        p->seg_base[u] = p->total_segments;
+        p->total_segments += (units_host[u].n_values + 4095) / 4096;
+        p->cache_extent = std::max<uint64_t>(p->cache_extent, units_host[u].cache_off + units_host[u].n_values);
     }
     // device image: the tile table, then (each 16-byte aligned) the index lists
     const ImageLayout L = image_layout(p);
@@ -164,6 +171,8 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
     if (n_units) {
         memcpy(p->image.data() + L.hash_off, p->hash_base.data(), (size_t)n_units * 8);
         memcpy(p->image.data() + L.first_off, p->unit_first.data(), (size_t)n_units * 4);
+        memcpy(p->image.data() + L.seg_off, p->seg_base.data(), (size_t)n_units * 8);
+        memcpy(p->image.data() + L.units_off, p->units.data(), (size_t)n_units * sizeof(ciera_unit));
     }
     *plan_out = p;
     return CIERA_OK;
@@ -212,6 +221,8 @@ extern "C" int ciera_plan_bind(ciera_plan* p, void* plan_dev, size_t plan_dev_by
     p->seq_first_dev = (const uint32_t*)(base + L.seq_off);
     p->hash_base_dev = (const unsigned long long*)(base + L.hash_off);
     p->unit_first_dev = (const uint32_t*)(base + L.first_off);
+    p->seg_base_dev = (const unsigned long long*)(base + L.seg_off);
+    p->units_dev = (const ciera_unit*)(base + L.units_off);
     return CIERA_OK;
 }
 

@@ -112,12 +112,17 @@ struct ciera_plan {
     std::vector<uint32_t> unit_first;  // first tile of every unit (0xffffffff: a unit without values)
     std::vector<uint64_t> hash_base;   // index of every unit's first block in a per-block hash cache
     uint64_t total_blocks = 0;
-    std::vector<uint8_t> image;        // device image: tiles, long_units, seq_first, hash_base, unit_first
+    std::vector<uint64_t> seg_base;    // index of every unit's first 4096-byte payload segment (entropy stage)
+    uint64_t total_segments = 0;
+    uint64_t cache_extent = 0;         // max over units of cache_off + n_values
+    std::vector<uint8_t> image;        // device image: tiles, long_units, seq_first, hash_base, unit_first, seg_base, units
     const ciera::TileDesc* tiles_dev = nullptr;
     const uint32_t* long_units_dev = nullptr;
     const uint32_t* seq_first_dev = nullptr;
     const unsigned long long* hash_base_dev = nullptr;
     const uint32_t* unit_first_dev = nullptr;
+    const unsigned long long* seg_base_dev = nullptr;
+    const ciera_unit* units_dev = nullptr;
 };
 
 namespace ciera {

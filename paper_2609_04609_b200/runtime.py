@@ -67,6 +67,21 @@ class LayerCodec:
         ciera.encode_hashed(self.plan, weights, self.hash_cache, self.msg_send, self.wire_bytes, self.changed_blocks,
                             self.hashed_workspace, stream)
 
+    # -- entropy stage around the transport --------------------------------------------------------
+    def _entropy_scratch(self) -> torch.Tensor:
+        if getattr(self, "entropy_scratch", None) is None:
+            self.entropy_scratch = torch.empty(max(self.plan.entropy_scratch_bytes, 16), dtype=torch.uint8,
+                                               device=self.device)
+        return self.entropy_scratch
+
+    def entropy_encode(self, stream=None) -> None:
+        """After encode: code the payloads of the messages to send (wire_bytes shrink)."""
+        ciera.entropy_encode(self.plan, self.msg_send, self.wire_bytes, self._entropy_scratch(), stream)
+
+    def entropy_decode(self, stream=None) -> None:
+        """After transport: restore the raw payloads of the received messages (wire_bytes grow back)."""
+        ciera.entropy_decode(self.plan, self.msg_recv, self.wire_bytes, self._entropy_scratch(), self.status, stream)
+
     # -- the three stages -----------------------------------------------------------------------
     def encode(self, weights: torch.Tensor, stream=None) -> None:
         ciera.encode(self.plan, weights, self.sender_cache, self.msg_send, self.wire_bytes, self.changed_blocks,
