@@ -61,6 +61,8 @@ def parse_args():
     ap.add_argument("--detect", default="compare", choices=["compare", "hash"],
                     help="sender-side change detection: exact comparison with an exponent cache, or a 128-bit "
                          "hash per block (ciera_encode_hashed)")
+    ap.add_argument("--entropy", action="store_true",
+                    help="rANS-code the changed exponents before the transport and restore them after it")
     ap.add_argument("--f", type=float, default=0.22, help="fraction of segments updated (clustered model)")
     ap.add_argument("--schedule", default="pipelined", choices=["pipelined", "serial"])
     ap.add_argument("--no-e2e", action="store_true")
@@ -391,8 +393,12 @@ def main():
     weight_bytes = n_values * vb
     s_enc = torch.cuda.Stream()
     s_dec = s_enc if args.schedule == "serial" else torch.cuda.Stream()
-    pipe = runtime.LayerPipeline(layers, s_enc, s_dec)
-    serial_pipe = runtime.LayerPipeline(layers, s_enc, s_enc)
+    if args.entropy:  # the stage's scratch is only used between a layer's launches: one buffer serves all layers
+        shared = layers[0]._entropy_scratch()
+        for c in layers[1:]:
+            c.entropy_scratch = shared
+    pipe = runtime.LayerPipeline(layers, s_enc, s_dec, entropy=args.entropy)
+    serial_pipe = runtime.LayerPipeline(layers, s_enc, s_enc, entropy=args.entropy)
 
     def weights_of(i):
         return wb if i % 2 == 0 else wa
@@ -455,6 +461,7 @@ def main():
     ovl_ms = [float(np.mean([t[2 * i].elapsed_time(t[2 * i + 1]) for t in timers])) for i in range(3)]
     enc_ms, tra_ms, dec_ms = [float(np.mean([t[2 * i].elapsed_time(t[2 * i + 1]) for t in serial_timers]))
                               for i in range(3)]
+    ent_ms = [float(np.mean([t[i].elapsed_time(t[i + 1]) for t in serial_timers])) for i in (6, 8)] if args.entropy else None
     n_layer = layers[0].plan.total_values
     a_enc, a_tra, a_dec = algorithmic_bytes(n_layer, q, args.dtype, args.block, args.detect)
     enc_gbs = a_enc / (enc_ms * 1e-3) / 1e9
@@ -501,6 +508,28 @@ def main():
                 verified = verified and np.array_equal(c.receiver_cache[co : co + n].cpu().numpy(), cache)
                 sampled += 1
 
+    coded = None
+    if args.entropy:
+        # one more (untimed) step, stopped after the entropy stage of every layer to read the coded sizes
+        nxt = weights_of(step_i)
+        coded_bytes = 0
+        for c, w in zip(layers, nxt):
+            c.encode(w)
+            raw_bytes_layer = c.paper_bytes()
+            c.entropy_encode()
+            coded_bytes += c.paper_bytes()
+            c.transport()
+            c.entropy_decode()
+            c.decode()
+        torch.cuda.synchronize()
+        for c in layers:
+            c.check_status()
+        step_i += 1
+        coded = {"bytes_ratio_coded": coded_bytes / weight_bytes,
+                 "entropy_encode_ms": ent_ms[0], "entropy_decode_ms": ent_ms[1],
+                 "per": "layer launch, serial re-run",
+                 "note": "rANS of the changed exponents, static 12-bit model per unit; one block per unit"}
+
     out = {
         "metric": METRIC,
         "value": whole_job_gbps(world, weight_bytes, ms_per_step),
@@ -518,6 +547,7 @@ def main():
         "gpu_launches": int(launches),
         "clocks": clocks,
         "verified_bit_exact": bool(verified),
+        "entropy_stage": coded,
         "oracle_sampled_units": sampled,
         "block_change_rate_q": q,
         "bytes_ratio": paper_bytes / weight_bytes,

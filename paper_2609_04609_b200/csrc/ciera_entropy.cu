@@ -42,6 +42,7 @@ entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long 
     __shared__ __align__(16) uint8_t s_seg[kEntWarps][kSegment];  // a warp's segment of raw payload
     __shared__ uint32_t s_hist[kEntWarps][256];
     __shared__ uint16_t s_f[256], s_c[256];
+    __shared__ unsigned long long s_rcp[256];  // ceil(2^64 / f): floor(x / f) = high half of x * rcp, exact for x < 2^32
     __shared__ uint32_t s_scan[kEntWarps];
     __shared__ unsigned long long s_total;
     const uint32_t unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
@@ -107,6 +108,11 @@ entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long 
         s_total = 0;
     }
     __syncthreads();
+    // x / f through a multiplication: rcp = ceil(2^64 / f) exceeds 2^64 / f by less than 1, so for
+    // x < 2^32 the product x * rcp / 2^64 exceeds x / f by less than 2^-32 -- too little to reach the
+    // next integer, because the fraction of x / f is at most 1 - 1/4096.  (f = 1 is handled apart.)
+    s_rcp[tid] = s_f[tid] > 1 ? (~0ull) / s_f[tid] + 1ull : 0ull;
+    __syncthreads();
 
     // 3. segments: warp w codes segments w, w + 8, ... into the unit's slots of the scratch
     const unsigned long long slot0 = seg_base[unit];
@@ -137,7 +143,10 @@ entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long 
                 x >>= 16;
             }
             nw += __popc(votes);
-            if (has) x = (x / f) * kProbScale + (x % f) + c;
+            if (has) {
+                const uint32_t q = f > 1 ? (uint32_t)__umul64hi((unsigned long long)x, s_rcp[s]) : x;
+                x = q * kProbScale + (x - q * f) + c;
+            }
         }
         reinterpret_cast<uint32_t*>(slot)[lane] = x;
         if (lane == 0) {
@@ -256,7 +265,7 @@ entropy_decode_kernel(const ciera_unit* __restrict__ units, uint32_t sm_bytes_pe
     if (tid == 0) {
         uint32_t run = 0;
         for (uint32_t s = 0; s < 256; ++s) {
-            sh.c[s] = (uint16_t)min(run, kProbScale - 1u);
+            sh.c[s] = (uint16_t)run;  // up to 4096 behind the last symbol that occurs
             run += sh.f[s];
         }
         if (run != kProbScale) sh.bad = 1;
@@ -266,7 +275,20 @@ entropy_decode_kernel(const ciera_unit* __restrict__ units, uint32_t sm_bytes_pe
         if (tid == 0 && status) atomicCAS(status, 0, (int32_t)CIERA_ERR_CORRUPT);
         return;
     }
-    for (uint32_t k = 0; k < sh.f[tid]; ++k) sh.sym[sh.c[tid] + k] = (uint8_t)tid;
+    // slot -> symbol: every thread looks up 16 consecutive slots.  The owner of a slot is the last
+    // symbol that starts at or below it (symbols that do not occur share their start with the next
+    // one, or start at 4096 behind the last occurring one): bisection over the 256 starts.
+    for (uint32_t slot = tid * 16; slot < tid * 16 + 16; ++slot) {
+        uint32_t lo = 0, hi = 255;
+        while (lo < hi) {
+            const uint32_t mid = (lo + hi + 1) >> 1;
+            if (sh.c[mid] <= slot)
+                lo = mid;
+            else
+                hi = mid - 1;
+        }
+        sh.sym[slot] = (uint8_t)lo;
+    }
     __syncthreads();
 
     const uint32_t* dir = reinterpret_cast<const uint32_t*>(pay + 512);

@@ -167,11 +167,14 @@ class LayerPipeline:
     Across iterations it keeps the dependency that the layers' buffers impose: the sender side of
     layer l in iteration i+1 (it overwrites the layer's messages, lengths and scratch) starts only
     after the decode of layer l in iteration i has finished.  ``timers``, if given, collects six CUDA
-    events per layer and step: around encode, transport (both on the sender stream) and decode."""
+    events per layer and step: around encode, transport (both on the sender stream) and decode; with
+    ``entropy`` the changed exponents are rANS-coded before the transport and restored after it, and
+    four more events are collected around those two stages."""
 
     def __init__(self, layers: List[LayerCodec], s_enc: Optional[torch.cuda.Stream] = None,
-                 s_dec: Optional[torch.cuda.Stream] = None):
+                 s_dec: Optional[torch.cuda.Stream] = None, entropy: bool = False):
         self.layers = layers
+        self.entropy = entropy
         self.s_enc = s_enc if s_enc is not None else torch.cuda.Stream()
         self.s_dec = s_dec if s_dec is not None else torch.cuda.Stream()
         self.serial = self.s_enc == self.s_dec
@@ -187,7 +190,7 @@ class LayerPipeline:
         for l, (codec, w) in enumerate(zip(self.layers, weights)):
             if not self.serial:
                 s_enc.wait_event(self.decoded[l])
-            t = [torch.cuda.Event(enable_timing=True) for _ in range(6)] if timers is not None else None
+            t = [torch.cuda.Event(enable_timing=True) for _ in range(10)] if timers is not None else None
             if t:
                 t[0].record(s_enc)
             if getattr(codec, "hash_cache", None) is not None:
@@ -196,6 +199,13 @@ class LayerPipeline:
                 codec.encode(w, s_enc)
             if t:
                 t[1].record(s_enc)
+            if self.entropy:
+                if t:
+                    t[6].record(s_enc)
+                codec.entropy_encode(s_enc)
+                if t:
+                    t[7].record(s_enc)
+            if t:
                 t[2].record(s_enc)
             codec.transport(s_enc)
             if t:
@@ -203,6 +213,12 @@ class LayerPipeline:
             if not self.serial:
                 self.sent[l].record(s_enc)
                 s_dec.wait_event(self.sent[l])
+            if self.entropy:
+                if t:
+                    t[8].record(s_dec)
+                codec.entropy_decode(s_dec)
+                if t:
+                    t[9].record(s_dec)
             if t:
                 t[4].record(s_dec)
             codec.decode(None if outs is None else outs[l], s_dec)
