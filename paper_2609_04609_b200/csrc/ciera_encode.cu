@@ -566,10 +566,17 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
                         // K = values-per-piece / B flags per piece; the warp's 32 pieces fill K whole
                         // words of the tile's block flags, 32 / K lanes to a word
                         const uint32_t k_l2 = (uint32_t)P::kLog2Values - log2b;  // log2 K, 0 .. 4
-                        uint32_t v = x.block_flags(c, log2b) << ((lane << k_l2) & 31u);
-                        for (uint32_t o = 1; o < (32u >> k_l2); o <<= 1) v |= __shfl_xor_sync(0xffffffffu, v, o);
-                        if ((lane & ((32u >> k_l2) - 1u)) == 0)
-                            ctl->bm[se][((p * kWarps + warp) << k_l2) + (lane >> (5u - k_l2))] = v;
+                        const uint32_t flags = x.block_flags(c, log2b);
+                        uint32_t* const words = &ctl->bm[se][(p * kWarps + warp) << k_l2];
+                        if (k_l2 == 3) {  // a byte of flags per piece: every lane stores its own
+                            reinterpret_cast<uint8_t*>(words)[lane] = (uint8_t)flags;
+                        } else if (k_l2 == 4) {  // two bytes per piece
+                            reinterpret_cast<uint16_t*>(words)[lane] = (uint16_t)flags;
+                        } else {
+                            uint32_t v = flags << ((lane << k_l2) & 31u);
+                            for (uint32_t o = 1; o < (32u >> k_l2); o <<= 1) v |= __shfl_xor_sync(0xffffffffu, v, o);
+                            if ((lane & ((32u >> k_l2) - 1u)) == 0) words[lane >> (5u - k_l2)] = v;
+                        }
                     }
                     // sign-plus-mantissa of every value
                     uint8_t* smdst = ti.sm_dst + (size_t)t0 * SMB;
