@@ -97,6 +97,7 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
         const ciera_unit& un = units_host[u];
         if ((un.weights_off | un.cache_off | un.msg_off) & 15ull) return CIERA_ERR_MISALIGNED;
         if (un.n_values >= (1ull << 48)) return CIERA_ERR_UNSUPPORTED;
+        if ((un.n_values + block - 1) / block > 0xffffffffull) return CIERA_ERR_UNSUPPORTED;  // block counts are 32-bit
         if (un.msg_capacity < ciera_message_capacity(un.n_values, dtype, block)) return CIERA_ERR_CAPACITY;
         n_tiles += (un.n_values + kTileValues - 1) / kTileValues;
         total += un.n_values;

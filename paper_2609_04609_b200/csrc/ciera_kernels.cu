@@ -47,14 +47,8 @@ cache_fill_kernel(const TileDesc* __restrict__ tiles, const uint8_t* __restrict_
 // stores); tile numbers, descriptors and reported lengths are fetched three, two and one tile
 // ahead, so that no step waits for them.
 
-#ifndef CIERA_COPY_THREADS
-#define CIERA_COPY_THREADS 256
-#endif
-#ifndef CIERA_COPY_UNROLL
-#define CIERA_COPY_UNROLL 8
-#endif
-constexpr int kCopyThreads = CIERA_COPY_THREADS;
-constexpr int kCopyUnroll = CIERA_COPY_UNROLL;
+constexpr int kCopyThreads = 256;
+constexpr int kCopyUnroll = 8;  // 128-bit loads in flight per lane
 
 // the part of a tile descriptor the copy needs (keeps the prefetched copies small in registers)
 struct CopyDesc {

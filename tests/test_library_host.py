@@ -70,6 +70,9 @@ def test_plan_validation(ciera):
     with pytest.raises(ciera.CieraError) as e:
         ciera.Plan(_units([(1000, 0, 0, 0, cap - 1)]), 0, 512)
     assert e.value.status == ciera.ERR_CAPACITY
+    with pytest.raises(ciera.CieraError) as e:  # more blocks than a 32-bit count holds
+        ciera.Plan(_units([(1 << 33, 0, 0, 0, ciera.message_capacity(1 << 33, 0, 1))]), 0, 1)
+    assert e.value.status == ciera.ERR_UNSUPPORTED
     with pytest.raises(ciera.CieraError) as e:
         ciera.Plan(good, 7, 512)
     assert e.value.status == ciera.ERR_INVALID_ARG
