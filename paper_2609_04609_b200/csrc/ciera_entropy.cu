@@ -18,7 +18,11 @@
 // 2 zero bytes if the count is odd].  It replaces the raw payload only if strictly shorter; the
 // receiver knows the raw length from the bitmap and so tells the two forms apart by the length.
 //
-// One thread block works on one unit: nothing waits for another block anywhere.
+// Work split: a unit of up to 64 segments' worth of values (262 144) is done by one thread block from
+// start to end (histogram, model, segments into a scratch, coded form into the message).  Longer
+// units go through a chain of launches whose grids run over chunks of 64 segments, so that their
+// work spreads over the GPU: sender = histogram, model, segments, layout, copy; receiver = layout,
+// segments, restore.  Nothing waits for another thread block anywhere.
 #include "ciera_bits.cuh"
 
 namespace ciera {
@@ -29,11 +33,232 @@ constexpr uint32_t kSegment = 4096;                              // bytes of raw
 constexpr uint32_t kSegWordsMax = kSegment * kProbBits / 16;     // 3072: a symbol adds at most 12 bits
 constexpr uint32_t kSegSlot = 4 * 32 + 2 * kSegWordsMax;         // 6272 bytes: states + words
 constexpr int kEntThreads = 256, kEntWarps = kEntThreads / 32;
+constexpr uint32_t kLongSegs = 64;  // units with more segment slots than this take the chunked path
 
 __host__ __device__ inline uint64_t segments_of(uint64_t bytes) { return (bytes + kSegment - 1) / kSegment; }
 __host__ __device__ inline uint32_t segment_bytes(uint32_t nw) { return 4u * 32u + 2u * nw + ((nw & 1u) ? 2u : 0u); }
 
+// ---------------------------------------------------------------------------------- shared pieces
+
+// Adds the bytes pay[lo, hi) to the warp-private histograms (lo a multiple of 16, pay 16-byte aligned).
+__device__ __forceinline__ void histogram_add(uint32_t (*hist)[256], const uint8_t* pay, uint64_t lo, uint64_t hi,
+                                              uint32_t tid) {
+    const uint32_t warp = tid >> 5;
+    for (uint64_t i = lo + (uint64_t)tid * 16; i < hi; i += (uint64_t)kEntThreads * 16) {
+        if (i + 16 <= hi) {
+            const uint4 v = *reinterpret_cast<const uint4*>(pay + i);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int k = 0; k < 16; ++k) atomicAdd(&hist[warp][(w[k >> 2] >> (8 * (k & 3))) & 0xFFu], 1u);
+        } else {
+            for (uint64_t k = i; k < hi; ++k) atomicAdd(&hist[warp][pay[k]], 1u);
+        }
+    }
+}
+
+// Frequencies from counts (h[256] in shared memory, P = their sum): thread s owns symbol s.  Ends
+// with a barrier; f is then final.
+__device__ __forceinline__ void normalise_model(const uint32_t* h, uint64_t P, uint16_t* f, uint32_t tid) {
+    {
+        uint32_t v = 0;
+        if (h[tid]) {
+            v = (uint32_t)((uint64_t)h[tid] * kProbScale / P);
+            if (v == 0) v = 1;
+        }
+        f[tid] = (uint16_t)v;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        uint32_t sum = 0, best = 0;
+        for (uint32_t s = 0; s < 256; ++s) {
+            sum += f[s];
+            if (h[s] > h[best]) best = s;
+        }
+        if (sum < kProbScale) {
+            f[best] = (uint16_t)(f[best] + (kProbScale - sum));
+        } else {
+            uint32_t excess = sum - kProbScale;
+            while (excess) {
+                uint32_t big = 0;
+                for (uint32_t s = 1; s < 256; ++s)
+                    if (f[s] > f[big]) big = s;
+                const uint32_t take = min((uint32_t)f[big] - 1u, excess);
+                f[big] = (uint16_t)(f[big] - take);
+                excess -= take;
+            }
+        }
+    }
+    __syncthreads();
+}
+
+// Starts c[] and reciprocals from final frequencies.  Ends with a barrier.
+// x / f through a multiplication: rcp = ceil(2^64 / f) exceeds 2^64 / f by less than 1, so for
+// x < 2^32 the product x * rcp / 2^64 exceeds x / f by less than 2^-32 -- too little to reach the next
+// integer, because the fraction of x / f is at most 1 - 1/4096.  (f = 1 is handled apart.)
+__device__ __forceinline__ void encoder_tables(const uint16_t* f, uint16_t* c, unsigned long long* rcp, uint32_t tid) {
+    if (tid == 0) {
+        uint32_t run = 0;
+        for (uint32_t s = 0; s < 256; ++s) {
+            c[s] = (uint16_t)run;
+            run += f[s];
+        }
+    }
+    rcp[tid] = f[tid] > 1 ? (~0ull) / f[tid] + 1ull : 0ull;
+    __syncthreads();
+}
+
+// One warp codes one segment: src[0, n) -> slot (32 states, then the words).  Returns the word count.
+__device__ __forceinline__ uint32_t encode_segment(const uint8_t* src, uint32_t n, uint8_t* stage, const uint16_t* f,
+                                                   const uint16_t* c, const unsigned long long* rcp, uint8_t* slot,
+                                                   uint32_t lane) {
+    for (uint32_t i = lane * 16; i < n; i += 32 * 16) {
+        if (i + 16 <= n) {
+            *reinterpret_cast<uint4*>(stage + i) = *reinterpret_cast<const uint4*>(src + i);
+        } else {
+            for (uint32_t k = i; k < n; ++k) stage[k] = src[k];
+        }
+    }
+    __syncwarp();
+    uint16_t* words = reinterpret_cast<uint16_t*>(slot + 4 * 32);
+    uint32_t x = kRansL, nw = 0;
+    const uint32_t steps = (n + 31u) >> 5;
+    for (uint32_t t = steps; t-- > 0;) {
+        const uint32_t i = 32u * t + lane;
+        const bool has = i < n;
+        const uint32_t s = has ? stage[i] : 0u;
+        const uint32_t fs = has ? f[s] : 1u, cs = c[s];
+        const bool emit = has && (x >> 20) >= fs;  // x >= f * 2^20
+        const uint32_t votes = __ballot_sync(0xffffffffu, emit);
+        if (emit) {
+            words[nw + __popc(votes & ((1u << lane) - 1u))] = (uint16_t)x;
+            x >>= 16;
+        }
+        nw += __popc(votes);
+        if (has) {
+            const uint32_t q = fs > 1 ? (uint32_t)__umul64hi((unsigned long long)x, rcp[s]) : x;
+            x = q * kProbScale + (x - q * fs) + cs;
+        }
+    }
+    reinterpret_cast<uint32_t*>(slot)[lane] = x;
+    if (lane == 0 && (nw & 1u)) words[nw] = 0;
+    __syncwarp();
+    return nw;
+}
+
+// Receiver tables from the transmitted frequencies (f[] already in shared memory and synced):
+// starts c[], slot -> symbol.  Returns false (in every thread) if the table does not sum to 4096.
+// The owner of a slot is the last symbol that starts at or below it (symbols that do not occur share
+// their start with the next one, or start at 4096 behind the last occurring one).
+__device__ __forceinline__ bool decoder_tables(const uint16_t* f, uint16_t* c, uint8_t* sym, uint32_t* flag, uint32_t tid) {
+    if (tid == 0) {
+        uint32_t run = 0;
+        for (uint32_t s = 0; s < 256; ++s) {
+            c[s] = (uint16_t)min(run, kProbScale);
+            run += f[s];
+        }
+        *flag = run == kProbScale ? 1u : 0u;
+    }
+    __syncthreads();
+    if (*flag == 0) return false;
+    for (uint32_t slot = tid * 16; slot < tid * 16 + 16; ++slot) {
+        uint32_t lo = 0, hi = 255;
+        while (lo < hi) {
+            const uint32_t mid = (lo + hi + 1) >> 1;
+            if (c[mid] <= slot)
+                lo = mid;
+            else
+                hi = mid - 1;
+        }
+        sym[slot] = (uint8_t)lo;
+    }
+    __syncthreads();
+    return true;
+}
+
+// One warp decodes one segment: coded (32 states + snw words, 4-byte aligned) -> out[0, n).
+// Returns false (in every lane) if the words run out, are left over, or a lane does not end in the
+// start state.
+__device__ __forceinline__ bool decode_segment(const uint8_t* coded, uint32_t snw, uint32_t n, uint8_t* stage,
+                                               const uint8_t* sym, const uint16_t* f, const uint16_t* c, uint8_t* out,
+                                               uint32_t lane) {
+    const uint32_t* from = reinterpret_cast<const uint32_t*>(coded);
+    uint32_t* st = reinterpret_cast<uint32_t*>(stage);
+    for (uint32_t i = lane; i < (segment_bytes(snw) >> 2); i += 32) st[i] = from[i];
+    __syncwarp();
+    const uint16_t* words = reinterpret_cast<const uint16_t*>(stage + 4 * 32);
+    uint32_t x = st[lane], ptr = snw;
+    const uint32_t steps = (n + 31u) >> 5;
+    bool ok = true;
+    for (uint32_t t = 0; t < steps; ++t) {
+        const uint32_t i = 32u * t + lane;
+        const bool has = i < n;
+        bool need = false;
+        if (has) {
+            const uint32_t slot = x & (kProbScale - 1u);
+            const uint32_t s = sym[slot];
+            out[i] = (uint8_t)s;
+            x = (uint32_t)f[s] * (x >> kProbBits) + slot - c[s];
+            need = x < kRansL;
+        }
+        const uint32_t votes = __ballot_sync(0xffffffffu, need);
+        const uint32_t k_need = __popc(votes);
+        if (k_need > ptr) {
+            ok = false;
+            break;
+        }
+        if (need) x = (x << 16) | words[ptr - k_need + __popc(votes & ((1u << lane) - 1u))];
+        ptr -= k_need;
+    }
+    ok = ok && ptr == 0 && !__any_sync(0xffffffffu, x != kRansL);
+    __syncwarp();
+    return ok;
+}
+
+// Raw payload length of a unit from its bitmap (block-wide; `acc` in shared memory, zeroed and
+// synced by the caller).  The bitmap's bits past the last block and the pad behind it are zero.
+__device__ __forceinline__ uint64_t raw_payload_bytes(const uint8_t* msg, uint64_t N, uint32_t log2b,
+                                                      unsigned long long* acc, uint32_t tid) {
+    const uint64_t words = (bitmap_bytes(N, log2b) + 3) >> 2;  // inside the 16-byte padded bitmap
+    const uint32_t* bm32 = reinterpret_cast<const uint32_t*>(msg);
+    uint32_t cnt = 0;
+    for (uint64_t i = tid; i < words; i += kEntThreads) cnt += __popc(bm32[i]);
+    cnt = __reduce_add_sync(0xffffffffu, cnt);
+    if ((tid & 31u) == 0 && cnt) atomicAdd(acc, (unsigned long long)cnt);
+    __syncthreads();
+    const uint32_t B = 1u << log2b;
+    uint64_t P = *acc << log2b;
+    const uint32_t rem = (uint32_t)(N & (B - 1u));
+    if (rem) {
+        const uint64_t kb = num_blocks(N, log2b) - 1;
+        if ((msg[kb >> 3] >> (kb & 7u)) & 1u) P -= (B - rem);
+    }
+    return P;
+}
+
+// Exclusive scan of one value per thread over the block; `scan` holds kEntWarps words.  Returns
+// the thread's offset; `total` gets the block's sum.  Contains barriers.
+__device__ __forceinline__ uint32_t block_scan(uint32_t v, uint32_t* scan, uint32_t tid, uint32_t& total) {
+    const uint32_t lane = tid & 31u, warp = tid >> 5;
+    uint32_t incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+        if ((int)lane >= o) incl += t;
+    }
+    __syncthreads();  // the previous use of scan[] is over
+    if (lane == 31) scan[warp] = incl;
+    __syncthreads();
+    uint32_t wbase = 0;
+    total = 0;
+    for (int w = 0; w < kEntWarps; ++w) {
+        if (w < (int)warp) wbase += scan[w];
+        total += scan[w];
+    }
+    return wbase + incl - v;
+}
+
 // ------------------------------------------------------------------------------------------ sender
+// units of up to kLongSegs segment slots: one thread block per unit, start to end
 
 __global__ void __launch_bounds__(kEntThreads)
 entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
@@ -42,342 +267,445 @@ entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long 
     __shared__ __align__(16) uint8_t s_seg[kEntWarps][kSegment];  // a warp's segment of raw payload
     __shared__ uint32_t s_hist[kEntWarps][256];
     __shared__ uint16_t s_f[256], s_c[256];
-    __shared__ unsigned long long s_rcp[256];  // ceil(2^64 / f): floor(x / f) = high half of x * rcp, exact for x < 2^32
+    __shared__ unsigned long long s_rcp[256];
     __shared__ uint32_t s_scan[kEntWarps];
     __shared__ unsigned long long s_total;
     const uint32_t unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     const ciera_unit un = units[unit];
-    if (un.n_values == 0) return;
+    if (un.n_values == 0 || segments_of(un.n_values) > kLongSegs) return;
     const uint64_t payoff = payload_offset(un.n_values, sm_bytes_per_value, log2b);
     const uint64_t P = wire_bytes[unit] - payoff;
-    if (P == 0 || P >= (1ull << 32)) return;  // nothing to code (or too much for 32-bit counts: stays raw)
+    if (P == 0) return;  // nothing to code
     uint8_t* const pay = msgs + un.msg_off + payoff;  // 16-byte aligned
     const uint32_t nseg = (uint32_t)segments_of(P);
 
-    // 1. histogram of the raw payload (one private copy per warp)
+    // 1. histogram of the raw payload (one private copy per warp), 2. the model
     for (uint32_t i = lane; i < 256; i += 32) s_hist[warp][i] = 0;
+    if (tid == 0) s_total = 0;
     __syncwarp();
-    for (uint64_t i = (uint64_t)tid * 16; i < P; i += (uint64_t)kEntThreads * 16) {
-        if (i + 16 <= P) {
-            const uint4 v = *reinterpret_cast<const uint4*>(pay + i);
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-            for (int k = 0; k < 16; ++k) atomicAdd(&s_hist[warp][(w[k >> 2] >> (8 * (k & 3))) & 0xFFu], 1u);
-        } else {
-            for (uint64_t k = i; k < P; ++k) atomicAdd(&s_hist[warp][pay[k]], 1u);
-        }
-    }
+    histogram_add(s_hist, pay, 0, P, tid);
     __syncthreads();
-    // 2. the model: thread s owns symbol s
     {
         uint32_t h = 0;
         for (int w = 0; w < kEntWarps; ++w) h += s_hist[w][tid];
-        uint32_t f = 0;
-        if (h) {
-            f = (uint32_t)((uint64_t)h * kProbScale / P);
-            if (f == 0) f = 1;
-        }
-        s_hist[0][tid] = h;  // every thread has read all copies of its own symbol only
-        s_f[tid] = (uint16_t)f;
+        __syncthreads();
+        s_hist[0][tid] = h;
     }
     __syncthreads();
-    if (tid == 0) {
-        uint32_t sum = 0, best = 0;
-        for (uint32_t s = 0; s < 256; ++s) {
-            sum += s_f[s];
-            if (s_hist[0][s] > s_hist[0][best]) best = s;
-        }
-        if (sum < kProbScale) {
-            s_f[best] = (uint16_t)(s_f[best] + (kProbScale - sum));
-        } else {
-            uint32_t excess = sum - kProbScale;
-            while (excess) {
-                uint32_t big = 0;
-                for (uint32_t s = 1; s < 256; ++s)
-                    if (s_f[s] > s_f[big]) big = s;
-                const uint32_t take = min((uint32_t)s_f[big] - 1u, excess);
-                s_f[big] = (uint16_t)(s_f[big] - take);
-                excess -= take;
-            }
-        }
-        uint32_t run = 0;
-        for (uint32_t s = 0; s < 256; ++s) {
-            s_c[s] = (uint16_t)run;
-            run += s_f[s];
-        }
-        s_total = 0;
-    }
-    __syncthreads();
-    // x / f through a multiplication: rcp = ceil(2^64 / f) exceeds 2^64 / f by less than 1, so for
-    // x < 2^32 the product x * rcp / 2^64 exceeds x / f by less than 2^-32 -- too little to reach the
-    // next integer, because the fraction of x / f is at most 1 - 1/4096.  (f = 1 is handled apart.)
-    s_rcp[tid] = s_f[tid] > 1 ? (~0ull) / s_f[tid] + 1ull : 0ull;
-    __syncthreads();
+    normalise_model(s_hist[0], P, s_f, tid);
+    encoder_tables(s_f, s_c, s_rcp, tid);
 
     // 3. segments: warp w codes segments w, w + 8, ... into the unit's slots of the scratch
     const unsigned long long slot0 = seg_base[unit];
     for (uint32_t g = warp; g < nseg; g += kEntWarps) {
         const uint32_t n = (uint32_t)min((uint64_t)kSegment, P - (uint64_t)g * kSegment);
-        const uint8_t* src = pay + (uint64_t)g * kSegment;
-        for (uint32_t i = lane * 16; i < n; i += 32 * 16) {
-            if (i + 16 <= n) {
-                *reinterpret_cast<uint4*>(&s_seg[warp][i]) = *reinterpret_cast<const uint4*>(src + i);
-            } else {
-                for (uint32_t k = i; k < n; ++k) s_seg[warp][k] = src[k];
-            }
-        }
-        __syncwarp();
-        uint8_t* slot = scratch_slots + (slot0 + g) * kSegSlot;
-        uint16_t* words = reinterpret_cast<uint16_t*>(slot + 4 * 32);
-        uint32_t x = kRansL, nw = 0;
-        const uint32_t steps = (n + 31u) >> 5;
-        for (uint32_t t = steps; t-- > 0;) {
-            const uint32_t i = 32u * t + lane;
-            const bool has = i < n;
-            const uint32_t s = has ? s_seg[warp][i] : 0u;
-            const uint32_t f = has ? s_f[s] : 1u, c = s_c[s];
-            const bool emit = has && (x >> 20) >= f;  // x >= f * 2^20
-            const uint32_t votes = __ballot_sync(0xffffffffu, emit);
-            if (emit) {
-                words[nw + __popc(votes & ((1u << lane) - 1u))] = (uint16_t)x;
-                x >>= 16;
-            }
-            nw += __popc(votes);
-            if (has) {
-                const uint32_t q = f > 1 ? (uint32_t)__umul64hi((unsigned long long)x, s_rcp[s]) : x;
-                x = q * kProbScale + (x - q * f) + c;
-            }
-        }
-        reinterpret_cast<uint32_t*>(slot)[lane] = x;
+        const uint32_t nw = encode_segment(pay + (uint64_t)g * kSegment, n, s_seg[warp], s_f, s_c, s_rcp,
+                                           scratch_slots + (slot0 + g) * kSegSlot, lane);
         if (lane == 0) {
-            if (nw & 1u) words[nw] = 0;
             scratch_nw[slot0 + g] = nw;
             atomicAdd(&s_total, (unsigned long long)segment_bytes(nw));
         }
-        __syncwarp();
     }
-    __threadfence_block();
     __syncthreads();  // every warp is done reading the raw payload and writing its slots
 
     // 4. keep the raw form unless the coded one is strictly shorter; else move it into the message
     const uint64_t C = 512ull + 4ull * nseg + s_total;
     if (C >= P) return;
-    uint16_t* table = reinterpret_cast<uint16_t*>(pay);
-    table[tid] = s_f[tid];
+    reinterpret_cast<uint16_t*>(pay)[tid] = s_f[tid];
     uint32_t* dir = reinterpret_cast<uint32_t*>(pay + 512);
     uint8_t* data = pay + 512 + 4ull * nseg;
-    uint64_t carry = 0;  // bytes of the segments before this chunk (same in every thread)
-    for (uint32_t g0 = 0; g0 < nseg; g0 += kEntThreads) {
-        const uint32_t g = g0 + tid;
-        const uint32_t nw = g < nseg ? scratch_nw[slot0 + g] : 0u;
-        const uint32_t size = g < nseg ? segment_bytes(nw) : 0u;
-        if (g < nseg) dir[g] = nw;
-        // exclusive scan of the sizes over the chunk
-        uint32_t incl = size;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
-            if ((int)lane >= o) incl += v;
-        }
-        if (lane == 31) s_scan[warp] = incl;
-        __syncthreads();
-        uint32_t wbase = 0, chunk_total = 0;
-        for (int w = 0; w < kEntWarps; ++w) {
-            if (w < (int)warp) wbase += s_scan[w];
-            chunk_total += s_scan[w];
-        }
-        // park (offset, size) of the chunk's segments where the warps can read them
-        uint32_t* s_off = &s_hist[1][0];
-        uint32_t* s_size = &s_hist[2][0];
-        s_off[tid] = wbase + incl - size;
-        s_size[tid] = size;
-        __syncthreads();
-        const uint32_t in_chunk = min((uint32_t)kEntThreads, nseg - g0);
-        for (uint32_t k = warp; k < in_chunk; k += kEntWarps) {
-            const uint32_t* from = reinterpret_cast<const uint32_t*>(scratch_slots + (slot0 + g0 + k) * kSegSlot);
-            uint32_t* to = reinterpret_cast<uint32_t*>(data + carry + s_off[k]);
-            for (uint32_t i = lane; i < (s_size[k] >> 2); i += 32) to[i] = from[i];
-        }
-        carry += chunk_total;
-        __syncthreads();
+    // nseg <= kLongSegs <= kEntThreads: one round
+    const uint32_t nw = tid < nseg ? scratch_nw[slot0 + tid] : 0u;
+    const uint32_t size = tid < nseg ? segment_bytes(nw) : 0u;
+    if (tid < nseg) dir[tid] = nw;
+    uint32_t total;
+    uint32_t* s_off = &s_hist[1][0];
+    uint32_t* s_size = &s_hist[2][0];
+    s_off[tid] = block_scan(size, s_scan, tid, total);
+    s_size[tid] = size;
+    __syncthreads();
+    for (uint32_t k = warp; k < nseg; k += kEntWarps) {
+        const uint32_t* from = reinterpret_cast<const uint32_t*>(scratch_slots + (slot0 + k) * kSegSlot);
+        uint32_t* to = reinterpret_cast<uint32_t*>(data + s_off[k]);
+        for (uint32_t i = lane; i < (s_size[k] >> 2); i += 32) to[i] = from[i];
     }
     if (tid == 0) wire_bytes[unit] = payoff + C;
 }
 
+// longer units: grids over chunks of kLongSegs segments.  A chunk record = {unit, first segment of
+// the chunk inside the unit, index of the unit among the long ones, 0}.  Per long unit the scratch
+// holds a record of 2048 bytes: 256 x u32 counts, 256 x u16 frequencies, then the words below.
+constexpr uint32_t kLongRec = 2048;
+struct LongState {            // at byte 1536 of a long unit's record
+    unsigned long long total;   // sender: bytes of all coded segments
+    unsigned long long P;       // raw payload length
+    uint32_t coded;             // 1: the coded form is (sender) / was (receiver) chosen
+    uint32_t bad;               // receiver: a segment did not decode
+    uint32_t nseg;              // segments of the raw payload
+    uint32_t pad;
+};
+__device__ __forceinline__ uint32_t* long_hist(uint8_t* recs, uint32_t li) { return reinterpret_cast<uint32_t*>(recs + (size_t)li * kLongRec); }
+__device__ __forceinline__ uint16_t* long_model(uint8_t* recs, uint32_t li) { return reinterpret_cast<uint16_t*>(recs + (size_t)li * kLongRec + 1024); }
+__device__ __forceinline__ LongState* long_state(uint8_t* recs, uint32_t li) { return reinterpret_cast<LongState*>(recs + (size_t)li * kLongRec + 1536); }
+
+// raw payload length of a unit on the sender (0: nothing to code or too much for 32-bit counts)
+__device__ __forceinline__ uint64_t sender_payload(const ciera_unit& un, uint32_t smb, uint32_t log2b,
+                                                   const unsigned long long* wire_bytes, uint32_t unit, uint64_t& payoff) {
+    payoff = payload_offset(un.n_values, smb, log2b);
+    const uint64_t P = wire_bytes[unit] - payoff;
+    return P < (1ull << 32) ? P : 0;
+}
+
+__global__ void __launch_bounds__(kEntThreads)
+entropy_long_hist_kernel(const ciera_unit* __restrict__ units, const uint4* __restrict__ chunks, uint32_t smb, uint32_t log2b,
+                         const uint8_t* msgs, const unsigned long long* wire_bytes, uint8_t* recs) {
+    __shared__ uint32_t s_hist[kEntWarps][256];
+    const uint4 ch = chunks[blockIdx.x];
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const ciera_unit un = units[ch.x];
+    uint64_t payoff;
+    const uint64_t P = sender_payload(un, smb, log2b, wire_bytes, ch.x, payoff);
+    const uint64_t lo = (uint64_t)ch.y * kSegment;
+    if (lo >= P) return;
+    const uint64_t hi = min(P, lo + (uint64_t)kLongSegs * kSegment);
+    for (uint32_t i = lane; i < 256; i += 32) s_hist[warp][i] = 0;
+    __syncwarp();
+    histogram_add(s_hist, msgs + un.msg_off + payoff, lo, hi, tid);
+    __syncthreads();
+    uint32_t h = 0;
+    for (int w = 0; w < kEntWarps; ++w) h += s_hist[w][tid];
+    if (h) atomicAdd(long_hist(recs, ch.z) + tid, h);
+}
+
+__global__ void __launch_bounds__(kEntThreads)
+entropy_long_model_kernel(const ciera_unit* __restrict__ units, const uint32_t* __restrict__ long_units, uint32_t smb,
+                          uint32_t log2b, const unsigned long long* wire_bytes, uint8_t* recs) {
+    __shared__ uint32_t s_h[256];
+    __shared__ uint16_t s_f[256];
+    const uint32_t li = blockIdx.x, tid = threadIdx.x, unit = long_units[li];
+    uint64_t payoff;
+    const uint64_t P = sender_payload(units[unit], smb, log2b, wire_bytes, unit, payoff);
+    if (tid == 0) {
+        LongState* st = long_state(recs, li);
+        st->total = 0;
+        st->coded = 0;
+        st->bad = 0;
+    }
+    if (P == 0) return;
+    s_h[tid] = long_hist(recs, li)[tid];
+    __syncthreads();
+    normalise_model(s_h, P, s_f, tid);
+    long_model(recs, li)[tid] = s_f[tid];
+}
+
+__global__ void __launch_bounds__(kEntThreads)
+entropy_long_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
+                           const uint4* __restrict__ chunks, uint32_t smb, uint32_t log2b, const uint8_t* msgs,
+                           const unsigned long long* wire_bytes, uint8_t* recs, uint8_t* scratch_slots,
+                           uint32_t* scratch_nw) {
+    __shared__ __align__(16) uint8_t s_seg[kEntWarps][kSegment];
+    __shared__ uint16_t s_f[256], s_c[256];
+    __shared__ unsigned long long s_rcp[256];
+    __shared__ unsigned long long s_total;
+    const uint4 ch = chunks[blockIdx.x];
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const ciera_unit un = units[ch.x];
+    uint64_t payoff;
+    const uint64_t P = sender_payload(un, smb, log2b, wire_bytes, ch.x, payoff);
+    if ((uint64_t)ch.y * kSegment >= P) return;
+    const uint32_t nseg = (uint32_t)segments_of(P);
+    const uint32_t g_end = min(nseg, ch.y + kLongSegs);
+    s_f[tid] = long_model(recs, ch.z)[tid];
+    if (tid == 0) s_total = 0;
+    __syncthreads();
+    encoder_tables(s_f, s_c, s_rcp, tid);
+    const uint8_t* pay = msgs + un.msg_off + payoff;
+    const unsigned long long slot0 = seg_base[ch.x];
+    for (uint32_t g = ch.y + warp; g < g_end; g += kEntWarps) {
+        const uint32_t n = (uint32_t)min((uint64_t)kSegment, P - (uint64_t)g * kSegment);
+        const uint32_t nw = encode_segment(pay + (uint64_t)g * kSegment, n, s_seg[warp], s_f, s_c, s_rcp,
+                                           scratch_slots + (slot0 + g) * kSegSlot, lane);
+        if (lane == 0) {
+            scratch_nw[slot0 + g] = nw;
+            atomicAdd(&s_total, (unsigned long long)segment_bytes(nw));
+        }
+    }
+    __syncthreads();
+    if (tid == 0) atomicAdd(&long_state(recs, ch.z)->total, s_total);
+}
+
+// decides raw or coded for a long unit; coded: table and word counts into the message, the byte
+// offset of every segment into the scratch
+__global__ void __launch_bounds__(kEntThreads)
+entropy_long_layout_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
+                           const uint32_t* __restrict__ long_units, uint32_t smb, uint32_t log2b, uint8_t* msgs,
+                           unsigned long long* wire_bytes, uint8_t* recs, const uint32_t* scratch_nw,
+                           uint32_t* scratch_off) {
+    __shared__ uint32_t s_scan[kEntWarps];
+    const uint32_t li = blockIdx.x, tid = threadIdx.x, unit = long_units[li];
+    const ciera_unit un = units[unit];
+    uint64_t payoff;
+    const uint64_t P = sender_payload(un, smb, log2b, wire_bytes, unit, payoff);
+    if (P == 0) return;
+    const uint32_t nseg = (uint32_t)segments_of(P);
+    LongState* st = long_state(recs, li);
+    const uint64_t C = 512ull + 4ull * nseg + st->total;
+    if (C >= P) return;
+    uint8_t* pay = msgs + un.msg_off + payoff;
+    reinterpret_cast<uint16_t*>(pay)[tid] = long_model(recs, li)[tid];
+    uint32_t* dir = reinterpret_cast<uint32_t*>(pay + 512);
+    const unsigned long long slot0 = seg_base[unit];
+    uint32_t carry = 0;  // C < P < 2^32: offsets fit
+    for (uint32_t g0 = 0; g0 < nseg; g0 += kEntThreads) {
+        const uint32_t g = g0 + tid;
+        const uint32_t nw = g < nseg ? scratch_nw[slot0 + g] : 0u;
+        if (g < nseg) dir[g] = nw;
+        uint32_t total;
+        const uint32_t off = block_scan(g < nseg ? segment_bytes(nw) : 0u, s_scan, tid, total);
+        if (g < nseg) scratch_off[slot0 + g] = carry + off;
+        carry += total;
+    }
+    if (tid == 0) {
+        st->coded = 1;
+        st->nseg = nseg;
+        wire_bytes[unit] = payoff + C;
+    }
+}
+
+__global__ void __launch_bounds__(kEntThreads)
+entropy_long_copy_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
+                         const uint4* __restrict__ chunks, uint32_t smb, uint32_t log2b, uint8_t* msgs, uint8_t* recs,
+                         const uint8_t* scratch_slots, const uint32_t* scratch_nw, const uint32_t* scratch_off) {
+    const uint4 ch = chunks[blockIdx.x];
+    const LongState* st = long_state(recs, ch.z);
+    if (st->coded == 0) return;
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const ciera_unit un = units[ch.x];
+    const uint32_t nseg = st->nseg;
+    uint8_t* data = msgs + un.msg_off + payload_offset(un.n_values, smb, log2b) + 512 + 4ull * nseg;
+    const unsigned long long slot0 = seg_base[ch.x];
+    const uint32_t g_end = min(nseg, ch.y + kLongSegs);
+    for (uint32_t g = ch.y + warp; g < g_end; g += kEntWarps) {
+        const uint32_t* from = reinterpret_cast<const uint32_t*>(scratch_slots + (slot0 + g) * kSegSlot);
+        uint32_t* to = reinterpret_cast<uint32_t*>(data + scratch_off[slot0 + g]);
+        const uint32_t words4 = segment_bytes(scratch_nw[slot0 + g]) >> 2;
+        for (uint32_t i = lane; i < words4; i += 32) to[i] = from[i];
+    }
+}
+
 // ---------------------------------------------------------------------------------------- receiver
+// units of up to kLongSegs segment slots: one thread block per unit, start to end
 
 struct DecodeShared {
     uint8_t sym[kProbScale];       // slot -> symbol
     uint16_t f[256], c[256];
-    uint32_t off[kEntThreads];     // per segment of a chunk: byte offset in the data part
-    uint32_t nw[kEntThreads];      //                         word count
+    uint32_t off[kEntThreads];     // per segment: byte offset in the data part
+    uint32_t nw[kEntThreads];      //              word count
     uint32_t scan[kEntWarps];
     unsigned long long changed;    // set bits of the unit's bitmap
-    uint32_t bad;
+    uint32_t flag, bad;
     __align__(16) uint8_t seg[kEntWarps][kSegSlot];  // a warp's coded segment
 };
 
+__device__ __forceinline__ void raise_corrupt(int32_t* status) {
+    if (status) atomicCAS(status, 0, (int32_t)CIERA_ERR_CORRUPT);
+}
+
 __global__ void __launch_bounds__(kEntThreads)
-entropy_decode_kernel(const ciera_unit* __restrict__ units, uint32_t sm_bytes_per_value, uint32_t log2b, uint8_t* msgs,
+entropy_decode_kernel(const ciera_unit* __restrict__ units, uint32_t smb, uint32_t log2b, uint8_t* msgs,
                       unsigned long long* wire_bytes, uint8_t* scratch_raw, int32_t* status) {
     extern __shared__ __align__(16) uint8_t smem_raw[];
     DecodeShared& sh = *reinterpret_cast<DecodeShared*>(smem_raw);
     const uint32_t unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     const ciera_unit un = units[unit];
     const uint64_t N = un.n_values;
-    if (N == 0) return;
+    if (N == 0 || segments_of(N) > kLongSegs) return;
     uint8_t* const msg = msgs + un.msg_off;
-    const uint64_t payoff = payload_offset(N, sm_bytes_per_value, log2b);
-    const uint32_t B = 1u << log2b;
+    const uint64_t payoff = payload_offset(N, smb, log2b);
     if (tid == 0) {
         sh.changed = 0;
         sh.bad = 0;
     }
     __syncthreads();
-    // raw payload length from the bitmap (its bits past the last block and the pad behind it are zero)
-    {
-        const uint64_t words = (bitmap_bytes(N, log2b) + 3) >> 2;  // inside the 16-byte padded bitmap
-        const uint32_t* bm32 = reinterpret_cast<const uint32_t*>(msg);
-        uint32_t cnt = 0;
-        for (uint64_t i = tid; i < words; i += kEntThreads) cnt += __popc(bm32[i]);
-        cnt = __reduce_add_sync(0xffffffffu, cnt);
-        if (lane == 0 && cnt) atomicAdd(&sh.changed, (unsigned long long)cnt);
-    }
-    __syncthreads();
-    uint64_t P = sh.changed << log2b;
-    const uint32_t rem = (uint32_t)(N & (B - 1u));
-    if (rem) {
-        const uint64_t kb = num_blocks(N, log2b) - 1;
-        if ((msg[kb >> 3] >> (kb & 7u)) & 1u) P -= (B - rem);
-    }
+    const uint64_t P = raw_payload_bytes(msg, N, log2b, &sh.changed, tid);
     const uint64_t wire = wire_bytes[unit];
     if (P == 0 || wire == payoff + P) return;  // nothing travelled, or the raw form did
     const uint64_t C = wire - payoff;
     const uint32_t nseg = (uint32_t)segments_of(P);
-    const uint8_t* const pay = msg + payoff;
+    uint8_t* const pay = msg + payoff;
     if (wire < payoff || C >= P || C < 512ull + 4ull * nseg) {
-        if (tid == 0 && status) atomicCAS(status, 0, (int32_t)CIERA_ERR_CORRUPT);
+        if (tid == 0) raise_corrupt(status);
         return;
     }
-    // the model
     sh.f[tid] = reinterpret_cast<const uint16_t*>(pay)[tid];
     __syncthreads();
-    if (tid == 0) {
-        uint32_t run = 0;
-        for (uint32_t s = 0; s < 256; ++s) {
-            sh.c[s] = (uint16_t)run;  // up to 4096 behind the last symbol that occurs
-            run += sh.f[s];
-        }
-        if (run != kProbScale) sh.bad = 1;
-    }
-    __syncthreads();
-    if (sh.bad) {
-        if (tid == 0 && status) atomicCAS(status, 0, (int32_t)CIERA_ERR_CORRUPT);
+    if (!decoder_tables(sh.f, sh.c, sh.sym, &sh.flag, tid)) {
+        if (tid == 0) raise_corrupt(status);
         return;
     }
-    // slot -> symbol: every thread looks up 16 consecutive slots.  The owner of a slot is the last
-    // symbol that starts at or below it (symbols that do not occur share their start with the next
-    // one, or start at 4096 behind the last occurring one): bisection over the 256 starts.
-    for (uint32_t slot = tid * 16; slot < tid * 16 + 16; ++slot) {
-        uint32_t lo = 0, hi = 255;
-        while (lo < hi) {
-            const uint32_t mid = (lo + hi + 1) >> 1;
-            if (sh.c[mid] <= slot)
-                lo = mid;
-            else
-                hi = mid - 1;
-        }
-        sh.sym[slot] = (uint8_t)lo;
-    }
-    __syncthreads();
-
+    // where the segments lie (nseg <= kLongSegs <= kEntThreads: one round)
     const uint32_t* dir = reinterpret_cast<const uint32_t*>(pay + 512);
     const uint8_t* data = pay + 512 + 4ull * nseg;
     const uint64_t data_bytes = C - 512ull - 4ull * nseg;
+    const uint32_t nw = tid < nseg ? dir[tid] : 0u;
+    if (nw > kSegWordsMax) sh.bad = 1;
+    uint32_t total;
+    sh.off[tid] = block_scan(tid < nseg ? segment_bytes(min(nw, kSegWordsMax)) : 0u, sh.scan, tid, total);
+    sh.nw[tid] = min(nw, kSegWordsMax);
+    __syncthreads();
+    if (sh.bad || total != data_bytes) {
+        if (tid == 0) raise_corrupt(status);
+        return;
+    }
     uint8_t* raw = scratch_raw + un.cache_off;  // the unit's stretch of the scratch (16-byte aligned)
+    for (uint32_t g = warp; g < nseg; g += kEntWarps) {
+        const uint32_t n = (uint32_t)min((uint64_t)kSegment, P - (uint64_t)g * kSegment);
+        if (!decode_segment(data + sh.off[g], sh.nw[g], n, sh.seg[warp], sh.sym, sh.f, sh.c, raw + (uint64_t)g * kSegment, lane))
+            sh.bad = 1;
+    }
+    __syncthreads();
+    if (sh.bad) {
+        if (tid == 0) raise_corrupt(status);
+        return;
+    }
+    // the raw payload goes back into the message, which then is what the sender step had written
+    for (uint64_t i = (uint64_t)tid * 16; i < P; i += (uint64_t)kEntThreads * 16) {
+        if (i + 16 <= P) {
+            *reinterpret_cast<uint4*>(pay + i) = *reinterpret_cast<const uint4*>(raw + i);
+        } else {
+            for (uint64_t k = i; k < P; ++k) pay[k] = raw[k];
+        }
+    }
+    if (tid == 0) wire_bytes[unit] = payoff + P;
+}
+
+// longer units: layout (one block per unit), segments and restore (grids over chunks)
+__global__ void __launch_bounds__(kEntThreads)
+entropy_long_parse_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
+                          const uint32_t* __restrict__ long_units, uint32_t smb, uint32_t log2b, const uint8_t* msgs,
+                          const unsigned long long* wire_bytes, uint8_t* recs, uint32_t* scratch_off, uint32_t* scratch_nw,
+                          int32_t* status) {
+    __shared__ uint32_t s_scan[kEntWarps];
+    __shared__ unsigned long long s_changed;
+    __shared__ uint32_t s_bad;
+    const uint32_t li = blockIdx.x, tid = threadIdx.x, unit = long_units[li];
+    const ciera_unit un = units[unit];
+    const uint64_t N = un.n_values;
+    LongState* st = long_state(recs, li);
+    if (tid == 0) {
+        st->coded = 0;
+        st->bad = 0;
+        s_changed = 0;
+        s_bad = 0;
+    }
+    __syncthreads();
+    const uint8_t* msg = msgs + un.msg_off;
+    const uint64_t payoff = payload_offset(N, smb, log2b);
+    const uint64_t P = raw_payload_bytes(msg, N, log2b, &s_changed, tid);
+    const uint64_t wire = wire_bytes[unit];
+    if (P == 0 || wire == payoff + P) return;
+    const uint64_t C = wire - payoff;
+    const uint64_t nseg64 = segments_of(P);
+    if (wire < payoff || C >= P || P >= (1ull << 32) || C < 512ull + 4ull * nseg64) {
+        if (tid == 0) raise_corrupt(status);
+        return;
+    }
+    const uint32_t nseg = (uint32_t)nseg64;
+    const uint8_t* pay = msg + payoff;
+    const uint32_t* dir = reinterpret_cast<const uint32_t*>(pay + 512);
+    const uint64_t data_bytes = C - 512ull - 4ull * nseg;
+    const unsigned long long slot0 = seg_base[unit];
     uint64_t carry = 0;
     for (uint32_t g0 = 0; g0 < nseg; g0 += kEntThreads) {
         const uint32_t g = g0 + tid;
         const uint32_t nw = g < nseg ? dir[g] : 0u;
-        const uint32_t size = g < nseg ? segment_bytes(min(nw, kSegWordsMax)) : 0u;
-        if (g < nseg && nw > kSegWordsMax) sh.bad = 1;
-        uint32_t incl = size;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
-            if ((int)lane >= o) incl += v;
+        if (nw > kSegWordsMax) s_bad = 1;
+        uint32_t total;
+        const uint32_t off = block_scan(g < nseg ? segment_bytes(min(nw, kSegWordsMax)) : 0u, s_scan, tid, total);
+        if (g < nseg) {
+            scratch_off[slot0 + g] = (uint32_t)(carry + off);
+            scratch_nw[slot0 + g] = min(nw, kSegWordsMax);
         }
-        if (lane == 31) sh.scan[warp] = incl;
-        __syncthreads();
-        uint32_t wbase = 0, chunk_total = 0;
-        for (int w = 0; w < kEntWarps; ++w) {
-            if (w < (int)warp) wbase += sh.scan[w];
-            chunk_total += sh.scan[w];
-        }
-        sh.off[tid] = wbase + incl - size;
-        sh.nw[tid] = min(nw, kSegWordsMax);
-        if (tid == 0 && carry + chunk_total > data_bytes) sh.bad = 1;  // sizes must stay inside the section
-        __syncthreads();
-        if (sh.bad) break;
-        const uint32_t in_chunk = min((uint32_t)kEntThreads, nseg - g0);
-        for (uint32_t k = warp; k < in_chunk; k += kEntWarps) {
-            const uint32_t gg = g0 + k;
-            const uint32_t n = (uint32_t)min((uint64_t)kSegment, P - (uint64_t)gg * kSegment);
-            const uint32_t snw = sh.nw[k];
-            // the coded segment into shared memory (4-byte aligned in the section)
-            const uint32_t* from = reinterpret_cast<const uint32_t*>(data + carry + sh.off[k]);
-            uint32_t* stage = reinterpret_cast<uint32_t*>(sh.seg[warp]);
-            for (uint32_t i = lane; i < (segment_bytes(snw) >> 2); i += 32) stage[i] = from[i];
-            __syncwarp();
-            const uint16_t* words = reinterpret_cast<const uint16_t*>(sh.seg[warp] + 4 * 32);
-            uint32_t x = stage[lane], ptr = snw;
-            uint8_t* out = raw + (uint64_t)gg * kSegment;
-            const uint32_t steps = (n + 31u) >> 5;
-            bool broken = false;
-            for (uint32_t t = 0; t < steps; ++t) {
-                const uint32_t i = 32u * t + lane;
-                const bool has = i < n;
-                bool need = false;
-                if (has) {
-                    const uint32_t slot = x & (kProbScale - 1u);
-                    const uint32_t s = sh.sym[slot];
-                    out[i] = (uint8_t)s;
-                    x = (uint32_t)sh.f[s] * (x >> kProbBits) + slot - sh.c[s];
-                    need = x < kRansL;
-                }
-                const uint32_t votes = __ballot_sync(0xffffffffu, need);
-                const uint32_t k_need = __popc(votes);
-                if (k_need > ptr) {
-                    broken = true;
-                    break;
-                }
-                if (need) x = (x << 16) | words[ptr - k_need + __popc(votes & ((1u << lane) - 1u))];
-                ptr -= k_need;
-            }
-            // all words used and every lane back at the start state, or the section is damaged
-            if (broken || ptr != 0 || __any_sync(0xffffffffu, x != kRansL)) sh.bad = 1;
-            __syncwarp();
-        }
-        carry += chunk_total;
-        __syncthreads();
-        if (sh.bad) break;
+        carry += total;
     }
     __syncthreads();
-    if (sh.bad || carry != data_bytes) {
-        if (tid == 0 && status) atomicCAS(status, 0, (int32_t)CIERA_ERR_CORRUPT);
+    if (s_bad || carry != data_bytes) {
+        if (tid == 0) raise_corrupt(status);
         return;
     }
-    // the raw payload goes back into the message, which then is what the sender step had written
-    __threadfence_block();
-    uint8_t* dst = msg + payoff;
-    for (uint64_t i = (uint64_t)tid * 16; i < P; i += (uint64_t)kEntThreads * 16) {
-        if (i + 16 <= P) {
-            *reinterpret_cast<uint4*>(dst + i) = *reinterpret_cast<const uint4*>(raw + i);
+    if (tid == 0) {
+        st->P = P;
+        st->nseg = nseg;
+        st->coded = 1;
+    }
+}
+
+__global__ void __launch_bounds__(kEntThreads)
+entropy_long_decode_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
+                           const uint4* __restrict__ chunks, uint32_t smb, uint32_t log2b, const uint8_t* msgs,
+                           uint8_t* recs, const uint32_t* scratch_off, const uint32_t* scratch_nw, uint8_t* scratch_raw,
+                           int32_t* status) {
+    extern __shared__ __align__(16) uint8_t smem_raw[];
+    DecodeShared& sh = *reinterpret_cast<DecodeShared*>(smem_raw);
+    const uint4 ch = chunks[blockIdx.x];
+    LongState* st = long_state(recs, ch.z);
+    if (st->coded == 0 || ch.y >= st->nseg) return;
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const ciera_unit un = units[ch.x];
+    const uint64_t P = st->P;
+    const uint32_t nseg = st->nseg;
+    const uint8_t* pay = msgs + un.msg_off + payload_offset(un.n_values, smb, log2b);
+    sh.f[tid] = reinterpret_cast<const uint16_t*>(pay)[tid];
+    if (tid == 0) sh.bad = 0;
+    __syncthreads();
+    if (!decoder_tables(sh.f, sh.c, sh.sym, &sh.flag, tid)) {
+        if (tid == 0) {
+            st->bad = 1;
+            raise_corrupt(status);
+        }
+        return;
+    }
+    const uint8_t* data = pay + 512 + 4ull * nseg;
+    uint8_t* raw = scratch_raw + un.cache_off;
+    const unsigned long long slot0 = seg_base[ch.x];
+    const uint32_t g_end = min(nseg, ch.y + kLongSegs);
+    for (uint32_t g = ch.y + warp; g < g_end; g += kEntWarps) {
+        const uint32_t n = (uint32_t)min((uint64_t)kSegment, P - (uint64_t)g * kSegment);
+        if (!decode_segment(data + scratch_off[slot0 + g], scratch_nw[slot0 + g], n, sh.seg[warp], sh.sym, sh.f, sh.c,
+                            raw + (uint64_t)g * kSegment, lane))
+            sh.bad = 1;
+    }
+    __syncthreads();
+    if (tid == 0 && sh.bad) {
+        st->bad = 1;
+        raise_corrupt(status);
+    }
+}
+
+__global__ void __launch_bounds__(kEntThreads)
+entropy_long_restore_kernel(const ciera_unit* __restrict__ units, const uint4* __restrict__ chunks, uint32_t smb,
+                            uint32_t log2b, uint8_t* msgs, unsigned long long* wire_bytes, const uint8_t* recs_c,
+                            const uint8_t* scratch_raw) {
+    const uint4 ch = chunks[blockIdx.x];
+    const LongState* st = long_state(const_cast<uint8_t*>(recs_c), ch.z);
+    if (st->coded == 0 || st->bad != 0) return;  // raw as received, or damaged: left as it is
+    const uint32_t tid = threadIdx.x;
+    const ciera_unit un = units[ch.x];
+    const uint64_t P = st->P;
+    const uint64_t lo = (uint64_t)ch.y * kSegment;
+    if (lo >= P) return;
+    const uint64_t hi = min(P, lo + (uint64_t)kLongSegs * kSegment);
+    const uint64_t payoff = payload_offset(un.n_values, smb, log2b);
+    uint8_t* pay = msgs + un.msg_off + payoff;
+    const uint8_t* raw = scratch_raw + un.cache_off;
+    for (uint64_t i = lo + (uint64_t)tid * 16; i < hi; i += (uint64_t)kEntThreads * 16) {
+        if (i + 16 <= hi) {
+            *reinterpret_cast<uint4*>(pay + i) = *reinterpret_cast<const uint4*>(raw + i);
         } else {
-            for (uint64_t k = i; k < P; ++k) dst[k] = raw[k];
+            for (uint64_t k = i; k < hi; ++k) pay[k] = raw[k];
         }
     }
-    if (tid == 0) wire_bytes[unit] = payoff + P;
+    if (ch.y == 0 && tid == 0) wire_bytes[ch.x] = payoff + P;
 }
 
 }  // namespace ciera
@@ -385,43 +713,81 @@ entropy_decode_kernel(const ciera_unit* __restrict__ units, uint32_t sm_bytes_pe
 using namespace ciera;
 
 static bool misaligned16(const void* p) { return ((uintptr_t)p & 15u) != 0; }
+static size_t up16(size_t x) { return (x + 15) / 16 * 16; }
 
-// scratch of the sender stage: per segment slot a word count and kSegSlot bytes
-static size_t encode_scratch_bytes(const ciera_plan* p) {
-    return ((size_t)p->total_segments * sizeof(uint32_t) + 15) / 16 * 16 + (size_t)p->total_segments * kSegSlot;
+// Scratch: [word count per segment slot][byte offset per segment slot][a record per long unit]
+// [body: the segment slots (sender) or the raw payloads at the units' cache offsets (receiver)]
+struct ScratchLayout {
+    size_t nw, off, recs, body, total;
+};
+static ScratchLayout scratch_layout(const ciera_plan* p) {
+    ScratchLayout L;
+    L.nw = 0;
+    L.off = L.nw + up16((size_t)p->total_segments * sizeof(uint32_t));
+    L.recs = L.off + up16((size_t)p->total_segments * sizeof(uint32_t));
+    L.body = L.recs + (size_t)p->ent_long_units.size() * kLongRec;
+    const size_t enc = (size_t)p->total_segments * kSegSlot, dec = (size_t)p->cache_extent;
+    L.total = L.body + (enc > dec ? enc : dec) + 16;
+    return L;
 }
 
-extern "C" size_t ciera_plan_entropy_scratch_bytes(const ciera_plan* p) {
-    if (!p) return 0;
-    const size_t enc = encode_scratch_bytes(p), dec = (size_t)p->cache_extent;
-    return (enc > dec ? enc : dec) + 16;
+extern "C" size_t ciera_plan_entropy_scratch_bytes(const ciera_plan* p) { return p ? scratch_layout(p).total : 0; }
+
+static int check_entropy_args(const ciera_plan* p, const void* messages_dev, const void* wire_bytes_dev,
+                              const void* scratch_dev) {
+    if (!p) return CIERA_ERR_INVALID_ARG;
+    if (!p->tiles.empty() && !p->tiles_dev) return CIERA_ERR_NOT_BOUND;
+    if (p->tiles.empty()) return CIERA_OK;
+    if (!messages_dev || !wire_bytes_dev || !scratch_dev) return CIERA_ERR_INVALID_ARG;
+    if (misaligned16(messages_dev) || misaligned16(scratch_dev) || ((uintptr_t)wire_bytes_dev & 7u))
+        return CIERA_ERR_MISALIGNED;
+    return CIERA_OK;
 }
 
 extern "C" int ciera_entropy_encode(const ciera_plan* p, void* messages_dev, uint64_t* wire_bytes_dev, void* scratch_dev,
                                     void* stream) {
-    if (!p) return CIERA_ERR_INVALID_ARG;
-    if (!p->tiles.empty() && !p->tiles_dev) return CIERA_ERR_NOT_BOUND;
-    if (p->tiles.empty()) return CIERA_OK;
-    if (!messages_dev || !wire_bytes_dev || !scratch_dev) return CIERA_ERR_INVALID_ARG;
-    if (misaligned16(messages_dev) || misaligned16(scratch_dev) || ((uintptr_t)wire_bytes_dev & 7u))
-        return CIERA_ERR_MISALIGNED;
-    uint32_t* nw = (uint32_t*)scratch_dev;
-    uint8_t* slots = (uint8_t*)scratch_dev + ((size_t)p->total_segments * sizeof(uint32_t) + 15) / 16 * 16;
-    entropy_encode_kernel<<<p->n_units, kEntThreads, 0, (cudaStream_t)stream>>>(
-        p->units_dev, p->seg_base_dev, p->dtype == CIERA_BF16 ? 1u : 3u, p->log2b, (uint8_t*)messages_dev,
-        (unsigned long long*)wire_bytes_dev, slots, nw);
-    count_launch();
-    return check_launch();
+    int rc = check_entropy_args(p, messages_dev, wire_bytes_dev, scratch_dev);
+    if (rc || p->tiles.empty()) return rc;
+    cudaStream_t s = (cudaStream_t)stream;
+    const ScratchLayout L = scratch_layout(p);
+    uint8_t* base = (uint8_t*)scratch_dev;
+    uint32_t* nw = (uint32_t*)(base + L.nw);
+    uint32_t* off = (uint32_t*)(base + L.off);
+    uint8_t* recs = base + L.recs;
+    uint8_t* slots = base + L.body;
+    const uint32_t smb = p->dtype == CIERA_BF16 ? 1u : 3u;
+    uint8_t* msgs = (uint8_t*)messages_dev;
+    unsigned long long* wire = (unsigned long long*)wire_bytes_dev;
+    const uint32_t n_long = (uint32_t)p->ent_long_units.size(), n_chunks = (uint32_t)p->ent_chunks.size();
+    if (n_long < p->n_units) {
+        entropy_encode_kernel<<<p->n_units, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, smb, p->log2b, msgs, wire,
+                                                                 slots, nw);
+        count_launch();
+        if ((rc = check_launch())) return rc;
+    }
+    if (n_long) {
+        cudaError_t e = cudaMemsetAsync(recs, 0, (size_t)n_long * kLongRec, s);  // the counts start at zero
+        if (e != cudaSuccess) return record_cuda_error(e);
+        entropy_long_hist_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->ent_chunks_dev, smb, p->log2b, msgs, wire,
+                                                                  recs);
+        entropy_long_model_kernel<<<n_long, kEntThreads, 0, s>>>(p->units_dev, p->ent_long_units_dev, smb, p->log2b, wire,
+                                                                 recs);
+        entropy_long_encode_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_chunks_dev, smb,
+                                                                    p->log2b, msgs, wire, recs, slots, nw);
+        entropy_long_layout_kernel<<<n_long, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_long_units_dev, smb,
+                                                                  p->log2b, msgs, wire, recs, nw, off);
+        entropy_long_copy_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_chunks_dev, smb,
+                                                                  p->log2b, msgs, recs, slots, nw, off);
+        for (int i = 0; i < 5; ++i) count_launch();
+        if ((rc = check_launch())) return rc;
+    }
+    return CIERA_OK;
 }
 
 extern "C" int ciera_entropy_decode(const ciera_plan* p, void* messages_dev, uint64_t* wire_bytes_dev, void* scratch_dev,
                                     int32_t* status_dev, void* stream) {
-    if (!p) return CIERA_ERR_INVALID_ARG;
-    if (!p->tiles.empty() && !p->tiles_dev) return CIERA_ERR_NOT_BOUND;
-    if (p->tiles.empty()) return CIERA_OK;
-    if (!messages_dev || !wire_bytes_dev || !scratch_dev) return CIERA_ERR_INVALID_ARG;
-    if (misaligned16(messages_dev) || misaligned16(scratch_dev) || ((uintptr_t)wire_bytes_dev & 7u))
-        return CIERA_ERR_MISALIGNED;
+    int rc = check_entropy_args(p, messages_dev, wire_bytes_dev, scratch_dev);
+    if (rc || p->tiles.empty()) return rc;
     static std::atomic<int> configured[64];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -431,11 +797,37 @@ extern "C" int ciera_entropy_decode(const ciera_plan* p, void* messages_dev, uin
         e = cudaFuncSetAttribute(entropy_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)sizeof(DecodeShared));
         if (e != cudaSuccess) return record_cuda_error(e);
+        e = cudaFuncSetAttribute(entropy_long_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)sizeof(DecodeShared));
+        if (e != cudaSuccess) return record_cuda_error(e);
         configured[dev].store(1, std::memory_order_release);
     }
-    entropy_decode_kernel<<<p->n_units, kEntThreads, sizeof(DecodeShared), (cudaStream_t)stream>>>(
-        p->units_dev, p->dtype == CIERA_BF16 ? 1u : 3u, p->log2b, (uint8_t*)messages_dev,
-        (unsigned long long*)wire_bytes_dev, (uint8_t*)scratch_dev, status_dev);
-    count_launch();
-    return check_launch();
+    cudaStream_t s = (cudaStream_t)stream;
+    const ScratchLayout L = scratch_layout(p);
+    uint8_t* base = (uint8_t*)scratch_dev;
+    uint32_t* nw = (uint32_t*)(base + L.nw);
+    uint32_t* off = (uint32_t*)(base + L.off);
+    uint8_t* recs = base + L.recs;
+    uint8_t* raw = base + L.body;
+    const uint32_t smb = p->dtype == CIERA_BF16 ? 1u : 3u;
+    uint8_t* msgs = (uint8_t*)messages_dev;
+    unsigned long long* wire = (unsigned long long*)wire_bytes_dev;
+    const uint32_t n_long = (uint32_t)p->ent_long_units.size(), n_chunks = (uint32_t)p->ent_chunks.size();
+    if (n_long < p->n_units) {
+        entropy_decode_kernel<<<p->n_units, kEntThreads, sizeof(DecodeShared), s>>>(p->units_dev, smb, p->log2b, msgs, wire,
+                                                                                   raw, status_dev);
+        count_launch();
+        if ((rc = check_launch())) return rc;
+    }
+    if (n_long) {
+        entropy_long_parse_kernel<<<n_long, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_long_units_dev, smb,
+                                                                 p->log2b, msgs, wire, recs, off, nw, status_dev);
+        entropy_long_decode_kernel<<<n_chunks, kEntThreads, sizeof(DecodeShared), s>>>(
+            p->units_dev, p->seg_base_dev, p->ent_chunks_dev, smb, p->log2b, msgs, recs, off, nw, raw, status_dev);
+        entropy_long_restore_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->ent_chunks_dev, smb, p->log2b, msgs,
+                                                                     wire, recs, raw);
+        for (int i = 0; i < 3; ++i) count_launch();
+        if ((rc = check_launch())) return rc;
+    }
+    return CIERA_OK;
 }

@@ -66,7 +66,7 @@ extern "C" size_t ciera_message_bytes(uint64_t n, int dtype, uint32_t block, uin
 
 namespace {
 struct ImageLayout {
-    size_t tiles, long_off, seq_off, hash_off, first_off, seg_off, units_off, total;
+    size_t tiles, long_off, seq_off, hash_off, first_off, seg_off, units_off, elong_off, echunk_off, total;
 };
 size_t up16(size_t x) { return (x + 15) / 16 * 16; }
 ImageLayout image_layout(const ciera_plan* p) {
@@ -78,7 +78,9 @@ ImageLayout image_layout(const ciera_plan* p) {
     L.first_off = L.hash_off + up16((size_t)p->n_units * sizeof(uint64_t));
     L.seg_off = L.first_off + up16((size_t)p->n_units * sizeof(uint32_t));
     L.units_off = L.seg_off + up16((size_t)p->n_units * sizeof(uint64_t));
-    L.total = L.units_off + up16((size_t)p->n_units * sizeof(ciera_unit)) + 16;
+    L.elong_off = L.units_off + up16((size_t)p->n_units * sizeof(ciera_unit));
+    L.echunk_off = L.elong_off + up16(p->ent_long_units.size() * sizeof(uint32_t));
+    L.total = L.echunk_off + p->ent_chunks.size() * sizeof(ciera_plan::EntChunk) + 16;
     return L;
 }
 }  // namespace
@@ -162,6 +164,12 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
         p->seg_base[u] = p->total_segments;
         p->total_segments += (units_host[u].n_values + 4095) / 4096;
         p->cache_extent = std::max<uint64_t>(p->cache_extent, units_host[u].cache_off + units_host[u].n_values);
+        const uint64_t slots = (units_host[u].n_values + 4095) / 4096;
+        if (slots > 64) {  // the entropy stage spreads such a unit over several thread blocks
+            const uint32_t li = (uint32_t)p->ent_long_units.size();
+            p->ent_long_units.push_back(u);
+            for (uint64_t g = 0; g < slots; g += 64) p->ent_chunks.push_back({u, (uint32_t)g, li, 0u});
+        }
     }
     // device image: the tile table, then (each 16-byte aligned) the index lists
     const ImageLayout L = image_layout(p);
@@ -174,6 +182,10 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
         memcpy(p->image.data() + L.first_off, p->unit_first.data(), (size_t)n_units * 4);
         memcpy(p->image.data() + L.seg_off, p->seg_base.data(), (size_t)n_units * 8);
         memcpy(p->image.data() + L.units_off, p->units.data(), (size_t)n_units * sizeof(ciera_unit));
+        if (!p->ent_long_units.empty()) {
+            memcpy(p->image.data() + L.elong_off, p->ent_long_units.data(), p->ent_long_units.size() * sizeof(uint32_t));
+            memcpy(p->image.data() + L.echunk_off, p->ent_chunks.data(), p->ent_chunks.size() * sizeof(ciera_plan::EntChunk));
+        }
     }
     *plan_out = p;
     return CIERA_OK;
@@ -224,6 +236,8 @@ extern "C" int ciera_plan_bind(ciera_plan* p, void* plan_dev, size_t plan_dev_by
     p->unit_first_dev = (const uint32_t*)(base + L.first_off);
     p->seg_base_dev = (const unsigned long long*)(base + L.seg_off);
     p->units_dev = (const ciera_unit*)(base + L.units_off);
+    p->ent_long_units_dev = (const uint32_t*)(base + L.elong_off);
+    p->ent_chunks_dev = (const uint4*)(base + L.echunk_off);
     return CIERA_OK;
 }
 

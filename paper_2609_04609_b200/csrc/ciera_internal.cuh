@@ -115,7 +115,17 @@ struct ciera_plan {
     std::vector<uint64_t> seg_base;    // index of every unit's first 4096-byte payload segment (entropy stage)
     uint64_t total_segments = 0;
     uint64_t cache_extent = 0;         // max over units of cache_off + n_values
-    std::vector<uint8_t> image;        // device image: tiles, long_units, seq_first, hash_base, unit_first, seg_base, units
+    // entropy stage: units of more than 64 segment slots, and their chunks of 64 slots
+    // {unit, first segment of the chunk inside the unit, index among the long units, 0}
+    struct EntChunk {
+        uint32_t unit, first_seg, long_index, zero;
+    };
+    std::vector<uint32_t> ent_long_units;
+    std::vector<EntChunk> ent_chunks;
+    const uint32_t* ent_long_units_dev = nullptr;
+    const uint4* ent_chunks_dev = nullptr;
+    std::vector<uint8_t> image;        // device image: tiles, long_units, seq_first, hash_base, unit_first, seg_base, units,
+                                       // ent_long_units, ent_chunks
     const ciera::TileDesc* tiles_dev = nullptr;
     const uint32_t* long_units_dev = nullptr;
     const uint32_t* seq_first_dev = nullptr;

@@ -114,9 +114,25 @@ def test_entropy_stage_unit_of_many_segments(rt):
     assert coded > 0
 
 
-def test_entropy_decode_flags_a_damaged_section(rt):
+def test_entropy_stage_long_and_short_units_mixed(rt):
+    """Units above and below 262 144 values in one table (the long ones are spread over several
+    thread blocks), a long unit with incompressible exponents among them."""
+    sizes = [300_000, 1000, 700_001, 262_144, 262_145, 50_000]
+    codec = rt[1].LayerCodec.from_tensors(sizes, 1, "bf16", 128, DEV)
+    n = codec.weights_bytes // 2
+    traj = [wl.as_bits(w) for w in wl.trajectory(n, "bf16", 21, 2, "adam")]
+    lo = int(codec.units[0]["weights_off"]) // 2
+    rng = np.random.default_rng(2)
+    for w in traj:  # unit 0: arbitrary bit patterns, new ones every step
+        w[lo : lo + 300_000] = rng.integers(0, 1 << 16, 300_000, dtype=np.uint64).astype(np.uint16)
+    coded = _run(rt, sizes, 1, 0, 128, [traj[0]] + traj, from_zero=True)
+    assert coded >= 4
+
+
+@pytest.mark.parametrize("n_values", [70_001, 600_001])
+def test_entropy_decode_flags_a_damaged_section(rt, n_values):
     ciera, runtime = rt
-    sizes = [70_001]
+    sizes = [n_values]
     codec = runtime.LayerCodec.from_tensors(sizes, 1, "bf16", 512, DEV)
     n = codec.weights_bytes // 2
     w = wl.as_bits(next(iter(wl.trajectory(n, "bf16", 3, 0, "adam"))))
@@ -125,10 +141,14 @@ def test_entropy_decode_flags_a_damaged_section(rt):
     codec.entropy_encode()
     codec.transport()
     torch.cuda.synchronize()
-    raw_len = ora.payload_offset(70_001, 0, 512) + 70_001
+    raw_len = ora.payload_offset(n_values, 0, 512) + n_values
     assert int(codec.wire_bytes[0].item()) < raw_len  # the coded form travelled
-    off = int(codec.units[0]["msg_off"]) + ora.payload_offset(70_001, 0, 512)
-    codec.msg_recv[off + 512 + 4 * 18 + 200] ^= 0x5A  # inside the first segment's words
+    off = int(codec.units[0]["msg_off"]) + ora.payload_offset(n_values, 0, 512)
+    nseg = -(-n_values // 4096)
+    before = codec.msg_recv.clone()
+    codec.msg_recv[off + 512 + 4 * nseg + 200] ^= 0x5A  # inside the first segment's words
+    damaged = codec.msg_recv.clone()
     codec.entropy_decode()
     torch.cuda.synchronize()
     assert int(codec.status.item()) == ciera.ERR_CORRUPT
+    assert torch.equal(codec.msg_recv, damaged) and not torch.equal(damaged, before)  # left as received
