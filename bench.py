@@ -68,7 +68,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-regimes", action="store_true")
-    ap.add_argument("--cpu-sample-units", type=int, default=1024)
+    ap.add_argument("--cpu-sample-units", type=int, default=3072, help="units per layer given to the CPU oracle")
+    ap.add_argument("--cpu-sample-layers", type=int, default=4, help="layers given to the CPU oracle")
     return ap.parse_args()
 
 
@@ -454,6 +455,12 @@ def main():
         c.check_status()
 
     # ---- what was moved: change rates and the paper's byte count of the last step
+    # element change rate c of the workload (reporting only): exponent fields of the two iterates of layer 0
+    shift, wdt_t = (7, torch.int16) if args.dtype == "bf16" else (23, torch.int32)
+    ea = (wa[0].view(wdt_t) >> shift) & 0xFF
+    eb = (wb[0].view(wdt_t) >> shift) & 0xFF
+    element_change_rate = float((ea != eb).float().mean().item())
+    del ea, eb
     changed = sum(int(c.changed_blocks.sum().item()) for c in layers)
     blocks = sum(c.n_blocks() for c in layers)
     q = changed / blocks
@@ -547,6 +554,7 @@ def main():
         "gpu_launches": int(launches),
         "clocks": clocks,
         "verified_bit_exact": bool(verified),
+        "element_change_rate_c": element_change_rate,
         "entropy_stage": coded,
         "oracle_sampled_units": sampled,
         "block_change_rate_q": q,
@@ -591,14 +599,22 @@ def main():
     # ---- the oracle on this machine's host cores (rank 0, one GPU only)
     if not args.no_cpu_baseline and rank == 0 and world == 1:
         threads = os.cpu_count() or 1
-        units = layers[0].units[: args.cpu_sample_units]
-        hi = int(units[-1]["weights_off"]) + int(units[-1]["n_values"]) * vb
-        a = wa[0][:hi].cpu().numpy()
-        b = wb[0][:hi].cpu().numpy()
-        dt, nv = oracle_roundtrip_units(units, a, b, ciera.DTYPE_CODES[args.dtype], args.block, vb, threads)
+        code = ciera.DTYPE_CODES[args.dtype]
+        dt = nv = nu = 0
+        for l in range(min(len(layers), args.cpu_sample_layers)):  # a bounded sample: some seconds of CPU work
+            units = layers[l].units[: args.cpu_sample_units]
+            hi = int(units[-1]["weights_off"]) + int(units[-1]["n_values"]) * vb
+            a = wa[l][:hi].cpu().numpy()
+            b = wb[l][:hi].cpu().numpy()
+            d, n = oracle_roundtrip_units(units, a, b, code, args.block, vb, threads)
+            dt, nv, nu = dt + d, nv + n, nu + len(units)
+        units1 = layers[0].units[: max(1, min(args.cpu_sample_units, 256))]
+        hi = int(units1[-1]["weights_off"]) + int(units1[-1]["n_values"]) * vb
+        d1, n1 = oracle_roundtrip_units(units1, wa[0][:hi].cpu().numpy(), wb[0][:hi].cpu().numpy(), code, args.block, vb, 1)
         out["cpu_baseline"] = {"value": nv * vb / dt / 1e9, "unit": "GB/s", "cores": threads, "kind": "oracle",
-                               "sample": f"{len(units)} of {sum(len(c.units) for c in layers)} units "
-                                         f"({nv} values), encode+decode round trip, {dt:.2f} s wall"}
+                               "sample": f"{nu} of {sum(len(c.units) for c in layers)} units ({nv} values), "
+                                         f"encode+decode round trip, {dt:.2f} s wall on {threads} threads",
+                               "single_thread_value": n1 * vb / d1 / 1e9}
     if rank == 0:
         print(json.dumps(out))
     if world > 1:
