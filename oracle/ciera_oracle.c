@@ -43,11 +43,32 @@
 #include <stdlib.h>
 #include <string.h>
 
-enum { ORA_BF16 = 0, ORA_FP32 = 1 };
+enum { ORA_BF16 = 0, ORA_FP32 = 1, ORA_FP16 = 2 };
 
-/* b = bits per value, m = sign+mantissa bits (b minus the 8 exponent bits). */
-static int ora_b(int dtype) { return dtype == ORA_BF16 ? 16 : 32; }
-static int ora_m(int dtype) { return ora_b(dtype) - 8; }
+/* b = bits per value, e = exponent bits, m = b - e = sign+mantissa bits (Section 3.1: a value is
+ * sign, exponent and mantissa bits).  bf16: 16 = 1 + 8 + 7; fp32: 32 = 1 + 8 + 23; fp16 (IEEE
+ * binary16): 16 = 1 + 5 + 10.  Caches hold one byte per value for every precision; on the wire an
+ * exponent takes e bits and a sign-plus-mantissa m bits, packed without gaps (reading: value j of a
+ * section occupies bits [j*w, (j+1)*w) of the section's bytes, bit i of a section = byte i >> 3,
+ * bit i & 7 -- for w = 8 and w = 24 this is one byte and three little-endian bytes per value). */
+static int ora_b(int dtype) { return dtype == ORA_FP32 ? 32 : 16; }
+static int ora_e(int dtype) { return dtype == ORA_FP16 ? 5 : 8; }
+static int ora_m(int dtype) { return ora_b(dtype) - ora_e(dtype); }
+
+static void put_bits(uint8_t* buf, uint64_t bitpos, int width, uint32_t value) {
+    for (int i = 0; i < width; ++i) {
+        uint64_t p = bitpos + (uint64_t)i;
+        if ((value >> i) & 1u) buf[p >> 3] |= (uint8_t)(1u << (p & 7));
+    }
+}
+static uint32_t get_bits(const uint8_t* buf, uint64_t bitpos, int width) {
+    uint32_t v = 0;
+    for (int i = 0; i < width; ++i) {
+        uint64_t p = bitpos + (uint64_t)i;
+        v |= (uint32_t)((buf[p >> 3] >> (p & 7)) & 1u) << i;
+    }
+    return v;
+}
 
 static uint64_t pad16(uint64_t x) { return (x + 15u) / 16u * 16u; }
 
@@ -57,8 +78,12 @@ uint64_t ora_num_blocks(uint64_t n, uint32_t block) { return (n + block - 1) / b
 /* S_bm = ceil(S_b / 8) bytes  (Section 3.2). */
 uint64_t ora_bitmap_bytes(uint64_t n, uint32_t block) { return (ora_num_blocks(n, block) + 7) / 8; }
 
-/* S_{s+m} = N * m / 8 bytes  (Section 3.2: S - S_e with S_e = N bytes). */
-uint64_t ora_sm_bytes(uint64_t n, int dtype) { return n * (uint64_t)ora_m(dtype) / 8; }
+/* S_{s+m} = N * m / 8 bytes  (Section 3.2: S - S_e), rounded up to whole bytes. */
+uint64_t ora_sm_bytes(uint64_t n, int dtype) { return (n * (uint64_t)ora_m(dtype) + 7) / 8; }
+
+/* Exponent bytes of one block of len values on the wire: len * e / 8, rounded up (every block of
+ * the payload starts on a byte boundary). */
+uint64_t ora_block_payload_bytes(uint64_t len, int dtype) { return (len * (uint64_t)ora_e(dtype) + 7) / 8; }
 
 uint64_t ora_sm_offset(uint64_t n, uint32_t block) { return pad16(ora_bitmap_bytes(n, block)); }
 
@@ -66,10 +91,13 @@ uint64_t ora_payload_offset(uint64_t n, int dtype, uint32_t block) {
     return ora_sm_offset(n, block) + pad16(ora_sm_bytes(n, dtype));
 }
 
-/* Worst case: every block changed, payload = N exponent bytes. */
+/* Worst case: every block changed (payload = N exponent bytes when e = 8). */
 uint64_t ora_message_capacity(uint64_t n, int dtype, uint32_t block) {
     if (n == 0) return 0;
-    return ora_payload_offset(n, dtype, block) + n;
+    uint64_t nb = ora_num_blocks(n, block);
+    uint64_t last = n - (nb - 1) * block;
+    return ora_payload_offset(n, dtype, block) + (nb - 1) * ora_block_payload_bytes(block, dtype) +
+           ora_block_payload_bytes(last, dtype);
 }
 
 /* The paper's transmitted-byte count S_{s+m} + S_bm + (changed exponent bytes). */
@@ -78,7 +106,7 @@ uint64_t ora_paper_bytes(uint64_t n, int dtype, uint32_t block, uint64_t payload
 }
 
 static uint32_t load_bits(const void* w, uint64_t j, int dtype) {
-    if (dtype == ORA_BF16) {
+    if (ora_b(dtype) == 16) {
         uint16_t v;
         memcpy(&v, (const uint8_t*)w + 2 * j, 2);
         return v;
@@ -89,7 +117,7 @@ static uint32_t load_bits(const void* w, uint64_t j, int dtype) {
 }
 
 static void store_bits(void* w, uint64_t j, int dtype, uint32_t bits) {
-    if (dtype == ORA_BF16) {
+    if (ora_b(dtype) == 16) {
         uint16_t v = (uint16_t)bits;
         memcpy((uint8_t*)w + 2 * j, &v, 2);
     } else {
@@ -101,7 +129,7 @@ static void store_bits(void* w, uint64_t j, int dtype, uint32_t bits) {
 static void split_value(uint32_t bits, int dtype, uint8_t* exp, uint32_t* sm) {
     int b = ora_b(dtype), m = ora_m(dtype);
     uint32_t sign = (bits >> (b - 1)) & 1u;
-    uint32_t expo = (bits >> (m - 1)) & 0xFFu;
+    uint32_t expo = (bits >> (m - 1)) & ((1u << ora_e(dtype)) - 1u);
     uint32_t mant = bits & ((1u << (m - 1)) - 1u);
     *exp = (uint8_t)expo;
     *sm = (sign << (m - 1)) | mant;
@@ -153,7 +181,7 @@ int ora_encode(const void* w, uint8_t* cache_s, uint64_t n, int dtype, uint32_t 
     if (n == 0) return 0;
     if (msg_capacity < ora_message_capacity(n, dtype, block)) return -2;
 
-    int m = ora_m(dtype);
+    int m = ora_m(dtype), e = ora_e(dtype);
     uint64_t nb = ora_num_blocks(n, block);
     uint64_t sm_off = ora_sm_offset(n, block);
     uint64_t pay_off = ora_payload_offset(n, dtype, block);
@@ -185,15 +213,7 @@ int ora_encode(const void* w, uint8_t* cache_s, uint64_t n, int dtype, uint32_t 
     }
 
     /* sign-plus-mantissa of all values. */
-    for (uint64_t j = 0; j < n; ++j) {
-        if (m == 8) {
-            msg[sm_off + j] = (uint8_t)sm[j];
-        } else {
-            msg[sm_off + 3 * j + 0] = (uint8_t)(sm[j] & 0xFF);
-            msg[sm_off + 3 * j + 1] = (uint8_t)((sm[j] >> 8) & 0xFF);
-            msg[sm_off + 3 * j + 2] = (uint8_t)((sm[j] >> 16) & 0xFF);
-        }
-    }
+    for (uint64_t j = 0; j < n; ++j) put_bits(msg + sm_off, j * (uint64_t)m, m, sm[j]);
 
     /* payload <- { exp[k] | bitmap[k] = 1 } in block order. */
     uint64_t plen = 0;
@@ -202,7 +222,10 @@ int ora_encode(const void* w, uint8_t* cache_s, uint64_t n, int dtype, uint32_t 
         if (!((msg[k >> 3] >> (k & 7)) & 1u)) continue;
         uint64_t lo = k * block;
         uint64_t hi = lo + block < n ? lo + block : n;
-        for (uint64_t j = lo; j < hi; ++j) msg[pay_off + plen++] = exp[j];
+        uint64_t nbytes = ora_block_payload_bytes(hi - lo, dtype);
+        memset(msg + pay_off + plen, 0, nbytes);
+        for (uint64_t j = lo; j < hi; ++j) put_bits(msg + pay_off + plen, (j - lo) * (uint64_t)e, e, exp[j]);
+        plen += nbytes;
         ++nchg;
     }
 
@@ -296,7 +319,7 @@ int ora_encode_hashed(const void* w, uint64_t* hash_cache, uint64_t n, int dtype
     if (n == 0) return 0;
     if (msg_capacity < ora_message_capacity(n, dtype, block)) return -2;
 
-    int m = ora_m(dtype);
+    int m = ora_m(dtype), e = ora_e(dtype);
     uint64_t nb = ora_num_blocks(n, block);
     uint64_t sm_off = ora_sm_offset(n, block);
     uint64_t pay_off = ora_payload_offset(n, dtype, block);
@@ -325,15 +348,7 @@ int ora_encode_hashed(const void* w, uint64_t* hash_cache, uint64_t n, int dtype
         }
     }
 
-    for (uint64_t j = 0; j < n; ++j) {
-        if (m == 8) {
-            msg[sm_off + j] = (uint8_t)sm[j];
-        } else {
-            msg[sm_off + 3 * j + 0] = (uint8_t)(sm[j] & 0xFF);
-            msg[sm_off + 3 * j + 1] = (uint8_t)((sm[j] >> 8) & 0xFF);
-            msg[sm_off + 3 * j + 2] = (uint8_t)((sm[j] >> 16) & 0xFF);
-        }
-    }
+    for (uint64_t j = 0; j < n; ++j) put_bits(msg + sm_off, j * (uint64_t)m, m, sm[j]);
 
     /* payload <- { exp[k] | bitmap[k] = 1 } in block order (no entropy stage, as in ora_encode) */
     uint64_t plen = 0;
@@ -342,7 +357,10 @@ int ora_encode_hashed(const void* w, uint64_t* hash_cache, uint64_t n, int dtype
         if (!((msg[k >> 3] >> (k & 7)) & 1u)) continue;
         uint64_t lo = k * block;
         uint64_t hi = lo + block < n ? lo + block : n;
-        for (uint64_t j = lo; j < hi; ++j) msg[pay_off + plen++] = exp[j];
+        uint64_t nbytes = ora_block_payload_bytes(hi - lo, dtype);
+        memset(msg + pay_off + plen, 0, nbytes);
+        for (uint64_t j = lo; j < hi; ++j) put_bits(msg + pay_off + plen, (j - lo) * (uint64_t)e, e, exp[j]);
+        plen += nbytes;
         ++nchg;
     }
     *payload_bytes = plen;
@@ -363,29 +381,23 @@ int ora_encode_hashed(const void* w, uint64_t* hash_cache, uint64_t n, int dtype
  */
 int ora_decode(const uint8_t* msg, uint8_t* cache_r, uint64_t n, int dtype, uint32_t block, void* w_out) {
     if (n == 0) return 0;
-    int m = ora_m(dtype);
+    int m = ora_m(dtype), e = ora_e(dtype);
     uint64_t nb = ora_num_blocks(n, block);
     uint64_t sm_off = ora_sm_offset(n, block);
     uint64_t pay_off = ora_payload_offset(n, dtype, block);
 
-    uint64_t j_pay = 0; /* read position in newExp */
+    uint64_t j_pay = 0; /* read position (bytes) in newExp */
     for (uint64_t k = 0; k < nb; ++k) {
         if (!((msg[k >> 3] >> (k & 7)) & 1u)) continue;
         uint64_t lo = k * block;
         uint64_t hi = lo + block < n ? lo + block : n;
-        for (uint64_t j = lo; j < hi; ++j) cache_r[j] = msg[pay_off + j_pay++];
+        for (uint64_t j = lo; j < hi; ++j) cache_r[j] = (uint8_t)get_bits(msg + pay_off + j_pay, (j - lo) * (uint64_t)e, e);
+        j_pay += ora_block_payload_bytes(hi - lo, dtype);
     }
 
     uint32_t* sm = (uint32_t*)malloc(n * sizeof(uint32_t));
     if (!sm) return -1;
-    for (uint64_t j = 0; j < n; ++j) {
-        if (m == 8) {
-            sm[j] = msg[sm_off + j];
-        } else {
-            sm[j] = (uint32_t)msg[sm_off + 3 * j] | ((uint32_t)msg[sm_off + 3 * j + 1] << 8) |
-                    ((uint32_t)msg[sm_off + 3 * j + 2] << 16);
-        }
-    }
+    for (uint64_t j = 0; j < n; ++j) sm[j] = get_bits(msg + sm_off, j * (uint64_t)m, m);
     ora_merge(cache_r, sm, n, dtype, w_out);
     free(sm);
     return 0;
@@ -415,7 +427,7 @@ double ora_gain(uint64_t n, int dtype, uint32_t block, double q, int world, doub
                 const double* table_bytes, const double* table_secs, int n_points, double t_hash, double t_cmp,
                 double t_decmp, int overlapped) {
     double S = (double)n * ora_b(dtype) / 8.0;
-    double S_e = (double)n; /* 8 exponent bits per value */
+    double S_e = (double)n * ora_e(dtype) / 8.0; /* exponent bits per value / 8 */
     double S_sm = S - S_e;
     double S_bm = (double)ora_bitmap_bytes(n, block);
     double sent = S_sm + S_bm + q * S_e;

@@ -17,6 +17,7 @@ import numpy as np
 
 BF16 = 0
 FP32 = 1
+FP16 = 2
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "ciera_oracle.c")
@@ -42,6 +43,7 @@ def lib() -> ctypes.CDLL:
             ("ora_num_blocks", [u64, u32]),
             ("ora_bitmap_bytes", [u64, u32]),
             ("ora_sm_bytes", [u64, i32]),
+            ("ora_block_payload_bytes", [u64, i32]),
             ("ora_sm_offset", [u64, u32]),
             ("ora_payload_offset", [u64, i32, u32]),
             ("ora_message_capacity", [u64, i32, u32]),
@@ -68,7 +70,7 @@ def lib() -> ctypes.CDLL:
 
 
 def _wdtype(dtype: int):
-    return np.uint16 if dtype == BF16 else np.uint32
+    return np.uint32 if dtype == FP32 else np.uint16
 
 
 def _ptr(a: np.ndarray) -> int:
@@ -86,6 +88,10 @@ def bitmap_bytes(n, block):
 
 def sm_bytes(n, dtype):
     return int(lib().ora_sm_bytes(n, dtype))
+
+
+def block_payload_bytes(length, dtype):
+    return int(lib().ora_block_payload_bytes(length, dtype))
 
 
 def sm_offset(n, block):

@@ -10,7 +10,7 @@ import numpy as np
 import pytest
 import torch
 
-from helpers import BF16, FP32, ieee_fields, parse_golden, shadow_blocks
+from helpers import BF16, FP16, FP32, FORMAT, ieee_fields, pack_fields, parse_golden, shadow_blocks, shadow_blocks_packed
 from paper_2609_04609_b200 import workloads as wl
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
@@ -20,7 +20,7 @@ GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
 
 def _check_fields(oracle, bits, dtype):
-    p = 7 if dtype == BF16 else 23
+    p = FORMAT[dtype][1]
     sign, E, M = ieee_fields(bits, dtype)
     exp, sm = oracle.split(bits, dtype)
     assert np.array_equal(exp.astype(np.int64), E), "exponent field differs from the IEEE definition"
@@ -35,6 +35,13 @@ def _check_fields(oracle, bits, dtype):
 def test_split_bf16_every_pattern_matches_ieee_definition(oracle):
     bits = np.arange(65536, dtype=np.uint16)
     _check_fields(oracle, bits, BF16)
+
+
+def test_split_fp16_every_pattern_matches_ieee_definition(oracle):
+    bits = np.arange(65536, dtype=np.uint16)
+    _check_fields(oracle, bits, FP16)
+    exp, _ = oracle.split(bits, FP16)
+    assert exp.max() == 31
 
 
 def test_split_fp32_random_and_special_patterns_match_ieee_definition(oracle):
@@ -53,12 +60,12 @@ def test_split_fp32_random_and_special_patterns_match_ieee_definition(oracle):
 
 
 @pytest.mark.parametrize("name", ["bf16_worked_example.txt", "fp32_worked_example.txt",
-                                  "small_block_worked_example.txt"])
+                                  "small_block_worked_example.txt", "fp16_worked_example.txt"])
 def test_hand_worked_examples(oracle, name):
     for st in parse_golden(os.path.join(GOLDEN, name)):
-        dtype = BF16 if st["dtype"][0] == "bf16" else FP32
+        dtype = {"bf16": BF16, "fp32": FP32, "fp16": FP16}[st["dtype"][0]]
         block = int(st["block"][0])
-        w = np.array([int(x, 16) for x in st["weights"]], np.uint16 if dtype == BF16 else np.uint32)
+        w = np.array([int(x, 16) for x in st["weights"]], np.uint32 if dtype == FP32 else np.uint16)
         hexb = lambda key: np.array([int(x, 16) for x in st.get(key, [])], np.uint8)
         cache = hexb("cache_before").copy()
         n = w.size
@@ -335,3 +342,69 @@ def test_gain_sign_cases(oracle):
     # a fast link makes every gain non-positive once decompression costs anything real
     fast = dict(kw, beta=1e13, alpha=0.0)
     assert oracle.gain(q=0.22, t_decmp=5e-6, overlapped=True, **fast) < 0
+
+
+# ------------------------------------------------------------------ fp16: packed sections
+
+
+def test_exhaustive_fp16_patterns_times_cache_values(oracle):
+    """All 32 cache values x all 65 536 fp16 patterns: the complete per-value map through encode and
+    decode, against numerically derived fields and a numpy restatement of the bit packing."""
+    pat = np.arange(65536, dtype=np.uint16)
+    sign, E, M = ieee_fields(pat, FP16)
+    w = np.tile(pat, 32)
+    exp_true = np.tile(E.astype(np.uint8), 32)
+    cache0 = np.repeat(np.arange(32, dtype=np.uint8), 65536)
+    block = 64
+    n = w.size
+    cache_s = cache0.copy()
+    msg, wire, pay, chg = oracle.encode(w, cache_s, FP16, block)
+    bitmap, payload, cache_after, chg_mask = shadow_blocks_packed(exp_true, cache0, block, 5)
+    sm_off, pay_off = oracle.sm_offset(n, block), oracle.payload_offset(n, FP16, block)
+    assert np.array_equal(msg[: bitmap.size], bitmap)
+    assert np.array_equal(msg[pay_off:], payload) and pay == payload.size and chg == int(chg_mask.sum())
+    assert np.array_equal(cache_s, cache_after) and np.array_equal(cache_s, exp_true)
+    # sm = sign << 10 | mantissa from the numeric fields (NaN payloads are covered by the round trip)
+    ok = M >= 0
+    sm_true = np.where(ok, sign << 10 | np.where(ok, M, 0), 0)
+    got = msg[sm_off : sm_off + 65536 * 11 // 8]
+    want = pack_fields(sm_true, 11)
+    # compare value by value where the mantissa has a numeric definition
+    got_fields = np.unpackbits(got, bitorder="little").reshape(65536, 11)
+    want_fields = np.unpackbits(want, bitorder="little").reshape(65536, 11)
+    assert np.array_equal(got_fields[ok], want_fields[ok])
+    cache_r = cache0.copy()
+    assert np.array_equal(oracle.decode(msg, cache_r, FP16, block), w)
+    assert np.array_equal(cache_r, exp_true)
+
+
+def test_fp16_byte_count_and_layout_over_ragged_sizes(oracle):
+    """S_{s+m} = ceil(11 N / 8), every changed block ceil(5 L / 8) bytes, capacity = all blocks changed."""
+    rng = np.random.default_rng(23)
+    for n, block in [(1, 64), (5, 2), (7, 8), (63, 64), (65, 64), (1000, 128), (4097, 512), (12345, 4096), (33, 1),
+                     (8193, 32), (100, 3)]:
+        w_prev = rng.integers(0, 1 << 16, size=n, dtype=np.uint64).astype(np.uint16)
+        w = w_prev.copy()
+        flip = rng.random(n) < 0.05
+        w[flip] = rng.integers(0, 1 << 16, size=int(flip.sum()), dtype=np.uint64).astype(np.uint16)
+        cache0 = oracle.cache_init(w_prev, n, FP16)
+        cache = cache0.copy()
+        msg, wire, pay, chg = oracle.encode(w, cache, FP16, block)
+        _, E, _ = ieee_fields(w, FP16)
+        bitmap, payload, cache_after, chg_mask = shadow_blocks_packed(E.astype(np.uint8), cache0, block, 5)
+        nb = -(-n // block)
+        lens = np.minimum(block, n - np.arange(nb) * block)
+        assert pay == int((-(-(lens[chg_mask] * 5) // 8)).sum()) == payload.size
+        s_bm, s_sm = -(-nb // 8), -(-(n * 11) // 8)
+        assert oracle.paper_bytes(n, FP16, block, pay) == s_sm + s_bm + pay
+        sm_off = -(-s_bm // 16) * 16
+        pay_off = sm_off + -(-s_sm // 16) * 16
+        assert (oracle.sm_offset(n, block), oracle.payload_offset(n, FP16, block)) == (sm_off, pay_off)
+        assert wire == pay_off + pay and msg.size == wire
+        assert oracle.message_capacity(n, FP16, block) == pay_off + int((-(-(lens * 5) // 8)).sum())
+        assert np.array_equal(msg[:s_bm], bitmap) and np.array_equal(msg[pay_off:], payload)
+        assert not msg[s_bm:sm_off].any() and not msg[sm_off + s_sm : pay_off].any()
+        assert np.array_equal(cache, cache_after)
+        cache_r = cache0.copy()
+        assert np.array_equal(oracle.decode(msg, cache_r, FP16, block), w)
+        assert np.array_equal(cache_r, cache_after)
