@@ -74,7 +74,13 @@ typedef enum ciera_status {
 
 typedef enum ciera_dtype {
     CIERA_BF16 = 0, /* b = 16: 1 sign, 8 exponent, 7 mantissa bits  -> m = 8  */
-    CIERA_FP32 = 1  /* b = 32: 1 sign, 8 exponent, 23 mantissa bits -> m = 24 */
+    CIERA_FP32 = 1, /* b = 32: 1 sign, 8 exponent, 23 mantissa bits -> m = 24 */
+    CIERA_FP16 = 2  /* b = 16: 1 sign, 5 exponent, 10 mantissa bits -> m = 11 (IEEE binary16).  On the
+                       wire its exponents take 5 bits and its sign-plus-mantissa 11 bits each, packed
+                       without gaps (value j of a section at bits [j*w, (j+1)*w), bit i of a section =
+                       byte i >> 3, bit i & 7); every changed block of the payload starts on a byte
+                       boundary; the caches still hold one byte per value.  Blocks of 32 values and
+                       more; no hashed sender, no entropy stage, no ciera_encode_noalloc. */
 } ciera_dtype;
 
 /* One unit = one shard of one tensor.  All offsets are in BYTES from the base pointer of the

@@ -17,7 +17,8 @@ from .workloads import UNIT_DTYPE
 
 BF16 = 0
 FP32 = 1
-DTYPE_CODES = {"bf16": BF16, "fp32": FP32}
+FP16 = 2
+DTYPE_CODES = {"bf16": BF16, "fp32": FP32, "fp16": FP16}
 
 OK = 0
 ERR_INVALID_ARG = -1

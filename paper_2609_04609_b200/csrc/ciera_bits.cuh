@@ -344,6 +344,41 @@ __device__ __forceinline__ int piece_valid(uint32_t start, uint32_t nv) {
     return start >= nv ? 0 : (int)min((uint32_t)Piece<DT>::kValues, nv - start);
 }
 
+// Block flags of a tile from the vote bits "my piece differs" (one warp).  `pl2` = log2 of the
+// values per piece.  Fills bm (one bit per block of the tile) and pre (set bits before each word);
+// returns the number of changed blocks of the tile.
+__device__ __forceinline__ uint32_t build_block_bitmap(const uint32_t* ballot, uint32_t* bm, uint16_t* pre,
+                                                       uint32_t log2b, uint32_t pl2, uint32_t lane) {
+    const uint32_t gl2 = log2b - pl2;           // log2(pieces per block)
+    const uint32_t nbt = kTileValues >> log2b;  // blocks of a full tile
+    uint32_t run = 0;
+    for (uint32_t base = 0; base < nbt; base += 32) {
+        const uint32_t i = base + lane;
+        bool f = false;
+        if (i < nbt) {
+            const uint32_t g0 = i << gl2;
+            if (gl2 <= 5) {
+                const uint32_t width = 1u << gl2;
+                const uint32_t m = width == 32 ? 0xffffffffu : ((1u << width) - 1u);
+                f = ((ballot[g0 >> 5] >> (g0 & 31)) & m) != 0;
+            } else {
+                const uint32_t nw = 1u << (gl2 - 5);
+                uint32_t acc = 0;
+                for (uint32_t j = 0; j < nw; ++j) acc |= ballot[(g0 >> 5) + j];
+                f = acc != 0;
+            }
+        }
+        const uint32_t word = __ballot_sync(0xffffffffu, f);
+        if (lane == 0) {
+            bm[base >> 5] = word;
+            pre[base >> 5] = (uint16_t)run;
+        }
+        run += __popc(word);
+    }
+    __syncwarp();
+    return run;
+}
+
 __device__ __forceinline__ TileDesc load_tile_desc(const TileDesc* t) {
     const uint4* p = reinterpret_cast<const uint4*>(t);
     uint4 a = __ldg(p), b = __ldg(p + 1), c = __ldg(p + 2);

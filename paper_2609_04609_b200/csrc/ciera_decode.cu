@@ -751,6 +751,9 @@ extern "C" int ciera_decode(const ciera_plan* p, const void* messages_dev, void*
         int rc = check_launch();
         if (rc) return rc;
     }
+    if (p->dtype == CIERA_FP16)
+        return fp16_decode(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,
+                           (const uint32_t*)workspace_dev, status_dev, s);
     const bool fine = is_fine(p->log2b);
     if (p->dtype == CIERA_BF16)
         return fine ? launch_decode<CIERA_BF16, true>(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,

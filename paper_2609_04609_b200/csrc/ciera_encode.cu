@@ -154,41 +154,6 @@ struct TileWalk {
     }
 };
 
-// Block flags of a tile from the vote bits "my piece differs" (one warp).  `pl2` = log2 of the
-// values per piece.  Fills bm (one bit per block of the tile) and pre (set bits before each word);
-// returns the number of changed blocks of the tile.
-__device__ __forceinline__ uint32_t build_block_bitmap(const uint32_t* ballot, uint32_t* bm, uint16_t* pre,
-                                                       uint32_t log2b, uint32_t pl2, uint32_t lane) {
-    const uint32_t gl2 = log2b - pl2;           // log2(pieces per block)
-    const uint32_t nbt = kTileValues >> log2b;  // blocks of a full tile
-    uint32_t run = 0;
-    for (uint32_t base = 0; base < nbt; base += 32) {
-        const uint32_t i = base + lane;
-        bool f = false;
-        if (i < nbt) {
-            const uint32_t g0 = i << gl2;
-            if (gl2 <= 5) {
-                const uint32_t width = 1u << gl2;
-                const uint32_t m = width == 32 ? 0xffffffffu : ((1u << width) - 1u);
-                f = ((ballot[g0 >> 5] >> (g0 & 31)) & m) != 0;
-            } else {
-                const uint32_t nw = 1u << (gl2 - 5);
-                uint32_t acc = 0;
-                for (uint32_t j = 0; j < nw; ++j) acc |= ballot[(g0 >> 5) + j];
-                f = acc != 0;
-            }
-        }
-        const uint32_t word = __ballot_sync(0xffffffffu, f);
-        if (lane == 0) {
-            bm[base >> 5] = word;
-            pre[base >> 5] = (uint16_t)run;
-        }
-        run += __popc(word);
-    }
-    __syncwarp();
-    return run;
-}
-
 // Fine blocks: the consumers have written the block flags themselves; fills pre (set bits before
 // each word) and returns the number of changed blocks of the tile (one warp).
 __device__ __forceinline__ uint32_t scan_block_bitmap(const uint32_t* bm, uint16_t* pre, uint32_t log2b, uint32_t lane) {
@@ -744,6 +709,9 @@ extern "C" int ciera_encode(const ciera_plan* p, const void* weights_dev, void* 
     if (misaligned16(weights_dev) || misaligned16(sender_cache_dev) || misaligned16(messages_dev) ||
         misaligned16(workspace_dev) || ((uintptr_t)wire_bytes_dev & 7u) || ((uintptr_t)changed_blocks_dev & 3u))
         return CIERA_ERR_MISALIGNED;
+    if (p->dtype == CIERA_FP16)  // three plain launches; the scratch needs no clearing
+        return fp16_encode(p, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev, changed_blocks_dev,
+                           workspace_dev, s);
     // scratch = one look-back status word per tile, then the unit counter; all of it starts at zero
     e = cudaMemsetAsync(workspace_dev, 0, sizeof(unsigned long long) * nt + 16, s);
     if (e != cudaSuccess) return record_cuda_error(e);
@@ -793,6 +761,7 @@ extern "C" int ciera_encode_noalloc(const ciera_plan* p, const void* weights_dev
     if (!p->tiles.empty() && !p->tiles_dev) return CIERA_ERR_NOT_BOUND;
     const uint32_t nt = (uint32_t)p->tiles.size();
     if (nt > CIERA_NOALLOC_MAX_TILES) return CIERA_ERR_TOO_LARGE;
+    if (p->dtype == CIERA_FP16) return CIERA_ERR_UNSUPPORTED;
     if (p->n_units == 0) return CIERA_OK;
     if (!wire_bytes_dev || !changed_blocks_dev) return CIERA_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)stream;

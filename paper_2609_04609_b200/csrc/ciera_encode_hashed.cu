@@ -21,17 +21,13 @@
 // cache, plus 16 bytes per block of HashCache traffic; the price is about 40 integer instructions
 // per 8 values for the two hashes.
 #include "ciera_bits.cuh"
+#include "ciera_multipass.cuh"
 
 namespace ciera {
 
 constexpr uint64_t kGamma = 0x9E3779B97F4A7C15ull;
 constexpr uint64_t kSeed1 = 0x0000000000000000ull;
 constexpr uint64_t kSeed2 = 0x6A09E667F3BCC908ull;
-// Scratch record of a tile: 16 words of block flags, the number of set flags, and the number of
-// set flags in the unit's earlier tiles.
-constexpr uint32_t kFlagWords = kBitmapWords;
-constexpr uint32_t kRecCount = kFlagWords, kRecPrefix = kFlagWords + 1, kRecWords = kFlagWords + 2;
-
 __device__ __forceinline__ uint64_t mix64(uint64_t z) {
     z ^= z >> 30;
     z *= 0xBF58476D1CE4E5B9ull;
@@ -137,84 +133,6 @@ hashed_scan_kernel(const TileDesc* __restrict__ tiles, const unsigned long long*
     if (tid == 0) ws[(size_t)tile * kRecWords + kRecCount] = s_count;
 }
 
-__device__ __forceinline__ uint32_t block_flag(const uint32_t* ws, uint32_t first_tile, uint32_t log2b, uint64_t k) {
-    const uint32_t nbt = kTileValues >> log2b;
-    const uint64_t t = k / nbt;
-    const uint32_t r = (uint32_t)(k % nbt);
-    return (ws[(size_t)(first_tile + t) * kRecWords + (r >> 5)] >> (r & 31u)) & 1u;
-}
-
-// One thread block per unit: payload offset of every tile, bitmap bytes, pads, reported totals.
-__global__ void __launch_bounds__(256)
-hashed_unit_kernel(const TileDesc* __restrict__ tiles, const uint32_t* __restrict__ unit_first, uint32_t log2b,
-                   uint32_t sm_bytes_per_value, uint8_t* msgs, uint32_t* ws,
-                   unsigned long long* __restrict__ wire_bytes, uint32_t* __restrict__ changed_blocks) {
-    __shared__ uint32_t s_warp[8];
-    __shared__ uint32_t s_carry;
-    const uint32_t unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
-    const uint32_t first = unit_first[unit];
-    if (first == 0xffffffffu) {  // a unit without values
-        if (tid == 0) {
-            wire_bytes[unit] = 0;
-            changed_blocks[unit] = 0;
-        }
-        return;
-    }
-    const TileDesc td0 = load_tile_desc(tiles + first);
-    const uint64_t N = td0.n_unit;
-    const uint32_t B = 1u << log2b;
-    const uint32_t nbt = kTileValues >> log2b;
-    const uint64_t nb = num_blocks(N, log2b);
-    uint8_t* msg = msgs + td0.msg_off;
-    if (tid == 0) s_carry = 0;
-    __syncthreads();
-    for (uint32_t j0 = 0; j0 < td0.n_tiles_unit; j0 += 256u) {
-        const uint32_t j = j0 + tid;
-        const uint32_t cnt = j < td0.n_tiles_unit ? ws[(size_t)(first + j) * kRecWords + kRecCount] : 0u;
-        uint32_t incl = cnt;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
-            if ((int)lane >= o) incl += t;
-        }
-        if (lane == 31) s_warp[warp] = incl;
-        __syncthreads();
-        uint32_t wbase = 0;
-        for (uint32_t w = 0; w < warp; ++w) wbase += s_warp[w];
-        const uint32_t carry = s_carry;
-        if (j < td0.n_tiles_unit) ws[(size_t)(first + j) * kRecWords + kRecPrefix] = carry + wbase + incl - cnt;
-        __syncthreads();
-        if (tid == 255) s_carry = carry + wbase + incl;
-        __syncthreads();
-    }
-    const uint64_t smoff = sm_offset(N, log2b);
-    const uint64_t payoff = smoff + pad16(N * sm_bytes_per_value);
-    if (tid == 0) {
-        const uint32_t total = s_carry;  // changed blocks of the unit
-        uint64_t bytes = (uint64_t)total << log2b;
-        const uint32_t rem = (uint32_t)(N & (B - 1u));
-        if (rem && block_flag(ws, first, log2b, nb - 1)) bytes -= (B - rem);  // a changed short last block
-        wire_bytes[unit] = payoff + bytes;
-        changed_blocks[unit] = total;
-    }
-    // bitmap bytes (bit k of the unit = block k, LSB first), then the two pads
-    const uint64_t bm_bytes = bitmap_bytes(N, log2b);
-    for (uint64_t i = tid; i < bm_bytes; i += 256u) {
-        uint32_t byte = 0;
-        if (nbt >= 32) {  // the byte's eight flags lie in one word of one tile
-            const uint64_t k = 8 * i;
-            const uint32_t r = (uint32_t)(k % nbt);
-            byte = (ws[(size_t)(first + k / nbt) * kRecWords + (r >> 5)] >> (r & 31u)) & 0xFFu;
-        } else {
-            for (uint32_t r = 0; r < 8; ++r)
-                if (8 * i + r < nb) byte |= block_flag(ws, first, log2b, 8 * i + r) << r;
-        }
-        msg[i] = (uint8_t)byte;
-    }
-    for (uint64_t b = bm_bytes + tid; b < smoff; b += 256u) msg[b] = 0;
-    for (uint64_t b = smoff + N * sm_bytes_per_value + tid; b < payoff; b += 256u) msg[b] = 0;
-}
-
 // One thread block per tile, every warp on its own (no barrier): exponents of the flagged blocks to
 // the payload.  A warp first looks at the flags of its own pieces and leaves if none is set;
 // otherwise it works out the ranks from the tile's scratch record with shuffles and fetches the
@@ -289,6 +207,7 @@ static int check_hashed_plan(const ciera_plan* p) {
     if (!p) return CIERA_ERR_INVALID_ARG;
     if (!p->tiles.empty() && !p->tiles_dev) return CIERA_ERR_NOT_BOUND;
     if (is_fine(p->log2b)) return CIERA_ERR_UNSUPPORTED;  // blocks of fewer than 16 values: exact comparison only
+    if (p->dtype == CIERA_FP16) return CIERA_ERR_UNSUPPORTED;
     return CIERA_OK;
 }
 
@@ -331,7 +250,6 @@ extern "C" int ciera_encode_hashed(const ciera_plan* p, const void* weights_dev,
     // scratch: one record of 18 words per tile; the scan pass writes every record's flags and count,
     // the unit pass its payload offset
     uint32_t* ws = (uint32_t*)workspace_dev;
-    const uint32_t smb = p->dtype == CIERA_BF16 ? 1u : 3u;
     if (nt != 0) {
         if (p->dtype == CIERA_BF16)
             hashed_scan_kernel<CIERA_BF16, false><<<nt, kThreads, 0, s>>>(
@@ -345,8 +263,9 @@ extern "C" int ciera_encode_hashed(const ciera_plan* p, const void* weights_dev,
         rc = check_launch();
         if (rc) return rc;
     }
-    hashed_unit_kernel<<<p->n_units, 256, 0, s>>>(p->tiles_dev, p->unit_first_dev, p->log2b, smb, (uint8_t*)messages_dev,
-                                                  ws, (unsigned long long*)wire_bytes_dev, changed_blocks_dev);
+    multipass_unit_kernel<<<p->n_units, 256, 0, s>>>(p->tiles_dev, p->unit_first_dev, p->log2b, p->dtype,
+                                                     (uint8_t*)messages_dev, ws, (unsigned long long*)wire_bytes_dev,
+                                                     changed_blocks_dev);
     count_launch();
     rc = check_launch();
     if (rc) return rc;

@@ -737,6 +737,7 @@ static int check_entropy_args(const ciera_plan* p, const void* messages_dev, con
                               const void* scratch_dev) {
     if (!p) return CIERA_ERR_INVALID_ARG;
     if (!p->tiles.empty() && !p->tiles_dev) return CIERA_ERR_NOT_BOUND;
+    if (p->dtype == CIERA_FP16) return CIERA_ERR_UNSUPPORTED;
     if (p->tiles.empty()) return CIERA_OK;
     if (!messages_dev || !wire_bytes_dev || !scratch_dev) return CIERA_ERR_INVALID_ARG;
     if (misaligned16(messages_dev) || misaligned16(scratch_dev) || ((uintptr_t)wire_bytes_dev & 7u))

@@ -22,9 +22,8 @@ int check_launch() {
     return CIERA_OK;
 }
 
-static bool valid_dtype(int dtype) { return dtype == CIERA_BF16 || dtype == CIERA_FP32; }
-static uint32_t sm_bytes_of(int dtype) { return dtype == CIERA_BF16 ? 1u : 3u; }
-static uint32_t value_bytes_of(int dtype) { return dtype == CIERA_BF16 ? 2u : 4u; }
+static bool valid_dtype(int dtype) { return dtype == CIERA_BF16 || dtype == CIERA_FP32 || dtype == CIERA_FP16; }
+static uint32_t value_bytes_of(int dtype) { return dtype == CIERA_FP32 ? 4u : 2u; }
 
 // log2 of a power of two, or -1.
 static int exact_log2(uint32_t x) {
@@ -48,18 +47,21 @@ extern "C" size_t ciera_sm_offset(uint64_t n, uint32_t block) {
 
 extern "C" size_t ciera_payload_offset(uint64_t n, int dtype, uint32_t block) {
     if (block == 0 || !valid_dtype(dtype)) return 0;
-    return ciera_sm_offset(n, block) + (size_t)pad16(n * sm_bytes_of(dtype));
+    return ciera_sm_offset(n, block) + (size_t)pad16(sm_section_bytes(n, dtype));
 }
 
 extern "C" size_t ciera_message_capacity(uint64_t n, int dtype, uint32_t block) {
     if (n == 0 || block == 0 || !valid_dtype(dtype)) return 0;
-    return ciera_payload_offset(n, dtype, block) + (size_t)n;
+    // every block changed: full blocks and the (possibly short) last one
+    const uint64_t nb = (n + block - 1) / block;
+    return ciera_payload_offset(n, dtype, block) +
+           (size_t)((nb - 1) * block_payload_bytes(block, dtype) + block_payload_bytes(n - (nb - 1) * block, dtype));
 }
 
 extern "C" size_t ciera_message_bytes(uint64_t n, int dtype, uint32_t block, uint64_t payload_bytes) {
     if (block == 0 || !valid_dtype(dtype)) return 0;
     uint64_t nb = (n + block - 1) / block;
-    return (size_t)(n * sm_bytes_of(dtype) + (nb + 7) / 8 + payload_bytes);
+    return (size_t)(sm_section_bytes(n, dtype) + (nb + 7) / 8 + payload_bytes);
 }
 
 // ---------------------------------------------------------------------------------- plan
@@ -93,6 +95,7 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
     if (block == 0) return CIERA_ERR_INVALID_ARG;
     int l2 = exact_log2(block);
     if (l2 < 0 || block < CIERA_MIN_BLOCK || block > CIERA_MAX_BLOCK) return CIERA_ERR_UNSUPPORTED;
+    if (dtype == CIERA_FP16 && block < 32) return CIERA_ERR_UNSUPPORTED;
 
     uint64_t n_tiles = 0, total = 0;
     for (uint32_t u = 0; u < n_units; ++u) {
@@ -142,7 +145,9 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
             t.n_tiles_unit = nt;
             p->tiles.push_back(t);
         }
-        const bool needs_prefix = is_fine(p->log2b) ? nt > 1 : (un.n_values + block - 1) / block > kDecodeDirectBlocks;
+        const bool needs_prefix = (is_fine(p->log2b) || dtype == CIERA_FP16)
+                                      ? nt > 1
+                                      : (un.n_values + block - 1) / block > kDecodeDirectBlocks;
         if (needs_prefix) p->long_units.push_back(first);
     };
     for (uint32_t u : shorts) {
@@ -203,8 +208,9 @@ extern "C" const void* ciera_plan_host_image(const ciera_plan* p) { return p ? p
 
 extern "C" size_t ciera_plan_workspace_bytes(const ciera_plan* p) {
     if (!p) return 0;
-    // one look-back status word per tile + the ticket counter
-    return p->tiles.size() * sizeof(unsigned long long) + 16;
+    // one look-back status word per tile + the ticket counter; fp16: a record of 18 words per tile
+    const size_t per_tile = p->dtype == CIERA_FP16 ? 18 * sizeof(uint32_t) : sizeof(unsigned long long);
+    return p->tiles.size() * per_tile + 16;
 }
 
 extern "C" size_t ciera_plan_hash_cache_bytes(const ciera_plan* p) { return p ? (size_t)p->total_blocks * 16 : 0; }
@@ -275,7 +281,7 @@ static int gain_of(const ciera_gain_in* in, double* g_out) {
     }
     const double n = (double)in->n_values;
     const double s_full = n * value_bytes_of(in->dtype);
-    const double s_exp = n;  // 8 exponent bits per value
+    const double s_exp = n * exp_bits_of(in->dtype) / 8.0;  // exponent bits per value / 8
     const double s_sm = s_full - s_exp;
     const uint64_t blocks = (in->n_values + in->block - 1) / in->block;
     const double s_bm = (double)((blocks + 7) / 8);

@@ -75,6 +75,17 @@ __host__ __device__ inline uint64_t payload_offset(uint64_t n, uint32_t sm_bytes
     return sm_offset(n, log2b) + pad16(n * sm_bytes_per_value);
 }
 
+// The same sizes by precision, for code that also handles fp16 (5 exponent bits and 11
+// sign-plus-mantissa bits per value, packed without gaps; every changed block of the payload starts
+// on a byte boundary).
+__host__ __device__ inline uint32_t sm_bits_of(int dtype) { return dtype == CIERA_FP32 ? 24u : dtype == CIERA_FP16 ? 11u : 8u; }
+__host__ __device__ inline uint32_t exp_bits_of(int dtype) { return dtype == CIERA_FP16 ? 5u : 8u; }
+__host__ __device__ inline uint64_t sm_section_bytes(uint64_t n, int dtype) { return (n * sm_bits_of(dtype) + 7) >> 3; }
+__host__ __device__ inline uint64_t block_payload_bytes(uint64_t len, int dtype) { return (len * exp_bits_of(dtype) + 7) >> 3; }
+__host__ __device__ inline uint64_t payload_offset_of(uint64_t n, int dtype, uint32_t log2b) {
+    return sm_offset(n, log2b) + pad16(sm_section_bytes(n, dtype));
+}
+
 // Units with more blocks than this get their per-tile "changed blocks before" counts from a
 // prefix kernel at decode time; shorter ones read them straight from the bitmap.  With fine
 // blocks every unit of more than one tile goes through the prefix kernel.
@@ -136,6 +147,12 @@ struct ciera_plan {
 };
 
 namespace ciera {
+// fp16 takes kernels of its own (ciera_fp16.cu)
+int fp16_cache_fill(const ciera_plan* p, void* cache_dev, const void* weights_dev, cudaStream_t s);
+int fp16_encode(const ciera_plan* p, const void* weights_dev, void* sender_cache_dev, void* messages_dev,
+                uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* workspace_dev, cudaStream_t s);
+int fp16_decode(const ciera_plan* p, const void* messages_dev, void* receiver_cache_dev, void* weights_out_dev,
+                const uint64_t* wire_bytes_dev, const uint32_t* ws_prefix, int32_t* status_dev, cudaStream_t s);
 int record_cuda_error(cudaError_t e);          // stores e for ciera_last_cuda_error, returns CIERA_ERR_CUDA
 void count_launch();                           // launch accounting
 int check_launch();                            // cudaGetLastError -> status

@@ -162,6 +162,7 @@ static int cache_fill(const ciera_plan* p, void* cache_dev, const void* weights_
     const uint32_t nt = (uint32_t)p->tiles.size();
     if (nt == 0) return CIERA_OK;
     cudaStream_t s = (cudaStream_t)stream;
+    if (p->dtype == CIERA_FP16) return fp16_cache_fill(p, cache_dev, weights_dev, s);
     if (p->dtype == CIERA_BF16)
         cache_fill_kernel<CIERA_BF16><<<nt, kThreads, 0, s>>>(p->tiles_dev, (const uint8_t*)weights_dev, (uint8_t*)cache_dev);
     else
@@ -198,7 +199,7 @@ extern "C" int ciera_transport(const ciera_plan* p, const void* src_messages_dev
     const uint32_t want = (nt + kCopyThreads / 32 - 1) / (kCopyThreads / 32);
     const uint32_t grid = want < (uint32_t)limit ? want : (uint32_t)limit;
     transport_kernel<<<grid, kCopyThreads, 0, (cudaStream_t)stream>>>(
-        p->tiles_dev, nt, transport_chunk_bytes(p->dtype == CIERA_BF16 ? 1u : 3u, p->log2b), (const uint8_t*)src_messages_dev, (uint8_t*)dst_messages_dev,
+        p->tiles_dev, nt, transport_chunk_bytes(p->dtype == CIERA_FP32 ? 3u : 1u, p->log2b), (const uint8_t*)src_messages_dev, (uint8_t*)dst_messages_dev,
         (const unsigned long long*)wire_bytes_dev, ticket);
     count_launch();
     return check_launch();

@@ -33,8 +33,8 @@ UNIT_DTYPE = np.dtype(
     ]
 )
 
-TORCH_DTYPES = {"bf16": torch.bfloat16, "fp32": torch.float32}
-VALUE_BYTES = {"bf16": 2, "fp32": 4}
+TORCH_DTYPES = {"bf16": torch.bfloat16, "fp32": torch.float32, "fp16": torch.float16}
+VALUE_BYTES = {"bf16": 2, "fp32": 4, "fp16": 2}
 
 
 def _align(x: int, a: int) -> int:
@@ -150,7 +150,7 @@ def step_clustered(w: torch.Tensor, gen: torch.Generator, f: float = 0.22, seg: 
 
 def as_bits(w: torch.Tensor) -> np.ndarray:
     """Raw bit patterns on the host: uint16 for bf16, uint32 for fp32."""
-    if w.dtype == torch.bfloat16:
+    if w.dtype in (torch.bfloat16, torch.float16):
         return w.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
     if w.dtype == torch.float32:
         return w.detach().cpu().contiguous().view(torch.int32).numpy().view(np.uint32)
@@ -169,34 +169,35 @@ def inject_exponent_changes(w: torch.Tensor, gen: torch.Generator, c: float, seg
     """Next iterate with an exact-rate exponent change.
 
     A Bernoulli(c) mask over values (``seg == 0``) or over ``seg``-aligned segments
-    (``seg > 0``, every value of a hit segment changes) selects the values whose 8-bit
-    exponent field moves by +-1 (kept inside 1..254, and always moving); every value gets
+    (``seg > 0``, every value of a hit segment changes) selects the values whose exponent
+    field moves by +-1 (kept inside 1..254, or 1..30 for fp16, and always moving); every value gets
     a fresh random mantissa; signs are kept.
     """
     n = w.numel()
     dev = w.device
-    if w.dtype == torch.bfloat16:
+    if w.dtype in (torch.bfloat16, torch.float16):
         bits = w.view(torch.int16).to(torch.int32) & 0xFFFF
-        mant_bits, total = 7, 16
+        mant_bits, total = (7, 16) if w.dtype == torch.bfloat16 else (10, 16)
     else:
         bits = w.view(torch.int32).to(torch.int64) & 0xFFFFFFFF
         mant_bits, total = 23, 32
+    emax = (1 << (total - 1 - mant_bits)) - 1  # all-ones exponent field: 255, or 31 for fp16
     if seg > 0:
         nseg = -(-n // seg)
         hit = torch.rand(nseg, generator=gen, device=dev) < c
         mask = hit.repeat_interleave(seg)[:n]
     else:
         mask = torch.rand(n, generator=gen, device=dev) < c
-    e = (bits >> mant_bits) & 0xFF
+    e = (bits >> mant_bits) & emax
     up = torch.rand(n, generator=gen, device=dev) < 0.5
-    up = (up | (e <= 1)) & ~(e >= 254)
+    up = (up | (e <= 1)) & ~(e >= emax - 1)
     e_new = torch.where(mask, torch.where(up, e + 1, e - 1), e)
     mant = torch.randint(0, 1 << mant_bits, (n,), generator=gen, device=dev, dtype=bits.dtype)
     sign = (bits >> (total - 1)) & 1
     out = (sign << (total - 1)) | (e_new << mant_bits) | mant
-    if w.dtype == torch.bfloat16:
+    if total == 16:
         out = torch.where(out >= 0x8000, out - 0x10000, out).to(torch.int16)
-        return out.view(torch.bfloat16)
+        return out.view(w.dtype)
     out = torch.where(out >= 0x80000000, out - 0x100000000, out).to(torch.int32)
     return out.view(torch.float32)
 

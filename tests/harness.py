@@ -7,8 +7,8 @@ import torch
 
 from oracle import ciera_oracle as ora
 
-VB = {0: 2, 1: 4}
-WDT = {0: np.uint16, 1: np.uint32}
+VB = {0: 2, 1: 4, 2: 2}
+WDT = {0: np.uint16, 1: np.uint32, 2: np.uint16}
 
 
 class OracleTable:
