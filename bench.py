@@ -52,7 +52,7 @@ def parse_args():
     ap.add_argument("--experts", type=int, default=64)
     ap.add_argument("--shards", type=int, default=16)
     ap.add_argument("--block", type=int, default=512)
-    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32", "fp16"])
     ap.add_argument("--update", default="clustered", choices=["clustered", "adam", "inject"])
     ap.add_argument("--inject", type=float, default=0.01, help="exponent change rate of the 'inject' update model")
     ap.add_argument("--shapes", default="olmoe", choices=["olmoe", "mixed"],
@@ -244,6 +244,14 @@ def algorithmic_bytes(n_values, q, dtype, block, detect="compare"):
     reads no exponent cache but reads the weights of changed blocks twice and keeps 16 bytes per block."""
     vb, smb = (2, 1) if dtype == "bf16" else (4, 3)
     bm = 1.0 / (8 * block)
+    if dtype == "fp16":
+        # packed on the wire (11 and 5 bits per value), one byte per value in the caches; the sender
+        # reads the weights of changed blocks a second time
+        sm, ex = 11 / 8, 5 / 8
+        enc = n_values * (2 + 1 + sm + bm + q * (ex + 1 + 2))
+        tra = 2 * n_values * (sm + bm + q * ex)
+        dec = n_values * (sm + bm + (1 - q) + q * ex + 2 + q)
+        return enc, tra, dec
     if detect == "hash":
         enc = n_values * (vb + smb + bm + q * (vb + 1) + 16.0 * (1 + q) / block)
     else:
@@ -261,7 +269,7 @@ def oracle_roundtrip_units(units, w_prev, w_cur, dtype_code, block, vb, threads)
     from oracle import ciera_oracle as ora
 
     ora.build()
-    wdt = np.uint16 if dtype_code == 0 else np.uint32
+    wdt = np.uint32 if dtype_code == 1 else np.uint16
     prev = w_prev.view(wdt)
     cur = w_cur.view(wdt)
     jobs = []
@@ -298,7 +306,7 @@ def run_reference(args):
     from oracle import ciera_oracle as ora
 
     ora.build()
-    code = 0 if args.dtype == "bf16" else 1
+    code = {"bf16": 0, "fp32": 1, "fp16": 2}[args.dtype]
     vb = wl.VALUE_BYTES[args.dtype]
     shapes = layer_numels(args)
     n_units = min(args.cpu_sample_units, len(shapes) * args.shards)
@@ -456,9 +464,10 @@ def main():
 
     # ---- what was moved: change rates and the paper's byte count of the last step
     # element change rate c of the workload (reporting only): exponent fields of the two iterates of layer 0
-    shift, wdt_t = (7, torch.int16) if args.dtype == "bf16" else (23, torch.int32)
-    ea = (wa[0].view(wdt_t) >> shift) & 0xFF
-    eb = (wb[0].view(wdt_t) >> shift) & 0xFF
+    shift, wdt_t, emask = {"bf16": (7, torch.int16, 0xFF), "fp32": (23, torch.int32, 0xFF),
+                           "fp16": (10, torch.int16, 0x1F)}[args.dtype]
+    ea = (wa[0].view(wdt_t) >> shift) & emask
+    eb = (wb[0].view(wdt_t) >> shift) & emask
     element_change_rate = float((ea != eb).float().mean().item())
     del ea, eb
     changed = sum(int(c.changed_blocks.sum().item()) for c in layers)
@@ -498,7 +507,7 @@ def main():
 
         ora.build()
         code = ciera.DTYPE_CODES[args.dtype]
-        wdt = np.uint16 if code == 0 else np.uint32
+        wdt = np.uint32 if code == 1 else np.uint16
         rng = np.random.default_rng(0)
         for l in sorted(set(rng.integers(0, len(layers), 4).tolist())):
             c = layers[l]
@@ -567,7 +576,7 @@ def main():
                                  "per": "layer launch inside the two-stream timed region (kernels overlap)"},
         "serial_ms_per_step": serial_ms_per_step,
         "roofline": {
-            "bound": "hbm", "kernel": "encode_kernel" if args.detect == "compare" else "hashed encode (scan + unit + payload launches)", "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
+            "bound": "hbm", "kernel": ("fp16 encode (scan + unit + payload launches)" if args.dtype == "fp16" else "encode_kernel" if args.detect == "compare" else "hashed encode (scan + unit + payload launches)"), "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
             "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBps": enc_gbs / NOMINAL_HBM_GBS,
             "traffic": (NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE * n_layer
                         if args.dtype == "bf16" and args.block == 512 and args.update == "clustered" else None),
@@ -589,7 +598,7 @@ def main():
         out["selection"] = selection_report(args, ciera, layers[-1], enc_ms, dec_ms)
 
     # ---- per-kernel numbers with each kernel alone on the GPU, three change regimes (one layer)
-    if not args.no_regimes and rank == 0 and args.detect == "compare":
+    if not args.no_regimes and rank == 0 and args.detect == "compare" and args.dtype != "fp16":
         out["kernels_alone"] = kernels_alone(args, layers[0], wa[0], wb[0], peak)
 
     # ---- end to end through the host-buffer entry point (weights start and end in host memory)
