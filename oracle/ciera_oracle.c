@@ -56,6 +56,10 @@ static int ora_e(int dtype) { return dtype == ORA_FP16 ? 5 : 8; }
 static int ora_m(int dtype) { return ora_b(dtype) - ora_e(dtype); }
 
 static void put_bits(uint8_t* buf, uint64_t bitpos, int width, uint32_t value) {
+    if (((bitpos | (uint64_t)width) & 7) == 0) { /* whole bytes (bf16, fp32): little-endian */
+        for (int i = 0; i < width / 8; ++i) buf[(bitpos >> 3) + i] |= (uint8_t)(value >> (8 * i));
+        return;
+    }
     for (int i = 0; i < width; ++i) {
         uint64_t p = bitpos + (uint64_t)i;
         if ((value >> i) & 1u) buf[p >> 3] |= (uint8_t)(1u << (p & 7));
@@ -63,6 +67,10 @@ static void put_bits(uint8_t* buf, uint64_t bitpos, int width, uint32_t value) {
 }
 static uint32_t get_bits(const uint8_t* buf, uint64_t bitpos, int width) {
     uint32_t v = 0;
+    if (((bitpos | (uint64_t)width) & 7) == 0) {
+        for (int i = 0; i < width / 8; ++i) v |= (uint32_t)buf[(bitpos >> 3) + i] << (8 * i);
+        return v;
+    }
     for (int i = 0; i < width; ++i) {
         uint64_t p = bitpos + (uint64_t)i;
         v |= (uint32_t)((buf[p >> 3] >> (p & 7)) & 1u) << i;
