@@ -276,13 +276,14 @@ fp16_payload_kernel(const TileDesc* __restrict__ tiles, uint32_t log2b, const ui
 
 // ---------------------------------------------------------------------------------------- receiver
 
+// One thread block per tile, every warp on its own (no barrier, no shared memory): a warp reads the
+// tile's words of the unit's bitmap itself and ranks them with shuffles.  What does not depend on
+// the flags -- the packed sign-plus-mantissa and the cached exponents of the warp's pieces -- is
+// requested first, so that those loads are under way while the flags arrive.
 __global__ void __launch_bounds__(kThreads)
 fp16_decode_kernel(const TileDesc* __restrict__ tiles, uint32_t log2b, const uint8_t* msgs, uint8_t* cache,
                    uint8_t* __restrict__ weights, const unsigned long long* __restrict__ wire_bytes,
                    const uint32_t* __restrict__ ws_prefix, int32_t* status) {
-    __shared__ uint32_t s_bm[kBitmapWords];
-    __shared__ uint32_t s_pre[kBitmapWords];
-    __shared__ uint32_t s_own;
     const uint32_t tile = blockIdx.x, tid = threadIdx.x, lane = tid & 31u;
     const TileDesc td = load_tile_desc(tiles + tile);
     const uint64_t N = td.n_unit;
@@ -290,66 +291,73 @@ fp16_decode_kernel(const TileDesc* __restrict__ tiles, uint32_t log2b, const uin
     const uint32_t nv = (uint32_t)min((uint64_t)kTileValues, N - v0);
     const bool full_tile = nv == (uint32_t)kTileValues;
     const uint32_t B = 1u << log2b;
-    const uint32_t nbt = kTileValues >> log2b;  // at most 256 blocks (B >= 32)
+    const uint32_t nbt = kTileValues >> log2b;  // at most 256 blocks (B >= 32): 8 words of flags
     const uint32_t nblk = (nv + B - 1u) >> log2b;
     const uint8_t* msg = msgs + td.msg_off;
-    // the tile's block flags from the unit's bitmap
-    if (tid < 32) {
-        const uint32_t* bm32 = reinterpret_cast<const uint32_t*>(msg);
-        const uint64_t kb0 = (uint64_t)td.tile_in_unit * nbt;
-        uint32_t word = 0;
-        if (nbt >= 32) {
-            if (lane < (nbt >> 5) && lane * 32u < nblk) {
-                word = bm32[(kb0 >> 5) + lane];
-                const uint32_t left = nblk - lane * 32u;
-                if (left < 32u) word &= (1u << left) - 1u;
-            }
-        } else if (lane == 0) {
-            word = (bm32[kb0 >> 5] >> (kb0 & 31u)) & ((1u << nblk) - 1u);
-        }
-        const uint32_t pc = __popc(word);
-        uint32_t incl = pc;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
-            if ((int)lane >= o) incl += t;
-        }
-        if (lane < kBitmapWords) {
-            s_bm[lane] = word;
-            s_pre[lane] = incl - pc;
-        }
-        if (lane == 31) s_own = incl;
-    }
-    __syncthreads();
-    const uint64_t before = td.tile_in_unit != 0 ? ws_prefix[tile] : 0u;  // changed blocks in the unit's earlier tiles
-    const uint32_t bpb = 5u * (B >> 3);
-    const uint64_t payoff = payload_offset_of(N, CIERA_FP16, log2b);
-    // integrity check by the unit's last tile: the bitmap fixes the message length
-    if (tid == 0 && wire_bytes != nullptr && status != nullptr && td.tile_in_unit == td.n_tiles_unit - 1u) {
-        uint64_t total = (before + s_own) * bpb;
-        const uint32_t rem = (uint32_t)(N & (B - 1u));
-        if (rem) {
-            const uint32_t kb = nv >> log2b;
-            if ((s_bm[kb >> 5] >> (kb & 31u)) & 1u) total -= bpb - (uint32_t)block_payload_bytes(rem, CIERA_FP16);
-        }
-        if (wire_bytes[td.unit] != payoff + total) atomicCAS(status, 0, (int32_t)CIERA_ERR_CORRUPT);
-    }
     const uint8_t* section = msg + sm_offset(N, log2b) + (v0 >> 3) * 11;
-    const uint8_t* pay = msg + payoff + before * bpb;
+
+    // 1. loads that need no flags
+    HalfPiece x[2];
+    uint32_t c[2][2];
+    int nvalid[2];
 #pragma unroll
     for (int p = 0; p < 2; ++p) {
         const uint32_t t0 = h_start(tid, p);
-        const int nvalid = t0 >= nv ? 0 : (int)min(8u, nv - t0);
-        HalfPiece x;
-        load_sm(x.s, section, t0, nvalid, full_tile, lane);
-        if (nvalid == 0) continue;
+        nvalid[p] = t0 >= nv ? 0 : (int)min(8u, nv - t0);
+        load_sm(x[p].s, section, t0, nvalid[p], full_tile, lane);
+        c[p][0] = c[p][1] = 0;
+        if (nvalid[p] > 0) load_exp_bytes(c[p], cache + td.c_off + t0, nvalid[p]);
+    }
+    // 2. the tile's block flags from the unit's bitmap, set flags before each word, their total
+    uint32_t word_l = 0;
+    {
+        const uint32_t* bm32 = reinterpret_cast<const uint32_t*>(msg);
+        const uint64_t kb0 = (uint64_t)td.tile_in_unit * nbt;
+        if (nbt >= 32) {
+            if (lane < (nbt >> 5) && lane * 32u < nblk) {
+                word_l = bm32[(kb0 >> 5) + lane];
+                const uint32_t left = nblk - lane * 32u;
+                if (left < 32u) word_l &= (1u << left) - 1u;
+            }
+        } else if (lane == 0) {
+            word_l = (bm32[kb0 >> 5] >> (kb0 & 31u)) & ((1u << nblk) - 1u);
+        }
+    }
+    const uint64_t before = td.tile_in_unit != 0 ? ws_prefix[tile] : 0u;  // changed blocks in the unit's earlier tiles
+    const uint32_t pc = __popc(word_l);
+    uint32_t incl = pc;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+        if ((int)lane >= o) incl += t;
+    }
+    const uint32_t pre_l = incl - pc;
+    const uint32_t own = __shfl_sync(0xffffffffu, incl, 31);
+    const uint32_t bpb = 5u * (B >> 3);
+    const uint64_t payoff = payload_offset_of(N, CIERA_FP16, log2b);
+    // integrity check by the unit's last tile: the bitmap fixes the message length
+    if (wire_bytes != nullptr && status != nullptr && td.tile_in_unit == td.n_tiles_unit - 1u && tid < 32) {
+        uint64_t total = (before + own) * bpb;
+        const uint32_t rem = (uint32_t)(N & (B - 1u));
+        const uint32_t kb = nv >> log2b;  // the short last block, if there is one
+        const uint32_t last_word = __shfl_sync(0xffffffffu, word_l, (kb >> 5) & 31u);
+        if (rem && ((last_word >> (kb & 31u)) & 1u)) total -= bpb - (uint32_t)block_payload_bytes(rem, CIERA_FP16);
+        if (lane == 0 && wire_bytes[td.unit] != payoff + total) atomicCAS(status, 0, (int32_t)CIERA_ERR_CORRUPT);
+    }
+    const uint8_t* pay = msg + payoff + before * bpb;
+    // 3. exponents of changed blocks from the payload, merge, store
+#pragma unroll
+    for (int p = 0; p < 2; ++p) {
+        const uint32_t t0 = h_start(tid, p);
         const uint32_t kb = t0 >> log2b;
-        const uint32_t word = s_bm[kb >> 5];
+        const uint32_t word = __shfl_sync(0xffffffffu, word_l, (kb >> 5) & 31u);
+        const uint32_t pre = __shfl_sync(0xffffffffu, pre_l, (kb >> 5) & 31u);
+        if (nvalid[p] == 0) continue;
         const bool chg = (word >> (kb & 31u)) & 1u;
         if (chg) {
-            const uint32_t rank = s_pre[kb >> 5] + __popc(word & ((1u << (kb & 31u)) - 1u));
+            const uint32_t rank = pre + __popc(word & ((1u << (kb & 31u)) - 1u));
             const uint8_t* src = pay + (uint64_t)rank * bpb + 5u * ((t0 & (B - 1u)) >> 3);
-            const int nbytes = (5 * nvalid + 7) >> 3;
+            const int nbytes = (5 * nvalid[p] + 7) >> 3;
             uint32_t lo = 0, hi = 0;
             for (int i = 0; i < nbytes; ++i) {
                 const uint32_t b = src[i];
@@ -358,19 +366,20 @@ fp16_decode_kernel(const TileDesc* __restrict__ tiles, uint32_t log2b, const uin
                 else
                     hi = b;
             }
-            x.unpack_exponents(lo, hi);
-            store_exp_bytes(cache + td.c_off + t0, x.e, nvalid);  // ExpCache[i,k] <- newExp[j]
+            x[p].unpack_exponents(lo, hi);
+            store_exp_bytes(cache + td.c_off + t0, x[p].e, nvalid[p]);  // ExpCache[i,k] <- newExp[j]
         } else {
-            load_exp_bytes(x.e, cache + td.c_off + t0, nvalid);
+            x[p].e[0] = c[p][0];
+            x[p].e[1] = c[p][1];
         }
         uint32_t w[4];
-        x.merge(w);
+        x[p].merge(w);
         uint8_t* dst = weights + td.w_off + (uint64_t)t0 * 2;
-        if (nvalid == 8) {
+        if (nvalid[p] == 8) {
             st_stream16(dst, make_uint4(w[0], w[1], w[2], w[3]));
         } else {
             uint16_t* d16 = reinterpret_cast<uint16_t*>(dst);
-            for (int i = 0; i < nvalid; ++i) d16[i] = (uint16_t)(w[i >> 1] >> (16 * (i & 1)));
+            for (int i = 0; i < nvalid[p]; ++i) d16[i] = (uint16_t)(w[i >> 1] >> (16 * (i & 1)));
         }
     }
 }
