@@ -238,9 +238,10 @@ CIERA_API int ciera_encode_hashed(const ciera_plan* plan, const void* weights_de
  * to the same slot of `dst_messages_dev` (one kernel; the lengths are read on the device).  This
  * stands where the Allgather of the messages would be.  `workspace_dev`: scratch of
  * ciera_plan_workspace_bytes() (holds the counter tiles are handed out from; cleared by the call;
- * not to be shared by calls that can overlap on the GPU). */
+ * not to be shared by calls that can overlap on the GPU).  `status_dev`: device int32 or NULL; the
+ * kernel's waits on its own copies are bounded and raise CIERA_ERR_TIMEOUT there. */
 CIERA_API int ciera_transport(const ciera_plan* plan, const void* src_messages_dev, void* dst_messages_dev,
-                    const uint64_t* wire_bytes_dev, void* workspace_dev, void* stream);
+                    const uint64_t* wire_bytes_dev, void* workspace_dev, int32_t* status_dev, void* stream);
 
 /* ---- receiver: Algorithm 1, receiver part; Section 3.1 ------------------------------------- */
 

@@ -80,7 +80,7 @@ _SIGS = {
     "ciera_plan_entropy_scratch_bytes": ([_vp], _sz),
     "ciera_entropy_encode": ([_vp] * 5, _i32),
     "ciera_entropy_decode": ([_vp] * 6, _i32),
-    "ciera_transport": ([_vp] * 6, _i32),
+    "ciera_transport": ([_vp] * 7, _i32),
     "ciera_decode": ([_vp] * 8, _i32),
     "ciera_roundtrip_host": ([_vp, _vp, _sz, _vp, _vp, _vp, _vp], _i32),
     "ciera_should_compress": ([ctypes.POINTER(GainIn), ctypes.POINTER(_dbl), ctypes.POINTER(_i32)], _i32),
@@ -260,10 +260,10 @@ def entropy_decode(plan: Plan, messages, wire_bytes, scratch, status=None, strea
                                      _stream(stream)))
 
 
-def transport(plan: Plan, src_messages, dst_messages, wire_bytes, workspace, stream=None) -> None:
+def transport(plan: Plan, src_messages, dst_messages, wire_bytes, workspace, status=None, stream=None) -> None:
     _check("ciera_transport",
            _lib.ciera_transport(plan.handle, _ptr(src_messages), _ptr(dst_messages), _ptr(wire_bytes),
-                                _ptr(workspace), _stream(stream)))
+                                _ptr(workspace), _ptr(status), _stream(stream)))
 
 
 def decode(plan: Plan, messages, receiver_cache, weights_out, wire_bytes=None, workspace=None, status=None,

@@ -40,15 +40,9 @@ cache_fill_kernel(const TileDesc* __restrict__ tiles, const uint8_t* __restrict_
 // ------------------------------------------------------------------------------------------
 // transport stand-in: copy the used bytes of every slot
 //
-// A persistent copy kernel in which every warp works on its own: it draws tile numbers from a
-// counter in the caller's scratch (so all SMs stay busy to the end whatever their pace); tile j of
-// a unit moves bytes [j * chunk, (j + 1) * chunk) of the unit's slot (chunk = 16 KB for bf16, 32 KB
-// for fp32, plus a tile's share of the bitmap when blocks are fine), the last tile also what lies beyond, cut off at the length the sender reported.  A warp moves 4 KB per step (eight 128-bit loads per lane in flight, then eight
-// stores); tile numbers, descriptors and reported lengths are fetched three, two and one tile
-// ahead, so that no step waits for them.
-
-constexpr int kCopyThreads = 256;
-constexpr int kCopyUnroll = 8;  // 128-bit loads in flight per lane
+// Tile j of a unit moves bytes [j * chunk, (j + 1) * chunk) of the unit's slot (chunk = 16 KB for
+// bf16 and fp16, 32 KB for fp32, plus a tile's share of the bitmap when blocks are fine), the last
+// tile also what lies beyond, cut off at the length the sender reported.
 
 // the part of a tile descriptor the copy needs (keeps the prefetched copies small in registers)
 struct CopyDesc {
@@ -66,70 +60,167 @@ __device__ __forceinline__ CopyDesc load_copy_desc(const TileDesc* t) {
     return d;
 }
 
-__global__ void __launch_bounds__(kCopyThreads)
-transport_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint64_t chunk,
-                 const uint8_t* __restrict__ src, uint8_t* __restrict__ dst,
-                 const unsigned long long* __restrict__ wire_bytes, unsigned int* ticket) {
-    const uint32_t lane = threadIdx.x & 31u;
-    auto draw = [&]() {
-        uint32_t t = 0;
-        if (lane == 0) t = atomicAdd(ticket, 1u);
-        return __shfl_sync(0xffffffffu, t, 0);
-    };
-    // three-deep software pipeline: tile number drawn (t_c), descriptor loaded (t_b, td_b), reported
-    // length loaded (t_a, td_a, used_a)
-    uint32_t t_a = draw(), t_b = draw(), t_c = draw();
-    CopyDesc td_a, td_b;
-    unsigned long long used_a = 0;
-    if (t_a < n_tiles) {
-        td_a = load_copy_desc(tiles + t_a);
-        used_a = __ldg(wire_bytes + td_a.unit);
-    }
-    if (t_b < n_tiles) td_b = load_copy_desc(tiles + t_b);
-    while (t_a < n_tiles) {
-        const CopyDesc td = td_a;
-        const uint64_t used = used_a;
-        // advance the pipeline; none of these loads is needed before the next iteration
-        const uint32_t t_d = t_c < n_tiles ? draw() : n_tiles;
-        td_a = td_b;
-        if (t_b < n_tiles) used_a = __ldg(wire_bytes + td_a.unit);
-        if (t_c < n_tiles) td_b = load_copy_desc(tiles + t_c);
-        t_a = t_b;
-        t_b = t_c;
-        t_c = t_d;
+// A persistent kernel in which the loads are done by the copy engine.  A producer warp draws tiles from the
+// counter, kPipeBatch at a time (one per lane: descriptors and reported lengths of a batch are
+// fetched in parallel and two batches ahead, so tiles beyond the used part of their messages cost
+// next to nothing), cuts each tile's byte range into pieces of at most kPipeStage bytes and starts
+// one bulk-async copy per piece into a ring of shared-memory stages; eight consumer warps move every
+// stage to its destination with 128-bit stores and hand it back.  Loads in flight then cost no
+// registers and no issue slots, and the stores of one stage overlap the loads of the next ones.
+constexpr uint32_t kPipeStage = 16384;
+constexpr int kPipeStages = 6;
+constexpr int kPipeConsumers = 8;                        // warps
+constexpr int kPipeThreads = 32 * (kPipeConsumers + 1);  // + the producer warp
+constexpr uint32_t kPipeBatch = 3;                       // tiles drawn at a time (measured: 3 beats 2, 4 and 8)
 
-        const uint64_t lo = (uint64_t)td.tile_in_unit * chunk;
-        if (lo >= used) continue;
-        // the unit's last tile also takes what lies beyond tiles * chunk
-        const bool last = td.tile_in_unit == td.n_tiles_unit - 1u;
-        const uint64_t hi = (last || lo + chunk >= used) ? used : lo + chunk;
-        const uint8_t* s = src + td.msg_off + lo;
-        uint8_t* d = dst + td.msg_off + lo;
-        const uint32_t nvec = (uint32_t)((hi - lo) >> 4);  // 16-byte pieces
-        uint32_t i = lane;
-        for (; i + 32u * (kCopyUnroll - 1) < nvec; i += 32u * kCopyUnroll) {
-            uint4 v[kCopyUnroll];
-#pragma unroll
-            for (int u = 0; u < kCopyUnroll; ++u) v[u] = ld_stream16(s + 16ull * (i + 32u * u));
-#pragma unroll
-            for (int u = 0; u < kCopyUnroll; ++u) st_stream16(d + 16ull * (i + 32u * u), v[u]);
+struct PipeSlot {
+    uint8_t* dst;
+    const uint8_t* tail_src;  // where the piece's last (hi - lo) % 16 bytes come from
+    uint32_t bytes;           // 0xffffffff: no more work
+    uint32_t pad;
+};
+struct PipeCtl {
+    uint64_t full[kPipeStages];
+    uint64_t empty[kPipeStages];
+    PipeSlot slot[kPipeStages];
+    int abort;
+    uint32_t issued, seen;
+};
+
+__global__ void __launch_bounds__(kPipeThreads, 2)
+transport_pipe_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint64_t chunk, const uint8_t* __restrict__ src,
+                      uint8_t* __restrict__ dst, const unsigned long long* __restrict__ wire_bytes, unsigned int* ticket,
+                      int32_t* status) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    PipeCtl* ctl = reinterpret_cast<PipeCtl*>(smem + (size_t)kPipeStages * kPipeStage);
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    volatile int* abort = &ctl->abort;
+    if (tid == 0) {
+        for (int s = 0; s < kPipeStages; ++s) {
+            mbar_init(&ctl->full[s], 1);
+            mbar_init(&ctl->empty[s], kPipeConsumers);
         }
-        for (; i < nvec; i += 32u) st_stream16(d + 16ull * i, ld_stream16(s + 16ull * i));
-        // a ragged end (fewer than 16 bytes; only the last tile of a message can have one)
-        const uint32_t tail = (uint32_t)((hi - lo) & 15ull);
-        if (lane < tail) d[16ull * nvec + lane] = s[16ull * nvec + lane];
+        ctl->abort = 0;
+        ctl->issued = 0;
+        ctl->seen = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+
+    if (warp == kPipeConsumers) {
+        // ---------------------------------------------------------------- producer warp
+        // every lane below kPipeBatch carries one tile through three steps: number (t_a), descriptor
+        // (td_b), descriptor and reported length (td_c, used_c); a step's loads are used one batch later
+        auto draw = [&]() {
+            uint32_t base = 0;
+            if (lane == 0) base = atomicAdd(ticket, kPipeBatch);
+            base = __shfl_sync(0xffffffffu, base, 0);
+            return lane < kPipeBatch ? base + lane : n_tiles;
+        };
+        uint32_t t_a = draw(), t_b = n_tiles, t_c = n_tiles;
+        CopyDesc td_b, td_c;
+        unsigned long long used_c = 0;
+        auto advance = [&]() {
+            td_c = td_b;
+            t_c = t_b;
+            if (t_c < n_tiles) used_c = __ldg(wire_bytes + td_c.unit);
+            t_b = t_a;
+            if (t_b < n_tiles) td_b = load_copy_desc(tiles + t_b);
+            // once a batch starts past the end there is nothing more to draw
+            t_a = __any_sync(0xffffffffu, t_a < n_tiles) ? draw() : n_tiles;
+        };
+        advance();
+        advance();
+        uint32_t k = 0;  // pieces issued so far (lane 0)
+        bool ok = true;
+        while (ok && __any_sync(0xffffffffu, t_c < n_tiles)) {
+            // this batch's byte ranges
+            uint64_t lo = 0, hi = 0, off = 0;
+            if (t_c < n_tiles) {
+                off = td_c.msg_off;
+                lo = (uint64_t)td_c.tile_in_unit * chunk;
+                const bool last = td_c.tile_in_unit == td_c.n_tiles_unit - 1u;
+                hi = (last || lo + chunk >= used_c) ? used_c : lo + chunk;
+                if (lo >= used_c) hi = lo;  // beyond the used part: nothing to move
+            }
+            advance();  // the next batches' loads go out before this batch is worked on
+            uint32_t todo = __ballot_sync(0xffffffffu, lo < hi);
+            while (ok && todo) {
+                const int l = __ffs(todo) - 1;
+                todo &= todo - 1;
+                uint64_t p_lo = __shfl_sync(0xffffffffu, lo, l);
+                const uint64_t p_hi = __shfl_sync(0xffffffffu, hi, l);
+                const uint64_t p_off = __shfl_sync(0xffffffffu, off, l);
+                if (lane == 0) {
+                    while (p_lo < p_hi) {
+                        const uint32_t bytes = (uint32_t)min((uint64_t)kPipeStage, p_hi - p_lo);
+                        const uint32_t st = k % kPipeStages;
+                        if (k >= (uint32_t)kPipeStages &&
+                            !mbar_wait(&ctl->empty[st], ((k / kPipeStages) & 1u) ^ 1u, abort, status)) {
+                            ok = false;
+                            break;
+                        }
+                        const uint32_t body = bytes & ~15u;
+                        ctl->slot[st].dst = dst + p_off + p_lo;
+                        ctl->slot[st].tail_src = src + p_off + p_lo + body;
+                        ctl->slot[st].bytes = bytes;
+                        if (body) {
+                            mbar_arrive_expect_tx(&ctl->full[st], body);
+                            bulk_load(smem + (size_t)st * kPipeStage, src + p_off + p_lo, body, &ctl->full[st]);
+                        } else {
+                            mbar_arrive(&ctl->full[st]);
+                        }
+                        ctl->issued = ++k;
+                        p_lo += bytes;
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            }
+        }
+        if (lane == 0 && ok) {  // end marker
+            const uint32_t st = k % kPipeStages;
+            if (k < (uint32_t)kPipeStages || mbar_wait(&ctl->empty[st], ((k / kPipeStages) & 1u) ^ 1u, abort, status)) {
+                ctl->slot[st].bytes = 0xffffffffu;
+                mbar_arrive(&ctl->full[st]);
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- consumers
+        for (uint32_t k = 0;; ++k) {
+            const uint32_t st = k % kPipeStages;
+            if (!mbar_wait(&ctl->full[st], (k / kPipeStages) & 1u, abort, status)) break;
+            if (tid == 0) ctl->seen = k + 1;
+            const PipeSlot sl = ctl->slot[st];
+            if (sl.bytes == 0xffffffffu) break;
+            const uint32_t nvec = sl.bytes >> 4;
+            const uint8_t* from = smem + (size_t)st * kPipeStage;
+            for (uint32_t i = tid; i < nvec; i += 32u * kPipeConsumers) st_stream16(sl.dst + 16ull * i, ld_shared16(from + 16ull * i));
+            const uint32_t tail = sl.bytes & 15u;  // only the last piece of a message can have one
+            if (warp == 0 && lane < tail) sl.dst[16ull * nvec + lane] = sl.tail_src[lane];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->empty[st]);
+        }
+    }
+    __syncthreads();
+    if (tid == 0 && ctl->abort) {  // after an aborted run wait (bounded) for bulk copies still in flight
+        for (uint32_t k = ctl->seen; k < ctl->issued; ++k)
+            for (uint32_t i = 0; i < kMaxBarrierPolls; ++i)
+                if (mbar_try_wait(&ctl->full[k % kPipeStages], (k / kPipeStages) & 1u)) break;
     }
 }
 
-static int transport_grid_limit(int* out) {
+static int transport_pipe_grid_limit(int* out) {
     static int cached[64] = {0};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return record_cuda_error(e);
     if (dev < 0 || dev >= 64) return CIERA_ERR_UNSUPPORTED;
     if (cached[dev] == 0) {
+        const size_t smem = (size_t)kPipeStages * kPipeStage + sizeof(PipeCtl);
+        e = cudaFuncSetAttribute(transport_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return record_cuda_error(e);
         int per_sm = 0, sms = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, transport_kernel, kCopyThreads, 0);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, transport_pipe_kernel, kPipeThreads, smem);
         if (e != cudaSuccess) return record_cuda_error(e);
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return record_cuda_error(e);
@@ -181,7 +272,7 @@ extern "C" int ciera_cache_update(const ciera_plan* plan, void* cache_dev, const
 }
 
 extern "C" int ciera_transport(const ciera_plan* p, const void* src_messages_dev, void* dst_messages_dev,
-                               const uint64_t* wire_bytes_dev, void* workspace_dev, void* stream) {
+                               const uint64_t* wire_bytes_dev, void* workspace_dev, int32_t* status_dev, void* stream) {
     int rc = check_plan(p);
     if (rc) return rc;
     const uint32_t nt = (uint32_t)p->tiles.size();
@@ -194,13 +285,13 @@ extern "C" int ciera_transport(const ciera_plan* p, const void* src_messages_dev
     cudaError_t me = cudaMemsetAsync(ticket, 0, 16, (cudaStream_t)stream);
     if (me != cudaSuccess) return record_cuda_error(me);
     int limit = 0;
-    rc = transport_grid_limit(&limit);
+    rc = transport_pipe_grid_limit(&limit);
     if (rc) return rc;
-    const uint32_t want = (nt + kCopyThreads / 32 - 1) / (kCopyThreads / 32);
-    const uint32_t grid = want < (uint32_t)limit ? want : (uint32_t)limit;
-    transport_kernel<<<grid, kCopyThreads, 0, (cudaStream_t)stream>>>(
-        p->tiles_dev, nt, transport_chunk_bytes(p->dtype == CIERA_FP32 ? 3u : 1u, p->log2b), (const uint8_t*)src_messages_dev, (uint8_t*)dst_messages_dev,
-        (const unsigned long long*)wire_bytes_dev, ticket);
+    const uint32_t want_blocks = (nt + kPipeBatch - 1) / kPipeBatch;
+    const uint32_t grid = want_blocks < (uint32_t)limit ? want_blocks : (uint32_t)limit;
+    transport_pipe_kernel<<<grid, kPipeThreads, (size_t)kPipeStages * kPipeStage + sizeof(PipeCtl), (cudaStream_t)stream>>>(
+        p->tiles_dev, nt, transport_chunk_bytes(p->dtype == CIERA_FP32 ? 3u : 1u, p->log2b), (const uint8_t*)src_messages_dev,
+        (uint8_t*)dst_messages_dev, (const unsigned long long*)wire_bytes_dev, ticket, status_dev);
     count_launch();
     return check_launch();
 }
@@ -218,7 +309,7 @@ extern "C" int ciera_roundtrip_host(const ciera_plan* p, const void* weights_hos
     rc = ciera_encode(p, b->weights_dev, b->sender_cache_dev, b->msg_send_dev, b->wire_bytes_dev, b->changed_blocks_dev,
                       b->workspace_dev, b->status_dev, stream);
     if (rc) return rc;
-    rc = ciera_transport(p, b->msg_send_dev, b->msg_recv_dev, b->wire_bytes_dev, b->workspace_dev, stream);
+    rc = ciera_transport(p, b->msg_send_dev, b->msg_recv_dev, b->wire_bytes_dev, b->workspace_dev, b->status_dev, stream);
     if (rc) return rc;
     rc = ciera_decode(p, b->msg_recv_dev, b->receiver_cache_dev, b->weights_out_dev, b->wire_bytes_dev,
                       b->workspace_dev, b->status_dev, stream);

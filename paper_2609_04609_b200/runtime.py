@@ -88,7 +88,7 @@ class LayerCodec:
                      self.workspace, self.status, stream)
 
     def transport(self, stream=None) -> None:
-        ciera.transport(self.plan, self.msg_send, self.msg_recv, self.wire_bytes, self.workspace, stream)
+        ciera.transport(self.plan, self.msg_send, self.msg_recv, self.wire_bytes, self.workspace, self.status, stream)
 
     def decode(self, weights_out: Optional[torch.Tensor] = None, stream=None, check_length: bool = True) -> None:
         out = self.weights_out if weights_out is None else weights_out
