@@ -38,7 +38,7 @@
 
 namespace ciera {
 
-constexpr int kResolvers = 3;                                    // resolver warps
+constexpr int kResolvers = 2;  // resolver warps (20 warps per block: two blocks per SM at 48 registers per thread)
 constexpr int kEncodeThreads = kThreads + 64 + 32 * kResolvers;  // consumers + producer + aggregator + resolvers
 constexpr int kProducerWarp = kWarps;                            // 16
 constexpr int kAggregatorWarp = kWarps + 1;                      // 17
