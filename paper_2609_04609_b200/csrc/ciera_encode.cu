@@ -485,10 +485,12 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
         // ---------------------------------------------------------------- consumers
         uint32_t k_end = kNoTile;  // slot of the first end marker, once seen
         uint32_t k = 0;
+        // stage and phase of slot k in the two rings, and of slot k - kDefer in the exponent ring, kept
+        // as running counters (the ring depths are no powers of two)
+        uint32_t sw = 0, pw = 0, se = 0, pe = 0, je = 0, pj = 0;
         for (;; ++k) {
-            const uint32_t sw = k % SW, se = k % SE;
-            if (!mbar_wait(&ctl->full_w[sw], (k / SW) & 1u, abort, status)) break;
-            if (!mbar_wait(&ctl->full_e[se], (k / SE) & 1u, abort, status)) break;
+            if (!mbar_wait(&ctl->full_w[sw], pw, abort, status)) break;
+            if (!mbar_wait(&ctl->full_e[se], pe, abort, status)) break;
             if (tid == 0) ctl->seen = k + 1;
             const bool marker = ctl->tile_idx[k % kDescRing] == kNoTile;
             if (marker) {
@@ -558,15 +560,28 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
             }
 
             // the changed exponents of the tile handled kDefer slots ago: its offset is known by now
-            if (k >= (uint32_t)kDefer && k - kDefer < k_end) {
-                const uint32_t j = k - kDefer, je = j % SE;
-                if (!mbar_wait(&ctl->resolved[je], (j / SE) & 1u, abort, status)) break;
-                send_changed<DT, FINE>(ctl->info[j % kDescRing], log2b, ctl->bm[je], ctl->pre[je], ctl->base[je],
-                                       ring_e + (size_t)je * kEBytes, tid);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&ctl->empty_e[je]);
+            if (k >= (uint32_t)kDefer) {
+                if (k - kDefer < k_end) {
+                    if (!mbar_wait(&ctl->resolved[je], pj, abort, status)) break;
+                    send_changed<DT, FINE>(ctl->info[(k - kDefer) % kDescRing], log2b, ctl->bm[je], ctl->pre[je],
+                                           ctl->base[je], ring_e + (size_t)je * kEBytes, tid);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&ctl->empty_e[je]);
+                }
+                if (++je == (uint32_t)SE) {
+                    je = 0;
+                    pj ^= 1u;
+                }
             }
             if (marker && k + 1u == k_end + (uint32_t)kResolvers) break;  // that was the last end marker
+            if (++sw == (uint32_t)SW) {
+                sw = 0;
+                pw ^= 1u;
+            }
+            if (++se == (uint32_t)SE) {
+                se = 0;
+                pe ^= 1u;
+            }
         }
         // tiles whose changed exponents are still to be sent (when kDefer > kResolvers)
         if (!*abort && k_end != kNoTile) {
