@@ -10,7 +10,11 @@
 
 namespace ciera {
 
-constexpr uint32_t kMaxBarrierPolls = 1u << 22;  // each poll may itself suspend for a short time slice
+// A poll suspends the thread in hardware until the phase completes or kSuspendNs have passed, so a
+// waiting warp takes (almost) no issue slots from the working ones; the bound on a wait is
+// kMaxBarrierPolls * kSuspendNs, about 1.3 s.
+constexpr uint32_t kSuspendNs = 20000;
+constexpr uint32_t kMaxBarrierPolls = 1u << 16;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -29,10 +33,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendNs)
         : "memory");
     return ok != 0;
 }
@@ -42,7 +46,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort, int32_t* status) {
     for (uint32_t i = 0; i < kMaxBarrierPolls; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 63u) == 63u && *abort) return false;
+        if (*abort) return false;
     }
     *abort = 1;
     if (status) atomicCAS(status, 0, (int32_t)CIERA_ERR_TIMEOUT);
