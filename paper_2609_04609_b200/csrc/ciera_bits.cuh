@@ -55,6 +55,7 @@ struct Global {
     static __device__ __forceinline__ void st16(uint8_t* p, uint4 v) { st_stream16(p, v); }
     static __device__ __forceinline__ void st8(uint8_t* p, uint2 v) { st_stream8(p, v); }
     static __device__ __forceinline__ uint32_t ld1(const uint8_t* p) { return __ldcs(p); }
+    static __device__ __forceinline__ uint32_t ld4(const uint8_t* p) { return __ldcs(reinterpret_cast<const uint32_t*>(p)); }
 };
 struct Shared {
     static __device__ __forceinline__ uint4 ld16(const uint8_t* p) { return ld_shared16(p); }
@@ -64,6 +65,11 @@ struct Shared {
     static __device__ __forceinline__ uint32_t ld1(const uint8_t* p) {
         uint32_t v;
         asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"((uint32_t)__cvta_generic_to_shared(p)));
+        return v;
+    }
+    static __device__ __forceinline__ uint32_t ld4(const uint8_t* p) {
+        uint32_t v;
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"((uint32_t)__cvta_generic_to_shared(p)));
         return v;
     }
 };
@@ -335,6 +341,170 @@ struct Piece<CIERA_FP32> {
 #pragma unroll
         for (int i = 0; i < 4; ++i) f |= word_block_flags(e[i] ^ o.e[i], log2b) << (per_word * i);
         return f;
+    }
+};
+
+// fp16: 8 values = 16 B of weights, 8 exponent bytes in the caches, and on the wire 11 bytes of
+// sign-plus-mantissa (8 x 11 bits, value j at bits [11 j, 11 j + 11)) and 5 bytes of exponents
+// (8 x 5 bits).  Thread -> value layout as for bf16.
+template <>
+struct Piece<CIERA_FP16> {
+    static constexpr int kValues = 8;
+    static constexpr int kLog2Values = 3;
+    static constexpr int kPerThread = 2;
+    static constexpr int kExpWords = 2;
+    static __device__ __forceinline__ uint32_t start(uint32_t tid, int p) {
+        return (uint32_t)p * (kTileValues / 2) + tid * 8u;
+    }
+
+    uint32_t e[2];  // 8 exponents, one byte each (0..31)
+    uint32_t s[3];  // 88 bits of sign-plus-mantissa
+
+    // w = eight fp16 values, two per word
+    __device__ __forceinline__ void split_words(const uint32_t w[4]) {
+        uint32_t e2[4], f[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            e2[i] = (w[i] >> 10) & 0x001F001Fu;
+            const uint32_t sm2 = (w[i] & 0x03FF03FFu) | ((w[i] >> 5) & 0x04000400u);
+            f[2 * i] = sm2 & 0xFFFFu;
+            f[2 * i + 1] = sm2 >> 16;
+        }
+        e[0] = __byte_perm(e2[0], e2[1], 0x6420);
+        e[1] = __byte_perm(e2[2], e2[3], 0x6420);
+        s[0] = f[0] | (f[1] << 11) | (f[2] << 22);
+        s[1] = (f[2] >> 10) | (f[3] << 1) | (f[4] << 12) | (f[5] << 23);
+        s[2] = (f[5] >> 9) | (f[6] << 2) | (f[7] << 13);
+    }
+    __device__ __forceinline__ void merge_words(uint32_t w[4]) const {
+        uint32_t f[8];
+        f[0] = s[0] & 0x7FFu;
+        f[1] = (s[0] >> 11) & 0x7FFu;
+        f[2] = ((s[0] >> 22) | (s[1] << 10)) & 0x7FFu;
+        f[3] = (s[1] >> 1) & 0x7FFu;
+        f[4] = (s[1] >> 12) & 0x7FFu;
+        f[5] = ((s[1] >> 23) | (s[2] << 9)) & 0x7FFu;
+        f[6] = (s[2] >> 2) & 0x7FFu;
+        f[7] = (s[2] >> 13) & 0x7FFu;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t ex = (e[i >> 2] >> (8 * (i & 3))) & 0x1Fu;
+            const uint32_t v = (f[i] & 0x3FFu) | ((f[i] & 0x400u) << 5) | (ex << 10);
+            if (i & 1)
+                w[i >> 1] |= v << 16;
+            else
+                w[i >> 1] = v;
+        }
+    }
+    template <class M>
+    __device__ __forceinline__ void split_full(const uint8_t* src) {
+        const uint4 v = M::ld16(src);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        split_words(w);
+    }
+    // the first nvalid (< 8) values; the others read as +0.0
+    __device__ __forceinline__ void split_partial(const uint8_t* src, int nvalid) {
+        const uint16_t* p = reinterpret_cast<const uint16_t*>(src);
+        uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (i < nvalid) w[i >> 1] |= (uint32_t)p[i] << (16 * (i & 1));
+        split_words(w);
+    }
+    template <class M>
+    __device__ __forceinline__ void merge_store_full(uint8_t* dst) const {
+        uint32_t w[4];
+        merge_words(w);
+        M::st16(dst, make_uint4(w[0], w[1], w[2], w[3]));
+    }
+    __device__ __forceinline__ void merge_store_partial(uint8_t* dst, int nvalid) const {
+        uint32_t w[4];
+        merge_words(w);
+        uint16_t* d16 = reinterpret_cast<uint16_t*>(dst);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (i < nvalid) d16[i] = (uint16_t)(w[i >> 1] >> (16 * (i & 1)));
+    }
+    template <class M>
+    __device__ __forceinline__ void load_exp_full(const uint8_t* src) {
+        const uint2 v = M::ld8(src);
+        e[0] = v.x; e[1] = v.y;
+    }
+    template <class M>
+    __device__ __forceinline__ void store_exp_full(uint8_t* dst) const { M::st8(dst, make_uint2(e[0], e[1])); }
+    __device__ __forceinline__ void load_exp_partial(const uint8_t* src, int nvalid) { load_bytes_partial<8>(e, src, nvalid); }
+    __device__ __forceinline__ void store_exp_partial(uint8_t* dst, int nvalid) const { store_bytes_partial<8>(dst, e, nvalid); }
+    __device__ __forceinline__ bool differs(const Piece& o) const { return ((e[0] ^ o.e[0]) | (e[1] ^ o.e[1])) != 0; }
+
+    // the 8 exponents as 40 bits: low word and high byte
+    __device__ __forceinline__ void pack_exponents(uint32_t& lo, uint32_t& hi) const {
+        uint32_t x[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[i] = (e[i >> 2] >> (8 * (i & 3))) & 0x1Fu;
+        lo = x[0] | (x[1] << 5) | (x[2] << 10) | (x[3] << 15) | (x[4] << 20) | (x[5] << 25) | (x[6] << 30);
+        hi = (x[6] >> 2) | (x[7] << 3);
+    }
+    __device__ __forceinline__ void unpack_exponents(uint32_t lo, uint32_t hi) {
+        uint32_t x[8];
+#pragma unroll
+        for (int i = 0; i < 6; ++i) x[i] = (lo >> (5 * i)) & 0x1Fu;
+        x[6] = ((lo >> 30) | (hi << 2)) & 0x1Fu;
+        x[7] = (hi >> 3) & 0x1Fu;
+        e[0] = x[0] | (x[1] << 8) | (x[2] << 16) | (x[3] << 24);
+        e[1] = x[4] | (x[5] << 8) | (x[6] << 16) | (x[7] << 24);
+    }
+    // the packed exponents of the piece from `src` (5 bytes, any alignment; nvalid < 8: fewer)
+    template <class M>
+    __device__ __forceinline__ void load_packed_exponents(const uint8_t* src, int nvalid) {
+        const int nbytes = (5 * nvalid + 7) >> 3;
+        uint32_t lo = 0, hi = 0;
+#pragma unroll
+        for (int i = 0; i < 5; ++i) {
+            if (i < nbytes) {
+                const uint32_t b = M::ld1(src + i);
+                if (i < 4)
+                    lo |= b << (8 * i);
+                else
+                    hi = b;
+            }
+        }
+        unpack_exponents(lo, hi);
+    }
+
+    // Packed sign-plus-mantissa of a piece in a section whose pieces are all complete: the four lanes
+    // 4k..4k+3 share 44 bytes = 11 aligned words, lane a holds bits [88a, 88a+88) of them.
+    // `section` = start of the tile's part of the section, `piece` = index of the piece in the tile.
+    template <class M>
+    __device__ __forceinline__ void load_sm_group(const uint8_t* section, uint32_t piece, uint32_t lane) {
+        const uint32_t a = lane & 3u;
+        // lane a's bits start at word {0, 2, 5, 8}, bit {0, 24, 16, 8} of the group
+        const uint32_t first = (11u * a) >> 2, sh = (88u * a) & 31u;
+        const uint8_t* src = section + (size_t)11 * (piece - a) + 4u * first;
+        const uint32_t w0 = M::ld4(src), w1 = M::ld4(src + 4), w2 = M::ld4(src + 8);
+        const uint32_t w3 = (a == 0u || a == 3u) ? 0u : M::ld4(src + 12);  // lanes 0 and 3 end inside their third word
+        s[0] = sh ? (w0 >> sh) | (w1 << (32u - sh)) : w0;
+        s[1] = sh ? (w1 >> sh) | (w2 << (32u - sh)) : w1;
+        s[2] = (sh ? (w2 >> sh) | (w3 << (32u - sh)) : w2) & 0x00FFFFFFu;
+    }
+    // lane a writes words 3a, 3a+1, 3a+2 of the group (lane 3: two words), taking the low bits of the
+    // next lane's first word where its own bits end inside a word.  All 32 lanes call this.
+    __device__ __forceinline__ void store_sm_group(uint8_t* section, uint32_t piece, uint32_t lane) const {
+        const uint32_t a = lane & 3u, sh = 8u * a;
+        const uint32_t next0 = __shfl_down_sync(0xffffffffu, s[0], 1);
+        uint32_t* dst = reinterpret_cast<uint32_t*>(section + (size_t)11 * (piece - a)) + 3u * a;
+        dst[0] = sh ? (s[0] >> sh) | (s[1] << (32u - sh)) : s[0];
+        dst[1] = sh ? (s[1] >> sh) | (s[2] << (32u - sh)) : s[1];
+        if (a != 3u) dst[2] = (s[2] >> sh) | (next0 << (24u - sh));
+    }
+    // byte by byte (pieces of a tile with a ragged end)
+    __device__ __forceinline__ void load_sm_bytes(const uint8_t* src, int nvalid) {
+        s[0] = s[1] = s[2] = 0;
+        const int nbytes = (11 * nvalid + 7) >> 3;
+        for (int i = 0; i < nbytes; ++i) s[i >> 2] |= (uint32_t)src[i] << (8 * (i & 3));
+    }
+    __device__ __forceinline__ void store_sm_bytes(uint8_t* dst, int nvalid) const {
+        const int nbytes = (11 * nvalid + 7) >> 3;
+        for (int i = 0; i < nbytes; ++i) dst[i] = (uint8_t)(s[i >> 2] >> (8 * (i & 3)));
     }
 };
 

@@ -54,6 +54,13 @@ struct DecodeCfg<CIERA_FP32, false> {
     static constexpr int kRing = 12;
 };
 template <>
+struct DecodeCfg<CIERA_FP16, false> {
+    static constexpr int kStages = 4;        // 4 x (11 KB sm + 8 KB cache span + 5 KB packed payload slice)
+    static constexpr int kBlocksPerSM = 2;
+    static constexpr bool kStageOut = false;
+    static constexpr int kRing = 12;
+};
+template <>
 struct DecodeCfg<CIERA_BF16, true> {
     static constexpr int kStages = 4;
     static constexpr int kBlocksPerSM = 2;
@@ -282,6 +289,16 @@ __device__ __forceinline__ void gather_changed(Piece<DT>& x, uint32_t km, uint32
     }
 }
 
+// Bytes of one shared-memory stage: the tile's sign-plus-mantissa, the span of cached exponents
+// (one byte per value), the payload slice (every block changed at most) and, where the slice need
+// not start on a 16-byte boundary (fine blocks, fp16), 16 bytes of slack.  Used by the kernel and by
+// the host when it sizes the dynamic shared memory.
+template <int DT, bool FINE>
+__host__ __device__ constexpr uint32_t decode_stage_bytes() {
+    return (uint32_t)sm_bytes_of_values<DT>(kTileValues) + (uint32_t)kTileValues +
+           (uint32_t)payload_bytes_of_blocks<DT>(kTileValues >> 5, 5) + ((FINE || DT == CIERA_FP16) ? 16u : 0u);
+}
+
 template <int DT, bool FINE>
 __global__ void __launch_bounds__(kDecodeThreads, DecodeCfg<DT, FINE>::kBlocksPerSM)
 decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log2b, const uint8_t* msgs, uint8_t* cache,
@@ -289,16 +306,18 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
               const uint32_t* __restrict__ ws_prefix, unsigned int* ticket, int32_t* status) {
     using P = Piece<DT>;
     constexpr int VB = Traits<DT>::kValueBytes;
-    constexpr int SMB = Traits<DT>::kSmBytes;
+    constexpr int SMB = Traits<DT>::kSmBytes;  // (not used for fp16)
+    constexpr bool kHalf = DT == CIERA_FP16;    // packed sections: see Piece<CIERA_FP16>
+    static_assert(!(kHalf && FINE), "fp16 takes blocks of 32 values and more");
     using Cfg = DecodeCfg<DT, FINE>;
     constexpr int S = Cfg::kStages;
     constexpr int kDecRing = Cfg::kRing;
     static_assert(S % kDecProducers == 0, "every producer cycles through stages of its own");
     static_assert(kDecRing > S + 2 * kDecProducers + 1, "a slot is refilled only after its tile is done");
     constexpr bool kStageOut = Cfg::kStageOut;
-    constexpr uint32_t kSmTile = kTileValues * SMB;                   // sign-plus-mantissa of a tile
-    // + cache span + payload slice (which, with fine blocks, need not start on a 16-byte boundary)
-    constexpr uint32_t kStageBytes = kSmTile + 2u * kTileValues + (FINE ? 16u : 0u);
+    constexpr uint32_t kSmTile = (uint32_t)sm_bytes_of_values<DT>(kTileValues);  // sign-plus-mantissa of a tile
+    constexpr bool kSkew = FINE || kHalf;  // the payload slice need not start on a 16-byte boundary
+    constexpr uint32_t kStageBytes = decode_stage_bytes<DT, FINE>();  // + cache span + payload slice
     constexpr uint32_t kOutBytes = kStageOut ? kTileValues * VB : 0u;  // reconstructed tile, staged for bulk stores
     constexpr uint32_t kWarpOutBytes = 32 * P::kValues * VB;           // one warp's contiguous slice of it
     extern __shared__ __align__(128) uint8_t smem[];
@@ -382,9 +401,10 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
             const uint64_t N = td.n_unit;
             const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
             const uint64_t smoff = sm_offset(N, log2b);
-            const uint64_t payoff = smoff + pad16(N * SMB);
+            const uint64_t payoff = smoff + pad16(sm_section_bytes(N, DT));
             const uint8_t* msg = msgs + td.msg_off;
-            const uint8_t* pay = msg + payoff + (before << log2b);  // this tile's slice of the payload
+            const uint64_t pay_before = payload_bytes_of_blocks<DT>(before, log2b);
+            const uint8_t* pay = msg + payoff + pay_before;  // this tile's slice of the payload
             uint8_t* st = smem + (size_t)stage * kStageBytes;
             const bool full_tile = N - v0 >= (uint64_t)kTileValues;
             uint32_t lo = 1, hi = 0;
@@ -398,7 +418,7 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
             if (lane == 0) {
                 r->w_dst = weights + td.w_off;
                 r->c_ptr = cache + td.c_off;
-                r->sm_src = msg + smoff + v0 * SMB;
+                r->sm_src = msg + smoff + sm_bytes_of_values<DT>(v0);
                 r->pay_src = pay;
                 r->nv = (uint32_t)min((uint64_t)kTileValues, N - v0);
 
@@ -406,11 +426,12 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                 if (wire_bytes != nullptr && status != nullptr && td.tile_in_unit == td.n_tiles_unit - 1u) {
                     const uint32_t B = 1u << log2b;
                     const uint32_t nv = (uint32_t)(N - v0);
-                    uint64_t total = (before + own) << log2b;
+                    uint64_t total = payload_bytes_of_blocks<DT>(before + own, log2b);
                     const uint32_t rem = nv & (B - 1u);
-                    if (rem) {
+                    if (rem) {  // a changed short last block carries fewer bytes
                         const uint32_t kb = nv >> log2b;
-                        if ((r->bm[kb >> 5] >> (kb & 31u)) & 1u) total -= (B - rem);
+                        if ((r->bm[kb >> 5] >> (kb & 31u)) & 1u)
+                            total -= block_payload_bytes(B, DT) - block_payload_bytes(rem, DT);
                     }
                     if (wire_bytes[td.unit] != payoff + total) atomicCAS(status, 0, (int32_t)CIERA_ERR_CORRUPT);
                 }
@@ -421,15 +442,15 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                     // cache is 16-byte aligned; the slice stays inside the unit's payload section,
                     // which holds at least the values up to the end of this full tile)
                     uint32_t span0 = lo << log2b, span = lo <= hi ? (hi - lo + 1u) << log2b : 0u;
-                    uint32_t skew = 0, slice = own << log2b;
-                    if (FINE) {
-                        if (span) {
-                            const uint32_t end = (span0 + span + 15u) & ~15u;
-                            span0 &= ~15u;
-                            span = end - span0;
-                        }
+                    uint32_t skew = 0, slice = (uint32_t)payload_bytes_of_blocks<DT>(own, log2b);
+                    if (FINE && span) {
+                        const uint32_t end = (span0 + span + 15u) & ~15u;
+                        span0 &= ~15u;
+                        span = end - span0;
+                    }
+                    if (kSkew) {
                         if (slice) {
-                            skew = (uint32_t)((before << log2b) & 15ull);
+                            skew = (uint32_t)(pay_before & 15ull);
                             slice = (skew + slice + 15u) & ~15u;
                         }
                         r->pay_skew = skew;
@@ -480,15 +501,27 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                     // exponents: the cached ones, or -- changed block -- the ones that came in the payload
                     const uint32_t rank = r->pre[kb >> 5] + __popc(word & ((1u << (kb & 31u)) - 1u));
                     P x;
-                    x.template load_sm_full<Shared>(st + (size_t)t0 * SMB);
                     bool chg;
-                    if (!FINE) {
+                    if constexpr (kHalf) {
+                        // 11 packed bytes of sign-plus-mantissa; 5 packed bytes of exponents if the block changed
+                        x.template load_sm_group<Shared>(st, t0 >> 3, lane);
+                        chg = (word >> (kb & 31u)) & 1u;
+                        if (chg)
+                            x.template load_packed_exponents<Shared>(
+                                st + kSmTile + kTileValues + r->pay_skew + (size_t)payload_bytes_of_blocks<DT>(rank, log2b) +
+                                    5u * ((t0 & bmask) >> 3),
+                                P::kValues);
+                        else
+                            x.template load_exp_full<Shared>(st + kSmTile + t0);
+                    } else if (!FINE) {
+                        x.template load_sm_full<Shared>(st + (size_t)t0 * SMB);
                         chg = (word >> (kb & 31u)) & 1u;
                         const uint8_t* esrc = chg ? st + kSmTile + kTileValues + ((size_t)rank << log2b) + (t0 & bmask)
                                                   : st + kSmTile + t0;
                         x.template load_exp_full<Shared>(esrc);
                     } else {
                         // the piece's flags (they never straddle a word) pick, block by block
+                        x.template load_sm_full<Shared>(st + (size_t)t0 * SMB);
                         const uint32_t km = (word >> (kb & 31u)) & ((1u << (P::kValues >> log2b)) - 1u);
                         chg = km != 0;
                         x.template load_exp_full<Shared>(st + kSmTile + t0);
@@ -531,7 +564,20 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                     const bool chg = km != 0;
                     const uint8_t* esrc = (chg && !FINE) ? pay_src + ((size_t)rank << log2b) + (t0 & bmask) : c_ptr + t0;
                     P x;
-                    if (nvalid == P::kValues) {
+                    if constexpr (kHalf) {
+                        x.load_sm_bytes(sm_src + (size_t)11 * (t0 >> 3), nvalid);
+                        if (chg) {
+                            x.template load_packed_exponents<Global>(
+                                pay_src + (size_t)payload_bytes_of_blocks<DT>(rank, log2b) + 5u * ((t0 & bmask) >> 3), nvalid);
+                            x.store_exp_partial(c_ptr + t0, nvalid);
+                        } else {
+                            x.load_exp_partial(c_ptr + t0, nvalid);
+                        }
+                        if (nvalid == P::kValues)
+                            x.template merge_store_full<Global>(w_dst + (size_t)t0 * VB);
+                        else
+                            x.merge_store_partial(w_dst + (size_t)t0 * VB, nvalid);
+                    } else if (nvalid == P::kValues) {
                         x.template load_sm_full<Global>(sm_src + (size_t)t0 * SMB);
                         x.template load_exp_full<Global>(esrc);
                         if (FINE && chg) gather_changed<DT, Global>(x, km, log2b, pay_src + ((size_t)rank << log2b), nvalid);
@@ -672,7 +718,7 @@ template <int DT, bool FINE>
 static size_t decode_smem_bytes() {
     using Cfg = DecodeCfg<DT, FINE>;
     constexpr int S = Cfg::kStages;
-    const size_t stage = (size_t)kTileValues * Traits<DT>::kSmBytes + 2u * kTileValues + (FINE ? 16u : 0u);
+    const size_t stage = decode_stage_bytes<DT, FINE>();
     const size_t out = Cfg::kStageOut ? (size_t)kTileValues * Traits<DT>::kValueBytes : 0;
     return (size_t)S * stage + out + sizeof(DecodeCtl<S, Cfg::kRing, FINE>);
 }
@@ -752,8 +798,8 @@ extern "C" int ciera_decode(const ciera_plan* p, const void* messages_dev, void*
         if (rc) return rc;
     }
     if (p->dtype == CIERA_FP16)
-        return fp16_decode(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,
-                           (const uint32_t*)workspace_dev, status_dev, s);
+        return launch_decode<CIERA_FP16, false>(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,
+                                                workspace_dev, ticket, status_dev, s);
     const bool fine = is_fine(p->log2b);
     if (p->dtype == CIERA_BF16)
         return fine ? launch_decode<CIERA_BF16, true>(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,

@@ -64,6 +64,23 @@ struct Traits<CIERA_FP32> {
     static constexpr int kValueBytes = 4;
     static constexpr int kSmBytes = 3;
 };
+// fp16: 11 bits of sign-plus-mantissa and 5 exponent bits per value on the wire, so the byte
+// counts below hold for multiples of 8 values only (kSmBytes is not used for it)
+template <>
+struct Traits<CIERA_FP16> {
+    static constexpr int kValueBytes = 2;
+    static constexpr int kSmBytes = 0;
+};
+// bytes of sign-plus-mantissa of `values` values (a multiple of 8 for fp16), and payload bytes of
+// `blocks` full blocks
+template <int DT>
+__host__ __device__ constexpr uint64_t sm_bytes_of_values(uint64_t values) {
+    return DT == CIERA_FP16 ? (values >> 3) * 11 : values * Traits<DT>::kSmBytes;
+}
+template <int DT>
+__host__ __device__ constexpr uint64_t payload_bytes_of_blocks(uint64_t blocks, uint32_t log2b) {
+    return DT == CIERA_FP16 ? blocks * (5ull << (log2b - 3)) : blocks << log2b;
+}
 
 __host__ __device__ inline uint64_t pad16(uint64_t x) { return (x + 15ull) & ~15ull; }
 __host__ __device__ inline uint64_t num_blocks(uint64_t n, uint32_t log2b) {
@@ -151,8 +168,6 @@ namespace ciera {
 int fp16_cache_fill(const ciera_plan* p, void* cache_dev, const void* weights_dev, cudaStream_t s);
 int fp16_encode(const ciera_plan* p, const void* weights_dev, void* sender_cache_dev, void* messages_dev,
                 uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* workspace_dev, cudaStream_t s);
-int fp16_decode(const ciera_plan* p, const void* messages_dev, void* receiver_cache_dev, void* weights_out_dev,
-                const uint64_t* wire_bytes_dev, const uint32_t* ws_prefix, int32_t* status_dev, cudaStream_t s);
 int record_cuda_error(cudaError_t e);          // stores e for ciera_last_cuda_error, returns CIERA_ERR_CUDA
 void count_launch();                           // launch accounting
 int check_launch();                            // cudaGetLastError -> status
