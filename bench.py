@@ -245,10 +245,9 @@ def algorithmic_bytes(n_values, q, dtype, block, detect="compare"):
     vb, smb = (2, 1) if dtype == "bf16" else (4, 3)
     bm = 1.0 / (8 * block)
     if dtype == "fp16":
-        # packed on the wire (11 and 5 bits per value), one byte per value in the caches; the sender
-        # reads the weights of changed blocks a second time
+        # packed on the wire (11 and 5 bits per value), one byte per value in the caches
         sm, ex = 11 / 8, 5 / 8
-        enc = n_values * (2 + 1 + sm + bm + q * (ex + 1 + 2))
+        enc = n_values * (2 + 1 + sm + bm + q * (ex + 1))
         tra = 2 * n_values * (sm + bm + q * ex)
         dec = n_values * (sm + bm + (1 - q) + q * ex + 2 + q)
         return enc, tra, dec
@@ -576,7 +575,7 @@ def main():
                                  "per": "layer launch inside the two-stream timed region (kernels overlap)"},
         "serial_ms_per_step": serial_ms_per_step,
         "roofline": {
-            "bound": "hbm", "kernel": ("fp16 encode (scan + unit + payload launches)" if args.dtype == "fp16" else "encode_kernel" if args.detect == "compare" else "hashed encode (scan + unit + payload launches)"), "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
+            "bound": "hbm", "kernel": ("encode_kernel" if args.detect == "compare" else "hashed encode (scan + unit + payload launches)"), "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
             "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBps": enc_gbs / NOMINAL_HBM_GBS,
             "traffic": (NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE * n_layer
                         if args.dtype == "bf16" and args.block == 512 and args.update == "clustered" else None),
@@ -598,7 +597,7 @@ def main():
         out["selection"] = selection_report(args, ciera, layers[-1], enc_ms, dec_ms)
 
     # ---- per-kernel numbers with each kernel alone on the GPU, three change regimes (one layer)
-    if not args.no_regimes and rank == 0 and args.detect == "compare" and args.dtype != "fp16":
+    if not args.no_regimes and rank == 0 and args.detect == "compare":
         out["kernels_alone"] = kernels_alone(args, layers[0], wa[0], wb[0], peak)
 
     # ---- end to end through the host-buffer entry point (weights start and end in host memory)
@@ -636,11 +635,13 @@ def kernels_alone(args, codec, w_a, w_b, peak):
     import torch
 
     res = {}
-    vb = 2 if args.dtype == "bf16" else 4
+    vb = 4 if args.dtype == "fp32" else 2
     n = codec.plan.total_values
     # lowest exponent bit flipped everywhere: every block changes
-    if vb == 2:
+    if args.dtype == "bf16":
         w_c = (w_a.view(torch.int16) ^ 0x0080).view(torch.uint8)
+    elif args.dtype == "fp16":
+        w_c = (w_a.view(torch.int16) ^ 0x0400).view(torch.uint8)
     else:
         w_c = (w_a.view(torch.int32) ^ 0x00800000).view(torch.uint8)
 

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libciera.so")
-SOURCES = ["ciera_host.cu", "ciera_encode.cu", "ciera_encode_hashed.cu", "ciera_decode.cu", "ciera_entropy.cu", "ciera_fp16.cu", "ciera_kernels.cu"]
+SOURCES = ["ciera_host.cu", "ciera_encode.cu", "ciera_encode_hashed.cu", "ciera_decode.cu", "ciera_entropy.cu", "ciera_kernels.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
     "-lineinfo", "-O3", "-std=c++17",

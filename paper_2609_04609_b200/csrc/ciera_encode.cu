@@ -66,6 +66,13 @@ struct EncodeCfg<CIERA_FP32, false> {
     static constexpr int kBmWords = kBitmapWords;
 };
 template <>
+struct EncodeCfg<CIERA_FP16, false> {  // as bf16: 16 KB weights tiles, 8 KB exponent tiles
+    static constexpr int kWStages = 3;
+    static constexpr int kEStages = 7;
+    static constexpr int kDefer = 3;
+    static constexpr int kBmWords = kBitmapWords;
+};
+template <>
 struct EncodeCfg<CIERA_BF16, true> {
     static constexpr int kWStages = 3;
     static constexpr int kEStages = 6;
@@ -192,11 +199,11 @@ __device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t 
                               : build_block_bitmap(ballot, bm, pre, log2b, Piece<DT>::kLog2Values, lane);
 
     // payload bytes of this tile: B per changed block, less for a changed short last block
-    uint64_t agg = (uint64_t)run << log2b;
+    uint64_t agg = payload_bytes_of_blocks<DT>(run, log2b);
     const uint32_t rem = nv & (B - 1u);
     if (rem) {
         const uint32_t kb = nv >> log2b;
-        if ((bm[kb >> 5] >> (kb & 31u)) & 1u) agg -= (B - rem);
+        if ((bm[kb >> 5] >> (kb & 31u)) & 1u) agg -= block_payload_bytes(B, DT) - block_payload_bytes(rem, DT);
     }
     if (publish) {
         // a unit's first tile knows its prefix (0) already
@@ -237,10 +244,26 @@ __device__ __forceinline__ void write_changed(const EncodeTileInfo& ti, uint32_t
         const uint32_t word = bm[kb >> 5];
         if (!((word >> (kb & 31u)) & 1u)) continue;
         const uint32_t rank = pre[kb >> 5] + __popc(word & ((1u << (kb & 31u)) - 1u));
-        uint8_t* pdst = ti.pay_dst + base + ((uint64_t)rank << log2b) + (t0 & ((1u << log2b) - 1u));
         uint8_t* cdst = ti.c_ptr + t0;
         P x;
         x.template load_exp_full<Shared>(s_exp + t0);
+        if constexpr (DT == CIERA_FP16) {
+            // five packed bytes per piece (fewer for the unit's last, short piece), byte by byte
+            uint8_t* pdst = ti.pay_dst + base + payload_bytes_of_blocks<DT>(rank, log2b) +
+                            5u * ((t0 & ((1u << log2b) - 1u)) >> 3);
+            uint32_t lo, hi;
+            x.pack_exponents(lo, hi);
+            const int nbytes = (5 * nvalid + 7) >> 3;
+#pragma unroll
+            for (int i = 0; i < 5; ++i)
+                if (i < nbytes) pdst[i] = (uint8_t)(i < 4 ? lo >> (8 * i) : hi);
+            if (nvalid == P::kValues)
+                x.template store_exp_full<Global>(cdst);
+            else
+                x.store_exp_partial(cdst, nvalid);
+            continue;
+        }
+        uint8_t* pdst = ti.pay_dst + base + ((uint64_t)rank << log2b) + (t0 & ((1u << log2b) - 1u));
         if (nvalid == P::kValues) {
             x.template store_exp_full<Global>(pdst);
             x.template store_exp_full<Global>(cdst);
@@ -405,8 +428,8 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
                 {
                     const uint64_t smoff = sm_offset(td.n_unit, log2b);
                     EncodeTileInfo ti;
-                    ti.sm_dst = msgs + td.msg_off + smoff + v0 * SMB;
-                    ti.pay_dst = msgs + td.msg_off + smoff + pad16(td.n_unit * SMB);
+                    ti.sm_dst = msgs + td.msg_off + smoff + sm_bytes_of_values<DT>(v0);
+                    ti.pay_dst = msgs + td.msg_off + smoff + pad16(sm_section_bytes(td.n_unit, DT));
                     ti.c_ptr = cache + td.c_off;
                     ti.w_src = weights + td.w_off;
                     ti.nv = (uint32_t)min((uint64_t)kTileValues, left);
@@ -526,7 +549,7 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
                     // leave the new exponents where the cached ones were staged: they are sent from
                     // there once the tile's place in the payload is known
                     x.template store_exp_full<Shared>(s_e + t0);
-                    if (!FINE) {
+                    if constexpr (!FINE) {
                         const uint32_t bal = __ballot_sync(0xffffffffu, x.differs(c));
                         if (lane == 0) ctl->ballot[se][p * kWarps + warp] = bal;
                     } else {
@@ -546,11 +569,20 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
                         }
                     }
                     // sign-plus-mantissa of every value
-                    uint8_t* smdst = ti.sm_dst + (size_t)t0 * SMB;
-                    if (nvalid == P::kValues)
-                        x.template store_sm_full<Global>(smdst);
-                    else if (nvalid > 0)
-                        x.store_sm_partial(smdst, nvalid);
+                    if constexpr (DT == CIERA_FP16) {
+                        // packed: whole groups of four lanes in a full tile (every lane takes part in the
+                        // group's shuffle), else byte by byte
+                        if (nv == (uint32_t)kTileValues)
+                            x.store_sm_group(ti.sm_dst, t0 >> 3, lane);
+                        else if (nvalid > 0)
+                            x.store_sm_bytes(ti.sm_dst + (size_t)11 * (t0 >> 3), nvalid);
+                    } else {
+                        uint8_t* smdst = ti.sm_dst + (size_t)t0 * SMB;
+                        if (nvalid == P::kValues)
+                            x.template store_sm_full<Global>(smdst);
+                        else if (nvalid > 0)
+                            x.store_sm_partial(smdst, nvalid);
+                    }
                 }
                 __syncwarp();  // the warp's shared-memory accesses above are ordered before lane 0's arrives
                 if (lane == 0) {
@@ -686,6 +718,9 @@ static int launch_encode_any(const ciera_plan* p, const void* weights_dev, void*
                              uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* scratch, int32_t* status_dev,
                              cudaStream_t s) {
     const bool fine = is_fine(p->log2b);
+    if (p->dtype == CIERA_FP16)
+        return launch_encode<CIERA_FP16, false>(p, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
+                                                changed_blocks_dev, scratch, status_dev, s);
     if (p->dtype == CIERA_BF16)
         return fine ? launch_encode<CIERA_BF16, true>(p, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
                                                       changed_blocks_dev, scratch, status_dev, s)
@@ -724,9 +759,6 @@ extern "C" int ciera_encode(const ciera_plan* p, const void* weights_dev, void* 
     if (misaligned16(weights_dev) || misaligned16(sender_cache_dev) || misaligned16(messages_dev) ||
         misaligned16(workspace_dev) || ((uintptr_t)wire_bytes_dev & 7u) || ((uintptr_t)changed_blocks_dev & 3u))
         return CIERA_ERR_MISALIGNED;
-    if (p->dtype == CIERA_FP16)  // three plain launches; the scratch needs no clearing
-        return fp16_encode(p, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev, changed_blocks_dev,
-                           workspace_dev, s);
     // scratch = one look-back status word per tile, then the unit counter; all of it starts at zero
     e = cudaMemsetAsync(workspace_dev, 0, sizeof(unsigned long long) * nt + 16, s);
     if (e != cudaSuccess) return record_cuda_error(e);
@@ -776,7 +808,6 @@ extern "C" int ciera_encode_noalloc(const ciera_plan* p, const void* weights_dev
     if (!p->tiles.empty() && !p->tiles_dev) return CIERA_ERR_NOT_BOUND;
     const uint32_t nt = (uint32_t)p->tiles.size();
     if (nt > CIERA_NOALLOC_MAX_TILES) return CIERA_ERR_TOO_LARGE;
-    if (p->dtype == CIERA_FP16) return CIERA_ERR_UNSUPPORTED;
     if (p->n_units == 0) return CIERA_OK;
     if (!wire_bytes_dev || !changed_blocks_dev) return CIERA_ERR_INVALID_ARG;
     cudaStream_t s = (cudaStream_t)stream;

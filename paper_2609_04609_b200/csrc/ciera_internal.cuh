@@ -164,10 +164,6 @@ struct ciera_plan {
 };
 
 namespace ciera {
-// fp16 takes kernels of its own (ciera_fp16.cu)
-int fp16_cache_fill(const ciera_plan* p, void* cache_dev, const void* weights_dev, cudaStream_t s);
-int fp16_encode(const ciera_plan* p, const void* weights_dev, void* sender_cache_dev, void* messages_dev,
-                uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* workspace_dev, cudaStream_t s);
 int record_cuda_error(cudaError_t e);          // stores e for ciera_last_cuda_error, returns CIERA_ERR_CUDA
 void count_launch();                           // launch accounting
 int check_launch();                            // cudaGetLastError -> status

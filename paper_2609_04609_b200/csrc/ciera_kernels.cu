@@ -253,8 +253,9 @@ static int cache_fill(const ciera_plan* p, void* cache_dev, const void* weights_
     const uint32_t nt = (uint32_t)p->tiles.size();
     if (nt == 0) return CIERA_OK;
     cudaStream_t s = (cudaStream_t)stream;
-    if (p->dtype == CIERA_FP16) return fp16_cache_fill(p, cache_dev, weights_dev, s);
-    if (p->dtype == CIERA_BF16)
+    if (p->dtype == CIERA_FP16)
+        cache_fill_kernel<CIERA_FP16><<<nt, kThreads, 0, s>>>(p->tiles_dev, (const uint8_t*)weights_dev, (uint8_t*)cache_dev);
+    else if (p->dtype == CIERA_BF16)
         cache_fill_kernel<CIERA_BF16><<<nt, kThreads, 0, s>>>(p->tiles_dev, (const uint8_t*)weights_dev, (uint8_t*)cache_dev);
     else
         cache_fill_kernel<CIERA_FP32><<<nt, kThreads, 0, s>>>(p->tiles_dev, (const uint8_t*)weights_dev, (uint8_t*)cache_dev);

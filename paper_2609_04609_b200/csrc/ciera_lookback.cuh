@@ -46,18 +46,23 @@ __device__ __forceinline__ uint64_t warp_sum_u64(uint64_t v) {
 template <int DT>
 __device__ __forceinline__ void finish_unit(const TileDesc& td, uint32_t log2b, uint64_t total, uint8_t* msgs,
                                             unsigned long long* wire_bytes, uint32_t* changed_blocks, uint32_t lane) {
-    constexpr int SMB = Traits<DT>::kSmBytes;
     const uint64_t N = td.n_unit;
-    const uint32_t B = 1u << log2b;
     uint8_t* msg = msgs + td.msg_off;
     const uint64_t smoff = sm_offset(N, log2b);
-    const uint64_t payoff = smoff + pad16(N * SMB);
+    const uint64_t sm_bytes = sm_section_bytes(N, DT);
+    const uint64_t payoff = smoff + pad16(sm_bytes);
     if (lane == 0) {
         wire_bytes[td.unit] = payoff + total;
-        changed_blocks[td.unit] = (uint32_t)((total + B - 1u) >> log2b);
+        // every changed block carries a full block's bytes except possibly the last one, which carries fewer
+        if (DT == CIERA_FP16) {
+            const uint64_t bpb = payload_bytes_of_blocks<DT>(1, log2b);
+            changed_blocks[td.unit] = (uint32_t)((total + bpb - 1u) / bpb);
+        } else {
+            changed_blocks[td.unit] = (uint32_t)((total + (1ull << log2b) - 1u) >> log2b);
+        }
     }
     for (uint64_t b = bitmap_bytes(N, log2b) + lane; b < smoff; b += 32) msg[b] = 0;
-    for (uint64_t b = smoff + N * SMB + lane; b < payoff; b += 32) msg[b] = 0;
+    for (uint64_t b = smoff + sm_bytes + lane; b < payoff; b += 32) msg[b] = 0;
 }
 
 // Resolver warp, one spread tile: exclusive prefix of the payload bytes over the earlier tiles of
