@@ -145,9 +145,7 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
             t.n_tiles_unit = nt;
             p->tiles.push_back(t);
         }
-        const bool needs_prefix = (is_fine(p->log2b) || dtype == CIERA_FP16)
-                                      ? nt > 1
-                                      : (un.n_values + block - 1) / block > kDecodeDirectBlocks;
+        const bool needs_prefix = is_fine(p->log2b) ? nt > 1 : (un.n_values + block - 1) / block > kDecodeDirectBlocks;
         if (needs_prefix) p->long_units.push_back(first);
     };
     for (uint32_t u : shorts) {
@@ -208,9 +206,8 @@ extern "C" const void* ciera_plan_host_image(const ciera_plan* p) { return p ? p
 
 extern "C" size_t ciera_plan_workspace_bytes(const ciera_plan* p) {
     if (!p) return 0;
-    // one look-back status word per tile + the ticket counter; fp16: a record of 18 words per tile
-    const size_t per_tile = p->dtype == CIERA_FP16 ? 18 * sizeof(uint32_t) : sizeof(unsigned long long);
-    return p->tiles.size() * per_tile + 16;
+    // one look-back status word per tile + the ticket counter
+    return p->tiles.size() * sizeof(unsigned long long) + 16;
 }
 
 extern "C" size_t ciera_plan_hash_cache_bytes(const ciera_plan* p) { return p ? (size_t)p->total_blocks * 16 : 0; }
