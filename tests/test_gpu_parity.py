@@ -335,3 +335,31 @@ def test_full_size_layer_sampled_units(rt, dtype, block):
         prev = cur
     q = int(codec.changed_blocks.sum().item()) / codec.n_blocks()
     assert q > (0.99 if block >= 256 else 0.8)  # the i.i.d. step changes (nearly) every block
+
+
+@pytest.mark.parametrize("sizes", [[], [0], [0, 0, 0]])
+@pytest.mark.parametrize("dtype_name", ["bf16", "fp32", "fp16"])
+def test_tables_without_values_run_through_every_entry_point(rt, sizes, dtype_name):
+    """No units, or only units without values: every call returns without touching anything."""
+    ciera, runtime = rt
+    codec = runtime.LayerCodec.from_tensors(sizes, 1, dtype_name, 64, DEV)
+    w = torch.zeros(16, dtype=torch.uint8, device=DEV)
+    codec.init_caches(None)
+    codec.init_caches(w)
+    launches0 = ciera.kernel_launch_count()
+    codec.step(w)
+    ciera.encode_noalloc(codec.plan, w, codec.sender_cache, codec.msg_send, codec.wire_bytes, codec.changed_blocks,
+                         codec.status)
+    if dtype_name != "fp16":
+        codec.init_hash_cache(None)
+        codec.encode_hashed(w)
+        codec.entropy_encode()
+        codec.entropy_decode()
+    host_in = torch.zeros(16, dtype=torch.uint8).pin_memory()
+    host_out = torch.zeros(16, dtype=torch.uint8).pin_memory()
+    wire_host = torch.zeros(max(len(codec.units), 1), dtype=torch.int64).pin_memory()
+    codec.step_host(host_in, host_out, w, wire_host)
+    torch.cuda.synchronize()
+    codec.check_status()
+    assert int(codec.wire_bytes.sum().item()) == 0 and int(codec.changed_blocks.sum().item()) == 0
+    assert ciera.kernel_launch_count() - launches0 <= 2  # at most the hashed sender's per-unit pass
