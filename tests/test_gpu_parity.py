@@ -363,3 +363,24 @@ def test_tables_without_values_run_through_every_entry_point(rt, sizes, dtype_na
     codec.check_status()
     assert int(codec.wire_bytes.sum().item()) == 0 and int(codec.changed_blocks.sum().item()) == 0
     assert ciera.kernel_launch_count() - launches0 <= 2  # at most the hashed sender's per-unit pass
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("block", [1, 64, 512])
+def test_tightly_packed_layout_in_shuffled_order(rt, dtype, block):
+    """Buffers laid out with the minimum alignment (16 bytes) and the units of the table listed in a
+    shuffled order: every offset the kernels derive must hold without the 256-byte padding of the
+    other tests."""
+    ciera, runtime = rt
+    sizes = [8192 * 2 + 24, 100, 70_001, 8, 40_000, 8192, 12_345, 0, 131_072]
+    code = dtype
+    units, wb, cb, mb = wl.layout_units(sizes, 1, 2 if dtype == 0 else 4,
+                                        lambda n: ciera.message_capacity(n, code, block), align=16)
+    rng = np.random.default_rng(12 + block)
+    units = units[rng.permutation(len(units))]
+    codec = runtime.LayerCodec(units, NAME[dtype], block, wb, cb, mb, DEV)
+    table = OracleTable(codec.units, dtype, block, codec.cache_bytes, codec.msg_bytes)
+    n = wb // (2 if dtype == 0 else 4)
+    traj = [wl.as_bits(w) for w in wl.trajectory(n, NAME[dtype], 90 + block, 2, "adam")]
+    _run_trajectory(rt, codec, table, traj, dtype, label=f"tight-{NAME[dtype]}-B{block}")
+    _run_trajectory(rt, codec, table, traj[:2], dtype, zero_cache=True, label=f"tight-zero-{NAME[dtype]}-B{block}")
