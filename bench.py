@@ -241,7 +241,8 @@ def selection_report(args, ciera, codec, enc_ms, dec_ms, alpha=20e-6, beta=8e9):
 def algorithmic_bytes(n_values, q, dtype, block, detect="compare"):
     """HBM bytes per launch the method needs: (encode, transport, decode).  q = share of the
     exponent bytes that travel (changed blocks); the bitmap is one bit per block.  The hashed sender
-    reads no exponent cache but reads the weights of changed blocks twice and keeps 16 bytes per block."""
+    reads no exponent cache and writes none; it reads 16 bytes of HashCache per block and writes them back
+    for the changed ones."""
     vb, smb = (2, 1) if dtype == "bf16" else (4, 3)
     bm = 1.0 / (8 * block)
     if dtype == "fp16":
@@ -252,7 +253,7 @@ def algorithmic_bytes(n_values, q, dtype, block, detect="compare"):
         dec = n_values * (sm + bm + (1 - q) + q * ex + 2 + q)
         return enc, tra, dec
     if detect == "hash":
-        enc = n_values * (vb + smb + bm + q * (vb + 1) + 16.0 * (1 + q) / block)
+        enc = n_values * (vb + smb + bm + q + 16.0 * (1 + q) / block)
     else:
         enc = n_values * (vb + 1 + smb + bm + 2 * q)
     tra = 2 * n_values * (smb + bm + q)
@@ -360,7 +361,7 @@ def workload_config(args):
         "schedule": args.schedule,
         "round_trip": "encode + device-to-device transport + decode",
         "change_detection": "exact comparison with a sender-side exponent cache" if args.detect == "compare"
-                            else "128-bit hash per block (HashCache), three launches per encode",
+                            else "128-bit hash per block (HashCache), the persistent kernel in its HashCache form",
     }
 
 
@@ -575,7 +576,7 @@ def main():
                                  "per": "layer launch inside the two-stream timed region (kernels overlap)"},
         "serial_ms_per_step": serial_ms_per_step,
         "roofline": {
-            "bound": "hbm", "kernel": ("encode_kernel" if args.detect == "compare" else "hashed encode (scan + unit + payload launches)"), "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
+            "bound": "hbm", "kernel": ("encode_kernel" if args.detect == "compare" else "encode_kernel (HashCache form)"), "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
             "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBps": enc_gbs / NOMINAL_HBM_GBS,
             "traffic": (NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE * n_layer
                         if args.dtype == "bf16" and args.block == 512 and args.update == "clustered" else None),

@@ -214,7 +214,7 @@ CIERA_API int ciera_encode_noalloc(const ciera_plan* plan, const void* weights_d
  * Blocks of 16 values and more only (CIERA_ERR_UNSUPPORTED otherwise). */
 
 /* Bytes of a HashCache for the whole plan (16 per block; units in table order), the offset of a
- * unit's first block in it, and the scratch ciera_encode_hashed needs (72 bytes per tile + 16). */
+ * unit's first block in it, and the scratch ciera_encode_hashed needs (8 bytes per tile + 16). */
 CIERA_API size_t ciera_plan_hash_cache_bytes(const ciera_plan* plan);
 CIERA_API size_t ciera_plan_unit_hash_offset(const ciera_plan* plan, uint32_t unit);
 CIERA_API size_t ciera_plan_hashed_workspace_bytes(const ciera_plan* plan);
@@ -224,13 +224,12 @@ CIERA_API size_t ciera_plan_hashed_workspace_bytes(const ciera_plan* plan);
  * 16-byte aligned.  Asynchronous on `stream`. */
 CIERA_API int ciera_hash_cache_init(const ciera_plan* plan, void* hash_cache_dev, const void* weights_dev, void* stream);
 
-/* Sender step with HashCache.  Arguments as for ciera_encode, with hash_cache_dev (in/out,
- * ciera_plan_hash_cache_bytes) in place of the exponent cache and a scratch of
- * ciera_plan_hashed_workspace_bytes (contents need not be initialised).  Three kernel launches on
- * `stream`; nothing waits inside the kernels, so there is no status word. */
+/* Sender step with HashCache.  Arguments, launch (one persistent kernel) and error behaviour as
+ * for ciera_encode, with hash_cache_dev (in/out, ciera_plan_hash_cache_bytes) in place of the
+ * exponent cache and a scratch of ciera_plan_hashed_workspace_bytes (cleared by the call). */
 CIERA_API int ciera_encode_hashed(const ciera_plan* plan, const void* weights_dev, void* hash_cache_dev,
                                   void* messages_dev, uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev,
-                                  void* workspace_dev, void* stream);
+                                  void* workspace_dev, int32_t* status_dev, void* stream);
 
 /* ---- transport stand-in: Send / Recv of Algorithm 1 on one GPU ----------------------------- */
 

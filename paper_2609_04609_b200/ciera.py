@@ -76,7 +76,7 @@ _SIGS = {
     "ciera_plan_unit_hash_offset": ([_vp, _u32], _sz),
     "ciera_plan_hashed_workspace_bytes": ([_vp], _sz),
     "ciera_hash_cache_init": ([_vp] * 4, _i32),
-    "ciera_encode_hashed": ([_vp] * 8, _i32),
+    "ciera_encode_hashed": ([_vp] * 9, _i32),
     "ciera_plan_entropy_scratch_bytes": ([_vp], _sz),
     "ciera_entropy_encode": ([_vp] * 5, _i32),
     "ciera_entropy_decode": ([_vp] * 6, _i32),
@@ -239,12 +239,13 @@ def hash_cache_init(plan: Plan, hash_cache: torch.Tensor, weights: Optional[torc
            _lib.ciera_hash_cache_init(plan.handle, _ptr(hash_cache), _ptr(weights), _stream(stream)))
 
 
-def encode_hashed(plan: Plan, weights, hash_cache, messages, wire_bytes, changed_blocks, workspace, stream=None) -> None:
+def encode_hashed(plan: Plan, weights, hash_cache, messages, wire_bytes, changed_blocks, workspace, status=None,
+                  stream=None) -> None:
     """Sender step with a 128-bit hash per block in place of the exponent cache (blocks of 16 values
     and more); ``workspace`` holds ``plan.hashed_workspace_bytes``."""
     _check("ciera_encode_hashed",
            _lib.ciera_encode_hashed(plan.handle, _ptr(weights), _ptr(hash_cache), _ptr(messages), _ptr(wire_bytes),
-                                    _ptr(changed_blocks), _ptr(workspace), _stream(stream)))
+                                    _ptr(changed_blocks), _ptr(workspace), _ptr(status), _stream(stream)))
 
 
 def entropy_encode(plan: Plan, messages, wire_bytes, scratch, stream=None) -> None:

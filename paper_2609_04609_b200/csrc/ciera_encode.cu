@@ -32,7 +32,15 @@
 // Only the resolvers ever wait for another thread block; the aggregator never does, and the
 // consumers only for a resolver that is several tiles late, so a tile's status is published as
 // soon as its votes are in.
+//
+// The same kernel serves the sender that keeps HashCache (a 128-bit hash per block, Section 3.1 and
+// Algorithm 1 as printed) instead of the previous exponents (template flag HASH): the producer then
+// stages the tile's cached hashes instead of cached exponents, the consumers turn their exponents
+// into hash terms and add them up over the lanes that share a block, and the aggregator finishes
+// the hashes, compares them with the cached ones, refreshes HashCache and derives the block flags
+// from the comparison.
 #include "ciera_bits.cuh"
+#include "ciera_hash.cuh"
 #include "ciera_lookback.cuh"
 #include "ciera_pipe.cuh"
 
@@ -87,12 +95,54 @@ struct EncodeCfg<CIERA_FP32, true> {
     static constexpr int kBmWords = kFineBitmapWords;
 };
 
+// With HashCache the exponent ring stages no cached exponents (it only keeps the new ones until
+// they are sent), so it is shorter; each of its stages has a companion with the tile's cached
+// hashes and the consumers' partial sums, sized at launch from the block size.
+template <int DT>
+struct EncodeHashCfg;
+template <>
+struct EncodeHashCfg<CIERA_BF16> {
+    static constexpr int kWStages = 3;
+    static constexpr int kEStages = 6;
+    static constexpr int kDefer = 3;
+    static constexpr int kBmWords = kBitmapWords;
+};
+template <>
+struct EncodeHashCfg<CIERA_FP32> {
+    static constexpr int kWStages = 2;
+    static constexpr int kEStages = 4;
+    static constexpr int kDefer = 2;
+    static constexpr int kBmWords = kBitmapWords;
+};
+template <int DT, bool FINE, bool HASH>
+struct EncodeCfgOf {
+    using type = EncodeCfg<DT, FINE>;
+};
+template <int DT>
+struct EncodeCfgOf<DT, false, true> {
+    using type = EncodeHashCfg<DT>;
+};
+
+// Shared-memory bytes of the cached hashes (`hold`) and of the partial sums (`part`) of one tile:
+// 16 bytes per block, and 16 bytes per group of lanes that add up their terms (a block's lanes, at
+// most a warp).
+template <int DT>
+__host__ __device__ constexpr uint32_t hash_hold_bytes(uint32_t log2b) {
+    return (uint32_t)(kTileValues >> log2b) * 16u;
+}
+template <int DT>
+__host__ __device__ constexpr uint32_t hash_part_bytes(uint32_t log2b) {
+    const uint32_t nbt = (uint32_t)kTileValues >> log2b;
+    const uint32_t warps = (uint32_t)kTileValues >> (5 + Piece<DT>::kLog2Values);  // warp-sized groups of pieces
+    return (nbt > warps ? nbt : warps) * 16u;
+}
+
 // What the consumers need of a tile, worked out once by the producer thread instead of by each
 // of the 512 consumer threads.
 struct __align__(16) EncodeTileInfo {
     uint8_t* sm_dst;       // where the tile's sign-plus-mantissa goes
     uint8_t* pay_dst;      // start of the unit's payload section
-    uint8_t* c_ptr;        // the tile's cached exponents
+    uint8_t* c_ptr;        // the tile's cached exponents (with HashCache: the cached hash of the tile's first block)
     const uint8_t* w_src;  // the tile's weights
     uint32_t nv;           // values in the tile
     uint32_t pad[3];
@@ -184,10 +234,96 @@ __device__ __forceinline__ uint32_t scan_block_bitmap(const uint32_t* bm, uint16
 // Aggregator warp, one tile: block flags, the tile's bitmap bytes, the tile's payload byte count.
 // With `publish` the count goes out at once as the tile's status word, so that later tiles never
 // wait for it longer than for the votes themselves.  Waits for nothing outside the thread block.
-template <int DT, bool FINE>
+// HashCache: block flags of a tile from the consumers' partial sums.  Lane i of a round takes one
+// block: adds up the block's partial sums, finishes the two hashes, compares them with the cached
+// pair and, where they differ, flags the block and stores the new pair (HashCache[i,k] <- h).
+// Returns the number of flagged blocks (one warp).
+template <int DT>
+__device__ __forceinline__ uint32_t hash_block_bitmap(const ulonglong2* part, const ulonglong2* hold, ulonglong2* hash_dst,
+                                                      uint32_t* bm, uint16_t* pre, uint32_t log2b, uint32_t nv,
+                                                      uint32_t lane) {
+    constexpr uint32_t kGroupL2 = 5 + Piece<DT>::kLog2Values;  // log2(values of a warp's pieces)
+    const uint32_t B = 1u << log2b;
+    const uint32_t nbt = kTileValues >> log2b;
+    const uint32_t nblk = (nv + B - 1u) >> log2b;
+    const uint32_t epb_l2 = log2b > kGroupL2 ? log2b - kGroupL2 : 0u;  // log2(partial sums per block)
+    uint32_t run = 0;
+    for (uint32_t base = 0; base < nbt; base += 32) {
+        const uint32_t i = base + lane;
+        bool f = false;
+        if (i < nblk) {
+            uint64_t a = 0, b = 0;
+            for (uint32_t e = 0; e < (1u << epb_l2); ++e) {
+                const ulonglong2 v = part[(i << epb_l2) + e];
+                a += v.x;
+                b += v.y;
+            }
+            const ulonglong2 h = hash_finish(a, b, min(B, nv - (i << log2b)));
+            const ulonglong2 old = hold[i];
+            f = h.x != old.x || h.y != old.y;
+            if (f) hash_dst[i] = h;
+        }
+        const uint32_t word = __ballot_sync(0xffffffffu, f);
+        if (lane == 0) {
+            bm[base >> 5] = word;
+            pre[base >> 5] = (uint16_t)run;
+        }
+        run += __popc(word);
+    }
+    __syncwarp();
+    return run;
+}
+
+// HashCache, consumers: adds up the pieces' sums of terms (a[p], b[p]: the two hashes' sums of piece
+// p of this thread) over groups of 2^l2 neighbouring lanes -- the lanes whose pieces lie in one block,
+// at most the warp -- and stores the group's totals as entry e0 (piece 0) and e1 (the thread's last
+// piece) of `part`, two 64-bit words each.  Instead of one butterfly per sum, the first exchanges
+// hand every lane fewer sums to carry on with (odd lanes keep the b's, even lanes the a's; then lanes
+// with bit 1 set keep the second piece's): 6 shuffles of 64 bits for four sums over a warp, not 20.
+template <int NP>
+__device__ __forceinline__ void reduce_hash_terms(const uint64_t* a, const uint64_t* b, uint32_t l2, uint32_t e0, uint32_t e1,
+                                                  uint64_t* part, uint32_t lane) {
+    const bool odd = (lane & 1u) != 0;
+    if (l2 == 0) {  // every lane a block of its own (NP = 1: a piece is a whole block at least)
+        part[2 * e0] = a[0];
+        part[2 * e0 + 1] = b[0];
+        return;
+    }
+    uint64_t k0 = (odd ? b[0] : a[0]) + __shfl_xor_sync(0xffffffffu, odd ? a[0] : b[0], 1);
+    if constexpr (NP == 1) {
+#pragma unroll
+        for (uint32_t o = 1; o < 5; ++o)
+            if (o < l2) k0 += __shfl_xor_sync(0xffffffffu, k0, 1u << o);
+        const uint32_t r = lane & ((1u << l2) - 1u);
+        if (r < 2) part[2 * e0 + r] = k0;  // lane 0 of the group: sum of a, lane 1: sum of b
+    } else {
+        uint64_t k1 = (odd ? b[1] : a[1]) + __shfl_xor_sync(0xffffffffu, odd ? a[1] : b[1], 1);
+        if (l2 == 1) {  // groups of two lanes
+            part[2 * e0 + (odd ? 1u : 0u)] = k0;
+            part[2 * e1 + (odd ? 1u : 0u)] = k1;
+            return;
+        }
+        const bool second = (lane & 2u) != 0;
+        uint64_t t = (second ? k1 : k0) + __shfl_xor_sync(0xffffffffu, second ? k0 : k1, 2);
+#pragma unroll
+        for (uint32_t o = 2; o < 5; ++o)
+            if (o < l2) t += __shfl_xor_sync(0xffffffffu, t, 1u << o);
+        const uint32_t r = lane & ((1u << l2) - 1u);
+        if (r < 4) part[2 * ((r & 2u) ? e1 : e0) + (r & 1u)] = t;  // lanes 0..3: a of piece 0, b of piece 0, a, b of piece 1
+    }
+}
+
+// what aggregate_tile needs besides the votes when the sender keeps HashCache
+struct HashTile {
+    const ulonglong2* part;
+    const ulonglong2* hold;
+    ulonglong2* dst;
+};
+
+template <int DT, bool FINE, bool HASH>
 __device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t tile, uint32_t log2b, bool publish,
                                                    const uint32_t* ballot, uint32_t* bm, uint16_t* pre, uint8_t* msgs,
-                                                   unsigned long long* tile_status, uint32_t lane) {
+                                                   unsigned long long* tile_status, const HashTile& ht, uint32_t lane) {
     const uint64_t N = td.n_unit;
     const uint32_t B = 1u << log2b;
     const uint32_t nbt = kTileValues >> log2b;
@@ -195,8 +331,12 @@ __device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t 
     const uint32_t nv = (uint32_t)min((uint64_t)kTileValues, N - v0);
     uint8_t* msg = msgs + td.msg_off;
 
-    const uint32_t run = FINE ? scan_block_bitmap(bm, pre, log2b, lane)
-                              : build_block_bitmap(ballot, bm, pre, log2b, Piece<DT>::kLog2Values, lane);
+    uint32_t run;
+    if constexpr (HASH)
+        run = hash_block_bitmap<DT>(ht.part, ht.hold, ht.dst, bm, pre, log2b, nv, lane);
+    else
+        run = FINE ? scan_block_bitmap(bm, pre, log2b, lane)
+                   : build_block_bitmap(ballot, bm, pre, log2b, Piece<DT>::kLog2Values, lane);
 
     // payload bytes of this tile: B per changed block, less for a changed short last block
     uint64_t agg = payload_bytes_of_blocks<DT>(run, log2b);
@@ -231,7 +371,8 @@ __device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t 
 // payload <- exponents of changed blocks in block order; cache refreshed for the same blocks.
 // Every consumer thread sends the exponents of its own pieces (left in the stage's shared-memory
 // tile) if their block changed; `base` is the tile's exclusive offset in the unit's payload.
-template <int DT>
+// (CACHE = false, the sender with HashCache: payload only.)
+template <int DT, bool CACHE>
 __device__ __forceinline__ void write_changed(const EncodeTileInfo& ti, uint32_t log2b, const uint32_t* bm,
                                               const uint16_t* pre, uint64_t base, const uint8_t* s_exp, uint32_t tid) {
     using P = Piece<DT>;
@@ -257,6 +398,7 @@ __device__ __forceinline__ void write_changed(const EncodeTileInfo& ti, uint32_t
 #pragma unroll
             for (int i = 0; i < 5; ++i)
                 if (i < nbytes) pdst[i] = (uint8_t)(i < 4 ? lo >> (8 * i) : hi);
+            if (!CACHE) continue;
             if (nvalid == P::kValues)
                 x.template store_exp_full<Global>(cdst);
             else
@@ -266,10 +408,10 @@ __device__ __forceinline__ void write_changed(const EncodeTileInfo& ti, uint32_t
         uint8_t* pdst = ti.pay_dst + base + ((uint64_t)rank << log2b) + (t0 & ((1u << log2b) - 1u));
         if (nvalid == P::kValues) {
             x.template store_exp_full<Global>(pdst);
-            x.template store_exp_full<Global>(cdst);
+            if (CACHE) x.template store_exp_full<Global>(cdst);
         } else {
             x.store_exp_partial(pdst, nvalid);
-            x.store_exp_partial(cdst, nvalid);
+            if (CACHE) x.store_exp_partial(cdst, nvalid);
         }
     }
 }
@@ -332,11 +474,11 @@ __device__ __forceinline__ void write_changed_fine(const EncodeTileInfo& ti, con
     }
 }
 
-template <int DT, bool FINE>
+template <int DT, bool FINE, bool HASH>
 __device__ __forceinline__ void send_changed(const EncodeTileInfo& ti, uint32_t log2b, const uint32_t* bm,
                                              const uint16_t* pre, uint64_t base, const uint8_t* s_exp, uint32_t tid) {
     if (!FINE) {
-        write_changed<DT>(ti, log2b, bm, pre, base, s_exp, tid);
+        write_changed<DT, !HASH>(ti, log2b, bm, pre, base, s_exp, tid);
     } else {
         switch (log2b) {
             case 0: write_changed_fine<0>(ti, bm, pre, base, s_exp, tid); break;
@@ -347,16 +489,19 @@ __device__ __forceinline__ void send_changed(const EncodeTileInfo& ti, uint32_t 
     }
 }
 
-template <int DT, bool FINE>
+// `cache` is the sender's exponent cache or, with HASH, its HashCache; `tile_hash` (HASH only) gives
+// the index of every tile's first block in it.
+template <int DT, bool FINE, bool HASH>
 __global__ void __launch_bounds__(kEncodeThreads, 2)
 encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32_t* __restrict__ seq_first,
               uint32_t n_short, uint32_t log2b, const uint8_t* __restrict__ weights, uint8_t* cache, uint8_t* msgs,
               unsigned long long* wire_bytes, uint32_t* changed_blocks, unsigned long long* tile_status,
-              unsigned int* unit_ticket, int32_t* status) {
+              unsigned int* unit_ticket, int32_t* status, const unsigned long long* __restrict__ tile_hash) {
+    static_assert(!(HASH && (FINE || DT == CIERA_FP16)), "HashCache: bf16 and fp32, blocks of 16 values and more");
     using P = Piece<DT>;
     constexpr int VB = Traits<DT>::kValueBytes;
     constexpr int SMB = Traits<DT>::kSmBytes;
-    using Cfg = EncodeCfg<DT, FINE>;
+    using Cfg = typename EncodeCfgOf<DT, FINE, HASH>::type;
     constexpr int SW = Cfg::kWStages;
     constexpr int SE = Cfg::kEStages;
     constexpr int kDefer = Cfg::kDefer;
@@ -368,6 +513,11 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
     uint8_t* const ring_e = smem + (size_t)SW * kWBytes;
     using Ctl = EncodeCtl<SW, SE, Cfg::kBmWords>;
     Ctl* ctl = reinterpret_cast<Ctl*>(ring_e + (size_t)SE * kEBytes);
+    // HASH: per stage of the exponent ring, the tile's cached hashes and then the partial sums
+    static_assert(sizeof(Ctl) % 16 == 0, "the hash stages follow the control block");
+    uint8_t* const ring_h = reinterpret_cast<uint8_t*>(ctl) + sizeof(Ctl);
+    const uint32_t kHoldBytes = HASH ? hash_hold_bytes<DT>(log2b) : 0u;
+    const uint32_t kHStage = HASH ? kHoldBytes + hash_part_bytes<DT>(log2b) : 0u;
 
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     volatile int* abort = &ctl->abort;
@@ -401,15 +551,23 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
             bool seq_nxt = false;
             uint32_t tile_nxt = walk.next(seq_nxt);
             TileDesc nxt;
-            if (tile_nxt != kNoTile) nxt = load_tile_desc(tiles + tile_nxt);  // descriptors are fetched one tile ahead
+            unsigned long long hb_nxt = 0;  // HASH: index of the tile's first block in HashCache
+            if (tile_nxt != kNoTile) {      // descriptors are fetched one tile ahead
+                nxt = load_tile_desc(tiles + tile_nxt);
+                if (HASH) hb_nxt = __ldg(tile_hash + tile_nxt);
+            }
             uint32_t markers = 0;
             for (uint32_t k = 0;; ++k) {
                 const TileDesc td = nxt;
                 const uint32_t tile = tile_nxt;
                 const bool seq = seq_nxt;
+                const unsigned long long hb = hb_nxt;
                 if (tile != kNoTile) {
                     tile_nxt = walk.next(seq_nxt);
-                    if (tile_nxt != kNoTile) nxt = load_tile_desc(tiles + tile_nxt);
+                    if (tile_nxt != kNoTile) {
+                        nxt = load_tile_desc(tiles + tile_nxt);
+                        if (HASH) hb_nxt = __ldg(tile_hash + tile_nxt);
+                    }
                 }
                 const uint32_t sw = k % SW, se = k % SE;
                 if (k >= (uint32_t)SW && !mbar_wait(&ctl->empty_w[sw], ((k / SW) & 1u) ^ 1u, abort, status)) break;
@@ -430,12 +588,23 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
                     EncodeTileInfo ti;
                     ti.sm_dst = msgs + td.msg_off + smoff + sm_bytes_of_values<DT>(v0);
                     ti.pay_dst = msgs + td.msg_off + smoff + pad16(sm_section_bytes(td.n_unit, DT));
-                    ti.c_ptr = cache + td.c_off;
+                    ti.c_ptr = HASH ? cache + hb * 16ull : cache + td.c_off;
                     ti.w_src = weights + td.w_off;
                     ti.nv = (uint32_t)min((uint64_t)kTileValues, left);
                     ctl->info[k % kDescRing] = ti;
                 }
-                if (left >= (uint64_t)kTileValues) {
+                if constexpr (HASH) {
+                    // the cached hashes of the tile's blocks (16 bytes each) come in for every tile
+                    if (left >= (uint64_t)kTileValues) {
+                        mbar_arrive_expect_tx(&ctl->full_w[sw], kWBytes);
+                        bulk_load(ring_w + (size_t)sw * kWBytes, weights + td.w_off, kWBytes, &ctl->full_w[sw]);
+                    } else {
+                        mbar_arrive(&ctl->full_w[sw]);
+                    }
+                    const uint32_t nblk = (uint32_t)((min((uint64_t)kTileValues, left) + (1u << log2b) - 1u) >> log2b);
+                    mbar_arrive_expect_tx(&ctl->full_e[se], nblk * 16u);
+                    bulk_load(ring_h + (size_t)se * kHStage, cache + hb * 16ull, nblk * 16u, &ctl->full_e[se]);
+                } else if (left >= (uint64_t)kTileValues) {
                     mbar_arrive_expect_tx(&ctl->full_w[sw], kWBytes);
                     bulk_load(ring_w + (size_t)sw * kWBytes, weights + td.w_off, kWBytes, &ctl->full_w[sw]);
                     mbar_arrive_expect_tx(&ctl->full_e[se], kEBytes);
@@ -464,8 +633,16 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
             }
             const TileDesc td = ctl->desc[k % kDescRing];
             const bool seq = ctl->seq[k % kDescRing] != 0;
-            const uint64_t agg = aggregate_tile<DT, FINE>(td, tile, log2b, !seq, ctl->ballot[se], ctl->bm[se], ctl->pre[se], msgs,
-                                                    tile_status, lane);
+            HashTile ht{nullptr, nullptr, nullptr};
+            if constexpr (HASH) {
+                // the cached hashes were staged by a bulk copy that completes on full_e: observe it here too
+                if (!mbar_wait(&ctl->full_e[se], (k / SE) & 1u, abort, status)) break;
+                ht.hold = reinterpret_cast<const ulonglong2*>(ring_h + (size_t)se * kHStage);
+                ht.part = reinterpret_cast<const ulonglong2*>(ring_h + (size_t)se * kHStage + kHoldBytes);
+                ht.dst = reinterpret_cast<ulonglong2*>(ctl->info[k % kDescRing].c_ptr);
+            }
+            const uint64_t agg = aggregate_tile<DT, FINE, HASH>(td, tile, log2b, !seq, ctl->ballot[se], ctl->bm[se],
+                                                                ctl->pre[se], msgs, tile_status, ht, lane);
             if (seq) {
                 // the whole unit is this block's: the tile's offset is the running sum
                 const uint64_t excl = td.tile_in_unit == 0 ? 0ull : run_incl;
@@ -511,6 +688,8 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
         // stage and phase of slot k in the two rings, and of slot k - kDefer in the exponent ring, kept
         // as running counters (the ring depths are no powers of two)
         uint32_t sw = 0, pw = 0, se = 0, pe = 0, je = 0, pj = 0;
+        // HASH: the lanes of a warp that share a block (a power of two, at most the warp) add up their terms
+        const uint32_t hash_lanes_l2 = min(5u, log2b - (uint32_t)P::kLog2Values);
         for (;; ++k) {
             if (!mbar_wait(&ctl->full_w[sw], pw, abort, status)) break;
             if (!mbar_wait(&ctl->full_e[se], pe, abort, status)) break;
@@ -529,6 +708,7 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
                 const uint32_t nv = ti.nv;
                 const uint8_t* const s_w = ring_w + (size_t)sw * kWBytes;
                 uint8_t* const s_e = ring_e + (size_t)se * kEBytes;
+                uint64_t hash_a[P::kPerThread], hash_b[P::kPerThread];  // HASH: the pieces' sums of terms
 #pragma unroll
                 for (int p = 0; p < P::kPerThread; ++p) {
                     const uint32_t t0 = P::start(tid, p);
@@ -537,19 +717,34 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
                     P x, c;
                     if (nv == (uint32_t)kTileValues) {
                         x.template split_full<Shared>(s_w + (size_t)t0 * VB);
-                        c.template load_exp_full<Shared>(s_e + t0);
+                        if (!HASH) c.template load_exp_full<Shared>(s_e + t0);
                     } else if (nvalid == P::kValues) {
                         x.template split_full<Global>(ti.w_src + (size_t)t0 * VB);
-                        c.template load_exp_full<Global>(ti.c_ptr + t0);
+                        if (!HASH) c.template load_exp_full<Global>(ti.c_ptr + t0);
                     } else {
                         // values past the end of the unit read as exponent 0 against a cached 0: never "changed"
                         x.split_partial(ti.w_src + (size_t)t0 * VB, nvalid);
-                        c.load_exp_partial(ti.c_ptr + t0, nvalid);
+                        if (!HASH) c.load_exp_partial(ti.c_ptr + t0, nvalid);
                     }
                     // leave the new exponents where the cached ones were staged: they are sent from
                     // there once the tile's place in the payload is known
                     x.template store_exp_full<Shared>(s_e + t0);
-                    if constexpr (!FINE) {
+                    if constexpr (HASH) {
+                        // h <- Hash128(exp[k]), first part: the terms of this piece's 64-bit words (words
+                        // past the end of the unit do not exist)
+                        uint64_t a = 0, b = 0;
+                        const uint32_t j0 = (t0 & ((1u << log2b) - 1u)) >> 3;
+#pragma unroll
+                        for (int w = 0; w < P::kExpWords / 2; ++w) {
+                            uint64_t ta, tb;
+                            hash_word_terms(j0 + (uint32_t)w, (uint64_t)x.e[2 * w] | ((uint64_t)x.e[2 * w + 1] << 32), ta, tb);
+                            const bool exists = nvalid > 8 * w;
+                            a += exists ? ta : 0ull;
+                            b += exists ? tb : 0ull;
+                        }
+                        hash_a[p] = a;
+                        hash_b[p] = b;
+                    } else if constexpr (!FINE) {
                         const uint32_t bal = __ballot_sync(0xffffffffu, x.differs(c));
                         if (lane == 0) ctl->ballot[se][p * kWarps + warp] = bal;
                     } else {
@@ -584,6 +779,11 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
                             x.store_sm_partial(smdst, nvalid);
                     }
                 }
+                if constexpr (HASH) {
+                    uint64_t* const part = reinterpret_cast<uint64_t*>(ring_h + (size_t)se * kHStage + kHoldBytes);
+                    reduce_hash_terms<P::kPerThread>(hash_a, hash_b, hash_lanes_l2, (P::start(tid, 0) >> P::kLog2Values) >> hash_lanes_l2,
+                                                     (P::start(tid, P::kPerThread - 1) >> P::kLog2Values) >> hash_lanes_l2, part, lane);
+                }
                 __syncwarp();  // the warp's shared-memory accesses above are ordered before lane 0's arrives
                 if (lane == 0) {
                     mbar_arrive(&ctl->empty_w[sw]);
@@ -595,8 +795,8 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
             if (k >= (uint32_t)kDefer) {
                 if (k - kDefer < k_end) {
                     if (!mbar_wait(&ctl->resolved[je], pj, abort, status)) break;
-                    send_changed<DT, FINE>(ctl->info[(k - kDefer) % kDescRing], log2b, ctl->bm[je], ctl->pre[je],
-                                           ctl->base[je], ring_e + (size_t)je * kEBytes, tid);
+                    send_changed<DT, FINE, HASH>(ctl->info[(k - kDefer) % kDescRing], log2b, ctl->bm[je], ctl->pre[je],
+                                                 ctl->base[je], ring_e + (size_t)je * kEBytes, tid);
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&ctl->empty_e[je]);
                 }
@@ -620,8 +820,8 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
             for (uint32_t j = k + 1u >= (uint32_t)kDefer ? k + 1u - kDefer : 0u; j < k_end; ++j) {
                 const uint32_t je = j % SE;
                 if (!mbar_wait(&ctl->resolved[je], (j / SE) & 1u, abort, status)) break;
-                send_changed<DT, FINE>(ctl->info[j % kDescRing], log2b, ctl->bm[je], ctl->pre[je], ctl->base[je],
-                                       ring_e + (size_t)je * kEBytes, tid);
+                send_changed<DT, FINE, HASH>(ctl->info[j % kDescRing], log2b, ctl->bm[je], ctl->pre[je], ctl->base[je],
+                                             ring_e + (size_t)je * kEBytes, tid);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&ctl->empty_e[je]);
             }
@@ -640,47 +840,51 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
     }
 }
 
-template <int DT, bool FINE>
-static size_t encode_smem_bytes() {
-    using Cfg = EncodeCfg<DT, FINE>;
+// (with HashCache the size depends on the block size: see hash_hold_bytes, hash_part_bytes)
+template <int DT, bool FINE, bool HASH>
+static size_t encode_smem_bytes(uint32_t log2b) {
+    using Cfg = typename EncodeCfgOf<DT, FINE, HASH>::type;
     constexpr int SW = Cfg::kWStages, SE = Cfg::kEStages;
+    const size_t hash_stage = HASH ? (size_t)hash_hold_bytes<DT>(log2b) + hash_part_bytes<DT>(log2b) : 0;
     return (size_t)SW * kTileValues * Traits<DT>::kValueBytes + (size_t)SE * kTileValues +
-           sizeof(EncodeCtl<SW, SE, Cfg::kBmWords>);
+           sizeof(EncodeCtl<SW, SE, Cfg::kBmWords>) + (size_t)SE * hash_stage;
 }
 
-// Largest grid whose blocks are all resident at once, per device (0 = not yet known).
-template <int DT, bool FINE>
-static int encode_grid_limit(int* out) {
-    static int cached[64] = {0};
+// Largest grid whose blocks are all resident at once, per device and block size (0 = not yet known).
+template <int DT, bool FINE, bool HASH>
+static int encode_grid_limit(uint32_t log2b, int* out) {
+    static int cached[64][16] = {{0}};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return record_cuda_error(e);
-    if (dev < 0 || dev >= 64) return CIERA_ERR_UNSUPPORTED;
-    if (cached[dev] == 0) {
-        const size_t smem = encode_smem_bytes<DT, FINE>();
-        e = cudaFuncSetAttribute(encode_kernel<DT, FINE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (dev < 0 || dev >= 64 || log2b >= 16) return CIERA_ERR_UNSUPPORTED;
+    if (cached[dev][log2b] == 0) {
+        const size_t smem = encode_smem_bytes<DT, FINE, HASH>(log2b);
+        // (the limit set here is the largest any block size asks for: the smallest block of the class)
+        e = cudaFuncSetAttribute(encode_kernel<DT, FINE, HASH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)encode_smem_bytes<DT, FINE, HASH>(FINE ? 0u : kFineLog2));
         if (e != cudaSuccess) return record_cuda_error(e);
         int per_sm = 0, sms = 0, coop = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, encode_kernel<DT, FINE>, kEncodeThreads, smem);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, encode_kernel<DT, FINE, HASH>, kEncodeThreads, smem);
         if (e != cudaSuccess) return record_cuda_error(e);
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return record_cuda_error(e);
         e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
         if (e != cudaSuccess) return record_cuda_error(e);
         if (per_sm < 1 || sms < 1 || !coop) return CIERA_ERR_UNSUPPORTED;
-        cached[dev] = per_sm * sms;
+        cached[dev][log2b] = per_sm * sms;
     }
-    *out = cached[dev];
+    *out = cached[dev][log2b];
     return CIERA_OK;
 }
 
 // `scratch`: one status word per tile, then the unit counter; all zero at kernel start.
-template <int DT, bool FINE>
+template <int DT, bool FINE, bool HASH = false>
 static int launch_encode(const ciera_plan* p, const void* weights_dev, void* sender_cache_dev, void* messages_dev,
                          uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* scratch, int32_t* status_dev,
                          cudaStream_t s) {
     int limit = 0;
-    const int rc = encode_grid_limit<DT, FINE>(&limit);
+    const int rc = encode_grid_limit<DT, FINE, HASH>(p->log2b, &limit);
     if (rc) return rc;
     const TileDesc* tiles = p->tiles_dev;
     uint32_t nt = (uint32_t)p->tiles.size();
@@ -694,18 +898,20 @@ static int launch_encode(const ciera_plan* p, const void* weights_dev, void* sen
     unsigned long long* wb = (unsigned long long*)wire_bytes_dev;
     unsigned long long* ts = (unsigned long long*)scratch;
     unsigned int* ticket = (unsigned int*)(ts + nt);
+    const unsigned long long* tile_hash = HASH ? p->tile_hash_dev : nullptr;
+    const size_t smem = encode_smem_bytes<DT, FINE, HASH>(log2b);
     const bool has_spread = p->seq_first.back() < nt;  // tiles of longer units: look-back between blocks
     cudaError_t e;
     if (has_spread) {
         // cooperative launch: the runtime starts the grid only when all of its blocks fit on the
         // GPU together, which is what the look-back between blocks relies on
         void* args[] = {&tiles, &nt, &seq_first, &n_short, &log2b, &w, &c, &m, &wb, &changed_blocks_dev, &ts, &ticket,
-                        &status_dev};
-        e = cudaLaunchCooperativeKernel((const void*)encode_kernel<DT, FINE>, dim3(grid), dim3(kEncodeThreads), args,
-                                        encode_smem_bytes<DT, FINE>(), s);
+                        &status_dev, &tile_hash};
+        e = cudaLaunchCooperativeKernel((const void*)encode_kernel<DT, FINE, HASH>, dim3(grid), dim3(kEncodeThreads), args,
+                                        smem, s);
     } else {
-        encode_kernel<DT, FINE><<<grid, kEncodeThreads, encode_smem_bytes<DT, FINE>(), s>>>(
-            tiles, nt, seq_first, n_short, log2b, w, c, m, wb, changed_blocks_dev, ts, ticket, status_dev);
+        encode_kernel<DT, FINE, HASH><<<grid, kEncodeThreads, smem, s>>>(
+            tiles, nt, seq_first, n_short, log2b, w, c, m, wb, changed_blocks_dev, ts, ticket, status_dev, tile_hash);
         e = cudaGetLastError();
     }
     if (e != cudaSuccess) return record_cuda_error(e);
@@ -730,6 +936,17 @@ static int launch_encode_any(const ciera_plan* p, const void* weights_dev, void*
                                                   changed_blocks_dev, scratch, status_dev, s)
                 : launch_encode<CIERA_FP32, false>(p, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
                                                    changed_blocks_dev, scratch, status_dev, s);
+}
+
+// the sender with HashCache: bf16 and fp32, blocks of 16 values and more (checked by the caller)
+int launch_encode_hashed(const ciera_plan* p, const void* weights_dev, void* hash_cache_dev, void* messages_dev,
+                         uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* scratch, int32_t* status_dev,
+                         cudaStream_t s) {
+    if (p->dtype == CIERA_BF16)
+        return launch_encode<CIERA_BF16, false, true>(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev,
+                                                      changed_blocks_dev, scratch, status_dev, s);
+    return launch_encode<CIERA_FP32, false, true>(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev,
+                                                  changed_blocks_dev, scratch, status_dev, s);
 }
 
 }  // namespace ciera

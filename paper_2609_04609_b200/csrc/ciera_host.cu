@@ -68,7 +68,7 @@ extern "C" size_t ciera_message_bytes(uint64_t n, int dtype, uint32_t block, uin
 
 namespace {
 struct ImageLayout {
-    size_t tiles, long_off, seq_off, hash_off, first_off, seg_off, units_off, elong_off, echunk_off, total;
+    size_t tiles, long_off, seq_off, hash_off, first_off, seg_off, units_off, elong_off, echunk_off, thash_off, total;
 };
 size_t up16(size_t x) { return (x + 15) / 16 * 16; }
 ImageLayout image_layout(const ciera_plan* p) {
@@ -82,7 +82,8 @@ ImageLayout image_layout(const ciera_plan* p) {
     L.units_off = L.seg_off + up16((size_t)p->n_units * sizeof(uint64_t));
     L.elong_off = L.units_off + up16((size_t)p->n_units * sizeof(ciera_unit));
     L.echunk_off = L.elong_off + up16(p->ent_long_units.size() * sizeof(uint32_t));
-    L.total = L.echunk_off + p->ent_chunks.size() * sizeof(ciera_plan::EntChunk) + 16;
+    L.thash_off = L.echunk_off + up16(p->ent_chunks.size() * sizeof(ciera_plan::EntChunk));
+    L.total = L.thash_off + p->tiles.size() * sizeof(uint64_t) + 16;
     return L;
 }
 }  // namespace
@@ -174,12 +175,16 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
             for (uint64_t g = 0; g < slots; g += 64) p->ent_chunks.push_back({u, (uint32_t)g, li, 0u});
         }
     }
+    p->tile_hash.resize(p->tiles.size());
+    for (size_t t = 0; t < p->tiles.size(); ++t)
+        p->tile_hash[t] = p->hash_base[p->tiles[t].unit] + (uint64_t)p->tiles[t].tile_in_unit * (kTileValues >> p->log2b);
     // device image: the tile table, then (each 16-byte aligned) the index lists
     const ImageLayout L = image_layout(p);
     p->image.assign(L.total, 0);
     if (L.tiles) memcpy(p->image.data(), p->tiles.data(), L.tiles);
     if (!p->long_units.empty()) memcpy(p->image.data() + L.long_off, p->long_units.data(), p->long_units.size() * 4);
     memcpy(p->image.data() + L.seq_off, p->seq_first.data(), p->seq_first.size() * 4);
+    if (!p->tile_hash.empty()) memcpy(p->image.data() + L.thash_off, p->tile_hash.data(), p->tile_hash.size() * 8);
     if (n_units) {
         memcpy(p->image.data() + L.hash_off, p->hash_base.data(), (size_t)n_units * 8);
         memcpy(p->image.data() + L.first_off, p->unit_first.data(), (size_t)n_units * 4);
@@ -216,8 +221,8 @@ extern "C" size_t ciera_plan_unit_hash_offset(const ciera_plan* p, uint32_t unit
 }
 extern "C" size_t ciera_plan_hashed_workspace_bytes(const ciera_plan* p) {
     if (!p) return 0;
-    // 16 words of block flags, a count and a payload offset per tile
-    return p->tiles.size() * (16 + 2) * sizeof(uint32_t) + 16;
+    // as for ciera_encode: one look-back status word per tile + the ticket counter
+    return p->tiles.size() * sizeof(unsigned long long) + 16;
 }
 
 extern "C" int ciera_plan_bind(ciera_plan* p, void* plan_dev, size_t plan_dev_bytes, void* stream) {
@@ -241,6 +246,7 @@ extern "C" int ciera_plan_bind(ciera_plan* p, void* plan_dev, size_t plan_dev_by
     p->units_dev = (const ciera_unit*)(base + L.units_off);
     p->ent_long_units_dev = (const uint32_t*)(base + L.elong_off);
     p->ent_chunks_dev = (const uint4*)(base + L.echunk_off);
+    p->tile_hash_dev = (const unsigned long long*)(base + L.thash_off);
     return CIERA_OK;
 }
 

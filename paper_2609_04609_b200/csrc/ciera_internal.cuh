@@ -139,6 +139,7 @@ struct ciera_plan {
     std::vector<uint32_t> seq_first;   // first tile of every short unit, in table order, + end marker
     std::vector<uint32_t> unit_first;  // first tile of every unit (0xffffffff: a unit without values)
     std::vector<uint64_t> hash_base;   // index of every unit's first block in a per-block hash cache
+    std::vector<uint64_t> tile_hash;   // the same for every tile's first block, in tile-table order
     uint64_t total_blocks = 0;
     std::vector<uint64_t> seg_base;    // index of every unit's first 4096-byte payload segment (entropy stage)
     uint64_t total_segments = 0;
@@ -153,11 +154,12 @@ struct ciera_plan {
     const uint32_t* ent_long_units_dev = nullptr;
     const uint4* ent_chunks_dev = nullptr;
     std::vector<uint8_t> image;        // device image: tiles, long_units, seq_first, hash_base, unit_first, seg_base, units,
-                                       // ent_long_units, ent_chunks
+                                       // ent_long_units, ent_chunks, tile_hash
     const ciera::TileDesc* tiles_dev = nullptr;
     const uint32_t* long_units_dev = nullptr;
     const uint32_t* seq_first_dev = nullptr;
     const unsigned long long* hash_base_dev = nullptr;
+    const unsigned long long* tile_hash_dev = nullptr;
     const uint32_t* unit_first_dev = nullptr;
     const unsigned long long* seg_base_dev = nullptr;
     const ciera_unit* units_dev = nullptr;
@@ -167,4 +169,8 @@ namespace ciera {
 int record_cuda_error(cudaError_t e);          // stores e for ciera_last_cuda_error, returns CIERA_ERR_CUDA
 void count_launch();                           // launch accounting
 int check_launch();                            // cudaGetLastError -> status
+// the persistent sender kernel with HashCache in place of the exponent cache (ciera_encode.cu)
+int launch_encode_hashed(const ciera_plan* p, const void* weights_dev, void* hash_cache_dev, void* messages_dev,
+                         uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* scratch, int32_t* status_dev,
+                         cudaStream_t s);
 }  // namespace ciera

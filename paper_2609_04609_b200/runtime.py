@@ -65,7 +65,7 @@ class LayerCodec:
 
     def encode_hashed(self, weights: torch.Tensor, stream=None) -> None:
         ciera.encode_hashed(self.plan, weights, self.hash_cache, self.msg_send, self.wire_bytes, self.changed_blocks,
-                            self.hashed_workspace, stream)
+                            self.hashed_workspace, self.status, stream)
 
     # -- entropy stage around the transport --------------------------------------------------------
     def _entropy_scratch(self) -> torch.Tensor:
