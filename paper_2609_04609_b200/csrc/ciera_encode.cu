@@ -98,29 +98,47 @@ struct EncodeCfg<CIERA_FP32, true> {
 // With HashCache the exponent ring stages no cached exponents (it only keeps the new ones until
 // they are sent), so it is shorter; each of its stages has a companion with the tile's cached
 // hashes and the consumers' partial sums, sized at launch from the block size.
-template <int DT>
+// The template argument HASH of the kernel is 0 (exponent cache), 1 (HashCache) or 2 (HashCache with
+// shorter rings: with blocks of 64 values and fewer the hash stages are large, and two thread blocks
+// still have to fit an SM).
+template <int DT, int HASH>
 struct EncodeHashCfg;
 template <>
-struct EncodeHashCfg<CIERA_BF16> {
+struct EncodeHashCfg<CIERA_BF16, 1> {
     static constexpr int kWStages = 3;
     static constexpr int kEStages = 6;
     static constexpr int kDefer = 3;
     static constexpr int kBmWords = kBitmapWords;
 };
 template <>
-struct EncodeHashCfg<CIERA_FP32> {
+struct EncodeHashCfg<CIERA_FP32, 1> {
     static constexpr int kWStages = 2;
     static constexpr int kEStages = 4;
     static constexpr int kDefer = 2;
     static constexpr int kBmWords = kBitmapWords;
 };
-template <int DT, bool FINE, bool HASH>
-struct EncodeCfgOf {
-    using type = EncodeCfg<DT, FINE>;
+template <>
+struct EncodeHashCfg<CIERA_BF16, 2> {
+    static constexpr int kWStages = 3;
+    static constexpr int kEStages = 4;
+    static constexpr int kDefer = 2;
+    static constexpr int kBmWords = kBitmapWords;
 };
-template <int DT>
-struct EncodeCfgOf<DT, false, true> {
-    using type = EncodeHashCfg<DT>;
+template <>
+struct EncodeHashCfg<CIERA_FP32, 2> {
+    static constexpr int kWStages = 2;
+    static constexpr int kEStages = 3;
+    static constexpr int kDefer = 1;
+    static constexpr int kBmWords = kBitmapWords;
+};
+constexpr uint32_t kHashShortRingsLog2 = 6;  // blocks of up to 2^6 values take the shorter rings
+template <int DT, bool FINE, int HASH>
+struct EncodeCfgOf {
+    using type = EncodeHashCfg<DT, HASH>;
+};
+template <int DT, bool FINE>
+struct EncodeCfgOf<DT, FINE, 0> {
+    using type = EncodeCfg<DT, FINE>;
 };
 
 // Shared-memory bytes of the cached hashes (`hold`) and of the partial sums (`part`) of one tile:
@@ -320,7 +338,7 @@ struct HashTile {
     ulonglong2* dst;
 };
 
-template <int DT, bool FINE, bool HASH>
+template <int DT, bool FINE, int HASH>
 __device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t tile, uint32_t log2b, bool publish,
                                                    const uint32_t* ballot, uint32_t* bm, uint16_t* pre, uint8_t* msgs,
                                                    unsigned long long* tile_status, const HashTile& ht, uint32_t lane) {
@@ -474,11 +492,11 @@ __device__ __forceinline__ void write_changed_fine(const EncodeTileInfo& ti, con
     }
 }
 
-template <int DT, bool FINE, bool HASH>
+template <int DT, bool FINE, int HASH>
 __device__ __forceinline__ void send_changed(const EncodeTileInfo& ti, uint32_t log2b, const uint32_t* bm,
                                              const uint16_t* pre, uint64_t base, const uint8_t* s_exp, uint32_t tid) {
     if (!FINE) {
-        write_changed<DT, !HASH>(ti, log2b, bm, pre, base, s_exp, tid);
+        write_changed<DT, HASH == 0>(ti, log2b, bm, pre, base, s_exp, tid);
     } else {
         switch (log2b) {
             case 0: write_changed_fine<0>(ti, bm, pre, base, s_exp, tid); break;
@@ -491,7 +509,7 @@ __device__ __forceinline__ void send_changed(const EncodeTileInfo& ti, uint32_t 
 
 // `cache` is the sender's exponent cache or, with HASH, its HashCache; `tile_hash` (HASH only) gives
 // the index of every tile's first block in it.
-template <int DT, bool FINE, bool HASH>
+template <int DT, bool FINE, int HASH>
 __global__ void __launch_bounds__(kEncodeThreads, 2)
 encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32_t* __restrict__ seq_first,
               uint32_t n_short, uint32_t log2b, const uint8_t* __restrict__ weights, uint8_t* cache, uint8_t* msgs,
@@ -732,15 +750,22 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
                     if constexpr (HASH) {
                         // h <- Hash128(exp[k]), first part: the terms of this piece's 64-bit words (words
                         // past the end of the unit do not exist)
-                        uint64_t a = 0, b = 0;
+                        constexpr int kWords = P::kExpWords / 2;
+                        uint64_t ta[kWords], tb[kWords];
                         const uint32_t j0 = (t0 & ((1u << log2b) - 1u)) >> 3;
 #pragma unroll
-                        for (int w = 0; w < P::kExpWords / 2; ++w) {
-                            uint64_t ta, tb;
-                            hash_word_terms(j0 + (uint32_t)w, (uint64_t)x.e[2 * w] | ((uint64_t)x.e[2 * w + 1] << 32), ta, tb);
-                            const bool exists = nvalid > 8 * w;
-                            a += exists ? ta : 0ull;
-                            b += exists ? tb : 0ull;
+                        for (int w = 0; w < kWords; ++w)
+                            hash_word_terms(j0 + (uint32_t)w, (uint64_t)x.e[2 * w] | ((uint64_t)x.e[2 * w + 1] << 32), ta[w], tb[w]);
+                        if (nvalid != P::kValues) {  // the unit's last pieces only
+#pragma unroll
+                            for (int w = 0; w < kWords; ++w)
+                                if (nvalid <= 8 * w) ta[w] = tb[w] = 0ull;
+                        }
+                        uint64_t a = ta[0], b = tb[0];
+#pragma unroll
+                        for (int w = 1; w < kWords; ++w) {
+                            a += ta[w];
+                            b += tb[w];
                         }
                         hash_a[p] = a;
                         hash_b[p] = b;
@@ -841,7 +866,7 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
 }
 
 // (with HashCache the size depends on the block size: see hash_hold_bytes, hash_part_bytes)
-template <int DT, bool FINE, bool HASH>
+template <int DT, bool FINE, int HASH>
 static size_t encode_smem_bytes(uint32_t log2b) {
     using Cfg = typename EncodeCfgOf<DT, FINE, HASH>::type;
     constexpr int SW = Cfg::kWStages, SE = Cfg::kEStages;
@@ -851,7 +876,7 @@ static size_t encode_smem_bytes(uint32_t log2b) {
 }
 
 // Largest grid whose blocks are all resident at once, per device and block size (0 = not yet known).
-template <int DT, bool FINE, bool HASH>
+template <int DT, bool FINE, int HASH>
 static int encode_grid_limit(uint32_t log2b, int* out) {
     static int cached[64][16] = {{0}};
     int dev = 0;
@@ -862,7 +887,7 @@ static int encode_grid_limit(uint32_t log2b, int* out) {
         const size_t smem = encode_smem_bytes<DT, FINE, HASH>(log2b);
         // (the limit set here is the largest any block size asks for: the smallest block of the class)
         e = cudaFuncSetAttribute(encode_kernel<DT, FINE, HASH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)encode_smem_bytes<DT, FINE, HASH>(FINE ? 0u : kFineLog2));
+                                 (int)encode_smem_bytes<DT, FINE, HASH>(FINE ? 0u : HASH == 1 ? kHashShortRingsLog2 + 1u : kFineLog2));
         if (e != cudaSuccess) return record_cuda_error(e);
         int per_sm = 0, sms = 0, coop = 0;
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, encode_kernel<DT, FINE, HASH>, kEncodeThreads, smem);
@@ -879,7 +904,7 @@ static int encode_grid_limit(uint32_t log2b, int* out) {
 }
 
 // `scratch`: one status word per tile, then the unit counter; all zero at kernel start.
-template <int DT, bool FINE, bool HASH = false>
+template <int DT, bool FINE, int HASH = 0>
 static int launch_encode(const ciera_plan* p, const void* weights_dev, void* sender_cache_dev, void* messages_dev,
                          uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* scratch, int32_t* status_dev,
                          cudaStream_t s) {
@@ -942,11 +967,16 @@ static int launch_encode_any(const ciera_plan* p, const void* weights_dev, void*
 int launch_encode_hashed(const ciera_plan* p, const void* weights_dev, void* hash_cache_dev, void* messages_dev,
                          uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* scratch, int32_t* status_dev,
                          cudaStream_t s) {
+    const bool short_rings = p->log2b <= kHashShortRingsLog2;
     if (p->dtype == CIERA_BF16)
-        return launch_encode<CIERA_BF16, false, true>(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev,
-                                                      changed_blocks_dev, scratch, status_dev, s);
-    return launch_encode<CIERA_FP32, false, true>(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev,
-                                                  changed_blocks_dev, scratch, status_dev, s);
+        return short_rings ? launch_encode<CIERA_BF16, false, 2>(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev,
+                                                                 changed_blocks_dev, scratch, status_dev, s)
+                           : launch_encode<CIERA_BF16, false, 1>(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev,
+                                                                 changed_blocks_dev, scratch, status_dev, s);
+    return short_rings ? launch_encode<CIERA_FP32, false, 2>(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev,
+                                                             changed_blocks_dev, scratch, status_dev, s)
+                       : launch_encode<CIERA_FP32, false, 1>(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev,
+                                                             changed_blocks_dev, scratch, status_dev, s);
 }
 
 }  // namespace ciera
