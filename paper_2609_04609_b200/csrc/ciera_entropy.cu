@@ -56,8 +56,46 @@ __device__ __forceinline__ void histogram_add(uint32_t (*hist)[256], const uint8
     }
 }
 
-// Frequencies from counts (h[256] in shared memory, P = their sum): thread s owns symbol s.  Ends
-// with a barrier; f is then final.
+// Exclusive running sums of f[0..255] by one warp (lane l owns symbols 8 l .. 8 l + 7): returns the sum of
+// the symbols before the lane's first one and leaves the sums inside its group in local[]; `total`
+// gets the sum of all.
+__device__ __forceinline__ uint32_t warp_prefix256(const uint16_t* f, uint32_t lane, uint32_t local[8], uint32_t& total) {
+    uint32_t run = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        local[i] = run;
+        run += f[8 * lane + i];
+    }
+    uint32_t incl = run;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+        if ((int)lane >= o) incl += t;
+    }
+    total = __shfl_sync(0xffffffffu, incl, 31);
+    return incl - run;
+}
+
+// Index of the largest of v[0..255], the lowest index among equals (one warp; v(s) gives the value).
+template <class V>
+__device__ __forceinline__ uint32_t warp_argmax256(V v, uint32_t lane) {
+    unsigned long long key = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint32_t s = 8 * lane + i;
+        const unsigned long long k = ((unsigned long long)v(s) << 8) | (255u - s);
+        key = k > key ? k : key;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long k = __shfl_xor_sync(0xffffffffu, key, o);
+        key = k > key ? k : key;
+    }
+    return 255u - (uint32_t)(key & 255u);
+}
+
+// Frequencies from counts (h[256] in shared memory, P = their sum): thread s owns symbol s, then the
+// first warp settles the sum.  Ends with a barrier; f is then final.
 __device__ __forceinline__ void normalise_model(const uint32_t* h, uint64_t P, uint16_t* f, uint32_t tid) {
     {
         uint32_t v = 0;
@@ -68,22 +106,20 @@ __device__ __forceinline__ void normalise_model(const uint32_t* h, uint64_t P, u
         f[tid] = (uint16_t)v;
     }
     __syncthreads();
-    if (tid == 0) {
-        uint32_t sum = 0, best = 0;
-        for (uint32_t s = 0; s < 256; ++s) {
-            sum += f[s];
-            if (h[s] > h[best]) best = s;
-        }
-        if (sum < kProbScale) {
-            f[best] = (uint16_t)(f[best] + (kProbScale - sum));
-        } else {
+    if (tid < 32) {
+        uint32_t local[8], sum;
+        warp_prefix256(f, tid, local, sum);
+        if (sum < kProbScale) {  // the shortfall goes to the most frequent symbol
+            const uint32_t best = warp_argmax256([&](uint32_t s) { return h[s]; }, tid);
+            if (tid == 0) f[best] = (uint16_t)(f[best] + (kProbScale - sum));
+        } else {  // an excess is taken from the largest entries
             uint32_t excess = sum - kProbScale;
             while (excess) {
-                uint32_t big = 0;
-                for (uint32_t s = 1; s < 256; ++s)
-                    if (f[s] > f[big]) big = s;
+                const uint32_t big = warp_argmax256([&](uint32_t s) { return (uint32_t)f[s]; }, tid);
                 const uint32_t take = min((uint32_t)f[big] - 1u, excess);
-                f[big] = (uint16_t)(f[big] - take);
+                __syncwarp();
+                if (tid == 0) f[big] = (uint16_t)(f[big] - take);
+                __syncwarp();
                 excess -= take;
             }
         }
@@ -96,12 +132,11 @@ __device__ __forceinline__ void normalise_model(const uint32_t* h, uint64_t P, u
 // x < 2^32 the product x * rcp / 2^64 exceeds x / f by less than 2^-32 -- too little to reach the next
 // integer, because the fraction of x / f is at most 1 - 1/4096.  (f = 1 is handled apart.)
 __device__ __forceinline__ void encoder_tables(const uint16_t* f, uint16_t* c, unsigned long long* rcp, uint32_t tid) {
-    if (tid == 0) {
-        uint32_t run = 0;
-        for (uint32_t s = 0; s < 256; ++s) {
-            c[s] = (uint16_t)run;
-            run += f[s];
-        }
+    if (tid < 32) {
+        uint32_t local[8], total;
+        const uint32_t base = warp_prefix256(f, tid, local, total);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) c[8 * tid + i] = (uint16_t)(base + local[i]);
     }
     rcp[tid] = f[tid] > 1 ? (~0ull) / f[tid] + 1ull : 0ull;
     __syncthreads();
@@ -150,13 +185,12 @@ __device__ __forceinline__ uint32_t encode_segment(const uint8_t* src, uint32_t 
 // The owner of a slot is the last symbol that starts at or below it (symbols that do not occur share
 // their start with the next one, or start at 4096 behind the last occurring one).
 __device__ __forceinline__ bool decoder_tables(const uint16_t* f, uint16_t* c, uint8_t* sym, uint32_t* flag, uint32_t tid) {
-    if (tid == 0) {
-        uint32_t run = 0;
-        for (uint32_t s = 0; s < 256; ++s) {
-            c[s] = (uint16_t)min(run, kProbScale);
-            run += f[s];
-        }
-        *flag = run == kProbScale ? 1u : 0u;
+    if (tid < 32) {
+        uint32_t local[8], total;
+        const uint32_t base = warp_prefix256(f, tid, local, total);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) c[8 * tid + i] = (uint16_t)min(base + local[i], kProbScale);
+        if (tid == 0) *flag = total == kProbScale ? 1u : 0u;
     }
     __syncthreads();
     if (*flag == 0) return false;
