@@ -131,21 +131,24 @@ __device__ __forceinline__ void normalise_model(const uint32_t* h, uint64_t P, u
 // x / f through a multiplication: rcp = ceil(2^64 / f) exceeds 2^64 / f by less than 1, so for
 // x < 2^32 the product x * rcp / 2^64 exceeds x / f by less than 2^-32 -- too little to reach the next
 // integer, because the fraction of x / f is at most 1 - 1/4096.  (f = 1 is handled apart.)
-__device__ __forceinline__ void encoder_tables(const uint16_t* f, uint16_t* c, unsigned long long* rcp, uint32_t tid) {
+// The coder reads one 16-byte entry per symbol: {rcp low, rcp high, f | c << 16, 0}.
+__device__ __forceinline__ void encoder_tables(const uint16_t* f, uint4* enc, uint32_t tid) {
+    const unsigned long long rcp = f[tid] > 1 ? (~0ull) / f[tid] + 1ull : 0ull;
+    enc[tid].x = (uint32_t)rcp;
+    enc[tid].y = (uint32_t)(rcp >> 32);
+    enc[tid].w = 0u;
     if (tid < 32) {
         uint32_t local[8], total;
         const uint32_t base = warp_prefix256(f, tid, local, total);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) c[8 * tid + i] = (uint16_t)(base + local[i]);
+        for (int i = 0; i < 8; ++i) enc[8 * tid + i].z = (uint32_t)f[8 * tid + i] | ((base + local[i]) << 16);
     }
-    rcp[tid] = f[tid] > 1 ? (~0ull) / f[tid] + 1ull : 0ull;
     __syncthreads();
 }
 
 // One warp codes one segment: src[0, n) -> slot (32 states, then the words).  Returns the word count.
-__device__ __forceinline__ uint32_t encode_segment(const uint8_t* src, uint32_t n, uint8_t* stage, const uint16_t* f,
-                                                   const uint16_t* c, const unsigned long long* rcp, uint8_t* slot,
-                                                   uint32_t lane) {
+__device__ __forceinline__ uint32_t encode_segment(const uint8_t* src, uint32_t n, uint8_t* stage, const uint4* enc,
+                                                   uint8_t* slot, uint32_t lane) {
     for (uint32_t i = lane * 16; i < n; i += 32 * 16) {
         if (i + 16 <= n) {
             *reinterpret_cast<uint4*>(stage + i) = *reinterpret_cast<const uint4*>(src + i);
@@ -156,24 +159,31 @@ __device__ __forceinline__ uint32_t encode_segment(const uint8_t* src, uint32_t 
     __syncwarp();
     uint16_t* words = reinterpret_cast<uint16_t*>(slot + 4 * 32);
     uint32_t x = kRansL, nw = 0;
-    const uint32_t steps = (n + 31u) >> 5;
-    for (uint32_t t = steps; t-- > 0;) {
-        const uint32_t i = 32u * t + lane;
-        const bool has = i < n;
-        const uint32_t s = has ? stage[i] : 0u;
-        const uint32_t fs = has ? f[s] : 1u, cs = c[s];
+    const uint32_t below = (1u << lane) - 1u;
+    // one coder step of this lane for symbol s
+    auto step = [&](uint32_t s, bool has) {
+        const uint4 en = enc[s];
+        const uint32_t fs = en.z & 0xFFFFu, cs = en.z >> 16;
         const bool emit = has && (x >> 20) >= fs;  // x >= f * 2^20
         const uint32_t votes = __ballot_sync(0xffffffffu, emit);
         if (emit) {
-            words[nw + __popc(votes & ((1u << lane) - 1u))] = (uint16_t)x;
+            words[nw + __popc(votes & below)] = (uint16_t)x;
             x >>= 16;
         }
         nw += __popc(votes);
         if (has) {
-            const uint32_t q = fs > 1 ? (uint32_t)__umul64hi((unsigned long long)x, rcp[s]) : x;
+            const unsigned long long rcp = (unsigned long long)en.x | ((unsigned long long)en.y << 32);
+            const uint32_t q = fs > 1 ? (uint32_t)__umul64hi((unsigned long long)x, rcp) : x;
             x = q * kProbScale + (x - q * fs) + cs;
         }
+    };
+    uint32_t t = (n + 31u) >> 5;
+    if (n & 31u) {  // the last, incomplete step comes first (the coder walks backwards)
+        --t;
+        const bool has = 32u * t + lane < n;
+        step(has ? stage[32u * t + lane] : 0u, has);
     }
+    while (t-- > 0) step(stage[32u * t + lane], true);
     reinterpret_cast<uint32_t*>(slot)[lane] = x;
     if (lane == 0 && (nw & 1u)) words[nw] = 0;
     __syncwarp();
@@ -181,10 +191,11 @@ __device__ __forceinline__ uint32_t encode_segment(const uint8_t* src, uint32_t 
 }
 
 // Receiver tables from the transmitted frequencies (f[] already in shared memory and synced):
-// starts c[], slot -> symbol.  Returns false (in every thread) if the table does not sum to 4096.
-// The owner of a slot is the last symbol that starts at or below it (symbols that do not occur share
-// their start with the next one, or start at 4096 behind the last occurring one).
-__device__ __forceinline__ bool decoder_tables(const uint16_t* f, uint16_t* c, uint8_t* sym, uint32_t* flag, uint32_t tid) {
+// starts c[], then one word per slot: symbol | (f - 1) << 8 | (slot - c) << 20.  Returns false (in every
+// thread) if the table does not sum to 4096.  The owner of a slot is the last symbol that starts at or
+// below it (symbols that do not occur share their start with the next one, or start at 4096 behind the
+// last occurring one).
+__device__ __forceinline__ bool decoder_tables(const uint16_t* f, uint16_t* c, uint32_t* tab, uint32_t* flag, uint32_t tid) {
     if (tid < 32) {
         uint32_t local[8], total;
         const uint32_t base = warp_prefix256(f, tid, local, total);
@@ -194,7 +205,9 @@ __device__ __forceinline__ bool decoder_tables(const uint16_t* f, uint16_t* c, u
     }
     __syncthreads();
     if (*flag == 0) return false;
-    for (uint32_t slot = tid * 16; slot < tid * 16 + 16; ++slot) {
+    // thread t fills slots 16 t .. 16 t + 15: a binary search for the owner of the first, then a walk
+    {
+        uint32_t slot = tid * 16;
         uint32_t lo = 0, hi = 255;
         while (lo < hi) {
             const uint32_t mid = (lo + hi + 1) >> 1;
@@ -203,7 +216,16 @@ __device__ __forceinline__ bool decoder_tables(const uint16_t* f, uint16_t* c, u
             else
                 hi = mid - 1;
         }
-        sym[slot] = (uint8_t)lo;
+        uint32_t cs = c[lo], fm1 = (uint32_t)f[lo] - 1u;
+        for (uint32_t k = 0; k < 16; ++k, ++slot) {
+            if (slot - cs > fm1) {  // past the owner's last slot: on to the next symbol that occurs
+                do ++lo; while (lo < 255u && c[lo + 1] <= slot);
+                cs = c[lo];
+                fm1 = (uint32_t)f[lo] - 1u;
+            }
+            // the owner occurs (f >= 1, its slots are [c, c + f)): the sum is 4096 and every slot has one
+            tab[slot] = lo | (fm1 & 0xFFFu) << 8 | ((slot - cs) & 0xFFFu) << 20;
+        }
     }
     __syncthreads();
     return true;
@@ -213,25 +235,23 @@ __device__ __forceinline__ bool decoder_tables(const uint16_t* f, uint16_t* c, u
 // Returns false (in every lane) if the words run out, are left over, or a lane does not end in the
 // start state.
 __device__ __forceinline__ bool decode_segment(const uint8_t* coded, uint32_t snw, uint32_t n, uint8_t* stage,
-                                               const uint8_t* sym, const uint16_t* f, const uint16_t* c, uint8_t* out,
-                                               uint32_t lane) {
+                                               const uint32_t* tab, uint8_t* out, uint32_t lane) {
     const uint32_t* from = reinterpret_cast<const uint32_t*>(coded);
     uint32_t* st = reinterpret_cast<uint32_t*>(stage);
     for (uint32_t i = lane; i < (segment_bytes(snw) >> 2); i += 32) st[i] = from[i];
     __syncwarp();
     const uint16_t* words = reinterpret_cast<const uint16_t*>(stage + 4 * 32);
     uint32_t x = st[lane], ptr = snw;
+    const uint32_t below = (1u << lane) - 1u;
     const uint32_t steps = (n + 31u) >> 5;
     bool ok = true;
     for (uint32_t t = 0; t < steps; ++t) {
         const uint32_t i = 32u * t + lane;
-        const bool has = i < n;
         bool need = false;
-        if (has) {
-            const uint32_t slot = x & (kProbScale - 1u);
-            const uint32_t s = sym[slot];
-            out[i] = (uint8_t)s;
-            x = (uint32_t)f[s] * (x >> kProbBits) + slot - c[s];
+        if (t + 1u < steps || i < n) {  // only the last step can be incomplete
+            const uint32_t en = tab[x & (kProbScale - 1u)];
+            out[i] = (uint8_t)en;
+            x = (((en >> 8) & 0xFFFu) + 1u) * (x >> kProbBits) + (en >> 20);
             need = x < kRansL;
         }
         const uint32_t votes = __ballot_sync(0xffffffffu, need);
@@ -240,7 +260,7 @@ __device__ __forceinline__ bool decode_segment(const uint8_t* coded, uint32_t sn
             ok = false;
             break;
         }
-        if (need) x = (x << 16) | words[ptr - k_need + __popc(votes & ((1u << lane) - 1u))];
+        if (need) x = (x << 16) | words[ptr - k_need + __popc(votes & below)];
         ptr -= k_need;
     }
     ok = ok && ptr == 0 && !__any_sync(0xffffffffu, x != kRansL);
@@ -294,14 +314,14 @@ __device__ __forceinline__ uint32_t block_scan(uint32_t v, uint32_t* scan, uint3
 // ------------------------------------------------------------------------------------------ sender
 // units of up to kLongSegs segment slots: one thread block per unit, start to end
 
-__global__ void __launch_bounds__(kEntThreads)
+__global__ void __launch_bounds__(kEntThreads, 5)
 entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
                       uint32_t sm_bytes_per_value, uint32_t log2b, uint8_t* msgs, unsigned long long* wire_bytes,
                       uint8_t* scratch_slots, uint32_t* scratch_nw) {
     __shared__ __align__(16) uint8_t s_seg[kEntWarps][kSegment];  // a warp's segment of raw payload
     __shared__ uint32_t s_hist[kEntWarps][256];
-    __shared__ uint16_t s_f[256], s_c[256];
-    __shared__ unsigned long long s_rcp[256];
+    __shared__ uint16_t s_f[256];
+    __shared__ uint4 s_enc[256];
     __shared__ uint32_t s_scan[kEntWarps];
     __shared__ unsigned long long s_total;
     const uint32_t unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
@@ -327,13 +347,13 @@ entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long 
     }
     __syncthreads();
     normalise_model(s_hist[0], P, s_f, tid);
-    encoder_tables(s_f, s_c, s_rcp, tid);
+    encoder_tables(s_f, s_enc, tid);
 
     // 3. segments: warp w codes segments w, w + 8, ... into the unit's slots of the scratch
     const unsigned long long slot0 = seg_base[unit];
     for (uint32_t g = warp; g < nseg; g += kEntWarps) {
         const uint32_t n = (uint32_t)min((uint64_t)kSegment, P - (uint64_t)g * kSegment);
-        const uint32_t nw = encode_segment(pay + (uint64_t)g * kSegment, n, s_seg[warp], s_f, s_c, s_rcp,
+        const uint32_t nw = encode_segment(pay + (uint64_t)g * kSegment, n, s_seg[warp], s_enc,
                                            scratch_slots + (slot0 + g) * kSegSlot, lane);
         if (lane == 0) {
             scratch_nw[slot0 + g] = nw;
@@ -438,8 +458,8 @@ entropy_long_encode_kernel(const ciera_unit* __restrict__ units, const unsigned 
                            const unsigned long long* wire_bytes, uint8_t* recs, uint8_t* scratch_slots,
                            uint32_t* scratch_nw) {
     __shared__ __align__(16) uint8_t s_seg[kEntWarps][kSegment];
-    __shared__ uint16_t s_f[256], s_c[256];
-    __shared__ unsigned long long s_rcp[256];
+    __shared__ uint16_t s_f[256];
+    __shared__ uint4 s_enc[256];
     __shared__ unsigned long long s_total;
     const uint4 ch = chunks[blockIdx.x];
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
@@ -452,12 +472,12 @@ entropy_long_encode_kernel(const ciera_unit* __restrict__ units, const unsigned 
     s_f[tid] = long_model(recs, ch.z)[tid];
     if (tid == 0) s_total = 0;
     __syncthreads();
-    encoder_tables(s_f, s_c, s_rcp, tid);
+    encoder_tables(s_f, s_enc, tid);
     const uint8_t* pay = msgs + un.msg_off + payoff;
     const unsigned long long slot0 = seg_base[ch.x];
     for (uint32_t g = ch.y + warp; g < g_end; g += kEntWarps) {
         const uint32_t n = (uint32_t)min((uint64_t)kSegment, P - (uint64_t)g * kSegment);
-        const uint32_t nw = encode_segment(pay + (uint64_t)g * kSegment, n, s_seg[warp], s_f, s_c, s_rcp,
+        const uint32_t nw = encode_segment(pay + (uint64_t)g * kSegment, n, s_seg[warp], s_enc,
                                            scratch_slots + (slot0 + g) * kSegSlot, lane);
         if (lane == 0) {
             scratch_nw[slot0 + g] = nw;
@@ -531,7 +551,7 @@ entropy_long_copy_kernel(const ciera_unit* __restrict__ units, const unsigned lo
 // units of up to kLongSegs segment slots: one thread block per unit, start to end
 
 struct DecodeShared {
-    uint8_t sym[kProbScale];       // slot -> symbol
+    uint32_t tab[kProbScale];      // slot -> symbol | (f - 1) << 8 | (slot - c) << 20
     uint16_t f[256], c[256];
     uint32_t off[kEntThreads];     // per segment: byte offset in the data part
     uint32_t nw[kEntThreads];      //              word count
@@ -573,7 +593,7 @@ entropy_decode_kernel(const ciera_unit* __restrict__ units, uint32_t smb, uint32
     }
     sh.f[tid] = reinterpret_cast<const uint16_t*>(pay)[tid];
     __syncthreads();
-    if (!decoder_tables(sh.f, sh.c, sh.sym, &sh.flag, tid)) {
+    if (!decoder_tables(sh.f, sh.c, sh.tab, &sh.flag, tid)) {
         if (tid == 0) raise_corrupt(status);
         return;
     }
@@ -594,7 +614,7 @@ entropy_decode_kernel(const ciera_unit* __restrict__ units, uint32_t smb, uint32
     uint8_t* raw = scratch_raw + un.cache_off;  // the unit's stretch of the scratch (16-byte aligned)
     for (uint32_t g = warp; g < nseg; g += kEntWarps) {
         const uint32_t n = (uint32_t)min((uint64_t)kSegment, P - (uint64_t)g * kSegment);
-        if (!decode_segment(data + sh.off[g], sh.nw[g], n, sh.seg[warp], sh.sym, sh.f, sh.c, raw + (uint64_t)g * kSegment, lane))
+        if (!decode_segment(data + sh.off[g], sh.nw[g], n, sh.seg[warp], sh.tab, raw + (uint64_t)g * kSegment, lane))
             sh.bad = 1;
     }
     __syncthreads();
@@ -692,7 +712,7 @@ entropy_long_decode_kernel(const ciera_unit* __restrict__ units, const unsigned 
     sh.f[tid] = reinterpret_cast<const uint16_t*>(pay)[tid];
     if (tid == 0) sh.bad = 0;
     __syncthreads();
-    if (!decoder_tables(sh.f, sh.c, sh.sym, &sh.flag, tid)) {
+    if (!decoder_tables(sh.f, sh.c, sh.tab, &sh.flag, tid)) {
         if (tid == 0) {
             st->bad = 1;
             raise_corrupt(status);
@@ -705,7 +725,7 @@ entropy_long_decode_kernel(const ciera_unit* __restrict__ units, const unsigned 
     const uint32_t g_end = min(nseg, ch.y + kLongSegs);
     for (uint32_t g = ch.y + warp; g < g_end; g += kEntWarps) {
         const uint32_t n = (uint32_t)min((uint64_t)kSegment, P - (uint64_t)g * kSegment);
-        if (!decode_segment(data + scratch_off[slot0 + g], scratch_nw[slot0 + g], n, sh.seg[warp], sh.sym, sh.f, sh.c,
+        if (!decode_segment(data + scratch_off[slot0 + g], scratch_nw[slot0 + g], n, sh.seg[warp], sh.tab,
                             raw + (uint64_t)g * kSegment, lane))
             sh.bad = 1;
     }
