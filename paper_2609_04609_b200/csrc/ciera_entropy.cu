@@ -160,9 +160,17 @@ __device__ __forceinline__ uint32_t encode_segment(const uint8_t* src, uint32_t 
     uint16_t* words = reinterpret_cast<uint16_t*>(slot + 4 * 32);
     uint32_t x = kRansL, nw = 0;
     const uint32_t below = (1u << lane) - 1u;
-    // one coder step of this lane for symbol s
-    auto step = [&](uint32_t s, bool has) {
-        const uint4 en = enc[s];
+    const uint32_t enc_a = (uint32_t)__cvta_generic_to_shared(enc);
+    const uint32_t stage_a = (uint32_t)__cvta_generic_to_shared(stage) + lane;
+    // one coder step of this lane for the symbol at byte 32 t + lane of the segment
+    auto step = [&](uint32_t t, bool has) {
+        uint32_t s = 0;
+        if (has) asm volatile("ld.shared.u8 %0, [%1];" : "=r"(s) : "r"(stage_a + 32u * t) : "memory");
+        uint4 en;
+        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(en.x), "=r"(en.y), "=r"(en.z), "=r"(en.w)
+                     : "r"(enc_a + (s << 4))
+                     : "memory");
         const uint32_t fs = en.z & 0xFFFFu, cs = en.z >> 16;
         const bool emit = has && (x >> 20) >= fs;  // x >= f * 2^20
         const uint32_t votes = __ballot_sync(0xffffffffu, emit);
@@ -180,10 +188,9 @@ __device__ __forceinline__ uint32_t encode_segment(const uint8_t* src, uint32_t 
     uint32_t t = (n + 31u) >> 5;
     if (n & 31u) {  // the last, incomplete step comes first (the coder walks backwards)
         --t;
-        const bool has = 32u * t + lane < n;
-        step(has ? stage[32u * t + lane] : 0u, has);
+        step(t, lane < (n & 31u));
     }
-    while (t-- > 0) step(stage[32u * t + lane], true);
+    while (t-- > 0) step(t, true);
     reinterpret_cast<uint32_t*>(slot)[lane] = x;
     if (lane == 0 && (nw & 1u)) words[nw] = 0;
     __syncwarp();
@@ -240,29 +247,38 @@ __device__ __forceinline__ bool decode_segment(const uint8_t* coded, uint32_t sn
     uint32_t* st = reinterpret_cast<uint32_t*>(stage);
     for (uint32_t i = lane; i < (segment_bytes(snw) >> 2); i += 32) st[i] = from[i];
     __syncwarp();
-    const uint16_t* words = reinterpret_cast<const uint16_t*>(stage + 4 * 32);
+    // shared-memory addresses of the word list and the slot table, and this lane's output position
+    const uint32_t words_a = (uint32_t)__cvta_generic_to_shared(stage + 4 * 32);
+    const uint32_t tab_a = (uint32_t)__cvta_generic_to_shared(tab);
     uint32_t x = st[lane], ptr = snw;
     const uint32_t below = (1u << lane) - 1u;
-    const uint32_t steps = (n + 31u) >> 5;
+    const uint32_t full = n >> 5;  // steps in which every lane has a symbol
+    uint8_t* o = out + lane;
     bool ok = true;
-    for (uint32_t t = 0; t < steps; ++t) {
-        const uint32_t i = 32u * t + lane;
+    // one step: `has` = this lane decodes a symbol in it
+    auto step = [&](bool has) -> bool {
         bool need = false;
-        if (t + 1u < steps || i < n) {  // only the last step can be incomplete
-            const uint32_t en = tab[x & (kProbScale - 1u)];
-            out[i] = (uint8_t)en;
+        if (has) {
+            uint32_t en;
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(en) : "r"(tab_a + ((x & (kProbScale - 1u)) << 2)) : "memory");
+            *o = (uint8_t)en;
             x = (((en >> 8) & 0xFFFu) + 1u) * (x >> kProbBits) + (en >> 20);
             need = x < kRansL;
         }
+        o += 32;
         const uint32_t votes = __ballot_sync(0xffffffffu, need);
         const uint32_t k_need = __popc(votes);
-        if (k_need > ptr) {
-            ok = false;
-            break;
-        }
-        if (need) x = (x << 16) | words[ptr - k_need + __popc(votes & below)];
+        if (k_need > ptr) return false;  // the words run out (the same in every lane)
         ptr -= k_need;
-    }
+        if (need) {
+            uint32_t w;
+            asm volatile("ld.shared.u16 %0, [%1];" : "=r"(w) : "r"(words_a + ((ptr + __popc(votes & below)) << 1)) : "memory");
+            x = (x << 16) | w;
+        }
+        return true;
+    };
+    for (uint32_t t = 0; t < full && ok; ++t) ok = step(true);
+    if (ok && (n & 31u)) ok = step(lane < (n & 31u));
     ok = ok && ptr == 0 && !__any_sync(0xffffffffu, x != kRansL);
     __syncwarp();
     return ok;
