@@ -238,19 +238,20 @@ __device__ __forceinline__ bool decoder_tables(const uint16_t* f, uint16_t* c, u
     return true;
 }
 
-// One warp decodes one segment: coded (32 states + snw words, 4-byte aligned) -> out[0, n).
+// One warp decodes one segment: coded (32 states + snw words, 4-byte aligned, in global memory) ->
+// out[0, n).  The words are read where they lie (a step takes a handful of neighbouring words from the
+// end of what is left, so the reads of a warp fall into one or two cache lines that stay in L1 for the
+// next steps); without a staged copy the kernel's shared memory is the slot table, and many warps per
+// SM hide the latency of a line's first touch.
 // Returns false (in every lane) if the words run out, are left over, or a lane does not end in the
 // start state.
-__device__ __forceinline__ bool decode_segment(const uint8_t* coded, uint32_t snw, uint32_t n, uint8_t* stage,
-                                               const uint32_t* tab, uint8_t* out, uint32_t lane) {
-    const uint32_t* from = reinterpret_cast<const uint32_t*>(coded);
-    uint32_t* st = reinterpret_cast<uint32_t*>(stage);
-    for (uint32_t i = lane; i < (segment_bytes(snw) >> 2); i += 32) st[i] = from[i];
-    __syncwarp();
-    // shared-memory addresses of the word list and the slot table, and this lane's output position
-    const uint32_t words_a = (uint32_t)__cvta_generic_to_shared(stage + 4 * 32);
+__device__ __forceinline__ bool decode_segment(const uint8_t* coded, uint32_t snw, uint32_t n, const uint32_t* tab,
+                                               uint8_t* out, uint32_t lane) {
+    const uint16_t* words = reinterpret_cast<const uint16_t*>(coded + 4 * 32);
+    for (uint32_t i = lane * 64u; i < snw; i += 32u * 64u)  // bring the word list towards the SM, a line per lane
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(words + i));
     const uint32_t tab_a = (uint32_t)__cvta_generic_to_shared(tab);
-    uint32_t x = st[lane], ptr = snw;
+    uint32_t x = reinterpret_cast<const uint32_t*>(coded)[lane], ptr = snw;
     const uint32_t below = (1u << lane) - 1u;
     const uint32_t full = n >> 5;  // steps in which every lane has a symbol
     uint8_t* o = out + lane;
@@ -270,11 +271,7 @@ __device__ __forceinline__ bool decode_segment(const uint8_t* coded, uint32_t sn
         const uint32_t k_need = __popc(votes);
         if (k_need > ptr) return false;  // the words run out (the same in every lane)
         ptr -= k_need;
-        if (need) {
-            uint32_t w;
-            asm volatile("ld.shared.u16 %0, [%1];" : "=r"(w) : "r"(words_a + ((ptr + __popc(votes & below)) << 1)) : "memory");
-            x = (x << 16) | w;
-        }
+        if (need) x = (x << 16) | words[ptr + __popc(votes & below)];
         return true;
     };
     for (uint32_t t = 0; t < full && ok; ++t) ok = step(true);
@@ -574,7 +571,6 @@ struct DecodeShared {
     uint32_t scan[kEntWarps];
     unsigned long long changed;    // set bits of the unit's bitmap
     uint32_t flag, bad;
-    __align__(16) uint8_t seg[kEntWarps][kSegSlot];  // a warp's coded segment
 };
 
 __device__ __forceinline__ void raise_corrupt(int32_t* status) {
@@ -630,7 +626,7 @@ entropy_decode_kernel(const ciera_unit* __restrict__ units, uint32_t smb, uint32
     uint8_t* raw = scratch_raw + un.cache_off;  // the unit's stretch of the scratch (16-byte aligned)
     for (uint32_t g = warp; g < nseg; g += kEntWarps) {
         const uint32_t n = (uint32_t)min((uint64_t)kSegment, P - (uint64_t)g * kSegment);
-        if (!decode_segment(data + sh.off[g], sh.nw[g], n, sh.seg[warp], sh.tab, raw + (uint64_t)g * kSegment, lane))
+        if (!decode_segment(data + sh.off[g], sh.nw[g], n, sh.tab, raw + (uint64_t)g * kSegment, lane))
             sh.bad = 1;
     }
     __syncthreads();
@@ -741,7 +737,7 @@ entropy_long_decode_kernel(const ciera_unit* __restrict__ units, const unsigned 
     const uint32_t g_end = min(nseg, ch.y + kLongSegs);
     for (uint32_t g = ch.y + warp; g < g_end; g += kEntWarps) {
         const uint32_t n = (uint32_t)min((uint64_t)kSegment, P - (uint64_t)g * kSegment);
-        if (!decode_segment(data + scratch_off[slot0 + g], scratch_nw[slot0 + g], n, sh.seg[warp], sh.tab,
+        if (!decode_segment(data + scratch_off[slot0 + g], scratch_nw[slot0 + g], n, sh.tab,
                             raw + (uint64_t)g * kSegment, lane))
             sh.bad = 1;
     }
