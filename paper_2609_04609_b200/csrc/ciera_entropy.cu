@@ -332,7 +332,10 @@ entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long 
                       uint32_t sm_bytes_per_value, uint32_t log2b, uint8_t* msgs, unsigned long long* wire_bytes,
                       uint8_t* scratch_slots, uint32_t* scratch_nw) {
     __shared__ __align__(16) uint8_t s_seg[kEntWarps][kSegment];  // a warp's segment of raw payload
-    __shared__ uint32_t s_hist[kEntWarps][256];
+    // the warps' private histograms are needed before the segments are staged, the two small lists of
+    // step 4 after: all of them lie in the first part of s_seg
+    uint32_t (*const s_hist)[256] = reinterpret_cast<uint32_t (*)[256]>(&s_seg[0][0]);
+    static_assert(sizeof(uint32_t) * 256 * kEntWarps <= sizeof(uint8_t) * kSegment * kEntWarps, "histograms overlay the stages");
     __shared__ uint16_t s_f[256];
     __shared__ uint4 s_enc[256];
     __shared__ uint32_t s_scan[kEntWarps];
