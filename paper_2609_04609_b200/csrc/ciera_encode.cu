@@ -39,6 +39,8 @@
 // into hash terms and add them up over the lanes that share a block, and the aggregator finishes
 // the hashes, compares them with the cached ones, refreshes HashCache and derives the block flags
 // from the comparison.
+#include <cstddef>
+
 #include "ciera_bits.cuh"
 #include "ciera_hash.cuh"
 #include "ciera_lookback.cuh"
@@ -180,7 +182,7 @@ struct EncodeCtl {
     uint32_t tile_idx[kDescRing];  // table index of the tile in desc[]; kNoTile = end marker
     uint32_t seq[kDescRing];       // 1: tile of a unit this block works through alone
     uint32_t ballot[SE][kVoteWords];  // coarse blocks: "my piece differs" votes
-    uint32_t bm[SE][BW];              // block flags of the tile
+    uint32_t bm[SE][BW];              // block flags of the tile (16-byte aligned: checked where the kernel starts)
     uint16_t pre[SE][BW];             // set flags before each word of bm
     unsigned long long agg[SE];
     unsigned long long base[SE];
@@ -231,8 +233,48 @@ struct TileWalk {
 
 // Fine blocks: the consumers have written the block flags themselves; fills pre (set bits before
 // each word) and returns the number of changed blocks of the tile (one warp).
+// Lane l takes the W = nwords / 32 consecutive words l W .. l W + W - 1 (1, 2, 4 or 8), so that one scan over
+// the lanes does for the whole tile.
+template <int W>
+__device__ __forceinline__ uint32_t scan_block_bitmap_w(const uint32_t* bm, uint16_t* pre, uint32_t lane) {
+    uint32_t w[W];
+    if constexpr (W >= 4) {
+#pragma unroll
+        for (int i = 0; i < W / 4; ++i) {
+            const uint4 v = reinterpret_cast<const uint4*>(bm)[lane * (W / 4) + i];
+            w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < W; ++i) w[i] = bm[lane * W + i];
+    }
+    uint32_t before[W], sum = 0;
+#pragma unroll
+    for (int i = 0; i < W; ++i) {
+        before[i] = sum;
+        sum += __popc(w[i]);
+    }
+    uint32_t incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+        if ((int)lane >= o) incl += t;
+    }
+    const uint32_t base = incl - sum;
+    if constexpr (W >= 2) {  // two 16-bit counts per store
+        uint32_t* pre32 = reinterpret_cast<uint32_t*>(pre) + lane * (W / 2);
+#pragma unroll
+        for (int i = 0; i < W / 2; ++i) pre32[i] = (base + before[2 * i]) | ((base + before[2 * i + 1]) << 16);
+    } else {
+        pre[lane] = (uint16_t)base;
+    }
+    const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
+    __syncwarp();
+    return total;
+}
 __device__ __forceinline__ uint32_t scan_block_bitmap(const uint32_t* bm, uint16_t* pre, uint32_t log2b, uint32_t lane) {
-    const uint32_t nwords = kTileValues >> (log2b + 5);  // 32 .. 256
+    if (log2b == 0) return scan_block_bitmap_w<8>(bm, pre, lane);  // 256 words: eight per lane, one scan
+    const uint32_t nwords = kTileValues >> (log2b + 5);  // 32 .. 128: a scan per 32 words
     uint32_t run = 0;
     for (uint32_t base = 0; base < nwords; base += 32) {
         const uint32_t pc = __popc(bm[base + lane]);
@@ -375,7 +417,10 @@ __device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t 
         const uint64_t byte0 = (uint64_t)td.tile_in_unit * (nbt >> 3);
         const uint32_t nbytes = (((nv + B - 1u) >> log2b) + 7u) >> 3;
         uint32_t* dst32 = reinterpret_cast<uint32_t*>(msg + byte0);
-        for (uint32_t w = lane; w < (nbytes >> 2); w += 32) dst32[w] = bm[w];
+        // 16 bytes at a time, then the last words, then the last bytes
+        const uint32_t quads = nbytes >> 4;
+        for (uint32_t c = lane; c < quads; c += 32) reinterpret_cast<uint4*>(dst32)[c] = reinterpret_cast<const uint4*>(bm)[c];
+        for (uint32_t w = 4u * quads + lane; w < (nbytes >> 2); w += 32) dst32[w] = bm[w];
         const uint32_t done = nbytes & ~3u;
         if (lane < nbytes - done) msg[byte0 + done + lane] = (uint8_t)(bm[done >> 2] >> (lane * 8u));
     } else if (nbt >= 8) {
@@ -533,6 +578,7 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
     Ctl* ctl = reinterpret_cast<Ctl*>(ring_e + (size_t)SE * kEBytes);
     // HASH: per stage of the exponent ring, the tile's cached hashes and then the partial sums
     static_assert(sizeof(Ctl) % 16 == 0, "the hash stages follow the control block");
+    static_assert(offsetof(Ctl, bm) % 16 == 0 && offsetof(Ctl, pre) % 4 == 0, "block flags are read 16 bytes at a time");
     uint8_t* const ring_h = reinterpret_cast<uint8_t*>(ctl) + sizeof(Ctl);
     const uint32_t kHoldBytes = HASH ? hash_hold_bytes<DT>(log2b) : 0u;
     const uint32_t kHStage = HASH ? kHoldBytes + hash_part_bytes<DT>(log2b) : 0u;
