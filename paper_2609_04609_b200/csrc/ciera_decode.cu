@@ -21,6 +21,8 @@
 // units of up to kDirectBlocks blocks a producer takes it straight from the bitmap (at most four
 // words per lane, fetched one tile ahead); longer units get it from a small prefix kernel that
 // runs first and writes one count per tile into the caller's scratch.
+#include <cstddef>
+
 #include "ciera_bits.cuh"
 #include "ciera_pipe.cuh"
 
@@ -97,6 +99,9 @@ struct __align__(16) DecodeRing {
     uint32_t raw_own[FINE ? 4 : kBitmapWords];               // words holding the tile's own bits
 };
 
+static_assert(offsetof(DecodeRing<true>, bm) % 16 == 0 && offsetof(DecodeRing<true>, pre) % 4 == 0,
+              "with blocks of one value the flags are digested 16 bytes at a time");
+
 template <int S, int R, bool FINE>
 struct DecodeCtl {
     uint64_t full[S];   // stage filled (producer arrive + bulk-copy bytes)
@@ -159,6 +164,40 @@ __device__ __forceinline__ uint64_t digest_bitmap(DecodeRing<FINE>* r, const Til
     const uint32_t nv = (uint32_t)min((uint64_t)kTileValues, td.n_unit - v0);
     const uint32_t nblk = (nv + (1u << log2b) - 1u) >> log2b;  // valid blocks of this tile
     uint32_t cnt = 0;
+    if (FINE && log2b == 0) {
+        // blocks of one value: 256 words; lane l takes words 8 l .. 8 l + 7, one scan does for the tile
+        uint32_t w[8], before8[8], sum = 0;
+        uint4* const bm4 = reinterpret_cast<uint4*>(r->bm) + 2u * lane;
+        const uint4 v0w = bm4[0], v1w = bm4[1];
+        w[0] = v0w.x; w[1] = v0w.y; w[2] = v0w.z; w[3] = v0w.w;
+        w[4] = v1w.x; w[5] = v1w.y; w[6] = v1w.z; w[7] = v1w.w;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t first = (8u * lane + (uint32_t)i) * 32u;  // the word's first block
+            // flags past the tile's last block are dropped (words past the bitmap's end were not fetched)
+            if (first >= nblk)
+                w[i] = 0;
+            else if (nblk - first < 32u)
+                w[i] &= (1u << (nblk - first)) - 1u;
+            before8[i] = sum;
+            sum += __popc(w[i]);
+        }
+        uint32_t incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+            if ((int)lane >= o) incl += t;
+        }
+        const uint32_t base = incl - sum;
+        bm4[0] = make_uint4(w[0], w[1], w[2], w[3]);
+        bm4[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        uint32_t* const pre32 = reinterpret_cast<uint32_t*>(r->pre) + 4u * lane;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) pre32[i] = (base + before8[2 * i]) | ((base + before8[2 * i + 1]) << 16);
+        own_total = __shfl_sync(0xffffffffu, incl, 31);
+        __syncwarp();
+        return td.tile_in_unit != 0 ? r->ws : 0u;
+    }
     if (FINE) {
         // flags past the tile's last block are dropped (words past the bitmap's end were not fetched)
         uint32_t run = 0;
