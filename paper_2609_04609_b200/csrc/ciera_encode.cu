@@ -828,10 +828,16 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
                             reinterpret_cast<uint8_t*>(words)[lane] = (uint8_t)flags;
                         } else if (k_l2 == 4) {  // two bytes per piece
                             reinterpret_cast<uint16_t*>(words)[lane] = (uint16_t)flags;
+                        } else if (k_l2 == 0) {  // one flag per piece: the vote is the word
+                            const uint32_t v = __ballot_sync(0xffffffffu, flags != 0);
+                            if (lane == 0) words[0] = v;
                         } else {
-                            uint32_t v = flags << ((lane << k_l2) & 31u);
-                            for (uint32_t o = 1; o < (32u >> k_l2); o <<= 1) v |= __shfl_xor_sync(0xffffffffu, v, o);
-                            if ((lane & ((32u >> k_l2) - 1u)) == 0) words[lane >> (5u - k_l2)] = v;
+                            // two or four flags per piece: 4 or 2 neighbouring lanes fill a byte
+                            uint32_t v = flags << ((lane << k_l2) & 7u);
+                            v |= __shfl_xor_sync(0xffffffffu, v, 1);
+                            if (k_l2 == 1) v |= __shfl_xor_sync(0xffffffffu, v, 2);
+                            if ((lane & ((8u >> k_l2) - 1u)) == 0)
+                                reinterpret_cast<uint8_t*>(words)[lane >> (3u - k_l2)] = (uint8_t)v;
                         }
                     }
                     // sign-plus-mantissa of every value
