@@ -55,6 +55,7 @@ struct Global {
     static __device__ __forceinline__ void st16(uint8_t* p, uint4 v) { st_stream16(p, v); }
     static __device__ __forceinline__ void st8(uint8_t* p, uint2 v) { st_stream8(p, v); }
     static __device__ __forceinline__ uint32_t ld1(const uint8_t* p) { return __ldcs(p); }
+    static __device__ __forceinline__ uint32_t ld2(const uint8_t* p) { return __ldcs(reinterpret_cast<const uint16_t*>(p)); }
     static __device__ __forceinline__ uint32_t ld4(const uint8_t* p) { return __ldcs(reinterpret_cast<const uint32_t*>(p)); }
 };
 struct Shared {
@@ -65,6 +66,11 @@ struct Shared {
     static __device__ __forceinline__ uint32_t ld1(const uint8_t* p) {
         uint32_t v;
         asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"((uint32_t)__cvta_generic_to_shared(p)));
+        return v;
+    }
+    static __device__ __forceinline__ uint32_t ld2(const uint8_t* p) {
+        uint32_t v;
+        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"((uint32_t)__cvta_generic_to_shared(p)));
         return v;
     }
     static __device__ __forceinline__ uint32_t ld4(const uint8_t* p) {

@@ -313,6 +313,40 @@ __device__ __forceinline__ void unchanged_span_fine(const uint32_t* bm, uint32_t
 // x.e value by value.  Only the first nvalid values exist.
 template <int DT, class M>
 __device__ __forceinline__ void gather_changed(Piece<DT>& x, uint32_t km, uint32_t log2b, const uint8_t* src, int nvalid) {
+    constexpr int kV = Piece<DT>::kValues;
+    if (nvalid == kV && log2b != 0) {
+        // a complete piece of blocks of 2, 4 or 8 values: a changed block's exponents come with one load
+        // (the payload holds whole blocks up to here, so `src` is a multiple of the block size)
+        if (log2b == 3) {
+#pragma unroll
+            for (int j = 0; j < kV / 8; ++j) {
+                if ((km >> j) & 1u) {
+                    const uint2 v = M::ld8(src);
+                    src += 8;
+                    x.e[2 * j] = v.x;
+                    x.e[2 * j + 1] = v.y;
+                }
+            }
+        } else if (log2b == 2) {
+#pragma unroll
+            for (int j = 0; j < kV / 4; ++j) {
+                if ((km >> j) & 1u) {
+                    x.e[j] = M::ld4(src);
+                    src += 4;
+                }
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < kV / 2; ++j) {
+                if ((km >> j) & 1u) {
+                    const uint32_t h = M::ld2(src);
+                    src += 2;
+                    x.e[j >> 1] = __byte_perm(x.e[j >> 1], h, (j & 1) ? 0x5410u : 0x3254u);
+                }
+            }
+        }
+        return;
+    }
     uint32_t cnt = 0;
 #pragma unroll
     for (int i = 0; i < Piece<DT>::kValues; ++i) {
