@@ -101,15 +101,17 @@ def test_hashed_reduced_moe_layer_and_zero_start(rt, dtype, block):
     _run(rt, sizes, 4, dtype, block, traj[:2], from_zero=True)
 
 
-def test_hashed_long_unit_of_many_tiles(rt):
-    """One unit of ~3 M values = 367 tiles: more than one chunk of the per-unit running count."""
+@pytest.mark.parametrize("dtype,block", [(0, 128), (0, 32), (1, 4096), (1, 64)])
+def test_hashed_long_unit_of_many_tiles(rt, dtype, block):
+    """One unit of ~3 M values = 367 tiles (its tiles are spread over the thread blocks and find their
+    payload offsets by look-back) beside a shorter one; long and short rings of the kernel."""
     sizes = [3_000_000 + 123, 600_000]
-    n = rt[1].LayerCodec.from_tensors(sizes, 1, "bf16", 128, DEV).weights_bytes // 2
-    gen = wl.make_generator(77)
-    w0 = wl.init_weights(n, "bf16", gen)
+    n = rt[1].LayerCodec.from_tensors(sizes, 1, NAME[dtype], block, DEV).weights_bytes // VB[dtype]
+    gen = wl.make_generator(77 + block)
+    w0 = wl.init_weights(n, NAME[dtype], gen)
     w1 = wl.inject_exponent_changes(w0, gen, 0.002)
     w2 = wl.inject_exponent_changes(w1, gen, 0.2)
-    _run(rt, sizes, 1, 0, 128, [wl.as_bits(w) for w in (w0, w1, w2)])
+    _run(rt, sizes, 1, dtype, block, [wl.as_bits(w) for w in (w0, w1, w2)])
 
 
 def test_hashed_rejects_fine_blocks(rt):
