@@ -368,19 +368,20 @@ struct Piece<CIERA_FP16> {
 
     // w = eight fp16 values, two per word
     __device__ __forceinline__ void split_words(const uint32_t w[4]) {
-        uint32_t e2[4], f[8];
+        // p[i] = the two values' 11-bit fields side by side (22 bits): mantissa bits 9:0 stay, the sign
+        // (bit 15) moves to bit 10, the second value's mantissa (bits 25:16) to 20:11, its sign (bit 31) to 21
+        uint32_t e2[4], p[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            e2[i] = (w[i] >> 10) & 0x001F001Fu;
-            const uint32_t sm2 = (w[i] & 0x03FF03FFu) | ((w[i] >> 5) & 0x04000400u);
-            f[2 * i] = sm2 & 0xFFFFu;
-            f[2 * i + 1] = sm2 >> 16;
+            const uint32_t t5 = w[i] >> 5, t10 = w[i] >> 10;
+            e2[i] = t10 & 0x001F001Fu;
+            p[i] = (w[i] & 0x000003FFu) | (t5 & 0x001FFC00u) | (t10 & 0x00200000u);
         }
         e[0] = __byte_perm(e2[0], e2[1], 0x6420);
         e[1] = __byte_perm(e2[2], e2[3], 0x6420);
-        s[0] = f[0] | (f[1] << 11) | (f[2] << 22);
-        s[1] = (f[2] >> 10) | (f[3] << 1) | (f[4] << 12) | (f[5] << 23);
-        s[2] = (f[5] >> 9) | (f[6] << 2) | (f[7] << 13);
+        s[0] = p[0] | (p[1] << 22);
+        s[1] = (p[1] >> 10) | (p[2] << 12);
+        s[2] = (p[2] >> 20) | (p[3] << 2);
     }
     __device__ __forceinline__ void merge_words(uint32_t w[4]) const {
         uint32_t f[8];
