@@ -96,6 +96,21 @@ def max_over_ranks(ms: float, world: int, device=None) -> float:
     return float(t.item())
 
 
+def host_memory_allows(need_bytes: int, world: int, device=None) -> bool:
+    """True on every rank iff on every rank `need_bytes` is at most 60 % of the free host memory."""
+    import psutil
+
+    ok = 1.0 if need_bytes <= 0.6 * psutil.virtual_memory().available else 0.0
+    if world > 1:
+        import torch
+        import torch.distributed as dist
+
+        t = torch.tensor([ok], dtype=torch.float64, device=device if device is not None else "cpu")
+        dist.all_reduce(t, op=dist.ReduceOp.MIN)
+        ok = float(t.item())
+    return ok > 0.5
+
+
 def whole_job_gbps(world: int, bytes_per_rank: int, ms_per_step: float) -> float:
     """Weak scaling: every rank processes its own stack; the job's throughput is the sum."""
     return world * bytes_per_rank / (ms_per_step * 1e-3) / 1e9
@@ -603,7 +618,13 @@ def main():
 
     # ---- end to end through the host-buffer entry point (weights start and end in host memory)
     if not args.no_e2e:
-        out["e2e"] = e2e(args, layers, wa, wb, world, rank, barrier)
+        # three pinned host copies of the stack per rank; all ranks of the node share its memory
+        need = 3 * sum(w.numel() for w in wa) * int(os.environ.get("LOCAL_WORLD_SIZE", str(world)))
+        if host_memory_allows(need, world, device):
+            out["e2e"] = e2e(args, layers, wa, wb, world, rank, barrier)
+        else:
+            out["e2e"] = {"value": None, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                          "skipped": f"{need} bytes of pinned host memory would be more than 60 % of what is free"}
 
     # ---- the oracle on this machine's host cores (rank 0, one GPU only)
     if not args.no_cpu_baseline and rank == 0 and world == 1:

@@ -22,7 +22,9 @@ def _worker(rank, world, port, out):
     local_ms = 1.0 if rank == 0 else 3.0
     ms = bench.max_over_ranks(local_ms, world)
     dist.barrier()
-    out[rank] = (ms, bench.whole_job_gbps(world, 12_000_000_000, ms), bench.rank_seed(rank))
+    # rank 1 asks for more host memory than any machine has: every rank must then hear "no"
+    allowed = (bench.host_memory_allows(1 << 20, world), bench.host_memory_allows((1 << 20) if rank == 0 else (1 << 60), world))
+    out[rank] = (ms, bench.whole_job_gbps(world, 12_000_000_000, ms), bench.rank_seed(rank), allowed)
     dist.destroy_process_group()
 
 
@@ -33,6 +35,7 @@ def test_two_gloo_ranks_agree_on_the_slowest_time_and_the_job_throughput():
     assert out[0][0] == out[1][0] == 3.0
     assert out[0][1] == pytest.approx(2 * 12e9 / 3e-3 / 1e9)
     assert out[0][2] != out[1][2]
+    assert out[0][3] == out[1][3] == (True, False)
 
 
 def test_single_rank_needs_no_process_group():
