@@ -1,7 +1,10 @@
 """Randomised differential test of the whole CUDA path against the oracles: random unit tables
 (empty, tiny, ragged and multi-tile units), every block size, both precisions, random update models
 and start states; with blocks of 16 values and more also the hashed sender and the entropy stage.
-Seeds are fixed: the cases are the same on every run."""
+Seeds are fixed: the cases are the same on every run.  CIERA_FUZZ_CASES=<n> in the environment runs n
+cases of each kind instead of the default 60 / 20 (a longer soak)."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -18,6 +21,8 @@ WDT = {0: np.uint16, 1: np.uint32, 2: np.uint16}
 VB = {0: 2, 1: 4, 2: 2}
 NAME = {0: "bf16", 1: "fp32", 2: "fp16"}
 BLOCKS = [1, 2, 4, 8, 16, 32, 64, 128, 256, 512, 1024, 2048, 4096]
+N_FULL = int(os.environ.get("CIERA_FUZZ_CASES", "60"))
+N_HASHED = int(os.environ.get("CIERA_FUZZ_CASES", "20"))
 
 
 @pytest.fixture(scope="module")
@@ -60,7 +65,7 @@ def _trajectory(rng, n, dtype):
     return [wl.as_bits(w) for w in wl.trajectory(n, NAME[dtype], int(rng.integers(1, 1 << 30)), 2, model, **kw)]
 
 
-@pytest.mark.parametrize("seed", range(60))
+@pytest.mark.parametrize("seed", range(N_FULL))
 def test_random_tables_full_step(rt, seed):
     ciera, runtime = rt
     rng, sizes, shards, dtype, block = _random_case(1000 + seed)
@@ -82,7 +87,7 @@ def test_random_tables_full_step(rt, seed):
         compare_recon(codec, exp, w, dtype, f"{label} t={t}")
 
 
-@pytest.mark.parametrize("seed", range(20))
+@pytest.mark.parametrize("seed", range(N_HASHED))
 def test_random_tables_hashed_sender_and_entropy_stage(rt, seed):
     ciera, runtime = rt
     rng, sizes, shards, dtype, block = _random_case(5000 + seed)
