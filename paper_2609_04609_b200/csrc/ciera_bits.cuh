@@ -528,6 +528,36 @@ __device__ __forceinline__ uint32_t build_block_bitmap(const uint32_t* ballot, u
                                                        uint32_t log2b, uint32_t pl2, uint32_t lane) {
     const uint32_t gl2 = log2b - pl2;           // log2(pieces per block)
     const uint32_t nbt = kTileValues >> log2b;  // blocks of a full tile
+    if (nbt > 32 && gl2 >= 1) {
+        // More than one word of block flags (2 to 16 pieces per block): lane l turns vote word l into
+        // its 32 >> gl2 block flags -- fold the votes of a block onto its first bit, gather those bits --
+        // the 2^gl2 lanes whose flags share a word of bm combine them, and one scan does for the tile.
+        const uint32_t vote_words = (uint32_t)kTileValues >> (pl2 + 5);  // 32 or 16
+        uint32_t t = lane < vote_words ? ballot[lane] : 0u;
+        for (uint32_t k = 0; k < gl2; ++k) t |= t >> (1u << k);
+        const uint32_t cnt = 32u >> gl2;
+        uint32_t fl = 0;
+        for (uint32_t j = 0; j < cnt; ++j) fl |= ((t >> (j << gl2)) & 1u) << j;
+        uint32_t v = fl << ((lane * cnt) & 31u);
+        for (uint32_t k = 0; k < gl2; ++k) v |= __shfl_xor_sync(0xffffffffu, v, 1u << k);
+        const uint32_t nwords = nbt >> 5;  // 2 .. 16
+        uint32_t word = __shfl_sync(0xffffffffu, v, (lane << gl2) & 31u);
+        if (lane >= nwords) word = 0u;
+        const uint32_t pc = __popc(word);
+        uint32_t incl = pc;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t u = __shfl_up_sync(0xffffffffu, incl, o);
+            if ((int)lane >= o) incl += u;
+        }
+        if (lane < nwords) {
+            bm[lane] = word;
+            pre[lane] = (uint16_t)(incl - pc);
+        }
+        const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
+        __syncwarp();
+        return total;
+    }
     uint32_t run = 0;
     for (uint32_t base = 0; base < nbt; base += 32) {
         const uint32_t i = base + lane;
