@@ -93,6 +93,7 @@ struct __align__(16) DecodeRing {
     uint32_t tile;                           // the tile's number, or kNoTile: this producer has no more work
     uint32_t pay_skew;                       // fine: bytes in front of the slice in its stage (0 .. 15)
     uint32_t ws;                             // count from the scratch (units that went through the prefix kernel)
+    uint32_t direct;                         // coarse: 1 = the few unchanged pieces read their cached exponents from global memory
     uint16_t pre[kBm];                       // set flags before each word
     // raw material of coarse blocks, fetched asynchronously one tile ahead:
     uint32_t raw_pre[FINE ? 4 : 32 * kDirectWordsPerLane];  // bitmap words before the tile
@@ -516,6 +517,14 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                     // which holds at least the values up to the end of this full tile)
                     uint32_t span0 = lo << log2b, span = lo <= hi ? (hi - lo + 1u) << log2b : 0u;
                     uint32_t skew = 0, slice = (uint32_t)payload_bytes_of_blocks<DT>(own, log2b);
+                    if (!FINE && !kHalf) {
+                        // a few unchanged blocks scattered over a long span: staging the span would mostly
+                        // move cached exponents that the payload replaces anyway
+                        const uint32_t unchanged = (uint32_t)kTileValues - (own << log2b);
+                        const bool direct = span != 0 && 4u * unchanged <= span;
+                        r->direct = direct ? 1u : 0u;
+                        if (direct) span = 0;
+                    }
                     if (FINE && span) {
                         const uint32_t end = (span0 + span + 15u) & ~15u;
                         span0 &= ~15u;
@@ -591,7 +600,10 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                         chg = (word >> (kb & 31u)) & 1u;
                         const uint8_t* esrc = chg ? st + kSmTile + kTileValues + ((size_t)rank << log2b) + (t0 & bmask)
                                                   : st + kSmTile + t0;
-                        x.template load_exp_full<Shared>(esrc);
+                        if (!chg && r->direct)
+                            x.template load_exp_full<Global>(c_ptr + t0);
+                        else
+                            x.template load_exp_full<Shared>(esrc);
                     } else {
                         // the piece's flags (they never straddle a word) pick, block by block
                         x.template load_sm_full<Shared>(st + (size_t)t0 * SMB);
