@@ -55,6 +55,8 @@ def parse_args():
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32", "fp16"])
     ap.add_argument("--update", default="clustered", choices=["clustered", "adam", "inject"])
     ap.add_argument("--inject", type=float, default=0.01, help="exponent change rate of the 'inject' update model")
+    ap.add_argument("--inject-seg", type=int, default=0,
+                    help="'inject' update model: 0 = every value changes independently; n = whole n-aligned segments change")
     ap.add_argument("--shapes", default="olmoe", choices=["olmoe", "mixed"],
                     help="olmoe: 64 experts x 3 matrices per layer; mixed: 256 fine-grained experts (2048x512, "
                          "2048x512, 512x2048) plus dense tensors of 4 KB ... 256 MB (the mixed-shape sweep)")
@@ -204,7 +206,7 @@ def build_stack(args, device, seed_base):
         elif args.update == "adam":
             step = lambda x: wl.step_adam_like(x, gen)
         else:
-            step = lambda x: wl.inject_exponent_changes(x, gen, args.inject)
+            step = lambda x: wl.inject_exponent_changes(x, gen, args.inject, args.inject_seg)
         for _ in range(4):  # iterations 1..4 of the trajectory
             w = step(w)
         w5 = step(w)  # iteration 5
@@ -335,7 +337,7 @@ def run_reference(args):
     elif args.update == "adam":
         w1 = wl.step_adam_like(w, gen)
     else:
-        w1 = wl.inject_exponent_changes(w, gen, args.inject)
+        w1 = wl.inject_exponent_changes(w, gen, args.inject, args.inject_seg)
     a = wl.as_bits(w).view(np.uint8)
     b = wl.as_bits(w1).view(np.uint8)
     threads = os.cpu_count() or 1
@@ -362,7 +364,7 @@ def run_reference(args):
 def workload_config(args):
     full = args.layers == 16 and args.experts == 64 and args.shapes == "olmoe"
     upd = f"update model {args.update}" + (f" f={args.f}" if args.update == "clustered" else "") + (
-        f" c={args.inject}" if args.update == "inject" else "")
+        f" c={args.inject}" + (f" in segments of {args.inject_seg}" if args.inject_seg else "") if args.update == "inject" else "")
     if args.shapes == "mixed":
         what = (f"mixed-shape sweep (config 5), {args.layers} x [256 fine-grained experts x (2048x512, 2048x512, "
                 f"512x2048) + dense tensors 4 KB..256 MB] {args.dtype}")
