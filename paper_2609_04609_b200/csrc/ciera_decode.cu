@@ -517,7 +517,15 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                     // which holds at least the values up to the end of this full tile)
                     uint32_t span0 = lo << log2b, span = lo <= hi ? (hi - lo + 1u) << log2b : 0u;
                     uint32_t skew = 0, slice = (uint32_t)payload_bytes_of_blocks<DT>(own, log2b);
-                    if (!FINE && !kHalf) {
+                    // Up to 32 blocks per tile (256 values and more each): one copy per run of unchanged
+                    // blocks instead of the span, so that no cached exponents of changed blocks are read.
+                    const uint32_t nbt_ = (uint32_t)kTileValues >> log2b;
+                    const bool by_runs = !FINE && !kStageOut && nbt_ <= 32u;  // (fp32, whose output goes through bulk stores, lost 6 % with it)
+                    if (by_runs) {
+                        const uint32_t zeros = ~r->bm[0] & (nbt_ == 32u ? 0xffffffffu : (1u << nbt_) - 1u);
+                        span = (uint32_t)__popc(zeros) << log2b;
+                        if (!kHalf) r->direct = 0u;
+                    } else if (!FINE && !kHalf) {
                         // a few unchanged blocks scattered over a long span: staging the span would mostly
                         // move cached exponents that the payload replaces anyway
                         const uint32_t unchanged = (uint32_t)kTileValues - (own << log2b);
@@ -539,14 +547,29 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                     }
                     mbar_arrive_expect_tx(&ctl->full[stage], kSmTile + span + slice);
                     bulk_load(st, r->sm_src, kSmTile, &ctl->full[stage]);
-                    if (span) bulk_load(st + kSmTile + span0, r->c_ptr + span0, span, &ctl->full[stage]);
+                    // (by_runs: the copies of the runs are started by the warp's lanes, one run each, below)
+                    if (!by_runs && span) bulk_load(st + kSmTile + span0, r->c_ptr + span0, span, &ctl->full[stage]);
                     if (slice) bulk_load(st + kSmTile + kTileValues, pay - skew, slice, &ctl->full[stage]);
                 } else {
                     mbar_arrive(&ctl->full[stage]);  // short tile: consumers read global memory themselves
                 }
-                atomicMax(&ctl->issued, k + 1u);
             }
             __syncwarp();
+            if (!FINE && !kStageOut && full_tile && ((uint32_t)kTileValues >> log2b) <= 32u) {
+                // lane i starts the copy of the i-th run of unchanged blocks (the bytes of all runs are
+                // already part of what lane 0 told the barrier to expect)
+                const uint32_t nbt_ = (uint32_t)kTileValues >> log2b;
+                const uint32_t zeros = ~r->bm[0] & (nbt_ == 32u ? 0xffffffffu : (1u << nbt_) - 1u);
+                const uint32_t starts = zeros & ~(zeros << 1);
+                if (lane < (uint32_t)__popc(starts)) {
+                    const uint32_t s0 = __fns(starts, 0u, (int)lane + 1);
+                    const uint32_t ones = ~(zeros >> s0);  // first set bit = the run's length (none: to bit 31)
+                    const uint32_t len = ones ? (uint32_t)__ffs(ones) - 1u : 32u - s0;
+                    bulk_load(st + kSmTile + (s0 << log2b), r->c_ptr + (s0 << log2b), len << log2b, &ctl->full[stage]);
+                }
+                __syncwarp();
+            }
+            if (lane == 0) atomicMax(&ctl->issued, k + 1u);
             t_cur = t_nxt;
             t_nxt = t_nn;
         }
