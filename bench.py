@@ -37,9 +37,11 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of one encode launch per value, from the ncu capture summarised in
 # profiles/ncu_full_one_layer_bf16.md: dram__bytes_read.sum + dram__bytes_write.sum of a one-layer
-# case (1.758 GB) divided by its 402 653 184 values; traffic grows in proportion to the values of
+# case (1.753 GB) divided by its 402 653 184 values; traffic grows in proportion to the values of
 # a launch, and every launch of the bench workload is one such layer.  bf16, B = 512, q = 0.22 only.
-NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE = 4.366
+# The same for the sender with HashCache (profiles/bench_hashed_encode_one_layer.md: 1.281 GB).
+NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE = 4.353
+NCU_HASHED_ENCODE_TRAFFIC_BYTES_PER_VALUE = 3.182
 
 
 def parse_args():
@@ -595,8 +597,10 @@ def main():
         "roofline": {
             "bound": "hbm", "kernel": ("encode_kernel" if args.detect == "compare" else "encode_kernel (HashCache form)"), "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
             "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBps": enc_gbs / NOMINAL_HBM_GBS,
-            "traffic": (NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE * n_layer
-                        if args.dtype == "bf16" and args.block == 512 and args.update == "clustered" else None),
+            "traffic": ((NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE if args.detect == "compare"
+                         else NCU_HASHED_ENCODE_TRAFFIC_BYTES_PER_VALUE) * n_layer
+                        if args.dtype == "bf16" and args.block == 512 and args.update == "clustered" and args.f == 0.22
+                        and args.shapes == "olmoe" else None),
             "algorithmic_bytes_per_launch": a_enc,
             "timed": "CUDA events around every encode launch, same K steps re-run on one stream so that "
                      "no other kernel overlaps it",
