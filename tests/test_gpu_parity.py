@@ -384,3 +384,21 @@ def test_tightly_packed_layout_in_shuffled_order(rt, dtype, block):
     traj = [wl.as_bits(w) for w in wl.trajectory(n, NAME[dtype], 90 + block, 2, "adam")]
     _run_trajectory(rt, codec, table, traj, dtype, label=f"tight-{NAME[dtype]}-B{block}")
     _run_trajectory(rt, codec, table, traj[:2], dtype, zero_cache=True, label=f"tight-zero-{NAME[dtype]}-B{block}")
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("block,rate", [(16, 0.9), (64, 0.9), (128, 0.95), (256, 0.5), (512, 0.5), (512, 0.06),
+                                        (4096, 0.5)])
+def test_scattered_unchanged_blocks(rt, dtype, block, rate):
+    """Whole blocks change at a given rate, the unchanged ones scattered between them: the receiver
+    fetches the cached exponents of unchanged blocks as a span, run by run, or piece by piece
+    depending on how many there are and how they lie."""
+    codec, table, n = _make(rt, [600_000, 131_072, 70_001], 2, dtype, block)
+    gen = wl.make_generator(4100 + block)
+    w0 = wl.init_weights(n, NAME[dtype], gen)
+    w1 = wl.inject_exponent_changes(w0, gen, rate, seg=block)
+    w2 = wl.inject_exponent_changes(w1, gen, rate, seg=block)
+    stats = _run_trajectory(rt, codec, table, [wl.as_bits(w) for w in (w0, w1, w2)], dtype,
+                            label=f"scattered-{NAME[dtype]}-B{block}-{rate}")
+    changed, blocks = stats[-1]
+    assert 0 < changed < blocks  # (segments are aligned in the buffer, not in every unit: the rate is only roughly `rate`)
