@@ -488,6 +488,23 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                 else
                     unchanged_span(r->bm, log2b, lane, lo, hi);
             }
+            // Coarse blocks (not fp32, whose output goes through bulk stores and which lost 6 % with it): the
+            // cached exponents of the unchanged blocks come run by run -- lane w looks at word w of the block
+            // flags and starts one bulk copy per run of unchanged blocks in it -- unless the runs are many
+            // (then the one span that covers them, or, where they are few and far apart, reads by the consumers).
+            bool by_runs = false;
+            uint32_t my_zeros = 0, unchanged_bytes = 0;
+            if (!FINE && !kStageOut && full_tile) {
+                const uint32_t nbt_ = (uint32_t)kTileValues >> log2b;
+                const uint32_t nwords = nbt_ >= 32u ? nbt_ >> 5 : 1u;
+                if (lane < nwords) my_zeros = ~r->bm[lane] & (nbt_ >= 32u ? 0xffffffffu : (1u << nbt_) - 1u);
+                const uint32_t nruns = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(my_zeros & ~(my_zeros << 1)));
+                const uint32_t unchanged = __reduce_add_sync(0xffffffffu, (uint32_t)__popc(my_zeros));
+                unchanged_bytes = unchanged << log2b;
+                const uint32_t span_bytes = lo <= hi ? (hi - lo + 1u) << log2b : 0u;
+                const bool sparse = span_bytes != 0 && 4u * unchanged_bytes <= span_bytes;  // consumers read them
+                by_runs = !sparse && nruns <= 32u && (!kHalf || nbt_ <= 32u);  // (fp16 with more than 32 blocks per tile: the span was faster)
+            }
 
             if (lane == 0) {
                 r->w_dst = weights + td.w_off;
@@ -517,13 +534,8 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                     // which holds at least the values up to the end of this full tile)
                     uint32_t span0 = lo << log2b, span = lo <= hi ? (hi - lo + 1u) << log2b : 0u;
                     uint32_t skew = 0, slice = (uint32_t)payload_bytes_of_blocks<DT>(own, log2b);
-                    // Up to 32 blocks per tile (256 values and more each): one copy per run of unchanged
-                    // blocks instead of the span, so that no cached exponents of changed blocks are read.
-                    const uint32_t nbt_ = (uint32_t)kTileValues >> log2b;
-                    const bool by_runs = !FINE && !kStageOut && nbt_ <= 32u;  // (fp32, whose output goes through bulk stores, lost 6 % with it)
                     if (by_runs) {
-                        const uint32_t zeros = ~r->bm[0] & (nbt_ == 32u ? 0xffffffffu : (1u << nbt_) - 1u);
-                        span = (uint32_t)__popc(zeros) << log2b;
+                        span = unchanged_bytes;  // no cached exponents of changed blocks are read
                         if (!kHalf) r->direct = 0u;
                     } else if (!FINE && !kHalf) {
                         // a few unchanged blocks scattered over a long span: staging the span would mostly
@@ -555,17 +567,16 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                 }
             }
             __syncwarp();
-            if (!FINE && !kStageOut && full_tile && ((uint32_t)kTileValues >> log2b) <= 32u) {
-                // lane i starts the copy of the i-th run of unchanged blocks (the bytes of all runs are
-                // already part of what lane 0 told the barrier to expect)
-                const uint32_t nbt_ = (uint32_t)kTileValues >> log2b;
-                const uint32_t zeros = ~r->bm[0] & (nbt_ == 32u ? 0xffffffffu : (1u << nbt_) - 1u);
-                const uint32_t starts = zeros & ~(zeros << 1);
-                if (lane < (uint32_t)__popc(starts)) {
-                    const uint32_t s0 = __fns(starts, 0u, (int)lane + 1);
+            if (by_runs) {
+                // (the bytes of all runs are already part of what lane 0 told the barrier to expect)
+                uint32_t zeros = my_zeros;
+                while (zeros) {
+                    const uint32_t s0 = (uint32_t)__ffs(zeros) - 1u;
                     const uint32_t ones = ~(zeros >> s0);  // first set bit = the run's length (none: to bit 31)
                     const uint32_t len = ones ? (uint32_t)__ffs(ones) - 1u : 32u - s0;
-                    bulk_load(st + kSmTile + (s0 << log2b), r->c_ptr + (s0 << log2b), len << log2b, &ctl->full[stage]);
+                    const uint32_t at = (32u * lane + s0) << log2b;
+                    bulk_load(st + kSmTile + at, r->c_ptr + at, len << log2b, &ctl->full[stage]);
+                    zeros &= ~((len == 32u ? 0xffffffffu : (1u << len) - 1u) << s0);
                 }
                 __syncwarp();
             }
