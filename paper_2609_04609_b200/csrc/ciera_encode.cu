@@ -40,6 +40,7 @@
 // the hashes, compares them with the cached ones, refreshes HashCache and derives the block flags
 // from the comparison.
 #include <cstddef>
+#include <type_traits>
 
 #include "ciera_bits.cuh"
 #include "ciera_hash.cuh"
@@ -773,88 +774,32 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
                 const uint8_t* const s_w = ring_w + (size_t)sw * kWBytes;
                 uint8_t* const s_e = ring_e + (size_t)se * kEBytes;
                 uint64_t hash_a[P::kPerThread], hash_b[P::kPerThread];  // HASH: the pieces' sums of terms
-#pragma unroll
-                for (int p = 0; p < P::kPerThread; ++p) {
-                    const uint32_t t0 = P::start(tid, p);
-                    const int nvalid = piece_valid<DT>(t0, nv);
-                    // (exp, mant) <- SplitExpMant, and the cached exponents of the same values
-                    P x, c;
-                    if (nv == (uint32_t)kTileValues) {
-                        x.template split_full<Shared>(s_w + (size_t)t0 * VB);
-                        if (!HASH) c.template load_exp_full<Shared>(s_e + t0);
-                    } else if (nvalid == P::kValues) {
-                        x.template split_full<Global>(ti.w_src + (size_t)t0 * VB);
-                        if (!HASH) c.template load_exp_full<Global>(ti.c_ptr + t0);
-                    } else {
-                        // values past the end of the unit read as exponent 0 against a cached 0: never "changed"
-                        x.split_partial(ti.w_src + (size_t)t0 * VB, nvalid);
-                        if (!HASH) c.load_exp_partial(ti.c_ptr + t0, nvalid);
-                    }
-                    // leave the new exponents where the cached ones were staged: they are sent from
-                    // there once the tile's place in the payload is known
-                    x.template store_exp_full<Shared>(s_e + t0);
-                    if constexpr (HASH) {
-                        // h <- Hash128(exp[k]), first part: the terms of this piece's 64-bit words (words
-                        // past the end of the unit do not exist)
-                        constexpr int kWords = P::kExpWords / 2;
-                        uint64_t ta[kWords], tb[kWords];
-                        const uint32_t j0 = (t0 & ((1u << log2b) - 1u)) >> 3;
-#pragma unroll
-                        for (int w = 0; w < kWords; ++w)
-                            hash_word_terms(j0 + (uint32_t)w, (uint64_t)x.e[2 * w] | ((uint64_t)x.e[2 * w + 1] << 32), ta[w], tb[w]);
-                        if (nvalid != P::kValues) {  // the unit's last pieces only
-#pragma unroll
-                            for (int w = 0; w < kWords; ++w)
-                                if (nvalid <= 8 * w) ta[w] = tb[w] = 0ull;
-                        }
-                        uint64_t a = ta[0], b = tb[0];
-#pragma unroll
-                        for (int w = 1; w < kWords; ++w) {
-                            a += ta[w];
-                            b += tb[w];
-                        }
-                        hash_a[p] = a;
-                        hash_b[p] = b;
-                    } else if constexpr (!FINE) {
-                        const uint32_t bal = __ballot_sync(0xffffffffu, x.differs(c));
-                        if (lane == 0) ctl->ballot[se][p * kWarps + warp] = bal;
-                    } else {
-                        // K = values-per-piece / B flags per piece; the warp's 32 pieces fill K whole
-                        // words of the tile's block flags, 32 / K lanes to a word
-                        const uint32_t k_l2 = (uint32_t)P::kLog2Values - log2b;  // log2 K, 0 .. 4
-                        const uint32_t flags = x.block_flags(c, log2b);
-                        uint32_t* const words = &ctl->bm[se][(p * kWarps + warp) << k_l2];
-                        if (k_l2 == 3) {  // a byte of flags per piece: every lane stores its own
-                            reinterpret_cast<uint8_t*>(words)[lane] = (uint8_t)flags;
-                        } else if (k_l2 == 4) {  // two bytes per piece
-                            reinterpret_cast<uint16_t*>(words)[lane] = (uint16_t)flags;
-                        } else if (k_l2 == 0) {  // one flag per piece: the vote is the word
-                            const uint32_t v = __ballot_sync(0xffffffffu, flags != 0);
-                            if (lane == 0) words[0] = v;
-                        } else {
-                            // two or four flags per piece: 4 or 2 neighbouring lanes fill a byte
-                            uint32_t v = flags << ((lane << k_l2) & 7u);
-                            v |= __shfl_xor_sync(0xffffffffu, v, 1);
-                            if (k_l2 == 1) v |= __shfl_xor_sync(0xffffffffu, v, 2);
-                            if ((lane & ((8u >> k_l2) - 1u)) == 0)
-                                reinterpret_cast<uint8_t*>(words)[lane >> (3u - k_l2)] = (uint8_t)v;
-                        }
-                    }
-                    // sign-plus-mantissa of every value
-                    if constexpr (DT == CIERA_FP16) {
-                        // packed: whole groups of four lanes in a full tile (every lane takes part in the
-                        // group's shuffle), else byte by byte
-                        if (nv == (uint32_t)kTileValues)
-                            x.store_sm_group(ti.sm_dst, t0 >> 3, lane);
-                        else if (nvalid > 0)
-                            x.store_sm_bytes(ti.sm_dst + (size_t)11 * (t0 >> 3), nvalid);
-                    } else {
-                        uint8_t* smdst = ti.sm_dst + (size_t)t0 * SMB;
-                        if (nvalid == P::kValues)
-                            x.template store_sm_full<Global>(smdst);
-                        else if (nvalid > 0)
-                            x.store_sm_partial(smdst, nvalid);
-                    }
+                // The pieces of this thread.  Most instances compile the loop twice: for full tiles (staged
+                // in shared memory, every piece complete, no tests on the way) and for a unit's last, short
+                // tile; that measured 2-12 % faster (fp16 most).  Two instances keep one loop that tests as it
+                // goes, which measured faster for them: bf16 with coarse blocks and the exponent cache (1 %),
+                // fp32 with HashCache (5 %).
+                constexpr bool kOneBody = (DT == CIERA_BF16 && !FINE && HASH == 0) || (DT == CIERA_FP32 && HASH != 0);
+                if constexpr (kOneBody) {
+                    // a plain loop that tests as it goes
+#define CIERA_PIECES_FULL false
+#define CIERA_PIECES_STAGED (nv == (uint32_t)kTileValues)
+#include "ciera_encode_pieces.inc"
+#undef CIERA_PIECES_FULL
+#undef CIERA_PIECES_STAGED
+                } else {
+                    auto pieces = [&](auto full_tag) {
+                        constexpr bool kFull = decltype(full_tag)::value;
+#define CIERA_PIECES_FULL kFull
+#define CIERA_PIECES_STAGED kFull
+#include "ciera_encode_pieces.inc"
+#undef CIERA_PIECES_FULL
+#undef CIERA_PIECES_STAGED
+                    };
+                    if (nv == (uint32_t)kTileValues)
+                        pieces(std::true_type{});
+                    else
+                        pieces(std::false_type{});
                 }
                 if constexpr (HASH) {
                     uint64_t* const part = reinterpret_cast<uint64_t*>(ring_h + (size_t)se * kHStage + kHoldBytes);
