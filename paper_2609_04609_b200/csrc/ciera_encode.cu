@@ -436,14 +436,15 @@ __device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t 
 // Every consumer thread sends the exponents of its own pieces (left in the stage's shared-memory
 // tile) if their block changed; `base` is the tile's exclusive offset in the unit's payload.
 // (CACHE = false, the sender with HashCache: payload only.)
-template <int DT, bool CACHE>
+// (FULL: the tile is a full one, every piece complete.)
+template <int DT, bool CACHE, bool FULL>
 __device__ __forceinline__ void write_changed(const EncodeTileInfo& ti, uint32_t log2b, const uint32_t* bm,
                                               const uint16_t* pre, uint64_t base, const uint8_t* s_exp, uint32_t tid) {
     using P = Piece<DT>;
 #pragma unroll
     for (int p = 0; p < P::kPerThread; ++p) {
         const uint32_t t0 = P::start(tid, p);
-        const int nvalid = piece_valid<DT>(t0, ti.nv);
+        const int nvalid = FULL ? (int)P::kValues : piece_valid<DT>(t0, ti.nv);
         if (nvalid == 0) continue;
         const uint32_t kb = t0 >> log2b;
         const uint32_t word = bm[kb >> 5];
@@ -542,7 +543,12 @@ template <int DT, bool FINE, int HASH>
 __device__ __forceinline__ void send_changed(const EncodeTileInfo& ti, uint32_t log2b, const uint32_t* bm,
                                              const uint16_t* pre, uint64_t base, const uint8_t* s_exp, uint32_t tid) {
     if (!FINE) {
-        write_changed<DT, HASH == 0>(ti, log2b, bm, pre, base, s_exp, tid);
+        // (as in the consumers' main loop: the two instances named there keep the one form that tests as it goes)
+        constexpr bool kOneBody = (DT == CIERA_BF16 && HASH == 0) || (DT == CIERA_FP32 && HASH != 0);
+        if (!kOneBody && ti.nv == (uint32_t)kTileValues)
+            write_changed<DT, HASH == 0, true>(ti, log2b, bm, pre, base, s_exp, tid);
+        else
+            write_changed<DT, HASH == 0, false>(ti, log2b, bm, pre, base, s_exp, tid);
     } else {
         switch (log2b) {
             case 0: write_changed_fine<0>(ti, bm, pre, base, s_exp, tid); break;
