@@ -106,6 +106,15 @@ def test_plan_tile_table(ciera):
             assert t["m"] == u["msg_off"]
             k += 1
     assert k == want_tiles
+    # HashCache: 16 bytes per block, units in table order; the image ends with the index of every tile's first
+    # block (8 bytes per tile, in tile-table order, then 16 spare bytes)
+    nblocks = [-(-n // 64) for n in sizes]
+    assert p.hash_cache_bytes == 16 * sum(nblocks)
+    base = np.concatenate([[0], np.cumsum(nblocks)])
+    assert [ciera.unit_hash_offset(p, u) for u in range(len(sizes))] == [16 * int(b) for b in base[:-1]]
+    assert p.hashed_workspace_bytes == p.workspace_bytes
+    tail = p.host_image()[-(8 * want_tiles + 16):-16].view("<u8")
+    assert [int(x) for x in tail] == [int(base[t["unit"]]) + int(t["j"]) * (T // 64) for t in img]
     # an empty table is legal
     e = ciera.Plan(np.zeros(0, UNIT_DTYPE), 0, 512)
     assert (e.n_units, e.n_tiles) == (0, 0)
