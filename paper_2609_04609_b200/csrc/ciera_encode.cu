@@ -275,6 +275,7 @@ __device__ __forceinline__ uint32_t scan_block_bitmap_w(const uint32_t* bm, uint
 }
 __device__ __forceinline__ uint32_t scan_block_bitmap(const uint32_t* bm, uint16_t* pre, uint32_t log2b, uint32_t lane) {
     if (log2b == 0) return scan_block_bitmap_w<8>(bm, pre, lane);  // 256 words: eight per lane, one scan
+    if (log2b == 1) return scan_block_bitmap_w<4>(bm, pre, lane);  // 128 words: four per lane
     const uint32_t nwords = kTileValues >> (log2b + 5);  // 32 .. 128: a scan per 32 words
     uint32_t run = 0;
     for (uint32_t base = 0; base < nwords; base += 32) {
