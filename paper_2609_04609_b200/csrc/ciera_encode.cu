@@ -309,23 +309,37 @@ __device__ __forceinline__ uint32_t hash_block_bitmap(const ulonglong2* part, co
     const uint32_t nbt = kTileValues >> log2b;
     const uint32_t nblk = (nv + B - 1u) >> log2b;
     const uint32_t epb_l2 = log2b > kGroupL2 ? log2b - kGroupL2 : 0u;  // log2(partial sums per block)
-    uint32_t run = 0;
-    for (uint32_t base = 0; base < nbt; base += 32) {
-        const uint32_t i = base + lane;
-        bool f = false;
-        if (i < nblk) {
-            uint64_t a = 0, b = 0;
-            for (uint32_t e = 0; e < (1u << epb_l2); ++e) {
-                const ulonglong2 v = part[(i << epb_l2) + e];
-                a += v.x;
-                b += v.y;
-            }
-            const ulonglong2 h = hash_finish(a, b, min(B, nv - (i << log2b)));
-            const ulonglong2 old = hold[i];
-            f = h.x != old.x || h.y != old.y;
-            if (f) hash_dst[i] = h;
+    // one block: true iff its hashes differ from the cached pair (which is then replaced)
+    auto finish_block = [&](uint32_t i) -> bool {
+        if (i >= nblk) return false;
+        uint64_t a = 0, b = 0;
+        for (uint32_t e = 0; e < (1u << epb_l2); ++e) {
+            const ulonglong2 v = part[(i << epb_l2) + e];
+            a += v.x;
+            b += v.y;
         }
-        const uint32_t word = __ballot_sync(0xffffffffu, f);
+        const ulonglong2 h = hash_finish(a, b, min(B, nv - (i << log2b)));
+        const ulonglong2 old = hold[i];
+        const bool f = h.x != old.x || h.y != old.y;
+        if (f) hash_dst[i] = h;
+        return f;
+    };
+    uint32_t run = 0;
+    uint32_t base = 0;
+    // two blocks per lane and round while there are 64 and more (their chains of multiplies overlap; four were slower)
+    for (; base + 64 <= nbt; base += 64) {
+        const bool f0 = finish_block(base + lane), f1 = finish_block(base + 32 + lane);
+        const uint32_t w0 = __ballot_sync(0xffffffffu, f0), w1 = __ballot_sync(0xffffffffu, f1);
+        if (lane == 0) {
+            bm[base >> 5] = w0;
+            pre[base >> 5] = (uint16_t)run;
+            bm[(base >> 5) + 1] = w1;
+            pre[(base >> 5) + 1] = (uint16_t)(run + __popc(w0));
+        }
+        run += __popc(w0) + __popc(w1);
+    }
+    for (; base < nbt; base += 32) {
+        const uint32_t word = __ballot_sync(0xffffffffu, finish_block(base + lane));
         if (lane == 0) {
             bm[base >> 5] = word;
             pre[base >> 5] = (uint16_t)run;
