@@ -5,10 +5,13 @@
 // the blocks (block c takes tiles T0 + c, T0 + c + G, ...; neighbouring tiles of a unit are then
 // worked on by neighbouring blocks at about the same time, and their payload offsets come from a
 // single-pass look-back over per-tile status words; this part needs all blocks resident, so a
-// plan with longer units is launched cooperatively).  Then it works through whole short units,
-// tile after tile, drawing the next unit's number from a counter in the scratch: a tile's place in
-// its unit's payload is then a running sum inside the block, nothing waits for another block, and
-// all SMs stay busy to the end whatever their individual pace.
+// plan with longer units is launched cooperatively).  Then it works through the short units in runs
+// of four tiles, drawing the next run's number from a counter in the scratch (every unit's first run
+// goes out before any unit's second run, and so on): a tile's place in its unit's payload is then a
+// running sum inside the block, which a run that does not start its unit takes over from the status
+// word of the tile before it -- written many draws earlier -- and all SMs stay busy to the end
+// whatever their individual pace (with whole units of 16 tiles as the piece of work drawn, the blocks
+// finished up to a unit apart: 0.921 of the copy peak against 0.935).
 // A thread block has four roles:
 //
 //   producer warp   runs ahead of the others: for each of its tiles it fetches the tile
@@ -181,7 +184,7 @@ struct EncodeCtl {
     TileDesc desc[kDescRing];
     EncodeTileInfo info[kDescRing];
     uint32_t tile_idx[kDescRing];  // table index of the tile in desc[]; kNoTile = end marker
-    uint32_t seq[kDescRing];       // 1: tile of a unit this block works through alone
+    uint32_t seq[kDescRing];       // kSeq* bits: tile of a run that this block works through alone, first / last of the run
     uint32_t ballot[SE][kVoteWords];  // coarse blocks: "my piece differs" votes
     uint32_t bm[SE][BW];              // block flags of the tile (16-byte aligned: checked where the kernel starts)
     uint16_t pre[SE][BW];             // set flags before each word of bm
@@ -194,40 +197,49 @@ struct EncodeCtl {
 
 constexpr uint32_t kNoTile = 0xffffffffu;
 
+// How a tile relates to the run of tiles it was handed out with (a short unit's tiles go out in runs of
+// kSeqRunTiles, see ciera_internal.cuh): bit 0 = the tile belongs to a run (else: a spread tile of a longer
+// unit), bit 1 = first tile of its run, bit 2 = last tile of its run.
+constexpr uint32_t kSeqTile = 1u, kSeqRunStart = 2u, kSeqRunEnd = 4u;
+
 // The sequence of tiles of one thread block (see the head of this file); used by the producer.
 struct TileWalk {
-    const uint32_t* seq_first;
-    unsigned int* unit_ticket;
-    uint32_t n_tiles, n_short, G;
-    uint32_t tile, end;      // current short unit: next tile, one past its last tile
-    uint32_t next_unit;      // the unit drawn ahead (its number arrives while the current one is worked on)
+    const uint2* seq_runs;
+    unsigned int* run_ticket;
+    uint32_t n_tiles, n_runs, G;
+    uint32_t tile, end;      // current run: next tile, one past its last tile
+    uint32_t next_run;       // the run drawn ahead (its number arrives while the current one is worked on)
     uint32_t spread_tile;    // next spread tile of this block
     bool spread;
 
-    __device__ TileWalk(const uint32_t* sf, unsigned int* ticket, uint32_t nshort, uint32_t nt, uint32_t grid, uint32_t block)
-        : seq_first(sf), unit_ticket(ticket), n_tiles(nt), n_short(nshort), G(grid), tile(0), end(0), spread(true) {
-        spread_tile = __ldg(sf + nshort) + block;  // tiles of longer units start after the short units' tiles
-        next_unit = nshort ? atomicAdd(ticket, 1u) : kNoTile;
+    __device__ TileWalk(const uint2* runs, unsigned int* ticket, uint32_t nruns, uint32_t spread_first, uint32_t nt,
+                        uint32_t grid, uint32_t block)
+        : seq_runs(runs), run_ticket(ticket), n_tiles(nt), n_runs(nruns), G(grid), tile(0), end(0), spread(true) {
+        spread_tile = spread_first + block;  // tiles of longer units start after the short units' tiles
+        next_run = nruns ? atomicAdd(ticket, 1u) : kNoTile;
     }
-    // next tile, or kNoTile; `seq` tells whether it belongs to a unit the block works through alone
-    __device__ uint32_t next(bool& seq) {
+    // next tile, or kNoTile; `seq` gets the kSeq* bits of the tile
+    __device__ uint32_t next(uint32_t& seq) {
         if (spread) {
             if (spread_tile < n_tiles) {
-                seq = false;
+                seq = 0;
                 const uint32_t t = spread_tile;
                 spread_tile += G;
                 return t;
             }
             spread = false;
         }
-        seq = true;
+        seq = kSeqTile;
         while (tile == end) {
-            const uint32_t u = next_unit;
-            if (u >= n_short) return kNoTile;
-            next_unit = atomicAdd(unit_ticket, 1u);
-            tile = __ldg(seq_first + u);
-            end = __ldg(seq_first + u + 1);
+            const uint32_t r = next_run;
+            if (r >= n_runs) return kNoTile;
+            next_run = atomicAdd(run_ticket, 1u);
+            const uint2 run = __ldg(seq_runs + r);
+            tile = run.x;
+            end = run.y;
+            seq |= kSeqRunStart;
         }
+        if (tile + 1u == end) seq |= kSeqRunEnd;
         return tile++;
     }
 };
@@ -578,8 +590,8 @@ __device__ __forceinline__ void send_changed(const EncodeTileInfo& ti, uint32_t 
 // the index of every tile's first block in it.
 template <int DT, bool FINE, int HASH>
 __global__ void __launch_bounds__(kEncodeThreads, 2)
-encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32_t* __restrict__ seq_first,
-              uint32_t n_short, uint32_t log2b, const uint8_t* __restrict__ weights, uint8_t* cache, uint8_t* msgs,
+encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint2* __restrict__ seq_runs, uint32_t n_runs,
+              uint32_t spread_first, uint32_t log2b, const uint8_t* __restrict__ weights, uint8_t* cache, uint8_t* msgs,
               unsigned long long* wire_bytes, uint32_t* changed_blocks, unsigned long long* tile_status,
               unsigned int* unit_ticket, int32_t* status, const unsigned long long* __restrict__ tile_hash) {
     static_assert(!(HASH && (FINE || DT == CIERA_FP16)), "HashCache: bf16 and fp32, blocks of 16 values and more");
@@ -633,8 +645,8 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
     if (warp == kProducerWarp) {
         // ---------------------------------------------------------------- producer
         if (lane == 0) {
-            TileWalk walk(seq_first, unit_ticket, n_short, n_tiles, gridDim.x, blockIdx.x);
-            bool seq_nxt = false;
+            TileWalk walk(seq_runs, unit_ticket, n_runs, spread_first, n_tiles, gridDim.x, blockIdx.x);
+            uint32_t seq_nxt = 0;
             uint32_t tile_nxt = walk.next(seq_nxt);
             TileDesc nxt;
             unsigned long long hb_nxt = 0;  // HASH: index of the tile's first block in HashCache
@@ -646,7 +658,7 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
             for (uint32_t k = 0;; ++k) {
                 const TileDesc td = nxt;
                 const uint32_t tile = tile_nxt;
-                const bool seq = seq_nxt;
+                const uint32_t seq = seq_nxt;
                 const unsigned long long hb = hb_nxt;
                 if (tile != kNoTile) {
                     tile_nxt = walk.next(seq_nxt);
@@ -666,7 +678,7 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
                     continue;
                 }
                 ctl->desc[k % kDescRing] = td;
-                ctl->seq[k % kDescRing] = seq ? 1u : 0u;
+                ctl->seq[k % kDescRing] = seq;
                 const uint64_t v0 = (uint64_t)td.tile_in_unit * kTileValues;
                 const uint64_t left = td.n_unit - v0;
                 {
@@ -718,7 +730,8 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
                 continue;
             }
             const TileDesc td = ctl->desc[k % kDescRing];
-            const bool seq = ctl->seq[k % kDescRing] != 0;
+            const uint32_t seq_bits = ctl->seq[k % kDescRing];
+            const bool seq = seq_bits != 0;
             HashTile ht{nullptr, nullptr, nullptr};
             if constexpr (HASH) {
                 // the cached hashes were staged by a bulk copy that completes on full_e: observe it here too
@@ -730,9 +743,18 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint32
             const uint64_t agg = aggregate_tile<DT, FINE, HASH>(td, tile, log2b, !seq, ctl->ballot[se], ctl->bm[se],
                                                                 ctl->pre[se], msgs, tile_status, ht, lane);
             if (seq) {
-                // the whole unit is this block's: the tile's offset is the running sum
-                const uint64_t excl = td.tile_in_unit == 0 ? 0ull : run_incl;
+                // the run is this block's: the tile's offset is the running sum; a run that does not start its
+                // unit carries on from the inclusive offset that the run before it left in its last tile's
+                // status word (that run went out many draws earlier; the wait is bounded all the same; reading
+                // the word in the producer thread instead, tiles ahead, was slower)
+                uint64_t excl = run_incl;
+                if (td.tile_in_unit == 0)
+                    excl = 0;
+                else if (seq_bits & kSeqRunStart)
+                    excl = wait_status(tile_status + tile - 1, status) & kValueMask;
                 run_incl = excl + agg;
+                if ((seq_bits & kSeqRunEnd) && td.tile_in_unit != td.n_tiles_unit - 1u && lane == 0)
+                    st_status(tile_status + tile, kFlagPrefix | run_incl);
                 const uint32_t nbt = kTileValues >> log2b;
                 const bool last = td.tile_in_unit == td.n_tiles_unit - 1u;
                 if (nbt < 8) {
@@ -932,8 +954,9 @@ static int launch_encode(const ciera_plan* p, const void* weights_dev, void* sen
     const TileDesc* tiles = p->tiles_dev;
     uint32_t nt = (uint32_t)p->tiles.size();
     const uint32_t grid = nt < (uint32_t)limit ? nt : (uint32_t)limit;
-    const uint32_t* seq_first = p->seq_first_dev;
-    uint32_t n_short = (uint32_t)p->seq_first.size() - 1u;
+    const uint2* seq_runs = p->seq_runs_dev;
+    uint32_t n_runs = (uint32_t)p->seq_runs.size();
+    uint32_t spread_first = p->seq_first.back();
     uint32_t log2b = p->log2b;
     const uint8_t* w = (const uint8_t*)weights_dev;
     uint8_t* c = (uint8_t*)sender_cache_dev;
@@ -948,13 +971,13 @@ static int launch_encode(const ciera_plan* p, const void* weights_dev, void* sen
     if (has_spread) {
         // cooperative launch: the runtime starts the grid only when all of its blocks fit on the
         // GPU together, which is what the look-back between blocks relies on
-        void* args[] = {&tiles, &nt, &seq_first, &n_short, &log2b, &w, &c, &m, &wb, &changed_blocks_dev, &ts, &ticket,
-                        &status_dev, &tile_hash};
+        void* args[] = {&tiles, &nt, &seq_runs, &n_runs, &spread_first, &log2b, &w, &c, &m, &wb, &changed_blocks_dev, &ts,
+                        &ticket, &status_dev, &tile_hash};
         e = cudaLaunchCooperativeKernel((const void*)encode_kernel<DT, FINE, HASH>, dim3(grid), dim3(kEncodeThreads), args,
                                         smem, s);
     } else {
         encode_kernel<DT, FINE, HASH><<<grid, kEncodeThreads, smem, s>>>(
-            tiles, nt, seq_first, n_short, log2b, w, c, m, wb, changed_blocks_dev, ts, ticket, status_dev, tile_hash);
+            tiles, nt, seq_runs, n_runs, spread_first, log2b, w, c, m, wb, changed_blocks_dev, ts, ticket, status_dev, tile_hash);
         e = cudaGetLastError();
     }
     if (e != cudaSuccess) return record_cuda_error(e);

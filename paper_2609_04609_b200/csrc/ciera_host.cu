@@ -68,7 +68,7 @@ extern "C" size_t ciera_message_bytes(uint64_t n, int dtype, uint32_t block, uin
 
 namespace {
 struct ImageLayout {
-    size_t tiles, long_off, seq_off, hash_off, first_off, seg_off, units_off, elong_off, echunk_off, thash_off, total;
+    size_t tiles, long_off, seq_off, hash_off, first_off, seg_off, units_off, elong_off, echunk_off, thash_off, runs_off, total;
 };
 size_t up16(size_t x) { return (x + 15) / 16 * 16; }
 ImageLayout image_layout(const ciera_plan* p) {
@@ -83,7 +83,8 @@ ImageLayout image_layout(const ciera_plan* p) {
     L.elong_off = L.units_off + up16((size_t)p->n_units * sizeof(ciera_unit));
     L.echunk_off = L.elong_off + up16(p->ent_long_units.size() * sizeof(uint32_t));
     L.thash_off = L.echunk_off + up16(p->ent_chunks.size() * sizeof(ciera_plan::EntChunk));
-    L.total = L.thash_off + p->tiles.size() * sizeof(uint64_t) + 16;
+    L.runs_off = L.thash_off + up16(p->tiles.size() * sizeof(uint64_t));
+    L.total = L.runs_off + p->seq_runs.size() * sizeof(ciera_plan::SeqRun) + 16;
     return L;
 }
 }  // namespace
@@ -154,6 +155,14 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
         emit(u);
     }
     p->seq_first.push_back((uint32_t)p->tiles.size());
+    // the short units' runs of kSeqRunTiles tiles: every unit's first run, then every unit's second run, ...
+    for (uint32_t pass = 0; pass * kSeqRunTiles < kSeqMaxTiles; ++pass) {
+        for (size_t i = 0; i + 1 < p->seq_first.size(); ++i) {
+            const uint32_t first = p->seq_first[i], end = p->seq_first[i + 1];
+            const uint32_t lo = first + pass * kSeqRunTiles;
+            if (lo < end) p->seq_runs.push_back({lo, std::min(lo + kSeqRunTiles, end)});
+        }
+    }
     for (uint32_t u : longs) emit(u);
     // per unit, in table order: where its tiles start and where its blocks start in a hash cache
     p->unit_first.assign(n_units, 0xffffffffu);
@@ -185,6 +194,8 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
     if (!p->long_units.empty()) memcpy(p->image.data() + L.long_off, p->long_units.data(), p->long_units.size() * 4);
     memcpy(p->image.data() + L.seq_off, p->seq_first.data(), p->seq_first.size() * 4);
     if (!p->tile_hash.empty()) memcpy(p->image.data() + L.thash_off, p->tile_hash.data(), p->tile_hash.size() * 8);
+    if (!p->seq_runs.empty())
+        memcpy(p->image.data() + L.runs_off, p->seq_runs.data(), p->seq_runs.size() * sizeof(ciera_plan::SeqRun));
     if (n_units) {
         memcpy(p->image.data() + L.hash_off, p->hash_base.data(), (size_t)n_units * 8);
         memcpy(p->image.data() + L.first_off, p->unit_first.data(), (size_t)n_units * 4);
@@ -247,6 +258,7 @@ extern "C" int ciera_plan_bind(ciera_plan* p, void* plan_dev, size_t plan_dev_by
     p->ent_long_units_dev = (const uint32_t*)(base + L.elong_off);
     p->ent_chunks_dev = (const uint4*)(base + L.echunk_off);
     p->tile_hash_dev = (const unsigned long long*)(base + L.thash_off);
+    p->seq_runs_dev = (const uint2*)(base + L.runs_off);
     return CIERA_OK;
 }
 

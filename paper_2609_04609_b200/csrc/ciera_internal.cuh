@@ -113,6 +113,11 @@ constexpr uint32_t kDecodeDirectBlocks = 4096;
 // a short unit tile after tile (the tile's place in the payload is then a running sum inside the
 // block) and spreads everything else tile by tile over all blocks.
 constexpr uint32_t kSeqMaxTiles = 32;
+// A short unit is handed out in runs of this many tiles (all units' first runs, then all second runs, ...): the
+// smaller the piece of work a thread block draws, the less the blocks differ in when they finish.  A run's first
+// tile takes its payload offset from the status word that the run before it left.  A multiple of 4, so that tiles
+// sharing a bitmap byte (blocks of 2048 and 4096 values) stay in one run.
+constexpr uint32_t kSeqRunTiles = 4;
 
 // Bytes of a message slot that tile j of a unit moves in the transport kernel: [j * chunk,
 // (j + 1) * chunk); the unit's last tile also moves whatever lies beyond (pads and, for coarse
@@ -137,6 +142,10 @@ struct ciera_plan {
     std::vector<ciera::TileDesc> tiles;
     std::vector<uint32_t> long_units;  // first tile of every unit whose decode needs the prefix kernel
     std::vector<uint32_t> seq_first;   // first tile of every short unit, in table order, + end marker
+    struct SeqRun {
+        uint32_t lo, hi;               // tiles [lo, hi) of the table
+    };
+    std::vector<SeqRun> seq_runs;      // the short units' runs of tiles in the order they are handed out
     std::vector<uint32_t> unit_first;  // first tile of every unit (0xffffffff: a unit without values)
     std::vector<uint64_t> hash_base;   // index of every unit's first block in a per-block hash cache
     std::vector<uint64_t> tile_hash;   // the same for every tile's first block, in tile-table order
@@ -154,10 +163,11 @@ struct ciera_plan {
     const uint32_t* ent_long_units_dev = nullptr;
     const uint4* ent_chunks_dev = nullptr;
     std::vector<uint8_t> image;        // device image: tiles, long_units, seq_first, hash_base, unit_first, seg_base, units,
-                                       // ent_long_units, ent_chunks, tile_hash
+                                       // ent_long_units, ent_chunks, tile_hash, seq_runs
     const ciera::TileDesc* tiles_dev = nullptr;
     const uint32_t* long_units_dev = nullptr;
     const uint32_t* seq_first_dev = nullptr;
+    const uint2* seq_runs_dev = nullptr;
     const unsigned long long* hash_base_dev = nullptr;
     const unsigned long long* tile_hash_dev = nullptr;
     const uint32_t* unit_first_dev = nullptr;

@@ -107,13 +107,27 @@ def test_plan_tile_table(ciera):
             k += 1
     assert k == want_tiles
     # HashCache: 16 bytes per block, units in table order; the image ends with the index of every tile's first
-    # block (8 bytes per tile, in tile-table order, then 16 spare bytes)
+    # block (8 bytes per tile, in tile-table order, padded to 16 bytes), the runs of tiles in which the short units
+    # are handed out (pairs of 32-bit tile numbers) and 16 spare bytes
     nblocks = [-(-n // 64) for n in sizes]
     assert p.hash_cache_bytes == 16 * sum(nblocks)
     base = np.concatenate([[0], np.cumsum(nblocks)])
     assert [ciera.unit_hash_offset(p, u) for u in range(len(sizes))] == [16 * int(b) for b in base[:-1]]
     assert p.hashed_workspace_bytes == p.workspace_bytes
-    tail = p.host_image()[-(8 * want_tiles + 16):-16].view("<u8")
+    RUN = 4  # tiles per run
+    runs = []
+    for pas in range(32 // RUN):
+        k0 = 0
+        for ui in short:
+            lo = k0 + pas * RUN
+            if lo < k0 + ntiles[ui]:
+                runs.append((lo, min(lo + RUN, k0 + ntiles[ui])))
+            k0 += ntiles[ui]
+    image = p.host_image()
+    got_runs = image[-(8 * len(runs) + 16):-16].view("<u4").reshape(-1, 2)
+    assert [tuple(int(x) for x in r) for r in got_runs] == runs
+    thash_bytes = (8 * want_tiles + 15) // 16 * 16
+    tail = image[-(8 * len(runs) + 16 + thash_bytes):-(8 * len(runs) + 16)][: 8 * want_tiles].view("<u8")
     assert [int(x) for x in tail] == [int(base[t["unit"]]) + int(t["j"]) * (T // 64) for t in img]
     # an empty table is legal
     e = ciera.Plan(np.zeros(0, UNIT_DTYPE), 0, 512)
