@@ -156,11 +156,15 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
     }
     p->seq_first.push_back((uint32_t)p->tiles.size());
     // the short units' runs of kSeqRunTiles tiles: every unit's first run, then every unit's second run, ...
-    for (uint32_t pass = 0; pass * kSeqRunTiles < kSeqMaxTiles; ++pass) {
+    // (With 16 to 128 values per block a tile has 64 to 512 blocks and the aggregator warp, which also waits
+    // for the status word at the start of a run, has the least time to spare: there whole units measured 2-3 %
+    // faster than runs, so a run is the whole unit.)
+    const uint32_t run_tiles = (p->log2b >= 4 && p->log2b <= 7) ? kSeqMaxTiles : kSeqRunTiles;
+    for (uint32_t pass = 0; pass * run_tiles < kSeqMaxTiles; ++pass) {
         for (size_t i = 0; i + 1 < p->seq_first.size(); ++i) {
             const uint32_t first = p->seq_first[i], end = p->seq_first[i + 1];
-            const uint32_t lo = first + pass * kSeqRunTiles;
-            if (lo < end) p->seq_runs.push_back({lo, std::min(lo + kSeqRunTiles, end)});
+            const uint32_t lo = first + pass * run_tiles;
+            if (lo < end) p->seq_runs.push_back({lo, std::min(lo + run_tiles, end)});
         }
     }
     for (uint32_t u : longs) emit(u);

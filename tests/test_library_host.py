@@ -114,18 +114,26 @@ def test_plan_tile_table(ciera):
     base = np.concatenate([[0], np.cumsum(nblocks)])
     assert [ciera.unit_hash_offset(p, u) for u in range(len(sizes))] == [16 * int(b) for b in base[:-1]]
     assert p.hashed_workspace_bytes == p.workspace_bytes
-    RUN = 4  # tiles per run
-    runs = []
-    for pas in range(32 // RUN):
-        k0 = 0
-        for ui in short:
-            lo = k0 + pas * RUN
-            if lo < k0 + ntiles[ui]:
-                runs.append((lo, min(lo + RUN, k0 + ntiles[ui])))
-            k0 += ntiles[ui]
+    def runs_of(run_tiles):
+        out = []
+        for pas in range(32 // run_tiles):
+            k0 = 0
+            for ui in short:
+                lo = k0 + pas * run_tiles
+                if lo < k0 + ntiles[ui]:
+                    out.append((lo, min(lo + run_tiles, k0 + ntiles[ui])))
+                k0 += ntiles[ui]
+        return out
+
+    # tiles per run: whole units with 16 to 128 values per block (this plan: 64), else 4 (checked on a second plan)
+    runs = runs_of(32)
     image = p.host_image()
     got_runs = image[-(8 * len(runs) + 16):-16].view("<u4").reshape(-1, 2)
     assert [tuple(int(x) for x in r) for r in got_runs] == runs
+    units512, _, _, _ = layout_units(sizes, 1, 4, lambda n: ciera.message_capacity(n, 1, 512))
+    runs4 = runs_of(4)
+    got4 = ciera.Plan(units512, 1, 512).host_image()[-(8 * len(runs4) + 16):-16].view("<u4").reshape(-1, 2)
+    assert [tuple(int(x) for x in r) for r in got4] == runs4
     thash_bytes = (8 * want_tiles + 15) // 16 * 16
     tail = image[-(8 * len(runs) + 16 + thash_bytes):-(8 * len(runs) + 16)][: 8 * want_tiles].view("<u8")
     assert [int(x) for x in tail] == [int(base[t["unit"]]) + int(t["j"]) * (T // 64) for t in img]
