@@ -37,10 +37,10 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of one encode launch per value, from the ncu capture summarised in
 # profiles/ncu_full_one_layer_bf16.md: dram__bytes_read.sum + dram__bytes_write.sum of a one-layer
-# case (1.753 GB) divided by its 402 653 184 values; traffic grows in proportion to the values of
+# case (1.755 GB) divided by its 402 653 184 values; traffic grows in proportion to the values of
 # a launch, and every launch of the bench workload is one such layer.  bf16, B = 512, q = 0.22 only.
 # The same for the sender with HashCache (profiles/bench_hashed_encode_one_layer.md: 1.281 GB).
-NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE = 4.353
+NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE = 4.359
 NCU_HASHED_ENCODE_TRAFFIC_BYTES_PER_VALUE = 3.182
 
 
