@@ -35,13 +35,35 @@ METRIC = "encode/decode GB/s of weights"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic of one encode launch per value, from the ncu capture summarised in
-# profiles/ncu_full_one_layer_bf16.md: dram__bytes_read.sum + dram__bytes_write.sum of a one-layer
-# case (1.755 GB) divided by its 402 653 184 values; traffic grows in proportion to the values of
-# a launch, and every launch of the bench workload is one such layer.  bf16, B = 512, q = 0.22 only.
-# The same for the sender with HashCache (profiles/bench_hashed_encode_one_layer.md: 1.281 GB).
-NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE = 4.359
-NCU_HASHED_ENCODE_TRAFFIC_BYTES_PER_VALUE = 3.182
+# Measured DRAM traffic per value of the headline encode launch (dram__bytes_read.sum + dram__bytes_write.sum of
+# one ncu capture, divided by the values of the launch; traffic grows in proportion to the values).  The figure
+# lives in a small data file beside the ncu summaries, together with a digest of the kernel sources it was
+# captured with; when the sources have changed since, the bench line says traffic: null and why.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_dram_traffic.json")
+CSRC_DIR = os.path.join(ROOT, "paper_2609_04609_b200", "csrc")
+
+
+def csrc_digest() -> str:
+    """sha256 over the kernel sources (names and contents, sorted by name)."""
+    import hashlib
+
+    h = hashlib.sha256()
+    for name in sorted(os.listdir(CSRC_DIR)):
+        h.update(name.encode())
+        with open(os.path.join(CSRC_DIR, name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def measured_traffic(key: str, n_values: int):
+    """(bytes per launch or None, note) for the capture stored under `key`."""
+    try:
+        entry = json.load(open(TRAFFIC_FILE))[key]
+    except Exception:
+        return None, "no ncu capture on record for this workload"
+    if entry.get("csrc_sha256") != csrc_digest():
+        return None, "kernel sources changed since the ncu capture on record; re-capture to fill this in"
+    return float(entry["dram_bytes_per_value"]) * n_values, f"ncu capture on record ({entry.get('captured', '')})"
 
 
 def parse_args():
@@ -72,6 +94,9 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-regimes", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the one-layer runs of the other configurations (config 2 worst case, fp32, mixed shapes, "
+                         "small blocks, fp16, hashed sender, entropy stage)")
     ap.add_argument("--cpu-sample-units", type=int, default=3072, help="units per layer given to the CPU oracle")
     ap.add_argument("--cpu-sample-layers", type=int, default=4, help="layers given to the CPU oracle")
     return ap.parse_args()
@@ -384,6 +409,52 @@ def workload_config(args):
     }
 
 
+def verify_stack(args, ciera, layers, last_w, prev_w, n_layer_picks, n_unit_picks, with_oracle=True):
+    """After a finished step from `prev_w` to `last_w`: the reconstructed weights equal the input everywhere and
+    the two caches agree (device-side comparison), and, for sampled units, message, length, changed-block count
+    and cache equal the CPU oracle's.  Returns (all of it held, number of units the oracle checked)."""
+    import torch
+
+    vb = 4 if args.dtype == "fp32" else 2
+
+    def same_weights(c, w):
+        """Exact comparison over the units' own bytes (alignment gaps between units carry nothing)."""
+        if int(c.units["n_values"].sum()) * vb == w.numel():
+            return torch.equal(c.weights_out[: w.numel()], w)
+        keep = np.zeros(w.numel(), dtype=bool)
+        for u in c.units:
+            keep[int(u["weights_off"]) : int(u["weights_off"]) + int(u["n_values"]) * vb] = True
+        keep = torch.from_numpy(keep).to(w.device)
+        return torch.equal(c.weights_out[: w.numel()][keep], w[keep])
+
+    verified = all(same_weights(c, w) for c, w in zip(layers, last_w))
+    if args.detect == "compare":
+        verified = verified and all(torch.equal(c.sender_cache, c.receiver_cache) for c in layers)
+    sampled = 0
+    if with_oracle:
+        from oracle import ciera_oracle as ora
+
+        ora.build()
+        code = ciera.DTYPE_CODES[args.dtype]
+        wdt = np.uint32 if code == 1 else np.uint16
+        rng = np.random.default_rng(0)
+        for l in sorted(set(rng.integers(0, len(layers), n_layer_picks).tolist())):
+            c = layers[l]
+            for ui in sorted(set(rng.integers(0, len(c.units), n_unit_picks).tolist())):
+                u = c.units[ui]
+                lo, n, mo, co = int(u["weights_off"]), int(u["n_values"]), int(u["msg_off"]), int(u["cache_off"])
+                w_prev = prev_w[l][lo : lo + n * vb].cpu().numpy().view(wdt)
+                w_cur = last_w[l][lo : lo + n * vb].cpu().numpy().view(wdt)
+                cache = ora.cache_init(w_prev, n, code)
+                m, wbytes, _, cb = ora.encode(w_cur, cache, code, args.block)
+                got = c.msg_recv[mo : mo + wbytes].cpu().numpy()
+                verified = verified and int(c.wire_bytes[ui].item()) == wbytes and np.array_equal(got, m)
+                verified = verified and int(c.changed_blocks[ui].item()) == cb
+                verified = verified and np.array_equal(c.receiver_cache[co : co + n].cpu().numpy(), cache)
+                sampled += 1
+    return bool(verified), sampled
+
+
 # --------------------------------------------------------------------------------- main arm
 
 
@@ -507,41 +578,8 @@ def main():
     # ---- correctness at full size: exact round trip everywhere, oracle on sampled units
     last_w = weights_of(step_i - 1)
     prev_w = weights_of(step_i)  # the iterate before the last one (the steps alternate)
-    def same_weights(c, w):
-        """Exact comparison over the units' own bytes (alignment gaps between units carry nothing)."""
-        if int(c.units["n_values"].sum()) * vb == w.numel():
-            return torch.equal(c.weights_out[: w.numel()], w)
-        keep = np.zeros(w.numel(), dtype=bool)
-        for u in c.units:
-            keep[int(u["weights_off"]) : int(u["weights_off"]) + int(u["n_values"]) * vb] = True
-        keep = torch.from_numpy(keep).to(w.device)
-        return torch.equal(c.weights_out[: w.numel()][keep], w[keep])
-
-    verified = all(same_weights(c, w) for c, w in zip(layers, last_w))
-    if args.detect == "compare":
-        verified = verified and all(torch.equal(c.sender_cache, c.receiver_cache) for c in layers)
-    sampled = 0
-    if rank == 0:
-        from oracle import ciera_oracle as ora
-
-        ora.build()
-        code = ciera.DTYPE_CODES[args.dtype]
-        wdt = np.uint32 if code == 1 else np.uint16
-        rng = np.random.default_rng(0)
-        for l in sorted(set(rng.integers(0, len(layers), 4).tolist())):
-            c = layers[l]
-            for ui in rng.integers(0, len(c.units), 4):
-                u = c.units[ui]
-                lo, n, mo, co = int(u["weights_off"]), int(u["n_values"]), int(u["msg_off"]), int(u["cache_off"])
-                w_prev = prev_w[l][lo : lo + n * vb].cpu().numpy().view(wdt)
-                w_cur = last_w[l][lo : lo + n * vb].cpu().numpy().view(wdt)
-                cache = ora.cache_init(w_prev, n, code)
-                m, wbytes, _, cb = ora.encode(w_cur, cache, code, args.block)
-                got = c.msg_recv[mo : mo + wbytes].cpu().numpy()
-                verified = verified and int(c.wire_bytes[ui].item()) == wbytes and np.array_equal(got, m)
-                verified = verified and int(c.changed_blocks[ui].item()) == cb
-                verified = verified and np.array_equal(c.receiver_cache[co : co + n].cpu().numpy(), cache)
-                sampled += 1
+    verified, sampled = verify_stack(args, ciera, layers, last_w, prev_w, n_layer_picks=4, n_unit_picks=16,
+                                     with_oracle=rank == 0)
 
     coded = None
     if args.entropy:
@@ -565,6 +603,11 @@ def main():
                  "per": "layer launch, serial re-run",
                  "note": "rANS of the changed exponents, static 12-bit model per unit; one block per unit"}
 
+    traffic, traffic_note = None, "no ncu capture on record for this workload"
+    if args.dtype == "bf16" and args.block == 512 and args.update == "clustered" and args.f == 0.22 and args.shapes == "olmoe":
+        traffic, traffic_note = measured_traffic("encode_exact_bf16_B512_clustered_f0.22" if args.detect == "compare"
+                                                 else "encode_hashed_bf16_B512_clustered_f0.22", n_layer)
+
     out = {
         "metric": METRIC,
         "value": whole_job_gbps(world, weight_bytes, ms_per_step),
@@ -581,7 +624,7 @@ def main():
         "config": workload_config(args),
         "gpu_launches": int(launches),
         "clocks": clocks,
-        "verified_bit_exact": bool(verified),
+        "verified_bit_exact": verified,
         "element_change_rate_c": element_change_rate,
         "entropy_stage": coded,
         "oracle_sampled_units": sampled,
@@ -597,10 +640,7 @@ def main():
         "roofline": {
             "bound": "hbm", "kernel": ("encode_kernel" if args.detect == "compare" else "encode_kernel (HashCache form)"), "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
             "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBps": enc_gbs / NOMINAL_HBM_GBS,
-            "traffic": ((NCU_ENCODE_TRAFFIC_BYTES_PER_VALUE if args.detect == "compare"
-                         else NCU_HASHED_ENCODE_TRAFFIC_BYTES_PER_VALUE) * n_layer
-                        if args.dtype == "bf16" and args.block == 512 and args.update == "clustered" and args.f == 0.22
-                        and args.shapes == "olmoe" else None),
+            "traffic": traffic, "traffic_note": traffic_note,
             "algorithmic_bytes_per_launch": a_enc,
             "timed": "CUDA events around every encode launch, same K steps re-run on one stream so that "
                      "no other kernel overlaps it",
@@ -621,6 +661,10 @@ def main():
     # ---- per-kernel numbers with each kernel alone on the GPU, three change regimes (one layer)
     if not args.no_regimes and rank == 0 and args.detect == "compare":
         out["kernels_alone"] = kernels_alone(args, layers[0], wa[0], wb[0], peak)
+
+    # ---- the other configurations, one layer each (rank 0, one GPU only)
+    if not args.no_other_configs and rank == 0 and world == 1:
+        out["other_configs"] = other_configs(args, device, peak)
 
     # ---- end to end through the host-buffer entry point (weights start and end in host memory)
     if not args.no_e2e:
@@ -655,6 +699,103 @@ def main():
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+# The other workloads of the build's configuration list, one layer each, kernels timed one after the other on one
+# stream (CUDA events around every launch).  They ride along in the bench line as `other_configs`; `value` is
+# never taken from them.
+OTHER_CONFIGS = [
+    # name, overrides of the command-line defaults
+    ("config2_one_layer_adam_like_update", dict(update="adam")),
+    ("config4_fp32_clustered", dict(dtype="fp32")),
+    ("config4_fp32_adam_like_update", dict(dtype="fp32", update="adam")),
+    ("config5_mixed_8_shards_1pct_iid", dict(shapes="mixed", shards=8, update="inject", inject=0.01, inject_seg=0)),
+    ("config5_mixed_64_shards_10pct_segments", dict(shapes="mixed", shards=64, update="inject", inject=0.1, inject_seg=512)),
+    ("block1_adam_like_update", dict(block=1, update="adam")),
+    ("block2_adam_like_update", dict(block=2, update="adam")),
+    ("block4_adam_like_update", dict(block=4, update="adam")),
+    ("block8_adam_like_update", dict(block=8, update="adam")),
+    ("block1_half_of_the_exponents_change", dict(block=1, update="inject", inject=0.5, inject_seg=0)),
+    ("block64_adam_like_update", dict(block=64, update="adam")),
+    ("fp16_clustered", dict(dtype="fp16")),
+    ("hashed_sender_bf16_block512", dict(detect="hash")),
+    ("hashed_sender_bf16_block32_adam_like_update", dict(detect="hash", block=32, update="adam")),
+    ("hashed_sender_fp32_block512", dict(detect="hash", dtype="fp32")),
+    ("entropy_stage_bf16_block512", dict(entropy=True)),
+]
+
+
+def one_layer_case(args, device, peak, over, steps=5):
+    """One layer of the workload `args` + `over`: three warm-up steps, then `steps` timed ones, all on one stream."""
+    import torch
+
+    from paper_2609_04609_b200 import ciera, runtime
+    from paper_2609_04609_b200 import workloads as wl
+
+    a = argparse.Namespace(**{**vars(args), "layers": 1, "experts": 64, "shards": 16, "block": 512, "dtype": "bf16",
+                              "update": "clustered", "f": 0.22, "shapes": "olmoe", "detect": "compare",
+                              "entropy": False, **over})
+    layers, wa, wb = build_stack(a, device, seed_base=4321)
+    codec = layers[0]
+    vb = wl.VALUE_BYTES[a.dtype]
+    stream = torch.cuda.Stream()
+    pipe = runtime.LayerPipeline(layers, stream, stream, entropy=a.entropy)
+    i = 0
+    for _ in range(3):
+        pipe.step(wb if i % 2 == 0 else wa)
+        i += 1
+    timers = []
+    for _ in range(steps):
+        pipe.step(wb if i % 2 == 0 else wa, None, timers)
+        i += 1
+    torch.cuda.synchronize()
+    codec.check_status()
+    last_w, prev_w = (wb, wa) if (i - 1) % 2 == 0 else (wa, wb)
+    verified, sampled = verify_stack(a, ciera, layers, last_w, prev_w, n_layer_picks=1, n_unit_picks=6)
+    n = codec.plan.total_values
+    q = int(codec.changed_blocks.sum().item()) / max(codec.n_blocks(), 1)
+    enc_ms, tra_ms, dec_ms = [float(np.mean([t[2 * k].elapsed_time(t[2 * k + 1]) for t in timers])) for k in range(3)]
+    a_enc, a_tra, a_dec = algorithmic_bytes(n, q, a.dtype, a.block, a.detect)
+    res = {
+        "workload": workload_config(a)["workload"], "values": n, "units": len(codec.units),
+        "block_change_rate_q": q, "bytes_ratio": codec.paper_bytes() / (n * vb),
+        "encode_ms": enc_ms, "transport_ms": tra_ms, "decode_ms": dec_ms,
+        "encode_frac": a_enc / (enc_ms * 1e-3) / 1e9 / peak, "transport_frac": a_tra / (tra_ms * 1e-3) / 1e9 / peak,
+        "decode_frac": a_dec / (dec_ms * 1e-3) / 1e9 / peak,
+        "encode_GBps_of_weights": n * vb / (enc_ms * 1e-3) / 1e9, "decode_GBps_of_weights": n * vb / (dec_ms * 1e-3) / 1e9,
+        "verified_bit_exact": verified, "oracle_sampled_units": sampled,
+    }
+    if a.entropy:
+        res["entropy_encode_ms"], res["entropy_decode_ms"] = [
+            float(np.mean([t[k].elapsed_time(t[k + 1]) for t in timers])) for k in (6, 8)]
+        # the coded size: one more sender step, read between the entropy stage and the transport
+        w = wb if i % 2 == 0 else wa
+        codec.encode(w[0])
+        raw = codec.paper_bytes()
+        codec.entropy_encode()
+        coded = codec.paper_bytes()
+        fixed = sum(ciera.message_bytes(int(u["n_values"]), codec.dtype, a.block, 0) for u in codec.units if int(u["n_values"]))
+        res["bytes_ratio_coded"] = coded / (n * vb)
+        res["payload_coded_over_raw"] = (coded - fixed) / (raw - fixed) if raw > fixed else None
+        codec.transport()
+        codec.entropy_decode()
+        codec.decode()
+        torch.cuda.synchronize()
+        codec.check_status()
+    del layers, wa, wb, pipe
+    torch.cuda.empty_cache()
+    return res
+
+
+def other_configs(args, device, peak):
+    out = {"per": "one layer; kernels one after the other on one stream, CUDA events around every launch; fractions "
+                  "are algorithmic bytes per launch over the measured copy bandwidth"}
+    for name, over in OTHER_CONFIGS:
+        try:
+            out[name] = one_layer_case(args, device, peak, over)
+        except Exception as e:  # one failing side case must not take the headline line with it
+            out[name] = {"error": f"{type(e).__name__}: {e}"}
+    return out
 
 
 def kernels_alone(args, codec, w_a, w_b, peak):

@@ -357,6 +357,21 @@ CIERA_API int ciera_select_shards(const ciera_gain_in* shards, uint32_t n_shards
 
 /* ---- diagnostics ---------------------------------------------------------------------------- */
 
+/* Self-test of the device-side failure path (no counterpart in the paper: Algorithm 1 has no failure
+ * handling).  Every wait inside the persistent kernels -- on a look-back status word of another tile,
+ * on a shared-memory barrier that a bulk copy or another warp completes -- is bounded: when the bound
+ * runs out the waiting role raises CIERA_ERR_TIMEOUT in the caller's status word, the thread block
+ * stops, and the kernel returns, so the context stays usable.  This call runs one tiny kernel (one
+ * thread block) that performs both kinds of wait with a limit of `max_polls` polls (1 .. 4096; a
+ * barrier poll suspends for at most 20 microseconds) on a word and a barrier that nothing completes.
+ *   scratch_dev  device, 8 bytes, 8-byte aligned: the status word that is polled (cleared by the call)
+ *   status_dev   device int32: receives CIERA_ERR_TIMEOUT if it was 0
+ *   report_dev   device, 4 x int32 (cleared by the call): [0] = 1 the status-word wait gave up,
+ *                [1] = 1 the barrier wait gave up, [2] = the block's abort flag, [3] = max_polls
+ * Asynchronous on `stream`. */
+CIERA_API int ciera_selftest_bounded_waits(uint32_t max_polls, void* scratch_dev, int32_t* status_dev,
+                                           int32_t* report_dev, void* stream);
+
 /* cudaError_t of the last failing runtime call made by the calling thread inside this library. */
 CIERA_API int ciera_last_cuda_error(void);
 /* Number of kernels this library has launched from the calling process (for launch accounting). */

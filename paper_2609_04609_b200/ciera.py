@@ -85,6 +85,7 @@ _SIGS = {
     "ciera_roundtrip_host": ([_vp, _vp, _sz, _vp, _vp, _vp, _vp], _i32),
     "ciera_should_compress": ([ctypes.POINTER(GainIn), ctypes.POINTER(_dbl), ctypes.POINTER(_i32)], _i32),
     "ciera_select_shards": ([ctypes.POINTER(GainIn), _u32, _u64, _i32, _vp, _vp, _vp, _vp, _vp], _i32),
+    "ciera_selftest_bounded_waits": ([_u32, _vp, _vp, _vp, _vp], _i32),
     "ciera_last_cuda_error": ([], _i32),
     "ciera_kernel_launch_count": ([], _u64),
     "ciera_status_string": ([_i32], ctypes.c_char_p),
@@ -143,6 +144,14 @@ def message_bytes(n: int, dtype: int, block: int, payload_bytes: int) -> int:
 
 def kernel_launch_count() -> int:
     return int(_lib.ciera_kernel_launch_count())
+
+
+def selftest_bounded_waits(max_polls: int, scratch: torch.Tensor, status: torch.Tensor, report: torch.Tensor,
+                           stream=None) -> None:
+    """Runs the library's two kinds of bounded device wait with a short limit on things nobody completes
+    (see ciera.h): ``status`` receives ERR_TIMEOUT, ``report`` (4 x int32) says which waits gave up."""
+    _check("ciera_selftest_bounded_waits",
+           _lib.ciera_selftest_bounded_waits(max_polls, _ptr(scratch), _ptr(status), _ptr(report), _stream(stream)))
 
 
 # ------------------------------------------------------------------------------ plan

@@ -345,7 +345,9 @@ entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long 
     if (un.n_values == 0 || segments_of(un.n_values) > kLongSegs) return;
     const uint64_t payoff = payload_offset(un.n_values, sm_bytes_per_value, log2b);
     const uint64_t P = wire_bytes[unit] - payoff;
-    if (P == 0) return;  // nothing to code
+    // nothing to code; or a length that no sender step reports (shorter than the fixed sections, or more
+    // than one payload byte per value): everything below is indexed by P, so such a unit is left alone
+    if (P == 0 || P > un.n_values) return;
     uint8_t* const pay = msgs + un.msg_off + payoff;  // 16-byte aligned
     const uint32_t nseg = (uint32_t)segments_of(P);
 
@@ -418,12 +420,17 @@ __device__ __forceinline__ uint32_t* long_hist(uint8_t* recs, uint32_t li) { ret
 __device__ __forceinline__ uint16_t* long_model(uint8_t* recs, uint32_t li) { return reinterpret_cast<uint16_t*>(recs + (size_t)li * kLongRec + 1024); }
 __device__ __forceinline__ LongState* long_state(uint8_t* recs, uint32_t li) { return reinterpret_cast<LongState*>(recs + (size_t)li * kLongRec + 1536); }
 
-// raw payload length of a unit on the sender (0: nothing to code or too much for 32-bit counts)
+// raw payload length of a unit on the sender (0: nothing to code).  A reported length that no sender
+// step can have produced -- shorter than the fixed sections, or a payload of more than one byte per
+// value, e.g. the stale word of a unit that an aborted encode never finished -- also gives 0: the
+// histogram, the segments and the scratch slots are all indexed by this length, so it must stay
+// inside the unit's slot (the entropy stage takes bf16 and fp32 only: one exponent byte per value,
+// and plans are limited to units whose block counts fit 32 bits).
 __device__ __forceinline__ uint64_t sender_payload(const ciera_unit& un, uint32_t smb, uint32_t log2b,
                                                    const unsigned long long* wire_bytes, uint32_t unit, uint64_t& payoff) {
     payoff = payload_offset(un.n_values, smb, log2b);
     const uint64_t P = wire_bytes[unit] - payoff;
-    return P < (1ull << 32) ? P : 0;
+    return (P <= un.n_values && P < (1ull << 32)) ? P : 0;
 }
 
 __global__ void __launch_bounds__(kEntThreads)

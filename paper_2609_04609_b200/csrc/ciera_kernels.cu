@@ -1,6 +1,7 @@
 // Auxiliary sm_100a kernels of libciera: cache initialisation, the transport stand-in, and the
 // host-buffer round trip.  (Encode and decode live in ciera_encode.cu / ciera_decode.cu.)
 #include "ciera_bits.cuh"
+#include "ciera_lookback.cuh"
 #include "ciera_pipe.cuh"
 
 namespace ciera {
@@ -42,11 +43,24 @@ cache_fill_kernel(const TileDesc* __restrict__ tiles, const uint8_t* __restrict_
 //
 // Tile j of a unit moves bytes [j * chunk, (j + 1) * chunk) of the unit's slot (chunk = 16 KB for
 // bf16 and fp16, 32 KB for fp32, plus a tile's share of the bitmap when blocks are fine), the last
-// tile also what lies beyond, cut off at the length the sender reported.
+// tile also what lies beyond, cut off at the length the sender reported.  A reported length beyond
+// what a message of the unit can ever take (every block changed) cannot come from a finished sender
+// step -- it is a stale or damaged word, e.g. of a unit that an aborted encode left unfinished: such a
+// unit moves nothing and raises CIERA_ERR_CORRUPT, so that no copy ever leaves the unit's slot.
+
+// largest message of a unit of n values: all sections with every block changed (device twin of
+// ciera_message_capacity)
+__device__ __forceinline__ uint64_t slot_capacity(uint64_t n, int dtype, uint32_t log2b) {
+    if (n == 0) return 0;
+    const uint64_t nb = num_blocks(n, log2b);
+    return payload_offset_of(n, dtype, log2b) + (nb - 1) * block_payload_bytes(1ull << log2b, dtype) +
+           block_payload_bytes(n - ((nb - 1) << log2b), dtype);
+}
 
 // the part of a tile descriptor the copy needs (keeps the prefetched copies small in registers)
 struct CopyDesc {
     uint64_t msg_off;
+    uint64_t n_unit;
     uint32_t unit, tile_in_unit, n_tiles_unit;
 };
 __device__ __forceinline__ CopyDesc load_copy_desc(const TileDesc* t) {
@@ -54,6 +68,7 @@ __device__ __forceinline__ CopyDesc load_copy_desc(const TileDesc* t) {
     const uint4 b = __ldg(p + 1), c = __ldg(p + 2);
     CopyDesc d;
     d.msg_off = (uint64_t)b.x | ((uint64_t)b.y << 32);
+    d.n_unit = (uint64_t)b.z | ((uint64_t)b.w << 32);
     d.unit = c.x;
     d.tile_in_unit = c.y;
     d.n_tiles_unit = c.w;
@@ -88,9 +103,9 @@ struct PipeCtl {
 };
 
 __global__ void __launch_bounds__(kPipeThreads, 2)
-transport_pipe_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint64_t chunk, const uint8_t* __restrict__ src,
-                      uint8_t* __restrict__ dst, const unsigned long long* __restrict__ wire_bytes, unsigned int* ticket,
-                      int32_t* status) {
+transport_pipe_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint64_t chunk, int dtype, uint32_t log2b,
+                      const uint8_t* __restrict__ src, uint8_t* __restrict__ dst,
+                      const unsigned long long* __restrict__ wire_bytes, unsigned int* ticket, int32_t* status) {
     extern __shared__ __align__(128) uint8_t smem[];
     PipeCtl* ctl = reinterpret_cast<PipeCtl*>(smem + (size_t)kPipeStages * kPipeStage);
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
@@ -123,7 +138,13 @@ transport_pipe_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint
         auto advance = [&]() {
             td_c = td_b;
             t_c = t_b;
-            if (t_c < n_tiles) used_c = __ldg(wire_bytes + td_c.unit);
+            if (t_c < n_tiles) {
+                used_c = __ldg(wire_bytes + td_c.unit);
+                if (used_c > slot_capacity(td_c.n_unit, dtype, log2b)) {  // not a length any sender step reports
+                    if (status) atomicCAS(status, 0, (int32_t)CIERA_ERR_CORRUPT);
+                    used_c = 0;
+                }
+            }
             t_b = t_a;
             if (t_b < n_tiles) td_b = load_copy_desc(tiles + t_b);
             // once a batch starts past the end there is nothing more to draw
@@ -231,6 +252,40 @@ static int transport_pipe_grid_limit(int* out) {
     return CIERA_OK;
 }
 
+// ------------------------------------------------------------------------------------------
+// Self-test of the bounded waits: both kinds of wait the persistent kernels use -- the poll of a
+// look-back status word in global memory and the wait on a shared-memory barrier -- are run with a
+// short limit on a word and a barrier that nobody ever completes.  Each must give up, raise
+// CIERA_ERR_TIMEOUT in the status word and return; the kernel then leaves normally.  Nothing traps,
+// nothing spins at the kernels' own limits, and no other kernel is involved.
+//   report[0] = 1: the status-word wait gave up and returned "prefix 0"
+//   report[1] = 1: the barrier wait gave up (returned false)
+//   report[2] = the block's abort flag afterwards (1 expected)
+//   report[3] = polls the barrier wait was given
+__global__ void __launch_bounds__(64)
+selftest_waits_kernel(const unsigned long long* never_written, uint32_t max_polls, int32_t* status, int32_t* report) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        mbar_fence_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned long long st = wait_status(never_written, status, max_polls);
+        report[0] = (st == kFlagPrefix) ? 1 : 0;
+    } else if (threadIdx.x == 32) {
+        const bool ok = mbar_wait(&bar, 0u, &abort_flag, status, max_polls);
+        report[1] = ok ? 0 : 1;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        report[2] = abort_flag;
+        report[3] = (int32_t)max_polls;
+    }
+}
+
 }  // namespace ciera
 
 // ------------------------------------------------------------------------------------------
@@ -291,8 +346,9 @@ extern "C" int ciera_transport(const ciera_plan* p, const void* src_messages_dev
     const uint32_t want_blocks = (nt + kPipeBatch - 1) / kPipeBatch;
     const uint32_t grid = want_blocks < (uint32_t)limit ? want_blocks : (uint32_t)limit;
     transport_pipe_kernel<<<grid, kPipeThreads, (size_t)kPipeStages * kPipeStage + sizeof(PipeCtl), (cudaStream_t)stream>>>(
-        p->tiles_dev, nt, transport_chunk_bytes(p->dtype == CIERA_FP32 ? 3u : 1u, p->log2b), (const uint8_t*)src_messages_dev,
-        (uint8_t*)dst_messages_dev, (const unsigned long long*)wire_bytes_dev, ticket, status_dev);
+        p->tiles_dev, nt, transport_chunk_bytes(p->dtype == CIERA_FP32 ? 3u : 1u, p->log2b), p->dtype, p->log2b,
+        (const uint8_t*)src_messages_dev, (uint8_t*)dst_messages_dev, (const unsigned long long*)wire_bytes_dev, ticket,
+        status_dev);
     count_launch();
     return check_launch();
 }
@@ -322,4 +378,20 @@ extern "C" int ciera_roundtrip_host(const ciera_plan* p, const void* weights_hos
         if (e != cudaSuccess) return record_cuda_error(e);
     }
     return CIERA_OK;
+}
+
+extern "C" int ciera_selftest_bounded_waits(uint32_t max_polls, void* scratch_dev, int32_t* status_dev, int32_t* report_dev,
+                                            void* stream) {
+    if (!scratch_dev || !status_dev || !report_dev) return CIERA_ERR_INVALID_ARG;
+    if (max_polls == 0 || max_polls > 4096) return CIERA_ERR_INVALID_ARG;  // a self-test, not a way to stall the GPU
+    if (((uintptr_t)scratch_dev & 7u) || ((uintptr_t)status_dev & 3u) || ((uintptr_t)report_dev & 3u))
+        return CIERA_ERR_MISALIGNED;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaMemsetAsync(scratch_dev, 0, 8, s);  // the word that is polled: empty, and nobody fills it
+    if (e != cudaSuccess) return record_cuda_error(e);
+    e = cudaMemsetAsync(report_dev, 0, 16, s);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    selftest_waits_kernel<<<1, 64, 0, s>>>((const unsigned long long*)scratch_dev, max_polls, status_dev, report_dev);
+    count_launch();
+    return check_launch();
 }

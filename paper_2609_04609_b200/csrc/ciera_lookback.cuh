@@ -19,14 +19,15 @@ __device__ __forceinline__ void st_status(unsigned long long* p, unsigned long l
     asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 
-// Polls a tile status word until its flag is set.  Bounded: after kMaxPolls reads it gives up,
-// raises CIERA_ERR_TIMEOUT and returns "prefix 0" so that the caller finishes (with unspecified
-// output) instead of hanging.
-__device__ __forceinline__ unsigned long long wait_status(const unsigned long long* p, int32_t* status) {
+// Polls a tile status word until its flag is set.  Bounded: after max_polls reads (kMaxPolls in the
+// kernels; the self-test passes a few dozen) it gives up, raises CIERA_ERR_TIMEOUT and returns
+// "prefix 0" so that the caller finishes (with unspecified output) instead of hanging.
+__device__ __forceinline__ unsigned long long wait_status(const unsigned long long* p, int32_t* status,
+                                                          uint32_t max_polls = kMaxPolls) {
     unsigned long long st = ld_status(p);
     uint32_t polls = 0;
     while ((st >> 62) == 0) {
-        if (++polls > kMaxPolls) {
+        if (++polls > max_polls) {
             if (status) atomicCAS(status, 0, (int32_t)CIERA_ERR_TIMEOUT);
             return kFlagPrefix;
         }

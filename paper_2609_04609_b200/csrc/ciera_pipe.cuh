@@ -42,9 +42,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 
 // Bounded wait for the phase with the given parity.  `abort` is a shared-memory flag common to
-// the thread block.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort, int32_t* status) {
-    for (uint32_t i = 0; i < kMaxBarrierPolls; ++i) {
+// the thread block.  max_polls: kMaxBarrierPolls in the kernels; the self-test passes a few dozen.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort, int32_t* status,
+                                          uint32_t max_polls = kMaxBarrierPolls) {
+    for (uint32_t i = 0; i < max_polls; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort) return false;
     }

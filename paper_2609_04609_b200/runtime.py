@@ -19,7 +19,9 @@ from .workloads import VALUE_BYTES, layout_units
 
 class LayerCodec:
     def __init__(self, units: np.ndarray, dtype: str, block: int, weights_bytes: int, cache_bytes: int,
-                 msg_bytes: int, device="cuda:0", with_output: bool = True):
+                 msg_bytes: int, device="cuda:0", with_output: bool = True, slack: int = 0):
+        """``slack``: extra bytes (entries, for the per-unit arrays) allocated behind every buffer; the
+        library is never told about them, so whatever a caller puts there must survive every call."""
         self.dtype_name = dtype
         self.dtype = ciera.DTYPE_CODES[dtype]
         self.block = block
@@ -27,16 +29,24 @@ class LayerCodec:
         self.plan = ciera.Plan(units, self.dtype, block, self.device)
         self.units = self.plan.units
         dev = self.device
-        u8 = dict(dtype=torch.uint8, device=dev)
         self.weights_bytes, self.cache_bytes, self.msg_bytes = weights_bytes, cache_bytes, msg_bytes
-        self.sender_cache = torch.zeros(max(cache_bytes, 16), **u8)
-        self.receiver_cache = torch.zeros(max(cache_bytes, 16), **u8)
-        self.msg_send = torch.zeros(max(msg_bytes, 16), **u8)
-        self.msg_recv = torch.zeros(max(msg_bytes, 16), **u8)
-        self.weights_out = torch.zeros(max(weights_bytes, 16), **u8) if with_output else None
+        # every buffer is a view of an allocation that is `slack` bytes (entries) longer
+        self.slack = slack
+        self.allocations = {}
+
+        def alloc(name, size, dt=torch.uint8):
+            full = torch.zeros(size + slack, dtype=dt, device=dev)
+            self.allocations[name] = full
+            return full[:size]
+
+        self.sender_cache = alloc("sender_cache", max(cache_bytes, 16))
+        self.receiver_cache = alloc("receiver_cache", max(cache_bytes, 16))
+        self.msg_send = alloc("msg_send", max(msg_bytes, 16))
+        self.msg_recv = alloc("msg_recv", max(msg_bytes, 16))
+        self.weights_out = alloc("weights_out", max(weights_bytes, 16)) if with_output else None
         n = max(self.plan.n_units, 1)
-        self.wire_bytes = torch.zeros(n, dtype=torch.int64, device=dev)
-        self.changed_blocks = torch.zeros(n, dtype=torch.int32, device=dev)
+        self.wire_bytes = alloc("wire_bytes", n, torch.int64)
+        self.changed_blocks = alloc("changed_blocks", n, torch.int32)
         self.workspace = self.plan.new_workspace()
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
 

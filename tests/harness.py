@@ -53,6 +53,78 @@ class OracleTable:
         return dict(msgs=msgs, wire=wire, chg=chg, pay=pay, recon=recon)
 
 
+class Canaries:
+    """Guard bytes around everything a step may write (the memory checker of the CUDA toolkit is not
+    available on the test machines).  The gaps that the layout leaves between the units inside
+    ``weights_out``, both caches and both message buffers, the ``slack`` bytes behind each of those
+    buffers, and the slack entries behind the per-unit outputs are filled with a pattern when the
+    object is made; ``check`` asserts that every one of them is untouched.  No kernel has any business
+    there: a store that lands in a gap corrupts a neighbouring tensor in a real run without showing up
+    in any comparison of the units' own bytes.  (Inside a message slot the bytes between the reported
+    length and the slot's capacity are unspecified, so only the bytes past the capacity are guarded.)"""
+
+    PATTERN = 0xA5
+
+    def __init__(self, codec):
+        self.codec = codec
+        vb = VB[codec.dtype]
+        u = codec.units
+        n = u["n_values"].astype(np.int64)
+        spans = {
+            "weights_out": (u["weights_off"].astype(np.int64), n * vb),
+            "sender_cache": (u["cache_off"].astype(np.int64), n),
+            "receiver_cache": (u["cache_off"].astype(np.int64), n),
+            "msg_send": (u["msg_off"].astype(np.int64), u["msg_capacity"].astype(np.int64)),
+            "msg_recv": (u["msg_off"].astype(np.int64), u["msg_capacity"].astype(np.int64)),
+        }
+        self.guards = {}
+        for name, (off, length) in spans.items():
+            full = codec.allocations.get(name)
+            if full is None:
+                continue
+            idx = torch.from_numpy(self._uncovered(off, length, full.numel())).to(full.device)
+            full[idx] = self.PATTERN
+            self.guards[name] = idx
+        self.tails = {}
+        for name, live in (("wire_bytes", len(u)), ("changed_blocks", len(u))):
+            full = codec.allocations[name]
+            live = max(live, 1)
+            full[live:] = 0x5A5A5A5A
+            self.tails[name] = live
+
+    @staticmethod
+    def _uncovered(off, length, total):
+        """Indices of [0, total) that lie in no [off_i, off_i + length_i)."""
+        keep = length > 0
+        off, length = off[keep], length[keep]
+        order = np.argsort(off, kind="stable")
+        off, end = off[order], (off + length)[order]
+        starts = np.concatenate([[0], end])
+        stops = np.concatenate([off, [total]])
+        assert np.all(stops >= starts), "units overlap"
+        parts = [np.arange(a, b, dtype=np.int64) for a, b in zip(starts, stops) if b > a]
+        return np.concatenate(parts) if parts else np.zeros(0, np.int64)
+
+    def guarded_bytes(self):
+        return sum(int(i.numel()) for i in self.guards.values())
+
+    def check(self, label=""):
+        for name, idx in self.guards.items():
+            full = self.codec.allocations[name]
+            bad = (full[idx] != self.PATTERN).nonzero()
+            assert bad.numel() == 0, (f"{label}: a store landed outside the units' bytes of {name}, first at byte "
+                                      f"{int(idx[bad[0, 0]])} of the buffer")
+        for name, live in self.tails.items():
+            full = self.codec.allocations[name]
+            assert bool((full[live:] == 0x5A5A5A5A).all()), f"{label}: entries past the last unit of {name} were written"
+
+
+def guard(codec):
+    """Arms the guard bytes of a codec made with ``slack`` > 0 (see Canaries); returns the codec."""
+    codec.canaries = Canaries(codec)
+    return codec
+
+
 def to_dev_bytes(bits: np.ndarray, device) -> torch.Tensor:
     """Raw bytes of a host bit-pattern array, on the device (padded to >= 16 bytes)."""
     b = np.ascontiguousarray(bits).view(np.uint8)
@@ -85,6 +157,8 @@ def compare_step(codec, exp, w_flat, label=""):
 
 
 def compare_caches(codec, table, label=""):
+    if getattr(codec, "canaries", None) is not None:
+        codec.canaries.check(label)
     cs = codec.sender_cache.cpu().numpy()
     cr = codec.receiver_cache.cpu().numpy()
     for i, u in enumerate(codec.units):

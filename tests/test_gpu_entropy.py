@@ -4,7 +4,7 @@ import numpy as np
 import pytest
 import torch
 
-from harness import to_dev_bytes
+from harness import guard, to_dev_bytes
 from oracle import ciera_oracle as ora
 from oracle import rans_oracle as rans
 from paper_2609_04609_b200 import workloads as wl
@@ -29,7 +29,7 @@ def rt():
 def _run(rt, sizes, n_shards, dtype, block, traj, from_zero):
     """Every step: encode, entropy-encode, transport, entropy-decode, decode; each stage against the oracle."""
     ciera, runtime = rt
-    codec = runtime.LayerCodec.from_tensors(sizes, n_shards, NAME[dtype], block, DEV)
+    codec = guard(runtime.LayerCodec.from_tensors(sizes, n_shards, NAME[dtype], block, DEV, slack=256))
     units = codec.units
 
     def unit_w(w, u):
@@ -72,6 +72,7 @@ def _run(rt, sizes, n_shards, dtype, block, traj, from_zero):
         for u in units:
             lo, n = int(u["weights_off"]) // VB[dtype], int(u["n_values"])
             assert np.array_equal(out[lo : lo + n], w[lo : lo + n]), f"t={t}: reconstruction differs"
+        codec.canaries.check(f"t={t}")
     return coded_units
 
 

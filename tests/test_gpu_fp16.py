@@ -4,7 +4,7 @@ import numpy as np
 import pytest
 import torch
 
-from harness import OracleTable, compare_caches, compare_recon, compare_step, to_dev_bytes
+from harness import OracleTable, compare_caches, compare_recon, compare_step, guard, to_dev_bytes
 from paper_2609_04609_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -25,7 +25,7 @@ def rt():
 
 def _run(rt, sizes, shards, block, traj_fn, zero_cache=False, label=""):
     ciera, runtime = rt
-    codec = runtime.LayerCodec.from_tensors(sizes, shards, "fp16", block, DEV)
+    codec = guard(runtime.LayerCodec.from_tensors(sizes, shards, "fp16", block, DEV, slack=256))
     table = OracleTable(codec.units, FP16, block, codec.cache_bytes, codec.msg_bytes)
     n = codec.weights_bytes // 2
     traj = traj_fn(n)

@@ -9,7 +9,7 @@ import numpy as np
 import pytest
 import torch
 
-from harness import OracleTable, compare_caches, compare_recon, compare_step, to_dev_bytes
+from harness import OracleTable, compare_caches, compare_recon, compare_step, guard, to_dev_bytes
 from oracle import ciera_oracle as ora
 from oracle import rans_oracle as rans
 from paper_2609_04609_b200 import workloads as wl
@@ -69,7 +69,7 @@ def _trajectory(rng, n, dtype):
 def test_random_tables_full_step(rt, seed):
     ciera, runtime = rt
     rng, sizes, shards, dtype, block = _random_case(1000 + seed)
-    codec = runtime.LayerCodec.from_tensors(sizes, shards, NAME[dtype], block, DEV)
+    codec = guard(runtime.LayerCodec.from_tensors(sizes, shards, NAME[dtype], block, DEV, slack=256))
     table = OracleTable(codec.units, dtype, block, codec.cache_bytes, codec.msg_bytes)
     n = codec.weights_bytes // VB[dtype]
     traj = _trajectory(rng, max(n, 1), dtype)
@@ -93,7 +93,7 @@ def test_random_tables_hashed_sender_and_entropy_stage(rt, seed):
     rng, sizes, shards, dtype, block = _random_case(5000 + seed)
     dtype = dtype % 2  # the hashed sender and the entropy stage take bf16 and fp32
     block = max(block, 16)
-    codec = runtime.LayerCodec.from_tensors(sizes, shards, NAME[dtype], block, DEV)
+    codec = guard(runtime.LayerCodec.from_tensors(sizes, shards, NAME[dtype], block, DEV, slack=256))
     units = codec.units
     n = codec.weights_bytes // VB[dtype]
     traj = _trajectory(rng, max(n, 1), dtype)
@@ -131,3 +131,4 @@ def test_random_tables_hashed_sender_and_entropy_stage(rt, seed):
         for u in units:
             lo, nn = int(u["weights_off"]) // VB[dtype], int(u["n_values"])
             assert np.array_equal(out[lo : lo + nn], w[lo : lo + nn]), f"{label} t={t}: reconstruction"
+        codec.canaries.check(f"{label} t={t}")

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 import torch
 
-from harness import to_dev_bytes
+from harness import guard, to_dev_bytes
 from oracle import ciera_oracle as ora
 from paper_2609_04609_b200 import workloads as wl
 
@@ -28,7 +28,7 @@ def rt():
 
 def _run(rt, sizes, n_shards, dtype, block, traj, from_zero=False):
     ciera, runtime = rt
-    codec = runtime.LayerCodec.from_tensors(sizes, n_shards, NAME[dtype], block, DEV)
+    codec = guard(runtime.LayerCodec.from_tensors(sizes, n_shards, NAME[dtype], block, DEV, slack=256))
     units = codec.units
     first = None if from_zero else traj[0]
 
@@ -72,6 +72,7 @@ def _run(rt, sizes, n_shards, dtype, block, traj, from_zero=False):
         for u in units:
             lo, n = int(u["weights_off"]) // VB[dtype], int(u["n_values"])
             assert np.array_equal(out[lo : lo + n], w[lo : lo + n]), f"t={t}: reconstruction differs"
+        codec.canaries.check(f"t={t}")
         changed_total.append(int(chg.sum()))
     return changed_total
 

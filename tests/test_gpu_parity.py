@@ -7,7 +7,7 @@ import numpy as np
 import pytest
 import torch
 
-from harness import OracleTable, compare_caches, compare_recon, compare_step, to_dev_bytes
+from harness import OracleTable, compare_caches, compare_recon, compare_step, guard, to_dev_bytes
 from paper_2609_04609_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -27,7 +27,7 @@ def rt():
 
 def _make(rt, sizes, n_shards, dtype, block):
     ciera, runtime = rt
-    codec = runtime.LayerCodec.from_tensors(sizes, n_shards, NAME[dtype], block, DEV)
+    codec = guard(runtime.LayerCodec.from_tensors(sizes, n_shards, NAME[dtype], block, DEV, slack=256))
     table = OracleTable(codec.units, dtype, block, codec.cache_bytes, codec.msg_bytes)
     n_flat = codec.weights_bytes // (2 if dtype == 0 else 4)
     return codec, table, n_flat
@@ -312,7 +312,8 @@ def test_full_size_layer_sampled_units(rt, dtype, block):
     b0, b1, b2 = (w.view(torch.uint8) for w in (w0, w1, w2))
     codec.init_caches(b0)
     rng = np.random.default_rng(5)
-    picks = sorted(set(rng.integers(0, len(codec.units), 12).tolist()) | {0, len(codec.units) - 1})
+    picks = sorted(set(rng.integers(0, len(codec.units), 80).tolist()) | {0, len(codec.units) - 1})
+    assert len(picks) >= 64
     wdt = WDT[dtype]
     prev = b0
     for cur in (b1, b2):
@@ -335,6 +336,80 @@ def test_full_size_layer_sampled_units(rt, dtype, block):
         prev = cur
     q = int(codec.changed_blocks.sum().item()) / codec.n_blocks()
     assert q > (0.99 if block >= 256 else 0.8)  # the i.i.d. step changes (nearly) every block
+
+
+@pytest.mark.parametrize("n_shards", [8, 64])
+def test_config5_full_size_mixed_shapes(rt, n_shards):
+    """The mixed-shape sweep at full size in ONE plan: 256 fine-grained experts x (2048x512, 2048x512, 512x2048)
+    plus dense tensors of 4 KB ... 256 MB (bf16) and one ragged 1000-value tensor, cut into 8 or 64 shards.  At 8
+    shards the 256 MB tensor gives units of 16.8 M values = 2048 tiles (tiles spread over the thread blocks,
+    look-back between them, cooperative launch, per-tile counts from the prefix kernel at decode time); at 64
+    shards the 4 KB tensor gives units of 32 values, far below the block size, and the ragged tensor a short-tail
+    unit and an empty one.  Exponent changes are injected at 0.1 %, 1 %, 10 % and 50 %, value by value and in
+    512-aligned segments, on the device.  After every step: the round trip is exact over the whole buffer (the
+    gaps between units hold guard bytes on both sides of the comparison), both caches agree, and messages,
+    lengths, counts and caches of sampled units equal the oracle's -- among them the first, a middle and the last
+    shard of the 256 MB tensor, a 32-value unit, the short-tail unit and the empty unit."""
+    ciera, runtime = rt
+    from oracle import ciera_oracle as ora
+
+    block = 512
+    dense = wl.dense_tensor_sizes()
+    sizes = [r * c for r, c in wl.fine_grained_layer_shapes(256)] + dense + [1000]
+    codec = guard(runtime.LayerCodec.from_tensors(sizes, n_shards, "bf16", block, DEV, slack=256))
+    units = codec.units
+    n = codec.weights_bytes // 2
+    first_of = lambda tensor: tensor * n_shards  # index of a tensor's first unit
+    big, small, ragged = first_of(256 * 3 + len(dense) - 1), first_of(256 * 3), first_of(256 * 3 + len(dense))
+    assert int(units[big]["n_values"]) == dense[-1] // n_shards
+    special = [big, big + n_shards // 2, big + n_shards - 1, small, small + n_shards - 1]
+    tail = [ragged + i for i in range(n_shards) if int(units[ragged + i]["n_values"]) < -(-1000 // n_shards)]
+    assert any(int(units[i]["n_values"]) == 0 for i in tail) or n_shards == 8
+    special += tail[:3]
+    rng = np.random.default_rng(77 + n_shards)
+    picks = sorted(set(special) | set(rng.integers(0, len(units), 16).tolist()))
+    if n_shards == 8:
+        assert codec.plan.n_tiles > 0 and int(units[big]["n_values"]) // 8192 == 2048
+    else:
+        assert int(units[small]["n_values"]) == 32
+
+    gen = wl.make_generator(5005 + n_shards, DEV)
+    w = wl.init_weights(n, "bf16", gen)
+    gaps = codec.canaries.guards["weights_out"]
+    gaps = gaps[gaps < w.numel() * 2]
+
+    def as_bytes(t):
+        b = t.view(torch.uint8)
+        b[gaps] = codec.canaries.PATTERN  # not part of any unit: make both sides of the comparison agree there
+        return b
+
+    prev = as_bytes(w)
+    codec.init_caches(prev)
+    for c, seg in [(0.001, 0), (0.01, 0), (0.1, 0), (0.5, 0), (0.001, 512), (0.01, 512), (0.1, 512), (0.5, 512)]:
+        w = wl.inject_exponent_changes(w, gen, c, seg)
+        cur = as_bytes(w)
+        codec.step(cur)
+        torch.cuda.synchronize()
+        codec.check_status()
+        label = f"config5 shards={n_shards} c={c} seg={seg}"
+        codec.canaries.check(label)
+        assert torch.equal(codec.weights_out[: cur.numel()], cur), f"{label}: round trip is not bit-exact"
+        assert torch.equal(codec.sender_cache, codec.receiver_cache), f"{label}: the two caches differ"
+        for ui in picks:
+            u = units[ui]
+            lo, nn, mo, co = int(u["weights_off"]), int(u["n_values"]), int(u["msg_off"]), int(u["cache_off"])
+            wp = prev[lo : lo + nn * 2].cpu().numpy().view(np.uint16)
+            wc = cur[lo : lo + nn * 2].cpu().numpy().view(np.uint16)
+            cache = ora.cache_init(wp, nn, 0)
+            m, wbytes, pay, cb = ora.encode(wc, cache, 0, block)
+            assert int(codec.wire_bytes[ui].item()) == wbytes, f"{label}: length of unit {ui} (N={nn})"
+            assert int(codec.changed_blocks[ui].item()) == cb, f"{label}: changed blocks of unit {ui} (N={nn})"
+            assert np.array_equal(codec.msg_send[mo : mo + wbytes].cpu().numpy(), m), f"{label}: message of unit {ui}"
+            assert np.array_equal(codec.msg_recv[mo : mo + wbytes].cpu().numpy(), m), f"{label}: transported {ui}"
+            assert np.array_equal(codec.sender_cache[co : co + nn].cpu().numpy(), cache), f"{label}: cache of {ui}"
+        q = int(codec.changed_blocks.sum().item()) / codec.n_blocks()
+        assert 0 < q <= 1
+        prev = cur
 
 
 @pytest.mark.parametrize("sizes", [[], [0], [0, 0, 0]])
@@ -378,7 +453,8 @@ def test_tightly_packed_layout_in_shuffled_order(rt, dtype, block):
                                         lambda n: ciera.message_capacity(n, code, block), align=16)
     rng = np.random.default_rng(12 + block)
     units = units[rng.permutation(len(units))]
-    codec = runtime.LayerCodec(units, NAME[dtype], block, wb, cb, mb, DEV)
+    codec = guard(runtime.LayerCodec(units, NAME[dtype], block, wb, cb, mb, DEV, slack=256))
+    assert codec.canaries.guarded_bytes() > 5 * 256  # the slack and the 16-byte alignment gaps
     table = OracleTable(codec.units, dtype, block, codec.cache_bytes, codec.msg_bytes)
     n = wb // (2 if dtype == 0 else 4)
     traj = [wl.as_bits(w) for w in wl.trajectory(n, NAME[dtype], 90 + block, 2, "adam")]
