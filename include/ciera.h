@@ -14,10 +14,13 @@
  * Conventions
  *   - Every function returns a ciera_status (0 = CIERA_OK, negative = error).  Nothing throws,
  *     nothing is printed, and no codec state lives in the library: caches, messages and scratch
- *     are the caller's buffers.
+ *     are the caller's buffers.  What the library does keep per process: the launch counter, the
+ *     thread's last CUDA error, and per device the grid sizes it has worked out for its kernels.
  *   - "dev" pointers are CUDA device pointers, "host" pointers are ordinary host pointers.
  *     The library never allocates device memory: the caller owns every device buffer and
- *     passes scratch space explicitly.  The only host allocation is the plan object.
+ *     passes scratch space explicitly.  The only host allocation is the plan object.  (One
+ *     exception, stated where it is declared: ciera_encode_noalloc works in a fixed device array
+ *     that is part of the library image, for callers that cannot supply scratch.)
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Device work is
  *     enqueued on it and the call returns without waiting, unless stated otherwise.
  *   - Errors found on the device (a wait that ran out, a message whose length contradicts its
@@ -130,9 +133,16 @@ CIERA_API uint64_t ciera_plan_total_values(const ciera_plan* plan);
 /* Bytes of device memory the table needs (>= 16), and the host image that has to be there. */
 CIERA_API size_t ciera_plan_device_bytes(const ciera_plan* plan);
 CIERA_API const void* ciera_plan_host_image(const ciera_plan* plan);
-/* Bytes of scratch one ciera_encode, ciera_transport or ciera_decode call needs (per-tile words
- * and a work counter). */
+/* Bytes of scratch ("workspace") that ciera_encode, ciera_transport and ciera_decode work in: 12 bytes per
+ * tile (a look-back status word for the sender, a count for the receiver) and a few counters. */
 CIERA_API size_t ciera_plan_workspace_bytes(const ciera_plan* plan);
+/* Zero-fills a workspace of ciera_plan_workspace_bytes(plan) bytes (16-byte aligned) on `stream`.  The sender
+ * calls (ciera_encode, ciera_encode_hashed, ciera_roundtrip_host) expect their part of the workspace all zero
+ * when they start and leave it all zero when they have finished, so that no launch is spent on clearing it
+ * before every call: initialise a workspace once after allocating it, and again after a call whose device
+ * status word came back with an error (a kernel that gave up leaves the workspace in an unspecified state).
+ * A plain cudaMemset of the whole workspace does the same. */
+CIERA_API int ciera_workspace_init(const ciera_plan* plan, void* workspace_dev, void* stream);
 
 /* Copies the table into caller-owned device memory `plan_dev` (>= ciera_plan_device_bytes,
  * 16-byte aligned) on `stream`, waits for the copy, and remembers the pointer.  The memory must
@@ -160,11 +170,12 @@ CIERA_API int ciera_cache_update(const ciera_plan* plan, void* cache_dev, const 
  *   wire_bytes_dev      out  [n_units] bytes that have to travel (payload offset + payload bytes;
  *                            0 for an empty unit)
  *   changed_blocks_dev  out  [n_units] number of set bitmap bits
- *   workspace_dev       scratch of ciera_plan_workspace_bytes(), 16-byte aligned (look-back status
- *                            words and the counter units are handed out from); cleared by the call
- *                            itself; must not be shared by calls that can overlap on the GPU
+ *   workspace_dev       i/o  scratch of ciera_plan_workspace_bytes(), 16-byte aligned (look-back status
+ *                            words, the counter that runs of tiles are handed out from); all zero on
+ *                            entry -- see ciera_workspace_init -- and handed back all zero; must not
+ *                            be shared by calls that can overlap on the GPU
  *   status_dev          i/o  device error word (may be NULL)
- * One kernel launch (plus one memset of the scratch) for the whole table.
+ * One kernel launch for the whole table, nothing else.
  */
 CIERA_API int ciera_encode(const ciera_plan* plan, const void* weights_dev, void* sender_cache_dev, void* messages_dev,
                  uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* workspace_dev,
@@ -214,7 +225,7 @@ CIERA_API int ciera_encode_noalloc(const ciera_plan* plan, const void* weights_d
  * Blocks of 16 values and more only (CIERA_ERR_UNSUPPORTED otherwise). */
 
 /* Bytes of a HashCache for the whole plan (16 per block; units in table order), the offset of a
- * unit's first block in it, and the scratch ciera_encode_hashed needs (8 bytes per tile + 16). */
+ * unit's first block in it, and the scratch ciera_encode_hashed needs (= ciera_plan_workspace_bytes). */
 CIERA_API size_t ciera_plan_hash_cache_bytes(const ciera_plan* plan);
 CIERA_API size_t ciera_plan_unit_hash_offset(const ciera_plan* plan, uint32_t unit);
 CIERA_API size_t ciera_plan_hashed_workspace_bytes(const ciera_plan* plan);
@@ -226,7 +237,8 @@ CIERA_API int ciera_hash_cache_init(const ciera_plan* plan, void* hash_cache_dev
 
 /* Sender step with HashCache.  Arguments, launch (one persistent kernel) and error behaviour as
  * for ciera_encode, with hash_cache_dev (in/out, ciera_plan_hash_cache_bytes) in place of the
- * exponent cache and a scratch of ciera_plan_hashed_workspace_bytes (cleared by the call). */
+ * exponent cache and a scratch of ciera_plan_hashed_workspace_bytes (all zero on entry and on return,
+ * as for ciera_encode). */
 CIERA_API int ciera_encode_hashed(const ciera_plan* plan, const void* weights_dev, void* hash_cache_dev,
                                   void* messages_dev, uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev,
                                   void* workspace_dev, int32_t* status_dev, void* stream);
@@ -236,8 +248,8 @@ CIERA_API int ciera_encode_hashed(const ciera_plan* plan, const void* weights_de
 /* Copies, for every unit, the first wire_bytes_dev[u] bytes of its slot from `src_messages_dev`
  * to the same slot of `dst_messages_dev` (one kernel; the lengths are read on the device).  This
  * stands where the Allgather of the messages would be.  `workspace_dev`: scratch of
- * ciera_plan_workspace_bytes() (holds the counter tiles are handed out from; cleared by the call;
- * not to be shared by calls that can overlap on the GPU).  `status_dev`: device int32 or NULL; the
+ * ciera_plan_workspace_bytes() (holds the counter tiles are handed out from, which the call sets to zero
+ * itself; not to be shared by calls that can overlap on the GPU).  `status_dev`: device int32 or NULL; the
  * kernel's waits on its own copies are bounded and raise CIERA_ERR_TIMEOUT there. */
 CIERA_API int ciera_transport(const ciera_plan* plan, const void* src_messages_dev, void* dst_messages_dev,
                     const uint64_t* wire_bytes_dev, void* workspace_dev, int32_t* status_dev, void* stream);
@@ -254,9 +266,10 @@ CIERA_API int ciera_transport(const ciera_plan* plan, const void* src_messages_d
  *                            whose bitmap implies a different length raises CIERA_ERR_CORRUPT in
  *                            status_dev (its output is then unspecified)
  *   workspace_dev       scratch of ciera_plan_workspace_bytes(), 16-byte aligned: the counter tiles
- *                            are handed out from (cleared by the call itself) and, when some unit has
+ *                            are handed out from (set to zero by the call itself) and, when some unit has
  *                            more than 4096 blocks, the per-tile counts of a small prefix kernel that
- *                            runs first.  Must not be shared by calls that can overlap on the GPU.
+ *                            runs first; the sender's part of the workspace is left alone.  Must not be
+ *                            shared by calls that can overlap on the GPU.
  */
 CIERA_API int ciera_decode(const ciera_plan* plan, const void* messages_dev, void* receiver_cache_dev,
                  void* weights_out_dev, const uint64_t* wire_bytes_dev, void* workspace_dev, int32_t* status_dev,
@@ -265,7 +278,8 @@ CIERA_API int ciera_decode(const ciera_plan* plan, const void* messages_dev, voi
 /* ---- whole step with host buffers ---------------------------------------------------------- */
 
 /* Device buffers one ciera_roundtrip_host call works in; all caller-owned, sized as for the
- * separate calls above (weights_dev / weights_out_dev: weights_bytes each). */
+ * separate calls above (weights_dev / weights_out_dev: weights_bytes each; workspace_dev initialised
+ * with ciera_workspace_init as for ciera_encode). */
 typedef struct ciera_device_buffers {
     void* weights_dev;
     void* sender_cache_dev;

@@ -67,6 +67,7 @@ _SIGS = {
     "ciera_plan_device_bytes": ([_vp], _sz),
     "ciera_plan_host_image": ([_vp], _vp),
     "ciera_plan_workspace_bytes": ([_vp], _sz),
+    "ciera_workspace_init": ([_vp, _vp, _vp], _i32),
     "ciera_plan_bind": ([_vp, _vp, _sz, _vp], _i32),
     "ciera_cache_init": ([_vp, _vp, _vp, _vp], _i32),
     "ciera_cache_update": ([_vp, _vp, _vp, _vp], _i32),
@@ -197,7 +198,10 @@ class Plan:
         return self
 
     def new_workspace(self) -> torch.Tensor:
-        return torch.empty(self.workspace_bytes, dtype=torch.uint8, device=self.table.device)
+        """A fresh workspace, zero-filled through ``ciera_workspace_init`` as the sender calls expect it."""
+        ws = torch.empty(max(self.workspace_bytes, 16), dtype=torch.uint8, device=self.table.device)
+        workspace_init(self, ws)
+        return ws
 
     @property
     def handle(self):
@@ -211,6 +215,12 @@ class Plan:
 
 
 # ------------------------------------------------------------------------------ device calls
+
+
+def workspace_init(plan: "Plan", workspace: torch.Tensor, stream=None) -> None:
+    """Zero-fills a workspace: once after allocating it, and again after a call that reported a device-side error."""
+    with torch.cuda.device(workspace.device):
+        _check("ciera_workspace_init", _lib.ciera_workspace_init(plan.handle, _ptr(workspace), _stream(stream)))
 
 
 def cache_init(plan: Plan, cache: torch.Tensor, weights: Optional[torch.Tensor], stream=None) -> None:

@@ -867,7 +867,7 @@ static int decode_grid_limit(int* out) {
 
 template <int DT, bool FINE>
 static int launch_decode(const ciera_plan* p, const void* messages_dev, void* receiver_cache_dev, void* weights_out_dev,
-                         const uint64_t* wire_bytes_dev, void* workspace_dev, unsigned int* ticket, int32_t* status_dev,
+                         const uint64_t* wire_bytes_dev, const uint32_t* ws_prefix, unsigned int* ticket, int32_t* status_dev,
                          cudaStream_t s) {
     int limit = 0;
     const int rc = decode_grid_limit<DT, FINE>(&limit);
@@ -876,7 +876,7 @@ static int launch_decode(const ciera_plan* p, const void* messages_dev, void* re
     const uint32_t grid = nt < (uint32_t)limit ? nt : (uint32_t)limit;
     decode_kernel<DT, FINE><<<grid, kDecodeThreads, decode_smem_bytes<DT, FINE>(), s>>>(
         p->tiles_dev, nt, p->log2b, (const uint8_t*)messages_dev, (uint8_t*)receiver_cache_dev, (uint8_t*)weights_out_dev,
-        (const unsigned long long*)wire_bytes_dev, (const uint32_t*)workspace_dev, ticket, status_dev);
+        (const unsigned long long*)wire_bytes_dev, ws_prefix, ticket, status_dev);
     count_launch();
     return check_launch();
 }
@@ -899,34 +899,35 @@ extern "C" int ciera_decode(const ciera_plan* p, const void* messages_dev, void*
         misaligned16(workspace_dev))
         return CIERA_ERR_MISALIGNED;
     cudaStream_t s = (cudaStream_t)stream;
-    // scratch = per-tile counts for long units (4 bytes per tile), then, past 8 bytes per tile, the
-    // tile counter, which starts at zero
-    unsigned int* ticket = (unsigned int*)((unsigned long long*)workspace_dev + nt);
+    // scratch: the tile counter, which starts at zero, behind the sender's status words (left alone), and
+    // behind it the per-tile counts of the units that go through the prefix kernel
+    unsigned int* ticket = (unsigned int*)((uint8_t*)workspace_dev + workspace_ticket_offset(nt));
+    uint32_t* ws_prefix = (uint32_t*)((uint8_t*)workspace_dev + workspace_prefix_offset(nt));
     cudaError_t me = cudaMemsetAsync(ticket, 0, 16, s);
     if (me != cudaSuccess) return record_cuda_error(me);
     const uint32_t n_long = (uint32_t)p->long_units.size();
     if (n_long) {
         if (is_fine(p->log2b))
             decode_prefix_fine_kernel<<<n_long, 256, 0, s>>>(p->tiles_dev, p->long_units_dev, p->log2b,
-                                                             (const uint8_t*)messages_dev, (uint32_t*)workspace_dev);
+                                                             (const uint8_t*)messages_dev, ws_prefix);
         else
             decode_prefix_kernel<<<n_long, 256, 0, s>>>(p->tiles_dev, p->long_units_dev, p->log2b,
-                                                        (const uint8_t*)messages_dev, (uint32_t*)workspace_dev);
+                                                        (const uint8_t*)messages_dev, ws_prefix);
         count_launch();
         int rc = check_launch();
         if (rc) return rc;
     }
     if (p->dtype == CIERA_FP16)
         return launch_decode<CIERA_FP16, false>(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,
-                                                workspace_dev, ticket, status_dev, s);
+                                                ws_prefix, ticket, status_dev, s);
     const bool fine = is_fine(p->log2b);
     if (p->dtype == CIERA_BF16)
         return fine ? launch_decode<CIERA_BF16, true>(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,
-                                                      workspace_dev, ticket, status_dev, s)
+                                                      ws_prefix, ticket, status_dev, s)
                     : launch_decode<CIERA_BF16, false>(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,
-                                                       workspace_dev, ticket, status_dev, s);
+                                                       ws_prefix, ticket, status_dev, s);
     return fine ? launch_decode<CIERA_FP32, true>(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,
-                                                  workspace_dev, ticket, status_dev, s)
+                                                  ws_prefix, ticket, status_dev, s)
                 : launch_decode<CIERA_FP32, false>(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,
-                                                   workspace_dev, ticket, status_dev, s);
+                                                   ws_prefix, ticket, status_dev, s);
 }

@@ -203,12 +203,20 @@ constexpr uint32_t kNoTile = 0xffffffffu;
 constexpr uint32_t kSeqTile = 1u, kSeqRunStart = 2u, kSeqRunEnd = 4u;
 
 // The sequence of tiles of one thread block (see the head of this file); used by the producer.
+// Runs of the short units: block b starts with runs b and b + G (no round trip to the counter stands between
+// the start of the kernel and the first loads); every run taken is paid for with one draw from the counter, so
+// the counter is drawn from exactly n_runs times in a launch, and the thread that makes the last draw puts it
+// back to zero for the next launch.  The walk keeps two runs in hand besides the current one: the number of
+// the run after next (its draw is on its way) and the table entry of the next run (its load is on its way), so
+// that at the start of a run neither the counter nor the table is waited for.
 struct TileWalk {
     const uint2* seq_runs;
     unsigned int* run_ticket;
     uint32_t n_tiles, n_runs, G;
     uint32_t tile, end;      // current run: next tile, one past its last tile
-    uint32_t next_run;       // the run drawn ahead (its number arrives while the current one is worked on)
+    uint2 next_range;        // the next run's tiles (valid if next_run < n_runs)
+    uint32_t next_run;       // number of the next run
+    uint32_t after_run;      // number of the run after that
     uint32_t spread_tile;    // next spread tile of this block
     bool spread;
 
@@ -216,7 +224,15 @@ struct TileWalk {
                         uint32_t grid, uint32_t block)
         : seq_runs(runs), run_ticket(ticket), n_tiles(nt), n_runs(nruns), G(grid), tile(0), end(0), spread(true) {
         spread_tile = spread_first + block;  // tiles of longer units start after the short units' tiles
-        next_run = nruns ? atomicAdd(ticket, 1u) : kNoTile;
+        next_run = block;
+        after_run = block + grid;
+        next_range = make_uint2(0u, 0u);
+        if (next_run < n_runs) next_range = __ldg(seq_runs + next_run);
+    }
+    __device__ uint32_t draw() {
+        const uint32_t d = atomicAdd(run_ticket, 1u);
+        if (d + 1u == n_runs) atomicExch(run_ticket, 0u);  // that was the launch's last draw
+        return d + 2u * G;
     }
     // next tile, or kNoTile; `seq` gets the kSeq* bits of the tile
     __device__ uint32_t next(uint32_t& seq) {
@@ -231,12 +247,12 @@ struct TileWalk {
         }
         seq = kSeqTile;
         while (tile == end) {
-            const uint32_t r = next_run;
-            if (r >= n_runs) return kNoTile;
-            next_run = atomicAdd(run_ticket, 1u);
-            const uint2 run = __ldg(seq_runs + r);
-            tile = run.x;
-            end = run.y;
+            if (next_run >= n_runs) return kNoTile;
+            tile = next_range.x;
+            end = next_range.y;
+            next_run = after_run;
+            if (next_run < n_runs) next_range = __ldg(seq_runs + next_run);
+            after_run = draw();
             seq |= kSeqRunStart;
         }
         if (tile + 1u == end) seq |= kSeqRunEnd;
@@ -593,7 +609,8 @@ __global__ void __launch_bounds__(kEncodeThreads, 2)
 encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint2* __restrict__ seq_runs, uint32_t n_runs,
               uint32_t spread_first, uint32_t log2b, const uint8_t* __restrict__ weights, uint8_t* cache, uint8_t* msgs,
               unsigned long long* wire_bytes, uint32_t* changed_blocks, unsigned long long* tile_status,
-              unsigned int* unit_ticket, int32_t* status, const unsigned long long* __restrict__ tile_hash) {
+              unsigned int* unit_ticket, unsigned int* blocks_done, int32_t* status,
+              const unsigned long long* __restrict__ tile_hash) {
     static_assert(!(HASH && (FINE || DT == CIERA_FP16)), "HashCache: bf16 and fp32, blocks of 16 values and more");
     using P = Piece<DT>;
     constexpr int VB = Traits<DT>::kValueBytes;
@@ -673,7 +690,7 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint2*
                 ctl->tile_idx[k % kDescRing] = tile;
                 if (tile == kNoTile) {  // end marker
                     mbar_arrive(&ctl->full_w[sw]);
-                    mbar_arrive(&ctl->full_e[se]);
+                    if (HASH) mbar_arrive(&ctl->full_e[se]);
                     if (++markers == (uint32_t)kResolvers) break;
                     continue;
                 }
@@ -703,14 +720,13 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint2*
                     mbar_arrive_expect_tx(&ctl->full_e[se], nblk * 16u);
                     bulk_load(ring_h + (size_t)se * kHStage, cache + hb * 16ull, nblk * 16u, &ctl->full_e[se]);
                 } else if (left >= (uint64_t)kTileValues) {
-                    mbar_arrive_expect_tx(&ctl->full_w[sw], kWBytes);
+                    // both copies of the tile complete on the one barrier the consumers wait for
+                    mbar_arrive_expect_tx(&ctl->full_w[sw], kWBytes + kEBytes);
                     bulk_load(ring_w + (size_t)sw * kWBytes, weights + td.w_off, kWBytes, &ctl->full_w[sw]);
-                    mbar_arrive_expect_tx(&ctl->full_e[se], kEBytes);
-                    bulk_load(ring_e + (size_t)se * kEBytes, cache + td.c_off, kEBytes, &ctl->full_e[se]);
+                    bulk_load(ring_e + (size_t)se * kEBytes, cache + td.c_off, kEBytes, &ctl->full_w[sw]);
                 } else {
                     // short tile: consumers read global memory themselves
                     mbar_arrive(&ctl->full_w[sw]);
-                    mbar_arrive(&ctl->full_e[se]);
                 }
                 ctl->issued = k + 1;
             }
@@ -750,8 +766,11 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint2*
                 uint64_t excl = run_incl;
                 if (td.tile_in_unit == 0)
                     excl = 0;
-                else if (seq_bits & kSeqRunStart)
+                else if (seq_bits & kSeqRunStart) {
                     excl = wait_status(tile_status + tile - 1, status) & kValueMask;
+                    __syncwarp();
+                    if (lane == 0) st_status(tile_status + tile - 1, 0ull);  // its one reader leaves the word empty again
+                }
                 run_incl = excl + agg;
                 if ((seq_bits & kSeqRunEnd) && td.tile_in_unit != td.n_tiles_unit - 1u && lane == 0)
                     st_status(tile_status + tile, kFlagPrefix | run_incl);
@@ -795,12 +814,14 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint2*
         uint32_t k = 0;
         // stage and phase of slot k in the two rings, and of slot k - kDefer in the exponent ring, kept
         // as running counters (the ring depths are no powers of two)
-        uint32_t sw = 0, pw = 0, se = 0, pe = 0, je = 0, pj = 0;
+        uint32_t sw = 0, pw = 0, se = 0, je = 0, pj = 0;
         // HASH: the lanes of a warp that share a block (a power of two, at most the warp) add up their terms
         const uint32_t hash_lanes_l2 = min(5u, log2b - (uint32_t)P::kLog2Values);
         for (;; ++k) {
+            // (the producer starts the loads of slot k only once both of its stages are free, and the cached
+            // exponents land on the same barrier as the weights; with HashCache the cached hashes, which only
+            // the aggregator reads, land on full_e)
             if (!mbar_wait(&ctl->full_w[sw], pw, abort, status)) break;
-            if (!mbar_wait(&ctl->full_e[se], pe, abort, status)) break;
             if (tid == 0) ctl->seen = k + 1;
             const bool marker = ctl->tile_idx[k % kDescRing] == kNoTile;
             if (marker) {
@@ -875,10 +896,7 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint2*
                 sw = 0;
                 pw ^= 1u;
             }
-            if (++se == (uint32_t)SE) {
-                se = 0;
-                pe ^= 1u;
-            }
+            if (++se == (uint32_t)SE) se = 0;
         }
         // tiles whose changed exponents are still to be sent (when kDefer > kResolvers)
         if (!*abort && k_end != kNoTile) {
@@ -899,9 +917,25 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint2*
         for (uint32_t k = ctl->seen; k < ctl->issued; ++k) {
             for (uint32_t i = 0; i < kMaxBarrierPolls; ++i)
                 if (mbar_try_wait(&ctl->full_w[k % SW], (k / SW) & 1u)) break;
-            for (uint32_t i = 0; i < kMaxBarrierPolls; ++i)
-                if (mbar_try_wait(&ctl->full_e[k % SE], (k / SE) & 1u)) break;
+            if (HASH) {
+                for (uint32_t i = 0; i < kMaxBarrierPolls; ++i)
+                    if (mbar_try_wait(&ctl->full_e[k % SE], (k / SE) & 1u)) break;
+            }
         }
+    }
+    // The scratch is handed back the way it was found, all zero: the hand-off words of the runs were emptied by
+    // their readers, the run counter by its last draw; the status words of the spread tiles (read by any number
+    // of later tiles) and the counter of finished blocks are emptied here by the block that finishes last.
+    __shared__ unsigned int s_last;
+    if (tid == 0) {
+        __threadfence();
+        s_last = atomicAdd(blocks_done, 1u) + 1u == gridDim.x ? 1u : 0u;
+    }
+    __syncthreads();
+    if (s_last) {
+        __threadfence();
+        for (uint32_t t = spread_first + tid; t < n_tiles; t += kEncodeThreads) st_status(tile_status + t, 0ull);
+        if (tid == 0) atomicExch(blocks_done, 0u);
     }
 }
 
@@ -943,7 +977,8 @@ static int encode_grid_limit(uint32_t log2b, int* out) {
     return CIERA_OK;
 }
 
-// `scratch`: one status word per tile, then the unit counter; all zero at kernel start.
+// `scratch`: one status word per tile, then the run counter and the counter of finished blocks; all zero when
+// the kernel starts, and all zero again when it has finished without a device-side error.
 template <int DT, bool FINE, int HASH = 0>
 static int launch_encode(const ciera_plan* p, const void* weights_dev, void* sender_cache_dev, void* messages_dev,
                          uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* scratch, int32_t* status_dev,
@@ -963,7 +998,8 @@ static int launch_encode(const ciera_plan* p, const void* weights_dev, void* sen
     uint8_t* m = (uint8_t*)messages_dev;
     unsigned long long* wb = (unsigned long long*)wire_bytes_dev;
     unsigned long long* ts = (unsigned long long*)scratch;
-    unsigned int* ticket = (unsigned int*)(ts + nt);
+    unsigned int* ticket = (unsigned int*)((uint8_t*)scratch + workspace_sender_counters_offset(nt));
+    unsigned int* done = ticket + 1;
     const unsigned long long* tile_hash = HASH ? p->tile_hash_dev : nullptr;
     const size_t smem = encode_smem_bytes<DT, FINE, HASH>(log2b);
     const bool has_spread = p->seq_first.back() < nt;  // tiles of longer units: look-back between blocks
@@ -972,12 +1008,13 @@ static int launch_encode(const ciera_plan* p, const void* weights_dev, void* sen
         // cooperative launch: the runtime starts the grid only when all of its blocks fit on the
         // GPU together, which is what the look-back between blocks relies on
         void* args[] = {&tiles, &nt, &seq_runs, &n_runs, &spread_first, &log2b, &w, &c, &m, &wb, &changed_blocks_dev, &ts,
-                        &ticket, &status_dev, &tile_hash};
+                        &ticket, &done, &status_dev, &tile_hash};
         e = cudaLaunchCooperativeKernel((const void*)encode_kernel<DT, FINE, HASH>, dim3(grid), dim3(kEncodeThreads), args,
                                         smem, s);
     } else {
         encode_kernel<DT, FINE, HASH><<<grid, kEncodeThreads, smem, s>>>(
-            tiles, nt, seq_runs, n_runs, spread_first, log2b, w, c, m, wb, changed_blocks_dev, ts, ticket, status_dev, tile_hash);
+            tiles, nt, seq_runs, n_runs, spread_first, log2b, w, c, m, wb, changed_blocks_dev, ts, ticket, done, status_dev,
+            tile_hash);
         e = cudaGetLastError();
     }
     if (e != cudaSuccess) return record_cuda_error(e);
@@ -1047,9 +1084,8 @@ extern "C" int ciera_encode(const ciera_plan* p, const void* weights_dev, void* 
     if (misaligned16(weights_dev) || misaligned16(sender_cache_dev) || misaligned16(messages_dev) ||
         misaligned16(workspace_dev) || ((uintptr_t)wire_bytes_dev & 7u) || ((uintptr_t)changed_blocks_dev & 3u))
         return CIERA_ERR_MISALIGNED;
-    // scratch = one look-back status word per tile, then the unit counter; all of it starts at zero
-    e = cudaMemsetAsync(workspace_dev, 0, sizeof(unsigned long long) * nt + 16, s);
-    if (e != cudaSuccess) return record_cuda_error(e);
+    // scratch = one look-back status word per tile, then two counters: all zero on entry (ciera_workspace_init,
+    // or left so by the previous call), and the kernel hands it back all zero
     return launch_encode_any(p, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev, changed_blocks_dev,
                              workspace_dev, status_dev, s);
 }

@@ -128,9 +128,7 @@ extern "C" int ciera_encode_hashed(const ciera_plan* p, const void* weights_dev,
     if (misaligned16(weights_dev) || misaligned16(hash_cache_dev) || misaligned16(messages_dev) ||
         misaligned16(workspace_dev) || ((uintptr_t)wire_bytes_dev & 7u) || ((uintptr_t)changed_blocks_dev & 3u))
         return CIERA_ERR_MISALIGNED;
-    // scratch = one look-back status word per tile, then the unit counter; all of it starts at zero
-    e = cudaMemsetAsync(workspace_dev, 0, sizeof(unsigned long long) * nt + 16, s);
-    if (e != cudaSuccess) return record_cuda_error(e);
+    // scratch as for ciera_encode: all zero on entry (ciera_workspace_init, or left so by the previous call)
     return launch_encode_hashed(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev, changed_blocks_dev,
                                 workspace_dev, status_dev, s);
 }

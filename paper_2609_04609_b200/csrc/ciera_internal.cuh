@@ -108,6 +108,20 @@ __host__ __device__ inline uint64_t payload_offset_of(uint64_t n, int dtype, uin
 // blocks every unit of more than one tile goes through the prefix kernel.
 constexpr uint32_t kDecodeDirectBlocks = 4096;
 
+// Layout of the scratch ("workspace") of a plan with nt tiles, shared by the sender, transport and receiver calls:
+//   [0, 8 nt)             one 64-bit look-back status word per tile                     (sender)
+//   [8 nt, + 16)          the sender's run counter and its counter of finished blocks   (sender)
+//   [8 nt + 16, + 16)     the counter that transport and receiver hand their tiles out from
+//   [8 nt + 32, + 4 nt)   changed blocks before each tile of the units that go through the receiver's prefix kernel
+// The sender needs its two parts all zero when it starts and leaves them so; transport and receiver set their
+// counter to zero themselves at the start of every call and touch nothing of the sender's.
+__host__ __device__ inline size_t workspace_sender_counters_offset(size_t nt) { return nt * sizeof(unsigned long long); }
+__host__ __device__ inline size_t workspace_ticket_offset(size_t nt) { return workspace_sender_counters_offset(nt) + 16; }
+__host__ __device__ inline size_t workspace_prefix_offset(size_t nt) { return workspace_ticket_offset(nt) + 16; }
+__host__ __device__ inline size_t workspace_total_bytes(size_t nt) {
+    return (workspace_prefix_offset(nt) + nt * sizeof(uint32_t) + 15) / 16 * 16;
+}
+
 // The tile table lists the tiles of "short" units (up to this many tiles) first, longest units
 // first, then the tiles of the longer units.  The encode kernel lets one thread block work through
 // a short unit tile after tile (the tile's place in the payload is then a running sum inside the

@@ -336,8 +336,8 @@ extern "C" int ciera_transport(const ciera_plan* p, const void* src_messages_dev
     if (!src_messages_dev || !dst_messages_dev || !wire_bytes_dev || !workspace_dev) return CIERA_ERR_INVALID_ARG;
     if (misaligned16(src_messages_dev) || misaligned16(dst_messages_dev) || misaligned16(workspace_dev))
         return CIERA_ERR_MISALIGNED;
-    // the tile counter sits past the per-tile words of the scratch and starts at zero
-    unsigned int* ticket = (unsigned int*)((unsigned long long*)workspace_dev + nt);
+    // the tile counter (see the layout of the scratch in ciera_internal.cuh) starts at zero
+    unsigned int* ticket = (unsigned int*)((uint8_t*)workspace_dev + workspace_ticket_offset(nt));
     cudaError_t me = cudaMemsetAsync(ticket, 0, 16, (cudaStream_t)stream);
     if (me != cudaSuccess) return record_cuda_error(me);
     int limit = 0;

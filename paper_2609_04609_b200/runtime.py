@@ -69,8 +69,7 @@ class LayerCodec:
         """Allocates (once) and fills the sender's HashCache and the scratch of the hashed encode."""
         if getattr(self, "hash_cache", None) is None:
             self.hash_cache = torch.zeros(max(self.plan.hash_cache_bytes, 16), dtype=torch.uint8, device=self.device)
-            self.hashed_workspace = torch.empty(max(self.plan.hashed_workspace_bytes, 16), dtype=torch.uint8,
-                                                device=self.device)
+            self.hashed_workspace = self.plan.new_workspace()
         ciera.hash_cache_init(self.plan, self.hash_cache, weights, stream)
 
     def encode_hashed(self, weights: torch.Tensor, stream=None) -> None:
@@ -132,6 +131,10 @@ class LayerCodec:
     def check_status(self) -> None:
         s = int(self.status.item())
         if s != 0:
+            # a kernel that gave up leaves its scratch in an unspecified state: make it usable again
+            ciera.workspace_init(self.plan, self.workspace)
+            if getattr(self, "hashed_workspace", None) is not None:
+                ciera.workspace_init(self.plan, self.hashed_workspace)
             raise ciera.CieraError("device status", s)
 
     # -- accounting -------------------------------------------------------------------------------
