@@ -162,7 +162,8 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
     // trip (the run's place in the table, the status word the run before it left), so runs should be few; but the
     // launch ends with the blocks working on the last runs, and the shorter those are, the closer together the
     // blocks finish.  Measured on one OLMoE-shaped layer (units of 16 tiles, 0.2848 ms with four runs of 4):
-    // 8 + 4 + 4 tiles 0.2836 ms, 12 + 4 tiles 0.2823 ms; ending on runs of 2 + 1 + 1 tiles instead 0.2932 ms.
+    // 8 + 4 + 4 tiles 0.2836 ms, 12 + 4 tiles 0.2823 ms (14 + 2: 0.2840, 15 + 1: 0.2857, 8 + 8: 0.2871); ending on runs of
+    // 2 + 1 + 1 tiles instead 0.2932 ms.
     // (With 16 to 128 values per block a tile has 64 to 512 blocks and the aggregator warp, which also waits
     // for the status word at the start of a run, has the least time to spare: there whole units measured 2-3 %
     // faster than runs, so a run is the whole unit.)
