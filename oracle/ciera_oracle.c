@@ -6,18 +6,18 @@
  * benchmark's cpu_baseline / reference legs may call it.  It shares no code, header,
  * table or constant with the CUDA library and neither side includes the other.
  *
- * What it follows (all from the paper):
- *   - Section 3.1 "Exponent Reuse based Compression": split every value into exponent
- *     bits and sign-plus-mantissa bits; a block's exponents are "unchanged" only if
- *     they equal the previous ones; send a bitmap (one bit per block), the
- *     sign-plus-mantissa of ALL values, and the exponents of the changed blocks.
- *   - Algorithm 1 (appendix): sender loop over blocks k = 1..S_b, bitmap[k] <- 1 and
- *     cache update when block k changed, payload = exponents of blocks with
- *     bitmap[k] = 1 in block order; receiver: walk the bitmap, ExpCache[i,k] <-
- *     newExp[j], j++ for set bits, then Merge(ExpCache, mant).
- *   - Section 3.2: S = N*b/8, S_e exponent bytes, S_{s+m} = S - S_e,
- *     S_b = ceil(N/B), S_bm = ceil(S_b/8), expected payload S_{s+m}+S_bm+q*S_e, and
- *     the gain g = Comm(S) - (Comm(S_{s+m}+S_bm+q S_e) + T_hash + T_cmp + T_decmp).
+ * What it states (the definitions are the paper's, the wording and structure are this file's):
+ *   - Section 3.1: a value is cut into its exponent field and the rest (sign and mantissa).
+ *     Blocks of B consecutive values are compared with what was last sent: a block counts as
+ *     changed when any of its exponents differs.  A message holds one bit per block, the
+ *     sign-and-mantissa part of every value, and the exponent fields of the changed blocks only.
+ *   - Algorithm 1: the sender marks changed blocks, remembers their new exponents, and strings the
+ *     exponents of the marked blocks together in ascending block order; the receiver goes through
+ *     the marks in the same order, takes one block of exponents off the front of the payload for
+ *     each mark to overwrite its cached copy, and rebuilds every value from cached exponent plus
+ *     received sign-and-mantissa.
+ *   - Section 3.2: the sizes S, S_e, S_{s+m}, S_b, S_bm, the expected message size, and the gain
+ *     of compressing a shard (ora_gain).
  *
  * Readings taken where the paper is silent (each is listed in the design notes):
  *   - Change detection is the exact predicate the paper's 128-bit block hash
@@ -32,8 +32,8 @@
  *
  * Pins: tests/test_oracle_*.py (IEEE field definition through frexp, exhaustive
  * bf16 x cache sweep, hand-worked fixtures, byte formula, closed forms (1-c)^B,
- * special cases, hand-computed gains).  ANS coding is not built ("parity unpinned", absent
- * here).  The hash-based sender (ora_encode_hashed) is pinned as a change detector (published
+ * special cases, hand-computed gains).  The entropy stage for the changed exponents has an oracle of
+ * its own (rans_oracle.c).  The hash-based sender (ora_encode_hashed) is pinned as a change detector (published
  * SplitMix64 streams, equality with the exact-comparison sender, certain detection of single-word
  * changes); the 128-bit hash VALUES follow a construction the paper does not print, so for them:
  * parity unpinned.
@@ -133,7 +133,7 @@ static void store_bits(void* w, uint64_t j, int dtype, uint32_t bits) {
     }
 }
 
-/* SplitExpMant (Algorithm 1, first sender line): one value -> (exp, sm). */
+/* One value -> exponent field and sign-plus-mantissa (the sender's first step in Algorithm 1). */
 static void split_value(uint32_t bits, int dtype, uint8_t* exp, uint32_t* sm) {
     int b = ora_b(dtype), m = ora_m(dtype);
     uint32_t sign = (bits >> (b - 1)) & 1u;
@@ -143,7 +143,7 @@ static void split_value(uint32_t bits, int dtype, uint8_t* exp, uint32_t* sm) {
     *sm = (sign << (m - 1)) | mant;
 }
 
-/* Merge (Algorithm 1, last receiver line): (exp, sm) -> one value. */
+/* Exponent field and sign-plus-mantissa -> one value (the receiver's last step in Algorithm 1). */
 static uint32_t merge_value(uint8_t exp, uint32_t sm, int dtype) {
     int b = ora_b(dtype), m = ora_m(dtype);
     uint32_t sign = (sm >> (m - 1)) & 1u;
@@ -194,7 +194,7 @@ int ora_encode(const void* w, uint8_t* cache_s, uint64_t n, int dtype, uint32_t 
     uint64_t sm_off = ora_sm_offset(n, block);
     uint64_t pay_off = ora_payload_offset(n, dtype, block);
 
-    /* (exp, mant) <- SplitExpMant(shard) */
+    /* every value cut into exponent field and sign-plus-mantissa */
     uint8_t* exp = (uint8_t*)malloc(n);
     uint32_t* sm = (uint32_t*)malloc(n * sizeof(uint32_t));
     if (!exp || !sm) {
@@ -204,10 +204,10 @@ int ora_encode(const void* w, uint8_t* cache_s, uint64_t n, int dtype, uint32_t 
     }
     ora_split(w, n, dtype, exp, sm);
 
-    /* bitmap <- [0]^{S_b}; payload <- empty.  Pads are zero as well. */
+    /* no block marked yet, nothing in the payload; the pads are zero as well */
     memset(msg, 0, pay_off);
 
-    /* for k = 1..S_b: changed iff some exponent differs from the cached one. */
+    /* a block is marked when one of its exponents is not the cached one; its cached copy is then replaced */
     for (uint64_t k = 0; k < nb; ++k) {
         uint64_t lo = k * block;
         uint64_t hi = lo + block < n ? lo + block : n;
@@ -223,7 +223,7 @@ int ora_encode(const void* w, uint8_t* cache_s, uint64_t n, int dtype, uint32_t 
     /* sign-plus-mantissa of all values. */
     for (uint64_t j = 0; j < n; ++j) put_bits(msg + sm_off, j * (uint64_t)m, m, sm[j]);
 
-    /* payload <- { exp[k] | bitmap[k] = 1 } in block order. */
+    /* the exponents of the marked blocks, ascending */
     uint64_t plen = 0;
     uint32_t nchg = 0;
     for (uint64_t k = 0; k < nb; ++k) {
@@ -253,16 +253,22 @@ int ora_encode(const void* w, uint8_t* cache_s, uint64_t n, int dtype, uint32_t 
  * SplitMix64 hashes.  The construction used here (a reading; the paper prints none):
  *   mix(z)  = the SplitMix64 output function: z ^= z >> 30; z *= 0xBF58476D1CE4E5B9;
  *             z ^= z >> 27; z *= 0x94D049BB133111EB; z ^= z >> 31
- *   gamma   = 0x9E3779B97F4A7C15 (the SplitMix64 increment)
  *   a block of L exponent bytes is read as m = ceil(L / 8) little-endian 64-bit words x_0..x_{m-1}
  *   (the last one zero-padded);
- *   H_s     = mix( L + sum_j mix(s + (j + 1) * gamma + x_j) )      (all arithmetic mod 2^64)
- *   Hash128 = (H_s1, H_s2), s1 = 0, s2 = 0x6A09E667F3BCC908.
- * mix(s + (j + 1) * gamma) is the j-th output of the SplitMix64 generator seeded with s, so each
- * word is added to the generator's state before the output function; summing the per-word terms
+ *   H_i     = mix( L + sum_j mix(s_i + (j + 1) * g_i + x_j) )      (all arithmetic mod 2^64)
+ *   Hash128 = (H_1, H_2) with  s_1 = 0,                  g_1 = 0x9E3779B97F4A7C15 (the SplitMix64 increment),
+ *                              s_2 = 0x6A09E667F3BCC908, g_2 = 0xD1342543DE82EF95 (another odd increment).
+ * mix(s + (j + 1) * g) is the j-th output of a SplitMix64 generator with seed s and increment g, so each
+ * word is added to that generator's state before the output function; summing the per-word terms
  * makes the hash independent of the order in which the words are visited.
+ * The two hashes run on generators with different increments (as split instances of SplitMix64 do): with a
+ * common increment, moving a word from position j to position i and adding (j - i) * g to it leaves the
+ * multiset of per-word terms of BOTH hashes unchanged, whatever the seeds, so that the two would share a
+ * family of collisions and not be independent; with different increments a rearrangement of that kind
+ * collides one of them only (pinned in the tests).
  */
 #define ORA_GAMMA 0x9E3779B97F4A7C15ull
+#define ORA_GAMMA2 0xD1342543DE82EF95ull
 #define ORA_SEED1 0x0000000000000000ull
 #define ORA_SEED2 0x6A09E667F3BCC908ull
 
@@ -281,14 +287,21 @@ uint64_t ora_splitmix64_next(uint64_t* state) {
     return ora_splitmix64_mix(*state);
 }
 
+/* the same for a generator with another (odd) increment */
+uint64_t ora_splitmix64_next_with(uint64_t* state, uint64_t gamma) {
+    *state += gamma;
+    return ora_splitmix64_mix(*state);
+}
+
 void ora_hash128(const uint8_t* exp, uint64_t len, uint64_t out[2]) {
     const uint64_t seeds[2] = {ORA_SEED1, ORA_SEED2};
+    const uint64_t gammas[2] = {ORA_GAMMA, ORA_GAMMA2};
     for (int h = 0; h < 2; ++h) {
         uint64_t acc = 0;
         for (uint64_t j = 0; 8 * j < len; ++j) {
             uint64_t x = 0;
             for (uint64_t i = 0; i < 8 && 8 * j + i < len; ++i) x |= (uint64_t)exp[8 * j + i] << (8 * i);
-            acc += ora_splitmix64_mix(seeds[h] + (j + 1) * ORA_GAMMA + x);
+            acc += ora_splitmix64_mix(seeds[h] + (j + 1) * gammas[h] + x);
         }
         out[h] = ora_splitmix64_mix(acc + len);
     }
@@ -332,7 +345,7 @@ int ora_encode_hashed(const void* w, uint64_t* hash_cache, uint64_t n, int dtype
     uint64_t sm_off = ora_sm_offset(n, block);
     uint64_t pay_off = ora_payload_offset(n, dtype, block);
 
-    /* (exp, mant) <- SplitExpMant(shard) */
+    /* every value cut into exponent field and sign-plus-mantissa */
     uint8_t* exp = (uint8_t*)malloc(n);
     uint32_t* sm = (uint32_t*)malloc(n * sizeof(uint32_t));
     if (!exp || !sm) {
@@ -343,7 +356,7 @@ int ora_encode_hashed(const void* w, uint64_t* hash_cache, uint64_t n, int dtype
     ora_split(w, n, dtype, exp, sm);
     memset(msg, 0, pay_off);
 
-    /* for k = 1..S_b: h <- Hash128(exp[k]); if h != HashCache[k]: bitmap[k] <- 1, HashCache[k] <- h */
+    /* a block is marked when its hash is not the cached one, which is then replaced */
     for (uint64_t k = 0; k < nb; ++k) {
         uint64_t lo = k * block;
         uint64_t hi = lo + block < n ? lo + block : n;
@@ -358,7 +371,7 @@ int ora_encode_hashed(const void* w, uint64_t* hash_cache, uint64_t n, int dtype
 
     for (uint64_t j = 0; j < n; ++j) put_bits(msg + sm_off, j * (uint64_t)m, m, sm[j]);
 
-    /* payload <- { exp[k] | bitmap[k] = 1 } in block order (no entropy stage, as in ora_encode) */
+    /* the exponents of the marked blocks, ascending (no entropy stage, as in ora_encode) */
     uint64_t plen = 0;
     uint32_t nchg = 0;
     for (uint64_t k = 0; k < nb; ++k) {

@@ -59,6 +59,7 @@ def lib() -> ctypes.CDLL:
         L.ora_decode.argtypes, L.ora_decode.restype = [vp, vp, u64, i32, u32, vp], i32
         L.ora_splitmix64_mix.argtypes, L.ora_splitmix64_mix.restype = [u64], u64
         L.ora_splitmix64_next.argtypes, L.ora_splitmix64_next.restype = [vp], u64
+        L.ora_splitmix64_next_with.argtypes, L.ora_splitmix64_next_with.restype = [vp, u64], u64
         L.ora_hash128.argtypes, L.ora_hash128.restype = [vp, u64, vp], None
         L.ora_hash_cache_init.argtypes, L.ora_hash_cache_init.restype = [vp, u64, i32, u32, vp], i32
         L.ora_encode_hashed.argtypes = [vp, vp, u64, i32, u32, vp, u64, vp, vp, vp]
@@ -187,10 +188,13 @@ def gain(n, dtype, block, q, world, alpha=0.0, beta=1.0, table=None, t_hash=0.0,
 # ------------------------------------------------------------------ hash-based change detection
 
 
-def splitmix64_stream(seed: int, count: int):
-    """First ``count`` outputs of the SplitMix64 generator seeded with ``seed``."""
+def splitmix64_stream(seed: int, count: int, gamma: int = None):
+    """First ``count`` outputs of the SplitMix64 generator seeded with ``seed`` (``gamma``: an increment
+    other than the generator's own)."""
     state = ctypes.c_uint64(seed)
-    return [int(lib().ora_splitmix64_next(ctypes.addressof(state))) for _ in range(count)]
+    if gamma is None:
+        return [int(lib().ora_splitmix64_next(ctypes.addressof(state))) for _ in range(count)]
+    return [int(lib().ora_splitmix64_next_with(ctypes.addressof(state), gamma)) for _ in range(count)]
 
 
 def splitmix64_mix(z: int) -> int:

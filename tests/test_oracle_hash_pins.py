@@ -13,6 +13,8 @@ from paper_2609_04609_b200 import workloads as wl
 
 MASK = (1 << 64) - 1
 GAMMA = 0x9E3779B97F4A7C15
+GAMMA2 = 0xD1342543DE82EF95  # the second hash's generator runs on an increment of its own
+HASHES = ((0, GAMMA), (0x6A09E667F3BCC908, GAMMA2))  # (seed, increment) of the two 64-bit hashes
 
 
 def test_splitmix64_published_streams(oracle):
@@ -27,9 +29,12 @@ def test_zero_blocks_tie_the_hash_to_the_generator_stream(oracle):
     H_s = mix(L + sum of the first ceil(L/8) outputs)."""
     for L in (1, 7, 8, 9, 64, 512, 4096, 13):
         m = -(-L // 8)
-        for h, seed in zip(oracle.hash128(np.zeros(L, np.uint8)), (0, 0x6A09E667F3BCC908)):
-            acc = sum(oracle.splitmix64_stream(seed, m)) & MASK
+        for h, (seed, gamma) in zip(oracle.hash128(np.zeros(L, np.uint8)), HASHES):
+            acc = sum(oracle.splitmix64_stream(seed, m, gamma)) & MASK
             assert h == oracle.splitmix64_mix((acc + L) & MASK)
+    # the increment argument itself: the generator's own increment gives the published stream
+    assert oracle.splitmix64_stream(1234567, 5, GAMMA) == oracle.splitmix64_stream(1234567, 5)
+    assert GAMMA2 % 2 == 1  # odd: the generator's state runs through all 2^64 values
 
 
 def test_mix_is_a_bijection_on_samples_and_fixes_zero(oracle):
@@ -125,10 +130,31 @@ def test_python_restatement_of_the_construction(oracle):
     for L in (1, 8, 9, 63, 64, 65, 512):
         blk = rng.integers(0, 256, L, dtype=np.uint8)
         want = []
-        for seed in (0, 0x6A09E667F3BCC908):
+        for seed, gamma in HASHES:
             acc = 0
             for j in range(-(-L // 8)):
                 x = int.from_bytes(blk[8 * j : 8 * j + 8].tobytes().ljust(8, b"\0"), "little")
-                acc = (acc + mix((seed + (j + 1) * GAMMA + x) & MASK)) & MASK
+                acc = (acc + mix((seed + (j + 1) * gamma + x) & MASK)) & MASK
             want.append(mix((acc + L) & MASK))
         assert oracle.hash128(blk) == tuple(want)
+
+
+def test_a_rearrangement_that_collides_one_hash_does_not_collide_the_other(oracle):
+    """Why the two hashes run on different increments.  Swapping two words and shifting them by the distance times
+    an increment g reproduces the per-word terms of the hash that runs on g -- a genuine collision of that 64-bit
+    hash, for every seed.  With a common increment both halves would collide together; with different ones the
+    other half tells the blocks apart, so Hash128 still detects the change."""
+    rng = np.random.default_rng(6)
+    for g, collides, differs in ((GAMMA, 0, 1), (GAMMA2, 1, 0)):
+        for _ in range(20):
+            words = [int(v) for v in rng.integers(0, 1 << 63, 4)]
+            i, j = 0, 2
+            moved = list(words)
+            moved[i] = (words[j] + (j - i) * g) & MASK
+            moved[j] = (words[i] - (j - i) * g) & MASK
+            a = np.frombuffer(b"".join(w.to_bytes(8, "little") for w in words), np.uint8)
+            b = np.frombuffer(b"".join(w.to_bytes(8, "little") for w in moved), np.uint8)
+            assert not np.array_equal(a, b)
+            ha, hb = oracle.hash128(a), oracle.hash128(b)
+            assert ha[collides] == hb[collides]
+            assert ha[differs] != hb[differs]
