@@ -765,6 +765,24 @@ def one_layer_case(args, device, peak, over, steps=5):
         "encode_GBps_of_weights": n * vb / (enc_ms * 1e-3) / 1e9, "decode_GBps_of_weights": n * vb / (dec_ms * 1e-3) / 1e9,
         "verified_bit_exact": verified, "oracle_sampled_units": sampled,
     }
+    if a.block < 32 and a.detect == "compare":
+        # Blocks smaller than a 32-byte DRAM sector: the caches (one byte per value) can only be refreshed by whole
+        # sectors, so the bytes that have to move are the sectors holding a changed exponent, not q bytes per value.
+        # s = share of the 32-value groups of the layer in which some exponent differs between the two iterates.
+        shift, wdt_t, emask = {"bf16": (7, torch.int16, 0xFF), "fp32": (23, torch.int32, 0xFF),
+                               "fp16": (10, torch.int16, 0x1F)}[a.dtype]
+        ea = (wa[0].view(wdt_t) >> shift) & emask
+        eb = (wb[0].view(wdt_t) >> shift) & emask
+        diff = ea != eb
+        m = diff.numel() // 32 * 32
+        s_rate = float(diff[:m].view(-1, 32).any(dim=1).float().mean().item())
+        del ea, eb, diff
+        extra = n * max(s_rate - q, 0.0)  # cache bytes beyond the q per value already counted
+        res["cache_sector_rate"] = s_rate
+        res["encode_frac_sector_granular"] = (a_enc + extra) / (enc_ms * 1e-3) / 1e9 / peak
+        res["decode_frac_sector_granular"] = (a_dec + extra) / (dec_ms * 1e-3) / 1e9 / peak
+        res["sector_note"] = ("the *_frac_sector_granular figures count the cache refresh as whole 32-byte sectors "
+                              "(cache_sector_rate bytes per value) instead of q bytes per value")
     if a.entropy:
         res["entropy_encode_ms"], res["entropy_decode_ms"] = [
             float(np.mean([t[k].elapsed_time(t[k + 1]) for t in timers])) for k in (6, 8)]

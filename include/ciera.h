@@ -217,11 +217,13 @@ CIERA_API int ciera_encode_noalloc(const ciera_plan* plan, const void* weights_d
  * Instead of the previous exponents the sender keeps HashCache: one 128-bit hash per block, built
  * from two independent 64-bit SplitMix64 hashes of the block's exponents.  A block travels iff its
  * hash differs from the cached one; the cached hash is then replaced.  The message is the same as
- * ciera_encode's (a collision, probability about 2^-128 per comparison, would leave a changed
- * block unsent).  The construction (the paper prints none): with mix() the SplitMix64 output
- * function and gamma its increment, a block of L exponent bytes read as little-endian 64-bit words
- * x_j (the last one zero-padded),  H_s = mix(L + sum_j mix(s + (j + 1) * gamma + x_j)) mod 2^64,
- * Hash128 = (H_0, H_0x6A09E667F3BCC908), stored as two little-endian 64-bit words per block.
+ * ciera_encode's (a collision -- both 64-bit halves at once, which behave like independent random
+ * functions of the block but are not a cryptographic hash -- would leave a changed block unsent).
+ * The construction (the paper prints none): with mix() the SplitMix64 output function, a block of L
+ * exponent bytes read as little-endian 64-bit words x_j (the last one zero-padded),
+ * H_i = mix(L + sum_j mix(s_i + (j + 1) * g_i + x_j)) mod 2^64, Hash128 = (H_1, H_2) with
+ * s_1 = 0, g_1 = 0x9E3779B97F4A7C15 (the generator's increment), s_2 = 0x6A09E667F3BCC908,
+ * g_2 = 0xD1342543DE82EF95; stored as two little-endian 64-bit words per block.
  * Blocks of 16 values and more only (CIERA_ERR_UNSUPPORTED otherwise). */
 
 /* Bytes of a HashCache for the whole plan (16 per block; units in table order), the offset of a
