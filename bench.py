@@ -377,12 +377,16 @@ def run_reference(args):
             times.append(dt)
     ms = 1e3 * float(np.mean(times))
     gbps = nvals * vb / (ms * 1e-3) / 1e9
-    sample = f"{n_units} of {len(shapes) * args.shards * args.layers} units ({nvals} values) per step"
+    total_units = len(shapes) * args.shards * args.layers
+    sample = f"{n_units} of {total_units} units ({nvals} values) per step"
+    config = workload_config(args)
+    config["workload"] += (f" -- each step of this arm is a sample of {n_units} of the {total_units} units; ms_per_step is "
+                           f"the time of that sample, value (GB/s of weights) is what compares with the other arm")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": gbps, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
-        "config": workload_config(args),
+        "config": config,
         "cpu_baseline": {"value": gbps, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": gbps, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -664,7 +668,7 @@ def main():
 
     # ---- the other configurations, one layer each (rank 0, one GPU only)
     if not args.no_other_configs and rank == 0 and world == 1:
-        out["other_configs"] = other_configs(args, device, peak)
+        out["other_configs"] = other_configs(args, device, peak, clocks.get("sm_mhz"))
 
     # ---- end to end through the host-buffer entry point (weights start and end in host memory)
     if not args.no_e2e:
@@ -725,7 +729,37 @@ OTHER_CONFIGS = [
 ]
 
 
-def one_layer_case(args, device, peak, over, steps=5):
+def raw_payload_symbols(codec, a):
+    """Changed exponents (one symbol each) that the entropy stage codes: the raw payload bytes of the last encode."""
+    from paper_2609_04609_b200 import ciera
+
+    wire = codec.wire_bytes.cpu().numpy()
+    return int(sum(int(w) - ciera.payload_offset(int(u["n_values"]), codec.dtype, a.block)
+                   for u, w in zip(codec.units, wire) if int(u["n_values"])))
+
+
+def entropy_roofline(symbols, enc_ms, dec_ms, sm_mhz, sms=148):
+    """The entropy stage moves little and computes a lot per byte: its bound is instruction issue.  Peak = SMs x 4
+    warp schedulers x one warp instruction per clock at the SM clock sampled during the run; the work is the ncu
+    count of warp instructions per coded symbol on record (profiles/) x the symbols of this launch."""
+    try:
+        rec = json.load(open(TRAFFIC_FILE))["entropy_stage_bf16_B512_clustered_f0.22"]
+    except Exception:
+        return None
+    peak = sms * 4 * (sm_mhz or 1965.0) * 1e6  # warp instructions per second
+    out = {"bound": "issue", "unit": "G warp-instructions/s", "peak": peak / 1e9, "symbols_per_launch": symbols,
+           "derivation": "148 SMs x 4 schedulers x 1 warp instruction per clock x sampled SM MHz"}
+    for name, ms, key in (("encode", enc_ms, "warp_instructions_per_symbol_encode"),
+                          ("decode", dec_ms, "warp_instructions_per_symbol_decode")):
+        ach = rec[key] * symbols / (ms * 1e-3)
+        out[name] = {"warp_instructions_per_symbol": rec[key], "achieved": ach / 1e9, "frac": ach / peak,
+                     "payload_GBps": symbols / (ms * 1e-3) / 1e9}
+    if rec.get("csrc_sha256") != csrc_digest():
+        out["note"] = "instruction counts per symbol are from an ncu capture of earlier kernel sources"
+    return out
+
+
+def one_layer_case(args, device, peak, over, steps=5, clocks_mhz=None):
     """One layer of the workload `args` + `over`: three warm-up steps, then `steps` timed ones, all on one stream."""
     import torch
 
@@ -790,7 +824,10 @@ def one_layer_case(args, device, peak, over, steps=5):
         w = wb if i % 2 == 0 else wa
         codec.encode(w[0])
         raw = codec.paper_bytes()
+        symbols = raw_payload_symbols(codec, a)
         codec.entropy_encode()
+        res["entropy_roofline"] = entropy_roofline(symbols, res["entropy_encode_ms"],
+                                                   res["entropy_decode_ms"], clocks_mhz)
         coded = codec.paper_bytes()
         fixed = sum(ciera.message_bytes(int(u["n_values"]), codec.dtype, a.block, 0) for u in codec.units if int(u["n_values"]))
         res["bytes_ratio_coded"] = coded / (n * vb)
@@ -805,12 +842,12 @@ def one_layer_case(args, device, peak, over, steps=5):
     return res
 
 
-def other_configs(args, device, peak):
+def other_configs(args, device, peak, clocks_mhz=None):
     out = {"per": "one layer; kernels one after the other on one stream, CUDA events around every launch; fractions "
                   "are algorithmic bytes per launch over the measured copy bandwidth"}
     for name, over in OTHER_CONFIGS:
         try:
-            out[name] = one_layer_case(args, device, peak, over)
+            out[name] = one_layer_case(args, device, peak, over, clocks_mhz=clocks_mhz)
         except Exception as e:  # one failing side case must not take the headline line with it
             out[name] = {"error": f"{type(e).__name__}: {e}"}
     return out

@@ -2,9 +2,10 @@
 
 TEST INFRASTRUCTURE ONLY (see ``ciera_oracle.py``); plain Python loops, no tuning.
 
-The paper: shard i has a per-iteration latency gain g_i and a cache footprint
-M_i = (W - 1) * S_e^i per GPU; only shards with positive gain are kept; the shards are
-ranked in descending order of g_i / M_i and selected until the cache budget is exhausted.
+What Section 3.2 defines: every shard has a gain g_i (seconds saved per iteration if it is
+compressed) and costs M_i = (W - 1) * S_e^i bytes of exponent cache on each GPU.  Candidates are the
+shards whose gain is positive; they are taken in order of gain per cached byte, best first, as long
+as the budget allows.
 
 Readings taken here (the paper gives no pseudo-code for this step):
   * ties in g_i / M_i keep the shards' original order;

@@ -844,12 +844,12 @@ static size_t decode_smem_bytes() {
 
 template <int DT, bool FINE>
 static int decode_grid_limit(int* out) {
-    static int cached[64] = {0};
+    static std::atomic<int> cached[64];  // (zero-initialised; any host thread may be the first to fill an entry)
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return record_cuda_error(e);
     if (dev < 0 || dev >= 64) return CIERA_ERR_UNSUPPORTED;
-    if (cached[dev] == 0) {
+    if (cached[dev].load(std::memory_order_acquire) == 0) {
         const size_t smem = decode_smem_bytes<DT, FINE>();
         e = cudaFuncSetAttribute(decode_kernel<DT, FINE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return record_cuda_error(e);
@@ -859,9 +859,9 @@ static int decode_grid_limit(int* out) {
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return record_cuda_error(e);
         if (per_sm < 1 || sms < 1) return CIERA_ERR_UNSUPPORTED;
-        cached[dev] = per_sm * sms;
+        cached[dev].store(per_sm * sms, std::memory_order_release);
     }
-    *out = cached[dev];
+    *out = cached[dev].load(std::memory_order_acquire);
     return CIERA_OK;
 }
 

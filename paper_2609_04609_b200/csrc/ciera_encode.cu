@@ -106,9 +106,9 @@ struct EncodeCfg<CIERA_FP32, true> {
 // With HashCache the exponent ring stages no cached exponents (it only keeps the new ones until
 // they are sent), so it is shorter; each of its stages has a companion with the tile's cached
 // hashes and the consumers' partial sums, sized at launch from the block size.
-// The template argument HASH of the kernel is 0 (exponent cache), 1 (HashCache) or 2 (HashCache with
+// The template argument HASH of the kernel is 0 (exponent cache), 1 (HashCache), 2 (HashCache with
 // shorter rings: with blocks of 64 values and fewer the hash stages are large, and two thread blocks
-// still have to fit an SM).
+// still have to fit an SM) or 3 (as 2, and the consumers finish the blocks' hashes).
 template <int DT, int HASH>
 struct EncodeHashCfg;
 template <>
@@ -139,7 +139,12 @@ struct EncodeHashCfg<CIERA_FP32, 2> {
     static constexpr int kDefer = 1;
     static constexpr int kBmWords = kBitmapWords;
 };
+template <int DT>
+struct EncodeHashCfg<DT, 3> : EncodeHashCfg<DT, 2> {};
 constexpr uint32_t kHashShortRingsLog2 = 6;  // blocks of up to 2^6 values take the shorter rings
+// With 256 and more blocks in a tile (16 and 32 values per block) the consumers finish the blocks' hashes
+// themselves: kernel instance HASH == 3 (see finish_hash_groups; blocks of at least two lanes' pieces).
+constexpr uint32_t kHashByConsumersLog2 = 5;
 template <int DT, bool FINE, int HASH>
 struct EncodeCfgOf {
     using type = EncodeHashCfg<DT, HASH>;
@@ -323,6 +328,13 @@ __device__ __forceinline__ uint32_t scan_block_bitmap(const uint32_t* bm, uint16
     return run;
 }
 
+// Blocks whose hashes the consumers finish themselves (see finish_hash_groups; kernel instance HASH == 3): many
+// per tile, and made of at least two lanes' pieces.
+template <int DT>
+__host__ __device__ __forceinline__ bool hash_finished_by_consumers(uint32_t log2b) {
+    return log2b <= kHashByConsumersLog2 && log2b > (uint32_t)Piece<DT>::kLog2Values;
+}
+
 // Aggregator warp, one tile: block flags, the tile's bitmap bytes, the tile's payload byte count.
 // With `publish` the count goes out at once as the tile's status word, so that later tiles never
 // wait for it longer than for the votes themselves.  Waits for nothing outside the thread block.
@@ -330,7 +342,7 @@ __device__ __forceinline__ uint32_t scan_block_bitmap(const uint32_t* bm, uint16
 // block: adds up the block's partial sums, finishes the two hashes, compares them with the cached
 // pair and, where they differ, flags the block and stores the new pair (HashCache[i,k] <- h).
 // Returns the number of flagged blocks (one warp).
-template <int DT>
+template <int DT, bool BY_CONSUMERS>
 __device__ __forceinline__ uint32_t hash_block_bitmap(const ulonglong2* part, const ulonglong2* hold, ulonglong2* hash_dst,
                                                       uint32_t* bm, uint16_t* pre, uint32_t log2b, uint32_t nv,
                                                       uint32_t lane) {
@@ -339,9 +351,11 @@ __device__ __forceinline__ uint32_t hash_block_bitmap(const ulonglong2* part, co
     const uint32_t nbt = kTileValues >> log2b;
     const uint32_t nblk = (nv + B - 1u) >> log2b;
     const uint32_t epb_l2 = log2b > kGroupL2 ? log2b - kGroupL2 : 0u;  // log2(partial sums per block)
+    const uint8_t* const verdicts = reinterpret_cast<const uint8_t*>(part);
     // one block: true iff its hashes differ from the cached pair (which is then replaced)
     auto finish_block = [&](uint32_t i) -> bool {
         if (i >= nblk) return false;
+        if (BY_CONSUMERS) return verdicts[i] != 0;  // finished, compared and stored by the consumers already
         uint64_t a = 0, b = 0;
         for (uint32_t e = 0; e < (1u << epb_l2); ++e) {
             const ulonglong2 v = part[(i << epb_l2) + e];
@@ -419,6 +433,66 @@ __device__ __forceinline__ void reduce_hash_terms(const uint64_t* a, const uint6
     }
 }
 
+// HashCache, consumers, kernel instance HASH == 3 (blocks that lie inside one warp's pieces and span at least two
+// lanes, l2 >= 1): the same reduction as reduce_hash_terms, but the lanes that end up with a block's sums
+// finish the block themselves -- each finishes one 64-bit half, compares it with its cached half, and the two
+// halves of a block (in neighbouring lanes) agree on the verdict with one exchange; a changed block's new hash
+// goes to HashCache at once (HashCache[i,k] <- h), and one byte per block tells the aggregator the verdict.
+// With 256 or 512 blocks in a tile the one aggregator warp, finishing them all by itself, set the pace of the
+// whole thread block (0.82 ms per layer with 32 values per block, 1.24 ms with 16, whatever the change rate);
+// with fewer blocks per tile the extra work in the consumers costs more than it saves (measured), so those
+// keep the aggregator's way.
+//   hold   the tile's cached hashes (two words per block), staged in shared memory
+//   dst    the same in global memory
+//   flags  one byte per block of the tile (written for every block below nblk)
+template <int DT, int NP>
+__device__ __forceinline__ void finish_hash_groups(const uint64_t* a, const uint64_t* b, uint32_t l2, uint32_t log2b,
+                                                   uint32_t nv, uint32_t tid, const uint64_t* hold, uint64_t* dst,
+                                                   uint8_t* flags, uint32_t lane) {
+    using P = Piece<DT>;
+    const bool odd = (lane & 1u) != 0;
+    const uint32_t B = 1u << log2b;
+    // One half of one block: `t` = the sum of the half's terms over the block (held by `leader` lanes, the half is
+    // the lane's parity), `piece` = which of the thread's pieces lies in that block.  Called by all lanes together.
+    auto finish_half = [&](uint64_t t, int piece, bool leader) {
+        const uint32_t blk = P::start(tid, piece) >> log2b;
+        const uint32_t first = blk << log2b;
+        const bool mine = leader && first < nv;
+        uint64_t h = 0;
+        uint32_t differs = 0;
+        if (mine) {
+            h = mix64(t + min(B, nv - first));
+            differs = h != hold[2u * blk + (odd ? 1u : 0u)] ? 1u : 0u;
+        }
+        differs |= __shfl_xor_sync(0xffffffffu, differs, 1);  // the block's two halves sit in neighbouring lanes
+        if (mine) {
+            if (differs) dst[2u * blk + (odd ? 1u : 0u)] = h;
+            if (!odd) flags[blk] = (uint8_t)differs;
+        }
+    };
+    const uint32_t r = lane & ((1u << l2) - 1u);
+    uint64_t k0 = (odd ? b[0] : a[0]) + __shfl_xor_sync(0xffffffffu, odd ? a[0] : b[0], 1);
+    if constexpr (NP == 1) {
+#pragma unroll
+        for (uint32_t o = 1; o < 5; ++o)
+            if (o < l2) k0 += __shfl_xor_sync(0xffffffffu, k0, 1u << o);
+        finish_half(k0, 0, r < 2u);
+    } else {
+        const uint64_t k1 = (odd ? b[1] : a[1]) + __shfl_xor_sync(0xffffffffu, odd ? a[1] : b[1], 1);
+        if (l2 == 1) {  // a block is two lanes' pieces: every lane finishes a half of each of its two blocks
+            finish_half(k0, 0, true);
+            finish_half(k1, NP - 1, true);
+        } else {
+            const bool second = (lane & 2u) != 0;
+            uint64_t t = (second ? k1 : k0) + __shfl_xor_sync(0xffffffffu, second ? k0 : k1, 2);
+#pragma unroll
+            for (uint32_t o = 2; o < 5; ++o)
+                if (o < l2) t += __shfl_xor_sync(0xffffffffu, t, 1u << o);
+            finish_half(t, second ? NP - 1 : 0, r < 4u);
+        }
+    }
+}
+
 // what aggregate_tile needs besides the votes when the sender keeps HashCache
 struct HashTile {
     const ulonglong2* part;
@@ -439,7 +513,7 @@ __device__ __forceinline__ uint64_t aggregate_tile(const TileDesc& td, uint32_t 
 
     uint32_t run;
     if constexpr (HASH)
-        run = hash_block_bitmap<DT>(ht.part, ht.hold, ht.dst, bm, pre, log2b, nv, lane);
+        run = hash_block_bitmap<DT, HASH == 3>(ht.part, ht.hold, ht.dst, bm, pre, log2b, nv, lane);
     else
         run = FINE ? scan_block_bitmap(bm, pre, log2b, lane)
                    : build_block_bitmap(ballot, bm, pre, log2b, Piece<DT>::kLog2Values, lane);
@@ -899,7 +973,7 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint2*
         uint32_t k = 0;
         // stage and phase of slot k in the two rings, and of slot k - kDefer in the exponent ring, kept
         // as running counters (the ring depths are no powers of two)
-        uint32_t sw = 0, pw = 0, se = 0, je = 0, pj = 0;
+        uint32_t sw = 0, pw = 0, se = 0, pe = 0, je = 0, pj = 0;
         // HASH: the lanes of a warp that share a block (a power of two, at most the warp) add up their terms
         const uint32_t hash_lanes_l2 = min(5u, log2b - (uint32_t)P::kLog2Values);
         for (;; ++k) {
@@ -952,8 +1026,17 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint2*
                 }
                 if constexpr (HASH) {
                     uint64_t* const part = reinterpret_cast<uint64_t*>(ring_h + (size_t)se * kHStage + kHoldBytes);
-                    reduce_hash_terms<P::kPerThread>(hash_a, hash_b, hash_lanes_l2, (P::start(tid, 0) >> P::kLog2Values) >> hash_lanes_l2,
-                                                     (P::start(tid, P::kPerThread - 1) >> P::kLog2Values) >> hash_lanes_l2, part, lane);
+                    if constexpr (HASH == 3) {
+                        // the tile's cached hashes have to be there now (they land on full_e)
+                        if (!mbar_wait(&ctl->full_e[se], pe, abort, status)) break;
+                        finish_hash_groups<DT, P::kPerThread>(hash_a, hash_b, hash_lanes_l2, log2b, nv, tid,
+                                                              reinterpret_cast<const uint64_t*>(ring_h + (size_t)se * kHStage),
+                                                              reinterpret_cast<uint64_t*>(ti.c_ptr),
+                                                              reinterpret_cast<uint8_t*>(part), lane);
+                    } else {
+                        reduce_hash_terms<P::kPerThread>(hash_a, hash_b, hash_lanes_l2, (P::start(tid, 0) >> P::kLog2Values) >> hash_lanes_l2,
+                                                         (P::start(tid, P::kPerThread - 1) >> P::kLog2Values) >> hash_lanes_l2, part, lane);
+                    }
                 }
                 __syncwarp();  // the warp's shared-memory accesses above are ordered before lane 0's arrives
                 if (lane == 0) {
@@ -982,7 +1065,10 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint2*
                 sw = 0;
                 pw ^= 1u;
             }
-            if (++se == (uint32_t)SE) se = 0;
+            if (++se == (uint32_t)SE) {
+                se = 0;
+                pe ^= 1u;
+            }
         }
         // tiles whose changed exponents are still to be sent (when kDefer > kResolvers)
         if (!*abort && k_end != kNoTile) {
@@ -1038,12 +1124,12 @@ static size_t encode_smem_bytes(uint32_t log2b) {
 // Largest grid whose blocks are all resident at once, per device and block size (0 = not yet known).
 template <int DT, bool FINE, int HASH>
 static int encode_grid_limit(uint32_t log2b, int* out) {
-    static int cached[64][16] = {{0}};
+    static std::atomic<int> cached[64][16];  // (zero-initialised; any host thread may be the first to fill an entry)
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return record_cuda_error(e);
     if (dev < 0 || dev >= 64 || log2b >= 16) return CIERA_ERR_UNSUPPORTED;
-    if (cached[dev][log2b] == 0) {
+    if (cached[dev][log2b].load(std::memory_order_acquire) == 0) {
         const size_t smem = encode_smem_bytes<DT, FINE, HASH>(log2b);
         // (the limit set here is the largest any block size asks for: the smallest block of the class)
         e = cudaFuncSetAttribute(encode_kernel<DT, FINE, HASH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1057,9 +1143,9 @@ static int encode_grid_limit(uint32_t log2b, int* out) {
         e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
         if (e != cudaSuccess) return record_cuda_error(e);
         if (per_sm < 1 || sms < 1 || !coop) return CIERA_ERR_UNSUPPORTED;
-        cached[dev][log2b] = per_sm * sms;
+        cached[dev][log2b].store(per_sm * sms, std::memory_order_release);
     }
-    *out = cached[dev][log2b];
+    *out = cached[dev][log2b].load(std::memory_order_acquire);
     return CIERA_OK;
 }
 
@@ -1132,6 +1218,12 @@ int launch_encode_hashed(const ciera_plan* p, const void* weights_dev, void* has
                          uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* scratch, int32_t* status_dev,
                          cudaStream_t s) {
     const bool short_rings = p->log2b <= kHashShortRingsLog2;
+    if (p->dtype == CIERA_BF16 && hash_finished_by_consumers<CIERA_BF16>(p->log2b))
+        return launch_encode<CIERA_BF16, false, 3>(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev,
+                                                   changed_blocks_dev, scratch, status_dev, s);
+    if (p->dtype == CIERA_FP32 && hash_finished_by_consumers<CIERA_FP32>(p->log2b))
+        return launch_encode<CIERA_FP32, false, 3>(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev,
+                                                   changed_blocks_dev, scratch, status_dev, s);
     if (p->dtype == CIERA_BF16)
         return short_rings ? launch_encode<CIERA_BF16, false, 2>(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev,
                                                                  changed_blocks_dev, scratch, status_dev, s)

@@ -1,5 +1,6 @@
-// Hash128 of a block of exponents (paper Section 3.1: a 128-bit hash built from two independent
-// 64-bit SplitMix64 hashes; Algorithm 1 keeps one per block in HashCache).
+// Hash128 of a block of exponents: the per-block fingerprint that the sender of Algorithm 1 keeps in
+// HashCache.  Section 3.1 asks for 128 bits made of two 64-bit SplitMix64-based hashes that do not
+// depend on each other.
 //
 // The paper fixes no more than that.  The construction used here:
 //   mix(z)  = the SplitMix64 output function;

@@ -231,12 +231,12 @@ transport_pipe_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint
 }
 
 static int transport_pipe_grid_limit(int* out) {
-    static int cached[64] = {0};
+    static std::atomic<int> cached[64];  // (zero-initialised; any host thread may be the first to fill an entry)
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return record_cuda_error(e);
     if (dev < 0 || dev >= 64) return CIERA_ERR_UNSUPPORTED;
-    if (cached[dev] == 0) {
+    if (cached[dev].load(std::memory_order_acquire) == 0) {
         const size_t smem = (size_t)kPipeStages * kPipeStage + sizeof(PipeCtl);
         e = cudaFuncSetAttribute(transport_pipe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return record_cuda_error(e);
@@ -246,9 +246,9 @@ static int transport_pipe_grid_limit(int* out) {
         e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return record_cuda_error(e);
         if (per_sm < 1 || sms < 1) return CIERA_ERR_UNSUPPORTED;
-        cached[dev] = per_sm * sms;
+        cached[dev].store(per_sm * sms, std::memory_order_release);
     }
-    *out = cached[dev];
+    *out = cached[dev].load(std::memory_order_acquire);
     return CIERA_OK;
 }
 
