@@ -159,7 +159,7 @@ class ClockSampler:
 
     def __init__(self, index: int, uuid: str = "", period_s: float = 0.05):
         self.index, self.period = index, period_s
-        self.samples, self.reasons = [], set()
+        self.samples, self.reasons, self.power = [], set(), []
         self.max_mhz = None
         self._stop = threading.Event()
         self._thr = None
@@ -188,6 +188,10 @@ class ClockSampler:
         while not self._stop.is_set():
             try:
                 self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
+                except Exception:
+                    pass
                 r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
                 for bit, name in names.items():
                     if r & bit:
@@ -208,7 +212,8 @@ class ClockSampler:
         if not self.samples:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
         return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
-                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+                "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "power_w": float(np.median(self.power)) if self.power else None}
 
 
 # --------------------------------------------------------------------------------- workload
@@ -641,6 +646,11 @@ def main():
         "kernel_ms_overlapped": {"encode": ovl_ms[0], "transport": ovl_ms[1], "decode": ovl_ms[2],
                                  "per": "layer launch inside the two-stream timed region (kernels overlap)"},
         "serial_ms_per_step": serial_ms_per_step,
+        "kernel_ms_x_sm_mhz": ({"encode": enc_ms * clocks["sm_mhz"], "transport": tra_ms * clocks["sm_mhz"],
+                                "decode": dec_ms * clocks["sm_mhz"],
+                                "note": "launch time x median SM MHz sampled in the timed region: constant across runs "
+                                        "for a kernel bound by the SM clock, proportional to the clock for one bound by HBM"}
+                               if clocks.get("sm_mhz") else None),
         "roofline": {
             "bound": "hbm", "kernel": ("encode_kernel" if args.detect == "compare" else "encode_kernel (HashCache form)"), "achieved": enc_gbs, "peak": peak, "unit": "GB/s",
             "frac": enc_gbs / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBps": enc_gbs / NOMINAL_HBM_GBS,
