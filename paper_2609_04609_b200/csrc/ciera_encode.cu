@@ -126,6 +126,8 @@ struct EncodeHashCfg<CIERA_FP32, 1> {
     static constexpr int kBmWords = kBitmapWords;
 };
 template <>
+struct EncodeHashCfg<CIERA_FP16, 1> : EncodeHashCfg<CIERA_BF16, 1> {};  // fp16: the tile sizes of bf16
+template <>
 struct EncodeHashCfg<CIERA_BF16, 2> {
     static constexpr int kWStages = 3;
     static constexpr int kEStages = 4;
@@ -139,6 +141,8 @@ struct EncodeHashCfg<CIERA_FP32, 2> {
     static constexpr int kDefer = 1;
     static constexpr int kBmWords = kBitmapWords;
 };
+template <>
+struct EncodeHashCfg<CIERA_FP16, 2> : EncodeHashCfg<CIERA_BF16, 2> {};
 template <int DT>
 struct EncodeHashCfg<DT, 3> : EncodeHashCfg<DT, 2> {};
 constexpr uint32_t kHashShortRingsLog2 = 6;  // blocks of up to 2^6 values take the shorter rings
@@ -765,7 +769,7 @@ encode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, const uint2*
               unsigned long long* wire_bytes, uint32_t* changed_blocks, unsigned long long* tile_status,
               unsigned int* unit_ticket, unsigned int* blocks_done, int32_t* status,
               const unsigned long long* __restrict__ tile_hash) {
-    static_assert(!(HASH && (FINE || DT == CIERA_FP16)), "HashCache: bf16 and fp32, blocks of 16 values and more");
+    static_assert(!(HASH && FINE), "HashCache: blocks of 16 values and more");
     using P = Piece<DT>;
     constexpr int VB = Traits<DT>::kValueBytes;
     constexpr int SMB = Traits<DT>::kSmBytes;
@@ -1213,7 +1217,7 @@ static int launch_encode_any(const ciera_plan* p, const void* weights_dev, void*
                                                    changed_blocks_dev, scratch, status_dev, s);
 }
 
-// the sender with HashCache: bf16 and fp32, blocks of 16 values and more (checked by the caller)
+// the sender with HashCache: blocks of 16 values and more, fp16 from 32 (checked by the caller)
 int launch_encode_hashed(const ciera_plan* p, const void* weights_dev, void* hash_cache_dev, void* messages_dev,
                          uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* scratch, int32_t* status_dev,
                          cudaStream_t s) {
@@ -1221,6 +1225,14 @@ int launch_encode_hashed(const ciera_plan* p, const void* weights_dev, void* has
     if (p->dtype == CIERA_BF16 && hash_finished_by_consumers<CIERA_BF16>(p->log2b))
         return launch_encode<CIERA_BF16, false, 3>(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev,
                                                    changed_blocks_dev, scratch, status_dev, s);
+    if (p->dtype == CIERA_FP16 && hash_finished_by_consumers<CIERA_FP16>(p->log2b))
+        return launch_encode<CIERA_FP16, false, 3>(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev,
+                                                   changed_blocks_dev, scratch, status_dev, s);
+    if (p->dtype == CIERA_FP16)
+        return short_rings ? launch_encode<CIERA_FP16, false, 2>(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev,
+                                                                 changed_blocks_dev, scratch, status_dev, s)
+                           : launch_encode<CIERA_FP16, false, 1>(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev,
+                                                                 changed_blocks_dev, scratch, status_dev, s);
     if (p->dtype == CIERA_FP32 && hash_finished_by_consumers<CIERA_FP32>(p->log2b))
         return launch_encode<CIERA_FP32, false, 3>(p, weights_dev, hash_cache_dev, messages_dev, wire_bytes_dev,
                                                    changed_blocks_dev, scratch, status_dev, s);

@@ -85,7 +85,6 @@ static int check_hashed_plan(const ciera_plan* p) {
     if (!p) return CIERA_ERR_INVALID_ARG;
     if (!p->tiles.empty() && !p->tiles_dev) return CIERA_ERR_NOT_BOUND;
     if (is_fine(p->log2b)) return CIERA_ERR_UNSUPPORTED;  // blocks of fewer than 16 values: exact comparison only
-    if (p->dtype == CIERA_FP16) return CIERA_ERR_UNSUPPORTED;
     return CIERA_OK;
 }
 
@@ -97,7 +96,10 @@ extern "C" int ciera_hash_cache_init(const ciera_plan* p, void* hash_cache_dev, 
     if (!hash_cache_dev) return CIERA_ERR_INVALID_ARG;
     if (misaligned16(hash_cache_dev) || misaligned16(weights_dev)) return CIERA_ERR_MISALIGNED;
     cudaStream_t s = (cudaStream_t)stream;
-    if (p->dtype == CIERA_BF16)
+    if (p->dtype == CIERA_FP16)
+        hash_cache_init_kernel<CIERA_FP16><<<nt, kThreads, 0, s>>>(p->tiles_dev, p->tile_hash_dev, p->log2b,
+                                                                   (const uint8_t*)weights_dev, (ulonglong2*)hash_cache_dev);
+    else if (p->dtype == CIERA_BF16)
         hash_cache_init_kernel<CIERA_BF16><<<nt, kThreads, 0, s>>>(p->tiles_dev, p->tile_hash_dev, p->log2b,
                                                                    (const uint8_t*)weights_dev, (ulonglong2*)hash_cache_dev);
     else

@@ -12,9 +12,9 @@ from paper_2609_04609_b200 import workloads as wl
 pytestmark = pytest.mark.gpu
 
 DEV = "cuda:0"
-WDT = {0: np.uint16, 1: np.uint32}
-VB = {0: 2, 1: 4}
-NAME = {0: "bf16", 1: "fp32"}
+WDT = {0: np.uint16, 1: np.uint32, 2: np.uint16}
+VB = {0: 2, 1: 4, 2: 2}
+NAME = {0: "bf16", 1: "fp32", 2: "fp16"}
 RAGGED = [0, 1, 5, 15, 16, 17, 100, 511, 512, 513, 4095, 4097, 8191, 8192, 8193, 20000, 3 * 8192 + 77, 70001]
 
 
@@ -82,7 +82,7 @@ def _run(rt, sizes, n_shards, dtype, block, traj, from_zero=False):
 def test_hashed_ragged_units_every_block_size(rt, dtype, block):
     n = rt[1].LayerCodec.from_tensors(RAGGED, 1, NAME[dtype], block, DEV).weights_bytes // VB[dtype]
     rng = np.random.default_rng(300 * dtype + block)
-    hi = 1 << (16 if dtype == 0 else 32)
+    hi = 1 << (32 if dtype == 1 else 16)
     w0 = rng.integers(0, hi, n, dtype=np.uint64).astype(WDT[dtype])
     w1 = w0.copy()
     flip = rng.random(n) < 0.01
@@ -92,7 +92,7 @@ def test_hashed_ragged_units_every_block_size(rt, dtype, block):
     assert chg[1] == 0  # the repeated iterate changes nothing
 
 
-@pytest.mark.parametrize("dtype,block", [(0, 512), (1, 512), (0, 64), (1, 16)])
+@pytest.mark.parametrize("dtype,block", [(0, 512), (1, 512), (0, 64), (1, 16), (2, 512), (2, 32)])
 def test_hashed_reduced_moe_layer_and_zero_start(rt, dtype, block):
     sizes = [r * c for r, c in wl.olmoe_layer_shapes(2)] + [70_001, 17, 0]
     n = rt[1].LayerCodec.from_tensors(sizes, 4, NAME[dtype], block, DEV).weights_bytes // VB[dtype]
@@ -102,7 +102,7 @@ def test_hashed_reduced_moe_layer_and_zero_start(rt, dtype, block):
     _run(rt, sizes, 4, dtype, block, traj[:2], from_zero=True)
 
 
-@pytest.mark.parametrize("dtype,block", [(0, 128), (0, 32), (1, 4096), (1, 64)])
+@pytest.mark.parametrize("dtype,block", [(0, 128), (0, 32), (1, 4096), (1, 64), (2, 64), (2, 2048)])
 def test_hashed_long_unit_of_many_tiles(rt, dtype, block):
     """One unit of ~3 M values = 367 tiles (its tiles are spread over the thread blocks and find their
     payload offsets by look-back) beside a shorter one; long and short rings of the kernel."""
@@ -121,3 +121,18 @@ def test_hashed_rejects_fine_blocks(rt):
     with pytest.raises(ciera.CieraError) as e:
         codec.init_hash_cache(None)
     assert e.value.status == ciera.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("block", [32, 64, 128, 256, 512, 1024, 4096])
+def test_hashed_fp16_ragged_units(rt, block):
+    """fp16 through the hashed sender (5-bit exponents and 11-bit sign-plus-mantissa packed on the wire, the
+    hash taken over the exponents one byte each, as the caches hold them): ragged units, random bit patterns."""
+    n = rt[1].LayerCodec.from_tensors(RAGGED, 1, "fp16", block, DEV).weights_bytes // 2
+    rng = np.random.default_rng(900 + block)
+    w0 = rng.integers(0, 1 << 16, n, dtype=np.uint64).astype(np.uint16)
+    w1 = w0.copy()
+    flip = rng.random(n) < 0.01
+    w1[flip] = rng.integers(0, 1 << 16, int(flip.sum()), dtype=np.uint64).astype(np.uint16)
+    w3 = rng.integers(0, 1 << 16, n, dtype=np.uint64).astype(np.uint16)
+    chg = _run(rt, RAGGED, 1, 2, block, [w0, w1, w1, w3])
+    assert chg[1] == 0
