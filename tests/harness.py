@@ -156,9 +156,21 @@ def compare_step(codec, exp, w_flat, label=""):
     return wire, chg
 
 
+def sender_scratch_is_clean(codec) -> bool:
+    """The sender finds its part of the workspace (one status word per tile, then 16 bytes of counters) all zero
+    and has to hand it back all zero: there is no clearing launch in front of the kernel."""
+    n = 8 * codec.plan.n_tiles + 16
+    clean = not bool(codec.workspace[:n].any().item())
+    hw = getattr(codec, "hashed_workspace", None)
+    if hw is not None:
+        clean = clean and not bool(hw[:n].any().item())
+    return clean
+
+
 def compare_caches(codec, table, label=""):
     if getattr(codec, "canaries", None) is not None:
         codec.canaries.check(label)
+    assert sender_scratch_is_clean(codec), f"{label}: the sender did not hand its scratch back all zero"
     cs = codec.sender_cache.cpu().numpy()
     cr = codec.receiver_cache.cpu().numpy()
     for i, u in enumerate(codec.units):

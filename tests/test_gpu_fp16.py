@@ -98,9 +98,7 @@ def test_fp16_sizes_and_limits(rt):
         runtime.LayerCodec.from_tensors([1000], 1, "fp16", 16, DEV)
     assert e.value.status == ciera.ERR_UNSUPPORTED
     codec = runtime.LayerCodec.from_tensors([1000], 1, "fp16", 64, DEV)
-    with pytest.raises(ciera.CieraError) as e:
-        codec.init_hash_cache(None)
-    assert e.value.status == ciera.ERR_UNSUPPORTED
+    codec.init_hash_cache(None)  # the hashed sender takes fp16 (tests/test_gpu_hashed.py); the entropy stage does not
     with pytest.raises(ciera.CieraError) as e:
         codec.entropy_encode()
     assert e.value.status == ciera.ERR_UNSUPPORTED

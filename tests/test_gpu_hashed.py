@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 import torch
 
-from harness import guard, to_dev_bytes
+from harness import guard, sender_scratch_is_clean, to_dev_bytes
 from oracle import ciera_oracle as ora
 from paper_2609_04609_b200 import workloads as wl
 
@@ -73,6 +73,7 @@ def _run(rt, sizes, n_shards, dtype, block, traj, from_zero=False):
             lo, n = int(u["weights_off"]) // VB[dtype], int(u["n_values"])
             assert np.array_equal(out[lo : lo + n], w[lo : lo + n]), f"t={t}: reconstruction differs"
         codec.canaries.check(f"t={t}")
+        assert sender_scratch_is_clean(codec), f"t={t}: scratch not handed back all zero"
         changed_total.append(int(chg.sum()))
     return changed_total
 

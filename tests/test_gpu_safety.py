@@ -139,3 +139,31 @@ def test_guard_bytes_notice_a_stray_store(rt):
     codec.allocations["wire_bytes"][len(codec.units)] = 0
     with pytest.raises(AssertionError, match="wire_bytes"):
         codec.canaries.check("planted")
+
+
+@pytest.mark.gpu
+def test_a_dirty_workspace_is_made_usable_again_by_workspace_init(rt):
+    """The sender expects its scratch all zero.  What a kernel that gave up would leave behind is imitated from the
+    host (the status words and counters overwritten with junk); `ciera_workspace_init` puts it right, and the next
+    step is bit-exact and leaves the scratch all zero again -- also for a plan whose long unit makes the thread
+    blocks look back on each other."""
+    from harness import sender_scratch_is_clean
+
+    ciera, runtime = rt
+    codec = guard(runtime.LayerCodec.from_tensors([3_000_000 + 5, 131_072, 70_001], 2, "bf16", 512, DEV, slack=256))
+    table = OracleTable(codec.units, 0, 512, codec.cache_bytes, codec.msg_bytes)
+    n = codec.weights_bytes // 2
+    traj = [wl.as_bits(w) for w in wl.trajectory(n, "bf16", 5150, 2, "clustered", f=0.3)]
+    codec.init_caches(to_dev_bytes(traj[0], DEV))
+    table.init_caches(traj[0])
+    for t in (1, 2):
+        codec.workspace.fill_(0xEE)
+        ciera.workspace_init(codec.plan, codec.workspace)
+        assert sender_scratch_is_clean(codec)
+        codec.step(to_dev_bytes(traj[t], DEV))
+        torch.cuda.synchronize()
+        codec.check_status()
+        exp = table.step(traj[t])
+        compare_step(codec, exp, traj[t], f"t={t}")
+        compare_caches(codec, table, f"t={t}")  # (checks the scratch as well)
+        compare_recon(codec, exp, traj[t], 0, f"t={t}")
