@@ -679,6 +679,7 @@ def main():
     # ---- the other configurations, one layer each (rank 0, one GPU only)
     if not args.no_other_configs and rank == 0 and world == 1:
         out["other_configs"] = other_configs(args, device, peak, clocks.get("sm_mhz"))
+        out["block_size_sweep"] = block_size_sweep(args, device, peak)
 
     # ---- end to end through the host-buffer entry point (weights start and end in host memory)
     if not args.no_e2e:
@@ -852,6 +853,23 @@ def one_layer_case(args, device, peak, over, steps=5, clocks_mhz=None):
     return res
 
 
+def block_size_sweep(args, device, peak):
+    """The paper's block-size sensitivity (64 ... 4096 values per block, default 512) on one synthetic layer: how the
+    share of changed blocks, the message size and the kernels' pace move with B, under the clustered update (changes
+    concentrated in 512-aligned segments) and under the literal Adam-like update (independent changes)."""
+    out = {"per": "one layer, bf16; kernels one after the other on one stream; fractions of the measured copy bandwidth"}
+    for update in ("clustered", "adam"):
+        for block in (16, 32, 64, 128, 256, 512, 1024, 2048, 4096):
+            try:
+                r = one_layer_case(args, device, peak, dict(block=block, update=update), steps=3)
+                out[f"{update}_B{block}"] = {k: r[k] for k in ("block_change_rate_q", "bytes_ratio", "encode_ms", "decode_ms",
+                                                                 "encode_frac", "transport_frac", "decode_frac",
+                                                                 "verified_bit_exact")}
+            except Exception as e:
+                out[f"{update}_B{block}"] = {"error": f"{type(e).__name__}: {e}"}
+    return out
+
+
 def other_configs(args, device, peak, clocks_mhz=None):
     out = {"per": "one layer; kernels one after the other on one stream, CUDA events around every launch; fractions "
                   "are algorithmic bytes per launch over the measured copy bandwidth"}
@@ -884,6 +902,7 @@ def kernels_alone(args, codec, w_a, w_b, peak):
         for _ in range(reps):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             torch.cuda.synchronize()
+            torch.cuda._sleep(300_000)  # keeps the stream busy while the host enqueues: no launch latency between the events
             e0.record()
             fn()
             e1.record()

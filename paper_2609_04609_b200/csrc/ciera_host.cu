@@ -164,15 +164,14 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
     // blocks finish.  Measured on one OLMoE-shaped layer (units of 16 tiles, 0.2848 ms with four runs of 4):
     // 8 + 4 + 4 tiles 0.2836 ms, 12 + 4 tiles 0.2823 ms (14 + 2: 0.2840, 15 + 1: 0.2857, 8 + 8: 0.2871); ending on runs of
     // 2 + 1 + 1 tiles instead 0.2932 ms.
-    // (With 16 to 128 values per block a tile has 64 to 512 blocks and the aggregator warp, which also waits
-    // for the status word at the start of a run, has the least time to spare: there whole units measured 2-3 %
-    // faster than runs, so a run is the whole unit.)
-    const bool whole_units = p->log2b >= 4 && p->log2b <= 7;
+    // (While a run's number and table entry were still waited for at its start, whole units were the faster way
+    // with 16 to 128 values per block, where the aggregator warp has the least time to spare; with the look-ahead
+    // runs win there too: 0.2874 against 0.2917 ms with 64 values per block, 0.2898 against 0.3005 with 128.)
     for (int pass = 0; pass < 2; ++pass) {
         for (size_t i = 0; i + 1 < p->seq_first.size(); ++i) {
             const uint32_t first = p->seq_first[i], end = p->seq_first[i + 1];
             const uint32_t n = end - first;
-            const uint32_t head = (whole_units || n <= kSeqRunTiles) ? n : (n - 1) / kSeqRunTiles * kSeqRunTiles;
+            const uint32_t head = n <= kSeqRunTiles ? n : (n - 1) / kSeqRunTiles * kSeqRunTiles;
             if (pass == 0)
                 p->seq_runs.push_back({first, first + head});
             else if (head < n)
