@@ -76,17 +76,20 @@ def decode(coded: np.ndarray, p: int) -> np.ndarray:
 # ------------------------------------------------------------------ whole unit messages
 
 
-def payload_bytes_from_bitmap(msg: np.ndarray, n: int, block: int) -> int:
-    """P = total length of the changed blocks, read off the message's bitmap."""
+def payload_bytes_from_bitmap(msg: np.ndarray, n: int, block: int, dtype: int = 0) -> int:
+    """P = total length in bytes of the changed blocks, read off the message's bitmap (a block of L values takes
+    L bytes, for fp16 -- five bits per exponent, every block starting on a byte boundary -- ceil(5 L / 8))."""
     nb = ora.num_blocks(n, block)
     flags = np.unpackbits(msg[: ora.bitmap_bytes(n, block)], bitorder="little")[:nb].astype(bool)
     lens = np.minimum(block, n - np.arange(nb, dtype=np.int64) * block)
-    return int(lens[flags].sum())
+    return int(sum(ora.block_payload_bytes(int(l), dtype) for l in lens[flags]))
 
 
 def entropy_encode_message(msg: np.ndarray, n: int, dtype: int, block: int) -> np.ndarray:
     """The sender's entropy stage on one unit's raw message: the payload is replaced by its coded
-    section iff that is strictly shorter."""
+    section iff that is strictly shorter.  The coder's symbols are the payload's BYTES whatever the precision: for
+    fp16 these are the bytes of the packed five-bit exponents as they travel (a reading: the paper names a byte-wise
+    general-purpose coder from a vendor library and says nothing about sub-byte symbols)."""
     pay_off = ora.payload_offset(n, dtype, block)
     p = msg.size - pay_off
     if p <= 0:
@@ -100,7 +103,7 @@ def entropy_encode_message(msg: np.ndarray, n: int, dtype: int, block: int) -> n
 def entropy_decode_message(msg: np.ndarray, n: int, dtype: int, block: int) -> np.ndarray:
     """The receiver's entropy stage: a message shorter than its bitmap implies holds a coded section."""
     pay_off = ora.payload_offset(n, dtype, block)
-    p = payload_bytes_from_bitmap(msg, n, block)
+    p = payload_bytes_from_bitmap(msg, n, block, dtype)
     if msg.size == pay_off + p:
         return msg.copy()
     return np.concatenate([msg[:pay_off], decode(msg[pay_off:], p)])

@@ -113,9 +113,31 @@ def test_message_level_stage_is_lossless_and_never_longer(oracle, dtype, n, bloc
     cache = oracle.cache_init(None, n, dtype)  # from empty caches: a large payload on the first step
     for w in traj:
         msg, wire, pay, chg = oracle.encode(w, cache, dtype, block)
-        assert rans.payload_bytes_from_bitmap(msg, n, block) == pay
+        assert rans.payload_bytes_from_bitmap(msg, n, block, dtype) == pay
         coded = rans.entropy_encode_message(msg, n, dtype, block)
         assert coded.size <= msg.size
         assert np.array_equal(rans.entropy_decode_message(coded, n, dtype, block), msg)
         if pay > 20_000:
             assert coded.size < msg.size - pay // 2  # exponents of Gaussian weights compress well
+
+
+@pytest.mark.parametrize("n,block", [(70_001, 512), (8192, 64), (1000, 32), (40_003, 4096)])
+def test_message_level_stage_on_packed_fp16_payloads(oracle, n, block):
+    """fp16: the payload holds five bits per exponent, every changed block starting on a byte boundary; the stage
+    codes those bytes as they are.  The receiver's payload length comes from the bitmap with ceil(5 L / 8) bytes
+    per block; the stage stays lossless and never lengthens a message, and still shortens large payloads."""
+    FP16 = 2
+    traj = [wl.as_bits(w) for w in wl.trajectory(n, "fp16", 177 + n, 2, "adam")]
+    cache = oracle.cache_init(None, n, FP16)
+    for w in traj:
+        msg, wire, pay, chg = oracle.encode(w, cache, FP16, block)
+        assert rans.payload_bytes_from_bitmap(msg, n, block, FP16) == pay
+        nb = -(-n // block)
+        assert pay <= (nb - 1) * ((5 * block + 7) // 8) + (5 * (n - (nb - 1) * block) + 7) // 8
+        coded = rans.entropy_encode_message(msg, n, FP16, block)
+        assert coded.size <= msg.size
+        assert np.array_equal(rans.entropy_decode_message(coded, n, FP16, block), msg)
+        if pay > 20_000:
+            # packed exponents of Gaussian weights still compress, if much less than whole bytes do (a byte of the
+            # packed stream mixes parts of two or three exponents at five different phases)
+            assert coded.size < msg.size - pay // 8
