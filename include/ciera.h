@@ -83,7 +83,8 @@ typedef enum ciera_dtype {
                        without gaps (value j of a section at bits [j*w, (j+1)*w), bit i of a section =
                        byte i >> 3, bit i & 7); every changed block of the payload starts on a byte
                        boundary; the caches still hold one byte per value.  Blocks of 32 values and
-                       more; the hashed sender takes it (from 32 values per block), the entropy stage does not. */
+                       more; the hashed sender takes it (from 32 values per block), and so does the entropy stage,
+                       which codes the bytes of the packed payload as they are. */
 } ciera_dtype;
 
 /* One unit = one shard of one tensor.  All offsets are in BYTES from the base pointer of the

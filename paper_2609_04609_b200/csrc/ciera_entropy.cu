@@ -283,7 +283,7 @@ __device__ __forceinline__ bool decode_segment(const uint8_t* coded, uint32_t sn
 
 // Raw payload length of a unit from its bitmap (block-wide; `acc` in shared memory, zeroed and
 // synced by the caller).  The bitmap's bits past the last block and the pad behind it are zero.
-__device__ __forceinline__ uint64_t raw_payload_bytes(const uint8_t* msg, uint64_t N, uint32_t log2b,
+__device__ __forceinline__ uint64_t raw_payload_bytes(const uint8_t* msg, uint64_t N, int dt, uint32_t log2b,
                                                       unsigned long long* acc, uint32_t tid) {
     const uint64_t words = (bitmap_bytes(N, log2b) + 3) >> 2;  // inside the 16-byte padded bitmap
     const uint32_t* bm32 = reinterpret_cast<const uint32_t*>(msg);
@@ -292,12 +292,14 @@ __device__ __forceinline__ uint64_t raw_payload_bytes(const uint8_t* msg, uint64
     cnt = __reduce_add_sync(0xffffffffu, cnt);
     if ((tid & 31u) == 0 && cnt) atomicAdd(acc, (unsigned long long)cnt);
     __syncthreads();
+    // every changed block carries a full block's bytes (one per exponent; fp16: five bits per exponent, rounded up
+    // to whole bytes per block), a changed short last block fewer
     const uint32_t B = 1u << log2b;
-    uint64_t P = *acc << log2b;
+    uint64_t P = *acc * block_payload_bytes(B, dt);
     const uint32_t rem = (uint32_t)(N & (B - 1u));
     if (rem) {
         const uint64_t kb = num_blocks(N, log2b) - 1;
-        if ((msg[kb >> 3] >> (kb & 7u)) & 1u) P -= (B - rem);
+        if ((msg[kb >> 3] >> (kb & 7u)) & 1u) P -= block_payload_bytes(B, dt) - block_payload_bytes(rem, dt);
     }
     return P;
 }
@@ -329,7 +331,7 @@ __device__ __forceinline__ uint32_t block_scan(uint32_t v, uint32_t* scan, uint3
 
 __global__ void __launch_bounds__(kEntThreads, 5)
 entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
-                      uint32_t sm_bytes_per_value, uint32_t log2b, uint8_t* msgs, unsigned long long* wire_bytes,
+                      int dt, uint32_t log2b, uint8_t* msgs, unsigned long long* wire_bytes,
                       uint8_t* scratch_slots, uint32_t* scratch_nw) {
     __shared__ __align__(16) uint8_t s_seg[kEntWarps][kSegment];  // a warp's segment of raw payload
     // the warps' private histograms are needed before the segments are staged, the two small lists of
@@ -343,7 +345,7 @@ entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long 
     const uint32_t unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     const ciera_unit un = units[unit];
     if (un.n_values == 0 || segments_of(un.n_values) > kLongSegs) return;
-    const uint64_t payoff = payload_offset(un.n_values, sm_bytes_per_value, log2b);
+    const uint64_t payoff = payload_offset_of(un.n_values, dt, log2b);
     const uint64_t P = wire_bytes[unit] - payoff;
     // nothing to code; or a length that no sender step reports (shorter than the fixed sections, or more
     // than one payload byte per value): everything below is indexed by P, so such a unit is left alone
@@ -426,22 +428,22 @@ __device__ __forceinline__ LongState* long_state(uint8_t* recs, uint32_t li) { r
 // histogram, the segments and the scratch slots are all indexed by this length, so it must stay
 // inside the unit's slot (the entropy stage takes bf16 and fp32 only: one exponent byte per value,
 // and plans are limited to units whose block counts fit 32 bits).
-__device__ __forceinline__ uint64_t sender_payload(const ciera_unit& un, uint32_t smb, uint32_t log2b,
+__device__ __forceinline__ uint64_t sender_payload(const ciera_unit& un, int dt, uint32_t log2b,
                                                    const unsigned long long* wire_bytes, uint32_t unit, uint64_t& payoff) {
-    payoff = payload_offset(un.n_values, smb, log2b);
+    payoff = payload_offset_of(un.n_values, dt, log2b);
     const uint64_t P = wire_bytes[unit] - payoff;
     return (P <= un.n_values && P < (1ull << 32)) ? P : 0;
 }
 
 __global__ void __launch_bounds__(kEntThreads)
-entropy_long_hist_kernel(const ciera_unit* __restrict__ units, const uint4* __restrict__ chunks, uint32_t smb, uint32_t log2b,
+entropy_long_hist_kernel(const ciera_unit* __restrict__ units, const uint4* __restrict__ chunks, int dt, uint32_t log2b,
                          const uint8_t* msgs, const unsigned long long* wire_bytes, uint8_t* recs) {
     __shared__ uint32_t s_hist[kEntWarps][256];
     const uint4 ch = chunks[blockIdx.x];
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     const ciera_unit un = units[ch.x];
     uint64_t payoff;
-    const uint64_t P = sender_payload(un, smb, log2b, wire_bytes, ch.x, payoff);
+    const uint64_t P = sender_payload(un, dt, log2b, wire_bytes, ch.x, payoff);
     const uint64_t lo = (uint64_t)ch.y * kSegment;
     if (lo >= P) return;
     const uint64_t hi = min(P, lo + (uint64_t)kLongSegs * kSegment);
@@ -455,13 +457,13 @@ entropy_long_hist_kernel(const ciera_unit* __restrict__ units, const uint4* __re
 }
 
 __global__ void __launch_bounds__(kEntThreads)
-entropy_long_model_kernel(const ciera_unit* __restrict__ units, const uint32_t* __restrict__ long_units, uint32_t smb,
+entropy_long_model_kernel(const ciera_unit* __restrict__ units, const uint32_t* __restrict__ long_units, int dt,
                           uint32_t log2b, const unsigned long long* wire_bytes, uint8_t* recs) {
     __shared__ uint32_t s_h[256];
     __shared__ uint16_t s_f[256];
     const uint32_t li = blockIdx.x, tid = threadIdx.x, unit = long_units[li];
     uint64_t payoff;
-    const uint64_t P = sender_payload(units[unit], smb, log2b, wire_bytes, unit, payoff);
+    const uint64_t P = sender_payload(units[unit], dt, log2b, wire_bytes, unit, payoff);
     if (tid == 0) {
         LongState* st = long_state(recs, li);
         st->total = 0;
@@ -477,7 +479,7 @@ entropy_long_model_kernel(const ciera_unit* __restrict__ units, const uint32_t* 
 
 __global__ void __launch_bounds__(kEntThreads)
 entropy_long_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
-                           const uint4* __restrict__ chunks, uint32_t smb, uint32_t log2b, const uint8_t* msgs,
+                           const uint4* __restrict__ chunks, int dt, uint32_t log2b, const uint8_t* msgs,
                            const unsigned long long* wire_bytes, uint8_t* recs, uint8_t* scratch_slots,
                            uint32_t* scratch_nw) {
     __shared__ __align__(16) uint8_t s_seg[kEntWarps][kSegment];
@@ -488,7 +490,7 @@ entropy_long_encode_kernel(const ciera_unit* __restrict__ units, const unsigned 
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     const ciera_unit un = units[ch.x];
     uint64_t payoff;
-    const uint64_t P = sender_payload(un, smb, log2b, wire_bytes, ch.x, payoff);
+    const uint64_t P = sender_payload(un, dt, log2b, wire_bytes, ch.x, payoff);
     if ((uint64_t)ch.y * kSegment >= P) return;
     const uint32_t nseg = (uint32_t)segments_of(P);
     const uint32_t g_end = min(nseg, ch.y + kLongSegs);
@@ -515,14 +517,14 @@ entropy_long_encode_kernel(const ciera_unit* __restrict__ units, const unsigned 
 // offset of every segment into the scratch
 __global__ void __launch_bounds__(kEntThreads)
 entropy_long_layout_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
-                           const uint32_t* __restrict__ long_units, uint32_t smb, uint32_t log2b, uint8_t* msgs,
+                           const uint32_t* __restrict__ long_units, int dt, uint32_t log2b, uint8_t* msgs,
                            unsigned long long* wire_bytes, uint8_t* recs, const uint32_t* scratch_nw,
                            uint32_t* scratch_off) {
     __shared__ uint32_t s_scan[kEntWarps];
     const uint32_t li = blockIdx.x, tid = threadIdx.x, unit = long_units[li];
     const ciera_unit un = units[unit];
     uint64_t payoff;
-    const uint64_t P = sender_payload(un, smb, log2b, wire_bytes, unit, payoff);
+    const uint64_t P = sender_payload(un, dt, log2b, wire_bytes, unit, payoff);
     if (P == 0) return;
     const uint32_t nseg = (uint32_t)segments_of(P);
     LongState* st = long_state(recs, li);
@@ -551,7 +553,7 @@ entropy_long_layout_kernel(const ciera_unit* __restrict__ units, const unsigned 
 
 __global__ void __launch_bounds__(kEntThreads)
 entropy_long_copy_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
-                         const uint4* __restrict__ chunks, uint32_t smb, uint32_t log2b, uint8_t* msgs, uint8_t* recs,
+                         const uint4* __restrict__ chunks, int dt, uint32_t log2b, uint8_t* msgs, uint8_t* recs,
                          const uint8_t* scratch_slots, const uint32_t* scratch_nw, const uint32_t* scratch_off) {
     const uint4 ch = chunks[blockIdx.x];
     const LongState* st = long_state(recs, ch.z);
@@ -559,7 +561,7 @@ entropy_long_copy_kernel(const ciera_unit* __restrict__ units, const unsigned lo
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     const ciera_unit un = units[ch.x];
     const uint32_t nseg = st->nseg;
-    uint8_t* data = msgs + un.msg_off + payload_offset(un.n_values, smb, log2b) + 512 + 4ull * nseg;
+    uint8_t* data = msgs + un.msg_off + payload_offset_of(un.n_values, dt, log2b) + 512 + 4ull * nseg;
     const unsigned long long slot0 = seg_base[ch.x];
     const uint32_t g_end = min(nseg, ch.y + kLongSegs);
     for (uint32_t g = ch.y + warp; g < g_end; g += kEntWarps) {
@@ -588,7 +590,7 @@ __device__ __forceinline__ void raise_corrupt(int32_t* status) {
 }
 
 __global__ void __launch_bounds__(kEntThreads)
-entropy_decode_kernel(const ciera_unit* __restrict__ units, uint32_t smb, uint32_t log2b, uint8_t* msgs,
+entropy_decode_kernel(const ciera_unit* __restrict__ units, int dt, uint32_t log2b, uint8_t* msgs,
                       unsigned long long* wire_bytes, uint8_t* scratch_raw, int32_t* status) {
     extern __shared__ __align__(16) uint8_t smem_raw[];
     DecodeShared& sh = *reinterpret_cast<DecodeShared*>(smem_raw);
@@ -597,13 +599,13 @@ entropy_decode_kernel(const ciera_unit* __restrict__ units, uint32_t smb, uint32
     const uint64_t N = un.n_values;
     if (N == 0 || segments_of(N) > kLongSegs) return;
     uint8_t* const msg = msgs + un.msg_off;
-    const uint64_t payoff = payload_offset(N, smb, log2b);
+    const uint64_t payoff = payload_offset_of(N, dt, log2b);
     if (tid == 0) {
         sh.changed = 0;
         sh.bad = 0;
     }
     __syncthreads();
-    const uint64_t P = raw_payload_bytes(msg, N, log2b, &sh.changed, tid);
+    const uint64_t P = raw_payload_bytes(msg, N, dt, log2b, &sh.changed, tid);
     const uint64_t wire = wire_bytes[unit];
     if (P == 0 || wire == payoff + P) return;  // nothing travelled, or the raw form did
     const uint64_t C = wire - payoff;
@@ -658,7 +660,7 @@ entropy_decode_kernel(const ciera_unit* __restrict__ units, uint32_t smb, uint32
 // longer units: layout (one block per unit), segments and restore (grids over chunks)
 __global__ void __launch_bounds__(kEntThreads)
 entropy_long_parse_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
-                          const uint32_t* __restrict__ long_units, uint32_t smb, uint32_t log2b, const uint8_t* msgs,
+                          const uint32_t* __restrict__ long_units, int dt, uint32_t log2b, const uint8_t* msgs,
                           const unsigned long long* wire_bytes, uint8_t* recs, uint32_t* scratch_off, uint32_t* scratch_nw,
                           int32_t* status) {
     __shared__ uint32_t s_scan[kEntWarps];
@@ -676,8 +678,8 @@ entropy_long_parse_kernel(const ciera_unit* __restrict__ units, const unsigned l
     }
     __syncthreads();
     const uint8_t* msg = msgs + un.msg_off;
-    const uint64_t payoff = payload_offset(N, smb, log2b);
-    const uint64_t P = raw_payload_bytes(msg, N, log2b, &s_changed, tid);
+    const uint64_t payoff = payload_offset_of(N, dt, log2b);
+    const uint64_t P = raw_payload_bytes(msg, N, dt, log2b, &s_changed, tid);
     const uint64_t wire = wire_bytes[unit];
     if (P == 0 || wire == payoff + P) return;
     const uint64_t C = wire - payoff;
@@ -718,7 +720,7 @@ entropy_long_parse_kernel(const ciera_unit* __restrict__ units, const unsigned l
 
 __global__ void __launch_bounds__(kEntThreads)
 entropy_long_decode_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
-                           const uint4* __restrict__ chunks, uint32_t smb, uint32_t log2b, const uint8_t* msgs,
+                           const uint4* __restrict__ chunks, int dt, uint32_t log2b, const uint8_t* msgs,
                            uint8_t* recs, const uint32_t* scratch_off, const uint32_t* scratch_nw, uint8_t* scratch_raw,
                            int32_t* status) {
     extern __shared__ __align__(16) uint8_t smem_raw[];
@@ -730,7 +732,7 @@ entropy_long_decode_kernel(const ciera_unit* __restrict__ units, const unsigned 
     const ciera_unit un = units[ch.x];
     const uint64_t P = st->P;
     const uint32_t nseg = st->nseg;
-    const uint8_t* pay = msgs + un.msg_off + payload_offset(un.n_values, smb, log2b);
+    const uint8_t* pay = msgs + un.msg_off + payload_offset_of(un.n_values, dt, log2b);
     sh.f[tid] = reinterpret_cast<const uint16_t*>(pay)[tid];
     if (tid == 0) sh.bad = 0;
     __syncthreads();
@@ -759,7 +761,7 @@ entropy_long_decode_kernel(const ciera_unit* __restrict__ units, const unsigned 
 }
 
 __global__ void __launch_bounds__(kEntThreads)
-entropy_long_restore_kernel(const ciera_unit* __restrict__ units, const uint4* __restrict__ chunks, uint32_t smb,
+entropy_long_restore_kernel(const ciera_unit* __restrict__ units, const uint4* __restrict__ chunks, int dt,
                             uint32_t log2b, uint8_t* msgs, unsigned long long* wire_bytes, const uint8_t* recs_c,
                             const uint8_t* scratch_raw) {
     const uint4 ch = chunks[blockIdx.x];
@@ -771,7 +773,7 @@ entropy_long_restore_kernel(const ciera_unit* __restrict__ units, const uint4* _
     const uint64_t lo = (uint64_t)ch.y * kSegment;
     if (lo >= P) return;
     const uint64_t hi = min(P, lo + (uint64_t)kLongSegs * kSegment);
-    const uint64_t payoff = payload_offset(un.n_values, smb, log2b);
+    const uint64_t payoff = payload_offset_of(un.n_values, dt, log2b);
     uint8_t* pay = msgs + un.msg_off + payoff;
     const uint8_t* raw = scratch_raw + un.cache_off;
     for (uint64_t i = lo + (uint64_t)tid * 16; i < hi; i += (uint64_t)kEntThreads * 16) {
@@ -813,7 +815,6 @@ static int check_entropy_args(const ciera_plan* p, const void* messages_dev, con
                               const void* scratch_dev) {
     if (!p) return CIERA_ERR_INVALID_ARG;
     if (!p->tiles.empty() && !p->tiles_dev) return CIERA_ERR_NOT_BOUND;
-    if (p->dtype == CIERA_FP16) return CIERA_ERR_UNSUPPORTED;
     if (p->tiles.empty()) return CIERA_OK;
     if (!messages_dev || !wire_bytes_dev || !scratch_dev) return CIERA_ERR_INVALID_ARG;
     if (misaligned16(messages_dev) || misaligned16(scratch_dev) || ((uintptr_t)wire_bytes_dev & 7u))
@@ -832,12 +833,12 @@ extern "C" int ciera_entropy_encode(const ciera_plan* p, void* messages_dev, uin
     uint32_t* off = (uint32_t*)(base + L.off);
     uint8_t* recs = base + L.recs;
     uint8_t* slots = base + L.body;
-    const uint32_t smb = p->dtype == CIERA_BF16 ? 1u : 3u;
+    const int dt = p->dtype;
     uint8_t* msgs = (uint8_t*)messages_dev;
     unsigned long long* wire = (unsigned long long*)wire_bytes_dev;
     const uint32_t n_long = (uint32_t)p->ent_long_units.size(), n_chunks = (uint32_t)p->ent_chunks.size();
     if (n_long < p->n_units) {
-        entropy_encode_kernel<<<p->n_units, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, smb, p->log2b, msgs, wire,
+        entropy_encode_kernel<<<p->n_units, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, dt, p->log2b, msgs, wire,
                                                                  slots, nw);
         count_launch();
         if ((rc = check_launch())) return rc;
@@ -845,15 +846,15 @@ extern "C" int ciera_entropy_encode(const ciera_plan* p, void* messages_dev, uin
     if (n_long) {
         cudaError_t e = cudaMemsetAsync(recs, 0, (size_t)n_long * kLongRec, s);  // the counts start at zero
         if (e != cudaSuccess) return record_cuda_error(e);
-        entropy_long_hist_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->ent_chunks_dev, smb, p->log2b, msgs, wire,
+        entropy_long_hist_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->ent_chunks_dev, dt, p->log2b, msgs, wire,
                                                                   recs);
-        entropy_long_model_kernel<<<n_long, kEntThreads, 0, s>>>(p->units_dev, p->ent_long_units_dev, smb, p->log2b, wire,
+        entropy_long_model_kernel<<<n_long, kEntThreads, 0, s>>>(p->units_dev, p->ent_long_units_dev, dt, p->log2b, wire,
                                                                  recs);
-        entropy_long_encode_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_chunks_dev, smb,
+        entropy_long_encode_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_chunks_dev, dt,
                                                                     p->log2b, msgs, wire, recs, slots, nw);
-        entropy_long_layout_kernel<<<n_long, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_long_units_dev, smb,
+        entropy_long_layout_kernel<<<n_long, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_long_units_dev, dt,
                                                                   p->log2b, msgs, wire, recs, nw, off);
-        entropy_long_copy_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_chunks_dev, smb,
+        entropy_long_copy_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_chunks_dev, dt,
                                                                   p->log2b, msgs, recs, slots, nw, off);
         for (int i = 0; i < 5; ++i) count_launch();
         if ((rc = check_launch())) return rc;
@@ -886,22 +887,22 @@ extern "C" int ciera_entropy_decode(const ciera_plan* p, void* messages_dev, uin
     uint32_t* off = (uint32_t*)(base + L.off);
     uint8_t* recs = base + L.recs;
     uint8_t* raw = base + L.body;
-    const uint32_t smb = p->dtype == CIERA_BF16 ? 1u : 3u;
+    const int dt = p->dtype;
     uint8_t* msgs = (uint8_t*)messages_dev;
     unsigned long long* wire = (unsigned long long*)wire_bytes_dev;
     const uint32_t n_long = (uint32_t)p->ent_long_units.size(), n_chunks = (uint32_t)p->ent_chunks.size();
     if (n_long < p->n_units) {
-        entropy_decode_kernel<<<p->n_units, kEntThreads, sizeof(DecodeShared), s>>>(p->units_dev, smb, p->log2b, msgs, wire,
+        entropy_decode_kernel<<<p->n_units, kEntThreads, sizeof(DecodeShared), s>>>(p->units_dev, dt, p->log2b, msgs, wire,
                                                                                    raw, status_dev);
         count_launch();
         if ((rc = check_launch())) return rc;
     }
     if (n_long) {
-        entropy_long_parse_kernel<<<n_long, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_long_units_dev, smb,
+        entropy_long_parse_kernel<<<n_long, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_long_units_dev, dt,
                                                                  p->log2b, msgs, wire, recs, off, nw, status_dev);
         entropy_long_decode_kernel<<<n_chunks, kEntThreads, sizeof(DecodeShared), s>>>(
-            p->units_dev, p->seg_base_dev, p->ent_chunks_dev, smb, p->log2b, msgs, recs, off, nw, raw, status_dev);
-        entropy_long_restore_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->ent_chunks_dev, smb, p->log2b, msgs,
+            p->units_dev, p->seg_base_dev, p->ent_chunks_dev, dt, p->log2b, msgs, recs, off, nw, raw, status_dev);
+        entropy_long_restore_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->ent_chunks_dev, dt, p->log2b, msgs,
                                                                      wire, recs, raw);
         for (int i = 0; i < 3; ++i) count_launch();
         if ((rc = check_launch())) return rc;

@@ -12,9 +12,9 @@ from paper_2609_04609_b200 import workloads as wl
 pytestmark = pytest.mark.gpu
 
 DEV = "cuda:0"
-WDT = {0: np.uint16, 1: np.uint32}
-VB = {0: 2, 1: 4}
-NAME = {0: "bf16", 1: "fp32"}
+WDT = {0: np.uint16, 1: np.uint32, 2: np.uint16}
+VB = {0: 2, 1: 4, 2: 2}
+NAME = {0: "bf16", 1: "fp32", 2: "fp16"}
 RAGGED = [0, 1, 5, 31, 33, 100, 511, 513, 4095, 4096, 4097, 8191, 8193, 20000, 3 * 8192 + 77, 70001, 140_000]
 
 
@@ -104,6 +104,22 @@ def test_entropy_stage_reduced_moe_layer(rt, dtype):
     traj = [wl.as_bits(w) for w in wl.trajectory(n, NAME[dtype], 4, 2, "clustered", f=0.3)]
     coded = _run(rt, sizes, 4, dtype, 512, traj, from_zero=False)
     assert coded > 0
+
+
+@pytest.mark.parametrize("block", [32, 64, 512, 4096])
+def test_entropy_stage_fp16(rt, block):
+    """fp16: the stage codes the bytes of the packed five-bit exponents; ragged units from empty caches (large
+    payloads), a reduced MoE layer under the clustered update, and a unit long enough for the chain of launches."""
+    n = rt[1].LayerCodec.from_tensors(RAGGED, 1, "fp16", block, DEV).weights_bytes // 2
+    traj = [wl.as_bits(w) for w in wl.trajectory(n, "fp16", 140 + block, 2, "adam")]
+    assert _run(rt, RAGGED, 1, 2, block, [traj[0]] + traj, from_zero=True) > 0
+    sizes = [r * c for r, c in wl.olmoe_layer_shapes(1)] + [700_001]
+    n = rt[1].LayerCodec.from_tensors(sizes, 4, "fp16", block, DEV).weights_bytes // 2
+    traj = [wl.as_bits(w) for w in wl.trajectory(n, "fp16", 9 + block, 2, "clustered", f=0.3)]
+    _run(rt, sizes, 4, 2, block, traj, from_zero=False)
+    n = rt[1].LayerCodec.from_tensors([700_001, 3000], 1, "fp16", block, DEV).weights_bytes // 2
+    w = wl.as_bits(next(iter(wl.trajectory(n, "fp16", 11 + block, 0, "adam"))))
+    assert _run(rt, [700_001, 3000], 1, 2, block, [w, w], from_zero=True) > 0
 
 
 def test_entropy_stage_unit_of_many_segments(rt):
