@@ -82,8 +82,8 @@ typedef enum ciera_dtype {
                        wire its exponents take 5 bits and its sign-plus-mantissa 11 bits each, packed
                        without gaps (value j of a section at bits [j*w, (j+1)*w), bit i of a section =
                        byte i >> 3, bit i & 7); every changed block of the payload starts on a byte
-                       boundary; the caches still hold one byte per value.  Blocks of 32 values and
-                       more; the hashed sender takes it (from 32 values per block), and so does the entropy stage,
+                       boundary; the caches still hold one byte per value.  Blocks of 16 values and
+                       more; the hashed sender takes it too, and so does the entropy stage,
                        which codes the bytes of the packed payload as they are. */
 } ciera_dtype;
 
@@ -225,7 +225,7 @@ CIERA_API int ciera_encode_noalloc(const ciera_plan* plan, const void* weights_d
  * H_i = mix(L + sum_j mix(s_i + (j + 1) * g_i + x_j)) mod 2^64, Hash128 = (H_1, H_2) with
  * s_1 = 0, g_1 = 0x9E3779B97F4A7C15 (the generator's increment), s_2 = 0x6A09E667F3BCC908,
  * g_2 = 0xD1342543DE82EF95; stored as two little-endian 64-bit words per block.
- * Blocks of 16 values and more only (fp16: 32 and more; CIERA_ERR_UNSUPPORTED otherwise).  The hash is taken
+ * Blocks of 16 values and more only (CIERA_ERR_UNSUPPORTED otherwise).  The hash is taken
  * over the exponents as the caches hold them, one byte each, for every precision. */
 
 /* Bytes of a HashCache for the whole plan (16 per block; units in table order), the offset of a

@@ -382,7 +382,7 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
     constexpr int VB = Traits<DT>::kValueBytes;
     constexpr int SMB = Traits<DT>::kSmBytes;  // (not used for fp16)
     constexpr bool kHalf = DT == CIERA_FP16;    // packed sections: see Piece<CIERA_FP16>
-    static_assert(!(kHalf && FINE), "fp16 takes blocks of 32 values and more");
+    static_assert(!(kHalf && FINE), "fp16 takes blocks of 16 values and more");
     using Cfg = DecodeCfg<DT, FINE>;
     constexpr int S = Cfg::kStages;
     constexpr int kDecRing = Cfg::kRing;

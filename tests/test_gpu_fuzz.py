@@ -44,7 +44,7 @@ def _random_case(seed):
     dtype = int(rng.integers(0, 3))
     block = int(rng.choice(BLOCKS))
     if dtype == 2:
-        block = max(block, 32)  # fp16: blocks of 32 values and more
+        block = max(block, 16)  # fp16: blocks of 16 values and more
     return rng, sizes, shards, dtype, block
 
 
@@ -91,7 +91,6 @@ def test_random_tables_full_step(rt, seed):
 def test_random_tables_hashed_sender_and_entropy_stage(rt, seed):
     ciera, runtime = rt
     rng, sizes, shards, dtype, block = _random_case(5000 + seed)
-    dtype = dtype % 2  # the hashed sender and the entropy stage take bf16 and fp32
     block = max(block, 16)
     codec = guard(runtime.LayerCodec.from_tensors(sizes, shards, NAME[dtype], block, DEV, slack=256))
     units = codec.units

@@ -124,7 +124,7 @@ def test_hashed_rejects_fine_blocks(rt):
     assert e.value.status == ciera.ERR_UNSUPPORTED
 
 
-@pytest.mark.parametrize("block", [32, 64, 128, 256, 512, 1024, 4096])
+@pytest.mark.parametrize("block", [16, 32, 64, 128, 256, 512, 1024, 4096])
 def test_hashed_fp16_ragged_units(rt, block):
     """fp16 through the hashed sender (5-bit exponents and 11-bit sign-plus-mantissa packed on the wire, the
     hash taken over the exponents one byte each, as the caches hold them): ragged units, random bit patterns."""

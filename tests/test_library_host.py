@@ -85,7 +85,7 @@ def test_plan_tile_table(ciera):
     """Every unit is cut into tiles of 8192 values; the table lists short units (<= 32 tiles) first, longest
     first and otherwise in table order, then the longer units; empty units have no tiles."""
     T = 8192
-    sizes = [0, 5, T, T + 1, 3 * T + 17, 0, 40000, 40 * T + 3, 33 * T]
+    sizes = [0, 5, T, T + 1, 3 * T + 17, 0, 40000, 40 * T + 3, 33 * T, 13 * T - 5]
     units, wb, cb, mb = layout_units(sizes, 1, 4, lambda n: ciera.message_capacity(n, 1, 64))
     p = ciera.Plan(units, 1, 64)
     ntiles = [-(-n // T) for n in sizes]
@@ -114,26 +114,26 @@ def test_plan_tile_table(ciera):
     base = np.concatenate([[0], np.cumsum(nblocks)])
     assert [ciera.unit_hash_offset(p, u) for u in range(len(sizes))] == [16 * int(b) for b in base[:-1]]
     assert p.hashed_workspace_bytes == p.workspace_bytes
-    def runs_of(run_tiles):
-        out = []
-        for pas in range(32 // run_tiles):
-            k0 = 0
-            for ui in short:
-                lo = k0 + pas * run_tiles
-                if lo < k0 + ntiles[ui]:
-                    out.append((lo, min(lo + run_tiles, k0 + ntiles[ui])))
-                k0 += ntiles[ui]
-        return out
+    def expected_runs():
+        """Every short unit's first run (all but its last one to four tiles), then every unit's last run."""
+        heads, tails, k0 = [], [], 0
+        for ui in short:
+            nt = ntiles[ui]
+            head = nt if nt <= 4 else (nt - 1) // 4 * 4
+            heads.append((k0, k0 + head))
+            if head < nt:
+                tails.append((k0 + head, k0 + nt))
+            k0 += nt
+        return heads + tails
 
-    # tiles per run: whole units with 16 to 128 values per block (this plan: 64), else 4 (checked on a second plan)
-    runs = runs_of(32)
+    runs = expected_runs()
+    assert any(hi - lo > 4 for lo, hi in runs) and len(runs) > len(short)  # the table has units of more than four tiles
     image = p.host_image()
     got_runs = image[-(8 * len(runs) + 16):-16].view("<u4").reshape(-1, 2)
     assert [tuple(int(x) for x in r) for r in got_runs] == runs
     units512, _, _, _ = layout_units(sizes, 1, 4, lambda n: ciera.message_capacity(n, 1, 512))
-    runs4 = runs_of(4)
-    got4 = ciera.Plan(units512, 1, 512).host_image()[-(8 * len(runs4) + 16):-16].view("<u4").reshape(-1, 2)
-    assert [tuple(int(x) for x in r) for r in got4] == runs4
+    got512 = ciera.Plan(units512, 1, 512).host_image()[-(8 * len(runs) + 16):-16].view("<u4").reshape(-1, 2)
+    assert [tuple(int(x) for x in r) for r in got512] == runs  # the same for every block size
     thash_bytes = (8 * want_tiles + 15) // 16 * 16
     tail = image[-(8 * len(runs) + 16 + thash_bytes):-(8 * len(runs) + 16)][: 8 * want_tiles].view("<u8")
     assert [int(x) for x in tail] == [int(base[t["unit"]]) + int(t["j"]) * (T // 64) for t in img]
