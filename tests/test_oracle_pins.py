@@ -56,6 +56,20 @@ def test_split_fp32_random_and_special_patterns_match_ieee_definition(oracle):
     _check_fields(oracle, np.concatenate([bits, special, grid.astype(np.uint32)]), FP32)
 
 
+def test_split_fp32_every_one_of_the_2_to_32_patterns(tmp_path):
+    """All 2^32 binary32 patterns through the oracle's split and merge against the numeric field definition
+    (frexpf / ldexpf), in a small C program of the test suite built together with the oracle's source: see
+    tests/exhaustive_fp32_fields.c.  About ten seconds on eight cores."""
+    import subprocess
+
+    here = os.path.dirname(os.path.abspath(__file__))
+    exe = str(tmp_path / "exhaustive_fp32_fields")
+    src = [os.path.join(here, "exhaustive_fp32_fields.c"), os.path.join(here, "..", "oracle", "ciera_oracle.c")]
+    subprocess.run(["gcc", "-O2", "-fopenmp", "-o", exe] + src + ["-lm"], check=True)
+    out = subprocess.run([exe], capture_output=True, text=True, timeout=1200)
+    assert out.returncode == 0 and out.stdout.strip() == "ok 4294967296", out.stdout + out.stderr
+
+
 # ------------------------------------------------------------------ hand-worked fixtures
 
 
