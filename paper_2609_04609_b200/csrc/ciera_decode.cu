@@ -503,7 +503,11 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                 unchanged_bytes = unchanged << log2b;
                 const uint32_t span_bytes = lo <= hi ? (hi - lo + 1u) << log2b : 0u;
                 const bool sparse = span_bytes != 0 && 4u * unchanged_bytes <= span_bytes;  // consumers read them
-                by_runs = !sparse && nruns <= 32u && (!kHalf || nbt_ <= 32u);  // (fp16 with more than 32 blocks per tile: the span was faster)
+                // (fp16 with more than 32 blocks per tile: the span was faster.  Runs of less than 512 bytes on
+                // average -- 32 values per block with two thirds of the blocks of a changed segment changed: copies of
+                // 32 to 64 bytes -- cost more than the bytes they save: 0.295 against 0.266 ms per layer with the span;
+                // a limit of 1024 bytes starts to cost with 64 values per block.)
+                by_runs = !sparse && nruns <= 32u && (!kHalf || nbt_ <= 32u) && unchanged_bytes >= nruns * 512u;
             }
 
             if (lane == 0) {
