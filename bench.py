@@ -976,9 +976,33 @@ def e2e(args, layers, wa, wb, world, rank, barrier):
     ms = max_over_ranks(t0.elapsed_time(t1) / steps, world, wa[0].device)
     ok = all(torch.equal(o, (host_b if (steps - 1) % 2 == 0 else host_a)[l]) for l, o in enumerate(host_out))
     nbytes = sum(h.numel() for h in host_a)
+    # what the link alone does on this machine: one layer's bytes in each direction at the same time, nothing else running
+    # (the end-to-end step cannot be faster than this; reported so that its figure can be read against the link)
+    link = None
+    try:
+        up, down = torch.empty_like(wa[0]), wa[0]
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        c0.record(cur)
+        for s in streams:
+            s.wait_event(c0)
+        for _ in range(4):
+            with torch.cuda.stream(streams[0]):
+                up.copy_(host_a[0], non_blocking=True)
+            with torch.cuda.stream(streams[1]):
+                host_out[0].copy_(down, non_blocking=True)
+        for s in streams:
+            cur.wait_stream(s)
+        c1.record(cur)
+        torch.cuda.synchronize()
+        link = 4 * host_a[0].numel() / (c0.elapsed_time(c1) * 1e-3) / 1e9
+    except Exception:
+        pass
     return {"value": whole_job_gbps(world, nbytes, ms), "unit": "GB/s", "ms_per_step": ms, "steps": steps,
             "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": nbytes + 8 * sum(len(c.units) for c in layers),
-            "bit_exact": bool(ok), "api": "ciera_roundtrip_host (pinned host weights in, host weights out)"}
+            "bit_exact": bool(ok), "api": "ciera_roundtrip_host (pinned host weights in, host weights out)",
+            "link_GBps_each_way_both_at_once": link,
+            "frac_of_link": (whole_job_gbps(1, nbytes, ms) / link) if link else None}
 
 
 if __name__ == "__main__":
