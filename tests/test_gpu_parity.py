@@ -149,28 +149,32 @@ def test_change_rate_sweep_mixed_shapes(rt):
         assert stats[0][0] > 0
 
 
-def test_repeated_runs_are_identical(rt):
-    """Same input twice from the same start state: every output byte equal (no order dependence
-    in the look-back)."""
+@pytest.mark.parametrize("dtype,block", [(0, 64), (0, 512), (0, 1), (0, 4096), (1, 8), (1, 256)])
+def test_repeated_runs_are_identical(rt, dtype, block):
+    """Same input three times from the same start state: every output byte equal (no order dependence in the
+    look-back between thread blocks, in the hand-off between runs of tiles or in the dynamic hand-out of work).
+    The table has a unit whose tiles are spread over the thread blocks, units worked through in runs, short ones."""
     ciera, runtime = rt
     outs = []
-    for _ in range(2):
-        codec, table, n = _make(rt, [2_000_000, 300_000, 131072], 2, 0, 64)
+    for _ in range(3):
+        codec, table, n = _make(rt, [2_000_000, 300_000, 131072, 8192 * 13 - 3, 70_001], 2, dtype, block)
         gen = wl.make_generator(31337)
-        w0 = wl.init_weights(n, "bf16", gen)
-        w1 = wl.step_adam_like(w0, gen)
+        w0 = wl.init_weights(n, NAME[dtype], gen)
+        w1 = wl.step_adam_like(w0, gen) if block < 256 else wl.step_clustered(w0, gen, f=0.4)
         codec.init_caches(to_dev_bytes(wl.as_bits(w0), DEV))
         codec.msg_send.zero_()
+        codec.msg_recv.zero_()
         codec.step(to_dev_bytes(wl.as_bits(w1), DEV))
         torch.cuda.synchronize()
         codec.check_status()
         wire = codec.wire_bytes.cpu().numpy()
         ms = codec.msg_send.cpu().numpy()
         used = np.concatenate([ms[int(u["msg_off"]) : int(u["msg_off"]) + int(wb)] for u, wb in zip(codec.units, wire)])
-        outs.append((wire.copy(), used, codec.sender_cache.cpu().numpy().copy(),
-                     codec.weights_out.cpu().numpy().copy()))
-    for a, b in zip(outs[0], outs[1]):
-        assert np.array_equal(a, b)
+        outs.append((wire.copy(), used, codec.changed_blocks.cpu().numpy().copy(), codec.sender_cache.cpu().numpy().copy(),
+                     codec.receiver_cache.cpu().numpy().copy(), codec.weights_out.cpu().numpy().copy()))
+    for other in outs[1:]:
+        for a, b in zip(outs[0], other):
+            assert np.array_equal(a, b)
 
 
 def test_length_check_flags_a_corrupted_message(rt):
