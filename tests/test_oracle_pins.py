@@ -65,7 +65,9 @@ def test_split_fp32_every_one_of_the_2_to_32_patterns(tmp_path):
     here = os.path.dirname(os.path.abspath(__file__))
     exe = str(tmp_path / "exhaustive_fp32_fields")
     src = [os.path.join(here, "exhaustive_fp32_fields.c"), os.path.join(here, "..", "oracle", "ciera_oracle.c")]
-    subprocess.run(["gcc", "-O2", "-fopenmp", "-o", exe] + src + ["-lm"], check=True)
+    built = subprocess.run(["gcc", "-O2", "-fopenmp", "-o", exe] + src + ["-lm"])
+    if built.returncode != 0:  # no OpenMP runtime on this machine: one thread, about a minute
+        subprocess.run(["gcc", "-O2", "-o", exe] + src + ["-lm"], check=True)
     out = subprocess.run([exe], capture_output=True, text=True, timeout=1200)
     assert out.returncode == 0 and out.stdout.strip() == "ok 4294967296", out.stdout + out.stderr
 
