@@ -33,9 +33,16 @@
  *
  * Coded section of a unit (replaces the raw payload when it is strictly shorter, which is how the
  * receiver tells the two apart -- it knows P from the bitmap):
- *   [256 x u16 f[s]] [n_seg x u32: number of 16-bit words of each segment] [segment 0] [segment 1] ...
+ *   [A x u16 f[s]] [n_seg x u32: number of 16-bit words of each segment] [segment 0] [segment 1] ...
  *   segment = [32 x u32 final lane states] [its 16-bit words] [2 zero bytes if their number is odd]
  * all little-endian; every segment starts on a 4-byte boundary of the section.
+ *
+ * Alphabet: Algorithm 1 codes the exponents themselves, {exp[k] | bitmap[k] = 1}.  For bf16 and fp32
+ * an exponent is a byte and the raw payload is the symbol sequence (A = 256 table entries).  An fp16
+ * exponent has five bits: the symbols are the exponents of the changed blocks in order, one per
+ * entry of raw[], all below 32, and only A = 32 table entries travel (the five-bit packing of the raw
+ * payload is undone before and redone after the coder by the caller; "raw length" in the rule above
+ * is then the length of the packed payload, while segments are cut every 4096 SYMBOLS).
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -100,32 +107,37 @@ int rans_encode_step(uint32_t* x, uint32_t f, uint32_t c, uint32_t* word) {
     return emitted;
 }
 
-/* Upper bound on the coded size of P raw bytes (what a caller must be able to hold). */
-uint64_t rans_coded_bound(uint64_t P) {
+/* Upper bound on the coded size of P symbols with A table entries (what a caller must be able to hold). */
+uint64_t rans_coded_bound_alphabet(uint64_t P, uint32_t A) {
     uint64_t nseg = (P + RANS_SEGMENT - 1) / RANS_SEGMENT;
     /* a symbol makes the state grow by at most 12 bits, a word takes 16 away */
-    return 512 + 4 * nseg + nseg * (4 * RANS_LANES + 4) + (P * RANS_PROB_BITS + 15) / 16 * 2;
+    return 2 * (uint64_t)A + 4 * nseg + nseg * (4 * RANS_LANES + 4) + (P * RANS_PROB_BITS + 15) / 16 * 2;
 }
+uint64_t rans_coded_bound(uint64_t P) { return rans_coded_bound_alphabet(P, 256); }
 
 /*
- * Codes raw[0..P) into out (at least rans_coded_bound(P) bytes).  Returns the coded size in
- * bytes, or 0 if P = 0.  The caller compares it with P to decide which form travels.
+ * Codes the symbols raw[0..P), each below A (A = 256 or 32), into out (at least
+ * rans_coded_bound_alphabet(P, A) bytes).  Returns the coded size in bytes, or 0 if P = 0 or a symbol
+ * does not fit the alphabet.  The caller compares it with the raw length to decide which form travels.
  */
-uint64_t rans_encode(const uint8_t* raw, uint64_t P, uint8_t* out) {
-    if (P == 0) return 0;
+uint64_t rans_encode_alphabet(const uint8_t* raw, uint64_t P, uint8_t* out, uint32_t A) {
+    if (P == 0 || (A != 256 && A != 32)) return 0;
     uint64_t h[256] = {0};
-    for (uint64_t i = 0; i < P; ++i) h[raw[i]]++;
+    for (uint64_t i = 0; i < P; ++i) {
+        if (raw[i] >= A) return 0;
+        h[raw[i]]++;
+    }
     uint16_t f[256];
     uint32_t c[256];
     rans_normalise(h, P, f);
     uint32_t run = 0;
-    for (int s = 0; s < 256; ++s) {
+    for (uint32_t s = 0; s < 256; ++s) {
         c[s] = run;
         run += f[s];
-        put16(out + 2 * s, f[s]);
+        if (s < A) put16(out + 2 * s, f[s]);
     }
     uint64_t nseg = (P + RANS_SEGMENT - 1) / RANS_SEGMENT;
-    uint8_t* dir = out + 512;
+    uint8_t* dir = out + 2 * A;
     uint8_t* dst = dir + 4 * nseg;
     uint16_t* words = (uint16_t*)malloc(sizeof(uint16_t) * RANS_SEGMENT);
     for (uint64_t g = 0; g < nseg; ++g) {
@@ -156,17 +168,20 @@ uint64_t rans_encode(const uint8_t* raw, uint64_t P, uint8_t* out) {
     free(words);
     return (uint64_t)(dst - out);
 }
+uint64_t rans_encode(const uint8_t* raw, uint64_t P, uint8_t* out) { return rans_encode_alphabet(raw, P, out, 256); }
 
-/* Decodes a coded section back into raw[0..P).  Returns 0, or -1 if the section is inconsistent
- * (sizes that do not add up to coded_bytes, a table that does not sum to 4096). */
-int rans_decode(const uint8_t* in, uint64_t coded_bytes, uint64_t P, uint8_t* raw) {
+/* Decodes a coded section with A table entries back into the symbols raw[0..P).  Returns 0, or -1 if
+ * the section is inconsistent (sizes that do not add up to coded_bytes, a table that does not sum to
+ * 4096). */
+int rans_decode_alphabet(const uint8_t* in, uint64_t coded_bytes, uint64_t P, uint8_t* raw, uint32_t A) {
+    if (A != 256 && A != 32) return -1;
     if (P == 0) return coded_bytes == 0 ? 0 : -1;
     uint64_t nseg = (P + RANS_SEGMENT - 1) / RANS_SEGMENT;
-    if (coded_bytes < 512 + 4 * nseg) return -1;
+    if (coded_bytes < 2 * (uint64_t)A + 4 * nseg) return -1;
     uint32_t f[256], c[256];
     uint8_t* sym = (uint8_t*)malloc(RANS_PROB_SCALE);
     uint32_t run = 0;
-    for (int s = 0; s < 256; ++s) {
+    for (uint32_t s = 0; s < A; ++s) {
         f[s] = get16(in + 2 * s);
         c[s] = run;
         if (run + f[s] > RANS_PROB_SCALE) {
@@ -180,7 +195,7 @@ int rans_decode(const uint8_t* in, uint64_t coded_bytes, uint64_t P, uint8_t* ra
         free(sym);
         return -1;
     }
-    const uint8_t* dir = in + 512;
+    const uint8_t* dir = in + 2 * A;
     const uint8_t* src = dir + 4 * nseg;
     int rc = 0;
     for (uint64_t g = 0; g < nseg && rc == 0; ++g) {
@@ -225,4 +240,7 @@ int rans_decode(const uint8_t* in, uint64_t coded_bytes, uint64_t P, uint8_t* ra
     if (rc == 0 && (uint64_t)(src - in) != coded_bytes) rc = -1;
     free(sym);
     return rc;
+}
+int rans_decode(const uint8_t* in, uint64_t coded_bytes, uint64_t P, uint8_t* raw) {
+    return rans_decode_alphabet(in, coded_bytes, P, raw, 256);
 }

@@ -121,11 +121,43 @@ def test_message_level_stage_is_lossless_and_never_longer(oracle, dtype, n, bloc
             assert coded.size < msg.size - pay // 2  # exponents of Gaussian weights compress well
 
 
-@pytest.mark.parametrize("n,block", [(70_001, 512), (8192, 64), (1000, 32), (40_003, 4096)])
-def test_message_level_stage_on_packed_fp16_payloads(oracle, n, block):
-    """fp16: the payload holds five bits per exponent, every changed block starting on a byte boundary; the stage
-    codes those bytes as they are.  The receiver's payload length comes from the bitmap with ceil(5 L / 8) bytes
-    per block; the stage stays lossless and never lengthens a message, and still shortens large payloads."""
+def test_five_bit_packing_by_hand():
+    """Exponents 1, 2, 3 of one block: 1 | 2 << 5 | 3 << 10 = 0x0C41, little-endian, one spare bit; two blocks
+    of 3 and 1 values start on byte boundaries."""
+    lens = np.array([3, 1])
+    packed = np.array([0x41, 0x0C, 0x1F], np.uint8)
+    assert rans.unpack_fp16_payload(packed, lens).tolist() == [1, 2, 3, 31]
+    assert rans.pack_fp16_payload(np.array([1, 2, 3, 31], np.uint8), lens).tolist() == [0x41, 0x0C, 0x1F]
+    with pytest.raises(ValueError):
+        rans.unpack_fp16_payload(packed, np.array([3]))  # a byte too many for one block of three
+
+
+def test_the_32_entry_table_is_the_256_entry_one_cut_short():
+    """Symbols below 32: the coded section with 32 table entries is the one with 256 entries without the 224
+    zero entries (same model, same segments), and decodes to the same symbols; a larger symbol is refused."""
+    rng = np.random.default_rng(5)
+    for n in (1, 31, 4096, 4097, 50_000):
+        raw = np.minimum(rng.geometric(0.3, n) + 9, 31).astype(np.uint8)
+        wide, narrow = rans.encode(raw), rans.encode(raw, 32)
+        assert narrow.size == wide.size - 448 == rans.coded_bound(n, 32) - (rans.coded_bound(n) - wide.size)
+        assert np.array_equal(narrow[:64], wide[:64]) and not wide[64:512].any()
+        assert np.array_equal(narrow[64:], wide[512:])
+        assert np.array_equal(rans.decode(narrow, n, 32), raw)
+    with pytest.raises(ValueError):
+        rans.encode(np.array([3, 32], np.uint8), 32)
+    bad = rans.encode(np.full(100, 7, np.uint8), 32)
+    bad[0] ^= 1  # the table no longer sums to 4096
+    with pytest.raises(ValueError):
+        rans.decode(bad, 100, 32)
+
+
+@pytest.mark.parametrize("n,block", [(70_001, 512), (8192, 64), (1000, 32), (40_003, 4096), (5_000, 16)])
+def test_message_level_stage_on_fp16_exponents(oracle, n, block):
+    """fp16: the payload holds five bits per exponent, every changed block starting on a byte boundary.  The
+    symbols the stage codes are the exponents themselves: unpacked they equal the exponent fields of the changed
+    blocks' values (taken with the codec oracle's split), packing them again gives the payload back, and the
+    stage stays lossless, never lengthens a message and shortens large payloads to well under five bits per
+    exponent."""
     FP16 = 2
     traj = [wl.as_bits(w) for w in wl.trajectory(n, "fp16", 177 + n, 2, "adam")]
     cache = oracle.cache_init(None, n, FP16)
@@ -134,10 +166,15 @@ def test_message_level_stage_on_packed_fp16_payloads(oracle, n, block):
         assert rans.payload_bytes_from_bitmap(msg, n, block, FP16) == pay
         nb = -(-n // block)
         assert pay <= (nb - 1) * ((5 * block + 7) // 8) + (5 * (n - (nb - 1) * block) + 7) // 8
+        pay_off = msg.size - pay
+        lens = rans.changed_block_lengths(msg, n, block)
+        symbols = rans.unpack_fp16_payload(msg[pay_off:], lens)
+        exp, _ = oracle.split(w, FP16)
+        flags = np.unpackbits(msg[: -(-nb // 8)], bitorder="little")[:nb].astype(bool)
+        assert np.array_equal(symbols, exp[np.repeat(flags, block)[:n]])
+        assert np.array_equal(rans.pack_fp16_payload(symbols, lens), msg[pay_off:])
         coded = rans.entropy_encode_message(msg, n, FP16, block)
         assert coded.size <= msg.size
         assert np.array_equal(rans.entropy_decode_message(coded, n, FP16, block), msg)
         if pay > 20_000:
-            # packed exponents of Gaussian weights still compress, if much less than whole bytes do (a byte of the
-            # packed stream mixes parts of two or three exponents at five different phases)
-            assert coded.size < msg.size - pay // 8
+            assert coded.size < msg.size - pay // 3  # under 3.4 of the 5 bits
