@@ -84,7 +84,8 @@ typedef enum ciera_dtype {
                        byte i >> 3, bit i & 7); every changed block of the payload starts on a byte
                        boundary; the caches still hold one byte per value.  Blocks of 16 values and
                        more; the hashed sender takes it too, and so does the entropy stage,
-                       which codes the bytes of the packed payload as they are. */
+                       which codes the 5-bit exponents as symbols of their own (it undoes the
+                       packing first; 32 table entries travel instead of 256). */
 } ciera_dtype;
 
 /* One unit = one shard of one tensor.  All offsets are in BYTES from the base pointer of the
@@ -315,10 +316,12 @@ CIERA_API int ciera_roundtrip_host(const ciera_plan* plan, const void* weights_h
  * payload in place (the receiver knows the raw length from the bitmap: a message of exactly that
  * length carries the raw form) and sets wire_bytes back to the raw length, so that ciera_decode
  * sees what the sender step had written.  The paper names a vendor library whose format is not
- * public; coder and layout are this library's own: static model per unit (256 symbols,
- * probabilities in 1/4096), 32-bit rANS states with 16-bit words, segments of 4096 payload bytes
- * coded by 32 interleaved coders each; coded section = [256 x u16 frequencies][per segment a u32
- * word count][segments: 32 x u32 final states, the words, 2 zero bytes if their number is odd].
+ * public; coder and layout are this library's own: static model per unit (a symbol = an exponent:
+ * 256 symbols for bf16 and fp32, 32 for fp16, whose 5-bit packing is undone before and redone after
+ * the coder; probabilities in 1/4096), 32-bit rANS states with 16-bit words, segments of 4096
+ * symbols coded by 32 interleaved coders each; coded section = [256 or 32 x u16 frequencies][per
+ * segment a u32 word count][segments: 32 x u32 final states, the words, 2 zero bytes if their
+ * number is odd].
  *   messages_dev    device, in/out
  *   wire_bytes_dev  device, n_units x uint64, in/out
  *   scratch_dev     device, ciera_plan_entropy_scratch_bytes(plan) bytes, 16-byte aligned; contents

@@ -14,9 +14,14 @@
 // 32 interleaved coders (lane l owns bytes 32 t + l).  The encoder walks the steps t backwards and
 // appends the words its lanes emit (ballot, rank = lanes below); the decoder walks forwards and
 // takes the words from the end of the list backwards, so neither side needs per-lane streams.
-// Coded section: [256 x u16 f] [n_seg x u32 word counts] [segments: 32 x u32 final states, words,
+// Coded section: [A x u16 f] [n_seg x u32 word counts] [segments: 32 x u32 final states, words,
 // 2 zero bytes if the count is odd].  It replaces the raw payload only if strictly shorter; the
 // receiver knows the raw length from the bitmap and so tells the two forms apart by the length.
+// The symbols are the exponents of the changed blocks (Algorithm 1 codes {exp[k] | bitmap[k] = 1}):
+// for bf16 and fp32 the payload's bytes as they are, A = 256 table entries.  For fp16 the five-bit
+// packing of the payload is undone into a scratch first (one symbol per byte, A = 32 entries travel),
+// segments are cut every 4096 symbols, "raw length" above is the packed payload's, and the receiver
+// packs the decoded symbols back into the message.
 //
 // Work split: a unit of up to 64 segments' worth of values (262 144) is done by one thread block from
 // start to end (histogram, model, segments into a scratch, coded form into the message).  Longer
@@ -37,6 +42,8 @@ constexpr uint32_t kLongSegs = 64;  // units with more segment slots than this t
 
 __host__ __device__ inline uint64_t segments_of(uint64_t bytes) { return (bytes + kSegment - 1) / kSegment; }
 __host__ __device__ inline uint32_t segment_bytes(uint32_t nw) { return 4u * 32u + 2u * nw + ((nw & 1u) ? 2u : 0u); }
+// bytes of the frequency table that travels: one u16 per symbol of the alphabet
+__host__ __device__ inline uint32_t model_bytes(int dt) { return dt == CIERA_FP16 ? 64u : 512u; }
 
 // ---------------------------------------------------------------------------------- shared pieces
 
@@ -281,10 +288,11 @@ __device__ __forceinline__ bool decode_segment(const uint8_t* coded, uint32_t sn
     return ok;
 }
 
-// Raw payload length of a unit from its bitmap (block-wide; `acc` in shared memory, zeroed and
-// synced by the caller).  The bitmap's bits past the last block and the pad behind it are zero.
+// Raw payload length Q in bytes and symbol count S of a unit from its bitmap (block-wide; `acc` in shared
+// memory, zeroed and synced by the caller).  The bitmap's bits past the last block and the pad behind it
+// are zero.
 __device__ __forceinline__ uint64_t raw_payload_bytes(const uint8_t* msg, uint64_t N, int dt, uint32_t log2b,
-                                                      unsigned long long* acc, uint32_t tid) {
+                                                      unsigned long long* acc, uint32_t tid, uint64_t& S) {
     const uint64_t words = (bitmap_bytes(N, log2b) + 3) >> 2;  // inside the 16-byte padded bitmap
     const uint32_t* bm32 = reinterpret_cast<const uint32_t*>(msg);
     uint32_t cnt = 0;
@@ -295,13 +303,74 @@ __device__ __forceinline__ uint64_t raw_payload_bytes(const uint8_t* msg, uint64
     // every changed block carries a full block's bytes (one per exponent; fp16: five bits per exponent, rounded up
     // to whole bytes per block), a changed short last block fewer
     const uint32_t B = 1u << log2b;
-    uint64_t P = *acc * block_payload_bytes(B, dt);
+    uint64_t Q = *acc * block_payload_bytes(B, dt);
+    S = *acc << log2b;
     const uint32_t rem = (uint32_t)(N & (B - 1u));
     if (rem) {
         const uint64_t kb = num_blocks(N, log2b) - 1;
-        if ((msg[kb >> 3] >> (kb & 7u)) & 1u) P -= block_payload_bytes(B, dt) - block_payload_bytes(rem, dt);
+        if ((msg[kb >> 3] >> (kb & 7u)) & 1u) {
+            Q -= block_payload_bytes(B, dt) - block_payload_bytes(rem, dt);
+            S -= B - rem;
+        }
     }
-    return P;
+    return Q;
+}
+
+// Symbol count of a sender's payload of Q bytes.  bf16, fp32: a byte each.  fp16: the changed blocks lie one
+// after the other, a full one taking block_payload_bytes(B) bytes, so Q and the last block's bit (a short last
+// block is the only one of another size) give the count.  0 if Q is not such a sum.
+__device__ __forceinline__ uint64_t symbols_of_payload(const uint8_t* msg, uint64_t N, int dt, uint32_t log2b, uint64_t Q) {
+    if (dt != CIERA_FP16) return Q;
+    const uint32_t B = 1u << log2b, full = (uint32_t)block_payload_bytes(B, dt);
+    const uint32_t rem = (uint32_t)(N & (B - 1u));
+    uint64_t tail_bytes = 0, tail_symbols = 0;
+    if (rem) {
+        const uint64_t kb = num_blocks(N, log2b) - 1;
+        if ((msg[kb >> 3] >> (kb & 7u)) & 1u) {
+            tail_bytes = block_payload_bytes(rem, dt);
+            tail_symbols = rem;
+        }
+    }
+    if (Q < tail_bytes || (Q - tail_bytes) % full != 0) return 0;
+    return ((Q - tail_bytes) / full << log2b) + tail_symbols;
+}
+
+// fp16: the symbols [lo, hi) of a payload between their packed form (five bits each, a block starting on a byte
+// boundary at block index x block_payload_bytes(B); all blocks before a short last one are full) and one byte
+// each.  lo is a multiple of 8 and of the block size where that is smaller; hi <= symbol count.  A group of 8
+// symbols is 5 bytes: one thread moves a group.  `sym` is 8-byte aligned.
+__device__ __forceinline__ uint64_t packed_group_offset(uint64_t s0, uint32_t log2b) {
+    const uint32_t B = 1u << log2b;
+    return (s0 >> log2b) * block_payload_bytes(B, CIERA_FP16) + (uint64_t)(((uint32_t)s0 & (B - 1u)) >> 3) * 5u;
+}
+__device__ __forceinline__ void unpack_symbols(const uint8_t* pay, uint8_t* sym, uint32_t log2b, uint64_t lo, uint64_t hi,
+                                               uint32_t tid, uint32_t threads) {
+    const uint32_t group = min(1u << log2b, 8u);
+    for (uint64_t s0 = lo + (uint64_t)tid * group; s0 < hi; s0 += (uint64_t)threads * group) {
+        const uint32_t ns = (uint32_t)min((uint64_t)group, hi - s0), nbytes = (5u * ns + 7u) >> 3;
+        const uint8_t* src = pay + packed_group_offset(s0, log2b);
+        unsigned long long v = 0;
+        for (uint32_t k = 0; k < nbytes; ++k) v |= (unsigned long long)src[k] << (8u * k);
+        if (ns == 8u) {
+            unsigned long long out = 0;
+#pragma unroll
+            for (uint32_t k = 0; k < 8u; ++k) out |= ((v >> (5u * k)) & 31ull) << (8u * k);
+            *reinterpret_cast<unsigned long long*>(sym + s0) = out;
+        } else {
+            for (uint32_t k = 0; k < ns; ++k) sym[s0 + k] = (uint8_t)((v >> (5u * k)) & 31u);
+        }
+    }
+}
+__device__ __forceinline__ void pack_symbols(const uint8_t* sym, uint8_t* pay, uint32_t log2b, uint64_t lo, uint64_t hi,
+                                             uint32_t tid, uint32_t threads) {
+    const uint32_t group = min(1u << log2b, 8u);
+    for (uint64_t s0 = lo + (uint64_t)tid * group; s0 < hi; s0 += (uint64_t)threads * group) {
+        const uint32_t ns = (uint32_t)min((uint64_t)group, hi - s0), nbytes = (5u * ns + 7u) >> 3;
+        unsigned long long v = 0;
+        for (uint32_t k = 0; k < ns; ++k) v |= (unsigned long long)(sym[s0 + k] & 31u) << (5u * k);
+        uint8_t* dst = pay + packed_group_offset(s0, log2b);
+        for (uint32_t k = 0; k < nbytes; ++k) dst[k] = (uint8_t)(v >> (8u * k));
+    }
 }
 
 // Exclusive scan of one value per thread over the block; `scan` holds kEntWarps words.  Returns
@@ -332,8 +401,8 @@ __device__ __forceinline__ uint32_t block_scan(uint32_t v, uint32_t* scan, uint3
 __global__ void __launch_bounds__(kEntThreads, 5)
 entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
                       int dt, uint32_t log2b, uint8_t* msgs, unsigned long long* wire_bytes,
-                      uint8_t* scratch_slots, uint32_t* scratch_nw) {
-    __shared__ __align__(16) uint8_t s_seg[kEntWarps][kSegment];  // a warp's segment of raw payload
+                      uint8_t* scratch_slots, uint32_t* scratch_nw, uint8_t* scratch_sym) {
+    __shared__ __align__(16) uint8_t s_seg[kEntWarps][kSegment];  // a warp's segment of symbols
     // the warps' private histograms are needed before the segments are staged, the two small lists of
     // step 4 after: all of them lie in the first part of s_seg
     uint32_t (*const s_hist)[256] = reinterpret_cast<uint32_t (*)[256]>(&s_seg[0][0]);
@@ -346,18 +415,29 @@ entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long 
     const ciera_unit un = units[unit];
     if (un.n_values == 0 || segments_of(un.n_values) > kLongSegs) return;
     const uint64_t payoff = payload_offset_of(un.n_values, dt, log2b);
-    const uint64_t P = wire_bytes[unit] - payoff;
-    // nothing to code; or a length that no sender step reports (shorter than the fixed sections, or more
-    // than one payload byte per value): everything below is indexed by P, so such a unit is left alone
+    const uint64_t Q = wire_bytes[unit] - payoff;
+    // nothing to code; or a length that no sender step reports (shorter than the fixed sections, more
+    // than one payload byte per value, not a sum of block sizes): everything below is indexed by the
+    // symbol count P, so such a unit is left alone
+    if (Q == 0 || Q > un.n_values) return;
+    const uint64_t P = symbols_of_payload(msgs + un.msg_off, un.n_values, dt, log2b, Q);
     if (P == 0 || P > un.n_values) return;
     uint8_t* const pay = msgs + un.msg_off + payoff;  // 16-byte aligned
     const uint32_t nseg = (uint32_t)segments_of(P);
+    const uint32_t hdr = model_bytes(dt);
+    const uint8_t* src = pay;  // the symbols, one per byte
+    if (dt == CIERA_FP16) {
+        uint8_t* sym = scratch_sym + un.cache_off;
+        unpack_symbols(pay, sym, log2b, 0, P, tid, kEntThreads);
+        src = sym;
+        __syncthreads();
+    }
 
-    // 1. histogram of the raw payload (one private copy per warp), 2. the model
+    // 1. histogram of the symbols (one private copy per warp), 2. the model
     for (uint32_t i = lane; i < 256; i += 32) s_hist[warp][i] = 0;
     if (tid == 0) s_total = 0;
     __syncwarp();
-    histogram_add(s_hist, pay, 0, P, tid);
+    histogram_add(s_hist, src, 0, P, tid);
     __syncthreads();
     {
         uint32_t h = 0;
@@ -373,7 +453,7 @@ entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long 
     const unsigned long long slot0 = seg_base[unit];
     for (uint32_t g = warp; g < nseg; g += kEntWarps) {
         const uint32_t n = (uint32_t)min((uint64_t)kSegment, P - (uint64_t)g * kSegment);
-        const uint32_t nw = encode_segment(pay + (uint64_t)g * kSegment, n, s_seg[warp], s_enc,
+        const uint32_t nw = encode_segment(src + (uint64_t)g * kSegment, n, s_seg[warp], s_enc,
                                            scratch_slots + (slot0 + g) * kSegSlot, lane);
         if (lane == 0) {
             scratch_nw[slot0 + g] = nw;
@@ -383,11 +463,11 @@ entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long 
     __syncthreads();  // every warp is done reading the raw payload and writing its slots
 
     // 4. keep the raw form unless the coded one is strictly shorter; else move it into the message
-    const uint64_t C = 512ull + 4ull * nseg + s_total;
-    if (C >= P) return;
-    reinterpret_cast<uint16_t*>(pay)[tid] = s_f[tid];
-    uint32_t* dir = reinterpret_cast<uint32_t*>(pay + 512);
-    uint8_t* data = pay + 512 + 4ull * nseg;
+    const uint64_t C = (uint64_t)hdr + 4ull * nseg + s_total;
+    if (C >= Q) return;
+    if (tid < hdr / 2u) reinterpret_cast<uint16_t*>(pay)[tid] = s_f[tid];
+    uint32_t* dir = reinterpret_cast<uint32_t*>(pay + hdr);
+    uint8_t* data = pay + hdr + 4ull * nseg;
     // nseg <= kLongSegs <= kEntThreads: one round
     const uint32_t nw = tid < nseg ? scratch_nw[slot0 + tid] : 0u;
     const uint32_t size = tid < nseg ? segment_bytes(nw) : 0u;
@@ -412,44 +492,68 @@ entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long 
 constexpr uint32_t kLongRec = 2048;
 struct LongState {            // at byte 1536 of a long unit's record
     unsigned long long total;   // sender: bytes of all coded segments
-    unsigned long long P;       // raw payload length
+    unsigned long long P;       // receiver: symbols of the raw payload
     uint32_t coded;             // 1: the coded form is (sender) / was (receiver) chosen
     uint32_t bad;               // receiver: a segment did not decode
-    uint32_t nseg;              // segments of the raw payload
+    uint32_t nseg;              // segments of the symbols
     uint32_t pad;
+    unsigned long long Q;       // receiver: raw payload length in bytes (P = its symbols)
 };
 __device__ __forceinline__ uint32_t* long_hist(uint8_t* recs, uint32_t li) { return reinterpret_cast<uint32_t*>(recs + (size_t)li * kLongRec); }
 __device__ __forceinline__ uint16_t* long_model(uint8_t* recs, uint32_t li) { return reinterpret_cast<uint16_t*>(recs + (size_t)li * kLongRec + 1024); }
 __device__ __forceinline__ LongState* long_state(uint8_t* recs, uint32_t li) { return reinterpret_cast<LongState*>(recs + (size_t)li * kLongRec + 1536); }
 
-// raw payload length of a unit on the sender (0: nothing to code).  A reported length that no sender
-// step can have produced -- shorter than the fixed sections, or a payload of more than one byte per
-// value, e.g. the stale word of a unit that an aborted encode never finished -- also gives 0: the
-// histogram, the segments and the scratch slots are all indexed by this length, so it must stay
-// inside the unit's slot (the entropy stage takes bf16 and fp32 only: one exponent byte per value,
-// and plans are limited to units whose block counts fit 32 bits).
-__device__ __forceinline__ uint64_t sender_payload(const ciera_unit& un, int dt, uint32_t log2b,
-                                                   const unsigned long long* wire_bytes, uint32_t unit, uint64_t& payoff) {
+// Symbol count of a unit's payload on the sender (0: nothing to code); Q gets the payload's length in bytes.
+// A reported length that no sender step can have produced -- shorter than the fixed sections, a payload of
+// more than one byte per value, not a sum of block sizes, e.g. the stale word of a unit that an aborted
+// encode never finished -- also gives 0: the histogram, the segments and the scratch slots are all indexed
+// by the symbol count, so it must stay inside the unit's slot (a value has one exponent, and plans are
+// limited to units whose block counts fit 32 bits).
+__device__ __forceinline__ uint64_t sender_payload(const ciera_unit& un, int dt, uint32_t log2b, const uint8_t* msgs,
+                                                   const unsigned long long* wire_bytes, uint32_t unit, uint64_t& payoff,
+                                                   uint64_t& Q) {
     payoff = payload_offset_of(un.n_values, dt, log2b);
-    const uint64_t P = wire_bytes[unit] - payoff;
+    Q = wire_bytes[unit] - payoff;
+    if (Q == 0 || Q > un.n_values || Q >= (1ull << 32)) return 0;
+    const uint64_t P = symbols_of_payload(msgs + un.msg_off, un.n_values, dt, log2b, Q);
     return (P <= un.n_values && P < (1ull << 32)) ? P : 0;
+}
+// where a unit's symbols lie, one per byte: in the message, or (fp16) unpacked in the scratch
+__device__ __forceinline__ const uint8_t* sender_symbols(const ciera_unit& un, int dt, const uint8_t* msgs, uint64_t payoff,
+                                                         const uint8_t* scratch_sym) {
+    return dt == CIERA_FP16 ? scratch_sym + un.cache_off : msgs + un.msg_off + payoff;
+}
+
+// fp16 only: the long units' payloads unpacked into the scratch, a chunk per thread block
+__global__ void __launch_bounds__(kEntThreads)
+entropy_long_unpack_kernel(const ciera_unit* __restrict__ units, const uint4* __restrict__ chunks, int dt, uint32_t log2b,
+                           const uint8_t* msgs, const unsigned long long* wire_bytes, uint8_t* scratch_sym) {
+    const uint4 ch = chunks[blockIdx.x];
+    const ciera_unit un = units[ch.x];
+    uint64_t payoff, Q;
+    const uint64_t P = sender_payload(un, dt, log2b, msgs, wire_bytes, ch.x, payoff, Q);
+    const uint64_t lo = (uint64_t)ch.y * kSegment;
+    if (lo >= P) return;
+    const uint64_t hi = min(P, lo + (uint64_t)kLongSegs * kSegment);
+    unpack_symbols(msgs + un.msg_off + payoff, scratch_sym + un.cache_off, log2b, lo, hi, threadIdx.x, kEntThreads);
 }
 
 __global__ void __launch_bounds__(kEntThreads)
 entropy_long_hist_kernel(const ciera_unit* __restrict__ units, const uint4* __restrict__ chunks, int dt, uint32_t log2b,
-                         const uint8_t* msgs, const unsigned long long* wire_bytes, uint8_t* recs) {
+                         const uint8_t* msgs, const unsigned long long* wire_bytes, uint8_t* recs,
+                         const uint8_t* scratch_sym) {
     __shared__ uint32_t s_hist[kEntWarps][256];
     const uint4 ch = chunks[blockIdx.x];
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     const ciera_unit un = units[ch.x];
-    uint64_t payoff;
-    const uint64_t P = sender_payload(un, dt, log2b, wire_bytes, ch.x, payoff);
+    uint64_t payoff, Q;
+    const uint64_t P = sender_payload(un, dt, log2b, msgs, wire_bytes, ch.x, payoff, Q);
     const uint64_t lo = (uint64_t)ch.y * kSegment;
     if (lo >= P) return;
     const uint64_t hi = min(P, lo + (uint64_t)kLongSegs * kSegment);
     for (uint32_t i = lane; i < 256; i += 32) s_hist[warp][i] = 0;
     __syncwarp();
-    histogram_add(s_hist, msgs + un.msg_off + payoff, lo, hi, tid);
+    histogram_add(s_hist, sender_symbols(un, dt, msgs, payoff, scratch_sym), lo, hi, tid);
     __syncthreads();
     uint32_t h = 0;
     for (int w = 0; w < kEntWarps; ++w) h += s_hist[w][tid];
@@ -458,12 +562,12 @@ entropy_long_hist_kernel(const ciera_unit* __restrict__ units, const uint4* __re
 
 __global__ void __launch_bounds__(kEntThreads)
 entropy_long_model_kernel(const ciera_unit* __restrict__ units, const uint32_t* __restrict__ long_units, int dt,
-                          uint32_t log2b, const unsigned long long* wire_bytes, uint8_t* recs) {
+                          uint32_t log2b, const uint8_t* msgs, const unsigned long long* wire_bytes, uint8_t* recs) {
     __shared__ uint32_t s_h[256];
     __shared__ uint16_t s_f[256];
     const uint32_t li = blockIdx.x, tid = threadIdx.x, unit = long_units[li];
-    uint64_t payoff;
-    const uint64_t P = sender_payload(units[unit], dt, log2b, wire_bytes, unit, payoff);
+    uint64_t payoff, Q;
+    const uint64_t P = sender_payload(units[unit], dt, log2b, msgs, wire_bytes, unit, payoff, Q);
     if (tid == 0) {
         LongState* st = long_state(recs, li);
         st->total = 0;
@@ -481,7 +585,7 @@ __global__ void __launch_bounds__(kEntThreads)
 entropy_long_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
                            const uint4* __restrict__ chunks, int dt, uint32_t log2b, const uint8_t* msgs,
                            const unsigned long long* wire_bytes, uint8_t* recs, uint8_t* scratch_slots,
-                           uint32_t* scratch_nw) {
+                           uint32_t* scratch_nw, const uint8_t* scratch_sym) {
     __shared__ __align__(16) uint8_t s_seg[kEntWarps][kSegment];
     __shared__ uint16_t s_f[256];
     __shared__ uint4 s_enc[256];
@@ -489,8 +593,8 @@ entropy_long_encode_kernel(const ciera_unit* __restrict__ units, const unsigned 
     const uint4 ch = chunks[blockIdx.x];
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     const ciera_unit un = units[ch.x];
-    uint64_t payoff;
-    const uint64_t P = sender_payload(un, dt, log2b, wire_bytes, ch.x, payoff);
+    uint64_t payoff, Q;
+    const uint64_t P = sender_payload(un, dt, log2b, msgs, wire_bytes, ch.x, payoff, Q);
     if ((uint64_t)ch.y * kSegment >= P) return;
     const uint32_t nseg = (uint32_t)segments_of(P);
     const uint32_t g_end = min(nseg, ch.y + kLongSegs);
@@ -498,7 +602,7 @@ entropy_long_encode_kernel(const ciera_unit* __restrict__ units, const unsigned 
     if (tid == 0) s_total = 0;
     __syncthreads();
     encoder_tables(s_f, s_enc, tid);
-    const uint8_t* pay = msgs + un.msg_off + payoff;
+    const uint8_t* pay = sender_symbols(un, dt, msgs, payoff, scratch_sym);
     const unsigned long long slot0 = seg_base[ch.x];
     for (uint32_t g = ch.y + warp; g < g_end; g += kEntWarps) {
         const uint32_t n = (uint32_t)min((uint64_t)kSegment, P - (uint64_t)g * kSegment);
@@ -523,18 +627,19 @@ entropy_long_layout_kernel(const ciera_unit* __restrict__ units, const unsigned 
     __shared__ uint32_t s_scan[kEntWarps];
     const uint32_t li = blockIdx.x, tid = threadIdx.x, unit = long_units[li];
     const ciera_unit un = units[unit];
-    uint64_t payoff;
-    const uint64_t P = sender_payload(un, dt, log2b, wire_bytes, unit, payoff);
+    uint64_t payoff, Q;
+    const uint64_t P = sender_payload(un, dt, log2b, msgs, wire_bytes, unit, payoff, Q);
     if (P == 0) return;
     const uint32_t nseg = (uint32_t)segments_of(P);
+    const uint32_t hdr = model_bytes(dt);
     LongState* st = long_state(recs, li);
-    const uint64_t C = 512ull + 4ull * nseg + st->total;
-    if (C >= P) return;
+    const uint64_t C = (uint64_t)hdr + 4ull * nseg + st->total;
+    if (C >= Q) return;
     uint8_t* pay = msgs + un.msg_off + payoff;
-    reinterpret_cast<uint16_t*>(pay)[tid] = long_model(recs, li)[tid];
-    uint32_t* dir = reinterpret_cast<uint32_t*>(pay + 512);
+    if (tid < hdr / 2u) reinterpret_cast<uint16_t*>(pay)[tid] = long_model(recs, li)[tid];
+    uint32_t* dir = reinterpret_cast<uint32_t*>(pay + hdr);
     const unsigned long long slot0 = seg_base[unit];
-    uint32_t carry = 0;  // C < P < 2^32: offsets fit
+    uint32_t carry = 0;  // C < Q < 2^32: offsets fit
     for (uint32_t g0 = 0; g0 < nseg; g0 += kEntThreads) {
         const uint32_t g = g0 + tid;
         const uint32_t nw = g < nseg ? scratch_nw[slot0 + g] : 0u;
@@ -561,7 +666,7 @@ entropy_long_copy_kernel(const ciera_unit* __restrict__ units, const unsigned lo
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     const ciera_unit un = units[ch.x];
     const uint32_t nseg = st->nseg;
-    uint8_t* data = msgs + un.msg_off + payload_offset_of(un.n_values, dt, log2b) + 512 + 4ull * nseg;
+    uint8_t* data = msgs + un.msg_off + payload_offset_of(un.n_values, dt, log2b) + model_bytes(dt) + 4ull * nseg;
     const unsigned long long slot0 = seg_base[ch.x];
     const uint32_t g_end = min(nseg, ch.y + kLongSegs);
     for (uint32_t g = ch.y + warp; g < g_end; g += kEntWarps) {
@@ -605,26 +710,28 @@ entropy_decode_kernel(const ciera_unit* __restrict__ units, int dt, uint32_t log
         sh.bad = 0;
     }
     __syncthreads();
-    const uint64_t P = raw_payload_bytes(msg, N, dt, log2b, &sh.changed, tid);
+    uint64_t P;  // symbols; Q = bytes of the raw payload
+    const uint64_t Q = raw_payload_bytes(msg, N, dt, log2b, &sh.changed, tid, P);
     const uint64_t wire = wire_bytes[unit];
-    if (P == 0 || wire == payoff + P) return;  // nothing travelled, or the raw form did
+    if (Q == 0 || wire == payoff + Q) return;  // nothing travelled, or the raw form did
     const uint64_t C = wire - payoff;
     const uint32_t nseg = (uint32_t)segments_of(P);
+    const uint32_t hdr = model_bytes(dt);
     uint8_t* const pay = msg + payoff;
-    if (wire < payoff || C >= P || C < 512ull + 4ull * nseg) {
+    if (wire < payoff || C >= Q || C < (uint64_t)hdr + 4ull * nseg) {
         if (tid == 0) raise_corrupt(status);
         return;
     }
-    sh.f[tid] = reinterpret_cast<const uint16_t*>(pay)[tid];
+    sh.f[tid] = tid < hdr / 2u ? reinterpret_cast<const uint16_t*>(pay)[tid] : (uint16_t)0;
     __syncthreads();
     if (!decoder_tables(sh.f, sh.c, sh.tab, &sh.flag, tid)) {
         if (tid == 0) raise_corrupt(status);
         return;
     }
     // where the segments lie (nseg <= kLongSegs <= kEntThreads: one round)
-    const uint32_t* dir = reinterpret_cast<const uint32_t*>(pay + 512);
-    const uint8_t* data = pay + 512 + 4ull * nseg;
-    const uint64_t data_bytes = C - 512ull - 4ull * nseg;
+    const uint32_t* dir = reinterpret_cast<const uint32_t*>(pay + hdr);
+    const uint8_t* data = pay + hdr + 4ull * nseg;
+    const uint64_t data_bytes = C - hdr - 4ull * nseg;
     const uint32_t nw = tid < nseg ? dir[tid] : 0u;
     if (nw > kSegWordsMax) sh.bad = 1;
     uint32_t total;
@@ -647,14 +754,18 @@ entropy_decode_kernel(const ciera_unit* __restrict__ units, int dt, uint32_t log
         return;
     }
     // the raw payload goes back into the message, which then is what the sender step had written
-    for (uint64_t i = (uint64_t)tid * 16; i < P; i += (uint64_t)kEntThreads * 16) {
-        if (i + 16 <= P) {
-            *reinterpret_cast<uint4*>(pay + i) = *reinterpret_cast<const uint4*>(raw + i);
-        } else {
-            for (uint64_t k = i; k < P; ++k) pay[k] = raw[k];
+    if (dt == CIERA_FP16) {
+        pack_symbols(raw, pay, log2b, 0, P, tid, kEntThreads);
+    } else {
+        for (uint64_t i = (uint64_t)tid * 16; i < P; i += (uint64_t)kEntThreads * 16) {
+            if (i + 16 <= P) {
+                *reinterpret_cast<uint4*>(pay + i) = *reinterpret_cast<const uint4*>(raw + i);
+            } else {
+                for (uint64_t k = i; k < P; ++k) pay[k] = raw[k];
+            }
         }
     }
-    if (tid == 0) wire_bytes[unit] = payoff + P;
+    if (tid == 0) wire_bytes[unit] = payoff + Q;
 }
 
 // longer units: layout (one block per unit), segments and restore (grids over chunks)
@@ -679,19 +790,21 @@ entropy_long_parse_kernel(const ciera_unit* __restrict__ units, const unsigned l
     __syncthreads();
     const uint8_t* msg = msgs + un.msg_off;
     const uint64_t payoff = payload_offset_of(N, dt, log2b);
-    const uint64_t P = raw_payload_bytes(msg, N, dt, log2b, &s_changed, tid);
+    uint64_t P;  // symbols; Q = bytes of the raw payload
+    const uint64_t Q = raw_payload_bytes(msg, N, dt, log2b, &s_changed, tid, P);
     const uint64_t wire = wire_bytes[unit];
-    if (P == 0 || wire == payoff + P) return;
+    if (Q == 0 || wire == payoff + Q) return;
     const uint64_t C = wire - payoff;
     const uint64_t nseg64 = segments_of(P);
-    if (wire < payoff || C >= P || P >= (1ull << 32) || C < 512ull + 4ull * nseg64) {
+    const uint32_t hdr = model_bytes(dt);
+    if (wire < payoff || C >= Q || P >= (1ull << 32) || C < (uint64_t)hdr + 4ull * nseg64) {
         if (tid == 0) raise_corrupt(status);
         return;
     }
     const uint32_t nseg = (uint32_t)nseg64;
     const uint8_t* pay = msg + payoff;
-    const uint32_t* dir = reinterpret_cast<const uint32_t*>(pay + 512);
-    const uint64_t data_bytes = C - 512ull - 4ull * nseg;
+    const uint32_t* dir = reinterpret_cast<const uint32_t*>(pay + hdr);
+    const uint64_t data_bytes = C - hdr - 4ull * nseg;
     const unsigned long long slot0 = seg_base[unit];
     uint64_t carry = 0;
     for (uint32_t g0 = 0; g0 < nseg; g0 += kEntThreads) {
@@ -713,6 +826,7 @@ entropy_long_parse_kernel(const ciera_unit* __restrict__ units, const unsigned l
     }
     if (tid == 0) {
         st->P = P;
+        st->Q = Q;
         st->nseg = nseg;
         st->coded = 1;
     }
@@ -733,7 +847,8 @@ entropy_long_decode_kernel(const ciera_unit* __restrict__ units, const unsigned 
     const uint64_t P = st->P;
     const uint32_t nseg = st->nseg;
     const uint8_t* pay = msgs + un.msg_off + payload_offset_of(un.n_values, dt, log2b);
-    sh.f[tid] = reinterpret_cast<const uint16_t*>(pay)[tid];
+    const uint32_t hdr = model_bytes(dt);
+    sh.f[tid] = tid < hdr / 2u ? reinterpret_cast<const uint16_t*>(pay)[tid] : (uint16_t)0;
     if (tid == 0) sh.bad = 0;
     __syncthreads();
     if (!decoder_tables(sh.f, sh.c, sh.tab, &sh.flag, tid)) {
@@ -743,7 +858,7 @@ entropy_long_decode_kernel(const ciera_unit* __restrict__ units, const unsigned 
         }
         return;
     }
-    const uint8_t* data = pay + 512 + 4ull * nseg;
+    const uint8_t* data = pay + hdr + 4ull * nseg;
     uint8_t* raw = scratch_raw + un.cache_off;
     const unsigned long long slot0 = seg_base[ch.x];
     const uint32_t g_end = min(nseg, ch.y + kLongSegs);
@@ -776,14 +891,18 @@ entropy_long_restore_kernel(const ciera_unit* __restrict__ units, const uint4* _
     const uint64_t payoff = payload_offset_of(un.n_values, dt, log2b);
     uint8_t* pay = msgs + un.msg_off + payoff;
     const uint8_t* raw = scratch_raw + un.cache_off;
-    for (uint64_t i = lo + (uint64_t)tid * 16; i < hi; i += (uint64_t)kEntThreads * 16) {
-        if (i + 16 <= hi) {
-            *reinterpret_cast<uint4*>(pay + i) = *reinterpret_cast<const uint4*>(raw + i);
-        } else {
-            for (uint64_t k = i; k < hi; ++k) pay[k] = raw[k];
+    if (dt == CIERA_FP16) {
+        pack_symbols(raw, pay, log2b, lo, hi, tid, kEntThreads);
+    } else {
+        for (uint64_t i = lo + (uint64_t)tid * 16; i < hi; i += (uint64_t)kEntThreads * 16) {
+            if (i + 16 <= hi) {
+                *reinterpret_cast<uint4*>(pay + i) = *reinterpret_cast<const uint4*>(raw + i);
+            } else {
+                for (uint64_t k = i; k < hi; ++k) pay[k] = raw[k];
+            }
         }
     }
-    if (ch.y == 0 && tid == 0) wire_bytes[ch.x] = payoff + P;
+    if (ch.y == 0 && tid == 0) wire_bytes[ch.x] = payoff + st->Q;
 }
 
 }  // namespace ciera
@@ -794,9 +913,10 @@ static bool misaligned16(const void* p) { return ((uintptr_t)p & 15u) != 0; }
 static size_t up16(size_t x) { return (x + 15) / 16 * 16; }
 
 // Scratch: [word count per segment slot][byte offset per segment slot][a record per long unit]
-// [body: the segment slots (sender) or the raw payloads at the units' cache offsets (receiver)]
+// [body: the segment slots (sender) or the decoded symbols at the units' cache offsets (receiver)]
+// [fp16 sender: the unpacked symbols at the units' cache offsets]
 struct ScratchLayout {
-    size_t nw, off, recs, body, total;
+    size_t nw, off, recs, body, sym, total;
 };
 static ScratchLayout scratch_layout(const ciera_plan* p) {
     ScratchLayout L;
@@ -805,7 +925,8 @@ static ScratchLayout scratch_layout(const ciera_plan* p) {
     L.recs = L.off + up16((size_t)p->total_segments * sizeof(uint32_t));
     L.body = L.recs + (size_t)p->ent_long_units.size() * kLongRec;
     const size_t enc = (size_t)p->total_segments * kSegSlot, dec = (size_t)p->cache_extent;
-    L.total = L.body + (enc > dec ? enc : dec) + 16;
+    L.sym = L.body + up16(enc > dec ? enc : dec);
+    L.total = L.sym + (p->dtype == CIERA_FP16 ? dec : 0) + 16;
     return L;
 }
 
@@ -833,25 +954,31 @@ extern "C" int ciera_entropy_encode(const ciera_plan* p, void* messages_dev, uin
     uint32_t* off = (uint32_t*)(base + L.off);
     uint8_t* recs = base + L.recs;
     uint8_t* slots = base + L.body;
+    uint8_t* sym = base + L.sym;
     const int dt = p->dtype;
     uint8_t* msgs = (uint8_t*)messages_dev;
     unsigned long long* wire = (unsigned long long*)wire_bytes_dev;
     const uint32_t n_long = (uint32_t)p->ent_long_units.size(), n_chunks = (uint32_t)p->ent_chunks.size();
     if (n_long < p->n_units) {
         entropy_encode_kernel<<<p->n_units, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, dt, p->log2b, msgs, wire,
-                                                                 slots, nw);
+                                                                 slots, nw, sym);
         count_launch();
         if ((rc = check_launch())) return rc;
     }
     if (n_long) {
         cudaError_t e = cudaMemsetAsync(recs, 0, (size_t)n_long * kLongRec, s);  // the counts start at zero
         if (e != cudaSuccess) return record_cuda_error(e);
+        if (dt == CIERA_FP16) {
+            entropy_long_unpack_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->ent_chunks_dev, dt, p->log2b, msgs,
+                                                                        wire, sym);
+            count_launch();
+        }
         entropy_long_hist_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->ent_chunks_dev, dt, p->log2b, msgs, wire,
-                                                                  recs);
-        entropy_long_model_kernel<<<n_long, kEntThreads, 0, s>>>(p->units_dev, p->ent_long_units_dev, dt, p->log2b, wire,
-                                                                 recs);
+                                                                  recs, sym);
+        entropy_long_model_kernel<<<n_long, kEntThreads, 0, s>>>(p->units_dev, p->ent_long_units_dev, dt, p->log2b, msgs,
+                                                                 wire, recs);
         entropy_long_encode_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_chunks_dev, dt,
-                                                                    p->log2b, msgs, wire, recs, slots, nw);
+                                                                    p->log2b, msgs, wire, recs, slots, nw, sym);
         entropy_long_layout_kernel<<<n_long, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_long_units_dev, dt,
                                                                   p->log2b, msgs, wire, recs, nw, off);
         entropy_long_copy_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_chunks_dev, dt,

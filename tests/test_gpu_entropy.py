@@ -106,10 +106,11 @@ def test_entropy_stage_reduced_moe_layer(rt, dtype):
     assert coded > 0
 
 
-@pytest.mark.parametrize("block", [32, 64, 512, 4096])
+@pytest.mark.parametrize("block", [16, 32, 64, 512, 4096])
 def test_entropy_stage_fp16(rt, block):
-    """fp16: the stage codes the bytes of the packed five-bit exponents; ragged units from empty caches (large
-    payloads), a reduced MoE layer under the clustered update, and a unit long enough for the chain of launches."""
+    """fp16: the stage codes the five-bit exponents as symbols of their own (unpacked before, packed after the
+    coder, 32 table entries); ragged units from empty caches (large payloads), a reduced MoE layer under the
+    clustered update, and a unit long enough for the chain of launches."""
     n = rt[1].LayerCodec.from_tensors(RAGGED, 1, "fp16", block, DEV).weights_bytes // 2
     traj = [wl.as_bits(w) for w in wl.trajectory(n, "fp16", 140 + block, 2, "adam")]
     assert _run(rt, RAGGED, 1, 2, block, [traj[0]] + traj, from_zero=True) > 0
@@ -146,24 +147,26 @@ def test_entropy_stage_long_and_short_units_mixed(rt):
     assert coded >= 4
 
 
+@pytest.mark.parametrize("dtype", [0, 2])
 @pytest.mark.parametrize("n_values", [70_001, 600_001])
-def test_entropy_decode_flags_a_damaged_section(rt, n_values):
+def test_entropy_decode_flags_a_damaged_section(rt, n_values, dtype):
     ciera, runtime = rt
     sizes = [n_values]
-    codec = runtime.LayerCodec.from_tensors(sizes, 1, "bf16", 512, DEV)
+    codec = runtime.LayerCodec.from_tensors(sizes, 1, NAME[dtype], 512, DEV)
     n = codec.weights_bytes // 2
-    w = wl.as_bits(next(iter(wl.trajectory(n, "bf16", 3, 0, "adam"))))
+    w = wl.as_bits(next(iter(wl.trajectory(n, NAME[dtype], 3, 0, "adam"))))
     codec.init_caches(None)
     codec.encode(to_dev_bytes(w, DEV))
     codec.entropy_encode()
     codec.transport()
     torch.cuda.synchronize()
-    raw_len = ora.payload_offset(n_values, 0, 512) + n_values
+    raw_len = ora.message_capacity(n_values, dtype, 512)  # from empty caches every block is changed
     assert int(codec.wire_bytes[0].item()) < raw_len  # the coded form travelled
-    off = int(codec.units[0]["msg_off"]) + ora.payload_offset(n_values, 0, 512)
+    off = int(codec.units[0]["msg_off"]) + ora.payload_offset(n_values, dtype, 512)
     nseg = -(-n_values // 4096)
+    table = 64 if dtype == 2 else 512
     before = codec.msg_recv.clone()
-    codec.msg_recv[off + 512 + 4 * nseg + 200] ^= 0x5A  # inside the first segment's words
+    codec.msg_recv[off + table + 4 * nseg + 200] ^= 0x5A  # inside the first segment's words
     damaged = codec.msg_recv.clone()
     codec.entropy_decode()
     torch.cuda.synchronize()
