@@ -737,16 +737,19 @@ OTHER_CONFIGS = [
     ("hashed_sender_bf16_block32_adam_like_update", dict(detect="hash", block=32, update="adam")),
     ("hashed_sender_fp32_block512", dict(detect="hash", dtype="fp32")),
     ("entropy_stage_bf16_block512", dict(entropy=True)),
+    ("entropy_stage_fp16_block512", dict(entropy=True, dtype="fp16")),
 ]
 
 
 def raw_payload_symbols(codec, a):
-    """Changed exponents (one symbol each) that the entropy stage codes: the raw payload bytes of the last encode."""
+    """Changed exponents (one symbol each) that the entropy stage codes: the raw payload bytes of the last encode
+    (fp16: five bits per exponent on the wire, so 8 symbols to 5 payload bytes; a short last block rounds up)."""
     from paper_2609_04609_b200 import ciera
 
     wire = codec.wire_bytes.cpu().numpy()
-    return int(sum(int(w) - ciera.payload_offset(int(u["n_values"]), codec.dtype, a.block)
-                   for u, w in zip(codec.units, wire) if int(u["n_values"])))
+    payload = int(sum(int(w) - ciera.payload_offset(int(u["n_values"]), codec.dtype, a.block)
+                      for u, w in zip(codec.units, wire) if int(u["n_values"])))
+    return payload * 8 // 5 if a.dtype == "fp16" else payload
 
 
 def entropy_roofline(symbols, enc_ms, dec_ms, sm_mhz, sms=148):
@@ -837,8 +840,12 @@ def one_layer_case(args, device, peak, over, steps=5, clocks_mhz=None):
         raw = codec.paper_bytes()
         symbols = raw_payload_symbols(codec, a)
         codec.entropy_encode()
-        res["entropy_roofline"] = entropy_roofline(symbols, res["entropy_encode_ms"],
-                                                   res["entropy_decode_ms"], clocks_mhz)
+        if a.dtype == "fp16":  # no instruction count on record for the unpacking and packing around the coder
+            res["entropy_symbols_per_launch"] = symbols
+            res["entropy_symbols_G_per_s"] = [symbols / (res[k] * 1e-3) / 1e9 for k in ("entropy_encode_ms", "entropy_decode_ms")]
+        else:
+            res["entropy_roofline"] = entropy_roofline(symbols, res["entropy_encode_ms"],
+                                                       res["entropy_decode_ms"], clocks_mhz)
         coded = codec.paper_bytes()
         fixed = sum(ciera.message_bytes(int(u["n_values"]), codec.dtype, a.block, 0) for u in codec.units if int(u["n_values"]))
         res["bytes_ratio_coded"] = coded / (n * vb)

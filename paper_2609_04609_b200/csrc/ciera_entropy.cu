@@ -398,6 +398,7 @@ __device__ __forceinline__ uint32_t block_scan(uint32_t v, uint32_t* scan, uint3
 // ------------------------------------------------------------------------------------------ sender
 // units of up to kLongSegs segment slots: one thread block per unit, start to end
 
+template <bool HALF>  // HALF: fp16, five-bit symbols (see the head of this file)
 __global__ void __launch_bounds__(kEntThreads, 5)
 entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
                       int dt, uint32_t log2b, uint8_t* msgs, unsigned long long* wire_bytes,
@@ -424,9 +425,9 @@ entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long 
     if (P == 0 || P > un.n_values) return;
     uint8_t* const pay = msgs + un.msg_off + payoff;  // 16-byte aligned
     const uint32_t nseg = (uint32_t)segments_of(P);
-    const uint32_t hdr = model_bytes(dt);
+    constexpr uint32_t hdr = HALF ? 64u : 512u;  // = model_bytes(dt)
     const uint8_t* src = pay;  // the symbols, one per byte
-    if (dt == CIERA_FP16) {
+    if (HALF) {
         uint8_t* sym = scratch_sym + un.cache_off;
         unpack_symbols(pay, sym, log2b, 0, P, tid, kEntThreads);
         src = sym;
@@ -581,6 +582,7 @@ entropy_long_model_kernel(const ciera_unit* __restrict__ units, const uint32_t* 
     long_model(recs, li)[tid] = s_f[tid];
 }
 
+template <bool HALF>  // HALF: fp16, five-bit symbols (see the head of this file)
 __global__ void __launch_bounds__(kEntThreads)
 entropy_long_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
                            const uint4* __restrict__ chunks, int dt, uint32_t log2b, const uint8_t* msgs,
@@ -602,7 +604,7 @@ entropy_long_encode_kernel(const ciera_unit* __restrict__ units, const unsigned 
     if (tid == 0) s_total = 0;
     __syncthreads();
     encoder_tables(s_f, s_enc, tid);
-    const uint8_t* pay = sender_symbols(un, dt, msgs, payoff, scratch_sym);
+    const uint8_t* pay = HALF ? scratch_sym + un.cache_off : msgs + un.msg_off + payoff;  // the symbols
     const unsigned long long slot0 = seg_base[ch.x];
     for (uint32_t g = ch.y + warp; g < g_end; g += kEntWarps) {
         const uint32_t n = (uint32_t)min((uint64_t)kSegment, P - (uint64_t)g * kSegment);
@@ -694,6 +696,7 @@ __device__ __forceinline__ void raise_corrupt(int32_t* status) {
     if (status) atomicCAS(status, 0, (int32_t)CIERA_ERR_CORRUPT);
 }
 
+template <bool HALF>  // HALF: fp16, five-bit symbols (see the head of this file)
 __global__ void __launch_bounds__(kEntThreads)
 entropy_decode_kernel(const ciera_unit* __restrict__ units, int dt, uint32_t log2b, uint8_t* msgs,
                       unsigned long long* wire_bytes, uint8_t* scratch_raw, int32_t* status) {
@@ -716,7 +719,7 @@ entropy_decode_kernel(const ciera_unit* __restrict__ units, int dt, uint32_t log
     if (Q == 0 || wire == payoff + Q) return;  // nothing travelled, or the raw form did
     const uint64_t C = wire - payoff;
     const uint32_t nseg = (uint32_t)segments_of(P);
-    const uint32_t hdr = model_bytes(dt);
+    constexpr uint32_t hdr = HALF ? 64u : 512u;  // = model_bytes(dt)
     uint8_t* const pay = msg + payoff;
     if (wire < payoff || C >= Q || C < (uint64_t)hdr + 4ull * nseg) {
         if (tid == 0) raise_corrupt(status);
@@ -754,7 +757,7 @@ entropy_decode_kernel(const ciera_unit* __restrict__ units, int dt, uint32_t log
         return;
     }
     // the raw payload goes back into the message, which then is what the sender step had written
-    if (dt == CIERA_FP16) {
+    if (HALF) {
         pack_symbols(raw, pay, log2b, 0, P, tid, kEntThreads);
     } else {
         for (uint64_t i = (uint64_t)tid * 16; i < P; i += (uint64_t)kEntThreads * 16) {
@@ -832,6 +835,7 @@ entropy_long_parse_kernel(const ciera_unit* __restrict__ units, const unsigned l
     }
 }
 
+template <bool HALF>  // HALF: fp16, five-bit symbols (see the head of this file)
 __global__ void __launch_bounds__(kEntThreads)
 entropy_long_decode_kernel(const ciera_unit* __restrict__ units, const unsigned long long* __restrict__ seg_base,
                            const uint4* __restrict__ chunks, int dt, uint32_t log2b, const uint8_t* msgs,
@@ -847,7 +851,7 @@ entropy_long_decode_kernel(const ciera_unit* __restrict__ units, const unsigned 
     const uint64_t P = st->P;
     const uint32_t nseg = st->nseg;
     const uint8_t* pay = msgs + un.msg_off + payload_offset_of(un.n_values, dt, log2b);
-    const uint32_t hdr = model_bytes(dt);
+    constexpr uint32_t hdr = HALF ? 64u : 512u;  // = model_bytes(dt)
     sh.f[tid] = tid < hdr / 2u ? reinterpret_cast<const uint16_t*>(pay)[tid] : (uint16_t)0;
     if (tid == 0) sh.bad = 0;
     __syncthreads();
@@ -960,8 +964,8 @@ extern "C" int ciera_entropy_encode(const ciera_plan* p, void* messages_dev, uin
     unsigned long long* wire = (unsigned long long*)wire_bytes_dev;
     const uint32_t n_long = (uint32_t)p->ent_long_units.size(), n_chunks = (uint32_t)p->ent_chunks.size();
     if (n_long < p->n_units) {
-        entropy_encode_kernel<<<p->n_units, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, dt, p->log2b, msgs, wire,
-                                                                 slots, nw, sym);
+        auto* k = dt == CIERA_FP16 ? entropy_encode_kernel<true> : entropy_encode_kernel<false>;
+        k<<<p->n_units, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, dt, p->log2b, msgs, wire, slots, nw, sym);
         count_launch();
         if ((rc = check_launch())) return rc;
     }
@@ -977,8 +981,9 @@ extern "C" int ciera_entropy_encode(const ciera_plan* p, void* messages_dev, uin
                                                                   recs, sym);
         entropy_long_model_kernel<<<n_long, kEntThreads, 0, s>>>(p->units_dev, p->ent_long_units_dev, dt, p->log2b, msgs,
                                                                  wire, recs);
-        entropy_long_encode_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_chunks_dev, dt,
-                                                                    p->log2b, msgs, wire, recs, slots, nw, sym);
+        auto* k = dt == CIERA_FP16 ? entropy_long_encode_kernel<true> : entropy_long_encode_kernel<false>;
+        k<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_chunks_dev, dt, p->log2b, msgs, wire, recs,
+                                           slots, nw, sym);
         entropy_long_layout_kernel<<<n_long, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_long_units_dev, dt,
                                                                   p->log2b, msgs, wire, recs, nw, off);
         entropy_long_copy_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_chunks_dev, dt,
@@ -999,12 +1004,14 @@ extern "C" int ciera_entropy_decode(const ciera_plan* p, void* messages_dev, uin
     if (e != cudaSuccess) return record_cuda_error(e);
     if (dev < 0 || dev >= 64) return CIERA_ERR_UNSUPPORTED;
     if (!configured[dev].load(std::memory_order_acquire)) {
-        e = cudaFuncSetAttribute(entropy_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)sizeof(DecodeShared));
-        if (e != cudaSuccess) return record_cuda_error(e);
-        e = cudaFuncSetAttribute(entropy_long_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)sizeof(DecodeShared));
-        if (e != cudaSuccess) return record_cuda_error(e);
+        for (auto* k : {entropy_decode_kernel<false>, entropy_decode_kernel<true>}) {
+            e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecodeShared));
+            if (e != cudaSuccess) return record_cuda_error(e);
+        }
+        for (auto* k : {entropy_long_decode_kernel<false>, entropy_long_decode_kernel<true>}) {
+            e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(DecodeShared));
+            if (e != cudaSuccess) return record_cuda_error(e);
+        }
         configured[dev].store(1, std::memory_order_release);
     }
     cudaStream_t s = (cudaStream_t)stream;
@@ -1019,16 +1026,17 @@ extern "C" int ciera_entropy_decode(const ciera_plan* p, void* messages_dev, uin
     unsigned long long* wire = (unsigned long long*)wire_bytes_dev;
     const uint32_t n_long = (uint32_t)p->ent_long_units.size(), n_chunks = (uint32_t)p->ent_chunks.size();
     if (n_long < p->n_units) {
-        entropy_decode_kernel<<<p->n_units, kEntThreads, sizeof(DecodeShared), s>>>(p->units_dev, dt, p->log2b, msgs, wire,
-                                                                                   raw, status_dev);
+        auto* k = dt == CIERA_FP16 ? entropy_decode_kernel<true> : entropy_decode_kernel<false>;
+        k<<<p->n_units, kEntThreads, sizeof(DecodeShared), s>>>(p->units_dev, dt, p->log2b, msgs, wire, raw, status_dev);
         count_launch();
         if ((rc = check_launch())) return rc;
     }
     if (n_long) {
         entropy_long_parse_kernel<<<n_long, kEntThreads, 0, s>>>(p->units_dev, p->seg_base_dev, p->ent_long_units_dev, dt,
                                                                  p->log2b, msgs, wire, recs, off, nw, status_dev);
-        entropy_long_decode_kernel<<<n_chunks, kEntThreads, sizeof(DecodeShared), s>>>(
-            p->units_dev, p->seg_base_dev, p->ent_chunks_dev, dt, p->log2b, msgs, recs, off, nw, raw, status_dev);
+        auto* k = dt == CIERA_FP16 ? entropy_long_decode_kernel<true> : entropy_long_decode_kernel<false>;
+        k<<<n_chunks, kEntThreads, sizeof(DecodeShared), s>>>(p->units_dev, p->seg_base_dev, p->ent_chunks_dev, dt, p->log2b,
+                                                              msgs, recs, off, nw, raw, status_dev);
         entropy_long_restore_kernel<<<n_chunks, kEntThreads, 0, s>>>(p->units_dev, p->ent_chunks_dev, dt, p->log2b, msgs,
                                                                      wire, recs, raw);
         for (int i = 0; i < 3; ++i) count_launch();
