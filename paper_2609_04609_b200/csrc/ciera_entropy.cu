@@ -418,9 +418,9 @@ entropy_encode_kernel(const ciera_unit* __restrict__ units, const unsigned long 
     const uint64_t payoff = payload_offset_of(un.n_values, dt, log2b);
     const uint64_t Q = wire_bytes[unit] - payoff;
     // nothing to code; or a length that no sender step reports (shorter than the fixed sections, more
-    // than one payload byte per value, not a sum of block sizes): everything below is indexed by the
+    // than the payload of a unit whose every block changed, not a sum of block sizes): everything below is indexed by the
     // symbol count P, so such a unit is left alone
-    if (Q == 0 || Q > un.n_values) return;
+    if (Q == 0 || Q > payload_bytes_max(un.n_values, dt, log2b)) return;
     const uint64_t P = symbols_of_payload(msgs + un.msg_off, un.n_values, dt, log2b, Q);
     if (P == 0 || P > un.n_values) return;
     uint8_t* const pay = msgs + un.msg_off + payoff;  // 16-byte aligned
@@ -505,8 +505,8 @@ __device__ __forceinline__ uint16_t* long_model(uint8_t* recs, uint32_t li) { re
 __device__ __forceinline__ LongState* long_state(uint8_t* recs, uint32_t li) { return reinterpret_cast<LongState*>(recs + (size_t)li * kLongRec + 1536); }
 
 // Symbol count of a unit's payload on the sender (0: nothing to code); Q gets the payload's length in bytes.
-// A reported length that no sender step can have produced -- shorter than the fixed sections, a payload of
-// more than one byte per value, not a sum of block sizes, e.g. the stale word of a unit that an aborted
+// A reported length that no sender step can have produced -- shorter than the fixed sections, a payload
+// longer than that of a unit whose every block changed, not a sum of block sizes, e.g. the stale word of a unit that an aborted
 // encode never finished -- also gives 0: the histogram, the segments and the scratch slots are all indexed
 // by the symbol count, so it must stay inside the unit's slot (a value has one exponent, and plans are
 // limited to units whose block counts fit 32 bits).
@@ -515,7 +515,7 @@ __device__ __forceinline__ uint64_t sender_payload(const ciera_unit& un, int dt,
                                                    uint64_t& Q) {
     payoff = payload_offset_of(un.n_values, dt, log2b);
     Q = wire_bytes[unit] - payoff;
-    if (Q == 0 || Q > un.n_values || Q >= (1ull << 32)) return 0;
+    if (Q == 0 || Q > payload_bytes_max(un.n_values, dt, log2b) || Q >= (1ull << 32)) return 0;
     const uint64_t P = symbols_of_payload(msgs + un.msg_off, un.n_values, dt, log2b, Q);
     return (P <= un.n_values && P < (1ull << 32)) ? P : 0;
 }

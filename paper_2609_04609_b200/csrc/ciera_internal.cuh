@@ -102,6 +102,12 @@ __host__ __device__ inline uint64_t block_payload_bytes(uint64_t len, int dtype)
 __host__ __device__ inline uint64_t payload_offset_of(uint64_t n, int dtype, uint32_t log2b) {
     return sm_offset(n, log2b) + pad16(sm_section_bytes(n, dtype));
 }
+// the largest payload a unit of n values can have: every block changed
+__host__ __device__ inline uint64_t payload_bytes_max(uint64_t n, int dtype, uint32_t log2b) {
+    const uint64_t nb = num_blocks(n, log2b);
+    if (nb == 0) return 0;
+    return (nb - 1) * block_payload_bytes(1ull << log2b, dtype) + block_payload_bytes(n - ((nb - 1) << log2b), dtype);
+}
 
 // Units with more blocks than this get their per-tile "changed blocks before" counts from a
 // prefix kernel at decode time; shorter ones read them straight from the bitmap.  With fine

@@ -41,7 +41,7 @@ def rt():
 
 def _clean_step_is_exact(rt, dtype=0, block=512):
     ciera, runtime = rt
-    name = {0: "bf16", 1: "fp32"}[dtype]
+    name = {0: "bf16", 1: "fp32", 2: "fp16"}[dtype]
     codec = guard(runtime.LayerCodec.from_tensors([3_000_000 + 5, 131_072, 70_001], 2, name, block, DEV, slack=256))
     table = OracleTable(codec.units, dtype, block, codec.cache_bytes, codec.msg_bytes)
     n = codec.weights_bytes // wl.VALUE_BYTES[name]
@@ -83,10 +83,10 @@ def test_bounded_waits_run_out_and_the_context_stays_usable(rt, max_polls):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("dtype,block", [(0, 512), (1, 64), (0, 4)])
+@pytest.mark.parametrize("dtype,block", [(0, 512), (1, 64), (0, 4), (2, 512), (2, 16)])
 def test_transport_never_leaves_a_slot_on_an_impossible_length(rt, dtype, block):
     ciera, runtime = rt
-    name = {0: "bf16", 1: "fp32"}[dtype]
+    name = {0: "bf16", 1: "fp32", 2: "fp16"}[dtype]
     sizes = [70_001, 131_072, 40_000, 8192 * 3]
     codec = guard(runtime.LayerCodec.from_tensors(sizes, 1, name, block, DEV, slack=256))
     n = codec.weights_bytes // wl.VALUE_BYTES[name]
@@ -123,6 +123,33 @@ def test_transport_never_leaves_a_slot_on_an_impossible_length(rt, dtype, block)
     assert torch.equal(codec.msg_send[mo : mo + cap], before[mo : mo + cap])
     codec.canaries.check("entropy stage with an impossible length")
     _clean_step_is_exact(rt, dtype, block if block >= 16 else 512)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("block", [16, 512])
+def test_entropy_stage_leaves_an_fp16_unit_alone_when_its_length_is_no_sum_of_block_sizes(rt, block):
+    """fp16: the sender's entropy stage gets the number of five-bit symbols from the payload's length.  A length
+    inside the slot that no set of changed blocks adds up to (here: one byte short) must make it leave the unit as
+    it is; the other units are coded as usual."""
+    ciera, runtime = rt
+    codec = guard(runtime.LayerCodec.from_tensors([70_001, 131_072, 40_000], 1, "fp16", block, DEV, slack=256))
+    n = codec.weights_bytes // 2
+    w = wl.as_bits(next(iter(wl.trajectory(n, "fp16", 12, 0, "adam"))))
+    codec.init_caches(None)  # from empty caches: every block is sent
+    codec.encode(to_dev_bytes(w, DEV))
+    torch.cuda.synchronize()
+    good = codec.wire_bytes.clone()
+    codec.wire_bytes[1] = int(good[1].item()) - 1
+    before = codec.msg_send.clone()
+    codec.entropy_encode()
+    torch.cuda.synchronize()
+    codec.check_status()
+    codec.canaries.check("entropy stage with a length that is no sum of block sizes")
+    mo, cap = int(codec.units[1]["msg_off"]), int(codec.units[1]["msg_capacity"])
+    assert torch.equal(codec.msg_send[mo : mo + cap], before[mo : mo + cap])
+    assert int(codec.wire_bytes[1].item()) == int(good[1].item()) - 1
+    for i in (0, 2):
+        assert int(codec.wire_bytes[i].item()) < int(good[i].item())  # coded
 
 
 @pytest.mark.gpu
