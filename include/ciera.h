@@ -138,12 +138,13 @@ CIERA_API const void* ciera_plan_host_image(const ciera_plan* plan);
 /* Bytes of scratch ("workspace") that ciera_encode, ciera_transport and ciera_decode work in: 12 bytes per
  * tile (a look-back status word for the sender, a count for the receiver) and a few counters. */
 CIERA_API size_t ciera_plan_workspace_bytes(const ciera_plan* plan);
-/* Zero-fills a workspace of ciera_plan_workspace_bytes(plan) bytes (16-byte aligned) on `stream`.  The sender
- * calls (ciera_encode, ciera_encode_hashed, ciera_roundtrip_host) expect their part of the workspace all zero
- * when they start and leave it all zero when they have finished, so that no launch is spent on clearing it
- * before every call: initialise a workspace once after allocating it, and again after a call whose device
- * status word came back with an error (a kernel that gave up leaves the workspace in an unspecified state).
- * A plain cudaMemset of the whole workspace does the same. */
+/* Zero-fills a workspace of ciera_plan_workspace_bytes(plan) bytes (16-byte aligned) on `stream`.  Every
+ * call that takes a workspace (ciera_encode, ciera_encode_hashed, ciera_transport, ciera_decode,
+ * ciera_roundtrip_host) expects its counters in it all zero when it starts and leaves them all zero when it
+ * has finished, so that no launch is spent on clearing them before every call: initialise a workspace once
+ * after allocating it, and again after a call whose device status word came back with an error (a kernel
+ * that gave up leaves the workspace in an unspecified state).  A plain cudaMemset of the whole workspace
+ * does the same. */
 CIERA_API int ciera_workspace_init(const ciera_plan* plan, void* workspace_dev, void* stream);
 
 /* Copies the table into caller-owned device memory `plan_dev` (>= ciera_plan_device_bytes,
@@ -253,8 +254,8 @@ CIERA_API int ciera_encode_hashed(const ciera_plan* plan, const void* weights_de
 /* Copies, for every unit, the first wire_bytes_dev[u] bytes of its slot from `src_messages_dev`
  * to the same slot of `dst_messages_dev` (one kernel; the lengths are read on the device).  This
  * stands where the Allgather of the messages would be.  `workspace_dev`: scratch of
- * ciera_plan_workspace_bytes() (holds the counter tiles are handed out from, which the call sets to zero
- * itself; not to be shared by calls that can overlap on the GPU).  `status_dev`: device int32 or NULL; the
+ * ciera_plan_workspace_bytes() (holds the counter tiles are handed out from: zero on entry -- see
+ * ciera_workspace_init -- and handed back at zero; not to be shared by calls that can overlap on the GPU).  `status_dev`: device int32 or NULL; the
  * kernel's waits on its own copies are bounded and raise CIERA_ERR_TIMEOUT there. */
 CIERA_API int ciera_transport(const ciera_plan* plan, const void* src_messages_dev, void* dst_messages_dev,
                     const uint64_t* wire_bytes_dev, void* workspace_dev, int32_t* status_dev, void* stream);
@@ -271,7 +272,8 @@ CIERA_API int ciera_transport(const ciera_plan* plan, const void* src_messages_d
  *                            whose bitmap implies a different length raises CIERA_ERR_CORRUPT in
  *                            status_dev (its output is then unspecified)
  *   workspace_dev       scratch of ciera_plan_workspace_bytes(), 16-byte aligned: the counter tiles
- *                            are handed out from (set to zero by the call itself) and, when some unit has
+ *                            are handed out from (zero on entry -- see ciera_workspace_init -- and handed
+ *                            back at zero) and, when some unit has
  *                            more than 4096 blocks, the per-tile counts of a small prefix kernel that
  *                            runs first; the sender's part of the workspace is left alone.  Must not be
  *                            shared by calls that can overlap on the GPU.

@@ -589,6 +589,16 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
             t_nxt = t_nn;
         }
         cp_async_wait<0>();
+        // this producer draws no more numbers: the last producer of the grid to get here hands the counter (and
+        // the count of producers that got here, in the word behind it) back at zero for the next call
+        if (lane == 0) {
+            __threadfence();
+            if (atomicAdd(ticket + 1, 1u) + 1u == gridDim.x * (uint32_t)kDecProducers) {
+                __threadfence();
+                ticket[0] = 0u;
+                ticket[1] = 0u;
+            }
+        }
     } else {
         // ---------------------------------------------------------------- consumers
         const uint32_t bmask = (1u << log2b) - 1u;
@@ -903,12 +913,10 @@ extern "C" int ciera_decode(const ciera_plan* p, const void* messages_dev, void*
         misaligned16(workspace_dev))
         return CIERA_ERR_MISALIGNED;
     cudaStream_t s = (cudaStream_t)stream;
-    // scratch: the tile counter, which starts at zero, behind the sender's status words (left alone), and
-    // behind it the per-tile counts of the units that go through the prefix kernel
+    // scratch: the tile counter (found at zero, handed back at zero) behind the sender's status words (left
+    // alone), and behind it the per-tile counts of the units that go through the prefix kernel
     unsigned int* ticket = (unsigned int*)((uint8_t*)workspace_dev + workspace_ticket_offset(nt));
     uint32_t* ws_prefix = (uint32_t*)((uint8_t*)workspace_dev + workspace_prefix_offset(nt));
-    cudaError_t me = cudaMemsetAsync(ticket, 0, 16, s);
-    if (me != cudaSuccess) return record_cuda_error(me);
     const uint32_t n_long = (uint32_t)p->long_units.size();
     if (n_long) {
         if (is_fine(p->log2b))

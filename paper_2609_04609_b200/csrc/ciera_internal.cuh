@@ -117,10 +117,12 @@ constexpr uint32_t kDecodeDirectBlocks = 4096;
 // Layout of the scratch ("workspace") of a plan with nt tiles, shared by the sender, transport and receiver calls:
 //   [0, 8 nt)             one 64-bit look-back status word per tile                     (sender)
 //   [8 nt, + 16)          the sender's run counter and its counter of finished blocks   (sender)
-//   [8 nt + 16, + 16)     the counter that transport and receiver hand their tiles out from
+//   [8 nt + 16, + 16)     the counter that transport and receiver hand their tiles out from, and their count of
+//                         thread blocks (producer warps) that have drawn their last number
 //   [8 nt + 32, + 4 nt)   changed blocks before each tile of the units that go through the receiver's prefix kernel
-// The sender needs its two parts all zero when it starts and leaves them so; transport and receiver set their
-// counter to zero themselves at the start of every call and touch nothing of the sender's.
+// Sender, transport and receiver each need their counters all zero when they start and leave them so (the last
+// thread block to finish clears them), so that no call needs a clearing launch in front of its kernel; transport
+// and receiver touch nothing of the sender's, and the per-tile counts need no initial value.
 __host__ __device__ inline size_t workspace_sender_counters_offset(size_t nt) { return nt * sizeof(unsigned long long); }
 __host__ __device__ inline size_t workspace_ticket_offset(size_t nt) { return workspace_sender_counters_offset(nt) + 16; }
 __host__ __device__ inline size_t workspace_prefix_offset(size_t nt) { return workspace_ticket_offset(nt) + 16; }

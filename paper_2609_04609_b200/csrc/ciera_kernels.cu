@@ -198,6 +198,16 @@ transport_pipe_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             }
         }
+        // this block draws no more numbers: the last block to get here hands the counter (and the count of
+        // blocks that got here, in the word behind it) back at zero, as the next call expects to find them
+        if (lane == 0) {
+            __threadfence();
+            if (atomicAdd(ticket + 1, 1u) + 1u == gridDim.x) {
+                __threadfence();
+                ticket[0] = 0u;
+                ticket[1] = 0u;
+            }
+        }
         if (lane == 0 && ok) {  // end marker
             const uint32_t st = k % kPipeStages;
             if (k < (uint32_t)kPipeStages || mbar_wait(&ctl->empty[st], ((k / kPipeStages) & 1u) ^ 1u, abort, status)) {
@@ -336,10 +346,8 @@ extern "C" int ciera_transport(const ciera_plan* p, const void* src_messages_dev
     if (!src_messages_dev || !dst_messages_dev || !wire_bytes_dev || !workspace_dev) return CIERA_ERR_INVALID_ARG;
     if (misaligned16(src_messages_dev) || misaligned16(dst_messages_dev) || misaligned16(workspace_dev))
         return CIERA_ERR_MISALIGNED;
-    // the tile counter (see the layout of the scratch in ciera_internal.cuh) starts at zero
+    // the tile counter (see the layout of the scratch in ciera_internal.cuh): found at zero, handed back at zero
     unsigned int* ticket = (unsigned int*)((uint8_t*)workspace_dev + workspace_ticket_offset(nt));
-    cudaError_t me = cudaMemsetAsync(ticket, 0, 16, (cudaStream_t)stream);
-    if (me != cudaSuccess) return record_cuda_error(me);
     int limit = 0;
     rc = transport_pipe_grid_limit(&limit);
     if (rc) return rc;

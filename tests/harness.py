@@ -157,9 +157,10 @@ def compare_step(codec, exp, w_flat, label=""):
 
 
 def sender_scratch_is_clean(codec) -> bool:
-    """The sender finds its part of the workspace (one status word per tile, then 16 bytes of counters) all zero
-    and has to hand it back all zero: there is no clearing launch in front of the kernel."""
-    n = 8 * codec.plan.n_tiles + 16
+    """The calls find their counters in the workspace (one status word per tile and 16 bytes of counters for the
+    sender, then 16 bytes for transport and receiver) all zero and have to hand them back all zero: there is no
+    clearing launch in front of any kernel."""
+    n = 8 * codec.plan.n_tiles + 32
     clean = not bool(codec.workspace[:n].any().item())
     hw = getattr(codec, "hashed_workspace", None)
     if hw is not None:
@@ -170,7 +171,7 @@ def sender_scratch_is_clean(codec) -> bool:
 def compare_caches(codec, table, label=""):
     if getattr(codec, "canaries", None) is not None:
         codec.canaries.check(label)
-    assert sender_scratch_is_clean(codec), f"{label}: the sender did not hand its scratch back all zero"
+    assert sender_scratch_is_clean(codec), f"{label}: the counters in the scratch were not handed back all zero"
     cs = codec.sender_cache.cpu().numpy()
     cr = codec.receiver_cache.cpu().numpy()
     for i, u in enumerate(codec.units):
