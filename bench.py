@@ -157,7 +157,7 @@ class ClockSampler:
     """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs
     (read-only queries)."""
 
-    def __init__(self, index: int, uuid: str = "", period_s: float = 0.05):
+    def __init__(self, index: int, uuid: str = "", period_s: float = 0.02):
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.power = [], set(), []
         self.max_mhz = None
