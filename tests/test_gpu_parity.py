@@ -416,6 +416,136 @@ def test_config5_full_size_mixed_shapes(rt, n_shards):
         prev = cur
 
 
+def test_buffers_beyond_four_gib(rt):
+    """One plan whose buffers are larger than 4 GiB each: 4.56 G bf16 values (9.1 GB of weights, 4.6 GB per cache,
+    9.1 GB per message buffer), so that byte offsets pass 2^32 in every buffer and 2^33 in weights and messages --
+    no 32-bit offset arithmetic survives this.  34 tensors of 128 Mi values in 4 shards (units of 4096 tiles: spread
+    tiles, look-back, cooperative launch, prefix kernel) between short units at the start and, beyond all the
+    marks, at the end.  Generated on the device in chunks.  After each of two steps (clustered, then 0.1 % of the
+    exponents changed in segments) the round trip is exact over the whole buffer, both caches agree, the guard
+    bytes are intact, and the units that straddle the 2^32 and 2^33 marks of each buffer, the first and the last
+    units equal the oracle's messages, lengths, counts and caches."""
+    ciera, runtime = rt
+    from oracle import ciera_oracle as ora
+
+    free, _ = torch.cuda.mem_get_info()
+    if free < 90e9:
+        pytest.skip("needs 90 GB of free device memory")
+    block, n_shards, big = 512, 4, 1 << 27
+    sizes = [1_000_001] + [big] * 34 + [1_000_001, 300_000, 4096 + 5]
+    codec = guard(runtime.LayerCodec.from_tensors(sizes, n_shards, "bf16", block, DEV, slack=256))
+    units = codec.units
+    n = codec.weights_bytes // 2
+    assert codec.weights_bytes > 2 ** 33 and codec.cache_bytes > 2 ** 32 and codec.msg_bytes > 2 ** 33
+
+    def straddlers(off_key, length_of, marks):
+        out = []
+        for i, u in enumerate(units):
+            lo = int(u[off_key])
+            hi = lo + length_of(u)
+            out += [i for m in marks if lo < m <= hi or (lo <= m < hi)]
+        return out
+
+    picks = set(straddlers("weights_off", lambda u: 2 * int(u["n_values"]), (2 ** 32, 2 ** 33)))
+    picks |= set(straddlers("cache_off", lambda u: int(u["n_values"]), (2 ** 32,)))
+    picks |= set(straddlers("msg_off", lambda u: int(u["msg_capacity"]), (2 ** 32, 2 ** 33)))
+    assert len(picks) >= 2
+    picks |= {i + d for i in picks for d in (-1, 1)}  # and their neighbours, which lie wholly beyond a mark
+    picks |= {0, 1, len(units) // 2} | set(range(len(units) - 3 * n_shards, len(units)))
+    picks = sorted(picks)
+    assert int(units[picks[-1]]["weights_off"]) > 2 ** 33 and int(units[picks[-1]]["cache_off"]) > 2 ** 32
+
+    gen = wl.make_generator(4242, DEV)
+    chunk = 1 << 28
+
+    def chunked(make, like=None):
+        out = torch.empty(n, dtype=torch.bfloat16, device=DEV)
+        for lo in range(0, n, chunk):
+            hi = min(n, lo + chunk)
+            out[lo:hi] = make(hi - lo) if like is None else make(like[lo:hi])
+        return out
+
+    gaps = codec.canaries.guards["weights_out"]
+    gaps = gaps[gaps < 2 * n]
+
+    def as_bytes(t):
+        b = t.view(torch.uint8)
+        b[gaps] = codec.canaries.PATTERN  # not part of any unit: make both sides of the comparison agree there
+        return b
+
+    w = chunked(lambda m: wl.init_weights(m, "bf16", gen))
+    prev = as_bytes(w)
+    codec.init_caches(prev)
+    steps = [lambda x: wl.step_clustered(x, gen, f=0.22), lambda x: wl.inject_exponent_changes(x, gen, 0.001, 512)]
+    for t, make in enumerate(steps):
+        w_next = chunked(make, like=w)
+        cur = as_bytes(w_next)
+        codec.step(cur)
+        torch.cuda.synchronize()
+        codec.check_status()
+        label = f"beyond 4 GiB, step {t}"
+        codec.canaries.check(label)
+        assert torch.equal(codec.weights_out[: cur.numel()], cur), f"{label}: round trip is not bit-exact"
+        assert torch.equal(codec.sender_cache, codec.receiver_cache), f"{label}: the two caches differ"
+        for ui in picks:
+            u = units[ui]
+            lo, nn, mo, co = int(u["weights_off"]), int(u["n_values"]), int(u["msg_off"]), int(u["cache_off"])
+            wp = prev[lo : lo + nn * 2].cpu().numpy().view(np.uint16)
+            wc = cur[lo : lo + nn * 2].cpu().numpy().view(np.uint16)
+            cache = ora.cache_init(wp, nn, 0)
+            m, wbytes, pay, cb = ora.encode(wc, cache, 0, block)
+            assert int(codec.wire_bytes[ui].item()) == wbytes, f"{label}: length of unit {ui} (N={nn})"
+            assert int(codec.changed_blocks[ui].item()) == cb, f"{label}: changed blocks of unit {ui} (N={nn})"
+            assert np.array_equal(codec.msg_send[mo : mo + wbytes].cpu().numpy(), m), f"{label}: message of unit {ui}"
+            assert np.array_equal(codec.msg_recv[mo : mo + wbytes].cpu().numpy(), m), f"{label}: transported {ui}"
+            assert np.array_equal(codec.sender_cache[co : co + nn].cpu().numpy(), cache), f"{label}: cache of {ui}"
+        q = int(codec.changed_blocks.sum().item()) / codec.n_blocks()
+        assert 0 < q < 0.5
+        del prev
+        w, prev = w_next, cur
+
+    # a third step through the hashed sender (its messages are the exact sender's) and the entropy stage, whose
+    # scratch (one slot per 4096 values) is larger than 4 GiB here as well
+    from oracle import rans_oracle as rans
+
+    codec.init_hash_cache(prev)
+    cur = as_bytes(chunked(lambda x: wl.step_clustered(x, gen, f=0.22), like=w))
+    codec.encode_hashed(cur)
+    torch.cuda.synchronize()
+    hashed_wire, hashed_changed = codec.wire_bytes.clone(), codec.changed_blocks.clone()
+    hashed_msgs = {ui: codec.msg_send[int(units[ui]["msg_off"]) : int(units[ui]["msg_off"]) + int(hashed_wire[ui].item())].clone()
+                   for ui in picks}
+    codec.msg_send.zero_()
+    guard(codec)  # (the fill went over the guard bytes between the slots: arm them again)
+    codec.encode(cur)
+    torch.cuda.synchronize()
+    assert torch.equal(codec.wire_bytes, hashed_wire) and torch.equal(codec.changed_blocks, hashed_changed)
+    raw_msgs = {}
+    for ui in picks:
+        mo = int(units[ui]["msg_off"])
+        raw_msgs[ui] = codec.msg_send[mo : mo + int(hashed_wire[ui].item())].cpu().numpy()
+        assert np.array_equal(raw_msgs[ui], hashed_msgs[ui].cpu().numpy()), f"hashed sender, unit {ui}"
+    assert codec.plan.entropy_scratch_bytes > 2 ** 32
+    codec.entropy_encode()
+    torch.cuda.synchronize()
+    for ui in picks:
+        u = units[ui]
+        want = rans.entropy_encode_message(raw_msgs[ui], int(u["n_values"]), 0, block)
+        assert int(codec.wire_bytes[ui].item()) == want.size, f"coded length of unit {ui}"
+        mo = int(u["msg_off"])
+        assert np.array_equal(codec.msg_send[mo : mo + want.size].cpu().numpy(), want), f"coded message of unit {ui}"
+    assert int(codec.wire_bytes.sum().item()) < int(hashed_wire.sum().item())
+    codec.transport()
+    codec.entropy_decode()
+    codec.decode()
+    torch.cuda.synchronize()
+    codec.check_status()
+    codec.canaries.check("beyond 4 GiB, hashed sender and entropy stage")
+    assert torch.equal(codec.wire_bytes, hashed_wire)
+    assert torch.equal(codec.weights_out[: cur.numel()], cur), "round trip through the entropy stage is not bit-exact"
+    assert torch.equal(codec.sender_cache, codec.receiver_cache)
+
+
 @pytest.mark.parametrize("sizes", [[], [0], [0, 0, 0]])
 @pytest.mark.parametrize("dtype_name", ["bf16", "fp32", "fp16"])
 def test_tables_without_values_run_through_every_entry_point(rt, sizes, dtype_name):
