@@ -546,6 +546,107 @@ def test_buffers_beyond_four_gib(rt):
     assert torch.equal(codec.sender_cache, codec.receiver_cache)
 
 
+def test_one_unit_of_more_than_two_to_the_32_values(rt):
+    """A single unit of 2^32 + 24 581 bf16 values (8.6 GB; 524 292 tiles, a short last block of 5 values): offsets
+    INSIDE the unit pass 2^32 in the sign-plus-mantissa section, in the payload (the look-back carries byte counts
+    beyond 32 bits) and in the caches.  The CPU oracle would need tens of GB of host memory for this, so the
+    message is checked on the device against the definition written with plain torch operations, chunk by
+    chunk: block flags = "some exponent of the block differs", bitmap = the flags LSB-first, sign-plus-mantissa
+    of every value, payload = the exponents of the flagged blocks in order, length and count, caches = the new
+    exponents, output = the input."""
+    ciera, runtime = rt
+    from oracle import ciera_oracle as ora
+
+    free, _ = torch.cuda.mem_get_info()
+    if free < 90e9:
+        pytest.skip("needs 90 GB of free device memory")
+    block, n = 512, 2 ** 32 + 3 * 8192 + 5
+    codec = guard(runtime.LayerCodec.from_tensors([n], 1, "bf16", block, DEV, slack=256))
+    assert len(codec.units) == 1 and int(codec.units[0]["n_values"]) == n
+    nb = -(-n // block)
+    pay_off = ora.payload_offset(n, 0, block)
+    sm_off = pay_off - (n + 15) // 16 * 16
+    assert sm_off == (-(-nb // 8) + 15) // 16 * 16
+    gen = wl.make_generator(99, DEV)
+    chunk = 1 << 28  # a multiple of the block size and of 8 blocks
+    w0 = torch.empty(n, dtype=torch.bfloat16, device=DEV)
+    w1 = torch.empty(n, dtype=torch.bfloat16, device=DEV)
+    for lo in range(0, n, chunk):
+        hi = min(n, lo + chunk)
+        w0[lo:hi] = wl.init_weights(hi - lo, "bf16", gen)
+        w1[lo:hi] = wl.step_clustered(w0[lo:hi], gen, f=0.22)
+    b0, b1 = w0.view(torch.uint8), w1.view(torch.uint8)
+    codec.init_caches(b0)
+    codec.step(b1)
+    torch.cuda.synchronize()
+    codec.check_status()
+    codec.canaries.check("one unit of more than 2^32 values")
+    assert torch.equal(codec.weights_out[: 2 * n], b1), "round trip is not bit-exact"
+
+    def exponents(w):  # bf16: bits 14..7
+        return ((w.view(torch.int16).to(torch.int32) >> 7) & 0xFF).to(torch.uint8)
+
+    def sign_mantissa(w):  # sign << 7 | mantissa
+        v = w.view(torch.int16).to(torch.int32)
+        return (((v >> 8) & 0x80) | (v & 0x7F)).to(torch.uint8)
+
+    msg = codec.msg_send
+    bit_weights = torch.tensor([1, 2, 4, 8, 16, 32, 64, 128], dtype=torch.int32, device=DEV)
+    sent = changed = 0
+    for lo in range(0, n, chunk):
+        hi = min(n, lo + chunk)
+        e0, e1 = exponents(w0[lo:hi]), exponents(w1[lo:hi])
+        assert torch.equal(codec.sender_cache[lo:hi], e1) and torch.equal(codec.receiver_cache[lo:hi], e1), f"caches at {lo}"
+        assert torch.equal(msg[sm_off + lo : sm_off + hi], sign_mantissa(w1[lo:hi])), f"sign-plus-mantissa at {lo}"
+        m = hi - lo
+        diff = e0 != e1
+        pad = (-m) % (8 * block)
+        if pad:
+            diff = torch.cat([diff, torch.zeros(pad, dtype=torch.bool, device=DEV)])
+        flags = diff.view(-1, block).any(dim=1)  # a multiple of 8 flags
+        want_bitmap = (flags.view(-1, 8).to(torch.int32) * bit_weights).sum(dim=1).to(torch.uint8)
+        first_byte = lo // block // 8
+        nbytes = -(-(-(-m // block)) // 8)
+        assert torch.equal(msg[first_byte : first_byte + nbytes], want_bitmap[:nbytes]), f"bitmap at {lo}"
+        mask = flags.repeat_interleave(block)[:m]
+        want_payload = e1[mask]
+        assert torch.equal(msg[pay_off + sent : pay_off + sent + want_payload.numel()], want_payload), f"payload at {lo}"
+        sent += int(want_payload.numel())
+        changed += int(flags.sum().item())
+    assert sent > 2 ** 30 // 2 and int(codec.changed_blocks[0].item()) == changed
+    assert int(codec.wire_bytes[0].item()) == pay_off + sent
+    assert pay_off > 2 ** 32 and torch.equal(codec.msg_recv[: pay_off + sent], msg[: pay_off + sent])
+
+    # the same step by the hashed sender gives the same message; then once through the entropy stage and back
+    # (its chain of launches for long units, a quarter of a million segments)
+    del e0, e1, diff, flags, mask, want_payload, want_bitmap
+    codec.init_caches(b0)
+    codec.init_hash_cache(b0)
+    # (the hashed call writes into msg_send: keep the exact message in msg_recv's place)
+    codec.msg_recv[: pay_off + sent].copy_(msg[: pay_off + sent])
+    msg.zero_()
+    guard(codec)
+    codec.encode_hashed(b1)
+    torch.cuda.synchronize()
+    codec.check_status()
+    assert int(codec.wire_bytes[0].item()) == pay_off + sent and int(codec.changed_blocks[0].item()) == changed
+    assert torch.equal(msg[: pay_off + sent], codec.msg_recv[: pay_off + sent]), "hashed sender's message differs"
+    codec.encode(b1)
+    codec.entropy_encode()
+    torch.cuda.synchronize()
+    coded = int(codec.wire_bytes[0].item())
+    assert pay_off < coded < pay_off + sent * 6 // 10  # exponents of Gaussian weights: well under 5 bits each
+    codec.transport()
+    codec.entropy_decode()
+    codec.decode()
+    torch.cuda.synchronize()
+    codec.check_status()
+    codec.canaries.check("one unit of more than 2^32 values, entropy stage")
+    assert int(codec.wire_bytes[0].item()) == pay_off + sent
+    assert torch.equal(codec.weights_out[: 2 * n], b1), "round trip through the entropy stage is not bit-exact"
+    assert torch.equal(codec.sender_cache[:n], codec.receiver_cache[:n])
+
+
 @pytest.mark.parametrize("sizes", [[], [0], [0, 0, 0]])
 @pytest.mark.parametrize("dtype_name", ["bf16", "fp32", "fp16"])
 def test_tables_without_values_run_through_every_entry_point(rt, sizes, dtype_name):
