@@ -428,6 +428,7 @@ def test_buffers_beyond_four_gib(rt):
     ciera, runtime = rt
     from oracle import ciera_oracle as ora
 
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     if free < 90e9:
         pytest.skip("needs 90 GB of free device memory")
@@ -557,6 +558,7 @@ def test_one_unit_of_more_than_two_to_the_32_values(rt):
     ciera, runtime = rt
     from oracle import ciera_oracle as ora
 
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     if free < 90e9:
         pytest.skip("needs 90 GB of free device memory")
