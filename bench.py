@@ -680,6 +680,7 @@ def main():
     if not args.no_other_configs and rank == 0 and world == 1:
         out["other_configs"] = other_configs(args, device, peak, clocks.get("sm_mhz"))
         out["block_size_sweep"] = block_size_sweep(args, device, peak)
+        out["graph_replay"] = graph_replay_latency(device)
 
     # ---- end to end through the host-buffer entry point (weights start and end in host memory)
     if not args.no_e2e:
@@ -858,6 +859,67 @@ def one_layer_case(args, device, peak, over, steps=5, clocks_mhz=None):
     del layers, wa, wb, pipe
     torch.cuda.empty_cache()
     return res
+
+
+def graph_replay_latency(device, reps=200):
+    """Small tables are bound by launch latency, not by HBM: config 1 (1024 x 512 bf16, 4 shards) and one expert's
+    three matrices on 16 shards, stepped eagerly through the binding and replayed from a CUDA graph that holds two
+    steps (A -> B -> A).  Microseconds per step (encode + transport + decode), CUDA events around `reps` pairs."""
+    import torch
+
+    from paper_2609_04609_b200 import runtime
+    from paper_2609_04609_b200 import workloads as wl
+
+    out = {"per": "step = encode + transport + decode of the whole table, one stream; us"}
+    cases = {"config1_1024x512_bf16_4_shards": ([1024 * 512], 4),
+             "one_expert_3_matrices_bf16_16_shards": ([r * c for r, c in wl.olmoe_layer_shapes(1)], 16)}
+    for name, (sizes, shards) in cases.items():
+        try:
+            codec = runtime.LayerCodec.from_tensors(sizes, shards, "bf16", 512, device)
+            gen = wl.make_generator(11, device)
+            n = codec.weights_bytes // 2
+            wa = wl.init_weights(n, "bf16", gen)
+            wb = wl.step_clustered(wa, gen, f=0.22)
+            a, b = wa.view(torch.uint8), wb.view(torch.uint8)
+            codec.init_caches(a)
+            stream = torch.cuda.Stream(device)
+            with torch.cuda.stream(stream):
+                for _ in range(3):
+                    codec.step(b)
+                    codec.step(a)
+                stream.synchronize()
+
+                def timed(fn):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    for _ in range(reps):
+                        fn()
+                    e1.record()
+                    e1.synchronize()
+                    return e0.elapsed_time(e1) * 1e3 / (2 * reps)
+
+                def eager():
+                    codec.step(b)
+                    codec.step(a)
+
+                eager_us = timed(eager)
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                codec.step(b)
+                codec.step(a)
+            with torch.cuda.stream(stream):
+                graph.replay()
+                graph_us = timed(graph.replay)
+            torch.cuda.synchronize()
+            codec.check_status()
+            ok = all(torch.equal(codec.weights_out[int(u["weights_off"]): int(u["weights_off"]) + 2 * int(u["n_values"])],
+                                 a[int(u["weights_off"]): int(u["weights_off"]) + 2 * int(u["n_values"])])
+                     for u in codec.units)
+            out[name] = {"values": int(codec.plan.total_values), "units": len(codec.units), "eager_us": eager_us,
+                         "graph_us": graph_us, "verified_bit_exact": bool(ok)}
+        except Exception as e:
+            out[name] = {"error": f"{type(e).__name__}: {e}"}
+    return out
 
 
 def block_size_sweep(args, device, peak):

@@ -23,6 +23,11 @@
  *     that is part of the library image, for callers that cannot supply scratch.)
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Device work is
  *     enqueued on it and the call returns without waiting, unless stated otherwise.
+ *     The sender, transport, receiver and entropy calls read every size they need on the device
+ *     and leave their scratch as they found it, so a step may be captured in a CUDA graph and
+ *     replayed; call each entry point once outside a capture first (its first call on a device
+ *     queries occupancy and sets kernel attributes).  The host-side launch counter does not see
+ *     replays.
  *   - Errors found on the device (a wait that ran out, a message whose length contradicts its
  *     bitmap) are written to the caller's `status_dev` word: 0 = none, otherwise the first
  *     ciera_status that was raised.  The word is only ever written on error; clear it yourself.

@@ -262,6 +262,40 @@ def test_pipelined_stack_equals_serial(rt):
             assert torch.equal(x, y)
 
 
+@pytest.mark.parametrize("sizes,dtype,block", [([3_000_005, 131_072, 70_001], 0, 512), ([200_000, 5, 8192 * 3], 0, 4),
+                                               ([131_072, 70_001], 1, 64), ([131_072, 70_001], 2, 512)])
+def test_steps_replayed_from_a_cuda_graph(rt, sizes, dtype, block):
+    """A whole step (sender, transport, receiver) is a handful of kernel launches that read their sizes on the
+    device and leave the scratch as they found it, so it can be captured once in a CUDA graph and replayed on new
+    weights in the same buffer.  Every replay must equal the oracle's step bit for bit, with a long unit
+    (cooperative launch, prefix kernel) in the table as well."""
+    ciera, runtime = rt
+    name = {0: "bf16", 1: "fp32", 2: "fp16"}[dtype]
+    codec = guard(runtime.LayerCodec.from_tensors(sizes, 2, name, block, DEV, slack=256))
+    table = OracleTable(codec.units, dtype, block, codec.cache_bytes, codec.msg_bytes)
+    n = codec.weights_bytes // wl.VALUE_BYTES[name]
+    traj = [wl.as_bits(w) for w in wl.trajectory(n, name, 321 + block, 4, "clustered", f=0.3)]
+    codec.init_caches(to_dev_bytes(traj[0], DEV))
+    table.init_caches(traj[0])
+    w_in = to_dev_bytes(traj[1], DEV).clone()
+    codec.step(w_in)  # outside the capture first: the first calls query occupancy and set kernel attributes
+    torch.cuda.synchronize()
+    codec.check_status()
+    compare_step(codec, table.step(traj[1]), traj[1], "eager")
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=torch.cuda.Stream()):
+        codec.step(w_in)
+    for t in (2, 3, 4):
+        w_in.copy_(to_dev_bytes(traj[t], DEV))
+        graph.replay()
+        torch.cuda.synchronize()
+        codec.check_status()
+        exp = table.step(traj[t])
+        compare_step(codec, exp, traj[t], f"replay t={t}")
+        compare_caches(codec, table, f"replay t={t}")
+        compare_recon(codec, exp, traj[t], dtype, f"replay t={t}")
+
+
 @pytest.mark.parametrize("n_layers", [1, 3])
 def test_pipeline_of_many_iterations_reuses_layer_buffers_safely(rt, n_layers):
     """Many iterations back to back on two streams, alternating between two iterates: with a single
