@@ -476,6 +476,9 @@ def main():
     import torch
     import torch.distributed as dist
 
+    from paper_2609_04609_b200 import build as libbuild
+
+    libbuild.ensure_library()  # a fresh checkout: built once, in-tree; an existing library is used as it is
     from paper_2609_04609_b200 import ciera, runtime
     from paper_2609_04609_b200 import workloads as wl
 

@@ -36,14 +36,35 @@ def needs_build() -> bool:
 def build_library(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return LIB
-    cmd = [_nvcc(), "-shared", "-o", LIB, "-I", os.path.join(ROOT, "include"), "-I", CSRC] + NVCC_FLAGS
+    tmp = f"{LIB}.{os.getpid()}.tmp"  # built beside its place and moved there whole: nobody loads half a library
+    cmd = [_nvcc(), "-shared", "-o", tmp, "-I", os.path.join(ROOT, "include"), "-I", CSRC] + NVCC_FLAGS
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or res.returncode != 0:
         print(res.stdout)
         print(res.stderr)
     if res.returncode != 0:
+        if os.path.exists(tmp):
+            os.remove(tmp)
         raise RuntimeError("nvcc failed building libciera.so")
+    os.replace(tmp, LIB)
+    return LIB
+
+
+def ensure_library(wait_s: float = 600.0) -> str:
+    """Builds the library if it is not there at all (a fresh checkout); a library that is there is used as it
+    is.  Of several processes started together (one per GPU) the one with LOCAL_RANK 0 builds, the others wait."""
+    import time
+
+    if os.path.exists(LIB):
+        return LIB
+    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        return build_library(force=True)
+    t0 = time.time()
+    while not os.path.exists(LIB):
+        if time.time() - t0 > wait_s:
+            raise RuntimeError("libciera.so did not appear: build it with python -m paper_2609_04609_b200.build")
+        time.sleep(1.0)
     return LIB
 
 

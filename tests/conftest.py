@@ -10,6 +10,13 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
+    # a fresh checkout has no built library yet (it is not tracked): build it once, in-tree
+    try:
+        from paper_2609_04609_b200 import build as libbuild
+
+        libbuild.ensure_library()
+    except Exception as e:  # the tests that need it will say so
+        print(f"libciera.so could not be built: {e}", file=sys.stderr)
 
 
 @pytest.fixture(scope="session")
