@@ -183,7 +183,8 @@ CIERA_API int ciera_cache_update(const ciera_plan* plan, void* cache_dev, const 
  *                            entry -- see ciera_workspace_init -- and handed back all zero; must not
  *                            be shared by calls that can overlap on the GPU
  *   status_dev          i/o  device error word (may be NULL)
- * One kernel launch for the whole table, nothing else.
+ * One kernel launch for the whole table, nothing else (a table that holds empty units: two small
+ * clearing operations in front of it, which write those units' zero lengths and counts).
  */
 CIERA_API int ciera_encode(const ciera_plan* plan, const void* weights_dev, void* sender_cache_dev, void* messages_dev,
                  uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* workspace_dev,
