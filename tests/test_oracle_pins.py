@@ -398,7 +398,7 @@ def test_fp16_byte_count_and_layout_over_ragged_sizes(oracle):
     """S_{s+m} = ceil(11 N / 8), every changed block ceil(5 L / 8) bytes, capacity = all blocks changed."""
     rng = np.random.default_rng(23)
     for n, block in [(1, 64), (5, 2), (7, 8), (63, 64), (65, 64), (1000, 128), (4097, 512), (12345, 4096), (33, 1),
-                     (8193, 32), (100, 3)]:
+                     (8193, 32), (100, 3), (1000, 4), (4099, 1), (777, 8), (2050, 2)]:
         w_prev = rng.integers(0, 1 << 16, size=n, dtype=np.uint64).astype(np.uint16)
         w = w_prev.copy()
         flip = rng.random(n) < 0.05

@@ -151,7 +151,8 @@ def test_the_32_entry_table_is_the_256_entry_one_cut_short():
         rans.decode(bad, 100, 32)
 
 
-@pytest.mark.parametrize("n,block", [(70_001, 512), (8192, 64), (1000, 32), (40_003, 4096), (5_000, 16)])
+@pytest.mark.parametrize("n,block", [(70_001, 512), (8192, 64), (1000, 32), (40_003, 4096), (5_000, 16), (30_001, 4),
+                                     (25_000, 1), (20_003, 8), (9_999, 2)])
 def test_message_level_stage_on_fp16_exponents(oracle, n, block):
     """fp16: the payload holds five bits per exponent, every changed block starting on a byte boundary.  The
     symbols the stage codes are the exponents themselves: unpacked they equal the exponent fields of the changed
