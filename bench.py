@@ -737,6 +737,7 @@ OTHER_CONFIGS = [
     ("block1_half_of_the_exponents_change", dict(block=1, update="inject", inject=0.5, inject_seg=0)),
     ("block64_adam_like_update", dict(block=64, update="adam")),
     ("fp16_clustered", dict(dtype="fp16")),
+    ("fp16_block1_adam_like_update", dict(dtype="fp16", block=1, update="adam")),
     ("hashed_sender_bf16_block512", dict(detect="hash")),
     ("hashed_sender_bf16_block32_adam_like_update", dict(detect="hash", block=32, update="adam")),
     ("hashed_sender_fp32_block512", dict(detect="hash", dtype="fp32")),

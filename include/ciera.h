@@ -87,10 +87,12 @@ typedef enum ciera_dtype {
                        wire its exponents take 5 bits and its sign-plus-mantissa 11 bits each, packed
                        without gaps (value j of a section at bits [j*w, (j+1)*w), bit i of a section =
                        byte i >> 3, bit i & 7); every changed block of the payload starts on a byte
-                       boundary; the caches still hold one byte per value.  Blocks of 16 values and
-                       more; the hashed sender takes it too, and so does the entropy stage,
-                       which codes the 5-bit exponents as symbols of their own (it undoes the
-                       packing first; 32 table entries travel instead of 256). */
+                       boundary (a block of 1, 2, 4, 8, 16 ... values takes 1, 2, 3, 5, 10 ... bytes);
+                       the caches still hold one byte per value.  Every block size; the hashed
+                       sender takes it too (blocks of 16 values and more, as for the other
+                       precisions), and so does the entropy stage, which codes the 5-bit exponents
+                       as symbols of their own (it undoes the packing first; 32 table entries
+                       travel instead of 256). */
 } ciera_dtype;
 
 /* One unit = one shard of one tensor.  All offsets are in BYTES from the base pointer of the

@@ -442,6 +442,13 @@ struct Piece<CIERA_FP16> {
     __device__ __forceinline__ void load_exp_partial(const uint8_t* src, int nvalid) { load_bytes_partial<8>(e, src, nvalid); }
     __device__ __forceinline__ void store_exp_partial(uint8_t* dst, int nvalid) const { store_bytes_partial<8>(dst, e, nvalid); }
     __device__ __forceinline__ bool differs(const Piece& o) const { return ((e[0] ^ o.e[0]) | (e[1] ^ o.e[1])) != 0; }
+    // one flag per block of 2^log2b values (log2b <= 3), lowest block first (the exponents lie one byte each, as for bf16)
+    __device__ __forceinline__ uint32_t block_flags(const Piece& o, uint32_t log2b) const {
+        if (log2b >= 3) return differs(o) ? 1u : 0u;
+        if (log2b == 0) return value_flags8(e[0] ^ o.e[0], e[1] ^ o.e[1]);
+        const uint32_t per_word = 4u >> log2b;
+        return word_block_flags(e[0] ^ o.e[0], log2b) | (word_block_flags(e[1] ^ o.e[1], log2b) << per_word);
+    }
 
     // the 8 exponents as 40 bits: low word and high byte
     __device__ __forceinline__ void pack_exponents(uint32_t& lo, uint32_t& hi) const {

@@ -70,6 +70,15 @@ struct DecodeCfg<CIERA_BF16, true> {
     static constexpr int kRing = 10;
 };
 template <>
+struct DecodeCfg<CIERA_FP16, true> {
+    // 4 x (11 KB sm + 8 KB cache span + 8 KB payload slice): one block per SM (two blocks with two stages each
+    // measured slower: 0.70 against 0.56 ms per layer)
+    static constexpr int kStages = 4;
+    static constexpr int kBlocksPerSM = 1;
+    static constexpr bool kStageOut = false;
+    static constexpr int kRing = 10;
+};
+template <>
 struct DecodeCfg<CIERA_FP32, true> {
     static constexpr int kStages = 4;
     static constexpr int kBlocksPerSM = 1;
@@ -312,9 +321,40 @@ __device__ __forceinline__ void unchanged_span_fine(const uint32_t* bm, uint32_t
 // Exponents of the changed blocks of one piece, fine blocks: `km` holds the piece's block flags,
 // `src` points at the exponents of its first changed block; they replace the cached exponents in
 // x.e value by value.  Only the first nvalid values exist.
+// (fp16: a changed block's exponents lie five bits each in 1, 2, 3 or 5 bytes for 1, 2, 4 or 8 values; the piece's
+// changed blocks take 8 bytes at most, read byte by byte -- never past the last block's bytes -- into one 64-bit
+// word from which every value of a changed block picks its field.)
 template <int DT, class M>
 __device__ __forceinline__ void gather_changed(Piece<DT>& x, uint32_t km, uint32_t log2b, const uint8_t* src, int nvalid) {
     constexpr int kV = Piece<DT>::kValues;
+    if constexpr (DT == CIERA_FP16) {
+        const uint32_t B = 1u << log2b;
+        const uint32_t block_bytes = (uint32_t)payload_bytes_of_blocks<DT>(1, log2b);
+        // bytes of the piece's changed blocks (a short last block of the unit carries fewer)
+        uint32_t nbytes = 0;
+#pragma unroll
+        for (int j = 0; j < kV; ++j) {
+            if (j < (kV >> log2b) && ((km >> j) & 1u)) {
+                const int len = min((int)B, nvalid - (j << log2b));
+                nbytes += len > 0 ? (5u * (uint32_t)len + 7u) >> 3 : 0u;
+            }
+        }
+        unsigned long long v = 0;
+#pragma unroll
+        for (uint32_t k = 0; k < 8u; ++k)
+            if (k < nbytes) v |= (unsigned long long)M::ld1(src + k) << (8u * k);
+#pragma unroll
+        for (int i = 0; i < kV; ++i) {
+            const uint32_t j = (uint32_t)i >> log2b;
+            if (((km >> j) & 1u) && i < nvalid) {
+                const uint32_t at = 8u * block_bytes * (uint32_t)__popc(km & ((1u << j) - 1u)) + 5u * ((uint32_t)i & (B - 1u));
+                const uint32_t b = (uint32_t)(v >> at) & 31u;
+                const uint32_t sel = (i & 3) == 0 ? 0x3214u : (i & 3) == 1 ? 0x3240u : (i & 3) == 2 ? 0x3410u : 0x4210u;
+                x.e[i >> 2] = __byte_perm(x.e[i >> 2], b, sel);
+            }
+        }
+        return;
+    }
     if (nvalid == kV && log2b != 0) {
         // a complete piece of blocks of 2, 4 or 8 values: a changed block's exponents come with one load
         // (the payload holds whole blocks up to here, so `src` is a multiple of the block size)
@@ -370,7 +410,8 @@ __device__ __forceinline__ void gather_changed(Piece<DT>& x, uint32_t km, uint32
 template <int DT, bool FINE>
 __host__ __device__ constexpr uint32_t decode_stage_bytes() {
     return (uint32_t)sm_bytes_of_values<DT>(kTileValues) + (uint32_t)kTileValues +
-           (uint32_t)payload_bytes_of_blocks<DT>(kTileValues >> 5, 5) + ((FINE || DT == CIERA_FP16) ? 16u : 0u);
+           (FINE ? (uint32_t)kTileValues : (uint32_t)payload_bytes_of_blocks<DT>(kTileValues >> 5, 5)) +
+           ((FINE || DT == CIERA_FP16) ? 16u : 0u);
 }
 
 template <int DT, bool FINE>
@@ -382,7 +423,6 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
     constexpr int VB = Traits<DT>::kValueBytes;
     constexpr int SMB = Traits<DT>::kSmBytes;  // (not used for fp16)
     constexpr bool kHalf = DT == CIERA_FP16;    // packed sections: see Piece<CIERA_FP16>
-    static_assert(!(kHalf && FINE), "fp16 takes blocks of 16 values and more");
     using Cfg = DecodeCfg<DT, FINE>;
     constexpr int S = Cfg::kStages;
     constexpr int kDecRing = Cfg::kRing;
@@ -632,7 +672,18 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                     const uint32_t rank = r->pre[kb >> 5] + __popc(word & ((1u << (kb & 31u)) - 1u));
                     P x;
                     bool chg;
-                    if constexpr (kHalf) {
+                    if constexpr (kHalf && FINE) {
+                        // 11 packed bytes of sign-plus-mantissa; the piece's flags pick, block by block
+                        x.template load_sm_group<Shared>(st, t0 >> 3, lane);
+                        const uint32_t km = (word >> (kb & 31u)) & ((1u << (P::kValues >> log2b)) - 1u);
+                        chg = km != 0;
+                        x.template load_exp_full<Shared>(st + kSmTile + t0);
+                        if (chg)
+                            gather_changed<DT, Shared>(x, km, log2b,
+                                                       st + kSmTile + kTileValues + r->pay_skew +
+                                                           (size_t)payload_bytes_of_blocks<DT>(rank, log2b),
+                                                       P::kValues);
+                    } else if constexpr (kHalf) {
                         // 11 packed bytes of sign-plus-mantissa; 5 packed bytes of exponents if the block changed
                         x.template load_sm_group<Shared>(st, t0 >> 3, lane);
                         chg = (word >> (kb & 31u)) & 1u;
@@ -697,7 +748,19 @@ decode_kernel(const TileDesc* __restrict__ tiles, uint32_t n_tiles, uint32_t log
                     const bool chg = km != 0;
                     const uint8_t* esrc = (chg && !FINE) ? pay_src + ((size_t)rank << log2b) + (t0 & bmask) : c_ptr + t0;
                     P x;
-                    if constexpr (kHalf) {
+                    if constexpr (kHalf && FINE) {
+                        x.load_sm_bytes(sm_src + (size_t)11 * (t0 >> 3), nvalid);
+                        x.load_exp_partial(c_ptr + t0, nvalid);
+                        if (chg) {
+                            gather_changed<DT, Global>(x, km, log2b, pay_src + (size_t)payload_bytes_of_blocks<DT>(rank, log2b),
+                                                       nvalid);
+                            x.store_exp_partial(c_ptr + t0, nvalid);
+                        }
+                        if (nvalid == P::kValues)
+                            x.template merge_store_full<Global>(w_dst + (size_t)t0 * VB);
+                        else
+                            x.merge_store_partial(w_dst + (size_t)t0 * VB, nvalid);
+                    } else if constexpr (kHalf) {
                         x.load_sm_bytes(sm_src + (size_t)11 * (t0 >> 3), nvalid);
                         if (chg) {
                             x.template load_packed_exponents<Global>(
@@ -929,10 +992,12 @@ extern "C" int ciera_decode(const ciera_plan* p, const void* messages_dev, void*
         int rc = check_launch();
         if (rc) return rc;
     }
-    if (p->dtype == CIERA_FP16)
-        return launch_decode<CIERA_FP16, false>(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,
-                                                ws_prefix, ticket, status_dev, s);
     const bool fine = is_fine(p->log2b);
+    if (p->dtype == CIERA_FP16)
+        return fine ? launch_decode<CIERA_FP16, true>(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,
+                                                      ws_prefix, ticket, status_dev, s)
+                    : launch_decode<CIERA_FP16, false>(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,
+                                                       ws_prefix, ticket, status_dev, s);
     if (p->dtype == CIERA_BF16)
         return fine ? launch_decode<CIERA_BF16, true>(p, messages_dev, receiver_cache_dev, weights_out_dev, wire_bytes_dev,
                                                       ws_prefix, ticket, status_dev, s)

@@ -96,6 +96,8 @@ struct EncodeCfg<CIERA_BF16, true> {
     static constexpr int kBmWords = kFineBitmapWords;
 };
 template <>
+struct EncodeCfg<CIERA_FP16, true> : EncodeCfg<CIERA_BF16, true> {};  // the tile sizes of bf16
+template <>
 struct EncodeCfg<CIERA_FP32, true> {
     static constexpr int kWStages = 2;
     static constexpr int kEStages = 3;
@@ -634,7 +636,9 @@ __device__ __forceinline__ void copy_block(uint8_t* dst, const uint8_t* s_src) {
 // unchanged ones among them equal the cached ones).  A store of single changed bytes would leave the sector
 // partly written in the L2 cache, to be completed from DRAM before it can be written back; whole sectors cost
 // the same DRAM traffic and one store instruction per thread instead of one per changed value.
-template <int LB>
+// (fp16: a changed block's exponents go out five bits each, the block rounded up to whole bytes -- 1, 2, 3 or 5
+// bytes for 1, 2, 4 or 8 values -- and byte by byte, since such blocks start on any byte.)
+template <int DT, int LB>
 __device__ __forceinline__ void write_changed_fine(const EncodeTileInfo& ti, const uint32_t* bm, const uint16_t* pre,
                                                    uint64_t base, const uint8_t* s_exp, uint32_t tid) {
     constexpr uint32_t B = 1u << LB;
@@ -653,6 +657,26 @@ __device__ __forceinline__ void write_changed_fine(const EncodeTileInfo& ti, con
     }
     if (bits == 0) return;
     const uint32_t rank = (uint32_t)pre[bit0 >> 5] + __popc(word & ((1u << sh) - 1u));
+    if constexpr (DT == CIERA_FP16) {
+        constexpr uint32_t kBlockBytes = (uint32_t)payload_bytes_of_blocks<DT>(1, LB);
+        uint8_t* pdst = ti.pay_dst + base + (uint64_t)rank * kBlockBytes;
+        while (bits) {
+            const uint32_t j = (uint32_t)__ffs(bits) - 1u;
+            bits &= bits - 1u;
+            const uint32_t v = (bit0 + j) << LB;
+            const uint32_t len = min(B, ti.nv - v);  // the unit's last block may be short
+            unsigned long long packed = 0;
+#pragma unroll
+            for (uint32_t i = 0; i < B; ++i)
+                if (i < len) packed |= (unsigned long long)(s_exp[v + i] & 31u) << (5u * i);
+            const uint32_t nbytes = (5u * len + 7u) >> 3;
+#pragma unroll
+            for (uint32_t k = 0; k < kBlockBytes; ++k)
+                if (k < nbytes) pdst[k] = (uint8_t)(packed >> (8u * k));
+            pdst += kBlockBytes;
+        }
+        return;
+    }
     uint8_t* pdst = ti.pay_dst + base + ((uint64_t)rank << LB);
     while (bits) {
         const uint32_t j = (uint32_t)__ffs(bits) - 1u;
@@ -742,7 +766,8 @@ __device__ __forceinline__ void send_changed(const EncodeTileInfo& ti, uint32_t 
             write_changed<DT, HASH == 0, true>(ti, log2b, bm, pre, base, s_exp, tid);
         else
             write_changed<DT, HASH == 0, false>(ti, log2b, bm, pre, base, s_exp, tid);
-    } else if (ti.nv == (uint32_t)kTileValues && tile_payload_bytes >= (uint32_t)kTileValues / kGatherDensity) {
+    } else if (DT != CIERA_FP16 && ti.nv == (uint32_t)kTileValues &&
+               tile_payload_bytes >= (uint32_t)kTileValues / kGatherDensity) {
         // a full tile in which many exponents changed: gathered in shared memory, written out in whole pieces
         switch (log2b) {
             case 0: write_changed_fine_full<0>(ti, bm, pre, base, s_exp, s_gather, tid); break;
@@ -750,12 +775,12 @@ __device__ __forceinline__ void send_changed(const EncodeTileInfo& ti, uint32_t 
             case 2: write_changed_fine_full<2>(ti, bm, pre, base, s_exp, s_gather, tid); break;
             default: write_changed_fine_full<3>(ti, bm, pre, base, s_exp, s_gather, tid); break;
         }
-    } else {  // few changes (a store per changed block is cheaper than the gathering), or a unit's last, short tile
+    } else {  // few changes (a store per changed block is cheaper than the gathering), a unit's last, short tile, or fp16
         switch (log2b) {
-            case 0: write_changed_fine<0>(ti, bm, pre, base, s_exp, tid); break;
-            case 1: write_changed_fine<1>(ti, bm, pre, base, s_exp, tid); break;
-            case 2: write_changed_fine<2>(ti, bm, pre, base, s_exp, tid); break;
-            default: write_changed_fine<3>(ti, bm, pre, base, s_exp, tid); break;
+            case 0: write_changed_fine<DT, 0>(ti, bm, pre, base, s_exp, tid); break;
+            case 1: write_changed_fine<DT, 1>(ti, bm, pre, base, s_exp, tid); break;
+            case 2: write_changed_fine<DT, 2>(ti, bm, pre, base, s_exp, tid); break;
+            default: write_changed_fine<DT, 3>(ti, bm, pre, base, s_exp, tid); break;
         }
     }
 }
@@ -1204,8 +1229,10 @@ static int launch_encode_any(const ciera_plan* p, const void* weights_dev, void*
                              cudaStream_t s) {
     const bool fine = is_fine(p->log2b);
     if (p->dtype == CIERA_FP16)
-        return launch_encode<CIERA_FP16, false>(p, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
-                                                changed_blocks_dev, scratch, status_dev, s);
+        return fine ? launch_encode<CIERA_FP16, true>(p, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
+                                                      changed_blocks_dev, scratch, status_dev, s)
+                    : launch_encode<CIERA_FP16, false>(p, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
+                                                       changed_blocks_dev, scratch, status_dev, s);
     if (p->dtype == CIERA_BF16)
         return fine ? launch_encode<CIERA_BF16, true>(p, weights_dev, sender_cache_dev, messages_dev, wire_bytes_dev,
                                                       changed_blocks_dev, scratch, status_dev, s)
@@ -1217,7 +1244,7 @@ static int launch_encode_any(const ciera_plan* p, const void* weights_dev, void*
                                                    changed_blocks_dev, scratch, status_dev, s);
 }
 
-// the sender with HashCache: blocks of 16 values and more, fp16 from 32 (checked by the caller)
+// the sender with HashCache: blocks of 16 values and more (checked by the caller)
 int launch_encode_hashed(const ciera_plan* p, const void* weights_dev, void* hash_cache_dev, void* messages_dev,
                          uint64_t* wire_bytes_dev, uint32_t* changed_blocks_dev, void* scratch, int32_t* status_dev,
                          cudaStream_t s) {

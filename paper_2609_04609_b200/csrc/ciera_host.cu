@@ -97,7 +97,6 @@ extern "C" int ciera_plan_create(const ciera_unit* units_host, uint32_t n_units,
     if (block == 0) return CIERA_ERR_INVALID_ARG;
     int l2 = exact_log2(block);
     if (l2 < 0 || block < CIERA_MIN_BLOCK || block > CIERA_MAX_BLOCK) return CIERA_ERR_UNSUPPORTED;
-    if (dtype == CIERA_FP16 && block < 16) return CIERA_ERR_UNSUPPORTED;
 
     uint64_t n_tiles = 0, total = 0;
     for (uint32_t u = 0; u < n_units; ++u) {

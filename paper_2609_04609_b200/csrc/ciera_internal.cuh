@@ -79,7 +79,8 @@ __host__ __device__ constexpr uint64_t sm_bytes_of_values(uint64_t values) {
 }
 template <int DT>
 __host__ __device__ constexpr uint64_t payload_bytes_of_blocks(uint64_t blocks, uint32_t log2b) {
-    return DT == CIERA_FP16 ? blocks * (5ull << (log2b - 3)) : blocks << log2b;
+    // fp16: five bits per exponent, a block rounded up to whole bytes (1, 2, 3, 5, 10, 20, ... bytes)
+    return DT == CIERA_FP16 ? blocks * (((5ull << log2b) + 7ull) >> 3) : blocks << log2b;
 }
 
 __host__ __device__ inline uint64_t pad16(uint64_t x) { return (x + 15ull) & ~15ull; }

@@ -106,7 +106,7 @@ def test_entropy_stage_reduced_moe_layer(rt, dtype):
     assert coded > 0
 
 
-@pytest.mark.parametrize("block", [16, 32, 64, 512, 4096])
+@pytest.mark.parametrize("block", [1, 2, 4, 8, 16, 32, 64, 512, 4096])
 def test_entropy_stage_fp16(rt, block):
     """fp16: the stage codes the five-bit exponents as symbols of their own (unpacked before, packed after the
     coder, 32 table entries); ragged units from empty caches (large payloads), a reduced MoE layer under the

@@ -46,7 +46,7 @@ def _run(rt, sizes, shards, block, traj_fn, zero_cache=False, label=""):
     return stats
 
 
-@pytest.mark.parametrize("block", [16, 32, 64, 128, 256, 512, 1024, 2048, 4096])
+@pytest.mark.parametrize("block", [1, 2, 4, 8, 16, 32, 64, 128, 256, 512, 1024, 2048, 4096])
 def test_fp16_ragged_units_every_block_size(rt, block):
     """Units shorter than a block, not multiples of 8 / of the block / of the tile, empty units;
     random bit patterns (NaN, Inf, subnormals, both zeros included)."""
@@ -64,7 +64,8 @@ def test_fp16_ragged_units_every_block_size(rt, block):
 
 
 @pytest.mark.parametrize("block,model,kw", [(512, "adam", {}), (512, "clustered", {"f": 0.22}), (64, "clustered", {"f": 0.5}),
-                                            (32, "adam", {}), (16, "adam", {})])
+                                            (32, "adam", {}), (16, "adam", {}), (8, "adam", {}), (4, "adam", {}),
+                                            (2, "adam", {}), (1, "adam", {}), (1, "clustered", {"f": 0.3})])
 def test_fp16_reduced_moe_layer(rt, block, model, kw):
     sizes = [r * c for r, c in wl.olmoe_layer_shapes(2)] + [70_001, 17, 0]
     stats = _run(rt, sizes, 4, block, lambda n: [wl.as_bits(w) for w in wl.trajectory(n, "fp16", 31 + block, 3, model, **kw)],
@@ -74,7 +75,7 @@ def test_fp16_reduced_moe_layer(rt, block, model, kw):
          zero_cache=True, label=f"fp16-moe-zero-B{block}")
 
 
-@pytest.mark.parametrize("block,c", [(512, 0.001), (64, 0.01), (4096, 0.3), (32, 0.05), (16, 0.1)])
+@pytest.mark.parametrize("block,c", [(512, 0.001), (64, 0.01), (4096, 0.3), (32, 0.05), (16, 0.1), (8, 0.01), (2, 0.3), (1, 0.02)])
 def test_fp16_long_units_of_many_tiles(rt, block, c):
     def traj(n):
         gen = wl.make_generator(4242 + block)
@@ -90,12 +91,14 @@ def test_fp16_sizes_and_limits(rt):
     ciera, runtime = rt
     from oracle import ciera_oracle as ora
     for n in (0, 1, 7, 8, 9, 1000, 131072, 70001):
-        for block in (32, 512, 4096):
+        for block in (1, 2, 4, 8, 32, 512, 4096):
             assert ciera.payload_offset(n, FP16, block) == ora.payload_offset(n, FP16, block)
             assert ciera.message_capacity(n, FP16, block) == ora.message_capacity(n, FP16, block)
             assert ciera.message_bytes(n, FP16, block, 17) == ora.paper_bytes(n, FP16, block, 17)
+    codec = runtime.LayerCodec.from_tensors([1000], 1, "fp16", 8, DEV)  # every block size from 1 value on
     with pytest.raises(ciera.CieraError) as e:
-        runtime.LayerCodec.from_tensors([1000], 1, "fp16", 8, DEV)
+        codec.init_hash_cache(None)
+        codec.encode_hashed(codec.weights_out)  # the hashed sender: blocks of 16 values and more
     assert e.value.status == ciera.ERR_UNSUPPORTED
     codec = runtime.LayerCodec.from_tensors([1000], 1, "fp16", 64, DEV)
     codec.init_hash_cache(None)  # the hashed sender and the entropy stage take fp16 (test_gpu_hashed.py, test_gpu_entropy.py)

@@ -43,8 +43,6 @@ def _random_case(seed):
     shards = int(rng.choice([1, 1, 2, 3, 8]))
     dtype = int(rng.integers(0, 3))
     block = int(rng.choice(BLOCKS))
-    if dtype == 2:
-        block = max(block, 16)  # fp16: blocks of 16 values and more
     return rng, sizes, shards, dtype, block
 
 

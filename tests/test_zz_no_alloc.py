@@ -65,7 +65,7 @@ def test_noalloc_encode_equals_encode_on_two_calls_in_a_row(dtype, block):
         assert torch.equal(new.weights_out[lo : lo + nb], traj[2][lo : lo + nb])
 
 
-@pytest.mark.parametrize("dtype,block", [("bf16", 512), ("bf16", 4), ("fp16", 64), ("fp32", 1)])
+@pytest.mark.parametrize("dtype,block", [("bf16", 512), ("bf16", 4), ("fp16", 64), ("fp16", 2), ("fp32", 1)])
 def test_noalloc_encode_with_long_units_equals_the_oracle(dtype, block):
     """Units of more than 32 tiles are spread over the thread blocks: their tiles find their place in the payload by
     a look-back over the status words in the built-in scratch, and the launch is a cooperative one.  The messages are
