@@ -296,6 +296,56 @@ def test_steps_replayed_from_a_cuda_graph(rt, sizes, dtype, block):
         compare_recon(codec, exp, traj[t], dtype, f"replay t={t}")
 
 
+@pytest.mark.parametrize("dtype,block", [(0, 512), (1, 4), (2, 64)])
+def test_resume_from_saved_caches_or_from_the_weights(rt, dtype, block):
+    """The codec's only persistent state are the two exponent caches (and the sender's HashCache), plain buffers of
+    the caller.  A run is resumed either by putting saved copies of them back into fresh buffers, or -- since
+    after every step both caches hold exactly the exponents of the weights just sent -- by rebuilding them from
+    those weights.  Both ways the next step is the one the uninterrupted run makes, bit for bit."""
+    ciera, runtime = rt
+    name = {0: "bf16", 1: "fp32", 2: "fp16"}[dtype]
+    sizes = [300_001, 131_072, 70_001]
+
+    def fresh():
+        return guard(runtime.LayerCodec.from_tensors(sizes, 2, name, block, DEV, slack=256))
+
+    first = fresh()
+    table = OracleTable(first.units, dtype, block, first.cache_bytes, first.msg_bytes)
+    n = first.weights_bytes // wl.VALUE_BYTES[name]
+    traj = [wl.as_bits(w) for w in wl.trajectory(n, name, 77 + block, 3, "clustered", f=0.3)]
+    first.init_caches(to_dev_bytes(traj[0], DEV))
+    table.init_caches(traj[0])
+    for t in (1, 2):
+        first.step(to_dev_bytes(traj[t], DEV))
+        torch.cuda.synchronize()
+        first.check_status()
+        compare_step(first, table.step(traj[t]), traj[t], f"t={t}")
+    saved_s, saved_r = first.sender_cache.cpu(), first.receiver_cache.cpu()  # the checkpoint
+    want = table.step(traj[3])  # what the uninterrupted run does next
+
+    restored = fresh()
+    restored.sender_cache.copy_(saved_s)
+    restored.receiver_cache.copy_(saved_r)
+    guard(restored)  # (the copies went over the guard bytes: arm them again)
+    rebuilt = fresh()
+    rebuilt.init_caches(to_dev_bytes(traj[2], DEV))
+    for label, codec in (("saved caches", restored), ("caches rebuilt from the weights", rebuilt)):
+        codec.step(to_dev_bytes(traj[3], DEV))
+        torch.cuda.synchronize()
+        codec.check_status()
+        compare_step(codec, want, traj[3], label)
+        compare_caches(codec, table, label)
+        compare_recon(codec, want, traj[3], dtype, label)
+    if block >= 16:  # the hashed sender resumes from a HashCache rebuilt from the weights of the last step sent
+        hashed = fresh()
+        hashed.init_hash_cache(to_dev_bytes(traj[2], DEV))
+        hashed.encode_hashed(to_dev_bytes(traj[3], DEV))
+        hashed.transport()
+        torch.cuda.synchronize()
+        hashed.check_status()
+        compare_step(hashed, want, traj[3], "HashCache rebuilt from the weights")
+
+
 @pytest.mark.parametrize("n_layers", [1, 3])
 def test_pipeline_of_many_iterations_reuses_layer_buffers_safely(rt, n_layers):
     """Many iterations back to back on two streams, alternating between two iterates: with a single
