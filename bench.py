@@ -561,6 +561,12 @@ def main():
     sev1.record(s_enc)
     barrier()
     serial_ms_per_step = sev0.elapsed_time(sev1) / args.steps
+    # spread over the steps (serial re-run: a step's first launch to its last; the paper reports p5 / p95 whiskers)
+    nl = len(layers)
+    per_step = [serial_timers[i * nl][0].elapsed_time(serial_timers[i * nl + nl - 1][5]) for i in range(args.steps)]
+    step_spread = {"mean": float(np.mean(per_step)), "min": float(np.min(per_step)), "p5": float(np.percentile(per_step, 5)),
+                   "p95": float(np.percentile(per_step, 95)), "max": float(np.max(per_step)), "steps": args.steps,
+                   "per": "serial re-run on one stream, first launch to last of each step, ms"}
     for c in layers:
         c.check_status()
 
@@ -649,6 +655,7 @@ def main():
         "kernel_ms_overlapped": {"encode": ovl_ms[0], "transport": ovl_ms[1], "decode": ovl_ms[2],
                                  "per": "layer launch inside the two-stream timed region (kernels overlap)"},
         "serial_ms_per_step": serial_ms_per_step,
+        "serial_step_ms_spread": step_spread,
         "kernel_ms_x_sm_mhz": ({"encode": enc_ms * clocks["sm_mhz"], "transport": tra_ms * clocks["sm_mhz"],
                                 "decode": dec_ms * clocks["sm_mhz"],
                                 "note": "launch time x median SM MHz sampled in the timed region: constant across runs "
