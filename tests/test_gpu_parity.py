@@ -296,6 +296,60 @@ def test_steps_replayed_from_a_cuda_graph(rt, sizes, dtype, block):
         compare_recon(codec, exp, traj[t], dtype, f"replay t={t}")
 
 
+@pytest.mark.parametrize("dtype,block", [(0, 1), (0, 8), (0, 512), (2, 1), (2, 4), (2, 64), (1, 2), (1, 512)])
+def test_every_pattern_against_every_cached_exponent(rt, dtype, block):
+    """The complete per-value map on the GPU: every 16-bit pattern of bf16 and fp16 (zeros, subnormals, infinities,
+    NaNs with every payload) against every value the cached exponent can have (256 / 32) -- 16.7 M / 2.1 M values in
+    one unit, cache rows shuffled so that changed and unchanged blocks mix; for fp32 every exponent field x both
+    signs x 4096 mantissas (the extreme ones among them) against eight cached exponents.  Message, length, count,
+    caches and output against the oracle."""
+    ciera, runtime = rt
+    from oracle import ciera_oracle as ora
+
+    rng = np.random.default_rng(1000 + 16 * dtype + block)
+    if dtype == 1:
+        mant = np.unique(np.concatenate([[0, 1, 2, (1 << 23) - 1, 1 << 22], rng.integers(0, 1 << 23, 4091)])).astype(np.uint32)
+        pat = (np.arange(512, dtype=np.uint32)[:, None] << 23 | mant[None, :]).reshape(-1)  # sign and exponent x mantissas
+        cached = np.array([0, 1, 126, 127, 128, 254, 255, 77], np.uint8)
+        name, wdt = "fp32", np.uint32
+        own = ((pat >> 23) & 0xFF).astype(np.uint8)
+    else:
+        pat = np.arange(1 << 16, dtype=np.uint16)
+        cached = np.arange(256 if dtype == 0 else 32, dtype=np.uint8)
+        name, wdt = ("bf16", np.uint16) if dtype == 0 else ("fp16", np.uint16)
+        own = ((pat >> 7) & 0xFF).astype(np.uint8) if dtype == 0 else ((pat >> 10) & 0x1F).astype(np.uint8)
+    w = np.tile(pat, cached.size).astype(wdt)
+    cache0 = np.repeat(cached, pat.size)
+    # in half of the rows the cache already holds the value's own exponent for most values: unchanged blocks too
+    keep = np.repeat(rng.random(cached.size) < 0.5, pat.size) & (rng.random(w.size) < 0.97)
+    cache0 = np.where(keep, np.tile(own, cached.size), cache0).astype(np.uint8)
+    n = w.size
+    codec = guard(runtime.LayerCodec.from_tensors([n], 1, name, block, DEV, slack=256))
+    assert len(codec.units) == 1
+    u = codec.units[0]
+    lo, mo, co = int(u["weights_off"]), int(u["msg_off"]), int(u["cache_off"])
+    w_dev = torch.zeros(codec.weights_bytes, dtype=torch.uint8, device=DEV)
+    w_dev[lo : lo + w.nbytes] = torch.from_numpy(w.view(np.uint8)).to(DEV)
+    for cache in (codec.sender_cache, codec.receiver_cache):
+        cache[co : co + n] = torch.from_numpy(cache0).to(DEV)
+    codec.step(w_dev)
+    torch.cuda.synchronize()
+    codec.check_status()
+    codec.canaries.check("every pattern")
+    cache_s = cache0.copy()
+    msg, wire, pay, chg = ora.encode(w, cache_s, dtype, block)
+    assert int(codec.wire_bytes[0].item()) == wire and int(codec.changed_blocks[0].item()) == chg
+    assert 0 < chg < -(-n // block) or block >= 64
+    assert np.array_equal(codec.msg_send[mo : mo + wire].cpu().numpy(), msg)
+    assert np.array_equal(codec.msg_recv[mo : mo + wire].cpu().numpy(), msg)
+    cache_r = cache0.copy()
+    out = ora.decode(msg, cache_r, dtype, block)
+    assert np.array_equal(out, w)
+    assert np.array_equal(codec.sender_cache[co : co + n].cpu().numpy(), cache_s)
+    assert np.array_equal(codec.receiver_cache[co : co + n].cpu().numpy(), cache_r)
+    assert np.array_equal(codec.weights_out[lo : lo + w.nbytes].cpu().numpy().view(wdt), w)
+
+
 @pytest.mark.parametrize("dtype,block", [(0, 512), (1, 4), (2, 64)])
 def test_resume_from_saved_caches_or_from_the_weights(rt, dtype, block):
     """The codec's only persistent state are the two exponent caches (and the sender's HashCache), plain buffers of
